@@ -1,0 +1,133 @@
+/* soap.h - C ABI of the B200 SOAP descriptor library (libsoap_b200.so).
+ *
+ * Computes, for every centre atom of a structure, the Smooth Overlap of Atomic
+ * Positions partial power spectrum and its analytic Cartesian Jacobian:
+ *
+ *   neighbours within r_cut (text under Eq. 1)
+ *   -> expansion coefficients c^mu_nlm of the Gaussian-smeared species
+ *      densities on a radial basis times real spherical harmonics
+ *      (Eq. 3; closed form Eq. 13 for Gaussian-type orbitals, the radial
+ *      Bessel integral Eqs. 18-19 for polynomials; on-site term included)
+ *   -> p^{mu nu}_{n n' l} = pi sqrt(8/(2l+1)) sum_m c^mu_nlm c^nu_n'lm   (Eq. 4)
+ *   -> d p / d R_j for every atom j inside the sphere and for the centre
+ *      (Eq. 5; Eq. 14 / Eq. 23 for the coefficient gradients).
+ *
+ * Conventions
+ *  - Pointers named d_* are DEVICE pointers owned by the caller; everything
+ *    else is host memory.  The handle owns its tables and scratch memory.
+ *  - Positions are fp32 Angstrom, row-major [N,3]; atomic numbers int32 [N].
+ *  - `cell` is host memory, 9 doubles, rows = lattice vectors a, b, c; it may
+ *    be NULL when no axis is periodic.  Positions need not be wrapped.
+ *  - `d_centers` lists the centre atoms (indices into the structure); NULL
+ *    means every atom, in order (then n_centers must equal n_atoms).
+ *  - `stream` is a cudaStream_t passed as void* (NULL = default stream).  All
+ *    calls enqueue work on it and return without waiting, except where noted.
+ *  - Feature order: species pairs mu <= nu (species sorted by atomic number),
+ *    then the radial pair (n, n') with n' >= n when mu == nu and all n, n'
+ *    otherwise (n outer), then l fastest.  F = S n_max (S n_max + 1)/2 (l_max+1).
+ *  - Every function returns SOAP_OK or a negative code; nothing throws.
+ *    Problems only the device can see (an atomic number outside the species
+ *    list, more pairs or rows than a buffer holds) are recorded in a sticky
+ *    status word that soap_status() returns after synchronising; when it is
+ *    set, the outputs of that call are unspecified.
+ *  - The library has no CPU fallback: without a CUDA device the compute
+ *    calls return SOAP_ERR_CUDA.
+ */
+#ifndef SOAP_B200_H
+#define SOAP_B200_H
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct soap_handle soap_t;
+
+enum {
+    SOAP_OK = 0,
+    SOAP_ERR_INVALID_ARG = -1,
+    SOAP_ERR_UNKNOWN_SPECIES = -2,  /* an atomic number is not in the species list */
+    SOAP_ERR_CAPACITY = -3,         /* a caller buffer or the planned scratch is too small */
+    SOAP_ERR_CUDA = -4,
+    SOAP_ERR_ALLOC = -5
+};
+
+enum { SOAP_RBF_GTO = 0, SOAP_RBF_POLYNOMIAL = 1 };
+
+/* Builds a descriptor object: basis constants of Eqs. 8-10 (GTO) or 15-17
+ * (polynomial) and the radial tables derived from Eq. 13 / Eqs. 18-19, all on
+ * the host in quad precision.  No GPU work happens here; device copies are
+ * made on first use.  species: n_species distinct atomic numbers (any order).
+ * Limits: 1 <= n_species <= 8, 1 <= n_max <= 16, 0 <= l_max <= 12,
+ * r_cut > 0 (> 1 A for GTO, whose width rule Eq. 10 starts at 1 A), sigma > 0.
+ * pbc: three flags, one per lattice vector. */
+int soap_create(soap_t **out, const int32_t *species, int n_species, double r_cut,
+                int n_max, int l_max, double sigma, int rbf, const int pbc[3]);
+
+void soap_destroy(soap_t *h);
+
+/* Number of features F per centre. */
+int soap_num_features(const soap_t *h, int64_t *n_features);
+
+/* (mu, nu, n, n', l) of feature f; mu, nu index the sorted species list. */
+int soap_feature_info(const soap_t *h, int64_t f, int *mu, int *nu, int *n, int *n2, int *l);
+
+/* Message of the last failing call on this handle (never NULL). */
+const char *soap_last_error(const soap_t *h);
+
+/* Host-side check of the radial tables: G_nl(d) and (dG_nl/dd)/d for all
+ * n_max*(l_max+1) channels (index n*(l_max+1)+l), where the pair term of
+ * Eq. 13 / Eq. 18 is G_nl(d) r^l Y_lm.  Needs no GPU. */
+int soap_radial_table(const soap_t *h, double d, double *G, double *Ghat);
+
+/* Neighbour search only (cell list + exact fp64 distance test), then WAITS
+ * for the stream.  Returns the number of (centre, neighbour image) pairs and
+ * the number of Jacobian rows (distinct atoms per sphere, plus the centre),
+ * and sizes the handle's scratch for later calls on structures of this size
+ * (with 25% headroom).  Call it before soap_derivatives to size d_jac. */
+int soap_neighbors(soap_t *h, const float *d_positions, const int32_t *d_numbers, int64_t n_atoms,
+                   const double *cell, const int32_t *d_centers, int64_t n_centers,
+                   int64_t *n_pairs, int64_t *n_rows, void *stream);
+
+/* Exports the neighbour list of the last soap_neighbors / soap_descriptor /
+ * soap_derivatives call: d_pair_ptr [n_centers+1]; for pair e of centre i
+ * (d_pair_ptr[i] <= e < d_pair_ptr[i+1]) the neighbour atom d_pair_atom[e] and
+ * its lattice translation d_pair_shift[3e..3e+2] (multiples of a, b, c; may be
+ * NULL).  Pairs of a centre are sorted by (atom, shift).  capacity_pairs is
+ * the length of the caller's arrays; too small sets SOAP_ERR_CAPACITY. */
+int soap_neighbor_list(soap_t *h, int64_t *d_pair_ptr, int32_t *d_pair_atom, int32_t *d_pair_shift,
+                       int64_t capacity_pairs, void *stream);
+
+/* Descriptor only: d_out [n_centers, F] fp32, fully overwritten (Eq. 4).
+ * Runs the neighbour search itself.  The first call for a structure size
+ * plans scratch memory like soap_neighbors (allocates and waits once). */
+int soap_descriptor(soap_t *h, const float *d_positions, const int32_t *d_numbers, int64_t n_atoms,
+                    const double *cell, const int32_t *d_centers, int64_t n_centers,
+                    float *d_out, void *stream);
+
+/* Descriptor and Jacobian (Eqs. 4 and 5).  Runs the neighbour search itself.
+ *   d_out_desc [n_centers, F]
+ *   d_row_ptr  [n_centers+1]   rows of centre i are d_row_ptr[i] .. d_row_ptr[i+1]-1
+ *   d_row_atom [capacity_rows] atom each row differentiates with respect to;
+ *                              ascending within a centre, the centre included
+ *   d_out_jac  [capacity_rows, 3, F]  d p_f / d (x,y,z of that atom); all other
+ *              entries of the dense (centre, atom, 3, F) Jacobian are zero.
+ * Periodic images of one atom add up in that atom's row.  Every row below
+ * d_row_ptr[n_centers] is fully overwritten.  If the structure has more rows
+ * than capacity_rows nothing is written and the status becomes
+ * SOAP_ERR_CAPACITY. */
+int soap_derivatives(soap_t *h, const float *d_positions, const int32_t *d_numbers, int64_t n_atoms,
+                     const double *cell, const int32_t *d_centers, int64_t n_centers,
+                     float *d_out_desc, float *d_out_jac, int64_t capacity_rows,
+                     int64_t *d_row_ptr, int32_t *d_row_atom, void *stream);
+
+/* Waits for `stream`, then returns and clears the sticky device status
+ * (SOAP_OK, SOAP_ERR_UNKNOWN_SPECIES or SOAP_ERR_CAPACITY); also reports the
+ * pair and row counts of the last call (either pointer may be NULL). */
+int soap_status(soap_t *h, int64_t *n_pairs, int64_t *n_rows, void *stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* SOAP_B200_H */

@@ -1,0 +1,204 @@
+"""ctypes binding of libsoap_b200.so (argument marshalling only)."""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from dataclasses import dataclass
+
+import numpy as np
+
+GTO, POLYNOMIAL = 0, 1
+
+EXPORTED_SYMBOLS = [
+    "soap_create", "soap_destroy", "soap_num_features", "soap_feature_info", "soap_last_error",
+    "soap_radial_table", "soap_neighbors", "soap_neighbor_list", "soap_descriptor",
+    "soap_derivatives", "soap_status",
+]
+
+_ERRORS = {-1: "SOAP_ERR_INVALID_ARG", -2: "SOAP_ERR_UNKNOWN_SPECIES", -3: "SOAP_ERR_CAPACITY",
+           -4: "SOAP_ERR_CUDA", -5: "SOAP_ERR_ALLOC"}
+
+
+class SoapError(RuntimeError):
+    def __init__(self, code, message):
+        super().__init__(f"{_ERRORS.get(code, code)}: {message}")
+        self.code = code
+
+
+def library_path() -> str:
+    return os.path.join(os.path.dirname(os.path.abspath(__file__)), "libsoap_b200.so")
+
+
+_LIB = None
+
+
+def load_library() -> C.CDLL:
+    """Loads the shared library (never builds it, never falls back)."""
+    global _LIB
+    if _LIB is not None:
+        return _LIB
+    path = library_path()
+    if not os.path.exists(path):
+        raise ImportError(f"{path} is missing: build it with `python -m paper_2609_05709_b200.build`")
+    lib = C.CDLL(path)
+    vp, i64, i32 = C.c_void_p, C.c_int64, C.c_int
+    lib.soap_create.argtypes = [C.POINTER(vp), C.POINTER(C.c_int32), i32, C.c_double, i32, i32, C.c_double, i32, C.POINTER(i32)]
+    lib.soap_destroy.argtypes = [vp]
+    lib.soap_destroy.restype = None
+    lib.soap_num_features.argtypes = [vp, C.POINTER(i64)]
+    lib.soap_feature_info.argtypes = [vp, i64] + [C.POINTER(i32)] * 5
+    lib.soap_last_error.argtypes = [vp]
+    lib.soap_last_error.restype = C.c_char_p
+    lib.soap_radial_table.argtypes = [vp, C.c_double, C.POINTER(C.c_double), C.POINTER(C.c_double)]
+    common = [vp, vp, vp, i64, C.POINTER(C.c_double), vp, i64]
+    lib.soap_neighbors.argtypes = common + [C.POINTER(i64), C.POINTER(i64), vp]
+    lib.soap_neighbor_list.argtypes = [vp, vp, vp, vp, i64, vp]
+    lib.soap_descriptor.argtypes = common + [vp, vp]
+    lib.soap_derivatives.argtypes = common + [vp, vp, i64, vp, vp, vp]
+    lib.soap_status.argtypes = [vp, C.POINTER(i64), C.POINTER(i64), vp]
+    for name in EXPORTED_SYMBOLS:
+        if name not in ("soap_destroy", "soap_last_error"):
+            getattr(lib, name).restype = C.c_int
+    _LIB = lib
+    return lib
+
+
+@dataclass
+class Derivatives:
+    descriptor: "torch.Tensor"   # (C, F) float32, device
+    jacobian: "torch.Tensor"     # (rows, 3, F) float32, device
+    row_ptr: "torch.Tensor"      # (C+1,) int64, device
+    row_atom: "torch.Tensor"     # (rows,) int32, device
+
+
+class Soap:
+    """One descriptor configuration (the arguments of soap_create)."""
+
+    def __init__(self, species, r_cut, n_max, l_max, sigma, rbf=GTO, pbc=(False, False, False)):
+        self._lib = load_library()
+        self._h = C.c_void_p()
+        sp = (C.c_int32 * len(species))(*[int(z) for z in species])
+        pb = (C.c_int * 3)(*[int(bool(p)) for p in pbc])
+        rc = self._lib.soap_create(C.byref(self._h), sp, len(species), float(r_cut), int(n_max), int(l_max),
+                                   float(sigma), int(rbf), pb)
+        if rc != 0:
+            msg = self._lib.soap_last_error(self._h).decode() if self._h else "allocation failed"
+            self.close()
+            raise SoapError(rc, msg)
+        n = C.c_int64()
+        self._check(self._lib.soap_num_features(self._h, C.byref(n)))
+        self.n_features = int(n.value)
+        self.n_channels = int(n_max) * (int(l_max) + 1)
+        self.pbc = tuple(bool(p) for p in pbc)
+
+    # ------------------------------------------------------------------ plumbing
+    def close(self):
+        if getattr(self, "_h", None):
+            self._lib.soap_destroy(self._h)
+            self._h = C.c_void_p()
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    def _check(self, rc):
+        if rc != 0:
+            raise SoapError(rc, self._lib.soap_last_error(self._h).decode())
+
+    @staticmethod
+    def _stream():
+        import torch
+        return C.c_void_p(torch.cuda.current_stream().cuda_stream)
+
+    @staticmethod
+    def _cell(cell):
+        if cell is None:
+            return None, None
+        arr = np.ascontiguousarray(np.asarray(cell, np.float64).reshape(9))
+        return arr, arr.ctypes.data_as(C.POINTER(C.c_double))
+
+    @staticmethod
+    def _inputs(positions, numbers, centers):
+        import torch
+        assert positions.is_cuda and positions.dtype == torch.float32 and positions.is_contiguous()
+        assert numbers.is_cuda and numbers.dtype == torch.int32 and numbers.is_contiguous()
+        n = positions.shape[0]
+        if centers is None:
+            return n, n, None
+        assert centers.is_cuda and centers.dtype == torch.int32 and centers.is_contiguous()
+        return n, centers.shape[0], C.c_void_p(centers.data_ptr())
+
+    # ------------------------------------------------------------------ host-only helpers
+    def feature_info(self, f):
+        out = [C.c_int() for _ in range(5)]
+        self._check(self._lib.soap_feature_info(self._h, int(f), *[C.byref(o) for o in out]))
+        return tuple(o.value for o in out)      # mu, nu, n, n', l
+
+    def radial_table(self, d):
+        G = np.empty(self.n_channels)
+        Gh = np.empty(self.n_channels)
+        self._check(self._lib.soap_radial_table(self._h, float(d), G.ctypes.data_as(C.POINTER(C.c_double)),
+                                                Gh.ctypes.data_as(C.POINTER(C.c_double))))
+        return G, Gh
+
+    # ------------------------------------------------------------------ device calls
+    def neighbors(self, positions, numbers, cell=None, centers=None):
+        """(n_pairs, n_rows); waits for the stream."""
+        n, c, cptr = self._inputs(positions, numbers, centers)
+        keep, cellp = self._cell(cell)
+        npairs, nrows = C.c_int64(), C.c_int64()
+        self._check(self._lib.soap_neighbors(self._h, positions.data_ptr(), numbers.data_ptr(), n, cellp, cptr, c,
+                                             C.byref(npairs), C.byref(nrows), self._stream()))
+        return int(npairs.value), int(nrows.value)
+
+    def neighbor_list(self, positions, numbers, cell=None, centers=None):
+        """pair_ptr (C+1,), pair_atom (E,), pair_shift (E,3) as device tensors."""
+        import torch
+        npairs, _ = self.neighbors(positions, numbers, cell, centers)
+        c = positions.shape[0] if centers is None else centers.shape[0]
+        ptr = torch.empty(c + 1, dtype=torch.int64, device=positions.device)
+        atom = torch.empty(max(npairs, 1), dtype=torch.int32, device=positions.device)
+        shift = torch.empty((max(npairs, 1), 3), dtype=torch.int32, device=positions.device)
+        self._check(self._lib.soap_neighbor_list(self._h, ptr.data_ptr(), atom.data_ptr(), shift.data_ptr(), npairs, self._stream()))
+        self.status()
+        return ptr, atom[:npairs], shift[:npairs]
+
+    def descriptor(self, positions, numbers, cell=None, centers=None, out=None):
+        import torch
+        n, c, cptr = self._inputs(positions, numbers, centers)
+        keep, cellp = self._cell(cell)
+        if out is None:
+            out = torch.empty((c, self.n_features), dtype=torch.float32, device=positions.device)
+        self._check(self._lib.soap_descriptor(self._h, positions.data_ptr(), numbers.data_ptr(), n, cellp, cptr, c,
+                                              out.data_ptr(), self._stream()))
+        return out
+
+    def derivatives_into(self, positions, numbers, cell, centers, desc, jac, row_ptr, row_atom):
+        """Asynchronous call into caller-provided buffers (jac: (capacity_rows, 3, F))."""
+        n, c, cptr = self._inputs(positions, numbers, centers)
+        keep, cellp = self._cell(cell)
+        self._check(self._lib.soap_derivatives(self._h, positions.data_ptr(), numbers.data_ptr(), n, cellp, cptr, c,
+                                               desc.data_ptr(), jac.data_ptr(), jac.shape[0], row_ptr.data_ptr(),
+                                               row_atom.data_ptr(), self._stream()))
+
+    def derivatives(self, positions, numbers, cell=None, centers=None) -> Derivatives:
+        """Sizes the Jacobian with one neighbour search, then computes it."""
+        import torch
+        _, nrows = self.neighbors(positions, numbers, cell, centers)
+        c = positions.shape[0] if centers is None else centers.shape[0]
+        dev = positions.device
+        desc = torch.empty((c, self.n_features), dtype=torch.float32, device=dev)
+        jac = torch.empty((max(nrows, 1), 3, self.n_features), dtype=torch.float32, device=dev)
+        row_ptr = torch.empty(c + 1, dtype=torch.int64, device=dev)
+        row_atom = torch.empty(max(nrows, 1), dtype=torch.int32, device=dev)
+        self.derivatives_into(positions, numbers, cell, centers, desc, jac, row_ptr, row_atom)
+        self.status()
+        return Derivatives(desc, jac[:nrows], row_ptr, row_atom[:nrows])
+
+    def status(self):
+        """Waits for the stream; raises if the device flagged a problem. Returns (n_pairs, n_rows)."""
+        npairs, nrows = C.c_int64(), C.c_int64()
+        self._check(self._lib.soap_status(self._h, C.byref(npairs), C.byref(nrows), self._stream()))
+        return int(npairs.value), int(nrows.value)

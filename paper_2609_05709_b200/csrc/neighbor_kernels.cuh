@@ -1,0 +1,382 @@
+// Cell list and neighbour compaction (the search step under Eq. 1).
+//
+// Atoms are binned in fractional coordinates of the cell (of the identity when
+// there is none); periodic axes are wrapped for binning only.  A centre visits
+// the stencil of bins around its own, and every candidate (atom j, lattice
+// translation n) passes the exact test
+//     0 < |(r_j - r_i) + ((n_a a + n_b b) + n_c c)|^2 < r_cut^2
+// in fp64 on the raw fp32 inputs, each operation rounded separately, so the set
+// does not depend on the binning and can be compared bit for bit with a
+// reference.  Pairs of a centre come out sorted by (atom, n_a, n_b, n_c).
+#pragma once
+#include "soap_device.cuh"
+
+namespace soap {
+
+// ---- order-preserving encoding of doubles for atomicMax ---------------------
+__device__ inline unsigned long long enc_double(double x) {
+    unsigned long long b = (unsigned long long)__double_as_longlong(x);
+    return (b >> 63) ? ~b : (b | 0x8000000000000000ull);
+}
+__device__ inline double dec_double(unsigned long long e) {
+    unsigned long long b = (e >> 63) ? (e & 0x7fffffffffffffffull) : ~e;
+    return __longlong_as_double((long long)b);
+}
+
+__device__ inline void frac_coords(const Geometry& g, float x, float y, float z, double s[3]) {
+    for (int a = 0; a < 3; ++a)
+        s[a] = (double)x * g.inv[0 + a] + (double)y * g.inv[3 + a] + (double)z * g.inv[6 + a];
+}
+
+// species index per atom, and the bounding box of the fractional coordinates
+// bbox[0..2] = enc(max s), bbox[3..5] = enc(max -s); zero-initialised by the host
+__global__ void species_bbox_kernel(const float* __restrict__ pos, const int* __restrict__ numbers, long long N,
+                                    Geometry geom, const int* __restrict__ z_lut, int* __restrict__ species_idx,
+                                    unsigned long long* bbox, Counters* counters) {
+    double hi[3] = {-1e300, -1e300, -1e300}, lo[3] = {-1e300, -1e300, -1e300};
+    bool bad = false;
+    for (long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x; i < N; i += (long long)gridDim.x * blockDim.x) {
+        int z = numbers[i];
+        int s = (z >= 0 && z < 128) ? z_lut[z] : -1;
+        if (s < 0) { bad = true; s = 0; }
+        species_idx[i] = s;
+        double f[3];
+        frac_coords(geom, pos[3 * i], pos[3 * i + 1], pos[3 * i + 2], f);
+        for (int a = 0; a < 3; ++a) { hi[a] = fmax(hi[a], f[a]); lo[a] = fmax(lo[a], -f[a]); }
+    }
+    for (int a = 0; a < 3; ++a)
+        for (int o = 16; o > 0; o >>= 1) {
+            hi[a] = fmax(hi[a], __shfl_xor_sync(0xffffffffu, hi[a], o));
+            lo[a] = fmax(lo[a], __shfl_xor_sync(0xffffffffu, lo[a], o));
+        }
+    if ((threadIdx.x & 31) == 0)
+        for (int a = 0; a < 3; ++a) {
+            atomicMax(&bbox[a], enc_double(hi[a]));
+            atomicMax(&bbox[3 + a], enc_double(lo[a]));
+        }
+    if (bad) atomicOr(&counters->status, kStatusUnknownSpecies);
+}
+
+// One thread: choose the bin grid.  Bin width (measured perpendicular to the
+// cell faces) is at least r_cut (1 + 1e-6) wherever more than one bin fits, so a
+// stencil of +-1 bin covers the sphere; short periodic axes get one bin and a
+// wider stencil of images.
+__global__ void grid_setup_kernel(const unsigned long long* bbox, Geometry geom, long long N, int cell_cap, GridParams* out) {
+    GridParams g;
+    const double rc = geom.r_cut * (1.0 + 1e-6);
+    double want[3];
+    for (int a = 0; a < 3; ++a) {
+        g.periodic[a] = geom.pbc[a];
+        if (geom.pbc[a]) {
+            g.smin[a] = 0.0;
+            want[a] = floor(geom.height[a] / rc);
+        } else {
+            double hi = N > 0 ? dec_double(bbox[a]) : 0.0, lo = N > 0 ? -dec_double(bbox[3 + a]) : 0.0;
+            g.smin[a] = lo;
+            want[a] = floor((hi - lo) * geom.height[a] / rc);
+        }
+        if (!(want[a] >= 1.0)) want[a] = 1.0;
+        if (want[a] > 1024.0) want[a] = 1024.0;
+    }
+    // respect the scratch capacity: shrink the grid uniformly
+    for (int it = 0; it < 64 && want[0] * want[1] * want[2] > (double)cell_cap; ++it)
+        for (int a = 0; a < 3; ++a) want[a] = fmax(1.0, floor(want[a] * 0.8));
+    for (int a = 0; a < 3; ++a) {
+        g.nb[a] = (int)want[a];
+        if (geom.pbc[a]) {
+            g.sscale[a] = (double)g.nb[a];
+            double width = geom.height[a] / g.nb[a];
+            g.R[a] = (int)ceil(rc / width);
+        } else {
+            double hi = N > 0 ? dec_double(bbox[a]) : 0.0;
+            double span = hi - g.smin[a];
+            g.sscale[a] = span > 0 ? g.nb[a] / span : 0.0;
+            g.R[a] = g.nb[a] > 1 ? 1 : 0;
+        }
+    }
+    g.n_cells = g.nb[0] * g.nb[1] * g.nb[2];
+    *out = g;
+}
+
+__device__ inline void bin_of(const Geometry& geom, const GridParams& g, float x, float y, float z, int b[3], int w[3]) {
+    double s[3];
+    frac_coords(geom, x, y, z, s);
+    for (int a = 0; a < 3; ++a) {
+        double t = s[a];
+        w[a] = 0;
+        if (g.periodic[a]) {
+            double fl = floor(t);
+            w[a] = (int)fl;
+            t -= fl;
+        }
+        int bi = (int)floor((t - g.smin[a]) * g.sscale[a]);
+        b[a] = min(max(bi, 0), g.nb[a] - 1);
+    }
+}
+
+__device__ inline int pack3(const int v[3]) { return ((v[0] + 512) << 20) | ((v[1] + 512) << 10) | (v[2] + 512); }
+__device__ inline void unpack3(int p, int v[3]) { v[0] = ((p >> 20) & 1023) - 512; v[1] = ((p >> 10) & 1023) - 512; v[2] = (p & 1023) - 512; }
+
+__global__ void bin_count_kernel(const float* __restrict__ pos, long long N, Geometry geom, const GridParams* __restrict__ gp,
+                                 int* __restrict__ atom_cell, int* __restrict__ atom_wrap, int* cell_count, Counters* counters) {
+    const GridParams g = *gp;
+    for (long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x; i < N; i += (long long)gridDim.x * blockDim.x) {
+        int b[3], w[3];
+        bin_of(geom, g, pos[3 * i], pos[3 * i + 1], pos[3 * i + 2], b, w);
+        if (abs(w[0]) > 100 || abs(w[1]) > 100 || abs(w[2]) > 100) {      // positions absurdly far outside the cell
+            atomicOr(&counters->status, kStatusShiftRange);
+            w[0] = w[1] = w[2] = 0;
+        }
+        int cell = (b[2] * g.nb[1] + b[1]) * g.nb[0] + b[0];
+        atom_cell[i] = cell;
+        atom_wrap[i] = pack3(w);
+        atomicAdd(&cell_count[cell], 1);
+    }
+}
+
+// Exclusive scan by ONE block (n is at most a few million here); out[n] = total.
+template <typename OutT>
+__global__ void scan_kernel(const int* __restrict__ in, OutT* __restrict__ out, long long n, long long* total_out) {
+    __shared__ long long warp_sums[32];
+    __shared__ long long carry_s;
+    if (threadIdx.x == 0) carry_s = 0;
+    __syncthreads();
+    const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5, nw = blockDim.x >> 5;
+    for (long long base = 0; base < n; base += blockDim.x) {
+        long long i = base + threadIdx.x;
+        long long v = i < n ? (long long)in[i] : 0, x = v;
+        for (int o = 1; o < 32; o <<= 1) {
+            long long y = __shfl_up_sync(0xffffffffu, x, o);
+            if (lane >= o) x += y;
+        }
+        if (lane == 31) warp_sums[wid] = x;
+        __syncthreads();
+        if (wid == 0) {
+            long long s = lane < nw ? warp_sums[lane] : 0;
+            for (int o = 1; o < 32; o <<= 1) {
+                long long y = __shfl_up_sync(0xffffffffu, s, o);
+                if (lane >= o) s += y;
+            }
+            warp_sums[lane] = s;
+        }
+        __syncthreads();
+        long long carry = carry_s;
+        long long excl = carry + (wid > 0 ? warp_sums[wid - 1] : 0) + x - v;
+        if (i < n) out[i] = (OutT)excl;
+        __syncthreads();
+        if (threadIdx.x == blockDim.x - 1) carry_s = carry + warp_sums[nw - 1];
+        __syncthreads();
+    }
+    if (threadIdx.x == 0) {
+        out[n] = (OutT)carry_s;
+        if (total_out) *total_out = carry_s;
+    }
+}
+
+__global__ void bin_fill_kernel(const float* __restrict__ pos, long long N, const int* __restrict__ atom_cell,
+                                const int* __restrict__ atom_wrap, const int* __restrict__ cell_start, int* cell_count,
+                                float4* __restrict__ s_pos, int* __restrict__ s_wrap) {
+    for (long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x; i < N; i += (long long)gridDim.x * blockDim.x) {
+        int cell = atom_cell[i];
+        int slot = cell_start[cell] + atomicSub(&cell_count[cell], 1) - 1;
+        s_pos[slot] = make_float4(pos[3 * i], pos[3 * i + 1], pos[3 * i + 2], __int_as_float((int)i));
+        s_wrap[slot] = atom_wrap[i];
+    }
+}
+
+// floor division / modulo for the periodic wrap of a bin coordinate
+__device__ inline void wrap_bin(int b, int nb, int& cell, int& image) {
+    image = (b >= 0) ? b / nb : -((-b + nb - 1) / nb);
+    cell = b - image * nb;
+}
+
+// Calls f(valid, key) for every lane in lock step, over all candidates of one centre.
+// key encodes (atom, lattice translation on the raw inputs); valid says whether this
+// lane holds a pair inside the cutoff.
+template <class F>
+__device__ inline void for_each_candidate(const Geometry& geom, const GridParams& g, const int* __restrict__ cell_start,
+                                          const float4* __restrict__ s_pos, const int* __restrict__ s_wrap,
+                                          float xi, float yi, float zi, const int bi[3], const int wi[3],
+                                          int lane, Counters* counters, F f) {
+    for (int oz = -g.R[2]; oz <= g.R[2]; ++oz) {
+        int cz, iz;
+        if (g.periodic[2]) wrap_bin(bi[2] + oz, g.nb[2], cz, iz);
+        else { cz = bi[2] + oz; iz = 0; if (cz < 0 || cz >= g.nb[2]) continue; }
+        for (int oy = -g.R[1]; oy <= g.R[1]; ++oy) {
+            int cy, iy;
+            if (g.periodic[1]) wrap_bin(bi[1] + oy, g.nb[1], cy, iy);
+            else { cy = bi[1] + oy; iy = 0; if (cy < 0 || cy >= g.nb[1]) continue; }
+            for (int ox = -g.R[0]; ox <= g.R[0]; ++ox) {
+                int cx, ix;
+                if (g.periodic[0]) wrap_bin(bi[0] + ox, g.nb[0], cx, ix);
+                else { cx = bi[0] + ox; ix = 0; if (cx < 0 || cx >= g.nb[0]) continue; }
+                const int cell = (cz * g.nb[1] + cy) * g.nb[0] + cx;
+                const int start = cell_start[cell], end = cell_start[cell + 1];
+                for (int t0 = start; t0 < end; t0 += 32) {
+                    const int t = t0 + lane;
+                    bool valid = false;
+                    unsigned long long key = 0;
+                    if (t < end) {
+                        const float4 pj = s_pos[t];
+                        int wj[3];
+                        unpack3(s_wrap[t], wj);
+                        // translation on the raw (unwrapped) inputs
+                        const int na = ix - wj[0] + wi[0], nb = iy - wj[1] + wi[1], nc = iz - wj[2] + wi[2];
+                        double dx = __dsub_rn((double)pj.x, (double)xi);
+                        double dy = __dsub_rn((double)pj.y, (double)yi);
+                        double dz = __dsub_rn((double)pj.z, (double)zi);
+                        if (g.periodic[0] | g.periodic[1] | g.periodic[2]) {
+                            // T = (n_a a + n_b b) + n_c c, each product and sum rounded on its own
+                            const double fa = (double)na, fb = (double)nb, fc = (double)nc;
+                            double tx = __dadd_rn(__dadd_rn(__dmul_rn(fa, geom.cell[0]), __dmul_rn(fb, geom.cell[3])), __dmul_rn(fc, geom.cell[6]));
+                            double ty = __dadd_rn(__dadd_rn(__dmul_rn(fa, geom.cell[1]), __dmul_rn(fb, geom.cell[4])), __dmul_rn(fc, geom.cell[7]));
+                            double tz = __dadd_rn(__dadd_rn(__dmul_rn(fa, geom.cell[2]), __dmul_rn(fb, geom.cell[5])), __dmul_rn(fc, geom.cell[8]));
+                            dx = __dadd_rn(dx, tx); dy = __dadd_rn(dy, ty); dz = __dadd_rn(dz, tz);
+                        }
+                        const double d2 = __dadd_rn(__dadd_rn(__dmul_rn(dx, dx), __dmul_rn(dy, dy)), __dmul_rn(dz, dz));
+                        valid = (d2 < geom.rc2) && (d2 > 0.0);
+                        if (valid && (abs(na) > 127 || abs(nb) > 127 || abs(nc) > 127)) {
+                            atomicOr(&counters->status, kStatusShiftRange);
+                            valid = false;
+                        }
+                        key = ((unsigned long long)(unsigned)__float_as_int(pj.w) << 24) |
+                              ((unsigned long long)(na + 128) << 16) | ((unsigned long long)(nb + 128) << 8) |
+                              (unsigned long long)(nc + 128);
+                    }
+                    f(valid, key);
+                }
+            }
+        }
+    }
+}
+
+// One warp per centre: number of pairs.
+__global__ void count_kernel(const float* __restrict__ pos, const int* __restrict__ centers, long long C, Geometry geom,
+                             const GridParams* __restrict__ gp, const int* __restrict__ atom_cell, const int* __restrict__ atom_wrap,
+                             const int* __restrict__ cell_start, const float4* __restrict__ s_pos, const int* __restrict__ s_wrap,
+                             int* __restrict__ pair_count, Counters* counters) {
+    const GridParams g = *gp;
+    const int lane = threadIdx.x & 31;
+    const long long c = blockIdx.x * (long long)(blockDim.x >> 5) + (threadIdx.x >> 5);
+    if (c >= C) return;
+    const int i = centers ? centers[c] : (int)c;
+    const float xi = pos[3 * (long long)i], yi = pos[3 * (long long)i + 1], zi = pos[3 * (long long)i + 2];
+    int bi[3], wi[3];
+    {
+        int cell = atom_cell[i];
+        bi[0] = cell % g.nb[0]; bi[1] = (cell / g.nb[0]) % g.nb[1]; bi[2] = cell / (g.nb[0] * g.nb[1]);
+        unpack3(atom_wrap[i], wi);
+    }
+    int cnt = 0;
+    for_each_candidate(geom, g, cell_start, s_pos, s_wrap, xi, yi, zi, bi, wi, lane, counters,
+                       [&](bool valid, unsigned long long) { cnt += __popc(__ballot_sync(0xffffffffu, valid)); });
+    if (lane == 0) pair_count[c] = cnt;
+}
+
+constexpr int kFillSmemKeys = 512;       // per warp; longer rows are sorted through global memory
+constexpr int kFillWarps = 4;
+
+// One warp per centre: collect the pairs, sort them by key, derive the Jacobian
+// row bookkeeping (distinct atoms, the centre's own position among them).
+__global__ void __launch_bounds__(kFillWarps * 32)
+fill_kernel(const float* __restrict__ pos, const int* __restrict__ centers, long long C, Geometry geom,
+            const GridParams* __restrict__ gp, const int* __restrict__ atom_cell, const int* __restrict__ atom_wrap,
+            const int* __restrict__ cell_start, const float4* __restrict__ s_pos, const int* __restrict__ s_wrap,
+            const long long* __restrict__ pair_ptr, long long pair_capacity,
+            unsigned long long* pair_tmp, unsigned long long* pair_key, int* __restrict__ pair_row,
+            int* __restrict__ row_count, int* __restrict__ self_row, Counters* counters) {
+    __shared__ unsigned long long s_raw[kFillWarps][kFillSmemKeys];
+    __shared__ unsigned long long s_sorted[kFillWarps][kFillSmemKeys];
+    const GridParams g = *gp;
+    const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
+    const long long c = blockIdx.x * (long long)kFillWarps + wid;
+    if (c >= C) return;
+    if (pair_ptr[C] > pair_capacity) {                       // scratch too small: report, write nothing
+        if (c == 0 && lane == 0) atomicOr(&counters->status, kStatusPairCapacity);
+        if (lane == 0) { row_count[c] = 0; self_row[c] = 0; }
+        return;
+    }
+    const int i = centers ? centers[c] : (int)c;
+    const float xi = pos[3 * (long long)i], yi = pos[3 * (long long)i + 1], zi = pos[3 * (long long)i + 2];
+    int bi[3], wi[3];
+    {
+        int cell = atom_cell[i];
+        bi[0] = cell % g.nb[0]; bi[1] = (cell / g.nb[0]) % g.nb[1]; bi[2] = cell / (g.nb[0] * g.nb[1]);
+        unpack3(atom_wrap[i], wi);
+    }
+    const long long base = pair_ptr[c];
+    const int k = (int)(pair_ptr[c + 1] - base);
+    const bool in_smem = k <= kFillSmemKeys;
+    volatile unsigned long long* raw = in_smem ? s_raw[wid] : pair_tmp + base;
+    volatile unsigned long long* sorted = in_smem ? s_sorted[wid] : pair_key + base;
+    int cnt = 0;
+    for_each_candidate(geom, g, cell_start, s_pos, s_wrap, xi, yi, zi, bi, wi, lane, counters,
+                       [&](bool valid, unsigned long long key) {
+                           unsigned m = __ballot_sync(0xffffffffu, valid);
+                           int at = cnt + __popc(m & ((1u << lane) - 1));
+                           if (valid && at < k) raw[at] = key;
+                           cnt += __popc(m);
+                       });
+    __syncwarp();
+    // rank sort (keys are distinct)
+    bool self_in = false;
+    for (int q = lane; q < k; q += 32) {
+        unsigned long long key = raw[q];
+        int rank = 0;
+        for (int r = 0; r < k; ++r) rank += raw[r] < key;
+        sorted[rank] = key;
+        if (in_smem) pair_key[base + rank] = key;
+        self_in |= key_atom(key) == i;
+    }
+    self_in = __any_sync(0xffffffffu, self_in);
+    __syncwarp();
+    // distinct atoms -> local Jacobian rows; the centre's own row sits in atom order
+    int uniq = 0, below = 0;
+    for (int q0 = 0; q0 < k; q0 += 32) {
+        const int q = q0 + lane;
+        int atom = -1, prev = -2;
+        if (q < k) {
+            atom = key_atom(sorted[q]);
+            prev = q > 0 ? key_atom(sorted[q - 1]) : -1;
+        }
+        const bool isnew = q < k && atom != prev;
+        const unsigned m = __ballot_sync(0xffffffffu, isnew);
+        const int u = uniq + __popc(m & ((1u << lane) - 1)) + (isnew ? 1 : 0) - 1;   // index among distinct atoms
+        if (q < k) {
+            int row = u + ((!self_in && atom > i) ? 1 : 0);
+            if (!isnew) row |= kRowContinuation;
+            if (atom == i) row |= kRowSelfImage;
+            pair_row[base + q] = row;
+        }
+        below += __popc(__ballot_sync(0xffffffffu, isnew && atom < i));
+        uniq += __popc(m);
+    }
+    if (lane == 0) {
+        row_count[c] = uniq + (self_in ? 0 : 1);
+        self_row[c] = below;
+    }
+}
+
+// Copies the sorted pair list out in a plain layout.
+__global__ void export_pairs_kernel(const long long* __restrict__ pair_ptr, const unsigned long long* __restrict__ pair_key,
+                                    long long C, long long capacity, long long* out_ptr, int* out_atom, int* out_shift,
+                                    Counters* counters) {
+    const long long total = pair_ptr[C];
+    for (long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x; i <= C; i += (long long)gridDim.x * blockDim.x)
+        out_ptr[i] = pair_ptr[i];
+    if (total > capacity) {
+        if (blockIdx.x == 0 && threadIdx.x == 0) atomicOr(&counters->status, kStatusPairCapacity);
+        return;
+    }
+    for (long long e = blockIdx.x * (long long)blockDim.x + threadIdx.x; e < total; e += (long long)gridDim.x * blockDim.x) {
+        unsigned long long key = pair_key[e];
+        out_atom[e] = key_atom(key);
+        if (out_shift) {
+            int s[3];
+            key_shift(key, s);
+            out_shift[3 * e] = s[0]; out_shift[3 * e + 1] = s[1]; out_shift[3 * e + 2] = s[2];
+        }
+    }
+}
+
+}  // namespace soap

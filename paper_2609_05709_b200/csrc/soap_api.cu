@@ -1,0 +1,440 @@
+// C ABI of libsoap_b200: handle, scratch memory and the launch sequences.
+#include <cuda_runtime.h>
+
+#include <algorithm>
+#include <cmath>
+#include <cstdio>
+#include <cstring>
+#include <new>
+#include <string>
+#include <vector>
+
+#include "basis_host.h"
+#include "center_kernel.cuh"
+#include "neighbor_kernels.cuh"
+#include "soap.h"
+
+using namespace soap;
+
+struct soap_handle {
+    // configuration
+    std::vector<int> species;            // sorted atomic numbers
+    int S = 0, n_max = 0, l_max = 0, rbf = 0;
+    double r_cut = 0, sigma = 0;
+    int pbc[3] = {0, 0, 0};
+    int64_t F = 0;
+    HostBasis basis;
+    std::vector<int> feat_pack;
+    std::string error;
+    // device state (created on first use)
+    int device = -1;
+    bool tables_ready = false;
+    float *d_table = nullptr, *d_self = nullptr, *d_anorm = nullptr, *d_dfact = nullptr, *d_kl = nullptr;
+    int *d_feat = nullptr, *d_zlut = nullptr;
+    Counters* d_counters = nullptr;
+    unsigned long long* d_bbox = nullptr;
+    GridParams* d_grid = nullptr;
+    Counters* h_counters = nullptr;      // pinned
+    // scratch, grown on demand
+    int64_t cap_atoms = 0, cap_centers = 0, cap_cells = 0, cap_pairs = 0;
+    int *d_species_idx = nullptr, *d_atom_cell = nullptr, *d_atom_wrap = nullptr, *d_s_wrap = nullptr;
+    float4* d_s_pos = nullptr;
+    int *d_cell_count = nullptr, *d_cell_start = nullptr;
+    int *d_pair_count = nullptr, *d_row_count = nullptr, *d_self_row = nullptr;
+    long long *d_pair_ptr = nullptr, *d_row_ptr = nullptr;
+    unsigned long long *d_pair_key = nullptr, *d_pair_tmp = nullptr;
+    int* d_pair_row = nullptr;
+    // plan
+    int64_t planned_atoms = -1, planned_centers = -1;
+    int64_t last_centers = 0;
+    int P_desc = 16, P_deriv = 16;
+    size_t smem_desc = 0, smem_deriv = 0;
+    bool attr_set = false;
+};
+
+namespace {
+
+int fail(soap_t* h, int code, const std::string& msg) {
+    if (h) h->error = msg;
+    return code;
+}
+int cuda_fail(soap_t* h, cudaError_t e, const char* what) {
+    return fail(h, SOAP_ERR_CUDA, std::string(what) + ": " + cudaGetErrorString(e));
+}
+#define CU(call)                                                   \
+    do {                                                           \
+        cudaError_t e_ = (call);                                   \
+        if (e_ != cudaSuccess) return cuda_fail(h, e_, #call);     \
+    } while (0)
+
+template <typename T>
+cudaError_t upload(T** dst, const std::vector<T>& src) {
+    cudaError_t e = cudaMalloc((void**)dst, std::max<size_t>(src.size(), 1) * sizeof(T));
+    if (e != cudaSuccess) return e;
+    return cudaMemcpy(*dst, src.data(), src.size() * sizeof(T), cudaMemcpyHostToDevice);
+}
+
+template <typename T>
+cudaError_t regrow(T** ptr, size_t count) {
+    if (*ptr) { cudaFree(*ptr); *ptr = nullptr; }
+    return cudaMalloc((void**)ptr, std::max<size_t>(count, 1) * sizeof(T));
+}
+
+bool invert3(const double m[9], double inv[9], double& det) {
+    det = m[0] * (m[4] * m[8] - m[5] * m[7]) - m[1] * (m[3] * m[8] - m[5] * m[6]) + m[2] * (m[3] * m[7] - m[4] * m[6]);
+    if (!(std::fabs(det) > 1e-12)) return false;
+    inv[0] = (m[4] * m[8] - m[5] * m[7]) / det; inv[1] = (m[2] * m[7] - m[1] * m[8]) / det; inv[2] = (m[1] * m[5] - m[2] * m[4]) / det;
+    inv[3] = (m[5] * m[6] - m[3] * m[8]) / det; inv[4] = (m[0] * m[8] - m[2] * m[6]) / det; inv[5] = (m[2] * m[3] - m[0] * m[5]) / det;
+    inv[6] = (m[3] * m[7] - m[4] * m[6]) / det; inv[7] = (m[1] * m[6] - m[0] * m[7]) / det; inv[8] = (m[0] * m[4] - m[1] * m[3]) / det;
+    return true;
+}
+
+int make_geometry(soap_t* h, const double* cell, Geometry& g) {
+    const bool periodic = h->pbc[0] || h->pbc[1] || h->pbc[2];
+    if (periodic && !cell) return fail(h, SOAP_ERR_INVALID_ARG, "a periodic axis needs a cell");
+    static const double ident[9] = {1, 0, 0, 0, 1, 0, 0, 0, 1};
+    std::memcpy(g.cell, cell ? cell : ident, sizeof(g.cell));
+    double det;
+    if (!invert3(g.cell, g.inv, det)) return fail(h, SOAP_ERR_INVALID_ARG, "the cell is singular");
+    for (int a = 0; a < 3; ++a) {
+        const double* u = &g.cell[3 * ((a + 1) % 3)];
+        const double* v = &g.cell[3 * ((a + 2) % 3)];
+        double cx = u[1] * v[2] - u[2] * v[1], cy = u[2] * v[0] - u[0] * v[2], cz = u[0] * v[1] - u[1] * v[0];
+        g.height[a] = std::fabs(det) / std::sqrt(cx * cx + cy * cy + cz * cz);
+        g.pbc[a] = h->pbc[a];
+        if (h->pbc[a] && std::ceil(h->r_cut / g.height[a]) > 100)
+            return fail(h, SOAP_ERR_INVALID_ARG, "the cell is too thin for this cutoff (more than 100 images along an axis)");
+    }
+    g.r_cut = h->r_cut;
+    g.rc2 = h->r_cut * h->r_cut;
+    return SOAP_OK;
+}
+
+int ensure_device(soap_t* h) {
+    int dev = -1;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return cuda_fail(h, e, "cudaGetDevice (is a CUDA device present? this library has no CPU path)");
+    if (h->tables_ready) {
+        if (dev != h->device) return fail(h, SOAP_ERR_INVALID_ARG, "handle was first used on another device");
+        return SOAP_OK;
+    }
+    h->device = dev;
+    CU(upload(&h->d_table, h->basis.table));
+    CU(upload(&h->d_self, h->basis.self_term));
+    CU(upload(&h->d_anorm, h->basis.anorm));
+    CU(upload(&h->d_dfact, h->basis.dfact));
+    CU(upload(&h->d_kl, h->basis.kl));
+    CU(upload(&h->d_feat, h->feat_pack));
+    std::vector<int> lut(128, -1);
+    for (int s = 0; s < h->S; ++s) lut[h->species[s]] = s;
+    CU(upload(&h->d_zlut, lut));
+    CU(cudaMalloc((void**)&h->d_counters, sizeof(Counters)));
+    CU(cudaMemset(h->d_counters, 0, sizeof(Counters)));
+    CU(cudaMalloc((void**)&h->d_bbox, 6 * sizeof(unsigned long long)));
+    CU(cudaMalloc((void**)&h->d_grid, sizeof(GridParams)));
+    CU(cudaMallocHost((void**)&h->h_counters, sizeof(Counters)));
+    // shared-memory plan of the per-centre kernels
+    int max_smem = 0;
+    CU(cudaDeviceGetAttribute(&max_smem, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev));
+    for (int deriv = 0; deriv < 2; ++deriv) {
+        int P = 16;
+        size_t bytes = 0;
+        for (; P >= 4; P -= 4) {
+            bytes = (size_t)make_layout(h->S, h->n_max, h->l_max, P, deriv).total * 4;
+            // aim for at least two CTAs per SM
+            if (bytes <= (size_t)max_smem / 2 - 1024 || P == 4) break;
+        }
+        if (bytes > (size_t)max_smem) return fail(h, SOAP_ERR_INVALID_ARG, "this basis does not fit the shared memory of the device");
+        if (deriv) { h->P_deriv = P; h->smem_deriv = bytes; } else { h->P_desc = P; h->smem_desc = bytes; }
+    }
+    CU(cudaFuncSetAttribute(center_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)h->smem_desc));
+    CU(cudaFuncSetAttribute(center_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)h->smem_deriv));
+    h->tables_ready = true;
+    return SOAP_OK;
+}
+
+int ensure_scratch(soap_t* h, int64_t N, int64_t C, int64_t pairs) {
+    if (N > h->cap_atoms) {
+        int64_t cap = N + N / 8 + 256;
+        CU(regrow(&h->d_species_idx, cap));
+        CU(regrow(&h->d_atom_cell, cap));
+        CU(regrow(&h->d_atom_wrap, cap));
+        CU(regrow(&h->d_s_wrap, cap));
+        CU(regrow(&h->d_s_pos, cap));
+        int64_t cells = std::min<int64_t>(std::max<int64_t>(2 * cap, 4096), (int64_t)1 << 26);
+        CU(regrow(&h->d_cell_count, cells + 1));
+        CU(regrow(&h->d_cell_start, cells + 1));
+        h->cap_cells = cells;
+        h->cap_atoms = cap;
+    }
+    if (C > h->cap_centers) {
+        int64_t cap = C + C / 8 + 256;
+        CU(regrow(&h->d_pair_count, cap));
+        CU(regrow(&h->d_row_count, cap));
+        CU(regrow(&h->d_self_row, cap));
+        CU(regrow(&h->d_pair_ptr, cap + 1));
+        CU(regrow(&h->d_row_ptr, cap + 1));
+        h->cap_centers = cap;
+    }
+    if (pairs > h->cap_pairs) {
+        int64_t cap = pairs + pairs / 4 + 1024;
+        CU(regrow(&h->d_pair_key, cap));
+        CU(regrow(&h->d_pair_tmp, cap));
+        CU(regrow(&h->d_pair_row, cap));
+        h->cap_pairs = cap;
+    }
+    return SOAP_OK;
+}
+
+int blocks_for(int64_t n, int threads, int cap = 4096) {
+    return (int)std::max<int64_t>(1, std::min<int64_t>((n + threads - 1) / threads, cap));
+}
+
+// Cell list and pair counts: everything up to the scan of the per-centre counts.
+int launch_count(soap_t* h, const float* pos, const int32_t* num, int64_t N, const Geometry& g,
+                 const int32_t* centers, int64_t C, cudaStream_t st) {
+    CU(cudaMemsetAsync(h->d_bbox, 0, 6 * sizeof(unsigned long long), st));
+    CU(cudaMemsetAsync(h->d_cell_count, 0, (h->cap_cells + 1) * sizeof(int), st));
+    if (N > 0) species_bbox_kernel<<<blocks_for(N, 256, 1024), 256, 0, st>>>(pos, num, N, g, h->d_zlut, h->d_species_idx, h->d_bbox, h->d_counters);
+    grid_setup_kernel<<<1, 1, 0, st>>>(h->d_bbox, g, N, (int)h->cap_cells, h->d_grid);
+    if (N > 0) bin_count_kernel<<<blocks_for(N, 256), 256, 0, st>>>(pos, N, g, h->d_grid, h->d_atom_cell, h->d_atom_wrap, h->d_cell_count, h->d_counters);
+    scan_kernel<int><<<1, 1024, 0, st>>>(h->d_cell_count, h->d_cell_start, h->cap_cells, nullptr);
+    if (N > 0) bin_fill_kernel<<<blocks_for(N, 256), 256, 0, st>>>(pos, N, h->d_atom_cell, h->d_atom_wrap, h->d_cell_start, h->d_cell_count, h->d_s_pos, h->d_s_wrap);
+    if (C > 0) count_kernel<<<(unsigned)((C + 7) / 8), 256, 0, st>>>(pos, centers, C, g, h->d_grid, h->d_atom_cell, h->d_atom_wrap, h->d_cell_start, h->d_s_pos, h->d_s_wrap, h->d_pair_count, h->d_counters);
+    scan_kernel<long long><<<1, 1024, 0, st>>>(h->d_pair_count, h->d_pair_ptr, C, &h->d_counters->n_pairs);
+    CU(cudaGetLastError());
+    return SOAP_OK;
+}
+
+// Sorted pair list and row bookkeeping; row_ptr goes to `row_ptr_out` (the caller's array or the handle's).
+int launch_fill(soap_t* h, const float* pos, const Geometry& g, const int32_t* centers, int64_t C,
+                long long* row_ptr_out, cudaStream_t st) {
+    if (C > 0) fill_kernel<<<(unsigned)((C + kFillWarps - 1) / kFillWarps), kFillWarps * 32, 0, st>>>(
+        pos, centers, C, g, h->d_grid, h->d_atom_cell, h->d_atom_wrap, h->d_cell_start, h->d_s_pos, h->d_s_wrap,
+        h->d_pair_ptr, h->cap_pairs, h->d_pair_tmp, h->d_pair_key, h->d_pair_row, h->d_row_count, h->d_self_row, h->d_counters);
+    scan_kernel<long long><<<1, 1024, 0, st>>>(h->d_row_count, row_ptr_out, C, &h->d_counters->n_rows);
+    CU(cudaGetLastError());
+    return SOAP_OK;
+}
+
+int check_inputs(soap_t* h, const float* pos, const int32_t* num, int64_t N, const int32_t* centers, int64_t C) {
+    if (!h) return SOAP_ERR_INVALID_ARG;
+    if (N < 0 || C < 0 || N > 2000000000LL) return fail(h, SOAP_ERR_INVALID_ARG, "atom or centre count out of range");
+    if (N > 0 && (!pos || !num)) return fail(h, SOAP_ERR_INVALID_ARG, "positions and numbers must not be NULL");
+    if (!centers && C != N) return fail(h, SOAP_ERR_INVALID_ARG, "without a centre list n_centers must equal n_atoms");
+    return SOAP_OK;
+}
+
+// Plans scratch for a structure of this size: count, read the total back, grow.
+int plan(soap_t* h, const float* pos, const int32_t* num, int64_t N, const Geometry& g,
+         const int32_t* centers, int64_t C, cudaStream_t st, int64_t* n_pairs_out) {
+    int rc = ensure_scratch(h, N, C, 0);
+    if (rc) return rc;
+    rc = launch_count(h, pos, num, N, g, centers, C, st);
+    if (rc) return rc;
+    CU(cudaMemcpyAsync(h->h_counters, h->d_counters, sizeof(Counters), cudaMemcpyDeviceToHost, st));
+    CU(cudaStreamSynchronize(st));
+    const int64_t pairs = h->h_counters->n_pairs;
+    rc = ensure_scratch(h, N, C, pairs + pairs / 4 + 1024);
+    if (rc) return rc;
+    h->planned_atoms = N;
+    h->planned_centers = C;
+    if (n_pairs_out) *n_pairs_out = pairs;
+    return SOAP_OK;
+}
+
+void fill_center_params(soap_t* h, CenterParams& cp, const float* pos, const int32_t* centers, int64_t C,
+                        const Geometry& g, bool deriv) {
+    cp.pos = pos; cp.centers = centers; cp.species_idx = h->d_species_idx; cp.n_centers = C; cp.geom = g;
+    cp.pair_ptr = h->d_pair_ptr; cp.pair_key = h->d_pair_key; cp.pair_row = h->d_pair_row;
+    cp.row_ptr = h->d_row_ptr; cp.self_row = h->d_self_row;
+    cp.pair_capacity = h->cap_pairs; cp.row_capacity = 0; cp.counters = h->d_counters;
+    cp.table = h->d_table; cp.self_term = h->d_self; cp.anorm = h->d_anorm; cp.dfact = h->d_dfact; cp.kl = h->d_kl;
+    cp.feat_pack = h->d_feat; cp.inv_h = (float)h->basis.inv_h; cp.n_intervals = h->basis.n_intervals;
+    cp.S = h->S; cp.n_max = h->n_max; cp.l_max = h->l_max; cp.F = (int)h->F;
+    cp.P = deriv ? h->P_deriv : h->P_desc;
+    cp.out_desc = nullptr; cp.out_jac = nullptr; cp.row_atom = nullptr;
+}
+
+}  // namespace
+
+extern "C" {
+
+int soap_create(soap_t** out, const int32_t* species, int n_species, double r_cut, int n_max, int l_max,
+                double sigma, int rbf, const int pbc[3]) {
+    if (!out) return SOAP_ERR_INVALID_ARG;
+    *out = nullptr;
+    soap_t* h = new (std::nothrow) soap_t();
+    if (!h) return SOAP_ERR_ALLOC;
+    auto bail = [&](int code, const std::string& msg) {
+        // keep the object so that soap_last_error can be read; the caller destroys it
+        h->error = msg;
+        *out = h;
+        return code;
+    };
+    if (!species || n_species < 1 || n_species > kMaxSpecies) return bail(SOAP_ERR_INVALID_ARG, "need 1 to 8 species");
+    h->species.assign(species, species + n_species);
+    std::sort(h->species.begin(), h->species.end());
+    for (int s = 0; s < n_species; ++s) {
+        if (h->species[s] < 1 || h->species[s] > 118) return bail(SOAP_ERR_INVALID_ARG, "atomic numbers must lie in 1..118");
+        if (s > 0 && h->species[s] == h->species[s - 1]) return bail(SOAP_ERR_INVALID_ARG, "duplicate species");
+    }
+    h->S = n_species; h->n_max = n_max; h->l_max = l_max; h->rbf = rbf; h->r_cut = r_cut; h->sigma = sigma;
+    for (int a = 0; a < 3; ++a) h->pbc[a] = (pbc && pbc[a]) ? 1 : 0;
+    std::string err;
+    int rc = build_basis(rbf, r_cut, n_max, l_max, sigma, h->basis, err);
+    if (rc) return bail(rc, err);
+    if ((int64_t)n_max * (l_max + 1) * (l_max + 1) > (int64_t)kMaxElemPerThread * kThreads)
+        return bail(SOAP_ERR_INVALID_ARG, "n_max (l_max+1)^2 must not exceed 2048");
+    // feature table: species pairs mu <= nu, radial pair (n' >= n on the diagonal), l fastest
+    for (int mu = 0; mu < h->S; ++mu)
+        for (int nu = mu; nu < h->S; ++nu)
+            for (int n = 0; n < n_max; ++n)
+                for (int n2 = (mu == nu ? n : 0); n2 < n_max; ++n2)
+                    for (int l = 0; l <= l_max; ++l)
+                        h->feat_pack.push_back(n | (n2 << 5) | (mu << 10) | (nu << 14) | (l << 18));
+    h->F = (int64_t)h->feat_pack.size();
+    *out = h;
+    return SOAP_OK;
+}
+
+void soap_destroy(soap_t* h) {
+    if (!h) return;
+    void* ptrs[] = {h->d_table, h->d_self, h->d_anorm, h->d_dfact, h->d_kl, h->d_feat, h->d_zlut, h->d_counters, h->d_bbox,
+                    h->d_grid, h->d_species_idx, h->d_atom_cell, h->d_atom_wrap, h->d_s_wrap, h->d_s_pos, h->d_cell_count,
+                    h->d_cell_start, h->d_pair_count, h->d_row_count, h->d_self_row, h->d_pair_ptr, h->d_row_ptr,
+                    h->d_pair_key, h->d_pair_tmp, h->d_pair_row};
+    for (void* p : ptrs) if (p) cudaFree(p);
+    if (h->h_counters) cudaFreeHost(h->h_counters);
+    delete h;
+}
+
+int soap_num_features(const soap_t* h, int64_t* n_features) {
+    if (!h || !n_features) return SOAP_ERR_INVALID_ARG;
+    *n_features = h->F;
+    return SOAP_OK;
+}
+
+int soap_feature_info(const soap_t* h, int64_t f, int* mu, int* nu, int* n, int* n2, int* l) {
+    if (!h || f < 0 || f >= h->F) return SOAP_ERR_INVALID_ARG;
+    const int pk = h->feat_pack[f];
+    if (n) *n = pk & 31;
+    if (n2) *n2 = (pk >> 5) & 31;
+    if (mu) *mu = (pk >> 10) & 15;
+    if (nu) *nu = (pk >> 14) & 15;
+    if (l) *l = (pk >> 18) & 15;
+    return SOAP_OK;
+}
+
+const char* soap_last_error(const soap_t* h) { return h ? h->error.c_str() : "null handle"; }
+
+int soap_radial_table(const soap_t* h, double d, double* G, double* Ghat) {
+    if (!h || !G || !Ghat || !(d >= 0) || d > h->r_cut) return SOAP_ERR_INVALID_ARG;
+    eval_table(h->basis, d, G, Ghat);
+    return SOAP_OK;
+}
+
+int soap_neighbors(soap_t* h, const float* d_positions, const int32_t* d_numbers, int64_t n_atoms, const double* cell,
+                   const int32_t* d_centers, int64_t n_centers, int64_t* n_pairs, int64_t* n_rows, void* stream) {
+    int rc = check_inputs(h, d_positions, d_numbers, n_atoms, d_centers, n_centers);
+    if (rc) return rc;
+    if ((rc = ensure_device(h))) return rc;
+    Geometry g;
+    if ((rc = make_geometry(h, cell, g))) return rc;
+    cudaStream_t st = (cudaStream_t)stream;
+    int64_t pairs = 0;
+    if ((rc = plan(h, d_positions, d_numbers, n_atoms, g, d_centers, n_centers, st, &pairs))) return rc;
+    if ((rc = launch_fill(h, d_positions, g, d_centers, n_centers, h->d_row_ptr, st))) return rc;
+    CU(cudaMemcpyAsync(h->h_counters, h->d_counters, sizeof(Counters), cudaMemcpyDeviceToHost, st));
+    CU(cudaStreamSynchronize(st));
+    h->last_centers = n_centers;
+    if (n_pairs) *n_pairs = h->h_counters->n_pairs;
+    if (n_rows) *n_rows = h->h_counters->n_rows;
+    return SOAP_OK;
+}
+
+int soap_neighbor_list(soap_t* h, int64_t* d_pair_ptr, int32_t* d_pair_atom, int32_t* d_pair_shift,
+                       int64_t capacity_pairs, void* stream) {
+    if (!h || !d_pair_ptr || !d_pair_atom || capacity_pairs < 0) return SOAP_ERR_INVALID_ARG;
+    if (!h->tables_ready || h->planned_atoms < 0) return fail(h, SOAP_ERR_INVALID_ARG, "no neighbour list has been built yet");
+    cudaStream_t st = (cudaStream_t)stream;
+    export_pairs_kernel<<<256, 256, 0, st>>>(h->d_pair_ptr, h->d_pair_key, h->last_centers, capacity_pairs,
+                                             (long long*)d_pair_ptr, d_pair_atom, d_pair_shift, h->d_counters);
+    CU(cudaGetLastError());
+    return SOAP_OK;
+}
+
+int soap_descriptor(soap_t* h, const float* d_positions, const int32_t* d_numbers, int64_t n_atoms, const double* cell,
+                    const int32_t* d_centers, int64_t n_centers, float* d_out, void* stream) {
+    int rc = check_inputs(h, d_positions, d_numbers, n_atoms, d_centers, n_centers);
+    if (rc) return rc;
+    if (n_centers > 0 && !d_out) return fail(h, SOAP_ERR_INVALID_ARG, "d_out must not be NULL");
+    if ((rc = ensure_device(h))) return rc;
+    Geometry g;
+    if ((rc = make_geometry(h, cell, g))) return rc;
+    cudaStream_t st = (cudaStream_t)stream;
+    if (h->planned_atoms != n_atoms || h->planned_centers != n_centers) {
+        if ((rc = plan(h, d_positions, d_numbers, n_atoms, g, d_centers, n_centers, st, nullptr))) return rc;
+    } else if ((rc = launch_count(h, d_positions, d_numbers, n_atoms, g, d_centers, n_centers, st))) {
+        return rc;
+    }
+    if ((rc = launch_fill(h, d_positions, g, d_centers, n_centers, h->d_row_ptr, st))) return rc;
+    h->last_centers = n_centers;
+    if (n_centers > 0) {
+        CenterParams cp;
+        fill_center_params(h, cp, d_positions, d_centers, n_centers, g, false);
+        cp.out_desc = d_out;
+        center_kernel<false><<<(unsigned)n_centers, kThreads, h->smem_desc, st>>>(cp);
+        CU(cudaGetLastError());
+    }
+    return SOAP_OK;
+}
+
+int soap_derivatives(soap_t* h, const float* d_positions, const int32_t* d_numbers, int64_t n_atoms, const double* cell,
+                     const int32_t* d_centers, int64_t n_centers, float* d_out_desc, float* d_out_jac,
+                     int64_t capacity_rows, int64_t* d_row_ptr, int32_t* d_row_atom, void* stream) {
+    int rc = check_inputs(h, d_positions, d_numbers, n_atoms, d_centers, n_centers);
+    if (rc) return rc;
+    if (!d_row_ptr || capacity_rows < 0) return fail(h, SOAP_ERR_INVALID_ARG, "d_row_ptr must not be NULL");
+    if (n_centers > 0 && (!d_out_desc || !d_out_jac || !d_row_atom)) return fail(h, SOAP_ERR_INVALID_ARG, "output pointers must not be NULL");
+    if ((rc = ensure_device(h))) return rc;
+    Geometry g;
+    if ((rc = make_geometry(h, cell, g))) return rc;
+    cudaStream_t st = (cudaStream_t)stream;
+    if (h->planned_atoms != n_atoms || h->planned_centers != n_centers) {
+        if ((rc = plan(h, d_positions, d_numbers, n_atoms, g, d_centers, n_centers, st, nullptr))) return rc;
+    } else if ((rc = launch_count(h, d_positions, d_numbers, n_atoms, g, d_centers, n_centers, st))) {
+        return rc;
+    }
+    if ((rc = launch_fill(h, d_positions, g, d_centers, n_centers, (long long*)d_row_ptr, st))) return rc;
+    h->last_centers = n_centers;
+    if (n_centers > 0) {
+        CenterParams cp;
+        fill_center_params(h, cp, d_positions, d_centers, n_centers, g, true);
+        cp.row_ptr = (const long long*)d_row_ptr;
+        cp.row_capacity = capacity_rows;
+        cp.out_desc = d_out_desc; cp.out_jac = d_out_jac; cp.row_atom = d_row_atom;
+        center_kernel<true><<<(unsigned)n_centers, kThreads, h->smem_deriv, st>>>(cp);
+        CU(cudaGetLastError());
+    }
+    return SOAP_OK;
+}
+
+int soap_status(soap_t* h, int64_t* n_pairs, int64_t* n_rows, void* stream) {
+    if (!h) return SOAP_ERR_INVALID_ARG;
+    if (!h->tables_ready) return SOAP_OK;
+    cudaStream_t st = (cudaStream_t)stream;
+    CU(cudaMemcpyAsync(h->h_counters, h->d_counters, sizeof(Counters), cudaMemcpyDeviceToHost, st));
+    CU(cudaMemsetAsync(&h->d_counters->status, 0, sizeof(int), st));
+    CU(cudaStreamSynchronize(st));
+    if (n_pairs) *n_pairs = h->h_counters->n_pairs;
+    if (n_rows) *n_rows = h->h_counters->n_rows;
+    const int s = h->h_counters->status;
+    if (s & kStatusUnknownSpecies) return fail(h, SOAP_ERR_UNKNOWN_SPECIES, "an atomic number is not in the species list");
+    if (s & kStatusShiftRange) return fail(h, SOAP_ERR_INVALID_ARG, "positions lie too many cells away from the unit cell");
+    if (s & kStatusPairCapacity) return fail(h, SOAP_ERR_CAPACITY, "more pairs than planned (call soap_neighbors again) or than the export buffer holds");
+    if (s & kStatusRowCapacity) return fail(h, SOAP_ERR_CAPACITY, "more Jacobian rows than capacity_rows");
+    return SOAP_OK;
+}
+
+}  // extern "C"

