@@ -154,7 +154,7 @@ int ensure_device(soap_t* h) {
 }
 
 int ensure_scratch(soap_t* h, int64_t N, int64_t C, int64_t pairs) {
-    if (N > h->cap_atoms) {
+    if (N > h->cap_atoms || h->cap_atoms == 0) {
         int64_t cap = N + N / 8 + 256;
         CU(regrow(&h->d_species_idx, cap));
         CU(regrow(&h->d_atom_cell, cap));
@@ -167,7 +167,7 @@ int ensure_scratch(soap_t* h, int64_t N, int64_t C, int64_t pairs) {
         h->cap_cells = cells;
         h->cap_atoms = cap;
     }
-    if (C > h->cap_centers) {
+    if (C > h->cap_centers || h->cap_centers == 0) {
         int64_t cap = C + C / 8 + 256;
         CU(regrow(&h->d_pair_count, cap));
         CU(regrow(&h->d_row_count, cap));
@@ -176,7 +176,7 @@ int ensure_scratch(soap_t* h, int64_t N, int64_t C, int64_t pairs) {
         CU(regrow(&h->d_row_ptr, cap + 1));
         h->cap_centers = cap;
     }
-    if (pairs > h->cap_pairs) {
+    if (pairs > h->cap_pairs || h->cap_pairs == 0) {
         int64_t cap = pairs + pairs / 4 + 1024;
         CU(regrow(&h->d_pair_key, cap));
         CU(regrow(&h->d_pair_tmp, cap));
