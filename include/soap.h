@@ -127,6 +127,15 @@ int soap_derivatives(soap_t *h, const float *d_positions, const int32_t *d_numbe
  * pair and row counts of the last call (either pointer may be NULL). */
 int soap_status(soap_t *h, int64_t *n_pairs, int64_t *n_rows, void *stream);
 
+/* Per-segment timing, the counterpart of the paper's companion profiler
+ * (end of its architecture section).  With profiling enabled,
+ * soap_descriptor and soap_derivatives record CUDA events on the caller's
+ * stream around (a) the neighbour search and (b) the fused per-centre kernel.
+ * soap_profile_read waits for the last call's events and returns both
+ * durations in milliseconds.  Events cost about a microsecond; off by default. */
+int soap_profile(soap_t *h, int enable);
+int soap_profile_read(soap_t *h, float *ms_neighbors, float *ms_center);
+
 #ifdef __cplusplus
 }
 #endif

@@ -12,7 +12,7 @@ GTO, POLYNOMIAL = 0, 1
 EXPORTED_SYMBOLS = [
     "soap_create", "soap_destroy", "soap_num_features", "soap_feature_info", "soap_last_error",
     "soap_radial_table", "soap_neighbors", "soap_neighbor_list", "soap_descriptor",
-    "soap_derivatives", "soap_status",
+    "soap_derivatives", "soap_status", "soap_profile", "soap_profile_read",
 ]
 
 _ERRORS = {-1: "SOAP_ERR_INVALID_ARG", -2: "SOAP_ERR_UNKNOWN_SPECIES", -3: "SOAP_ERR_CAPACITY",
@@ -56,6 +56,8 @@ def load_library() -> C.CDLL:
     lib.soap_descriptor.argtypes = common + [vp, vp]
     lib.soap_derivatives.argtypes = common + [vp, vp, i64, vp, vp, vp]
     lib.soap_status.argtypes = [vp, C.POINTER(i64), C.POINTER(i64), vp]
+    lib.soap_profile.argtypes = [vp, i32]
+    lib.soap_profile_read.argtypes = [vp, C.POINTER(C.c_float), C.POINTER(C.c_float)]
     for name in EXPORTED_SYMBOLS:
         if name not in ("soap_destroy", "soap_last_error"):
             getattr(lib, name).restype = C.c_int
@@ -196,6 +198,27 @@ class Soap:
         self.derivatives_into(positions, numbers, cell, centers, desc, jac, row_ptr, row_atom)
         self.status()
         return Derivatives(desc, jac[:nrows], row_ptr, row_atom[:nrows])
+
+    def profile(self, enable=True):
+        self._check(self._lib.soap_profile(self._h, int(bool(enable))))
+
+    def profile_read(self):
+        """(ms in the neighbour search, ms in the fused per-centre kernel) of the last call."""
+        a, b = C.c_float(), C.c_float()
+        self._check(self._lib.soap_profile_read(self._h, C.byref(a), C.byref(b)))
+        return float(a.value), float(b.value)
+
+    def derivatives_host(self, positions, numbers, cell, host_out, dev_buf):
+        """End-to-end call on HOST buffers: copies the (pinned) inputs to the device,
+        computes, and copies descriptor, Jacobian, row_ptr and row_atom back into the
+        pinned tensors of `host_out`.  `dev_buf` holds the device staging tensors.
+        Everything is enqueued on the current stream; the caller synchronises."""
+        dev_buf["pos"].copy_(positions, non_blocking=True)
+        dev_buf["num"].copy_(numbers, non_blocking=True)
+        self.derivatives_into(dev_buf["pos"], dev_buf["num"], cell, None, dev_buf["desc"], dev_buf["jac"],
+                              dev_buf["row_ptr"], dev_buf["row_atom"])
+        for k in ("desc", "jac", "row_ptr", "row_atom"):
+            host_out[k].copy_(dev_buf[k], non_blocking=True)
 
     def status(self):
         """Waits for the stream; raises if the device flagged a problem. Returns (n_pairs, n_rows)."""

@@ -49,7 +49,9 @@ struct soap_handle {
     int64_t last_centers = 0;
     int P_desc = 16, P_deriv = 16;
     size_t smem_desc = 0, smem_deriv = 0;
-    bool attr_set = false;
+    // optional per-segment timing (events on the caller's stream)
+    bool profiling = false;
+    cudaEvent_t ev[3] = {nullptr, nullptr, nullptr};
 };
 
 namespace {
@@ -306,6 +308,7 @@ void soap_destroy(soap_t* h) {
                     h->d_pair_key, h->d_pair_tmp, h->d_pair_row};
     for (void* p : ptrs) if (p) cudaFree(p);
     if (h->h_counters) cudaFreeHost(h->h_counters);
+    for (cudaEvent_t e : h->ev) if (e) cudaEventDestroy(e);
     delete h;
 }
 
@@ -373,12 +376,14 @@ int soap_descriptor(soap_t* h, const float* d_positions, const int32_t* d_number
     Geometry g;
     if ((rc = make_geometry(h, cell, g))) return rc;
     cudaStream_t st = (cudaStream_t)stream;
+    if (h->profiling) CU(cudaEventRecord(h->ev[0], st));
     if (h->planned_atoms != n_atoms || h->planned_centers != n_centers) {
         if ((rc = plan(h, d_positions, d_numbers, n_atoms, g, d_centers, n_centers, st, nullptr))) return rc;
     } else if ((rc = launch_count(h, d_positions, d_numbers, n_atoms, g, d_centers, n_centers, st))) {
         return rc;
     }
     if ((rc = launch_fill(h, d_positions, g, d_centers, n_centers, h->d_row_ptr, st))) return rc;
+    if (h->profiling) CU(cudaEventRecord(h->ev[1], st));
     h->last_centers = n_centers;
     if (n_centers > 0) {
         CenterParams cp;
@@ -387,6 +392,7 @@ int soap_descriptor(soap_t* h, const float* d_positions, const int32_t* d_number
         center_kernel<false><<<(unsigned)n_centers, kThreads, h->smem_desc, st>>>(cp);
         CU(cudaGetLastError());
     }
+    if (h->profiling) CU(cudaEventRecord(h->ev[2], st));
     return SOAP_OK;
 }
 
@@ -401,12 +407,14 @@ int soap_derivatives(soap_t* h, const float* d_positions, const int32_t* d_numbe
     Geometry g;
     if ((rc = make_geometry(h, cell, g))) return rc;
     cudaStream_t st = (cudaStream_t)stream;
+    if (h->profiling) CU(cudaEventRecord(h->ev[0], st));
     if (h->planned_atoms != n_atoms || h->planned_centers != n_centers) {
         if ((rc = plan(h, d_positions, d_numbers, n_atoms, g, d_centers, n_centers, st, nullptr))) return rc;
     } else if ((rc = launch_count(h, d_positions, d_numbers, n_atoms, g, d_centers, n_centers, st))) {
         return rc;
     }
     if ((rc = launch_fill(h, d_positions, g, d_centers, n_centers, (long long*)d_row_ptr, st))) return rc;
+    if (h->profiling) CU(cudaEventRecord(h->ev[1], st));
     h->last_centers = n_centers;
     if (n_centers > 0) {
         CenterParams cp;
@@ -417,6 +425,7 @@ int soap_derivatives(soap_t* h, const float* d_positions, const int32_t* d_numbe
         center_kernel<true><<<(unsigned)n_centers, kThreads, h->smem_deriv, st>>>(cp);
         CU(cudaGetLastError());
     }
+    if (h->profiling) CU(cudaEventRecord(h->ev[2], st));
     return SOAP_OK;
 }
 
@@ -434,6 +443,29 @@ int soap_status(soap_t* h, int64_t* n_pairs, int64_t* n_rows, void* stream) {
     if (s & kStatusShiftRange) return fail(h, SOAP_ERR_INVALID_ARG, "positions lie too many cells away from the unit cell");
     if (s & kStatusPairCapacity) return fail(h, SOAP_ERR_CAPACITY, "more pairs than planned (call soap_neighbors again) or than the export buffer holds");
     if (s & kStatusRowCapacity) return fail(h, SOAP_ERR_CAPACITY, "more Jacobian rows than capacity_rows");
+    return SOAP_OK;
+}
+
+int soap_profile(soap_t* h, int enable) {
+    if (!h) return SOAP_ERR_INVALID_ARG;
+    if (enable) {
+        int rc = ensure_device(h);
+        if (rc) return rc;
+        for (cudaEvent_t& e : h->ev)
+            if (!e) CU(cudaEventCreate(&e));
+    }
+    h->profiling = enable != 0;
+    return SOAP_OK;
+}
+
+int soap_profile_read(soap_t* h, float* ms_neighbors, float* ms_center) {
+    if (!h || !h->ev[2]) return SOAP_ERR_INVALID_ARG;
+    CU(cudaEventSynchronize(h->ev[2]));
+    float a = 0.f, b = 0.f;
+    CU(cudaEventElapsedTime(&a, h->ev[0], h->ev[1]));
+    CU(cudaEventElapsedTime(&b, h->ev[1], h->ev[2]));
+    if (ms_neighbors) *ms_neighbors = a;
+    if (ms_center) *ms_center = b;
     return SOAP_OK;
 }
 
