@@ -32,6 +32,7 @@ WORKLOADS = {
     # name: (generator, generator args, species, r_cut, n_max, l_max, sigma, rbf)
     "water1000_gto_n8_l6_rc6": ("water", 1000, [1, 8], 6.0, 8, 6, 0.5, 0),
     "water8_gto_n4_l3_rc5": ("water", 8, [1, 8], 5.0, 4, 3, 0.5, 0),
+    "water300_gto_n8_l6_rc6": ("water", 300, [1, 8], 6.0, 8, 6, 0.5, 0),      # small case for ncu captures
     "chno2000_poly_n8_l8_rc5": ("box", 2000, [1, 6, 7, 8], 5.0, 8, 8, 0.4, 1),
 }
 DEFAULT_WORKLOAD = "water1000_gto_n8_l6_rc6"
@@ -224,11 +225,13 @@ def run_cuda(args):
     soap.status()
     total_ms = sum(step_ms)
     # ---- end to end on host buffers: H2D of the inputs, compute, D2H of every output ----
-    host_out = {k: torch.empty(v.shape, dtype=v.dtype).pin_memory() for k, v in dev.items() if k not in ("pos", "num")}
-    for _ in range(2):
-        soap.derivatives_host(pos_host, num_host, s.cell, host_out, dev)
+    e2e_steps = 0 if args.kernel_only else max(3, min(args.steps, 10))
+    host_out = {}
+    if e2e_steps:
+        host_out = {k: torch.empty(v.shape, dtype=v.dtype).pin_memory() for k, v in dev.items() if k not in ("pos", "num")}
+        for _ in range(2):
+            soap.derivatives_host(pos_host, num_host, s.cell, host_out, dev)
     torch.cuda.synchronize()
-    e2e_steps = max(3, min(args.steps, 10))
     barrier()
     e2e_ms = []
     for _ in range(e2e_steps):
@@ -251,7 +254,7 @@ def run_cuda(args):
         return
     ms_per_step = total_ms / args.steps
     value = world * C / (ms_per_step * 1e-3)
-    e2e_value = world * C / (e2e_total / e2e_steps * 1e-3)
+    e2e_value = world * C / (e2e_total / e2e_steps * 1e-3) if e2e_steps else None
     # ---- roofline of the dominant kernel (the fused per-centre kernel): HBM-write bound ----
     # algorithmic bytes per launch: Jacobian rows + descriptor + row_atom written, pair list and positions read
     alg_bytes = n_rows * 3 * F * 4 + C * F * 4 + n_rows * 4 + n_pairs * (8 + 4 + 12) + (C + 1) * 16
@@ -262,14 +265,17 @@ def run_cuda(args):
     d2h = sum(v.numel() * v.element_size() for v in host_out.values())
     # ---- oracle on the host cores, bounded sample ----
     n_sample = 600 if name == DEFAULT_WORKLOAD else 64
-    cpu_value, cpu_times, _ = oracle_rate(name, n_sample)
+    if args.kernel_only:
+        cpu_value, cpu_times = None, [0.0]
+    else:
+        cpu_value, cpu_times, _ = oracle_rate(name, n_sample)
     print(json.dumps({
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3),
         "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "f32", "data": "synthetic", "config": config_dict(name, s),
         "clocks": clocks,
         "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
-                "ms_per_step": e2e_total / e2e_steps, "steps": e2e_steps},
+                "ms_per_step": e2e_total / e2e_steps if e2e_steps else None, "steps": e2e_steps},
         "gpu_launches": KERNELS_PER_STEP * args.steps,
         "roofline": {"bound": "hbm", "kernel": "center_kernel<true>", "achieved": achieved, "peak": peak, "unit": "GB/s",
                      "frac": achieved / peak, "peak_source": peak_src, "traffic": None,
@@ -291,6 +297,8 @@ def main():
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="cuda", choices=["cuda", "reference"])
     ap.add_argument("--workload", default=DEFAULT_WORKLOAD, choices=sorted(WORKLOADS))
+    ap.add_argument("--kernel-only", action="store_true",
+                    help="skip the end-to-end and CPU-baseline legs (for profiler captures)")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)

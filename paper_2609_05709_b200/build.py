@@ -4,6 +4,7 @@ from __future__ import annotations
 import os
 import subprocess
 import sys
+from concurrent.futures import ThreadPoolExecutor
 
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
@@ -12,6 +13,7 @@ LIB = os.path.join(HERE, "libsoap_b200.so")
 
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-O3", "-lineinfo", "-std=c++17",
               "--expt-relaxed-constexpr", "-Xcompiler", "-fPIC", "-Xptxas", "-v"]
+CUDA_UNITS = ["soap_api", "center_g0", "center_g1", "center_g2", "center_g3"]
 
 
 def _newer(target, sources):
@@ -21,25 +23,32 @@ def _newer(target, sources):
     return any(os.path.getmtime(s) > t for s in sources)
 
 
+def _run(cmd, verbose, log):
+    res = subprocess.run(cmd, capture_output=True, text=True)
+    log.append(" ".join(cmd) + "\n" + res.stdout + res.stderr)
+    if res.returncode != 0:
+        sys.stderr.write(log[-1])
+        raise RuntimeError("build failed: " + " ".join(cmd))
+
+
 def build(force: bool = False, verbose: bool = False) -> str:
-    sources = [os.path.join(CSRC, f) for f in sorted(os.listdir(CSRC))] + [os.path.join(INCLUDE, "soap.h")]
+    sources = [os.path.join(CSRC, f) for f in sorted(os.listdir(CSRC)) if not f.endswith(".o")]
+    sources.append(os.path.join(INCLUDE, "soap.h"))
     if not force and not _newer(LIB, sources):
         return LIB
     nvcc = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
-    obj_host = os.path.join(CSRC, "basis_host.o")
-    obj_api = os.path.join(CSRC, "soap_api.o")
-    cmds = [
-        ["g++", "-O2", "-std=gnu++17", "-fPIC", "-ffp-contract=off", "-I", INCLUDE, "-I", CSRC,
-         "-c", os.path.join(CSRC, "basis_host.cpp"), "-o", obj_host],
-        [nvcc, *NVCC_FLAGS, "-I", INCLUDE, "-I", CSRC, "-c", os.path.join(CSRC, "soap_api.cu"), "-o", obj_api],
-        [nvcc, "-shared", "-o", LIB, obj_api, obj_host, "-lquadmath", "-cudart", "static"],
-    ]
-    for cmd in cmds:
-        res = subprocess.run(cmd, capture_output=True, text=True)
-        if verbose or res.returncode != 0:
-            sys.stderr.write(" ".join(cmd) + "\n" + res.stdout + res.stderr)
-        if res.returncode != 0:
-            raise RuntimeError("build failed: " + " ".join(cmd))
+    obj = lambda name: os.path.join(CSRC, name + ".o")
+    cmds = [["g++", "-O2", "-std=gnu++17", "-fPIC", "-ffp-contract=off", "-I", INCLUDE, "-I", CSRC,
+             "-c", os.path.join(CSRC, "basis_host.cpp"), "-o", obj("basis_host")]]
+    for unit in CUDA_UNITS:
+        cmds.append([nvcc, *NVCC_FLAGS, "-I", INCLUDE, "-I", CSRC, "-c", os.path.join(CSRC, unit + ".cu"), "-o", obj(unit)])
+    log = []
+    with ThreadPoolExecutor(max_workers=len(cmds)) as pool:
+        list(pool.map(lambda c: _run(c, verbose, log), cmds))
+    _run([nvcc, "-shared", "-o", LIB, *[obj(u) for u in CUDA_UNITS], obj("basis_host"), "-lquadmath", "-cudart", "static"],
+         verbose, log)
+    if verbose:
+        sys.stderr.write("\n".join(log))
     return LIB
 
 

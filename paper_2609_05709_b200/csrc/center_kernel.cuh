@@ -1,28 +1,95 @@
 // The fused per-centre kernel: one CTA owns one centre atom and produces its
 // descriptor row (Eq. 4) and, in the derivative build, all of its Jacobian
 // rows (Eq. 5).  Nothing per pair ever goes to HBM: radial factors, solid
-// harmonics and the precontracted U/V live in shared memory for a chunk of
-// pairs at a time; the expansion coefficients c^mu_nlm of the centre stay in
-// shared memory for the whole CTA lifetime.
+// harmonics and the precontracted U/V live in shared memory; the expansion
+// coefficients c^mu_nlm of the centre stay in shared memory for the CTA's life.
 //
 // Per pair (displacement d = r_j + T - r_i, species Z of j):
 //   c^Z_nlm        += G_nl(|d|) S_lm(d)                               (Eq. 13 / 18)
 //   grad_j c^Z_nlm  = G_nl grad S_lm + Ghat_nl d S_lm,  Ghat = G'/|d|  (Eq. 14 / 23)
 // with S_lm = r^l Y_lm the real solid harmonic and G_nl, G'_nl read from the
-// degree-5 tables.  Pass 1 accumulates c and D = sum_j grad_j c (for the
-// centre's own row, which is minus the sum over the neighbours).  Pass 2 forms,
-// per pair, U^nu_{n'l} = K_l sum_m S_lm c^nu_{n'lm} and V likewise with grad S,
-// and then each output element of Eq. 5 is two fused multiply-adds per term.
+// degree-5 tables.
+//   Pass 1 (whole CTA per chunk of pairs) accumulates c and D = sum_j grad_j c;
+//   the centre's own Jacobian row is minus the sum over its neighbours, which is
+//   a contraction of D with c.
+//   Pass 2 (one warp per pair, no block barriers) forms U^nu_{n'l} = K_l sum_m
+//   S_lm c^nu_{n'lm} and V likewise with grad S, after which every output
+//   element of Eq. 5 is two fused multiply-adds per term, and streams the row
+//   out with lanes on consecutive features.
+// l_max is a template parameter so that the harmonic recursions unroll and the
+// index arithmetic folds; n_max and the species count stay run-time values.
 #pragma once
 #include "soap_device.cuh"
 
 namespace soap {
 
-__device__ inline int tri_index(int l, int m) { return l * (l + 1) / 2 + m; }
+// Real solid harmonics S_{l,+m}, S_{l,-m} (and gradients) for one (l, m >= 0):
+//   S_{l,+m} = a_lm Q_l^m Re (x+iy)^m,   S_{l,-m} = a_lm Q_l^m Im (x+iy)^m,
+//   Q_l^m = r^(l-m) d^m P_l(t)/dt^m at t = z/r, by the recurrence
+//   (l-m) Q_l^m = (2l-1) z Q_{l-1}^m - (l+m-1) r^2 Q_{l-2}^m,  Q_m^m = (2m-1)!!,
+//   dQ_l^m/dx = -x Q_{l-1}^{m+1},  dQ_l^m/dy = -y Q_{l-1}^{m+1},  dQ_l^m/dz = (l+m) Q_{l-1}^m.
+// Every lane runs the same unrolled, predicated recurrences for its own (l, m).
+template <int L, bool GRAD>
+__device__ __forceinline__ void solid_harmonic_item(float x, float y, float z, float r2, int l, int m,
+                                                    const float* __restrict__ anorm, const float* __restrict__ dfact,
+                                                    const float* __restrict__ inv_int,
+                                                    float4& plus, float4& minus) {
+    float cm = 1.f, sm = 0.f, cp = 0.f, sp = 0.f;          // (x+iy)^m and (x+iy)^(m-1)
+#pragma unroll
+    for (int t = 0; t < L; ++t)
+        if (t < m) {
+            cp = cm; sp = sm;
+            const float cn = x * cm - y * sm;
+            sm = x * sm + y * cm;
+            cm = cn;
+        }
+    float qa = __ldg(dfact + m), qb = 0.f;                  // Q_ll^m, Q_{ll-1}^m
+    float qc = 0.f, qd = 0.f;                               // Q_ll^{m+1}, Q_{ll-1}^{m+1} (up to ll = l-1)
+    if (GRAD && m + 1 <= l - 1) qc = __ldg(dfact + m + 1);
+#pragma unroll
+    for (int ll = 1; ll <= L; ++ll) {
+        if (ll > m && ll <= l) {
+            const float qn = ((2 * ll - 1) * z * qa - (ll + m - 1) * r2 * qb) * __ldg(inv_int + ll - m);
+            qb = qa; qa = qn;
+        }
+        if (GRAD && ll > m + 1 && ll <= l - 1) {
+            const float qn = ((2 * ll - 1) * z * qc - (ll + m) * r2 * qd) * __ldg(inv_int + ll - m - 1);
+            qd = qc; qc = qn;
+        }
+    }
+    const float a = __ldg(anorm + l * (l + 1) / 2 + m);
+    const float aq = a * qa;
+    if (!GRAD) {
+        plus.x = aq * cm;
+        minus.x = aq * sm;
+        return;
+    }
+    const float qz = (l > m) ? a * (l + m) * qb : 0.f;      // a dQ/dz
+    const float qx = a * qc;                                // a Q_{l-1}^{m+1} (0 when it does not exist)
+    const float mq = m * aq;
+    plus = make_float4(aq * cm, -x * qx * cm + mq * cp, -y * qx * cm - mq * sp, qz * cm);
+    minus = make_float4(aq * sm, -x * qx * sm + mq * sp, -y * qx * sm + mq * cp, qz * sm);
+}
 
-template <bool DERIV>
-__global__ void __launch_bounds__(kThreads)
+// Degree-5 table lookup: value and derivative with respect to the interval coordinate t.
+__device__ __forceinline__ void radial_lookup(const float* __restrict__ table, int qi, int n_ch, int ch, float t,
+                                              float& v, float& dv) {
+    const float2* cf = reinterpret_cast<const float2*>(table + ((size_t)qi * n_ch + ch) * 6);
+    const float2 a = __ldg(cf), b = __ldg(cf + 1), c = __ldg(cf + 2);
+    v = c.y; dv = 0.f;
+    dv = fmaf(dv, t, v); v = fmaf(v, t, c.x);
+    dv = fmaf(dv, t, v); v = fmaf(v, t, b.y);
+    dv = fmaf(dv, t, v); v = fmaf(v, t, b.x);
+    dv = fmaf(dv, t, v); v = fmaf(v, t, a.y);
+    dv = fmaf(dv, t, v); v = fmaf(v, t, a.x);
+}
+
+template <bool DERIV, int L>
+__global__ void __launch_bounds__(kThreads, DERIV ? 3 : 4)
 center_kernel(const CenterParams p) {
+    constexpr int L1 = L + 1, LM = L1 * L1, NQ = L1 * (L1 + 1) / 2;
+    constexpr int KE = (16 * LM + kThreads - 1) / kThreads < kMaxElemPerThread ? (16 * LM + kThreads - 1) / kThreads
+                                                                                : kMaxElemPerThread;
     extern __shared__ __align__(16) float smem[];
     const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
     const long long c_idx = blockIdx.x;
@@ -32,20 +99,16 @@ center_kernel(const CenterParams p) {
         if (c_idx == 0 && tid == 0) atomicOr(&p.counters->status, kStatusRowCapacity);
         return;
     }
-    const int S = p.S, NMAX = p.n_max, L = p.l_max, L1 = L + 1, LM = L1 * L1, NCH = NMAX * L1;
-    const int NE = NMAX * LM, CT = S * NE, NQ = L1 * (L1 + 1) / 2, P = p.P, F = p.F;
+    const int S = p.S, NMAX = p.n_max, NCH = NMAX * L1, NE = NMAX * LM, CT = S * NE, P = p.P, F = p.F;
     const SmemLayout lay = make_layout(S, NMAX, L, P, DERIV);
     float* c_t = smem + lay.c;
-    float* D_t = smem + lay.D;                             // [3][CT]
-    float4* sd = reinterpret_cast<float4*>(smem + lay.sd); // dx, dy, dz, r
-    int2* sinfo = reinterpret_cast<int2*>(smem + lay.sinfo);   // species | moving<<8 ; pair_row word
-    float* sS = smem + lay.sSD;                            // desc: [P][LM]
-    float4* sSD4 = reinterpret_cast<float4*>(smem + lay.sSD);  // deriv: [P][LM] (S, dSx, dSy, dSz)
-    float* sG1 = smem + lay.sG;                            // desc: [P][NCH]
-    float2* sG2 = reinterpret_cast<float2*>(smem + lay.sG);    // deriv: [P][NCH] (G, Ghat)
-    float* sQ = smem + lay.sQ;                             // [P][NQ]
-    float2* sCS = reinterpret_cast<float2*>(smem + lay.sCS);   // [P][L1]
-    float4* sUV = reinterpret_cast<float4*>(smem + lay.sUV);   // [P][S*NCH]
+    float4* geo_d = reinterpret_cast<float4*>(smem + lay.geo);             // [GP] dx, dy, dz, r
+    int4* geo_i = reinterpret_cast<int4*>(smem + lay.geo + 4 * kGeoPairs);   // [GP] interval, t bits, species|moving<<8, row word
+    float* D_t = smem + lay.D;                                             // [3][CT]           (pass 1)
+    float* sS = smem + lay.sSD;                                            // [P][LM]           (pass 1, descriptor build)
+    float4* sSD4 = reinterpret_cast<float4*>(smem + lay.sSD);              // [P][LM]           (pass 1, derivative build)
+    float* sG1 = smem + lay.sG;
+    float2* sG2 = reinterpret_cast<float2*>(smem + lay.sG);                // [P][NCH]
 
     const int ci = p.centers ? p.centers[c_idx] : (int)c_idx;
     const float xi = p.pos[3 * (long long)ci], yi = p.pos[3 * (long long)ci + 1], zi = p.pos[3 * (long long)ci + 2];
@@ -59,22 +122,19 @@ center_kernel(const CenterParams p) {
     }
 
     // elements (n, lm) this thread accumulates in pass 1
-    int el_lm[kMaxElemPerThread], el_ch[kMaxElemPerThread];
+    int el_lm[KE], el_ch[KE];
 #pragma unroll
-    for (int k = 0; k < kMaxElemPerThread; ++k) {
-        int e = tid + k * kThreads;
-        int n = e / LM, lm = e - n * LM;
-        int l = (int)sqrtf((float)lm);
-        while ((l + 1) * (l + 1) <= lm) ++l;
-        while (l * l > lm) --l;
+    for (int k = 0; k < KE; ++k) {
+        const int e = tid + k * kThreads;
+        const int n = e / LM, lm = e - n * LM;
         el_lm[k] = e < NE ? lm : -1;
-        el_ch[k] = n * L1 + l;
+        el_ch[k] = n * L1 + __ldg(p.l_of_lm + lm);
     }
 
-    // ---- stage one chunk of pairs: geometry, radial factors, solid harmonics ----
-    auto stage_chunk = [&](int q0, int pc) {
-        if (tid < pc) {
-            const unsigned long long key = p.pair_key[pair_base + q0 + tid];
+    // ---- geometry of up to kGeoPairs pairs, one thread each ----
+    auto stage_geometry = [&](int g0, int gc) {
+        if (tid < gc) {
+            const unsigned long long key = p.pair_key[pair_base + g0 + tid];
             const int j = key_atom(key);
             double dx = (double)p.pos[3 * (long long)j] - (double)xi;
             double dy = (double)p.pos[3 * (long long)j + 1] - (double)yi;
@@ -87,134 +147,95 @@ center_kernel(const CenterParams p) {
                 dz += s[0] * p.geom.cell[2] + s[1] * p.geom.cell[5] + s[2] * p.geom.cell[8];
             }
             const double r = sqrt(dx * dx + dy * dy + dz * dz);
-            sd[tid] = make_float4((float)dx, (float)dy, (float)dz, (float)r);
-            const int rw = p.pair_row[pair_base + q0 + tid];
-            sinfo[tid] = make_int2(p.species_idx[j] | ((rw & kRowSelfImage) ? 0 : 256), rw);
+            geo_d[tid] = make_float4((float)dx, (float)dy, (float)dz, (float)r);
+            const int rw = p.pair_row[pair_base + g0 + tid];
             // interval and offset in the radial table, in fp64 so that the offset keeps its digits
-            double u = r * (double)p.inv_h;
-            int qi = min((int)u, p.n_intervals - 1);
-            sCS[tid * L1] = make_float2(__int_as_float(qi), (float)(u - qi));   // parked here until the harmonics overwrite it
+            const double u = r * (double)p.inv_h;
+            const int qi = min((int)u, p.n_intervals - 1);
+            geo_i[tid] = make_int4(qi, __float_as_int((float)(u - qi)),
+                                   p.species_idx[j] | ((rw & kRowSelfImage) ? 0 : 256), rw);
         }
-        __syncthreads();
-        // radial factors: thread <-> (pair, channel)
-        for (int idx = tid; idx < pc * NCH; idx += kThreads) {
-            const int pr = idx / NCH, ch = idx - pr * NCH;
-            const float2 it = sCS[pr * L1];
-            const int qi = __float_as_int(it.x);
-            const float t = it.y;
-            const float2* cf = reinterpret_cast<const float2*>(p.table + ((size_t)qi * NCH + ch) * 6);
-            const float2 a = __ldg(cf), b = __ldg(cf + 1), cc = __ldg(cf + 2);
-            float v = cc.y, dv = 0.f;
-            dv = fmaf(dv, t, v); v = fmaf(v, t, cc.x);
-            dv = fmaf(dv, t, v); v = fmaf(v, t, b.y);
-            dv = fmaf(dv, t, v); v = fmaf(v, t, b.x);
-            dv = fmaf(dv, t, v); v = fmaf(v, t, a.y);
-            dv = fmaf(dv, t, v); v = fmaf(v, t, a.x);
-            if (DERIV) sG2[pr * NCH + ch] = make_float2(v, dv * p.inv_h / sd[pr].w);
-            else sG1[pr * NCH + ch] = v;
-        }
-        __syncthreads();
-        // harmonics, step 1: thread <-> (pair, m): (x+iy)^m and the column Q_l^m, l = m..L
-        for (int idx = tid; idx < pc * L1; idx += kThreads) {
-            const int pr = idx / L1, m = idx - pr * L1;
-            const float4 d = sd[pr];
-            float cm = 1.f, sm = 0.f;
-            for (int t = 0; t < m; ++t) {
-                const float cn = d.x * cm - d.y * sm;
-                sm = d.x * sm + d.y * cm;
-                cm = cn;
-            }
-            sCS[pr * L1 + m] = make_float2(cm, sm);
-            const float r2 = d.w * d.w;
-            float q0v = 0.f, q1v = __ldg(p.dfact + m);          // Q_m^m = (2m-1)!!
-            sQ[pr * NQ + tri_index(m, m)] = q1v;
-            for (int l = m + 1; l <= L; ++l) {
-                // (l-m) Q_l^m = (2l-1) z Q_{l-1}^m - (l+m-1) r^2 Q_{l-2}^m
-                const float qn = ((2 * l - 1) * d.z * q1v - (l + m - 1) * r2 * q0v) / (float)(l - m);
-                q0v = q1v; q1v = qn;
-                sQ[pr * NQ + tri_index(l, m)] = qn;
-            }
-        }
-        __syncthreads();
-        // harmonics, step 2: thread <-> (pair, l, m >= 0): S_{l,+-m} and, for the Jacobian, their gradients
-        for (int idx = tid; idx < pc * NQ; idx += kThreads) {
-            const int pr = idx / NQ, t = idx - pr * NQ;
-            int l = (int)((sqrtf(8.f * t + 1.f) - 1.f) * 0.5f);
-            while (tri_index(l + 1, 0) <= t) ++l;
-            while (tri_index(l, 0) > t) --l;
-            const int m = t - tri_index(l, 0);
-            const float a = __ldg(p.anorm + t);
-            const float Q = sQ[pr * NQ + t];
-            const float2 cs = sCS[pr * L1 + m];
-            const int lm0 = l * l + l;
-            if (!DERIV) {
-                if (m == 0) sS[pr * LM + lm0] = a * Q;
-                else { sS[pr * LM + lm0 + m] = a * Q * cs.x; sS[pr * LM + lm0 - m] = a * Q * cs.y; }
-            } else {
-                const float4 d = sd[pr];
-                // dQ_l^m/dx = -x Q_{l-1}^{m+1}, dQ_l^m/dy = -y Q_{l-1}^{m+1}, dQ_l^m/dz = (l+m) Q_{l-1}^m
-                const float Qx = (l - 1 >= m + 1) ? sQ[pr * NQ + tri_index(l - 1, m + 1)] : 0.f;
-                const float Qz = (l - 1 >= m) ? (l + m) * sQ[pr * NQ + tri_index(l - 1, m)] : 0.f;
-                if (m == 0) {
-                    sSD4[pr * LM + lm0] = make_float4(a * Q, -a * d.x * Qx, -a * d.y * Qx, a * Qz);
-                } else {
-                    const float2 cp = sCS[pr * L1 + m - 1];
-                    const float mq = m * Q;
-                    // d/dx (x+iy)^m = m (x+iy)^(m-1), d/dy = i m (x+iy)^(m-1)
-                    sSD4[pr * LM + lm0 + m] = make_float4(a * Q * cs.x, a * (-d.x * Qx * cs.x + mq * cp.x),
-                                                         a * (-d.y * Qx * cs.x - mq * cp.y), a * Qz * cs.x);
-                    sSD4[pr * LM + lm0 - m] = make_float4(a * Q * cs.y, a * (-d.x * Qx * cs.y + mq * cp.y),
-                                                         a * (-d.y * Qx * cs.y + mq * cp.x), a * Qz * cs.y);
-                }
-            }
-        }
-        __syncthreads();
     };
 
     // =========================== pass 1: c (and D) ===========================
-    for (int q0 = 0; q0 < k_pairs; q0 += P) {
-        const int pc = min(P, k_pairs - q0);
-        stage_chunk(q0, pc);
-        for (int s = 0; s < S; ++s) {
-            float ac[kMaxElemPerThread], ax[kMaxElemPerThread], ay[kMaxElemPerThread], az[kMaxElemPerThread];
-#pragma unroll
-            for (int k = 0; k < kMaxElemPerThread; ++k) ac[k] = ax[k] = ay[k] = az[k] = 0.f;
-            bool any = false;
-            for (int pr = 0; pr < pc; ++pr) {
-                const int info = sinfo[pr].x;
-                if ((info & 255) != s) continue;
-                any = true;
-                if (!DERIV) {
-#pragma unroll
-                    for (int k = 0; k < kMaxElemPerThread; ++k)
-                        if (el_lm[k] >= 0) ac[k] = fmaf(sG1[pr * NCH + el_ch[k]], sS[pr * LM + el_lm[k]], ac[k]);
+    for (int g0 = 0; g0 < k_pairs; g0 += kGeoPairs) {
+        const int gc = min(kGeoPairs, k_pairs - g0);
+        __syncthreads();
+        stage_geometry(g0, gc);
+        __syncthreads();
+        for (int q0 = 0; q0 < gc; q0 += P) {
+            const int pc = min(P, gc - q0);
+            // radial factors: warp <-> pair, lane <-> channel
+            for (int pr = wid; pr < pc; pr += kWarps) {
+                const int4 gi = geo_i[q0 + pr];
+                const float t = __int_as_float(gi.y);
+                const float rinv_h = p.inv_h / geo_d[q0 + pr].w;
+                for (int ch = lane; ch < NCH; ch += 32) {
+                    float v, dv;
+                    radial_lookup(p.table, gi.x, NCH, ch, t, v, dv);
+                    if (DERIV) sG2[pr * NCH + ch] = make_float2(v, dv * rinv_h);
+                    else sG1[pr * NCH + ch] = v;
+                }
+            }
+            // solid harmonics: thread <-> (pair, (l, m >= 0))
+            for (int idx = tid; idx < pc * NQ; idx += kThreads) {
+                const int pr = idx / NQ, t = idx - pr * NQ;
+                const int lmp = __ldg(p.lm_of_t + t);
+                const int l = lmp >> 4, m = lmp & 15;
+                const float4 d = geo_d[q0 + pr];
+                float4 plus, minus;
+                solid_harmonic_item<L, DERIV>(d.x, d.y, d.z, d.w * d.w, l, m, p.anorm, p.dfact, p.inv_int, plus, minus);
+                const int lm0 = l * l + l;
+                if (DERIV) {
+                    sSD4[pr * LM + lm0 + m] = plus;
+                    if (m) sSD4[pr * LM + lm0 - m] = minus;
                 } else {
-                    const float4 d = sd[pr];
-                    const float mv = (info & 256) ? 1.f : 0.f;   // an image of the centre does not move relative to it
+                    sS[pr * LM + lm0 + m] = plus.x;
+                    if (m) sS[pr * LM + lm0 - m] = minus.x;
+                }
+            }
+            __syncthreads();
+            for (int s = 0; s < S; ++s) {
+                float ac[KE], ax[KE], ay[KE], az[KE];
 #pragma unroll
-                    for (int k = 0; k < kMaxElemPerThread; ++k)
+                for (int k = 0; k < KE; ++k) ac[k] = ax[k] = ay[k] = az[k] = 0.f;
+                bool any = false;
+                for (int pr = 0; pr < pc; ++pr) {
+                    const int info = geo_i[q0 + pr].z;
+                    if ((info & 255) != s) continue;
+                    any = true;
+                    if (!DERIV) {
+#pragma unroll
+                        for (int k = 0; k < KE; ++k)
+                            if (el_lm[k] >= 0) ac[k] = fmaf(sG1[pr * NCH + el_ch[k]], sS[pr * LM + el_lm[k]], ac[k]);
+                    } else {
+                        const float4 d = geo_d[q0 + pr];
+                        const float mv = (info & 256) ? 1.f : 0.f;   // an image of the centre does not move relative to it
+#pragma unroll
+                        for (int k = 0; k < KE; ++k)
+                            if (el_lm[k] >= 0) {
+                                const float2 g = sG2[pr * NCH + el_ch[k]];
+                                const float4 h = sSD4[pr * LM + el_lm[k]];
+                                ac[k] = fmaf(g.x, h.x, ac[k]);
+                                const float gm = g.x * mv, t = g.y * h.x * mv;
+                                ax[k] = fmaf(gm, h.y, fmaf(t, d.x, ax[k]));
+                                ay[k] = fmaf(gm, h.z, fmaf(t, d.y, ay[k]));
+                                az[k] = fmaf(gm, h.w, fmaf(t, d.z, az[k]));
+                            }
+                    }
+                }
+                if (any) {
+#pragma unroll
+                    for (int k = 0; k < KE; ++k)
                         if (el_lm[k] >= 0) {
-                            const float2 g = sG2[pr * NCH + el_ch[k]];
-                            const float4 h = sSD4[pr * LM + el_lm[k]];
-                            ac[k] = fmaf(g.x, h.x, ac[k]);
-                            const float gm = g.x * mv, t = g.y * h.x * mv;
-                            ax[k] = fmaf(gm, h.y, fmaf(t, d.x, ax[k]));
-                            ay[k] = fmaf(gm, h.z, fmaf(t, d.y, ay[k]));
-                            az[k] = fmaf(gm, h.w, fmaf(t, d.z, az[k]));
+                            const int e = s * NE + tid + k * kThreads;
+                            c_t[e] += ac[k];
+                            if (DERIV) { D_t[e] += ax[k]; D_t[CT + e] += ay[k]; D_t[2 * CT + e] += az[k]; }
                         }
                 }
             }
-            if (any) {
-#pragma unroll
-                for (int k = 0; k < kMaxElemPerThread; ++k)
-                    if (el_lm[k] >= 0) {
-                        const int e = s * NE + tid + k * kThreads;
-                        c_t[e] += ac[k];
-                        if (DERIV) { D_t[e] += ax[k]; D_t[CT + e] += ay[k]; D_t[2 * CT + e] += az[k]; }
-                    }
-            }
+            __syncthreads();
         }
-        __syncthreads();
     }
     __syncthreads();
     // on-site term: the centre's own Gaussian, l = 0 only (second term of Eq. 13)
@@ -244,71 +265,83 @@ center_kernel(const CenterParams p) {
             const int n1 = pk & 31, n2 = (pk >> 5) & 31, mu = (pk >> 10) & 15, nu = (pk >> 14) & 15, l = (pk >> 18) & 15;
             const int ia = (mu * NMAX + n1) * LM + l * l, ib = (nu * NMAX + n2) * LM + l * l;
             const float kl = -__ldg(p.kl + l);
-            for (int dir = 0; dir < 3; ++dir) {
-                const float* Da = D_t + dir * CT + ia;
-                const float* Db = D_t + dir * CT + ib;
-                float acc = 0.f;
-                for (int m = 0; m <= 2 * l; ++m) acc = fmaf(Da[m], c_t[ib + m], fmaf(c_t[ia + m], Db[m], acc));
-                out[(size_t)dir * F + f] = kl * acc;
+            float ax = 0.f, ay = 0.f, az = 0.f;
+            for (int m = 0; m <= 2 * l; ++m) {
+                const float ca = c_t[ia + m], cb = c_t[ib + m];
+                ax = fmaf(D_t[ia + m], cb, fmaf(ca, D_t[ib + m], ax));
+                ay = fmaf(D_t[CT + ia + m], cb, fmaf(ca, D_t[CT + ib + m], ay));
+                az = fmaf(D_t[2 * CT + ia + m], cb, fmaf(ca, D_t[2 * CT + ib + m], az));
             }
+            out[f] = kl * ax; out[(size_t)F + f] = kl * ay; out[(size_t)2 * F + f] = kl * az;
         }
         if (tid == 0) p.row_atom[row_base + my_row] = ci;
     }
     __syncthreads();
-    // fold K_l into c for pass 2 (D is dead from here; its space becomes the U/V staging)
-    for (int e = tid; e < CT; e += kThreads) {
-        int lm = e % LM;
-        int l = (int)sqrtf((float)lm);
-        while ((l + 1) * (l + 1) <= lm) ++l;
-        while (l * l > lm) --l;
-        c_t[e] *= __ldg(p.kl + l);
-    }
-    __syncthreads();
+    // fold K_l into c for pass 2 (D and the pass-1 staging are dead from here; their space
+    // becomes the per-warp staging of pass 2)
+    for (int e = tid; e < CT; e += kThreads) c_t[e] *= __ldg(p.kl + __ldg(p.l_of_lm + e % LM));
 
-    // lane-fixed channels j = (n', l) of phase C
-    const int NI = S * NCH;
     // =========================== pass 2: the Jacobian rows ===========================
-    for (int q0 = 0; q0 < k_pairs; q0 += P) {
-        const int pc = min(P, k_pairs - q0);
-        stage_chunk(q0, pc);
-        // ---- phase B: U, V per pair and (nu, n', l); a thread serves 4 pairs of one item ----
-        const int groups = (pc + 3) >> 2;
-        for (int unit = tid; unit < groups * NI; unit += kThreads) {
-            const int pg = unit / NI, item = unit - pg * NI;
-            const int l = item % L1;
-            const float* cp = c_t + (item / L1) * LM + l * l;
-            float4 acc[4];
-#pragma unroll
-            for (int a = 0; a < 4; ++a) acc[a] = make_float4(0.f, 0.f, 0.f, 0.f);
-            for (int m = 0; m <= 2 * l; ++m) {
-                const float cv = cp[m];
-#pragma unroll
-                for (int a = 0; a < 4; ++a) {
-                    const float4 h = sSD4[(pg * 4 + a) * LM + l * l + m];
-                    acc[a].x = fmaf(cv, h.x, acc[a].x);
-                    acc[a].y = fmaf(cv, h.y, acc[a].y);
-                    acc[a].z = fmaf(cv, h.z, acc[a].z);
-                    acc[a].w = fmaf(cv, h.w, acc[a].w);
-                }
-            }
-#pragma unroll
-            for (int a = 0; a < 4; ++a) sUV[(pg * 4 + a) * NI + item] = acc[a];
-        }
+    const int NI = S * NCH;
+    float4* wSD = reinterpret_cast<float4*>(smem + lay.w2 + wid * lay.w2_stride);         // [LM]
+    float2* wG = reinterpret_cast<float2*>(smem + lay.w2 + wid * lay.w2_stride + 4 * LM);  // [NCH]
+    float4* wUV = reinterpret_cast<float4*>(smem + lay.w2 + wid * lay.w2_stride + 4 * LM + ((2 * NCH + 3) & ~3));   // [NI]
+    for (int g0 = 0; g0 < k_pairs; g0 += kGeoPairs) {
+        const int gc = min(kGeoPairs, k_pairs - g0);
         __syncthreads();
-        // ---- phase C: product rule and store; a warp owns whole rows ----
-        for (int pr = 0; pr < pc; ++pr) {
-            const int2 info = sinfo[pr];
-            const int rw = info.y;
+        if (g0 > 0 || k_pairs > kGeoPairs) stage_geometry(g0, gc);     // otherwise still valid from pass 1
+        __syncthreads();
+        for (int pr = 0; pr < gc; ++pr) {
+            const int4 gi = geo_i[pr];
+            const int rw = gi.w;
             if (rw & kRowSelfImage) continue;
             const int row = rw & kRowMask;
-            if ((row % kWarps) != wid) continue;
+            if ((row & (kWarps - 1)) != wid) continue;
             const bool accumulate = rw & kRowContinuation;
-            const int Z = info.x & 255;
-            const float4 d = sd[pr];
+            const int Z = gi.z & 255;
+            const float4 d = geo_d[pr];
+            __syncwarp();
+            // ---- radial factors and harmonics of this pair ----
+            {
+                const float t = __int_as_float(gi.y);
+                const float rinv_h = p.inv_h / d.w;
+                for (int ch = lane; ch < NCH; ch += 32) {
+                    float v, dv;
+                    radial_lookup(p.table, gi.x, NCH, ch, t, v, dv);
+                    wG[ch] = make_float2(v, dv * rinv_h);
+                }
+                for (int t2 = lane; t2 < NQ; t2 += 32) {
+                    const int lmp = __ldg(p.lm_of_t + t2);
+                    const int l = lmp >> 4, m = lmp & 15;
+                    float4 plus, minus;
+                    solid_harmonic_item<L, true>(d.x, d.y, d.z, d.w * d.w, l, m, p.anorm, p.dfact, p.inv_int, plus, minus);
+                    const int lm0 = l * l + l;
+                    wSD[lm0 + m] = plus;
+                    if (m) wSD[lm0 - m] = minus;
+                }
+            }
+            __syncwarp();
+            // ---- U, V for every (nu, n', l); items ordered l-major so that a warp's trip counts agree ----
+            {
+                const int SN = S * NMAX;
+                for (int it = lane; it < NI; it += 32) {
+                    const int l = it / SN, sn = it - l * SN;            // sn = nu * NMAX + n'
+                    const float* cp = c_t + sn * LM + l * l;
+                    const float4* hp = wSD + l * l;
+                    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+                    for (int m = 0; m <= 2 * l; ++m) {
+                        const float cv = cp[m];
+                        const float4 h = hp[m];
+                        acc.x = fmaf(cv, h.x, acc.x); acc.y = fmaf(cv, h.y, acc.y);
+                        acc.z = fmaf(cv, h.z, acc.z); acc.w = fmaf(cv, h.w, acc.w);
+                    }
+                    wUV[sn * L1 + l] = acc;                           // [nu][n'][l]
+                }
+            }
+            __syncwarp();
+            // ---- product rule and store ----
             float* out = p.out_jac + (size_t)(row_base + row) * 3 * F;
-            if (!accumulate && lane == 0) p.row_atom[row_base + row] = key_atom(p.pair_key[pair_base + q0 + pr]);
-            const float2* G = sG2 + pr * NCH;
-            const float4* UV = sUV + pr * NI;
+            if (!accumulate && lane == 0) p.row_atom[row_base + row] = key_atom(p.pair_key[pair_base + g0 + pr]);
             int boff = 0;
             for (int mu = 0; mu < S; ++mu) {
                 for (int nu = mu; nu < S; ++nu) {
@@ -318,55 +351,64 @@ center_kernel(const CenterParams p) {
                         if (!accumulate)
                             for (int f = lane; f < bsize; f += 32) { ob[f] = 0.f; ob[F + f] = 0.f; ob[2 * F + f] = 0.f; }
                     } else if (mu == nu) {
-                        // both terms; features (n1 <= n2, l) at tri(n1) + (n2-n1) L1 + l
+                        // both terms; feature (n1 <= n2, l) sits at L1 (n1 NMAX - n1(n1-1)/2) + (n2-n1) L1 + l
+                        const float4* UVz = wUV + Z * NCH;
                         for (int j = lane; j < NCH; j += 32) {
                             const int n2 = j / L1, l = j - n2 * L1;
-                            const float2 gj = G[j];
-                            const float4 uj = UV[Z * NCH + j];
-                            const float tj = gj.y;
+                            const float2 gj = wG[j];
+                            const float4 uj = UVz[j];
+                            const float2* g1p = wG + l;
+                            const float4* u1p = UVz + l;
+                            float* o = ob + j;
                             for (int n1 = 0; n1 <= n2; ++n1) {
-                                const int i1 = n1 * L1 + l;
-                                const float2 g1 = G[i1];
-                                const float4 u1 = UV[Z * NCH + i1];
-                                const float w = g1.y * uj.x + tj * u1.x;          // Ghat_n1 U_n2 + Ghat_n2 U_n1
+                                const float2 g1 = *g1p;
+                                const float4 u1 = *u1p;
+                                const float w = fmaf(g1.y, uj.x, gj.y * u1.x);    // Ghat_n1 U_n2 + Ghat_n2 U_n1
                                 const float vx = fmaf(g1.x, uj.y, fmaf(gj.x, u1.y, w * d.x));
                                 const float vy = fmaf(g1.x, uj.z, fmaf(gj.x, u1.z, w * d.y));
                                 const float vz = fmaf(g1.x, uj.w, fmaf(gj.x, u1.w, w * d.z));
-                                const int f = (n1 * NMAX - n1 * (n1 - 1) / 2) * L1 + (n2 - n1) * L1 + l;
-                                if (accumulate) { ob[f] += vx; ob[F + f] += vy; ob[2 * F + f] += vz; }
-                                else { ob[f] = vx; ob[F + f] = vy; ob[2 * F + f] = vz; }
+                                if (accumulate) { o[0] += vx; o[F] += vy; o[2 * F] += vz; }
+                                else { o[0] = vx; o[F] = vy; o[2 * F] = vz; }
+                                g1p += L1; u1p += L1;
+                                o += (NMAX - n1 - 1) * L1;
                             }
                         }
                     } else if (mu == Z) {
                         // (grad c^mu_{n1 l}) c^nu_{n2 l}: G_{n1 l} V^nu_{n2 l} + Ghat_{n1 l} d U^nu_{n2 l}
                         for (int j = lane; j < NCH; j += 32) {
                             const int l = j % L1;
-                            const float4 uj = UV[nu * NCH + j];
+                            const float4 uj = wUV[nu * NCH + j];
                             const float xx = uj.x * d.x, xy = uj.x * d.y, xz = uj.x * d.z;
+                            const float2* g1p = wG + l;
+                            float* o = ob + j;
+#pragma unroll 4
                             for (int n1 = 0; n1 < NMAX; ++n1) {
-                                const float2 g1 = G[n1 * L1 + l];
+                                const float2 g1 = *g1p;
                                 const float vx = fmaf(g1.x, uj.y, g1.y * xx);
                                 const float vy = fmaf(g1.x, uj.z, g1.y * xy);
                                 const float vz = fmaf(g1.x, uj.w, g1.y * xz);
-                                const int f = n1 * NCH + j;
-                                if (accumulate) { ob[f] += vx; ob[F + f] += vy; ob[2 * F + f] += vz; }
-                                else { ob[f] = vx; ob[F + f] = vy; ob[2 * F + f] = vz; }
+                                if (accumulate) { o[0] += vx; o[F] += vy; o[2 * F] += vz; }
+                                else { o[0] = vx; o[F] = vy; o[2 * F] = vz; }
+                                g1p += L1; o += NCH;
                             }
                         }
                     } else {
                         // c^mu_{n1 l} (grad c^nu_{n2 l}): G_{n2 l} V^mu_{n1 l} + Ghat_{n2 l} d U^mu_{n1 l}
                         for (int j = lane; j < NCH; j += 32) {
                             const int l = j % L1;
-                            const float2 gj = G[j];
+                            const float2 gj = wG[j];
                             const float gx = gj.y * d.x, gy = gj.y * d.y, gz = gj.y * d.z;
+                            const float4* u1p = wUV + mu * NCH + l;
+                            float* o = ob + j;
+#pragma unroll 4
                             for (int n1 = 0; n1 < NMAX; ++n1) {
-                                const float4 u1 = UV[mu * NCH + n1 * L1 + l];
+                                const float4 u1 = *u1p;
                                 const float vx = fmaf(gj.x, u1.y, gx * u1.x);
                                 const float vy = fmaf(gj.x, u1.z, gy * u1.x);
                                 const float vz = fmaf(gj.x, u1.w, gz * u1.x);
-                                const int f = n1 * NCH + j;
-                                if (accumulate) { ob[f] += vx; ob[F + f] += vy; ob[2 * F + f] += vz; }
-                                else { ob[f] = vx; ob[F + f] = vy; ob[2 * F + f] = vz; }
+                                if (accumulate) { o[0] += vx; o[F] += vy; o[2 * F] += vz; }
+                                else { o[0] = vx; o[F] = vy; o[2 * F] = vz; }
+                                u1p += L1; o += NCH;
                             }
                         }
                     }
@@ -374,7 +416,6 @@ center_kernel(const CenterParams p) {
                 }
             }
         }
-        __syncthreads();
     }
 }
 

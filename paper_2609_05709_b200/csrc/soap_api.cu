@@ -10,11 +10,31 @@
 #include <vector>
 
 #include "basis_host.h"
-#include "center_kernel.cuh"
+#include "center_launch.h"
 #include "neighbor_kernels.cuh"
 #include "soap.h"
 
 using namespace soap;
+
+namespace soap {
+static int group_of(int l_max) { return l_max <= 5 ? 0 : l_max <= 8 ? 1 : l_max <= 10 ? 2 : 3; }
+cudaError_t center_set_smem(bool deriv, int l_max, int bytes) {
+    switch (group_of(l_max)) {
+        case 0: return center_set_smem_g0(deriv, l_max, bytes);
+        case 1: return center_set_smem_g1(deriv, l_max, bytes);
+        case 2: return center_set_smem_g2(deriv, l_max, bytes);
+        default: return center_set_smem_g3(deriv, l_max, bytes);
+    }
+}
+cudaError_t center_launch(bool deriv, int l_max, const CenterParams& p, unsigned grid, size_t smem, cudaStream_t st) {
+    switch (group_of(l_max)) {
+        case 0: return center_launch_g0(deriv, l_max, p, grid, smem, st);
+        case 1: return center_launch_g1(deriv, l_max, p, grid, smem, st);
+        case 2: return center_launch_g2(deriv, l_max, p, grid, smem, st);
+        default: return center_launch_g3(deriv, l_max, p, grid, smem, st);
+    }
+}
+}  // namespace soap
 
 struct soap_handle {
     // configuration
@@ -29,8 +49,8 @@ struct soap_handle {
     // device state (created on first use)
     int device = -1;
     bool tables_ready = false;
-    float *d_table = nullptr, *d_self = nullptr, *d_anorm = nullptr, *d_dfact = nullptr, *d_kl = nullptr;
-    int *d_feat = nullptr, *d_zlut = nullptr;
+    float *d_table = nullptr, *d_self = nullptr, *d_anorm = nullptr, *d_dfact = nullptr, *d_kl = nullptr, *d_inv_int = nullptr;
+    int *d_feat = nullptr, *d_zlut = nullptr, *d_lm_of_t = nullptr, *d_l_of_lm = nullptr;
     Counters* d_counters = nullptr;
     unsigned long long* d_bbox = nullptr;
     GridParams* d_grid = nullptr;
@@ -127,6 +147,18 @@ int ensure_device(soap_t* h) {
     CU(upload(&h->d_dfact, h->basis.dfact));
     CU(upload(&h->d_kl, h->basis.kl));
     CU(upload(&h->d_feat, h->feat_pack));
+    {
+        std::vector<float> inv(32, 0.f);
+        for (int k = 1; k < 32; ++k) inv[k] = 1.0f / k;
+        CU(upload(&h->d_inv_int, inv));
+        std::vector<int> lm_of_t, l_of_lm;
+        for (int l = 0; l <= h->l_max; ++l) {
+            for (int m = 0; m <= l; ++m) lm_of_t.push_back((l << 4) | m);
+            for (int m = -l; m <= l; ++m) l_of_lm.push_back(l);
+        }
+        CU(upload(&h->d_lm_of_t, lm_of_t));
+        CU(upload(&h->d_l_of_lm, l_of_lm));
+    }
     std::vector<int> lut(128, -1);
     for (int s = 0; s < h->S; ++s) lut[h->species[s]] = s;
     CU(upload(&h->d_zlut, lut));
@@ -141,16 +173,16 @@ int ensure_device(soap_t* h) {
     for (int deriv = 0; deriv < 2; ++deriv) {
         int P = 16;
         size_t bytes = 0;
-        for (; P >= 4; P -= 4) {
+        for (; P >= 2; P /= 2) {
             bytes = (size_t)make_layout(h->S, h->n_max, h->l_max, P, deriv).total * 4;
             // aim for at least two CTAs per SM
-            if (bytes <= (size_t)max_smem / 2 - 1024 || P == 4) break;
+            if (bytes <= (size_t)max_smem / 2 - 1024 || P == 2) break;
         }
         if (bytes > (size_t)max_smem) return fail(h, SOAP_ERR_INVALID_ARG, "this basis does not fit the shared memory of the device");
         if (deriv) { h->P_deriv = P; h->smem_deriv = bytes; } else { h->P_desc = P; h->smem_desc = bytes; }
     }
-    CU(cudaFuncSetAttribute(center_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)h->smem_desc));
-    CU(cudaFuncSetAttribute(center_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)h->smem_deriv));
+    CU(center_set_smem(false, h->l_max, (int)h->smem_desc));
+    CU(center_set_smem(true, h->l_max, (int)h->smem_deriv));
     h->tables_ready = true;
     return SOAP_OK;
 }
@@ -252,6 +284,7 @@ void fill_center_params(soap_t* h, CenterParams& cp, const float* pos, const int
     cp.row_ptr = h->d_row_ptr; cp.self_row = h->d_self_row;
     cp.pair_capacity = h->cap_pairs; cp.row_capacity = 0; cp.counters = h->d_counters;
     cp.table = h->d_table; cp.self_term = h->d_self; cp.anorm = h->d_anorm; cp.dfact = h->d_dfact; cp.kl = h->d_kl;
+    cp.inv_int = h->d_inv_int; cp.lm_of_t = h->d_lm_of_t; cp.l_of_lm = h->d_l_of_lm;
     cp.feat_pack = h->d_feat; cp.inv_h = (float)h->basis.inv_h; cp.n_intervals = h->basis.n_intervals;
     cp.S = h->S; cp.n_max = h->n_max; cp.l_max = h->l_max; cp.F = (int)h->F;
     cp.P = deriv ? h->P_deriv : h->P_desc;
@@ -302,7 +335,7 @@ int soap_create(soap_t** out, const int32_t* species, int n_species, double r_cu
 
 void soap_destroy(soap_t* h) {
     if (!h) return;
-    void* ptrs[] = {h->d_table, h->d_self, h->d_anorm, h->d_dfact, h->d_kl, h->d_feat, h->d_zlut, h->d_counters, h->d_bbox,
+    void* ptrs[] = {h->d_table, h->d_self, h->d_anorm, h->d_dfact, h->d_kl, h->d_feat, h->d_zlut, h->d_inv_int, h->d_lm_of_t, h->d_l_of_lm, h->d_counters, h->d_bbox,
                     h->d_grid, h->d_species_idx, h->d_atom_cell, h->d_atom_wrap, h->d_s_wrap, h->d_s_pos, h->d_cell_count,
                     h->d_cell_start, h->d_pair_count, h->d_row_count, h->d_self_row, h->d_pair_ptr, h->d_row_ptr,
                     h->d_pair_key, h->d_pair_tmp, h->d_pair_row};
@@ -389,8 +422,7 @@ int soap_descriptor(soap_t* h, const float* d_positions, const int32_t* d_number
         CenterParams cp;
         fill_center_params(h, cp, d_positions, d_centers, n_centers, g, false);
         cp.out_desc = d_out;
-        center_kernel<false><<<(unsigned)n_centers, kThreads, h->smem_desc, st>>>(cp);
-        CU(cudaGetLastError());
+        CU(center_launch(false, h->l_max, cp, (unsigned)n_centers, h->smem_desc, st));
     }
     if (h->profiling) CU(cudaEventRecord(h->ev[2], st));
     return SOAP_OK;
@@ -422,8 +454,7 @@ int soap_derivatives(soap_t* h, const float* d_positions, const int32_t* d_numbe
         cp.row_ptr = (const long long*)d_row_ptr;
         cp.row_capacity = capacity_rows;
         cp.out_desc = d_out_desc; cp.out_jac = d_out_jac; cp.row_atom = d_row_atom;
-        center_kernel<true><<<(unsigned)n_centers, kThreads, h->smem_deriv, st>>>(cp);
-        CU(cudaGetLastError());
+        CU(center_launch(true, h->l_max, cp, (unsigned)n_centers, h->smem_deriv, st));
     }
     if (h->profiling) CU(cudaEventRecord(h->ev[2], st));
     return SOAP_OK;

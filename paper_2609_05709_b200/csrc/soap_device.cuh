@@ -65,14 +65,17 @@ struct CenterParams {
     // basis
     const float* table;           // [nint][n_ch][6]
     const float* self_term;       // [n_max]
-    const float* anorm;
-    const float* dfact;
+    const float* anorm;           // [(l,m)] harmonic normalisation
+    const float* dfact;           // [m] (2m-1)!!
+    const float* inv_int;         // [k] 1/k
+    const int* lm_of_t;           // [(l,m) index] -> l<<4 | m
+    const int* l_of_lm;           // [lm] -> l
     const float* kl;
     const int* feat_pack;         // [F] n | n'<<5 | mu<<10 | nu<<14 | l<<18
     float inv_h;
     int n_intervals;
     int S, n_max, l_max, F;
-    int P;                        // pairs per chunk (multiple of 4, <= 32)
+    int P;                        // pairs per pass-1 chunk
     // outputs
     float* out_desc;              // [C,F]
     float* out_jac;               // [rows,3,F]
@@ -86,28 +89,32 @@ __host__ __device__ inline void key_shift(unsigned long long k, int s[3]) {
     s[2] = (int)(k & 255) - 128;
 }
 
-// Shared-memory carve-up of the per-centre kernel, in 4-byte words.
+// Shared-memory carve-up of the per-centre kernel, in 4-byte words.  Every region
+// starts on a 16-byte boundary.  The pass-1 regions (D tiles, chunk staging) and
+// the per-warp staging of pass 2 never live at the same time and share space.
+constexpr int kGeoPairs = 128;           // pairs whose geometry is staged at once
+
 struct SmemLayout {
-    int c, D, sd, sinfo, sSD, sG, sQ, sCS, sUV, total;
+    int c, geo, D, sSD, sG, w2, w2_stride, total;
 };
+__host__ __device__ inline int align4(int x) { return (x + 3) & ~3; }
 __host__ __device__ inline SmemLayout make_layout(int S, int n_max, int l_max, int P, bool deriv) {
     const int L1 = l_max + 1, LM = L1 * L1, NCH = n_max * L1, CT = S * n_max * LM;
     SmemLayout o;
-    int off = 0;                                   // every region starts on a 16-byte boundary
-    o.c = off; off = (off + CT + 3) & ~3;
-    o.sd = off; off += P * 4;
-    o.sinfo = off; off = (off + P * 2 + 3) & ~3;
-    o.sSD = off; off = (off + (deriv ? P * LM * 4 : P * LM) + 3) & ~3;
-    o.sG = off; off = (off + (deriv ? P * NCH * 2 : P * NCH) + 3) & ~3;
-    o.sQ = off; off = (off + P * (L1 * (L1 + 1) / 2) + 3) & ~3;
-    o.sCS = off; off = (off + P * L1 * 2 + 3) & ~3;
-    // the D tiles (pass 1) and the U/V staging (pass 2) never live at the same time
-    o.D = off; o.sUV = off;
-    if (deriv) {
-        int a = 3 * CT, b = P * S * NCH * 4;
-        off += a > b ? a : b;
-    }
-    o.total = off;
+    int off = 0;
+    o.c = off; off = align4(off + CT);
+    o.geo = off; off += kGeoPairs * 8;
+    const int u = off;
+    // pass 1
+    o.D = off; if (deriv) off = align4(off + 3 * CT);
+    o.sSD = off; off = align4(off + (deriv ? P * LM * 4 : P * LM));
+    o.sG = off; off = align4(off + (deriv ? P * NCH * 2 : P * NCH));
+    const int end1 = off;
+    // pass 2: per warp [LM] float4 harmonics, [NCH] float2 radial, [S*NCH] float4 U/V
+    o.w2 = u;
+    o.w2_stride = 4 * LM + align4(2 * NCH) + 4 * S * NCH;
+    const int end2 = deriv ? u + kWarps * o.w2_stride : u;
+    o.total = end1 > end2 ? end1 : end2;
     return o;
 }
 
