@@ -13,7 +13,7 @@ LIB = os.path.join(HERE, "libsoap_b200.so")
 
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-O3", "-lineinfo", "-std=c++17",
               "--expt-relaxed-constexpr", "-Xcompiler", "-fPIC", "-Xptxas", "-v"]
-CUDA_UNITS = ["soap_api", "center_g0", "center_g1", "center_g2", "center_g3"]
+CUDA_UNITS = ["soap_api"] + [f"center_l{l}" for l in range(13)]
 
 
 def _newer(target, sources):
@@ -43,7 +43,7 @@ def build(force: bool = False, verbose: bool = False) -> str:
     for unit in CUDA_UNITS:
         cmds.append([nvcc, *NVCC_FLAGS, "-I", INCLUDE, "-I", CSRC, "-c", os.path.join(CSRC, unit + ".cu"), "-o", obj(unit)])
     log = []
-    with ThreadPoolExecutor(max_workers=len(cmds)) as pool:
+    with ThreadPoolExecutor(max_workers=min(len(cmds), os.cpu_count() or 4)) as pool:
         list(pool.map(lambda c: _run(c, verbose, log), cmds))
     _run([nvcc, "-shared", "-o", LIB, *[obj(u) for u in CUDA_UNITS], obj("basis_host"), "-lquadmath", "-cudart", "static"],
          verbose, log)

@@ -9,67 +9,22 @@
 //   grad_j c^Z_nlm  = G_nl grad S_lm + Ghat_nl d S_lm,  Ghat = G'/|d|  (Eq. 14 / 23)
 // with S_lm = r^l Y_lm the real solid harmonic and G_nl, G'_nl read from the
 // degree-5 tables.
-//   Pass 1 (whole CTA per chunk of pairs) accumulates c and D = sum_j grad_j c;
-//   the centre's own Jacobian row is minus the sum over its neighbours, which is
-//   a contraction of D with c.
-//   Pass 2 (one warp per pair, no block barriers) forms U^nu_{n'l} = K_l sum_m
-//   S_lm c^nu_{n'lm} and V likewise with grad S, after which every output
-//   element of Eq. 5 is two fused multiply-adds per term, and streams the row
-//   out with lanes on consecutive features.
-// l_max is a template parameter so that the harmonic recursions unroll and the
-// index arithmetic folds; n_max and the species count stay run-time values.
+//   Staging (whole CTA, a chunk of up to 32 pairs): radial factors with a warp per
+//   pair and lanes on channels; solid harmonics with lanes on pairs and warps on
+//   the columns m of the recursion, so that control flow is uniform.
+//   Pass 1 accumulates c and D = sum_j grad_j c with thread-owned elements; the
+//   centre's own Jacobian row is minus the sum over its neighbours, which is a
+//   contraction of D with c.
+//   Pass 2 gives every pair to one warp: it forms U^nu_{n'l} = K_l sum_m S_lm
+//   c^nu_{n'lm} and V likewise with grad S, after which every output element of
+//   Eq. 5 is two fused multiply-adds per term, and streams the row out with lanes
+//   on consecutive features.
+// l_max and n_max are template parameters (n_max = 0 means "read it at run
+// time") so that loops unroll and the store addresses become immediates.
 #pragma once
 #include "soap_device.cuh"
 
 namespace soap {
-
-// Real solid harmonics S_{l,+m}, S_{l,-m} (and gradients) for one (l, m >= 0):
-//   S_{l,+m} = a_lm Q_l^m Re (x+iy)^m,   S_{l,-m} = a_lm Q_l^m Im (x+iy)^m,
-//   Q_l^m = r^(l-m) d^m P_l(t)/dt^m at t = z/r, by the recurrence
-//   (l-m) Q_l^m = (2l-1) z Q_{l-1}^m - (l+m-1) r^2 Q_{l-2}^m,  Q_m^m = (2m-1)!!,
-//   dQ_l^m/dx = -x Q_{l-1}^{m+1},  dQ_l^m/dy = -y Q_{l-1}^{m+1},  dQ_l^m/dz = (l+m) Q_{l-1}^m.
-// Every lane runs the same unrolled, predicated recurrences for its own (l, m).
-template <int L, bool GRAD>
-__device__ __forceinline__ void solid_harmonic_item(float x, float y, float z, float r2, int l, int m,
-                                                    const float* __restrict__ anorm, const float* __restrict__ dfact,
-                                                    const float* __restrict__ inv_int,
-                                                    float4& plus, float4& minus) {
-    float cm = 1.f, sm = 0.f, cp = 0.f, sp = 0.f;          // (x+iy)^m and (x+iy)^(m-1)
-#pragma unroll
-    for (int t = 0; t < L; ++t)
-        if (t < m) {
-            cp = cm; sp = sm;
-            const float cn = x * cm - y * sm;
-            sm = x * sm + y * cm;
-            cm = cn;
-        }
-    float qa = __ldg(dfact + m), qb = 0.f;                  // Q_ll^m, Q_{ll-1}^m
-    float qc = 0.f, qd = 0.f;                               // Q_ll^{m+1}, Q_{ll-1}^{m+1} (up to ll = l-1)
-    if (GRAD && m + 1 <= l - 1) qc = __ldg(dfact + m + 1);
-#pragma unroll
-    for (int ll = 1; ll <= L; ++ll) {
-        if (ll > m && ll <= l) {
-            const float qn = ((2 * ll - 1) * z * qa - (ll + m - 1) * r2 * qb) * __ldg(inv_int + ll - m);
-            qb = qa; qa = qn;
-        }
-        if (GRAD && ll > m + 1 && ll <= l - 1) {
-            const float qn = ((2 * ll - 1) * z * qc - (ll + m) * r2 * qd) * __ldg(inv_int + ll - m - 1);
-            qd = qc; qc = qn;
-        }
-    }
-    const float a = __ldg(anorm + l * (l + 1) / 2 + m);
-    const float aq = a * qa;
-    if (!GRAD) {
-        plus.x = aq * cm;
-        minus.x = aq * sm;
-        return;
-    }
-    const float qz = (l > m) ? a * (l + m) * qb : 0.f;      // a dQ/dz
-    const float qx = a * qc;                                // a Q_{l-1}^{m+1} (0 when it does not exist)
-    const float mq = m * aq;
-    plus = make_float4(aq * cm, -x * qx * cm + mq * cp, -y * qx * cm - mq * sp, qz * cm);
-    minus = make_float4(aq * sm, -x * qx * sm + mq * sp, -y * qx * sm + mq * cp, qz * sm);
-}
 
 // Degree-5 table lookup: value and derivative with respect to the interval coordinate t.
 __device__ __forceinline__ void radial_lookup(const float* __restrict__ table, int qi, int n_ch, int ch, float t,
@@ -84,12 +39,60 @@ __device__ __forceinline__ void radial_lookup(const float* __restrict__ table, i
     dv = fmaf(dv, t, v); v = fmaf(v, t, a.x);
 }
 
-template <bool DERIV, int L>
+// Real solid harmonics of one pair per lane; this warp covers the columns
+// m = wid, wid + kWarps, ... of
+//   S_{l,+m} = a_lm Q_l^m Re (x+iy)^m,   S_{l,-m} = a_lm Q_l^m Im (x+iy)^m,
+//   Q_l^m = r^(l-m) d^m P_l(t)/dt^m at t = z/r,
+//   (l-m) Q_l^m = (2l-1) z Q_{l-1}^m - (l+m-1) r^2 Q_{l-2}^m,   Q_m^m = (2m-1)!!,
+//   dQ_l^m/dx = -x Q_{l-1}^{m+1},  dQ_l^m/dy = -y Q_{l-1}^{m+1},  dQ_l^m/dz = (l+m) Q_{l-1}^m.
+// Columns m and m+1 are advanced in lock step, so a step needs four registers.
+template <bool GRAD>
+__device__ __forceinline__ void harmonics_columns(int L, int wid, float4 d, const float* __restrict__ anorm,
+                                                  const float* __restrict__ dfact, const float* __restrict__ inv_int,
+                                                  float4* __restrict__ out4, float* __restrict__ out1) {
+    const float x = d.x, y = d.y, z = d.z, r2 = d.w * d.w;
+    for (int m = wid; m <= L; m += kWarps) {
+        float cm = 1.f, sm = 0.f, cp = 0.f, sp = 0.f;           // (x+iy)^m and (x+iy)^(m-1)
+        for (int t = 0; t < m; ++t) {
+            cp = cm; sp = sm;
+            const float cn = x * cm - y * sm;
+            sm = x * sm + y * cm;
+            cm = cn;
+        }
+        float a1 = __ldg(dfact + m), a0 = 0.f;                  // Q_l^m, Q_{l-1}^m
+        float b1 = 0.f, b0 = 0.f;                               // Q_l^{m+1}, Q_{l-1}^{m+1}
+        const float fm = (float)m;
+        for (int l = m; l <= L; ++l) {
+            const float a = __ldg(anorm + l * (l + 1) / 2 + m);
+            const float aq = a * a1;
+            const int lm0 = l * l + l;
+            if (!GRAD) {
+                out1[lm0 + m] = aq * cm;
+                if (m) out1[lm0 - m] = aq * sm;
+            } else {
+                const float qz = a * (float)(l + m) * a0;       // a dQ/dz (a0 = 0 when l = m)
+                const float qx = a * b0;                        // a Q_{l-1}^{m+1}
+                const float mq = fm * aq;
+                out4[lm0 + m] = make_float4(aq * cm, mq * cp - x * qx * cm, -mq * sp - y * qx * cm, qz * cm);
+                if (m) out4[lm0 - m] = make_float4(aq * sm, mq * sp - x * qx * sm, mq * cp - y * qx * sm, qz * sm);
+            }
+            // advance both columns to l + 1
+            const float zz = (float)(2 * l + 1) * z;
+            const float an = (zz * a1 - (float)(l + m) * r2 * a0) * __ldg(inv_int + l + 1 - m);
+            a0 = a1; a1 = an;
+            const float bn = (l == m) ? __ldg(dfact + m + 1) : (zz * b1 - (float)(l + m + 1) * r2 * b0) * __ldg(inv_int + l - m);
+            b0 = b1; b1 = bn;
+        }
+    }
+}
+
+template <bool DERIV, int L, int NMAX_T>
 __global__ void __launch_bounds__(kThreads, DERIV ? 3 : 4)
 center_kernel(const CenterParams p) {
-    constexpr int L1 = L + 1, LM = L1 * L1, NQ = L1 * (L1 + 1) / 2;
-    constexpr int KE = (16 * LM + kThreads - 1) / kThreads < kMaxElemPerThread ? (16 * LM + kThreads - 1) / kThreads
-                                                                                : kMaxElemPerThread;
+    constexpr int L1 = L + 1, LM = L1 * L1, LMP = LM | 1;      // odd row stride: no shared-memory bank conflicts
+    constexpr int NMAX_BOUND = NMAX_T ? NMAX_T : 16;
+    constexpr int KE_RAW = (NMAX_BOUND * LM + kThreads - 1) / kThreads;
+    constexpr int KE = KE_RAW < kMaxElemPerThread ? KE_RAW : kMaxElemPerThread;
     extern __shared__ __align__(16) float smem[];
     const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
     const long long c_idx = blockIdx.x;
@@ -99,14 +102,16 @@ center_kernel(const CenterParams p) {
         if (c_idx == 0 && tid == 0) atomicOr(&p.counters->status, kStatusRowCapacity);
         return;
     }
-    const int S = p.S, NMAX = p.n_max, NCH = NMAX * L1, NE = NMAX * LM, CT = S * NE, P = p.P, F = p.F;
+    const int S = p.S, NMAX = NMAX_T ? NMAX_T : p.n_max, NCH = NMAX * L1, NE = NMAX * LM;
+    const int CT = S * NMAX * LMP, P = p.P, F = p.F;
     const SmemLayout lay = make_layout(S, NMAX, L, P, DERIV);
-    float* c_t = smem + lay.c;
+    float* c_t = smem + lay.c;                                             // [S][NMAX][LMP]
     float4* geo_d = reinterpret_cast<float4*>(smem + lay.geo);             // [GP] dx, dy, dz, r
     int4* geo_i = reinterpret_cast<int4*>(smem + lay.geo + 4 * kGeoPairs);   // [GP] interval, t bits, species|moving<<8, row word
-    float* D_t = smem + lay.D;                                             // [3][CT]           (pass 1)
-    float* sS = smem + lay.sSD;                                            // [P][LM]           (pass 1, descriptor build)
-    float4* sSD4 = reinterpret_cast<float4*>(smem + lay.sSD);              // [P][LM]           (pass 1, derivative build)
+    int* geo_j = reinterpret_cast<int*>(smem + lay.geo + 8 * kGeoPairs);     // [GP] neighbour atom
+    float* D_t = smem + lay.D;                                             // [3][CT]           (pass 1 only)
+    float* sS = smem + lay.sSD;                                            // [P][LMP]          (descriptor build)
+    float4* sSD4 = reinterpret_cast<float4*>(smem + lay.sSD);              // [P][LMP]          (derivative build)
     float* sG1 = smem + lay.sG;
     float2* sG2 = reinterpret_cast<float2*>(smem + lay.sG);                // [P][NCH]
 
@@ -121,13 +126,14 @@ center_kernel(const CenterParams p) {
         if (e < CT) c_t[e] = 0.f; else D_t[e - CT] = 0.f;
     }
 
-    // elements (n, lm) this thread accumulates in pass 1
-    int el_lm[KE], el_ch[KE];
+    // elements (n, lm) this thread accumulates in pass 1: offsets into a c tile and into the staging rows
+    int el_c[KE], el_lm[KE], el_ch[KE];
 #pragma unroll
     for (int k = 0; k < KE; ++k) {
         const int e = tid + k * kThreads;
         const int n = e / LM, lm = e - n * LM;
         el_lm[k] = e < NE ? lm : -1;
+        el_c[k] = n * LMP + lm;
         el_ch[k] = n * L1 + __ldg(p.l_of_lm + lm);
     }
 
@@ -154,7 +160,25 @@ center_kernel(const CenterParams p) {
             const int qi = min((int)u, p.n_intervals - 1);
             geo_i[tid] = make_int4(qi, __float_as_int((float)(u - qi)),
                                    p.species_idx[j] | ((rw & kRowSelfImage) ? 0 : 256), rw);
+            geo_j[tid] = j;
         }
+    };
+
+    // ---- radial factors and solid harmonics of the pairs g .. g + pc - 1 of the staged geometry ----
+    auto stage_chunk = [&](int g, int pc) {
+        for (int pr = wid; pr < pc; pr += kWarps) {
+            const int4 gi = geo_i[g + pr];
+            const float t = __int_as_float(gi.y);
+            const float rinv_h = p.inv_h / geo_d[g + pr].w;
+            for (int ch = lane; ch < NCH; ch += 32) {
+                float v, dv;
+                radial_lookup(p.table, gi.x, NCH, ch, t, v, dv);
+                if (DERIV) sG2[pr * NCH + ch] = make_float2(v, dv * rinv_h);
+                else sG1[pr * NCH + ch] = v;
+            }
+        }
+        if (lane < pc)
+            harmonics_columns<DERIV>(L, wid, geo_d[g + lane], p.anorm, p.dfact, p.inv_int, sSD4 + lane * LMP, sS + lane * LMP);
     };
 
     // =========================== pass 1: c (and D) ===========================
@@ -165,35 +189,7 @@ center_kernel(const CenterParams p) {
         __syncthreads();
         for (int q0 = 0; q0 < gc; q0 += P) {
             const int pc = min(P, gc - q0);
-            // radial factors: warp <-> pair, lane <-> channel
-            for (int pr = wid; pr < pc; pr += kWarps) {
-                const int4 gi = geo_i[q0 + pr];
-                const float t = __int_as_float(gi.y);
-                const float rinv_h = p.inv_h / geo_d[q0 + pr].w;
-                for (int ch = lane; ch < NCH; ch += 32) {
-                    float v, dv;
-                    radial_lookup(p.table, gi.x, NCH, ch, t, v, dv);
-                    if (DERIV) sG2[pr * NCH + ch] = make_float2(v, dv * rinv_h);
-                    else sG1[pr * NCH + ch] = v;
-                }
-            }
-            // solid harmonics: thread <-> (pair, (l, m >= 0))
-            for (int idx = tid; idx < pc * NQ; idx += kThreads) {
-                const int pr = idx / NQ, t = idx - pr * NQ;
-                const int lmp = __ldg(p.lm_of_t + t);
-                const int l = lmp >> 4, m = lmp & 15;
-                const float4 d = geo_d[q0 + pr];
-                float4 plus, minus;
-                solid_harmonic_item<L, DERIV>(d.x, d.y, d.z, d.w * d.w, l, m, p.anorm, p.dfact, p.inv_int, plus, minus);
-                const int lm0 = l * l + l;
-                if (DERIV) {
-                    sSD4[pr * LM + lm0 + m] = plus;
-                    if (m) sSD4[pr * LM + lm0 - m] = minus;
-                } else {
-                    sS[pr * LM + lm0 + m] = plus.x;
-                    if (m) sS[pr * LM + lm0 - m] = minus.x;
-                }
-            }
+            stage_chunk(q0, pc);
             __syncthreads();
             for (int s = 0; s < S; ++s) {
                 float ac[KE], ax[KE], ay[KE], az[KE];
@@ -207,20 +203,21 @@ center_kernel(const CenterParams p) {
                     if (!DERIV) {
 #pragma unroll
                         for (int k = 0; k < KE; ++k)
-                            if (el_lm[k] >= 0) ac[k] = fmaf(sG1[pr * NCH + el_ch[k]], sS[pr * LM + el_lm[k]], ac[k]);
+                            if (el_lm[k] >= 0) ac[k] = fmaf(sG1[pr * NCH + el_ch[k]], sS[pr * LMP + el_lm[k]], ac[k]);
                     } else {
                         const float4 d = geo_d[q0 + pr];
                         const float mv = (info & 256) ? 1.f : 0.f;   // an image of the centre does not move relative to it
+                        const float dxm = d.x * mv, dym = d.y * mv, dzm = d.z * mv;
 #pragma unroll
                         for (int k = 0; k < KE; ++k)
                             if (el_lm[k] >= 0) {
                                 const float2 g = sG2[pr * NCH + el_ch[k]];
-                                const float4 h = sSD4[pr * LM + el_lm[k]];
+                                const float4 h = sSD4[pr * LMP + el_lm[k]];
                                 ac[k] = fmaf(g.x, h.x, ac[k]);
-                                const float gm = g.x * mv, t = g.y * h.x * mv;
-                                ax[k] = fmaf(gm, h.y, fmaf(t, d.x, ax[k]));
-                                ay[k] = fmaf(gm, h.z, fmaf(t, d.y, ay[k]));
-                                az[k] = fmaf(gm, h.w, fmaf(t, d.z, az[k]));
+                                const float gm = g.x * mv, t = g.y * h.x;
+                                ax[k] = fmaf(gm, h.y, fmaf(t, dxm, ax[k]));
+                                ay[k] = fmaf(gm, h.z, fmaf(t, dym, ay[k]));
+                                az[k] = fmaf(gm, h.w, fmaf(t, dzm, az[k]));
                             }
                     }
                 }
@@ -228,7 +225,7 @@ center_kernel(const CenterParams p) {
 #pragma unroll
                     for (int k = 0; k < KE; ++k)
                         if (el_lm[k] >= 0) {
-                            const int e = s * NE + tid + k * kThreads;
+                            const int e = s * NMAX * LMP + el_c[k];
                             c_t[e] += ac[k];
                             if (DERIV) { D_t[e] += ax[k]; D_t[CT + e] += ay[k]; D_t[2 * CT + e] += az[k]; }
                         }
@@ -239,7 +236,7 @@ center_kernel(const CenterParams p) {
     }
     __syncthreads();
     // on-site term: the centre's own Gaussian, l = 0 only (second term of Eq. 13)
-    if (tid < NMAX) c_t[(zi_species * NMAX + tid) * LM] += __ldg(p.self_term + tid);
+    if (tid < NMAX) c_t[(zi_species * NMAX + tid) * LMP] += __ldg(p.self_term + tid);
     __syncthreads();
 
     // ====================== power spectrum, Eq. 4 ======================
@@ -247,8 +244,8 @@ center_kernel(const CenterParams p) {
     for (int f = tid; f < F; f += kThreads) {
         const int pk = __ldg(p.feat_pack + f);
         const int n1 = pk & 31, n2 = (pk >> 5) & 31, mu = (pk >> 10) & 15, nu = (pk >> 14) & 15, l = (pk >> 18) & 15;
-        const float* a = c_t + (mu * NMAX + n1) * LM + l * l;
-        const float* b = c_t + (nu * NMAX + n2) * LM + l * l;
+        const float* a = c_t + (mu * NMAX + n1) * LMP + l * l;
+        const float* b = c_t + (nu * NMAX + n2) * LMP + l * l;
         float acc = 0.f;
         for (int m = 0; m <= 2 * l; ++m) acc = fmaf(a[m], b[m], acc);
         desc_row[f] = __ldg(p.kl + l) * acc;
@@ -263,7 +260,7 @@ center_kernel(const CenterParams p) {
         for (int f = tid; f < F; f += kThreads) {
             const int pk = __ldg(p.feat_pack + f);
             const int n1 = pk & 31, n2 = (pk >> 5) & 31, mu = (pk >> 10) & 15, nu = (pk >> 14) & 15, l = (pk >> 18) & 15;
-            const int ia = (mu * NMAX + n1) * LM + l * l, ib = (nu * NMAX + n2) * LM + l * l;
+            const int ia = (mu * NMAX + n1) * LMP + l * l, ib = (nu * NMAX + n2) * LMP + l * l;
             const float kl = -__ldg(p.kl + l);
             float ax = 0.f, ay = 0.f, az = 0.f;
             for (int m = 0; m <= 2 * l; ++m) {
@@ -277,144 +274,167 @@ center_kernel(const CenterParams p) {
         if (tid == 0) p.row_atom[row_base + my_row] = ci;
     }
     __syncthreads();
-    // fold K_l into c for pass 2 (D and the pass-1 staging are dead from here; their space
-    // becomes the per-warp staging of pass 2)
-    for (int e = tid; e < CT; e += kThreads) c_t[e] *= __ldg(p.kl + __ldg(p.l_of_lm + e % LM));
+    // fold K_l into c for pass 2 (D is dead from here; its space becomes the U/V staging)
+    for (int e = tid; e < S * NMAX * LM; e += kThreads) {
+        const int row = e / LM, lm = e - row * LM;
+        c_t[row * LMP + lm] *= __ldg(p.kl + __ldg(p.l_of_lm + lm));
+    }
 
     // =========================== pass 2: the Jacobian rows ===========================
-    const int NI = S * NCH;
-    float4* wSD = reinterpret_cast<float4*>(smem + lay.w2 + wid * lay.w2_stride);         // [LM]
-    float2* wG = reinterpret_cast<float2*>(smem + lay.w2 + wid * lay.w2_stride + 4 * LM);  // [NCH]
-    float4* wUV = reinterpret_cast<float4*>(smem + lay.w2 + wid * lay.w2_stride + 4 * LM + ((2 * NCH + 3) & ~3));   // [NI]
+    const int NI = S * NCH, SN = S * NMAX;
+    float4* wUV = reinterpret_cast<float4*>(smem + lay.wUV) + wid * NI;       // [nu][n'][l]
     for (int g0 = 0; g0 < k_pairs; g0 += kGeoPairs) {
         const int gc = min(kGeoPairs, k_pairs - g0);
         __syncthreads();
         if (g0 > 0 || k_pairs > kGeoPairs) stage_geometry(g0, gc);     // otherwise still valid from pass 1
         __syncthreads();
-        for (int pr = 0; pr < gc; ++pr) {
-            const int4 gi = geo_i[pr];
-            const int rw = gi.w;
-            if (rw & kRowSelfImage) continue;
-            const int row = rw & kRowMask;
-            if ((row & (kWarps - 1)) != wid) continue;
-            const bool accumulate = rw & kRowContinuation;
-            const int Z = gi.z & 255;
-            const float4 d = geo_d[pr];
-            __syncwarp();
-            // ---- radial factors and harmonics of this pair ----
-            {
-                const float t = __int_as_float(gi.y);
-                const float rinv_h = p.inv_h / d.w;
-                for (int ch = lane; ch < NCH; ch += 32) {
-                    float v, dv;
-                    radial_lookup(p.table, gi.x, NCH, ch, t, v, dv);
-                    wG[ch] = make_float2(v, dv * rinv_h);
-                }
-                for (int t2 = lane; t2 < NQ; t2 += 32) {
-                    const int lmp = __ldg(p.lm_of_t + t2);
-                    const int l = lmp >> 4, m = lmp & 15;
-                    float4 plus, minus;
-                    solid_harmonic_item<L, true>(d.x, d.y, d.z, d.w * d.w, l, m, p.anorm, p.dfact, p.inv_int, plus, minus);
-                    const int lm0 = l * l + l;
-                    wSD[lm0 + m] = plus;
-                    if (m) wSD[lm0 - m] = minus;
-                }
-            }
-            __syncwarp();
-            // ---- U, V for every (nu, n', l); items ordered l-major so that a warp's trip counts agree ----
-            {
-                const int SN = S * NMAX;
-                for (int it = lane; it < NI; it += 32) {
-                    const int l = it / SN, sn = it - l * SN;            // sn = nu * NMAX + n'
-                    const float* cp = c_t + sn * LM + l * l;
-                    const float4* hp = wSD + l * l;
-                    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-                    for (int m = 0; m <= 2 * l; ++m) {
-                        const float cv = cp[m];
-                        const float4 h = hp[m];
-                        acc.x = fmaf(cv, h.x, acc.x); acc.y = fmaf(cv, h.y, acc.y);
-                        acc.z = fmaf(cv, h.z, acc.z); acc.w = fmaf(cv, h.w, acc.w);
-                    }
-                    wUV[sn * L1 + l] = acc;                           // [nu][n'][l]
-                }
-            }
-            __syncwarp();
-            // ---- product rule and store ----
-            float* out = p.out_jac + (size_t)(row_base + row) * 3 * F;
-            if (!accumulate && lane == 0) p.row_atom[row_base + row] = key_atom(p.pair_key[pair_base + g0 + pr]);
-            int boff = 0;
-            for (int mu = 0; mu < S; ++mu) {
-                for (int nu = mu; nu < S; ++nu) {
-                    const int bsize = (mu == nu) ? (NMAX * (NMAX + 1) / 2) * L1 : NMAX * NCH;
-                    float* ob = out + boff;
-                    if (mu != Z && nu != Z) {
-                        if (!accumulate)
-                            for (int f = lane; f < bsize; f += 32) { ob[f] = 0.f; ob[F + f] = 0.f; ob[2 * F + f] = 0.f; }
-                    } else if (mu == nu) {
-                        // both terms; feature (n1 <= n2, l) sits at L1 (n1 NMAX - n1(n1-1)/2) + (n2-n1) L1 + l
-                        const float4* UVz = wUV + Z * NCH;
-                        for (int j = lane; j < NCH; j += 32) {
-                            const int n2 = j / L1, l = j - n2 * L1;
-                            const float2 gj = wG[j];
-                            const float4 uj = UVz[j];
-                            const float2* g1p = wG + l;
-                            const float4* u1p = UVz + l;
-                            float* o = ob + j;
-                            for (int n1 = 0; n1 <= n2; ++n1) {
-                                const float2 g1 = *g1p;
-                                const float4 u1 = *u1p;
-                                const float w = fmaf(g1.y, uj.x, gj.y * u1.x);    // Ghat_n1 U_n2 + Ghat_n2 U_n1
-                                const float vx = fmaf(g1.x, uj.y, fmaf(gj.x, u1.y, w * d.x));
-                                const float vy = fmaf(g1.x, uj.z, fmaf(gj.x, u1.z, w * d.y));
-                                const float vz = fmaf(g1.x, uj.w, fmaf(gj.x, u1.w, w * d.z));
-                                if (accumulate) { o[0] += vx; o[F] += vy; o[2 * F] += vz; }
-                                else { o[0] = vx; o[F] = vy; o[2 * F] = vz; }
-                                g1p += L1; u1p += L1;
-                                o += (NMAX - n1 - 1) * L1;
+        for (int q0 = 0; q0 < gc; q0 += P) {
+            const int pc = min(P, gc - q0);
+            stage_chunk(q0, pc);
+            __syncthreads();
+            for (int pr = 0; pr < pc; ++pr) {
+                const int4 gi = geo_i[q0 + pr];
+                const int rw = gi.w;
+                if (rw & kRowSelfImage) continue;
+                const int row = rw & kRowMask;
+                if ((row & (kWarps - 1)) != wid) continue;
+                const bool accumulate = rw & kRowContinuation;
+                const int Z = gi.z & 255;
+                const float4 d = geo_d[q0 + pr];
+                const float2* wG = sG2 + pr * NCH;
+                const float4* wSD = sSD4 + pr * LMP;
+                __syncwarp();
+                // ---- U, V for every (nu, n', l) ----
+                if (SN <= 16) {
+                    // lane <-> (nu n', half): half 0 accumulates (U, Vx), half 1 (Vy, Vz)
+                    const int sn = lane >> 1, half = lane & 1;
+                    if (sn < SN) {
+                        const float* cp = c_t + sn * LMP;
+                        const float2* hp = reinterpret_cast<const float2*>(wSD) + half;
+                        float2* up = reinterpret_cast<float2*>(wUV + sn * L1) + half;
+#pragma unroll
+                        for (int l = 0; l <= L; ++l) {
+                            float2 acc = make_float2(0.f, 0.f);
+#pragma unroll
+                            for (int m = 0; m <= 2 * l; ++m) {
+                                const float cv = cp[l * l + m];
+                                const float2 h = hp[2 * (l * l + m)];
+                                acc.x = fmaf(cv, h.x, acc.x); acc.y = fmaf(cv, h.y, acc.y);
                             }
-                        }
-                    } else if (mu == Z) {
-                        // (grad c^mu_{n1 l}) c^nu_{n2 l}: G_{n1 l} V^nu_{n2 l} + Ghat_{n1 l} d U^nu_{n2 l}
-                        for (int j = lane; j < NCH; j += 32) {
-                            const int l = j % L1;
-                            const float4 uj = wUV[nu * NCH + j];
-                            const float xx = uj.x * d.x, xy = uj.x * d.y, xz = uj.x * d.z;
-                            const float2* g1p = wG + l;
-                            float* o = ob + j;
-#pragma unroll 4
-                            for (int n1 = 0; n1 < NMAX; ++n1) {
-                                const float2 g1 = *g1p;
-                                const float vx = fmaf(g1.x, uj.y, g1.y * xx);
-                                const float vy = fmaf(g1.x, uj.z, g1.y * xy);
-                                const float vz = fmaf(g1.x, uj.w, g1.y * xz);
-                                if (accumulate) { o[0] += vx; o[F] += vy; o[2 * F] += vz; }
-                                else { o[0] = vx; o[F] = vy; o[2 * F] = vz; }
-                                g1p += L1; o += NCH;
-                            }
-                        }
-                    } else {
-                        // c^mu_{n1 l} (grad c^nu_{n2 l}): G_{n2 l} V^mu_{n1 l} + Ghat_{n2 l} d U^mu_{n1 l}
-                        for (int j = lane; j < NCH; j += 32) {
-                            const int l = j % L1;
-                            const float2 gj = wG[j];
-                            const float gx = gj.y * d.x, gy = gj.y * d.y, gz = gj.y * d.z;
-                            const float4* u1p = wUV + mu * NCH + l;
-                            float* o = ob + j;
-#pragma unroll 4
-                            for (int n1 = 0; n1 < NMAX; ++n1) {
-                                const float4 u1 = *u1p;
-                                const float vx = fmaf(gj.x, u1.y, gx * u1.x);
-                                const float vy = fmaf(gj.x, u1.z, gy * u1.x);
-                                const float vz = fmaf(gj.x, u1.w, gz * u1.x);
-                                if (accumulate) { o[0] += vx; o[F] += vy; o[2 * F] += vz; }
-                                else { o[0] = vx; o[F] = vy; o[2 * F] = vz; }
-                                u1p += L1; o += NCH;
-                            }
+                            up[2 * l] = acc;
                         }
                     }
-                    boff += bsize;
+                } else {
+                    for (int sn = lane; sn < SN; sn += 32) {
+                        const float* cp = c_t + sn * LMP;
+#pragma unroll
+                        for (int l = 0; l <= L; ++l) {
+                            float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+                            for (int m = 0; m <= 2 * l; ++m) {
+                                const float cv = cp[l * l + m];
+                                const float4 h = wSD[l * l + m];
+                                acc.x = fmaf(cv, h.x, acc.x); acc.y = fmaf(cv, h.y, acc.y);
+                                acc.z = fmaf(cv, h.z, acc.z); acc.w = fmaf(cv, h.w, acc.w);
+                            }
+                            wUV[sn * L1 + l] = acc;
+                        }
+                    }
+                }
+                __syncwarp();
+                // ---- product rule and store ----
+                float* out = p.out_jac + (size_t)(row_base + row) * 3 * F;
+                if (!accumulate && lane == 0) p.row_atom[row_base + row] = geo_j[q0 + pr];
+                int boff = 0;
+                for (int mu = 0; mu < S; ++mu) {
+                    for (int nu = mu; nu < S; ++nu) {
+                        const int bsize = (mu == nu) ? (NMAX * (NMAX + 1) / 2) * L1 : NMAX * NCH;
+                        float* ob = out + boff;
+                        boff += bsize;
+                        if (mu != Z && nu != Z) {
+                            if (!accumulate) {
+                                float *o0 = ob + lane, *o1 = o0 + F, *o2 = o1 + F;
+                                int f = lane;
+                                for (; f + 96 < bsize; f += 128) {
+#pragma unroll
+                                    for (int u = 0; u < 4; ++u) { o0[32 * u] = 0.f; o1[32 * u] = 0.f; o2[32 * u] = 0.f; }
+                                    o0 += 128; o1 += 128; o2 += 128;
+                                }
+                                for (; f < bsize; f += 32) { *o0 = 0.f; *o1 = 0.f; *o2 = 0.f; o0 += 32; o1 += 32; o2 += 32; }
+                            }
+                        } else if (mu == nu) {
+                            // both terms; feature (n1 <= n2, l) sits at L1 (n1 NMAX - n1(n1-1)/2) + (n2-n1) L1 + l
+                            const float4* UVz = wUV + Z * NCH;
+                            for (int j0 = 0; j0 < NCH; j0 += 32) {
+                                const int j = j0 + lane;
+                                const bool live = j < NCH;
+                                const int jj = live ? j : 0;
+                                const int n2 = jj / L1, l = jj - n2 * L1;
+                                const float2 gj = wG[jj];
+                                const float4 uj = UVz[jj];
+                                const float2* g1p = wG + l;
+                                const float4* u1p = UVz + l;
+                                float *o0 = ob + jj, *o1 = o0 + F, *o2 = o1 + F;
+                                const int n1_hi = min(NMAX - 1, (j0 + 31) / L1);     // no lane of this round goes beyond
+#pragma unroll
+                                for (int n1 = 0; n1 < NMAX_BOUND; ++n1) {
+                                    if (n1 > n1_hi) break;
+                                    const int off = (n1 * NMAX - n1 * (n1 + 1) / 2) * L1;   // feature offset relative to n1 = 0
+                                    if (live && n1 <= n2) {
+                                        const float2 g1 = g1p[n1 * L1];
+                                        const float4 u1 = u1p[n1 * L1];
+                                        const float w = fmaf(g1.y, uj.x, gj.y * u1.x);    // Ghat_n1 U_n2 + Ghat_n2 U_n1
+                                        const float vx = fmaf(g1.x, uj.y, fmaf(gj.x, u1.y, w * d.x));
+                                        const float vy = fmaf(g1.x, uj.z, fmaf(gj.x, u1.z, w * d.y));
+                                        const float vz = fmaf(g1.x, uj.w, fmaf(gj.x, u1.w, w * d.z));
+                                        if (accumulate) { o0[off] += vx; o1[off] += vy; o2[off] += vz; }
+                                        else { o0[off] = vx; o1[off] = vy; o2[off] = vz; }
+                                    }
+                                }
+                            }
+                        } else if (mu == Z) {
+                            // (grad c^mu_{n1 l}) c^nu_{n2 l}: G_{n1 l} V^nu_{n2 l} + Ghat_{n1 l} d U^nu_{n2 l}
+                            for (int j = lane; j < NCH; j += 32) {
+                                const int l = j % L1;
+                                const float4 uj = wUV[nu * NCH + j];
+                                const float xx = uj.x * d.x, xy = uj.x * d.y, xz = uj.x * d.z;
+                                const float2* g1p = wG + l;
+                                float *o0 = ob + j, *o1 = o0 + F, *o2 = o1 + F;
+#pragma unroll
+                                for (int n1 = 0; n1 < NMAX_BOUND; ++n1) {
+                                    if (n1 >= NMAX) break;
+                                    const float2 g1 = g1p[n1 * L1];
+                                    const float vx = fmaf(g1.x, uj.y, g1.y * xx);
+                                    const float vy = fmaf(g1.x, uj.z, g1.y * xy);
+                                    const float vz = fmaf(g1.x, uj.w, g1.y * xz);
+                                    if (accumulate) { o0[n1 * NCH] += vx; o1[n1 * NCH] += vy; o2[n1 * NCH] += vz; }
+                                    else { o0[n1 * NCH] = vx; o1[n1 * NCH] = vy; o2[n1 * NCH] = vz; }
+                                }
+                            }
+                        } else {
+                            // c^mu_{n1 l} (grad c^nu_{n2 l}): G_{n2 l} V^mu_{n1 l} + Ghat_{n2 l} d U^mu_{n1 l}
+                            for (int j = lane; j < NCH; j += 32) {
+                                const int l = j % L1;
+                                const float2 gj = wG[j];
+                                const float gx = gj.y * d.x, gy = gj.y * d.y, gz = gj.y * d.z;
+                                const float4* u1p = wUV + mu * NCH + l;
+                                float *o0 = ob + j, *o1 = o0 + F, *o2 = o1 + F;
+#pragma unroll
+                                for (int n1 = 0; n1 < NMAX_BOUND; ++n1) {
+                                    if (n1 >= NMAX) break;
+                                    const float4 u1 = u1p[n1 * L1];
+                                    const float vx = fmaf(gj.x, u1.y, gx * u1.x);
+                                    const float vy = fmaf(gj.x, u1.z, gy * u1.x);
+                                    const float vz = fmaf(gj.x, u1.w, gz * u1.x);
+                                    if (accumulate) { o0[n1 * NCH] += vx; o1[n1 * NCH] += vy; o2[n1 * NCH] += vz; }
+                                    else { o0[n1 * NCH] = vx; o1[n1 * NCH] = vy; o2[n1 * NCH] = vz; }
+                                }
+                            }
+                        }
+                    }
                 }
             }
+            __syncthreads();
         }
     }
 }

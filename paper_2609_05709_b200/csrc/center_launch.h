@@ -1,13 +1,21 @@
-// Dispatch of the per-centre kernel over its compile-time l_max (0..12).
+// Dispatch of the per-centre kernel over its compile-time l_max (0..12) and n_max.
 #pragma once
 #include "soap_device.cuh"
 
 namespace soap {
-cudaError_t center_set_smem(bool deriv, int l_max, int bytes);
-cudaError_t center_launch(bool deriv, int l_max, const CenterParams& p, unsigned grid, size_t smem, cudaStream_t st);
-// one group of l_max values per translation unit, so that they compile in parallel
-cudaError_t center_set_smem_g0(bool, int, int);  cudaError_t center_launch_g0(bool, int, const CenterParams&, unsigned, size_t, cudaStream_t);
-cudaError_t center_set_smem_g1(bool, int, int);  cudaError_t center_launch_g1(bool, int, const CenterParams&, unsigned, size_t, cudaStream_t);
-cudaError_t center_set_smem_g2(bool, int, int);  cudaError_t center_launch_g2(bool, int, const CenterParams&, unsigned, size_t, cudaStream_t);
-cudaError_t center_set_smem_g3(bool, int, int);  cudaError_t center_launch_g3(bool, int, const CenterParams&, unsigned, size_t, cudaStream_t);
+// n_max values with their own instantiation of the derivative kernel; others run the
+// variant that reads n_max at run time.
+inline bool center_has_fixed_nmax(bool deriv, int n_max) {
+    if (deriv) return n_max >= 2 && n_max <= 12 && n_max % 2 == 0;
+    return n_max == 8;
+}
+cudaError_t center_set_smem(bool deriv, int l_max, int n_max, int bytes);
+cudaError_t center_launch(bool deriv, int l_max, int n_max, const CenterParams& p, unsigned grid, size_t smem, cudaStream_t st);
+
+#define SOAP_DECLARE_L(LV)                                                                                       \
+    cudaError_t center_set_smem_l##LV(bool deriv, int n_max, int bytes);                                        \
+    cudaError_t center_launch_l##LV(bool deriv, int n_max, const CenterParams& p, unsigned grid, size_t smem, cudaStream_t st);
+SOAP_DECLARE_L(0) SOAP_DECLARE_L(1) SOAP_DECLARE_L(2) SOAP_DECLARE_L(3) SOAP_DECLARE_L(4) SOAP_DECLARE_L(5) SOAP_DECLARE_L(6)
+SOAP_DECLARE_L(7) SOAP_DECLARE_L(8) SOAP_DECLARE_L(9) SOAP_DECLARE_L(10) SOAP_DECLARE_L(11) SOAP_DECLARE_L(12)
+#undef SOAP_DECLARE_L
 }  // namespace soap

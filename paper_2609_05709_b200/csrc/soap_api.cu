@@ -17,22 +17,21 @@
 using namespace soap;
 
 namespace soap {
-static int group_of(int l_max) { return l_max <= 5 ? 0 : l_max <= 8 ? 1 : l_max <= 10 ? 2 : 3; }
-cudaError_t center_set_smem(bool deriv, int l_max, int bytes) {
-    switch (group_of(l_max)) {
-        case 0: return center_set_smem_g0(deriv, l_max, bytes);
-        case 1: return center_set_smem_g1(deriv, l_max, bytes);
-        case 2: return center_set_smem_g2(deriv, l_max, bytes);
-        default: return center_set_smem_g3(deriv, l_max, bytes);
+cudaError_t center_set_smem(bool deriv, int l_max, int n_max, int bytes) {
+    switch (l_max) {
+#define X(LV) case LV: return center_set_smem_l##LV(deriv, n_max, bytes);
+        X(0) X(1) X(2) X(3) X(4) X(5) X(6) X(7) X(8) X(9) X(10) X(11) X(12)
+#undef X
     }
+    return cudaErrorInvalidValue;
 }
-cudaError_t center_launch(bool deriv, int l_max, const CenterParams& p, unsigned grid, size_t smem, cudaStream_t st) {
-    switch (group_of(l_max)) {
-        case 0: return center_launch_g0(deriv, l_max, p, grid, smem, st);
-        case 1: return center_launch_g1(deriv, l_max, p, grid, smem, st);
-        case 2: return center_launch_g2(deriv, l_max, p, grid, smem, st);
-        default: return center_launch_g3(deriv, l_max, p, grid, smem, st);
+cudaError_t center_launch(bool deriv, int l_max, int n_max, const CenterParams& p, unsigned grid, size_t smem, cudaStream_t st) {
+    switch (l_max) {
+#define X(LV) case LV: return center_launch_l##LV(deriv, n_max, p, grid, smem, st);
+        X(0) X(1) X(2) X(3) X(4) X(5) X(6) X(7) X(8) X(9) X(10) X(11) X(12)
+#undef X
     }
+    return cudaErrorInvalidValue;
 }
 }  // namespace soap
 
@@ -171,18 +170,25 @@ int ensure_device(soap_t* h) {
     int max_smem = 0;
     CU(cudaDeviceGetAttribute(&max_smem, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev));
     for (int deriv = 0; deriv < 2; ++deriv) {
-        int P = 16;
+        // largest chunk that still leaves room for three CTAs per SM, else two, else whatever fits
+        int P = 32;
         size_t bytes = 0;
-        for (; P >= 2; P /= 2) {
-            bytes = (size_t)make_layout(h->S, h->n_max, h->l_max, P, deriv).total * 4;
-            // aim for at least two CTAs per SM
-            if (bytes <= (size_t)max_smem / 2 - 1024 || P == 2) break;
+        const size_t budget3 = (size_t)228 * 1024 / 3 - 1024, budget2 = (size_t)228 * 1024 / 2 - 1024;
+        for (int pass = 0; pass < 3; ++pass) {
+            const size_t budget = pass == 0 ? budget3 : pass == 1 ? budget2 : (size_t)max_smem;
+            for (P = 32; P >= 4; P /= 2) {
+                bytes = (size_t)make_layout(h->S, h->n_max, h->l_max, P, deriv).total * 4;
+                if (bytes <= budget) break;
+            }
+            if (P >= (pass == 2 ? 4 : 8) && bytes <= budget) break;
+            if (P < 4) P = 4;
         }
+        bytes = (size_t)make_layout(h->S, h->n_max, h->l_max, P, deriv).total * 4;
         if (bytes > (size_t)max_smem) return fail(h, SOAP_ERR_INVALID_ARG, "this basis does not fit the shared memory of the device");
         if (deriv) { h->P_deriv = P; h->smem_deriv = bytes; } else { h->P_desc = P; h->smem_desc = bytes; }
     }
-    CU(center_set_smem(false, h->l_max, (int)h->smem_desc));
-    CU(center_set_smem(true, h->l_max, (int)h->smem_deriv));
+    CU(center_set_smem(false, h->l_max, h->n_max, (int)h->smem_desc));
+    CU(center_set_smem(true, h->l_max, h->n_max, (int)h->smem_deriv));
     h->tables_ready = true;
     return SOAP_OK;
 }
@@ -422,7 +428,7 @@ int soap_descriptor(soap_t* h, const float* d_positions, const int32_t* d_number
         CenterParams cp;
         fill_center_params(h, cp, d_positions, d_centers, n_centers, g, false);
         cp.out_desc = d_out;
-        CU(center_launch(false, h->l_max, cp, (unsigned)n_centers, h->smem_desc, st));
+        CU(center_launch(false, h->l_max, h->n_max, cp, (unsigned)n_centers, h->smem_desc, st));
     }
     if (h->profiling) CU(cudaEventRecord(h->ev[2], st));
     return SOAP_OK;
@@ -454,7 +460,7 @@ int soap_derivatives(soap_t* h, const float* d_positions, const int32_t* d_numbe
         cp.row_ptr = (const long long*)d_row_ptr;
         cp.row_capacity = capacity_rows;
         cp.out_desc = d_out_desc; cp.out_jac = d_out_jac; cp.row_atom = d_row_atom;
-        CU(center_launch(true, h->l_max, cp, (unsigned)n_centers, h->smem_deriv, st));
+        CU(center_launch(true, h->l_max, h->n_max, cp, (unsigned)n_centers, h->smem_deriv, st));
     }
     if (h->profiling) CU(cudaEventRecord(h->ev[2], st));
     return SOAP_OK;

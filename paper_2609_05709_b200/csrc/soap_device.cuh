@@ -75,7 +75,7 @@ struct CenterParams {
     float inv_h;
     int n_intervals;
     int S, n_max, l_max, F;
-    int P;                        // pairs per pass-1 chunk
+    int P;                        // pairs per staged chunk (<= 32)
     // outputs
     float* out_desc;              // [C,F]
     float* out_jac;               // [rows,3,F]
@@ -90,31 +90,30 @@ __host__ __device__ inline void key_shift(unsigned long long k, int s[3]) {
 }
 
 // Shared-memory carve-up of the per-centre kernel, in 4-byte words.  Every region
-// starts on a 16-byte boundary.  The pass-1 regions (D tiles, chunk staging) and
-// the per-warp staging of pass 2 never live at the same time and share space.
+// starts on a 16-byte boundary.  Rows of the coefficient tiles and of the harmonics
+// staging have the odd stride (l_max+1)^2 | 1, which keeps strided accesses off a
+// single bank.  The D tiles (pass 1) and the per-warp U/V staging (pass 2) never
+// live at the same time and share space.
 constexpr int kGeoPairs = 128;           // pairs whose geometry is staged at once
 
 struct SmemLayout {
-    int c, geo, D, sSD, sG, w2, w2_stride, total;
+    int c, geo, D, wUV, sSD, sG, total;
 };
 __host__ __device__ inline int align4(int x) { return (x + 3) & ~3; }
 __host__ __device__ inline SmemLayout make_layout(int S, int n_max, int l_max, int P, bool deriv) {
-    const int L1 = l_max + 1, LM = L1 * L1, NCH = n_max * L1, CT = S * n_max * LM;
+    const int L1 = l_max + 1, LMP = (L1 * L1) | 1, NCH = n_max * L1, CT = S * n_max * LMP;
     SmemLayout o;
     int off = 0;
     o.c = off; off = align4(off + CT);
-    o.geo = off; off += kGeoPairs * 8;
-    const int u = off;
-    // pass 1
-    o.D = off; if (deriv) off = align4(off + 3 * CT);
-    o.sSD = off; off = align4(off + (deriv ? P * LM * 4 : P * LM));
+    o.geo = off; off = align4(off + kGeoPairs * 9);
+    o.D = off; o.wUV = off;
+    if (deriv) {
+        const int a = 3 * CT, b = kWarps * S * NCH * 4;
+        off = align4(off + (a > b ? a : b));
+    }
+    o.sSD = off; off = align4(off + (deriv ? P * LMP * 4 : P * LMP));
     o.sG = off; off = align4(off + (deriv ? P * NCH * 2 : P * NCH));
-    const int end1 = off;
-    // pass 2: per warp [LM] float4 harmonics, [NCH] float2 radial, [S*NCH] float4 U/V
-    o.w2 = u;
-    o.w2_stride = 4 * LM + align4(2 * NCH) + 4 * S * NCH;
-    const int end2 = deriv ? u + kWarps * o.w2_stride : u;
-    o.total = end1 > end2 ? end1 : end2;
+    o.total = off;
     return o;
 }
 
