@@ -26,7 +26,8 @@ class SoapError(RuntimeError):
 
 
 def library_path() -> str:
-    return os.path.join(os.path.dirname(os.path.abspath(__file__)), "libsoap_b200.so")
+    """The in-tree build, unless SOAP_B200_LIB names another build of the same library."""
+    return os.environ.get("SOAP_B200_LIB") or os.path.join(os.path.dirname(os.path.abspath(__file__)), "libsoap_b200.so")
 
 
 _LIB = None

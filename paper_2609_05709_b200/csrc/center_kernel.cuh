@@ -13,8 +13,8 @@
 //   pair and lanes on channels; solid harmonics with lanes on pairs and warps on
 //   the columns m of the recursion, so that control flow is uniform.
 //   Pass 1 accumulates c and D = sum_j grad_j c with thread-owned elements; the
-//   centre's own Jacobian row is minus the sum over its neighbours, which is a
-//   contraction of D with c.
+//   centre's own Jacobian row is minus the sum over its neighbours (translation
+//   invariance, text below Eq. 5), which is a contraction of D with c.
 //   Pass 2 gives every pair to one warp: it forms U^nu_{n'l} = K_l sum_m S_lm
 //   c^nu_{n'lm} and V likewise with grad S, after which every output element of
 //   Eq. 5 is two fused multiply-adds per term, and streams the row out with lanes
@@ -22,7 +22,13 @@
 // l_max and n_max are template parameters (n_max = 0 means "read it at run
 // time") so that loops unroll and the store addresses become immediates.
 #pragma once
+#include <type_traits>
+
 #include "soap_device.cuh"
+
+#ifndef SOAP_DEBUG_SKIP
+#define SOAP_DEBUG_SKIP 0
+#endif
 
 namespace soap {
 
@@ -109,11 +115,11 @@ center_kernel(const CenterParams p) {
     float4* geo_d = reinterpret_cast<float4*>(smem + lay.geo);             // [GP] dx, dy, dz, r
     int4* geo_i = reinterpret_cast<int4*>(smem + lay.geo + 4 * kGeoPairs);   // [GP] interval, t bits, species|moving<<8, row word
     int* geo_j = reinterpret_cast<int*>(smem + lay.geo + 8 * kGeoPairs);     // [GP] neighbour atom
-    float* D_t = smem + lay.D;                                             // [3][CT]           (pass 1 only)
-    float* sS = smem + lay.sSD;                                            // [P][LMP]          (descriptor build)
-    float4* sSD4 = reinterpret_cast<float4*>(smem + lay.sSD);              // [P][LMP]          (derivative build)
-    float* sG1 = smem + lay.sG;
-    float2* sG2 = reinterpret_cast<float2*>(smem + lay.sG);                // [P][NCH]
+    float* D_t = smem + lay.D;                                             // [3][CT]    (pass 1 and the centre's row)
+    float* sS = smem + lay.sSD;                                            // [P][LMP]   values            (descriptor build)
+    float4* sSD4 = reinterpret_cast<float4*>(smem + lay.sSD);              // [P][LMP]   (S, dSx, dSy, dSz) (derivative build)
+    float* sG1 = smem + lay.sG;                                            // [P][NCH]   G
+    float2* sG2 = reinterpret_cast<float2*>(smem + lay.sG);                // [P][NCH]   (G, Ghat)
 
     const int ci = p.centers ? p.centers[c_idx] : (int)c_idx;
     const float xi = p.pos[3 * (long long)ci], yi = p.pos[3 * (long long)ci + 1], zi = p.pos[3 * (long long)ci + 2];
@@ -137,8 +143,10 @@ center_kernel(const CenterParams p) {
         el_ch[k] = n * L1 + __ldg(p.l_of_lm + lm);
     }
 
-    // ---- geometry of up to kGeoPairs pairs, one thread each ----
-    auto stage_geometry = [&](int g0, int gc) {
+    // ---- geometry of up to kGeoPairs pairs, one thread each; returns whether any pair of the
+    //      batch shares its row with another or is an image of the centre ----
+    auto stage_geometry = [&](int g0, int gc) -> bool {
+        int special = 0;
         if (tid < gc) {
             const unsigned long long key = p.pair_key[pair_base + g0 + tid];
             const int j = key_atom(key);
@@ -155,6 +163,7 @@ center_kernel(const CenterParams p) {
             const double r = sqrt(dx * dx + dy * dy + dz * dz);
             geo_d[tid] = make_float4((float)dx, (float)dy, (float)dz, (float)r);
             const int rw = p.pair_row[pair_base + g0 + tid];
+            special = rw & (kRowSelfImage | kRowContinuation);
             // interval and offset in the radial table, in fp64 so that the offset keeps its digits
             const double u = r * (double)p.inv_h;
             const int qi = min((int)u, p.n_intervals - 1);
@@ -162,36 +171,39 @@ center_kernel(const CenterParams p) {
                                    p.species_idx[j] | ((rw & kRowSelfImage) ? 0 : 256), rw);
             geo_j[tid] = j;
         }
+        return __syncthreads_or(special) != 0;
     };
 
     // ---- radial factors and solid harmonics of the pairs g .. g + pc - 1 of the staged geometry ----
-    auto stage_chunk = [&](int g, int pc) {
+    auto stage_chunk = [&](int g, int pc, auto grad_tag) {
+        constexpr bool GRAD = decltype(grad_tag)::value;
+        if (SOAP_DEBUG_SKIP & 16) return;
         for (int pr = wid; pr < pc; pr += kWarps) {
             const int4 gi = geo_i[g + pr];
             const float t = __int_as_float(gi.y);
-            const float rinv_h = p.inv_h / geo_d[g + pr].w;
+            const float rinv_h = GRAD ? p.inv_h / geo_d[g + pr].w : 0.f;
             for (int ch = lane; ch < NCH; ch += 32) {
                 float v, dv;
                 radial_lookup(p.table, gi.x, NCH, ch, t, v, dv);
-                if (DERIV) sG2[pr * NCH + ch] = make_float2(v, dv * rinv_h);
+                if (GRAD) sG2[pr * NCH + ch] = make_float2(v, dv * rinv_h);
                 else sG1[pr * NCH + ch] = v;
             }
         }
         if (lane < pc)
-            harmonics_columns<DERIV>(L, wid, geo_d[g + lane], p.anorm, p.dfact, p.inv_int, sSD4 + lane * LMP, sS + lane * LMP);
+            harmonics_columns<GRAD>(L, wid, geo_d[g + lane], p.anorm, p.dfact, p.inv_int, sSD4 + lane * LMP, sS + lane * LMP);
     };
 
     // =========================== pass 1: c (and D) ===========================
+    bool special = false;
     for (int g0 = 0; g0 < k_pairs; g0 += kGeoPairs) {
         const int gc = min(kGeoPairs, k_pairs - g0);
         __syncthreads();
-        stage_geometry(g0, gc);
-        __syncthreads();
+        special = stage_geometry(g0, gc);
         for (int q0 = 0; q0 < gc; q0 += P) {
             const int pc = min(P, gc - q0);
-            stage_chunk(q0, pc);
+            stage_chunk(q0, pc, std::integral_constant<bool, DERIV>{});
             __syncthreads();
-            for (int s = 0; s < S; ++s) {
+            for (int s = 0; s < ((SOAP_DEBUG_SKIP & 4) ? 0 : S); ++s) {
                 float ac[KE], ax[KE], ay[KE], az[KE];
 #pragma unroll
                 for (int k = 0; k < KE; ++k) ac[k] = ax[k] = ay[k] = az[k] = 0.f;
@@ -239,42 +251,38 @@ center_kernel(const CenterParams p) {
     if (tid < NMAX) c_t[(zi_species * NMAX + tid) * LMP] += __ldg(p.self_term + tid);
     __syncthreads();
 
-    // ====================== power spectrum, Eq. 4 ======================
-    float* desc_row = p.out_desc + (size_t)c_idx * F;
-    for (int f = tid; f < F; f += kThreads) {
-        const int pk = __ldg(p.feat_pack + f);
-        const int n1 = pk & 31, n2 = (pk >> 5) & 31, mu = (pk >> 10) & 15, nu = (pk >> 14) & 15, l = (pk >> 18) & 15;
-        const float* a = c_t + (mu * NMAX + n1) * LMP + l * l;
-        const float* b = c_t + (nu * NMAX + n2) * LMP + l * l;
-        float acc = 0.f;
-        for (int m = 0; m <= 2 * l; ++m) acc = fmaf(a[m], b[m], acc);
-        desc_row[f] = __ldg(p.kl + l) * acc;
-    }
-    if (!DERIV) return;
-
-    // ============ the centre's own row: minus the sum over its neighbours ============
-    const long long row_base = p.row_ptr[c_idx];
-    const int my_row = p.self_row[c_idx];
+    // ============ power spectrum (Eq. 4) and the centre's own row ============
+    // threads walk the features l-major so that the lanes of a warp share the trip count 2l+1;
+    // the centre's row is minus the sum over its neighbours: -K_l sum_m (D^mu c^nu + c^mu D^nu)
+    const long long row_base = DERIV ? p.row_ptr[c_idx] : 0;
     {
-        float* out = p.out_jac + (size_t)(row_base + my_row) * 3 * F;
-        for (int f = tid; f < F; f += kThreads) {
+        float* desc_row = p.out_desc + (size_t)c_idx * F;
+        float* own = DERIV ? p.out_jac + (size_t)(row_base + p.self_row[c_idx]) * 3 * F : nullptr;
+        const int NP = F / L1;                                  // (species pair, n, n') combinations
+        for (int g = tid; g < ((SOAP_DEBUG_SKIP & 8) ? 0 : F); g += kThreads) {
+            const int l = g / NP, f = (g - l * NP) * L1 + l;
             const int pk = __ldg(p.feat_pack + f);
-            const int n1 = pk & 31, n2 = (pk >> 5) & 31, mu = (pk >> 10) & 15, nu = (pk >> 14) & 15, l = (pk >> 18) & 15;
+            const int n1 = pk & 31, n2 = (pk >> 5) & 31, mu = (pk >> 10) & 15, nu = (pk >> 14) & 15;
             const int ia = (mu * NMAX + n1) * LMP + l * l, ib = (nu * NMAX + n2) * LMP + l * l;
-            const float kl = -__ldg(p.kl + l);
-            float ax = 0.f, ay = 0.f, az = 0.f;
+            const float kl = __ldg(p.kl + l);
+            float acc = 0.f, ax = 0.f, ay = 0.f, az = 0.f;
             for (int m = 0; m <= 2 * l; ++m) {
                 const float ca = c_t[ia + m], cb = c_t[ib + m];
-                ax = fmaf(D_t[ia + m], cb, fmaf(ca, D_t[ib + m], ax));
-                ay = fmaf(D_t[CT + ia + m], cb, fmaf(ca, D_t[CT + ib + m], ay));
-                az = fmaf(D_t[2 * CT + ia + m], cb, fmaf(ca, D_t[2 * CT + ib + m], az));
+                acc = fmaf(ca, cb, acc);
+                if (DERIV) {
+                    ax = fmaf(D_t[ia + m], cb, fmaf(ca, D_t[ib + m], ax));
+                    ay = fmaf(D_t[CT + ia + m], cb, fmaf(ca, D_t[CT + ib + m], ay));
+                    az = fmaf(D_t[2 * CT + ia + m], cb, fmaf(ca, D_t[2 * CT + ib + m], az));
+                }
             }
-            out[f] = kl * ax; out[(size_t)F + f] = kl * ay; out[(size_t)2 * F + f] = kl * az;
+            desc_row[f] = kl * acc;
+            if (DERIV) { own[f] = -kl * ax; own[(size_t)F + f] = -kl * ay; own[(size_t)2 * F + f] = -kl * az; }
         }
-        if (tid == 0) p.row_atom[row_base + my_row] = ci;
+        if (DERIV && tid == 0) p.row_atom[row_base + p.self_row[c_idx]] = ci;
     }
+    if (!DERIV) return;
     __syncthreads();
-    // fold K_l into c for pass 2 (D is dead from here; its space becomes the U/V staging)
+    // fold K_l into c for pass 2
     for (int e = tid; e < S * NMAX * LM; e += kThreads) {
         const int row = e / LM, lm = e - row * LM;
         c_t[row * LMP + lm] *= __ldg(p.kl + __ldg(p.l_of_lm + lm));
@@ -283,155 +291,169 @@ center_kernel(const CenterParams p) {
     // =========================== pass 2: the Jacobian rows ===========================
     const int NI = S * NCH, SN = S * NMAX;
     float4* wUV = reinterpret_cast<float4*>(smem + lay.wUV) + wid * NI;       // [nu][n'][l]
-    for (int g0 = 0; g0 < k_pairs; g0 += kGeoPairs) {
-        const int gc = min(kGeoPairs, k_pairs - g0);
-        __syncthreads();
-        if (g0 > 0 || k_pairs > kGeoPairs) stage_geometry(g0, gc);     // otherwise still valid from pass 1
-        __syncthreads();
-        for (int q0 = 0; q0 < gc; q0 += P) {
-            const int pc = min(P, gc - q0);
-            stage_chunk(q0, pc);
-            __syncthreads();
-            for (int pr = 0; pr < pc; ++pr) {
-                const int4 gi = geo_i[q0 + pr];
-                const int rw = gi.w;
-                if (rw & kRowSelfImage) continue;
-                const int row = rw & kRowMask;
-                if ((row & (kWarps - 1)) != wid) continue;
-                const bool accumulate = rw & kRowContinuation;
-                const int Z = gi.z & 255;
-                const float4 d = geo_d[q0 + pr];
-                const float2* wG = sG2 + pr * NCH;
-                const float4* wSD = sSD4 + pr * LMP;
-                __syncwarp();
-                // ---- U, V for every (nu, n', l) ----
-                if (SN <= 16) {
-                    // lane <-> (nu n', half): half 0 accumulates (U, Vx), half 1 (Vy, Vz)
-                    const int sn = lane >> 1, half = lane & 1;
-                    if (sn < SN) {
-                        const float* cp = c_t + sn * LMP;
-                        const float2* hp = reinterpret_cast<const float2*>(wSD) + half;
-                        float2* up = reinterpret_cast<float2*>(wUV + sn * L1) + half;
+
+    // product rule of one pair: stores the row (or adds to it when another image of the same atom
+    // already wrote it) and subtracts it from the centre's row
+    auto product_rule = [&](auto acc_tag, int Z, float4 d, const float2* wG, float* out) {
+        constexpr bool ACC = decltype(acc_tag)::value;
+        auto emit = [&](float* o, float v) {
+            if (ACC) *o += v; else *o = v;
+        };
+        int boff = 0;
+        for (int mu = 0; mu < S; ++mu) {
+            for (int nu = mu; nu < S; ++nu) {
+                const int bsize = (mu == nu) ? (NMAX * (NMAX + 1) / 2) * L1 : NMAX * NCH;
+                float* ob = out + boff;
+                boff += bsize;
+                if (mu != Z && nu != Z) {
+                    if (!ACC) {
+                        float *o0 = ob + lane, *o1 = o0 + F, *o2 = o1 + F;
+                        for (int f = lane; f < bsize; f += 32) { *o0 = 0.f; *o1 = 0.f; *o2 = 0.f; o0 += 32; o1 += 32; o2 += 32; }
+                    }
+                } else if (mu == nu) {
+                    // both terms; feature (n1 <= n2, l) sits at L1 (n1 NMAX - n1(n1-1)/2) + (n2-n1) L1 + l
+                    const float4* UVz = wUV + Z * NCH;
+                    for (int j0 = 0; j0 < NCH; j0 += 32) {
+                        const int j = j0 + lane;
+                        const bool live = j < NCH;
+                        const int jj = live ? j : 0;
+                        const int n2 = jj / L1, l = jj - n2 * L1;
+                        const float2 gj = wG[jj];
+                        const float4 uj = UVz[jj];
+                        const float2* g1p = wG + l;
+                        const float4* u1p = UVz + l;
+                        float *o0 = ob + jj, *o1 = o0 + F, *o2 = o1 + F;
+                        const int n1_hi = min(NMAX - 1, (j0 + 31) / L1);     // no lane of this round goes beyond
 #pragma unroll
-                        for (int l = 0; l <= L; ++l) {
-                            float2 acc = make_float2(0.f, 0.f);
-#pragma unroll
-                            for (int m = 0; m <= 2 * l; ++m) {
-                                const float cv = cp[l * l + m];
-                                const float2 h = hp[2 * (l * l + m)];
-                                acc.x = fmaf(cv, h.x, acc.x); acc.y = fmaf(cv, h.y, acc.y);
+                        for (int n1 = 0; n1 < NMAX_BOUND; ++n1) {
+                            if (n1 > n1_hi) break;
+                            const int off = (n1 * NMAX - n1 * (n1 + 1) / 2) * L1;   // feature offset relative to n1 = 0
+                            if (live && n1 <= n2) {
+                                const float2 g1 = g1p[n1 * L1];
+                                const float4 u1 = u1p[n1 * L1];
+                                const float w = fmaf(g1.y, uj.x, gj.y * u1.x);    // Ghat_n1 U_n2 + Ghat_n2 U_n1
+                                emit(o0 + off, fmaf(g1.x, uj.y, fmaf(gj.x, u1.y, w * d.x)));
+                                emit(o1 + off, fmaf(g1.x, uj.z, fmaf(gj.x, u1.z, w * d.y)));
+                                emit(o2 + off, fmaf(g1.x, uj.w, fmaf(gj.x, u1.w, w * d.z)));
                             }
-                            up[2 * l] = acc;
+                        }
+                    }
+                } else if (mu == Z) {
+                    // (grad c^mu_{n1 l}) c^nu_{n2 l}: G_{n1 l} V^nu_{n2 l} + Ghat_{n1 l} d U^nu_{n2 l}
+                    for (int j = lane; j < NCH; j += 32) {
+                        const int l = j % L1;
+                        const float4 uj = wUV[nu * NCH + j];
+                        const float xx = uj.x * d.x, xy = uj.x * d.y, xz = uj.x * d.z;
+                        const float2* g1p = wG + l;
+                        float *o0 = ob + j, *o1 = o0 + F, *o2 = o1 + F;
+#pragma unroll
+                        for (int n1 = 0; n1 < NMAX_BOUND; ++n1) {
+                            if (n1 >= NMAX) break;
+                            const float2 g1 = g1p[n1 * L1];
+                            emit(o0 + n1 * NCH, fmaf(g1.x, uj.y, g1.y * xx));
+                            emit(o1 + n1 * NCH, fmaf(g1.x, uj.z, g1.y * xy));
+                            emit(o2 + n1 * NCH, fmaf(g1.x, uj.w, g1.y * xz));
                         }
                     }
                 } else {
-                    for (int sn = lane; sn < SN; sn += 32) {
-                        const float* cp = c_t + sn * LMP;
+                    // c^mu_{n1 l} (grad c^nu_{n2 l}): G_{n2 l} V^mu_{n1 l} + Ghat_{n2 l} d U^mu_{n1 l}
+                    for (int j = lane; j < NCH; j += 32) {
+                        const int l = j % L1;
+                        const float2 gj = wG[j];
+                        const float gx = gj.y * d.x, gy = gj.y * d.y, gz = gj.y * d.z;
+                        const float4* u1p = wUV + mu * NCH + l;
+                        float *o0 = ob + j, *o1 = o0 + F, *o2 = o1 + F;
 #pragma unroll
-                        for (int l = 0; l <= L; ++l) {
-                            float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-#pragma unroll
-                            for (int m = 0; m <= 2 * l; ++m) {
-                                const float cv = cp[l * l + m];
-                                const float4 h = wSD[l * l + m];
-                                acc.x = fmaf(cv, h.x, acc.x); acc.y = fmaf(cv, h.y, acc.y);
-                                acc.z = fmaf(cv, h.z, acc.z); acc.w = fmaf(cv, h.w, acc.w);
-                            }
-                            wUV[sn * L1 + l] = acc;
+                        for (int n1 = 0; n1 < NMAX_BOUND; ++n1) {
+                            if (n1 >= NMAX) break;
+                            const float4 u1 = u1p[n1 * L1];
+                            emit(o0 + n1 * NCH, fmaf(gj.x, u1.y, gx * u1.x));
+                            emit(o1 + n1 * NCH, fmaf(gj.x, u1.z, gy * u1.x));
+                            emit(o2 + n1 * NCH, fmaf(gj.x, u1.w, gz * u1.x));
                         }
                     }
                 }
-                __syncwarp();
-                // ---- product rule and store ----
-                float* out = p.out_jac + (size_t)(row_base + row) * 3 * F;
-                if (!accumulate && lane == 0) p.row_atom[row_base + row] = geo_j[q0 + pr];
-                int boff = 0;
-                for (int mu = 0; mu < S; ++mu) {
-                    for (int nu = mu; nu < S; ++nu) {
-                        const int bsize = (mu == nu) ? (NMAX * (NMAX + 1) / 2) * L1 : NMAX * NCH;
-                        float* ob = out + boff;
-                        boff += bsize;
-                        if (mu != Z && nu != Z) {
-                            if (!accumulate) {
-                                float *o0 = ob + lane, *o1 = o0 + F, *o2 = o1 + F;
-                                int f = lane;
-                                for (; f + 96 < bsize; f += 128) {
+            }
+        }
+    };
+
+    // everything one warp does for one pair of the staged chunk
+    auto do_pair = [&](int g, int pr) {
+        const int4 gi = geo_i[g];
+        const int rw = gi.w;
+        const int row = rw & kRowMask;
+        const int Z = gi.z & 255;
+        const float4 d = geo_d[g];
+        const float2* wG = sG2 + pr * NCH;
+        const float4* wSD = sSD4 + pr * LMP;
+        __syncwarp();
+        // ---- U, V for every (nu, n', l) ----
+        if (SOAP_DEBUG_SKIP & 2) {
+        } else if (SN <= 16) {
+            // lane <-> (nu n', half): half 0 accumulates (U, Vx), half 1 (Vy, Vz)
+            const int sn = lane >> 1, half = lane & 1;
+            if (sn < SN) {
+                const float* cp = c_t + sn * LMP;
+                const float2* hp = reinterpret_cast<const float2*>(wSD) + half;
+                float2* up = reinterpret_cast<float2*>(wUV + sn * L1) + half;
 #pragma unroll
-                                    for (int u = 0; u < 4; ++u) { o0[32 * u] = 0.f; o1[32 * u] = 0.f; o2[32 * u] = 0.f; }
-                                    o0 += 128; o1 += 128; o2 += 128;
-                                }
-                                for (; f < bsize; f += 32) { *o0 = 0.f; *o1 = 0.f; *o2 = 0.f; o0 += 32; o1 += 32; o2 += 32; }
-                            }
-                        } else if (mu == nu) {
-                            // both terms; feature (n1 <= n2, l) sits at L1 (n1 NMAX - n1(n1-1)/2) + (n2-n1) L1 + l
-                            const float4* UVz = wUV + Z * NCH;
-                            for (int j0 = 0; j0 < NCH; j0 += 32) {
-                                const int j = j0 + lane;
-                                const bool live = j < NCH;
-                                const int jj = live ? j : 0;
-                                const int n2 = jj / L1, l = jj - n2 * L1;
-                                const float2 gj = wG[jj];
-                                const float4 uj = UVz[jj];
-                                const float2* g1p = wG + l;
-                                const float4* u1p = UVz + l;
-                                float *o0 = ob + jj, *o1 = o0 + F, *o2 = o1 + F;
-                                const int n1_hi = min(NMAX - 1, (j0 + 31) / L1);     // no lane of this round goes beyond
+                for (int l = 0; l <= L; ++l) {
+                    float2 acc = make_float2(0.f, 0.f);
 #pragma unroll
-                                for (int n1 = 0; n1 < NMAX_BOUND; ++n1) {
-                                    if (n1 > n1_hi) break;
-                                    const int off = (n1 * NMAX - n1 * (n1 + 1) / 2) * L1;   // feature offset relative to n1 = 0
-                                    if (live && n1 <= n2) {
-                                        const float2 g1 = g1p[n1 * L1];
-                                        const float4 u1 = u1p[n1 * L1];
-                                        const float w = fmaf(g1.y, uj.x, gj.y * u1.x);    // Ghat_n1 U_n2 + Ghat_n2 U_n1
-                                        const float vx = fmaf(g1.x, uj.y, fmaf(gj.x, u1.y, w * d.x));
-                                        const float vy = fmaf(g1.x, uj.z, fmaf(gj.x, u1.z, w * d.y));
-                                        const float vz = fmaf(g1.x, uj.w, fmaf(gj.x, u1.w, w * d.z));
-                                        if (accumulate) { o0[off] += vx; o1[off] += vy; o2[off] += vz; }
-                                        else { o0[off] = vx; o1[off] = vy; o2[off] = vz; }
-                                    }
-                                }
-                            }
-                        } else if (mu == Z) {
-                            // (grad c^mu_{n1 l}) c^nu_{n2 l}: G_{n1 l} V^nu_{n2 l} + Ghat_{n1 l} d U^nu_{n2 l}
-                            for (int j = lane; j < NCH; j += 32) {
-                                const int l = j % L1;
-                                const float4 uj = wUV[nu * NCH + j];
-                                const float xx = uj.x * d.x, xy = uj.x * d.y, xz = uj.x * d.z;
-                                const float2* g1p = wG + l;
-                                float *o0 = ob + j, *o1 = o0 + F, *o2 = o1 + F;
-#pragma unroll
-                                for (int n1 = 0; n1 < NMAX_BOUND; ++n1) {
-                                    if (n1 >= NMAX) break;
-                                    const float2 g1 = g1p[n1 * L1];
-                                    const float vx = fmaf(g1.x, uj.y, g1.y * xx);
-                                    const float vy = fmaf(g1.x, uj.z, g1.y * xy);
-                                    const float vz = fmaf(g1.x, uj.w, g1.y * xz);
-                                    if (accumulate) { o0[n1 * NCH] += vx; o1[n1 * NCH] += vy; o2[n1 * NCH] += vz; }
-                                    else { o0[n1 * NCH] = vx; o1[n1 * NCH] = vy; o2[n1 * NCH] = vz; }
-                                }
-                            }
-                        } else {
-                            // c^mu_{n1 l} (grad c^nu_{n2 l}): G_{n2 l} V^mu_{n1 l} + Ghat_{n2 l} d U^mu_{n1 l}
-                            for (int j = lane; j < NCH; j += 32) {
-                                const int l = j % L1;
-                                const float2 gj = wG[j];
-                                const float gx = gj.y * d.x, gy = gj.y * d.y, gz = gj.y * d.z;
-                                const float4* u1p = wUV + mu * NCH + l;
-                                float *o0 = ob + j, *o1 = o0 + F, *o2 = o1 + F;
-#pragma unroll
-                                for (int n1 = 0; n1 < NMAX_BOUND; ++n1) {
-                                    if (n1 >= NMAX) break;
-                                    const float4 u1 = u1p[n1 * L1];
-                                    const float vx = fmaf(gj.x, u1.y, gx * u1.x);
-                                    const float vy = fmaf(gj.x, u1.z, gy * u1.x);
-                                    const float vz = fmaf(gj.x, u1.w, gz * u1.x);
-                                    if (accumulate) { o0[n1 * NCH] += vx; o1[n1 * NCH] += vy; o2[n1 * NCH] += vz; }
-                                    else { o0[n1 * NCH] = vx; o1[n1 * NCH] = vy; o2[n1 * NCH] = vz; }
-                                }
-                            }
-                        }
+                    for (int m = 0; m <= 2 * l; ++m) {
+                        const float cv = cp[l * l + m];
+                        const float2 h = hp[2 * (l * l + m)];
+                        acc.x = fmaf(cv, h.x, acc.x); acc.y = fmaf(cv, h.y, acc.y);
                     }
+                    up[2 * l] = acc;
+                }
+            }
+        } else {
+            for (int sn = lane; sn < SN; sn += 32) {
+                const float* cp = c_t + sn * LMP;
+#pragma unroll
+                for (int l = 0; l <= L; ++l) {
+                    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+                    for (int m = 0; m <= 2 * l; ++m) {
+                        const float cv = cp[l * l + m];
+                        const float4 h = wSD[l * l + m];
+                        acc.x = fmaf(cv, h.x, acc.x); acc.y = fmaf(cv, h.y, acc.y);
+                        acc.z = fmaf(cv, h.z, acc.z); acc.w = fmaf(cv, h.w, acc.w);
+                    }
+                    wUV[sn * L1 + l] = acc;
+                }
+            }
+        }
+        __syncwarp();
+        if (SOAP_DEBUG_SKIP & 1) return;
+        float* out = p.out_jac + (size_t)(row_base + row) * 3 * F;
+        if (rw & kRowContinuation) {
+            product_rule(std::true_type{}, Z, d, wG, out);
+        } else {
+            if (lane == 0) p.row_atom[row_base + row] = geo_j[g];
+            product_rule(std::false_type{}, Z, d, wG, out);
+        }
+    };
+
+    for (int g0 = 0; g0 < k_pairs; g0 += kGeoPairs) {
+        const int gc = min(kGeoPairs, k_pairs - g0);
+        __syncthreads();
+        if (g0 > 0 || k_pairs > kGeoPairs) special = stage_geometry(g0, gc);     // otherwise still valid from pass 1
+        for (int q0 = 0; q0 < gc; q0 += P) {
+            const int pc = min(P, gc - q0);
+            stage_chunk(q0, pc, std::true_type{});
+            __syncthreads();
+            if (!special) {
+                // every pair has a row of its own: deal them out round-robin
+                for (int pr = wid; pr < pc; pr += kWarps) do_pair(q0 + pr, pr);
+            } else {
+                // images of one atom share a row and must stay with one warp, in order;
+                // images of the centre itself do not move relative to it and are skipped
+                for (int pr = 0; pr < pc; ++pr) {
+                    const int rw = geo_i[q0 + pr].w;
+                    if ((rw & kRowSelfImage) || ((rw & kRowMask) & (kWarps - 1)) != wid) continue;
+                    do_pair(q0 + pr, pr);
                 }
             }
             __syncthreads();

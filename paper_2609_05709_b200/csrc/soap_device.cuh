@@ -92,8 +92,7 @@ __host__ __device__ inline void key_shift(unsigned long long k, int s[3]) {
 // Shared-memory carve-up of the per-centre kernel, in 4-byte words.  Every region
 // starts on a 16-byte boundary.  Rows of the coefficient tiles and of the harmonics
 // staging have the odd stride (l_max+1)^2 | 1, which keeps strided accesses off a
-// single bank.  The D tiles (pass 1) and the per-warp U/V staging (pass 2) never
-// live at the same time and share space.
+// single bank.
 constexpr int kGeoPairs = 128;           // pairs whose geometry is staged at once
 
 struct SmemLayout {
@@ -106,6 +105,8 @@ __host__ __device__ inline SmemLayout make_layout(int S, int n_max, int l_max, i
     int off = 0;
     o.c = off; off = align4(off + CT);
     o.geo = off; off = align4(off + kGeoPairs * 9);
+    // the D tiles (pass 1, centre's row) and the per-warp U/V staging (pass 2) never live
+    // at the same time and share space
     o.D = off; o.wUV = off;
     if (deriv) {
         const int a = 3 * CT, b = kWarps * S * NCH * 4;
