@@ -29,8 +29,18 @@
 #ifndef SOAP_DEBUG_SKIP
 #define SOAP_DEBUG_SKIP 0
 #endif
+#ifndef SOAP_MIN_CTAS_DERIV
+#define SOAP_MIN_CTAS_DERIV 3          // resident CTAs per SM the derivative kernel is compiled for
+#endif
 
 namespace soap {
+
+// Universal small tables for the harmonic recursion (l_max <= 12), read with
+// warp-uniform indices, hence constant memory.  Each translation unit that
+// includes this file gets its own copy, filled in at load time.
+__device__ __constant__ float kc_anorm[91] = {0};    // [(l,m)] sqrt((2l+1)/4pi (l-m)!/(l+m)!) (times sqrt2 for m > 0)
+__device__ __constant__ float kc_dfact[16] = {0};    // [m] (2m-1)!!
+__device__ __constant__ float kc_inv_int[32] = {0};  // [k] 1/k
 
 // Degree-5 table lookup: value and derivative with respect to the interval coordinate t.
 __device__ __forceinline__ void radial_lookup(const float* __restrict__ table, int qi, int n_ch, int ch, float t,
@@ -53,9 +63,8 @@ __device__ __forceinline__ void radial_lookup(const float* __restrict__ table, i
 //   dQ_l^m/dx = -x Q_{l-1}^{m+1},  dQ_l^m/dy = -y Q_{l-1}^{m+1},  dQ_l^m/dz = (l+m) Q_{l-1}^m.
 // Columns m and m+1 are advanced in lock step, so a step needs four registers.
 template <bool GRAD>
-__device__ __forceinline__ void harmonics_columns(int L, int wid, float4 d, const float* __restrict__ anorm,
-                                                  const float* __restrict__ dfact, const float* __restrict__ inv_int,
-                                                  float4* __restrict__ out4, float* __restrict__ out1) {
+__device__ __forceinline__ void harmonics_columns(int L, int wid, float4 d, float4* __restrict__ out4,
+                                                  float* __restrict__ out1) {
     const float x = d.x, y = d.y, z = d.z, r2 = d.w * d.w;
     for (int m = wid; m <= L; m += kWarps) {
         float cm = 1.f, sm = 0.f, cp = 0.f, sp = 0.f;           // (x+iy)^m and (x+iy)^(m-1)
@@ -65,11 +74,11 @@ __device__ __forceinline__ void harmonics_columns(int L, int wid, float4 d, cons
             sm = x * sm + y * cm;
             cm = cn;
         }
-        float a1 = __ldg(dfact + m), a0 = 0.f;                  // Q_l^m, Q_{l-1}^m
+        float a1 = kc_dfact[m], a0 = 0.f;                  // Q_l^m, Q_{l-1}^m
         float b1 = 0.f, b0 = 0.f;                               // Q_l^{m+1}, Q_{l-1}^{m+1}
         const float fm = (float)m;
         for (int l = m; l <= L; ++l) {
-            const float a = __ldg(anorm + l * (l + 1) / 2 + m);
+            const float a = kc_anorm[l * (l + 1) / 2 + m];
             const float aq = a * a1;
             const int lm0 = l * l + l;
             if (!GRAD) {
@@ -84,16 +93,16 @@ __device__ __forceinline__ void harmonics_columns(int L, int wid, float4 d, cons
             }
             // advance both columns to l + 1
             const float zz = (float)(2 * l + 1) * z;
-            const float an = (zz * a1 - (float)(l + m) * r2 * a0) * __ldg(inv_int + l + 1 - m);
+            const float an = (zz * a1 - (float)(l + m) * r2 * a0) * kc_inv_int[l + 1 - m];
             a0 = a1; a1 = an;
-            const float bn = (l == m) ? __ldg(dfact + m + 1) : (zz * b1 - (float)(l + m + 1) * r2 * b0) * __ldg(inv_int + l - m);
+            const float bn = (l == m) ? kc_dfact[m + 1] : (zz * b1 - (float)(l + m + 1) * r2 * b0) * kc_inv_int[l - m];
             b0 = b1; b1 = bn;
         }
     }
 }
 
 template <bool DERIV, int L, int NMAX_T>
-__global__ void __launch_bounds__(kThreads, DERIV ? 3 : 4)
+__global__ void __launch_bounds__(kThreads, DERIV ? SOAP_MIN_CTAS_DERIV : 4)
 center_kernel(const CenterParams p) {
     constexpr int L1 = L + 1, LM = L1 * L1, LMP = LM | 1;      // odd row stride: no shared-memory bank conflicts
     constexpr int NMAX_BOUND = NMAX_T ? NMAX_T : 16;
@@ -190,7 +199,7 @@ center_kernel(const CenterParams p) {
             }
         }
         if (lane < pc)
-            harmonics_columns<GRAD>(L, wid, geo_d[g + lane], p.anorm, p.dfact, p.inv_int, sSD4 + lane * LMP, sS + lane * LMP);
+            harmonics_columns<GRAD>(L, wid, geo_d[g + lane], sSD4 + lane * LMP, sS + lane * LMP);
     };
 
     // =========================== pass 1: c (and D) ===========================
@@ -296,7 +305,9 @@ center_kernel(const CenterParams p) {
     // already wrote it) and subtracts it from the centre's row
     auto product_rule = [&](auto acc_tag, int Z, float4 d, const float2* wG, float* out) {
         constexpr bool ACC = decltype(acc_tag)::value;
+        float dbg_sink = 0.f;
         auto emit = [&](float* o, float v) {
+            if (SOAP_DEBUG_SKIP & 32) { dbg_sink += v; return; }
             if (ACC) *o += v; else *o = v;
         };
         int boff = 0;
@@ -306,7 +317,7 @@ center_kernel(const CenterParams p) {
                 float* ob = out + boff;
                 boff += bsize;
                 if (mu != Z && nu != Z) {
-                    if (!ACC) {
+                    if (!ACC && !(SOAP_DEBUG_SKIP & 64)) {
                         float *o0 = ob + lane, *o1 = o0 + F, *o2 = o1 + F;
                         for (int f = lane; f < bsize; f += 32) { *o0 = 0.f; *o1 = 0.f; *o2 = 0.f; o0 += 32; o1 += 32; o2 += 32; }
                     }
@@ -375,6 +386,7 @@ center_kernel(const CenterParams p) {
                 }
             }
         }
+        if ((SOAP_DEBUG_SKIP & 32) && dbg_sink == 123.456f) out[lane] = dbg_sink;
     };
 
     // everything one warp does for one pair of the staged chunk

@@ -4,6 +4,7 @@
 #include <algorithm>
 #include <cmath>
 #include <cstdio>
+#include <cstdlib>
 #include <cstring>
 #include <new>
 #include <string>
@@ -17,6 +18,14 @@
 using namespace soap;
 
 namespace soap {
+cudaError_t center_constants(int l_max, const float* anorm91, const float* dfact16, const float* inv32) {
+    switch (l_max) {
+#define X(LV) case LV: return center_constants_l##LV(anorm91, dfact16, inv32);
+        X(0) X(1) X(2) X(3) X(4) X(5) X(6) X(7) X(8) X(9) X(10) X(11) X(12)
+#undef X
+    }
+    return cudaErrorInvalidValue;
+}
 cudaError_t center_set_smem(bool deriv, int l_max, int n_max, int bytes) {
     switch (l_max) {
 #define X(LV) case LV: return center_set_smem_l##LV(deriv, n_max, bytes);
@@ -183,9 +192,21 @@ int ensure_device(soap_t* h) {
             if (P >= (pass == 2 ? 4 : 8) && bytes <= budget) break;
             if (P < 4) P = 4;
         }
+        if (const char* env = std::getenv("SOAP_B200_CHUNK")) {       // tuning knob: pairs staged per chunk (4..32)
+            const int v = std::atoi(env);
+            if (v >= 4 && v <= 32) P = v;
+        }
         bytes = (size_t)make_layout(h->S, h->n_max, h->l_max, P, deriv).total * 4;
         if (bytes > (size_t)max_smem) return fail(h, SOAP_ERR_INVALID_ARG, "this basis does not fit the shared memory of the device");
         if (deriv) { h->P_deriv = P; h->smem_deriv = bytes; } else { h->P_desc = P; h->smem_desc = bytes; }
+    }
+    {
+        // universal harmonic tables up to l = 12 (the handle's own tables stop at its l_max)
+        std::vector<float> anorm(91, 0.f), dfact(16, 0.f), inv(32, 0.f);
+        for (size_t i = 0; i < h->basis.anorm.size(); ++i) anorm[i] = h->basis.anorm[i];
+        for (size_t i = 0; i < h->basis.dfact.size(); ++i) dfact[i] = h->basis.dfact[i];
+        for (int k = 1; k < 32; ++k) inv[k] = 1.0f / k;
+        CU(center_constants(h->l_max, anorm.data(), dfact.data(), inv.data()));
     }
     CU(center_set_smem(false, h->l_max, h->n_max, (int)h->smem_desc));
     CU(center_set_smem(true, h->l_max, h->n_max, (int)h->smem_deriv));
