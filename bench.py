@@ -290,6 +290,84 @@ def run_cuda(args):
         dist.destroy_process_group()
 
 
+def time_case(struct, species, r_cut, n_max, l_max, sigma, rbf, mode, steps, warmup=3):
+    """Device-resident timing of one configuration; returns a dict for the tables in the benchmark spec."""
+    import torch
+    import paper_2609_05709_b200 as pkg
+    pbc = (True, True, True) if struct.cell is not None else (False, False, False)
+    soap = pkg.Soap(species, r_cut, n_max, l_max, sigma, rbf, pbc)
+    F, C = soap.n_features, struct.n_atoms
+    pos = torch.from_numpy(struct.positions).cuda()
+    num = torch.from_numpy(struct.numbers).cuda()
+    n_pairs, n_rows = soap.neighbors(pos, num, struct.cell)
+    desc = torch.empty((C, F), device="cuda")
+    if mode == "derivatives":
+        jac = torch.empty((n_rows, 3, F), device="cuda")
+        row_ptr = torch.empty(C + 1, dtype=torch.int64, device="cuda")
+        row_atom = torch.empty(n_rows, dtype=torch.int32, device="cuda")
+        step = lambda: soap.derivatives_into(pos, num, struct.cell, None, desc, jac, row_ptr, row_atom)
+        alg_bytes = n_rows * 3 * F * 4 + C * F * 4 + n_rows * 4 + n_pairs * 24 + (C + 1) * 16
+    else:
+        step = lambda: soap.descriptor(pos, num, struct.cell, None, out=desc)
+        alg_bytes = C * F * 4 + n_pairs * 24 + (C + 1) * 8
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
+    soap.profile(True)
+    for _ in range(warmup):
+        step()
+    soap.status()
+    total, kern, nbr = [], [], []
+    for _ in range(steps):
+        flush.fill_(1)
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        step()
+        e1.record()
+        e1.synchronize()
+        total.append(e0.elapsed_time(e1))
+        a, b = soap.profile_read()
+        nbr.append(a)
+        kern.append(b)
+    soap.status()
+    ms = statistics.median(total)
+    peak, _ = measured_peaks()
+    k_ms = statistics.median(kern)
+    out = {"mode": mode, "atoms": C, "n_max": n_max, "l_max": l_max, "features": F, "pairs": n_pairs, "rows": n_rows,
+           "ms_per_step": ms, "atoms_per_s": C / (ms * 1e-3), "kernel_ms": k_ms, "neighbour_search_ms": statistics.median(nbr),
+           "algorithmic_bytes": alg_bytes, "kernel_GBps": alg_bytes / (k_ms * 1e-3) / 1e9,
+           "hbm_frac_of_measured_peak": alg_bytes / (k_ms * 1e-3) / 1e9 / peak}
+    del soap
+    torch.cuda.empty_cache()
+    return out
+
+
+def run_suite(args):
+    import torch
+    from soap_inputs import multispecies_box, water_cluster
+    torch.cuda.set_device(0)
+    steps = args.steps
+    if args.suite == "map":
+        s = water_cluster(1000, 0)
+        for n_max in (2, 4, 6, 8, 10, 12):
+            for l_max in (2, 4, 6, 8, 10, 12):
+                r = time_case(s, [1, 8], 6.0, n_max, l_max, 0.5, 0, "derivatives", steps)
+                r["case"] = "map"
+                print(json.dumps(r), flush=True)
+    elif args.suite == "scaling":
+        for n_mol in (1000, 10000, 100000, 333334):
+            s = water_cluster(n_mol, 0)
+            r = time_case(s, [1, 8], 5.0, 8, 6, 0.5, 0, "descriptor", steps)
+            r["case"] = "scaling"
+            print(json.dumps(r), flush=True)
+    else:
+        for name in ("water8_gto_n4_l3_rc5", "water1000_gto_n8_l6_rc6", "chno2000_poly_n8_l8_rc5"):
+            kind, n, species, r_cut, n_max, l_max, sigma, rbf = WORKLOADS[name]
+            s = make_structure(name)
+            for mode in ("derivatives", "descriptor"):
+                r = time_case(s, species, r_cut, n_max, l_max, sigma, rbf, mode, steps)
+                r["case"] = name
+                print(json.dumps(r), flush=True)
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -299,9 +377,16 @@ def main():
     ap.add_argument("--workload", default=DEFAULT_WORKLOAD, choices=sorted(WORKLOADS))
     ap.add_argument("--kernel-only", action="store_true",
                     help="skip the end-to-end and CPU-baseline legs (for profiler captures)")
+    ap.add_argument("--suite", choices=["map", "scaling", "configs"],
+                    help="extra measurements beside the headline line: 'map' = descriptor+Jacobian over "
+                         "n_max x l_max on the 1000-molecule cluster, 'scaling' = descriptor-only on "
+                         "3k..1M atoms, 'configs' = the periodic multi-species box and the tiny cluster; "
+                         "prints one JSON line per case")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)
+    elif args.suite:
+        run_suite(args)
     else:
         run_cuda(args)
 
