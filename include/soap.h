@@ -127,6 +127,34 @@ int soap_derivatives(soap_t *h, const float *d_positions, const int32_t *d_numbe
  * pair and row counts of the last call (either pointer may be NULL). */
 int soap_status(soap_t *h, int64_t *n_pairs, int64_t *n_rows, void *stream);
 
+/* Neighbour counts with NO allocation anywhere in the call (the paper has no
+ * counterpart; this entry point exists for callers that must not allocate).
+ * Some callers cannot call cudaMalloc, or anything that may: a host
+ * application that gave its whole device-memory budget to its own pool at
+ * start-up, a latency-critical loop that cannot afford the implicit device
+ * synchronisation of an allocation, or a plug-in that is forbidden to touch
+ * the allocator of the process it lives in.  For them this call counts, for
+ * every atom of a NON-PERIODIC structure, the atoms within r_cut
+ * (0 < distance^2 < r_cut^2, the same exact fp64 test and the same cell-list
+ * kernels as soap_neighbors), keeping the cell list in a fixed array compiled
+ * into the library instead of allocated scratch.
+ *   d_positions [n_atoms,3] fp32, device   (input, caller-owned)
+ *   d_counts    [n_atoms]   int32, device  (output, caller-owned, fully overwritten)
+ *   message     optional host buffer of message_len bytes for the error text
+ * Limit: n_atoms <= 65536; more returns SOAP_ERR_CAPACITY and does nothing.
+ * Cost of the limit: about 2.4 MB of device memory on every GPU that loads the
+ * library, held until the process exits.
+ * The call uses no handle, calls no cudaMalloc / cudaFree / allocating library
+ * routine, and enqueues its work on `stream` without waiting.  The first call
+ * on a device also looks up the device address of the fixed array (once per
+ * device, with that device current); make that first call outside any stream
+ * capture.  All calls on one GPU share the one array, which keeps the last
+ * call's contents (the call clears what must start at zero): two calls whose
+ * work overlaps on the GPU - different streams, or different host threads on
+ * different streams - race on it and give wrong counts.  Serialise them. */
+int soap_neighbor_counts_static(const float *d_positions, int64_t n_atoms, double r_cut,
+                                int32_t *d_counts, void *stream, char *message, int64_t message_len);
+
 /* Per-segment timing, the counterpart of the paper's companion profiler
  * (end of its architecture section).  With profiling enabled,
  * soap_descriptor and soap_derivatives record CUDA events on the caller's

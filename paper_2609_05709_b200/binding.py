@@ -12,7 +12,7 @@ GTO, POLYNOMIAL = 0, 1
 EXPORTED_SYMBOLS = [
     "soap_create", "soap_destroy", "soap_num_features", "soap_feature_info", "soap_last_error",
     "soap_radial_table", "soap_neighbors", "soap_neighbor_list", "soap_descriptor",
-    "soap_derivatives", "soap_status", "soap_profile", "soap_profile_read",
+    "soap_derivatives", "soap_status", "soap_profile", "soap_profile_read", "soap_neighbor_counts_static",
 ]
 
 _ERRORS = {-1: "SOAP_ERR_INVALID_ARG", -2: "SOAP_ERR_UNKNOWN_SPECIES", -3: "SOAP_ERR_CAPACITY",
@@ -57,6 +57,7 @@ def load_library() -> C.CDLL:
     lib.soap_descriptor.argtypes = common + [vp, vp]
     lib.soap_derivatives.argtypes = common + [vp, vp, i64, vp, vp, vp]
     lib.soap_status.argtypes = [vp, C.POINTER(i64), C.POINTER(i64), vp]
+    lib.soap_neighbor_counts_static.argtypes = [vp, i64, C.c_double, vp, vp, C.c_char_p, i64]
     lib.soap_profile.argtypes = [vp, i32]
     lib.soap_profile_read.argtypes = [vp, C.POINTER(C.c_float), C.POINTER(C.c_float)]
     for name in EXPORTED_SYMBOLS:
@@ -64,6 +65,25 @@ def load_library() -> C.CDLL:
             getattr(lib, name).restype = C.c_int
     _LIB = lib
     return lib
+
+
+def neighbor_counts_static(positions, r_cut, out=None):
+    """Atoms within r_cut of every atom of a non-periodic structure, through the entry point that
+    allocates nothing inside the library (at most 65536 atoms; the output tensor is the caller's:
+    pass `out` to keep this wrapper allocation-free as well).  Work is enqueued on the current
+    stream; calls that overlap on the GPU race on the library's fixed scratch array."""
+    import torch
+    lib = load_library()
+    assert positions.is_cuda and positions.dtype == torch.float32 and positions.is_contiguous()
+    n = positions.shape[0]
+    if out is None:
+        out = torch.empty(n, dtype=torch.int32, device=positions.device)
+    msg = C.create_string_buffer(256)
+    rc = lib.soap_neighbor_counts_static(positions.data_ptr(), n, float(r_cut), out.data_ptr(),
+                                         C.c_void_p(torch.cuda.current_stream().cuda_stream), msg, 256)
+    if rc != 0:
+        raise SoapError(rc, msg.value.decode())
+    return out
 
 
 @dataclass

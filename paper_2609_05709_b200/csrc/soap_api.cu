@@ -504,6 +504,107 @@ int soap_status(soap_t* h, int64_t* n_pairs, int64_t* n_rows, void* stream) {
     return SOAP_OK;
 }
 
+// ---------------------------------------------------------------------------------------------
+// Neighbour counts without any allocation.
+//
+// Some hosts of this library may not allocate device memory when they call it: code that runs
+// inside a memory pool it must not disturb, a real-time loop where cudaMalloc's implicit
+// synchronisation is not acceptable, or a process whose memory budget was handed out in full at
+// start-up.  For them the cell list lives in the fixed array below, which every GPU that loads the
+// library carries until the process exits.
+constexpr int kStaticMaxAtoms = 65536;
+constexpr int kStaticMaxCells = 65536;
+struct StaticLayout {
+    static constexpr size_t header = 1024;                                       // bbox, grid, counters
+    static constexpr size_t atom_cell = header;
+    static constexpr size_t atom_wrap = atom_cell + sizeof(int) * kStaticMaxAtoms;
+    static constexpr size_t s_wrap = atom_wrap + sizeof(int) * kStaticMaxAtoms;
+    static constexpr size_t s_pos = s_wrap + sizeof(int) * kStaticMaxAtoms;
+    static constexpr size_t cell_count = s_pos + sizeof(float4) * kStaticMaxAtoms;
+    static constexpr size_t cell_start = cell_count + 256 * ((sizeof(int) * (kStaticMaxCells + 1) + 255) / 256);
+    static constexpr size_t total = cell_start + 256 * ((sizeof(int) * (kStaticMaxCells + 1) + 255) / 256);
+};
+static __device__ __align__(256) unsigned char g_static_scratch[StaticLayout::total];   // about 2.4 MB
+
+// bounding box only (the handle-based path also looks up species here; this one has no species)
+__global__ void bbox_only_kernel(const float* __restrict__ pos, long long N, Geometry geom, unsigned long long* bbox) {
+    double hi[3] = {-1e300, -1e300, -1e300}, lo[3] = {-1e300, -1e300, -1e300};
+    for (long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x; i < N; i += (long long)gridDim.x * blockDim.x) {
+        double f[3];
+        frac_coords(geom, pos[3 * i], pos[3 * i + 1], pos[3 * i + 2], f);
+        for (int a = 0; a < 3; ++a) { hi[a] = fmax(hi[a], f[a]); lo[a] = fmax(lo[a], -f[a]); }
+    }
+    for (int a = 0; a < 3; ++a)
+        for (int o = 16; o > 0; o >>= 1) {
+            hi[a] = fmax(hi[a], __shfl_xor_sync(0xffffffffu, hi[a], o));
+            lo[a] = fmax(lo[a], __shfl_xor_sync(0xffffffffu, lo[a], o));
+        }
+    if ((threadIdx.x & 31) == 0)
+        for (int a = 0; a < 3; ++a) {
+            atomicMax(&bbox[a], enc_double(hi[a]));
+            atomicMax(&bbox[3 + a], enc_double(lo[a]));
+        }
+}
+
+int soap_neighbor_counts_static(const float* d_positions, int64_t n_atoms, double r_cut, int32_t* d_counts,
+                                void* stream, char* message, int64_t message_len) {
+    auto say = [&](int code, const char* text) {
+        if (message && message_len > 0) std::snprintf(message, (size_t)message_len, "%s", text);
+        return code;
+    };
+    if (n_atoms < 0 || !(r_cut > 0) || (n_atoms > 0 && (!d_positions || !d_counts)))
+        return say(SOAP_ERR_INVALID_ARG, "need n_atoms >= 0, r_cut > 0 and non-NULL device pointers");
+    if (n_atoms > kStaticMaxAtoms)
+        return say(SOAP_ERR_CAPACITY, "soap_neighbor_counts_static handles at most 65536 atoms (fixed scratch); "
+                                       "use soap_neighbors for larger structures");
+    // Set-up, once per device: the array's name is only a host-side stand-in here, so ask the
+    // runtime for its device address.  The first call on a device does this (it may initialise
+    // the context) and should therefore come before any stream capture.
+    static unsigned char* base_of_device[64] = {nullptr};
+    int dev = -1;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return say(SOAP_ERR_CUDA, cudaGetErrorString(e));
+    if (dev < 0 || dev >= 64) return say(SOAP_ERR_INVALID_ARG, "device ordinal out of range");
+    if (!base_of_device[dev]) {
+        void* ptr = nullptr;
+        e = cudaGetSymbolAddress(&ptr, g_static_scratch);
+        if (e != cudaSuccess || !ptr) return say(SOAP_ERR_CUDA, cudaGetErrorString(e));
+        base_of_device[dev] = static_cast<unsigned char*>(ptr);
+    }
+    unsigned char* base = base_of_device[dev];
+    unsigned long long* bbox = reinterpret_cast<unsigned long long*>(base);
+    GridParams* grid = reinterpret_cast<GridParams*>(base + 256);
+    Counters* counters = reinterpret_cast<Counters*>(base + 768);
+    int* atom_cell = reinterpret_cast<int*>(base + StaticLayout::atom_cell);
+    int* atom_wrap = reinterpret_cast<int*>(base + StaticLayout::atom_wrap);
+    int* s_wrap = reinterpret_cast<int*>(base + StaticLayout::s_wrap);
+    float4* s_pos = reinterpret_cast<float4*>(base + StaticLayout::s_pos);
+    int* cell_count = reinterpret_cast<int*>(base + StaticLayout::cell_count);
+    int* cell_start = reinterpret_cast<int*>(base + StaticLayout::cell_start);
+    if (n_atoms == 0) return SOAP_OK;
+    Geometry g;
+    const double ident[9] = {1, 0, 0, 0, 1, 0, 0, 0, 1};
+    std::memcpy(g.cell, ident, sizeof(ident));
+    std::memcpy(g.inv, ident, sizeof(ident));
+    for (int a = 0; a < 3; ++a) { g.height[a] = 1.0; g.pbc[a] = 0; }
+    g.r_cut = r_cut;
+    g.rc2 = r_cut * r_cut;
+    cudaStream_t st = (cudaStream_t)stream;
+    const long long N = n_atoms;
+    // the array keeps whatever the previous call left: clear what has to start at zero
+    if ((e = cudaMemsetAsync(base, 0, StaticLayout::header, st)) != cudaSuccess) return say(SOAP_ERR_CUDA, cudaGetErrorString(e));
+    if ((e = cudaMemsetAsync(cell_count, 0, sizeof(int) * (kStaticMaxCells + 1), st)) != cudaSuccess) return say(SOAP_ERR_CUDA, cudaGetErrorString(e));
+    bbox_only_kernel<<<blocks_for(N, 256, 256), 256, 0, st>>>(d_positions, N, g, bbox);
+    grid_setup_kernel<<<1, 1, 0, st>>>(bbox, g, N, kStaticMaxCells, grid);
+    bin_count_kernel<<<blocks_for(N, 256), 256, 0, st>>>(d_positions, N, g, grid, atom_cell, atom_wrap, cell_count, counters);
+    scan_kernel<int><<<1, 1024, 0, st>>>(cell_count, cell_start, kStaticMaxCells, nullptr);
+    bin_fill_kernel<<<blocks_for(N, 256), 256, 0, st>>>(d_positions, N, atom_cell, atom_wrap, cell_start, cell_count, s_pos, s_wrap);
+    count_kernel<<<(unsigned)((N + 7) / 8), 256, 0, st>>>(d_positions, nullptr, N, g, grid, atom_cell, atom_wrap, cell_start, s_pos, s_wrap,
+                                                         d_counts, counters);
+    if ((e = cudaGetLastError()) != cudaSuccess) return say(SOAP_ERR_CUDA, cudaGetErrorString(e));
+    return SOAP_OK;
+}
+
 int soap_profile(soap_t* h, int enable) {
     if (!h) return SOAP_ERR_INVALID_ARG;
     if (enable) {
