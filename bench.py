@@ -165,6 +165,7 @@ def run_cuda(args):
     import torch
     import torch.distributed as dist
     import paper_2609_05709_b200 as pkg
+    from paper_2609_05709_b200.replicas import job_throughput, max_over_ranks
 
     world = int(os.environ.get("WORLD_SIZE", "1"))
     rank = int(os.environ.get("RANK", "0"))
@@ -244,17 +245,14 @@ def run_cuda(args):
         e2e_ms.append(e0.elapsed_time(e1))
     barrier()
     e2e_total = sum(e2e_ms)
-    if world > 1:
-        t = torch.tensor([total_ms, e2e_total], device="cuda", dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        total_ms, e2e_total = float(t[0]), float(t[1])
+    total_ms, e2e_total = max_over_ranks([total_ms, e2e_total], device="cuda")     # slowest rank decides
     if rank != 0:
         if world > 1:
             dist.destroy_process_group()
         return
     ms_per_step = total_ms / args.steps
-    value = world * C / (ms_per_step * 1e-3)
-    e2e_value = world * C / (e2e_total / e2e_steps * 1e-3) if e2e_steps else None
+    value = job_throughput(C, world, ms_per_step)
+    e2e_value = job_throughput(C, world, e2e_total / e2e_steps) if e2e_steps else None
     # ---- roofline of the dominant kernel (the fused per-centre kernel): HBM-write bound ----
     # algorithmic bytes per launch: Jacobian rows + descriptor + row_atom written, pair list and positions read
     alg_bytes = n_rows * 3 * F * 4 + C * F * 4 + n_rows * 4 + n_pairs * (8 + 4 + 12) + (C + 1) * 16
