@@ -106,8 +106,10 @@ __global__ void __launch_bounds__(kThreads, DERIV ? SOAP_MIN_CTAS_DERIV : 4)
 center_kernel(const CenterParams p) {
     constexpr int L1 = L + 1, LM = L1 * L1, LMP = LM | 1;      // odd row stride: no shared-memory bank conflicts
     constexpr int NMAX_BOUND = NMAX_T ? NMAX_T : 16;
-    constexpr int KE_RAW = (NMAX_BOUND * LM + kThreads - 1) / kThreads;
-    constexpr int KE = KE_RAW < kMaxElemPerThread ? KE_RAW : kMaxElemPerThread;
+    // pass-1 ownership: W_LM warps cover the lm index, SLOTS such groups split the n index
+    constexpr int W_LM = (LM + 31) / 32, SLOTS = kWarps / W_LM;
+    constexpr int NPT_RAW = (NMAX_BOUND + SLOTS - 1) / SLOTS;      // radial functions per thread ...
+    constexpr int NPT = NPT_RAW < 8 ? NPT_RAW : 8;                // ... at most 8 at a time (register budget)
     extern __shared__ __align__(16) float smem[];
     const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
     const long long c_idx = blockIdx.x;
@@ -141,46 +143,71 @@ center_kernel(const CenterParams p) {
         if (e < CT) c_t[e] = 0.f; else D_t[e - CT] = 0.f;
     }
 
-    // elements (n, lm) this thread accumulates in pass 1: offsets into a c tile and into the staging rows
-    int el_c[KE], el_lm[KE], el_ch[KE];
-#pragma unroll
-    for (int k = 0; k < KE; ++k) {
-        const int e = tid + k * kThreads;
-        const int n = e / LM, lm = e - n * LM;
-        el_lm[k] = e < NE ? lm : -1;
-        el_c[k] = n * LMP + lm;
-        el_ch[k] = n * L1 + __ldg(p.l_of_lm + lm);
-    }
+    // pass-1 ownership of this thread: one lm, and the radial functions slot, slot + SLOTS, ...
+    const int own_slot = wid / W_LM, own_lm = (wid - own_slot * W_LM) * 32 + lane;
+    const bool owner = own_slot < SLOTS && own_lm < LM;
+    const int own_l = owner ? __ldg(p.l_of_lm + own_lm) : 0;
 
-    // ---- geometry of up to kGeoPairs pairs, one thread each; returns whether any pair of the
-    //      batch shares its row with another or is an image of the centre ----
+    // ---- geometry of up to kGeoPairs pairs, one thread each, stored grouped by the neighbour's
+    //      species (stable, so images of one atom stay adjacent and in order); seg[s] .. seg[s+1]
+    //      are the pairs of species s.  Returns whether any pair of the batch shares its row with
+    //      another or is an image of the centre ----
+    int* seg = reinterpret_cast<int*>(smem + lay.geo + 9 * kGeoPairs);       // [kMaxSpecies + 1]
+    int* seg_warp = seg + kMaxSpecies + 1;                                   // [4 warps][kMaxSpecies]
     auto stage_geometry = [&](int g0, int gc) -> bool {
-        int special = 0;
-        if (tid < gc) {
-            const unsigned long long key = p.pair_key[pair_base + g0 + tid];
-            const int j = key_atom(key);
-            double dx = (double)p.pos[3 * (long long)j] - (double)xi;
-            double dy = (double)p.pos[3 * (long long)j + 1] - (double)yi;
-            double dz = (double)p.pos[3 * (long long)j + 2] - (double)zi;
-            if (periodic) {
-                int s[3];
-                key_shift(key, s);
-                dx += s[0] * p.geom.cell[0] + s[1] * p.geom.cell[3] + s[2] * p.geom.cell[6];
-                dy += s[0] * p.geom.cell[1] + s[1] * p.geom.cell[4] + s[2] * p.geom.cell[7];
-                dz += s[0] * p.geom.cell[2] + s[1] * p.geom.cell[5] + s[2] * p.geom.cell[8];
+        int special = 0, sp = -1, rank = 0, rw = 0, j = 0;
+        float4 dd = make_float4(0.f, 0.f, 0.f, 0.f);
+        int qi = 0;
+        float tt = 0.f;
+        if (tid < kGeoPairs) {
+            if (tid < gc) {
+                const unsigned long long key = p.pair_key[pair_base + g0 + tid];
+                j = key_atom(key);
+                double dx = (double)p.pos[3 * (long long)j] - (double)xi;
+                double dy = (double)p.pos[3 * (long long)j + 1] - (double)yi;
+                double dz = (double)p.pos[3 * (long long)j + 2] - (double)zi;
+                if (periodic) {
+                    int s[3];
+                    key_shift(key, s);
+                    dx += s[0] * p.geom.cell[0] + s[1] * p.geom.cell[3] + s[2] * p.geom.cell[6];
+                    dy += s[0] * p.geom.cell[1] + s[1] * p.geom.cell[4] + s[2] * p.geom.cell[7];
+                    dz += s[0] * p.geom.cell[2] + s[1] * p.geom.cell[5] + s[2] * p.geom.cell[8];
+                }
+                const double r = sqrt(dx * dx + dy * dy + dz * dz);
+                dd = make_float4((float)dx, (float)dy, (float)dz, (float)r);
+                rw = p.pair_row[pair_base + g0 + tid];
+                special = rw & (kRowSelfImage | kRowContinuation);
+                // interval and offset in the radial table, in fp64 so that the offset keeps its digits
+                const double u = r * (double)p.inv_h;
+                qi = min((int)u, p.n_intervals - 1);
+                tt = (float)(u - qi);
+                sp = p.species_idx[j];
             }
-            const double r = sqrt(dx * dx + dy * dy + dz * dz);
-            geo_d[tid] = make_float4((float)dx, (float)dy, (float)dz, (float)r);
-            const int rw = p.pair_row[pair_base + g0 + tid];
-            special = rw & (kRowSelfImage | kRowContinuation);
-            // interval and offset in the radial table, in fp64 so that the offset keeps its digits
-            const double u = r * (double)p.inv_h;
-            const int qi = min((int)u, p.n_intervals - 1);
-            geo_i[tid] = make_int4(qi, __float_as_int((float)(u - qi)),
-                                   p.species_idx[j] | ((rw & kRowSelfImage) ? 0 : 256), rw);
-            geo_j[tid] = j;
+            // stable partition by species: rank inside the warp, then offsets across warps
+            for (int s = 0; s < S; ++s) {
+                const unsigned m = __ballot_sync(0xffffffffu, sp == s);
+                if (sp == s) rank = __popc(m & ((1u << lane) - 1));
+                if (lane == 0) seg_warp[wid * kMaxSpecies + s] = __popc(m);
+            }
         }
-        return __syncthreads_or(special) != 0;
+        const bool any_special = __syncthreads_or(special) != 0;
+        if (tid < gc) {
+            int at = rank;
+            for (int s = 0; s < sp; ++s)
+                for (int w = 0; w < kGeoPairs / 32; ++w) at += seg_warp[w * kMaxSpecies + s];
+            for (int w = 0; w < wid; ++w) at += seg_warp[w * kMaxSpecies + sp];
+            geo_d[at] = dd;
+            geo_i[at] = make_int4(qi, __float_as_int(tt), sp | ((rw & kRowSelfImage) ? 0 : 256), rw);
+            geo_j[at] = j;
+        }
+        if (tid <= S) {
+            int at = 0;
+            for (int s = 0; s < tid; ++s)
+                for (int w = 0; w < kGeoPairs / 32; ++w) at += seg_warp[w * kMaxSpecies + s];
+            seg[tid] = at;
+        }
+        __syncthreads();
+        return any_special;
     };
 
     // ---- radial factors and solid harmonics of the pairs g .. g + pc - 1 of the staged geometry ----
@@ -203,56 +230,73 @@ center_kernel(const CenterParams p) {
     };
 
     // =========================== pass 1: c (and D) ===========================
+    // A thread owns c[s][n][own_lm] (and the three D tiles) for its n and keeps the sums of the
+    // species it is working on in registers; pairs arrive grouped by species, so the sums go to
+    // shared memory once per species and batch.
     bool special = false;
-    for (int g0 = 0; g0 < k_pairs; g0 += kGeoPairs) {
-        const int gc = min(kGeoPairs, k_pairs - g0);
-        __syncthreads();
-        special = stage_geometry(g0, gc);
-        for (int q0 = 0; q0 < gc; q0 += P) {
-            const int pc = min(P, gc - q0);
-            stage_chunk(q0, pc, std::integral_constant<bool, DERIV>{});
+    for (int n0 = 0; n0 < NMAX; n0 += SLOTS * NPT) {             // one trip unless n_max > 8 SLOTS
+        for (int g0 = 0; g0 < k_pairs; g0 += kGeoPairs) {
+            const int gc = min(kGeoPairs, k_pairs - g0);
             __syncthreads();
-            for (int s = 0; s < ((SOAP_DEBUG_SKIP & 4) ? 0 : S); ++s) {
-                float ac[KE], ax[KE], ay[KE], az[KE];
+            special = stage_geometry(g0, gc);
+            float ac[NPT], ax[NPT], ay[NPT], az[NPT];
 #pragma unroll
-                for (int k = 0; k < KE; ++k) ac[k] = ax[k] = ay[k] = az[k] = 0.f;
-                bool any = false;
-                for (int pr = 0; pr < pc; ++pr) {
-                    const int info = geo_i[q0 + pr].z;
-                    if ((info & 255) != s) continue;
-                    any = true;
-                    if (!DERIV) {
+            for (int k = 0; k < NPT; ++k) ac[k] = ax[k] = ay[k] = az[k] = 0.f;
+            int cur = -1;
+            auto flush = [&]() {
+                if (cur < 0 || !owner) return;
 #pragma unroll
-                        for (int k = 0; k < KE; ++k)
-                            if (el_lm[k] >= 0) ac[k] = fmaf(sG1[pr * NCH + el_ch[k]], sS[pr * LMP + el_lm[k]], ac[k]);
-                    } else {
-                        const float4 d = geo_d[q0 + pr];
-                        const float mv = (info & 256) ? 1.f : 0.f;   // an image of the centre does not move relative to it
-                        const float dxm = d.x * mv, dym = d.y * mv, dzm = d.z * mv;
+                for (int k = 0; k < NPT; ++k) {
+                    const int n = n0 + own_slot + k * SLOTS;
+                    if (n < NMAX) {
+                        const int e = (cur * NMAX + n) * LMP + own_lm;
+                        c_t[e] += ac[k];
+                        if (DERIV) { D_t[e] += ax[k]; D_t[CT + e] += ay[k]; D_t[2 * CT + e] += az[k]; }
+                    }
+                    ac[k] = ax[k] = ay[k] = az[k] = 0.f;
+                }
+            };
+            for (int q0 = 0; q0 < gc; q0 += P) {
+                const int pc = min(P, gc - q0);
+                stage_chunk(q0, pc, std::integral_constant<bool, DERIV>{});
+                __syncthreads();
+                if (owner && !(SOAP_DEBUG_SKIP & 4)) {
+                    for (int s = 0; s < S; ++s) {
+                        const int a = max(seg[s], q0), b = min(seg[s + 1], q0 + pc);
+                        if (a >= b) continue;
+                        if (s != cur) { flush(); cur = s; }
+                        for (int g = a; g < b; ++g) {
+                            const int pr = g - q0;
+                            if (!DERIV) {
+                                const float h = sS[pr * LMP + own_lm];
+                                const float* gp = sG1 + pr * NCH + (n0 + own_slot) * L1 + own_l;
 #pragma unroll
-                        for (int k = 0; k < KE; ++k)
-                            if (el_lm[k] >= 0) {
-                                const float2 g = sG2[pr * NCH + el_ch[k]];
-                                const float4 h = sSD4[pr * LMP + el_lm[k]];
-                                ac[k] = fmaf(g.x, h.x, ac[k]);
-                                const float gm = g.x * mv, t = g.y * h.x;
-                                ax[k] = fmaf(gm, h.y, fmaf(t, dxm, ax[k]));
-                                ay[k] = fmaf(gm, h.z, fmaf(t, dym, ay[k]));
-                                az[k] = fmaf(gm, h.w, fmaf(t, dzm, az[k]));
+                                for (int k = 0; k < NPT; ++k)
+                                    if (n0 + own_slot + k * SLOTS < NMAX) ac[k] = fmaf(gp[k * SLOTS * L1], h, ac[k]);
+                            } else {
+                                const float4 h = sSD4[pr * LMP + own_lm];
+                                const float4 d = geo_d[g];
+                                // an image of the centre does not move relative to it: no contribution to D
+                                const float mv = (geo_i[g].z & 256) ? 1.f : 0.f;
+                                const float hy = h.y * mv, hz = h.z * mv, hw = h.w * mv;
+                                const float tx = h.x * d.x * mv, ty = h.x * d.y * mv, tz = h.x * d.z * mv;
+                                const float2* gp = sG2 + pr * NCH + (n0 + own_slot) * L1 + own_l;
+#pragma unroll
+                                for (int k = 0; k < NPT; ++k)
+                                    if (n0 + own_slot + k * SLOTS < NMAX) {
+                                        const float2 gg = gp[k * SLOTS * L1];
+                                        ac[k] = fmaf(gg.x, h.x, ac[k]);
+                                        ax[k] = fmaf(gg.x, hy, fmaf(gg.y, tx, ax[k]));
+                                        ay[k] = fmaf(gg.x, hz, fmaf(gg.y, ty, ay[k]));
+                                        az[k] = fmaf(gg.x, hw, fmaf(gg.y, tz, az[k]));
+                                    }
                             }
+                        }
                     }
                 }
-                if (any) {
-#pragma unroll
-                    for (int k = 0; k < KE; ++k)
-                        if (el_lm[k] >= 0) {
-                            const int e = s * NMAX * LMP + el_c[k];
-                            c_t[e] += ac[k];
-                            if (DERIV) { D_t[e] += ax[k]; D_t[CT + e] += ay[k]; D_t[2 * CT + e] += az[k]; }
-                        }
-                }
+                __syncthreads();
             }
-            __syncthreads();
+            flush();
         }
     }
     __syncthreads();

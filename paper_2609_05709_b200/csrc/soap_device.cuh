@@ -104,7 +104,7 @@ __host__ __device__ inline SmemLayout make_layout(int S, int n_max, int l_max, i
     SmemLayout o;
     int off = 0;
     o.c = off; off = align4(off + CT);
-    o.geo = off; off = align4(off + kGeoPairs * 9);
+    o.geo = off; off = align4(off + kGeoPairs * 9 + (kMaxSpecies + 1) + (kGeoPairs / 32) * kMaxSpecies);   // + species segments
     // the D tiles (pass 1, centre's row) and the per-warp U/V staging (pass 2) never live
     // at the same time and share space
     o.D = off; o.wUV = off;
