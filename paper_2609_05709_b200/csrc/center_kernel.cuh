@@ -143,6 +143,16 @@ center_kernel(const CenterParams p) {
         if (e < CT) c_t[e] = 0.f; else D_t[e - CT] = 0.f;
     }
 
+    // same-species blocks: feature index -> (n1 L1 + l) | (n2 L1 + l) << 8, rows n1 of (NMAX - n1) L1 entries
+    unsigned short* tri_dec = reinterpret_cast<unsigned short*>(smem + lay.tri);
+    if (DERIV)
+        for (int e = tid; e < (NMAX * (NMAX + 1) / 2) * L1; e += kThreads) {
+            int n1 = 0, r = e;
+            while (r >= (NMAX - n1) * L1) { r -= (NMAX - n1) * L1; ++n1; }
+            const int n2 = n1 + r / L1, l = r % L1;
+            tri_dec[e] = (unsigned short)((n1 * L1 + l) | ((n2 * L1 + l) << 8));
+        }
+
     // pass-1 ownership of this thread: one lm, and the radial functions slot, slot + SLOTS, ...
     const int own_slot = wid / W_LM, own_lm = (wid - own_slot * W_LM) * 32 + lane;
     const bool owner = own_slot < SLOTS && own_lm < LM;
@@ -305,31 +315,58 @@ center_kernel(const CenterParams p) {
     __syncthreads();
 
     // ============ power spectrum (Eq. 4) and the centre's own row ============
-    // threads walk the features l-major so that the lanes of a warp share the trip count 2l+1;
-    // the centre's row is minus the sum over its neighbours: -K_l sum_m (D^mu c^nu + c^mu D^nu)
+    // Threads walk the features l-major so that the lanes of a warp share the trip count 2l+1; the
+    // centre's row is minus the sum over its neighbours: -K_l sum_m (D^mu c^nu + c^mu D^nu).  Results
+    // pass through the (now idle) staging area in slabs, so that global memory is written in
+    // feature order, whole sectors at a time.
     const long long row_base = DERIV ? p.row_ptr[c_idx] : 0;
     {
         float* desc_row = p.out_desc + (size_t)c_idx * F;
         float* own = DERIV ? p.out_jac + (size_t)(row_base + p.self_row[c_idx]) * 3 * F : nullptr;
-        const int NP = F / L1;                                  // (species pair, n, n') combinations
-        for (int g = tid; g < ((SOAP_DEBUG_SKIP & 8) ? 0 : F); g += kThreads) {
-            const int l = g / NP, f = (g - l * NP) * L1 + l;
-            const int pk = __ldg(p.feat_pack + f);
-            const int n1 = pk & 31, n2 = (pk >> 5) & 31, mu = (pk >> 10) & 15, nu = (pk >> 14) & 15;
-            const int ia = (mu * NMAX + n1) * LMP + l * l, ib = (nu * NMAX + n2) * LMP + l * l;
-            const float kl = __ldg(p.kl + l);
-            float acc = 0.f, ax = 0.f, ay = 0.f, az = 0.f;
-            for (int m = 0; m <= 2 * l; ++m) {
-                const float ca = c_t[ia + m], cb = c_t[ib + m];
-                acc = fmaf(ca, cb, acc);
-                if (DERIV) {
-                    ax = fmaf(D_t[ia + m], cb, fmaf(ca, D_t[ib + m], ax));
-                    ay = fmaf(D_t[CT + ia + m], cb, fmaf(ca, D_t[CT + ib + m], ay));
-                    az = fmaf(D_t[2 * CT + ia + m], cb, fmaf(ca, D_t[2 * CT + ib + m], az));
+        float* slab = smem + lay.sSD;
+        constexpr int NV = DERIV ? 4 : 1;                                   // values per feature
+        const int NP = F / L1;                                              // (species pair, n, n') groups
+        int gp = ((lay.total - lay.sSD) / NV) / L1;                         // groups per slab
+        gp = gp < 1 ? 1 : (gp > NP ? NP : gp);
+        const bool staged = (lay.total - lay.sSD) >= NV * L1 && !(SOAP_DEBUG_SKIP & 8);
+        for (int q0 = 0; q0 < ((SOAP_DEBUG_SKIP & 8) ? 0 : NP); q0 += gp) {
+            const int nq = min(gp, NP - q0), nf = nq * L1, f0 = q0 * L1;
+            for (int g = tid; g < nf; g += kThreads) {
+                const int l = g / nq, fl = (g - l * nq) * L1 + l;             // feature index inside the slab
+                const int pk = __ldg(p.feat_pack + f0 + fl);
+                const int n1 = pk & 31, n2 = (pk >> 5) & 31, mu = (pk >> 10) & 15, nu = (pk >> 14) & 15;
+                const int ia = (mu * NMAX + n1) * LMP + l * l, ib = (nu * NMAX + n2) * LMP + l * l;
+                const float kl = __ldg(p.kl + l);
+                float acc = 0.f, ax = 0.f, ay = 0.f, az = 0.f;
+                for (int m = 0; m <= 2 * l; ++m) {
+                    const float ca = c_t[ia + m], cb = c_t[ib + m];
+                    acc = fmaf(ca, cb, acc);
+                    if (DERIV) {
+                        ax = fmaf(D_t[ia + m], cb, fmaf(ca, D_t[ib + m], ax));
+                        ay = fmaf(D_t[CT + ia + m], cb, fmaf(ca, D_t[CT + ib + m], ay));
+                        az = fmaf(D_t[2 * CT + ia + m], cb, fmaf(ca, D_t[2 * CT + ib + m], az));
+                    }
+                }
+                if (staged) {
+                    slab[fl] = kl * acc;
+                    if (DERIV) { slab[nf + fl] = -kl * ax; slab[2 * nf + fl] = -kl * ay; slab[3 * nf + fl] = -kl * az; }
+                } else {
+                    desc_row[f0 + fl] = kl * acc;
+                    if (DERIV) { own[f0 + fl] = -kl * ax; own[(size_t)F + f0 + fl] = -kl * ay; own[(size_t)2 * F + f0 + fl] = -kl * az; }
                 }
             }
-            desc_row[f] = kl * acc;
-            if (DERIV) { own[f] = -kl * ax; own[(size_t)F + f] = -kl * ay; own[(size_t)2 * F + f] = -kl * az; }
+            if (staged) {
+                __syncthreads();
+                for (int e = tid; e < nf; e += kThreads) {
+                    desc_row[f0 + e] = slab[e];
+                    if (DERIV) {
+                        own[f0 + e] = slab[nf + e];
+                        own[(size_t)F + f0 + e] = slab[2 * nf + e];
+                        own[(size_t)2 * F + f0 + e] = slab[3 * nf + e];
+                    }
+                }
+                __syncthreads();
+            }
         }
         if (DERIV && tid == 0) p.row_atom[row_base + p.self_row[c_idx]] = ci;
     }
@@ -345,92 +382,65 @@ center_kernel(const CenterParams p) {
     const int NI = S * NCH, SN = S * NMAX;
     float4* wUV = reinterpret_cast<float4*>(smem + lay.wUV) + wid * NI;       // [nu][n'][l]
 
-    // product rule of one pair: stores the row (or adds to it when another image of the same atom
-    // already wrote it) and subtracts it from the centre's row
+    // Product rule of one pair (Eq. 5).  Lanes take consecutive features of the row in sweeps that
+    // are aligned to the row's start, so every warp store covers whole 32-byte sectors of each of the
+    // three direction planes (sectors written in two pieces halve the achievable write bandwidth).
+    // Feature (mu, nu, n1, n2, l) of a neighbour of species Z:
+    //   mu == Z:  G_{n1 l} V^nu_{n2 l} + Ghat_{n1 l} U^nu_{n2 l} d      (grad c^mu_{n1 l}) c^nu_{n2 l}
+    //   nu == Z:  G_{n2 l} V^mu_{n1 l} + Ghat_{n2 l} U^mu_{n1 l} d      c^mu_{n1 l} (grad c^nu_{n2 l})
+    // (both when mu == nu == Z, zero when neither).  Stores the row, or adds to it when another
+    // image of the same atom already wrote it.
     auto product_rule = [&](auto acc_tag, int Z, float4 d, const float2* wG, float* out) {
         constexpr bool ACC = decltype(acc_tag)::value;
-        float dbg_sink = 0.f;
-        auto emit = [&](float* o, float v) {
-            if (SOAP_DEBUG_SKIP & 32) { dbg_sink += v; return; }
-            if (ACC) *o += v; else *o = v;
+        const int F2 = 2 * F;
+        auto put = [&](int f, float vx, float vy, float vz) {
+            if (SOAP_DEBUG_SKIP & 128) vx = vy = vz = 1.f;
+            if (ACC) { out[f] += vx; out[F + f] += vy; out[F2 + f] += vz; }
+            else { out[f] = vx; out[F + f] = vy; out[F2 + f] = vz; }
         };
-        int boff = 0;
+        int lo = 0;
         for (int mu = 0; mu < S; ++mu) {
             for (int nu = mu; nu < S; ++nu) {
-                const int bsize = (mu == nu) ? (NMAX * (NMAX + 1) / 2) * L1 : NMAX * NCH;
-                float* ob = out + boff;
-                boff += bsize;
+                const int hi = lo + ((mu == nu) ? (NMAX * (NMAX + 1) / 2) * L1 : NMAX * NCH);
+                const int first = lo & ~31;
                 if (mu != Z && nu != Z) {
-                    if (!ACC && !(SOAP_DEBUG_SKIP & 64)) {
-                        float *o0 = ob + lane, *o1 = o0 + F, *o2 = o1 + F;
-                        for (int f = lane; f < bsize; f += 32) { *o0 = 0.f; *o1 = 0.f; *o2 = 0.f; o0 += 32; o1 += 32; o2 += 32; }
-                    }
+                    if (!ACC)
+                        for (int f = first + lane; f < hi; f += 32)
+                            if (f >= lo) put(f, 0.f, 0.f, 0.f);
                 } else if (mu == nu) {
-                    // both terms; feature (n1 <= n2, l) sits at L1 (n1 NMAX - n1(n1-1)/2) + (n2-n1) L1 + l
                     const float4* UVz = wUV + Z * NCH;
-                    for (int j0 = 0; j0 < NCH; j0 += 32) {
-                        const int j = j0 + lane;
-                        const bool live = j < NCH;
-                        const int jj = live ? j : 0;
-                        const int n2 = jj / L1, l = jj - n2 * L1;
-                        const float2 gj = wG[jj];
-                        const float4 uj = UVz[jj];
-                        const float2* g1p = wG + l;
-                        const float4* u1p = UVz + l;
-                        float *o0 = ob + jj, *o1 = o0 + F, *o2 = o1 + F;
-                        const int n1_hi = min(NMAX - 1, (j0 + 31) / L1);     // no lane of this round goes beyond
-#pragma unroll
-                        for (int n1 = 0; n1 < NMAX_BOUND; ++n1) {
-                            if (n1 > n1_hi) break;
-                            const int off = (n1 * NMAX - n1 * (n1 + 1) / 2) * L1;   // feature offset relative to n1 = 0
-                            if (live && n1 <= n2) {
-                                const float2 g1 = g1p[n1 * L1];
-                                const float4 u1 = u1p[n1 * L1];
-                                const float w = fmaf(g1.y, uj.x, gj.y * u1.x);    // Ghat_n1 U_n2 + Ghat_n2 U_n1
-                                emit(o0 + off, fmaf(g1.x, uj.y, fmaf(gj.x, u1.y, w * d.x)));
-                                emit(o1 + off, fmaf(g1.x, uj.z, fmaf(gj.x, u1.z, w * d.y)));
-                                emit(o2 + off, fmaf(g1.x, uj.w, fmaf(gj.x, u1.w, w * d.z)));
-                            }
-                        }
-                    }
-                } else if (mu == Z) {
-                    // (grad c^mu_{n1 l}) c^nu_{n2 l}: G_{n1 l} V^nu_{n2 l} + Ghat_{n1 l} d U^nu_{n2 l}
-                    for (int j = lane; j < NCH; j += 32) {
-                        const int l = j % L1;
-                        const float4 uj = wUV[nu * NCH + j];
-                        const float xx = uj.x * d.x, xy = uj.x * d.y, xz = uj.x * d.z;
-                        const float2* g1p = wG + l;
-                        float *o0 = ob + j, *o1 = o0 + F, *o2 = o1 + F;
-#pragma unroll
-                        for (int n1 = 0; n1 < NMAX_BOUND; ++n1) {
-                            if (n1 >= NMAX) break;
-                            const float2 g1 = g1p[n1 * L1];
-                            emit(o0 + n1 * NCH, fmaf(g1.x, uj.y, g1.y * xx));
-                            emit(o1 + n1 * NCH, fmaf(g1.x, uj.z, g1.y * xy));
-                            emit(o2 + n1 * NCH, fmaf(g1.x, uj.w, g1.y * xz));
-                        }
+#pragma unroll 2
+                    for (int f = first + lane; f < hi; f += 32) {
+                        if (f < lo) continue;
+                        const unsigned dec = tri_dec[f - lo];                 // (n1 L1 + l) | (n2 L1 + l) << 8
+                        const int iA = dec & 255, iB = dec >> 8;
+                        const float2 g1 = wG[iA], g2 = wG[iB];
+                        const float4 u1 = UVz[iA], u2 = UVz[iB];
+                        const float t = fmaf(g1.y, u2.x, g2.y * u1.x);      // Ghat_n1 U_n2 + Ghat_n2 U_n1
+                        put(f, fmaf(g1.x, u2.y, fmaf(g2.x, u1.y, t * d.x)), fmaf(g1.x, u2.z, fmaf(g2.x, u1.z, t * d.y)),
+                            fmaf(g1.x, u2.w, fmaf(g2.x, u1.w, t * d.z)));
                     }
                 } else {
-                    // c^mu_{n1 l} (grad c^nu_{n2 l}): G_{n2 l} V^mu_{n1 l} + Ghat_{n2 l} d U^mu_{n1 l}
-                    for (int j = lane; j < NCH; j += 32) {
-                        const int l = j % L1;
-                        const float2 gj = wG[j];
-                        const float gx = gj.y * d.x, gy = gj.y * d.y, gz = gj.y * d.z;
-                        const float4* u1p = wUV + mu * NCH + l;
-                        float *o0 = ob + j, *o1 = o0 + F, *o2 = o1 + F;
-#pragma unroll
-                        for (int n1 = 0; n1 < NMAX_BOUND; ++n1) {
-                            if (n1 >= NMAX) break;
-                            const float4 u1 = u1p[n1 * L1];
-                            emit(o0 + n1 * NCH, fmaf(gj.x, u1.y, gx * u1.x));
-                            emit(o1 + n1 * NCH, fmaf(gj.x, u1.z, gy * u1.x));
-                            emit(o2 + n1 * NCH, fmaf(gj.x, u1.w, gz * u1.x));
-                        }
+                    // block index e = n1 NCH + n2 L1 + l; the radial factor belongs to the neighbour's
+                    // species, U/V to the other one
+                    const bool first_term = (mu == Z);
+                    const float4* UVo = wUV + (first_term ? nu : mu) * NCH;
+#pragma unroll 2
+                    for (int f = first + lane; f < hi; f += 32) {
+                        if (f < lo) continue;
+                        const int e = f - lo;
+                        const int n1 = (int)__umulhi((unsigned)e, p.nch_magic);
+                        const int j = e - n1 * NCH;                           // n2 L1 + l
+                        const int i1 = n1 * L1 + (j % L1);                    // n1 L1 + l
+                        const float2 g = wG[first_term ? i1 : j];
+                        const float4 u = UVo[first_term ? j : i1];
+                        const float t = g.y * u.x;
+                        put(f, fmaf(g.x, u.y, t * d.x), fmaf(g.x, u.z, t * d.y), fmaf(g.x, u.w, t * d.z));
                     }
                 }
+                lo = hi;
             }
         }
-        if ((SOAP_DEBUG_SKIP & 32) && dbg_sink == 123.456f) out[lane] = dbg_sink;
     };
 
     // everything one warp does for one pair of the staged chunk

@@ -312,7 +312,7 @@ void fill_center_params(soap_t* h, CenterParams& cp, const float* pos, const int
     cp.pair_capacity = h->cap_pairs; cp.row_capacity = 0; cp.counters = h->d_counters;
     cp.table = h->d_table; cp.self_term = h->d_self; cp.anorm = h->d_anorm; cp.dfact = h->d_dfact; cp.kl = h->d_kl;
     cp.inv_int = h->d_inv_int; cp.lm_of_t = h->d_lm_of_t; cp.l_of_lm = h->d_l_of_lm;
-    cp.feat_pack = h->d_feat; cp.inv_h = (float)h->basis.inv_h; cp.n_intervals = h->basis.n_intervals;
+    cp.feat_pack = h->d_feat; cp.nch_magic = (unsigned)((1ull << 32) / (unsigned)(h->n_max * (h->l_max + 1))) + 1u; cp.inv_h = (float)h->basis.inv_h; cp.n_intervals = h->basis.n_intervals;
     cp.S = h->S; cp.n_max = h->n_max; cp.l_max = h->l_max; cp.F = (int)h->F;
     cp.P = deriv ? h->P_deriv : h->P_desc;
     cp.out_desc = nullptr; cp.out_jac = nullptr; cp.row_atom = nullptr;
@@ -353,8 +353,9 @@ int soap_create(soap_t** out, const int32_t* species, int n_species, double r_cu
         for (int nu = mu; nu < h->S; ++nu)
             for (int n = 0; n < n_max; ++n)
                 for (int n2 = (mu == nu ? n : 0); n2 < n_max; ++n2)
-                    for (int l = 0; l <= l_max; ++l)
+                    for (int l = 0; l <= l_max; ++l) {
                         h->feat_pack.push_back(n | (n2 << 5) | (mu << 10) | (nu << 14) | (l << 18));
+                    }
     h->F = (int64_t)h->feat_pack.size();
     *out = h;
     return SOAP_OK;

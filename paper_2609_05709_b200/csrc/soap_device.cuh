@@ -76,6 +76,7 @@ struct CenterParams {
     int n_intervals;
     int S, n_max, l_max, F;
     int P;                        // pairs per staged chunk (<= 32)
+    unsigned nch_magic;           // floor(2^32 / (n_max (l_max+1))) + 1: x / n_ch == umulhi(x, magic) for x < 65536
     // outputs
     float* out_desc;              // [C,F]
     float* out_jac;               // [rows,3,F]
@@ -96,7 +97,7 @@ __host__ __device__ inline void key_shift(unsigned long long k, int s[3]) {
 constexpr int kGeoPairs = 128;           // pairs whose geometry is staged at once
 
 struct SmemLayout {
-    int c, geo, D, wUV, sSD, sG, total;
+    int c, geo, tri, D, wUV, sSD, sG, total;
 };
 __host__ __device__ inline int align4(int x) { return (x + 3) & ~3; }
 __host__ __device__ inline SmemLayout make_layout(int S, int n_max, int l_max, int P, bool deriv) {
@@ -105,6 +106,7 @@ __host__ __device__ inline SmemLayout make_layout(int S, int n_max, int l_max, i
     int off = 0;
     o.c = off; off = align4(off + CT);
     o.geo = off; off = align4(off + kGeoPairs * 9 + (kMaxSpecies + 1) + (kGeoPairs / 32) * kMaxSpecies);   // + species segments
+    o.tri = off; if (deriv) off = align4(off + ((n_max * (n_max + 1) / 2) * L1 + 1) / 2);   // 16-bit entries
     // the D tiles (pass 1, centre's row) and the per-warp U/V staging (pass 2) never live
     // at the same time and share space
     o.D = off; o.wUV = off;
