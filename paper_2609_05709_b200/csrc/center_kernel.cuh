@@ -420,6 +420,52 @@ center_kernel(const CenterParams p) {
                         put(f, fmaf(g1.x, u2.y, fmaf(g2.x, u1.y, t * d.x)), fmaf(g1.x, u2.z, fmaf(g2.x, u1.z, t * d.y)),
                             fmaf(g1.x, u2.w, fmaf(g2.x, u1.w, t * d.z)));
                     }
+                } else if ((NCH & 7) == 0) {
+                    // Cross-species block, n_ch a multiple of 8: rows n1 of n_ch floats follow each other, so
+                    // windows of n_ch floats that start `shift` floats before a row start are sector-aligned
+                    // for every n1.  A lane keeps one window position i: its (n2, l) = i - shift (mod n_ch)
+                    // is fixed, so the operand that depends on (n2, l) stays in registers over the n1 loop;
+                    // the lanes in front of the row start (i < shift) serve the tail of the previous row.
+                    const bool first_term = (mu == Z);
+                    const float4* UVo = wUV + (first_term ? nu : mu) * NCH;
+                    const int shift = lo & 7;
+                    for (int i0 = 0; i0 < NCH; i0 += 32) {
+                        const int i = i0 + lane;
+                        if (i >= NCH) break;
+                        const bool prev = i < shift;                          // belongs to row n1 - 1
+                        const int j = prev ? i - shift + NCH : i - shift;      // n2 L1 + l
+                        const int l = j % L1;
+                        float* o = out + (lo - shift + i);
+                        if (first_term) {
+                            const float4 u = UVo[j];
+                            const float xx = u.x * d.x, xy = u.x * d.y, xz = u.x * d.z;
+                            const float2* gp = wG + l - (prev ? L1 : 0);
+#pragma unroll
+                            for (int n1 = 0; n1 <= NMAX_BOUND; ++n1) {
+                                if (n1 > NMAX) break;
+                                if (prev ? (n1 >= 1) : (n1 < NMAX)) {
+                                    const float2 g = gp[n1 * L1];
+                                    const float vx = fmaf(g.x, u.y, g.y * xx), vy = fmaf(g.x, u.z, g.y * xy), vz = fmaf(g.x, u.w, g.y * xz);
+                                    if (ACC) { o[n1 * NCH] += vx; o[F + n1 * NCH] += vy; o[F2 + n1 * NCH] += vz; }
+                                    else { o[n1 * NCH] = vx; o[F + n1 * NCH] = vy; o[F2 + n1 * NCH] = vz; }
+                                }
+                            }
+                        } else {
+                            const float2 g = wG[j];
+                            const float gx = g.y * d.x, gy = g.y * d.y, gz = g.y * d.z;
+                            const float4* up = UVo + l - (prev ? L1 : 0);
+#pragma unroll
+                            for (int n1 = 0; n1 <= NMAX_BOUND; ++n1) {
+                                if (n1 > NMAX) break;
+                                if (prev ? (n1 >= 1) : (n1 < NMAX)) {
+                                    const float4 u = up[n1 * L1];
+                                    const float vx = fmaf(g.x, u.y, gx * u.x), vy = fmaf(g.x, u.z, gy * u.x), vz = fmaf(g.x, u.w, gz * u.x);
+                                    if (ACC) { o[n1 * NCH] += vx; o[F + n1 * NCH] += vy; o[F2 + n1 * NCH] += vz; }
+                                    else { o[n1 * NCH] = vx; o[F + n1 * NCH] = vy; o[F2 + n1 * NCH] = vz; }
+                                }
+                            }
+                        }
+                    }
                 } else {
                     // block index e = n1 NCH + n2 L1 + l; the radial factor belongs to the neighbour's
                     // species, U/V to the other one
