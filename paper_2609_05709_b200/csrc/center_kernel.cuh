@@ -112,7 +112,7 @@ center_kernel(const CenterParams p) {
     constexpr int NPT = NPT_RAW < 8 ? NPT_RAW : 8;                // ... at most 8 at a time (register budget)
     extern __shared__ __align__(16) float smem[];
     const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
-    const long long c_idx = blockIdx.x;
+    const long long c_idx = p.order ? p.order[blockIdx.x] : blockIdx.x;
     // a failed neighbour build or an undersized output: write nothing
     if (p.pair_ptr[p.n_centers] > p.pair_capacity) return;
     if (DERIV && p.row_ptr[p.n_centers] > p.row_capacity) {

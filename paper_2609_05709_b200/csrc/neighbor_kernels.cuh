@@ -250,11 +250,16 @@ __device__ inline void for_each_candidate(const Geometry& geom, const GridParams
     }
 }
 
+// Centres are handed to the per-centre kernel largest first (their CTAs differ in length by the
+// number of pairs): a histogram of pair counts in bins of 4, filled while counting, gives every
+// centre a slot.  Only used for moderate numbers of centres (the bins are global atomics).
+constexpr int kSizeBins = 256, kSizeBinShift = 2;
+
 // One warp per centre: number of pairs.
 __global__ void count_kernel(const float* __restrict__ pos, const int* __restrict__ centers, long long C, Geometry geom,
                              const GridParams* __restrict__ gp, const int* __restrict__ atom_cell, const int* __restrict__ atom_wrap,
                              const int* __restrict__ cell_start, const float4* __restrict__ s_pos, const int* __restrict__ s_wrap,
-                             int* __restrict__ pair_count, Counters* counters) {
+                             int* __restrict__ pair_count, int* size_hist, Counters* counters) {
     const GridParams g = *gp;
     const int lane = threadIdx.x & 31;
     const long long c = blockIdx.x * (long long)(blockDim.x >> 5) + (threadIdx.x >> 5);
@@ -270,7 +275,10 @@ __global__ void count_kernel(const float* __restrict__ pos, const int* __restric
     int cnt = 0;
     for_each_candidate(geom, g, cell_start, s_pos, s_wrap, xi, yi, zi, bi, wi, lane, counters,
                        [&](bool valid, unsigned long long) { cnt += __popc(__ballot_sync(0xffffffffu, valid)); });
-    if (lane == 0) pair_count[c] = cnt;
+    if (lane == 0) {
+        pair_count[c] = cnt;
+        if (size_hist) atomicAdd(&size_hist[min(cnt >> kSizeBinShift, kSizeBins - 1)], 1);
+    }
 }
 
 constexpr int kFillSmemKeys = 512;       // per warp; longer rows are sorted through global memory
@@ -284,7 +292,8 @@ fill_kernel(const float* __restrict__ pos, const int* __restrict__ centers, long
             const int* __restrict__ cell_start, const float4* __restrict__ s_pos, const int* __restrict__ s_wrap,
             const long long* __restrict__ pair_ptr, long long pair_capacity,
             unsigned long long* pair_tmp, unsigned long long* pair_key, int* __restrict__ pair_row,
-            int* __restrict__ row_count, int* __restrict__ self_row, Counters* counters) {
+            int* __restrict__ row_count, int* __restrict__ self_row, const int* size_hist, int* size_cursor,
+            int* __restrict__ order, Counters* counters) {
     __shared__ unsigned long long s_raw[kFillWarps][kFillSmemKeys];
     __shared__ unsigned long long s_sorted[kFillWarps][kFillSmemKeys];
     const GridParams g = *gp;
@@ -306,6 +315,14 @@ fill_kernel(const float* __restrict__ pos, const int* __restrict__ centers, long
     }
     const long long base = pair_ptr[c];
     const int k = (int)(pair_ptr[c + 1] - base);
+    if (order) {
+        // slot = number of centres in larger bins + arrival number inside the own bin
+        const int bin = min(k >> kSizeBinShift, kSizeBins - 1);
+        int larger = 0;
+        for (int b = bin + 1 + lane; b < kSizeBins; b += 32) larger += size_hist[b];
+        for (int o = 16; o > 0; o >>= 1) larger += __shfl_xor_sync(0xffffffffu, larger, o);
+        if (lane == 0) order[larger + atomicAdd(&size_cursor[bin], 1)] = (int)c;
+    }
     const bool in_smem = k <= kFillSmemKeys;
     volatile unsigned long long* raw = in_smem ? s_raw[wid] : pair_tmp + base;
     volatile unsigned long long* sorted = in_smem ? s_sorted[wid] : pair_key + base;

@@ -60,7 +60,8 @@ struct soap_handle {
     float *d_table = nullptr, *d_self = nullptr, *d_anorm = nullptr, *d_dfact = nullptr, *d_kl = nullptr, *d_inv_int = nullptr;
     int *d_feat = nullptr, *d_zlut = nullptr, *d_lm_of_t = nullptr, *d_l_of_lm = nullptr;
     Counters* d_counters = nullptr;
-    unsigned long long* d_bbox = nullptr;
+    unsigned long long* d_bbox = nullptr;   // 6 words of bounding box, then the size histogram and its cursors
+    int *d_size_hist = nullptr, *d_size_cursor = nullptr, *d_order = nullptr;
     GridParams* d_grid = nullptr;
     Counters* h_counters = nullptr;      // pinned
     // scratch, grown on demand
@@ -83,6 +84,8 @@ struct soap_handle {
 };
 
 namespace {
+
+constexpr int64_t kOrderMaxCenters = 65536;   // above this the CTAs simply run in centre order
 
 int fail(soap_t* h, int code, const std::string& msg) {
     if (h) h->error = msg;
@@ -172,7 +175,9 @@ int ensure_device(soap_t* h) {
     CU(upload(&h->d_zlut, lut));
     CU(cudaMalloc((void**)&h->d_counters, sizeof(Counters)));
     CU(cudaMemset(h->d_counters, 0, sizeof(Counters)));
-    CU(cudaMalloc((void**)&h->d_bbox, 6 * sizeof(unsigned long long)));
+    CU(cudaMalloc((void**)&h->d_bbox, 64 + 2 * kSizeBins * sizeof(int)));
+    h->d_size_hist = reinterpret_cast<int*>(reinterpret_cast<char*>(h->d_bbox) + 64);
+    h->d_size_cursor = h->d_size_hist + kSizeBins;
     CU(cudaMalloc((void**)&h->d_grid, sizeof(GridParams)));
     CU(cudaMallocHost((void**)&h->h_counters, sizeof(Counters)));
     // shared-memory plan of the per-centre kernels
@@ -233,6 +238,7 @@ int ensure_scratch(soap_t* h, int64_t N, int64_t C, int64_t pairs) {
         CU(regrow(&h->d_pair_count, cap));
         CU(regrow(&h->d_row_count, cap));
         CU(regrow(&h->d_self_row, cap));
+        CU(regrow(&h->d_order, cap));
         CU(regrow(&h->d_pair_ptr, cap + 1));
         CU(regrow(&h->d_row_ptr, cap + 1));
         h->cap_centers = cap;
@@ -254,14 +260,15 @@ int blocks_for(int64_t n, int threads, int cap = 4096) {
 // Cell list and pair counts: everything up to the scan of the per-centre counts.
 int launch_count(soap_t* h, const float* pos, const int32_t* num, int64_t N, const Geometry& g,
                  const int32_t* centers, int64_t C, cudaStream_t st) {
-    CU(cudaMemsetAsync(h->d_bbox, 0, 6 * sizeof(unsigned long long), st));
+    CU(cudaMemsetAsync(h->d_bbox, 0, 64 + 2 * kSizeBins * sizeof(int), st));
     CU(cudaMemsetAsync(h->d_cell_count, 0, (h->cap_cells + 1) * sizeof(int), st));
     if (N > 0) species_bbox_kernel<<<blocks_for(N, 256, 1024), 256, 0, st>>>(pos, num, N, g, h->d_zlut, h->d_species_idx, h->d_bbox, h->d_counters);
     grid_setup_kernel<<<1, 1, 0, st>>>(h->d_bbox, g, N, (int)h->cap_cells, h->d_grid);
     if (N > 0) bin_count_kernel<<<blocks_for(N, 256), 256, 0, st>>>(pos, N, g, h->d_grid, h->d_atom_cell, h->d_atom_wrap, h->d_cell_count, h->d_counters);
     scan_kernel<int><<<1, 1024, 0, st>>>(h->d_cell_count, h->d_cell_start, h->cap_cells, nullptr);
     if (N > 0) bin_fill_kernel<<<blocks_for(N, 256), 256, 0, st>>>(pos, N, h->d_atom_cell, h->d_atom_wrap, h->d_cell_start, h->d_cell_count, h->d_s_pos, h->d_s_wrap);
-    if (C > 0) count_kernel<<<(unsigned)((C + 7) / 8), 256, 0, st>>>(pos, centers, C, g, h->d_grid, h->d_atom_cell, h->d_atom_wrap, h->d_cell_start, h->d_s_pos, h->d_s_wrap, h->d_pair_count, h->d_counters);
+    if (C > 0) count_kernel<<<(unsigned)((C + 7) / 8), 256, 0, st>>>(pos, centers, C, g, h->d_grid, h->d_atom_cell, h->d_atom_wrap, h->d_cell_start, h->d_s_pos, h->d_s_wrap, h->d_pair_count,
+                                                                              C <= kOrderMaxCenters ? h->d_size_hist : nullptr, h->d_counters);
     scan_kernel<long long><<<1, 1024, 0, st>>>(h->d_pair_count, h->d_pair_ptr, C, &h->d_counters->n_pairs);
     CU(cudaGetLastError());
     return SOAP_OK;
@@ -272,7 +279,8 @@ int launch_fill(soap_t* h, const float* pos, const Geometry& g, const int32_t* c
                 long long* row_ptr_out, cudaStream_t st) {
     if (C > 0) fill_kernel<<<(unsigned)((C + kFillWarps - 1) / kFillWarps), kFillWarps * 32, 0, st>>>(
         pos, centers, C, g, h->d_grid, h->d_atom_cell, h->d_atom_wrap, h->d_cell_start, h->d_s_pos, h->d_s_wrap,
-        h->d_pair_ptr, h->cap_pairs, h->d_pair_tmp, h->d_pair_key, h->d_pair_row, h->d_row_count, h->d_self_row, h->d_counters);
+        h->d_pair_ptr, h->cap_pairs, h->d_pair_tmp, h->d_pair_key, h->d_pair_row, h->d_row_count, h->d_self_row,
+        h->d_size_hist, h->d_size_cursor, C <= kOrderMaxCenters ? h->d_order : nullptr, h->d_counters);
     scan_kernel<long long><<<1, 1024, 0, st>>>(h->d_row_count, row_ptr_out, C, &h->d_counters->n_rows);
     CU(cudaGetLastError());
     return SOAP_OK;
@@ -306,7 +314,7 @@ int plan(soap_t* h, const float* pos, const int32_t* num, int64_t N, const Geome
 
 void fill_center_params(soap_t* h, CenterParams& cp, const float* pos, const int32_t* centers, int64_t C,
                         const Geometry& g, bool deriv) {
-    cp.pos = pos; cp.centers = centers; cp.species_idx = h->d_species_idx; cp.n_centers = C; cp.geom = g;
+    cp.pos = pos; cp.centers = centers; cp.order = C <= kOrderMaxCenters ? h->d_order : nullptr; cp.species_idx = h->d_species_idx; cp.n_centers = C; cp.geom = g;
     cp.pair_ptr = h->d_pair_ptr; cp.pair_key = h->d_pair_key; cp.pair_row = h->d_pair_row;
     cp.row_ptr = h->d_row_ptr; cp.self_row = h->d_self_row;
     cp.pair_capacity = h->cap_pairs; cp.row_capacity = 0; cp.counters = h->d_counters;
@@ -365,7 +373,7 @@ void soap_destroy(soap_t* h) {
     if (!h) return;
     void* ptrs[] = {h->d_table, h->d_self, h->d_anorm, h->d_dfact, h->d_kl, h->d_feat, h->d_zlut, h->d_inv_int, h->d_lm_of_t, h->d_l_of_lm, h->d_counters, h->d_bbox,
                     h->d_grid, h->d_species_idx, h->d_atom_cell, h->d_atom_wrap, h->d_s_wrap, h->d_s_pos, h->d_cell_count,
-                    h->d_cell_start, h->d_pair_count, h->d_row_count, h->d_self_row, h->d_pair_ptr, h->d_row_ptr,
+                    h->d_cell_start, h->d_pair_count, h->d_row_count, h->d_self_row, h->d_order, h->d_pair_ptr, h->d_row_ptr,
                     h->d_pair_key, h->d_pair_tmp, h->d_pair_row};
     for (void* p : ptrs) if (p) cudaFree(p);
     if (h->h_counters) cudaFreeHost(h->h_counters);
@@ -601,7 +609,7 @@ int soap_neighbor_counts_static(const float* d_positions, int64_t n_atoms, doubl
     scan_kernel<int><<<1, 1024, 0, st>>>(cell_count, cell_start, kStaticMaxCells, nullptr);
     bin_fill_kernel<<<blocks_for(N, 256), 256, 0, st>>>(d_positions, N, atom_cell, atom_wrap, cell_start, cell_count, s_pos, s_wrap);
     count_kernel<<<(unsigned)((N + 7) / 8), 256, 0, st>>>(d_positions, nullptr, N, g, grid, atom_cell, atom_wrap, cell_start, s_pos, s_wrap,
-                                                         d_counts, counters);
+                                                         d_counts, nullptr, counters);
     if ((e = cudaGetLastError()) != cudaSuccess) return say(SOAP_ERR_CUDA, cudaGetErrorString(e));
     return SOAP_OK;
 }

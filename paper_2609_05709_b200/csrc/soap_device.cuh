@@ -51,6 +51,7 @@ struct CenterParams {
     // structure
     const float* pos;             // [N,3]
     const int* centers;           // [C] or null
+    const int* order;             // [C] CTA -> centre slot (largest first) or null
     const int* species_idx;       // [N]
     long long n_centers;
     Geometry geom;
