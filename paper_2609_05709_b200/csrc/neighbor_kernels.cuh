@@ -136,7 +136,9 @@ __global__ void bin_count_kernel(const float* __restrict__ pos, long long N, Geo
 
 // Exclusive scan by ONE block (n is at most a few million here); out[n] = total.
 template <typename OutT>
-__global__ void scan_kernel(const int* __restrict__ in, OutT* __restrict__ out, long long n, long long* total_out) {
+__global__ void scan_kernel(const int* __restrict__ in, OutT* __restrict__ out, long long n, long long* total_out,
+                            const int* n_dev = nullptr) {
+    if (n_dev) n = min(n, (long long)*n_dev);          // only the bins the grid really uses
     __shared__ long long warp_sums[32];
     __shared__ long long carry_s;
     if (threadIdx.x == 0) carry_s = 0;
@@ -193,59 +195,86 @@ __device__ inline void wrap_bin(int b, int nb, int& cell, int& image) {
 // Calls f(valid, key) for every lane in lock step, over all candidates of one centre.
 // key encodes (atom, lattice translation on the raw inputs); valid says whether this
 // lane holds a pair inside the cutoff.
+// The stencil is walked 32 bins at a time: each lane fetches the atom range of one bin (a single
+// memory round trip for all of them), a warp scan turns the counts into offsets, and the lanes
+// then run over the concatenated candidates, so they stay busy whatever the bin occupancy.
 template <class F>
 __device__ inline void for_each_candidate(const Geometry& geom, const GridParams& g, const int* __restrict__ cell_start,
                                           const float4* __restrict__ s_pos, const int* __restrict__ s_wrap,
                                           float xi, float yi, float zi, const int bi[3], const int wi[3],
                                           int lane, Counters* counters, F f) {
-    for (int oz = -g.R[2]; oz <= g.R[2]; ++oz) {
-        int cz, iz;
-        if (g.periodic[2]) wrap_bin(bi[2] + oz, g.nb[2], cz, iz);
-        else { cz = bi[2] + oz; iz = 0; if (cz < 0 || cz >= g.nb[2]) continue; }
-        for (int oy = -g.R[1]; oy <= g.R[1]; ++oy) {
-            int cy, iy;
-            if (g.periodic[1]) wrap_bin(bi[1] + oy, g.nb[1], cy, iy);
-            else { cy = bi[1] + oy; iy = 0; if (cy < 0 || cy >= g.nb[1]) continue; }
-            for (int ox = -g.R[0]; ox <= g.R[0]; ++ox) {
-                int cx, ix;
-                if (g.periodic[0]) wrap_bin(bi[0] + ox, g.nb[0], cx, ix);
-                else { cx = bi[0] + ox; ix = 0; if (cx < 0 || cx >= g.nb[0]) continue; }
-                const int cell = (cz * g.nb[1] + cy) * g.nb[0] + cx;
-                const int start = cell_start[cell], end = cell_start[cell + 1];
-                for (int t0 = start; t0 < end; t0 += 32) {
-                    const int t = t0 + lane;
-                    bool valid = false;
-                    unsigned long long key = 0;
-                    if (t < end) {
-                        const float4 pj = s_pos[t];
-                        int wj[3];
-                        unpack3(s_wrap[t], wj);
-                        // translation on the raw (unwrapped) inputs
-                        const int na = ix - wj[0] + wi[0], nb = iy - wj[1] + wi[1], nc = iz - wj[2] + wi[2];
-                        double dx = __dsub_rn((double)pj.x, (double)xi);
-                        double dy = __dsub_rn((double)pj.y, (double)yi);
-                        double dz = __dsub_rn((double)pj.z, (double)zi);
-                        if (g.periodic[0] | g.periodic[1] | g.periodic[2]) {
-                            // T = (n_a a + n_b b) + n_c c, each product and sum rounded on its own
-                            const double fa = (double)na, fb = (double)nb, fc = (double)nc;
-                            double tx = __dadd_rn(__dadd_rn(__dmul_rn(fa, geom.cell[0]), __dmul_rn(fb, geom.cell[3])), __dmul_rn(fc, geom.cell[6]));
-                            double ty = __dadd_rn(__dadd_rn(__dmul_rn(fa, geom.cell[1]), __dmul_rn(fb, geom.cell[4])), __dmul_rn(fc, geom.cell[7]));
-                            double tz = __dadd_rn(__dadd_rn(__dmul_rn(fa, geom.cell[2]), __dmul_rn(fb, geom.cell[5])), __dmul_rn(fc, geom.cell[8]));
-                            dx = __dadd_rn(dx, tx); dy = __dadd_rn(dy, ty); dz = __dadd_rn(dz, tz);
-                        }
-                        const double d2 = __dadd_rn(__dadd_rn(__dmul_rn(dx, dx), __dmul_rn(dy, dy)), __dmul_rn(dz, dz));
-                        valid = (d2 < geom.rc2) && (d2 > 0.0);
-                        if (valid && (abs(na) > 127 || abs(nb) > 127 || abs(nc) > 127)) {
-                            atomicOr(&counters->status, kStatusShiftRange);
-                            valid = false;
-                        }
-                        key = ((unsigned long long)(unsigned)__float_as_int(pj.w) << 24) |
-                              ((unsigned long long)(na + 128) << 16) | ((unsigned long long)(nb + 128) << 8) |
-                              (unsigned long long)(nc + 128);
-                    }
-                    f(valid, key);
-                }
+    const int w0 = 2 * g.R[0] + 1, w1 = 2 * g.R[1] + 1, w2 = 2 * g.R[2] + 1;
+    const int n_stencil = w0 * w1 * w2;
+    const bool any_periodic = g.periodic[0] | g.periodic[1] | g.periodic[2];
+    for (int q0 = 0; q0 < n_stencil; q0 += 32) {
+        // ---- this lane's bin of the stencil ----
+        const int q = q0 + lane;
+        int start = 0, cnt = 0, img = 0;                  // img: packed image of the bin (periodic axes)
+        if (q < n_stencil) {
+            int o[3] = {q % w0 - g.R[0], (q / w0) % w1 - g.R[1], q / (w0 * w1) - g.R[2]};
+            int c[3], im[3];
+            bool inside = true;
+            for (int a = 0; a < 3; ++a) {
+                if (g.periodic[a]) wrap_bin(bi[a] + o[a], g.nb[a], c[a], im[a]);
+                else { c[a] = bi[a] + o[a]; im[a] = 0; inside &= (c[a] >= 0 && c[a] < g.nb[a]); }
             }
+            if (inside) {
+                const int cell = (c[2] * g.nb[1] + c[1]) * g.nb[0] + c[0];
+                start = cell_start[cell];
+                cnt = cell_start[cell + 1] - start;
+                img = pack3(im);
+            }
+        }
+        // ---- offsets of the bins in the concatenated candidate list ----
+        int incl = cnt;
+        for (int d = 1; d < 32; d <<= 1) {
+            const int y = __shfl_up_sync(0xffffffffu, incl, d);
+            if (lane >= d) incl += y;
+        }
+        const int total = __shfl_sync(0xffffffffu, incl, 31);
+        for (int t0 = 0; t0 < total; t0 += 32) {
+            const int t = t0 + lane;
+            // bin of candidate t: the first lane whose inclusive offset exceeds t (binary search by shuffles)
+            int lo = 0;
+            for (int step = 16; step > 0; step >>= 1) {
+                const int probe = __shfl_sync(0xffffffffu, incl, lo + step - 1);
+                if (probe <= t) lo += step;
+            }
+            lo = min(lo, 31);
+            const int b_incl = __shfl_sync(0xffffffffu, incl, lo), b_cnt = __shfl_sync(0xffffffffu, cnt, lo);
+            const int b_start = __shfl_sync(0xffffffffu, start, lo), b_img = __shfl_sync(0xffffffffu, img, lo);
+            bool valid = false;
+            unsigned long long key = 0;
+            if (t < total) {
+                const int at = b_start + (t - (b_incl - b_cnt));
+                const float4 pj = s_pos[at];
+                int wj[3], im[3];
+                unpack3(s_wrap[at], wj);
+                unpack3(b_img, im);
+                // translation on the raw (unwrapped) inputs
+                const int na = im[0] - wj[0] + wi[0], nb = im[1] - wj[1] + wi[1], nc = im[2] - wj[2] + wi[2];
+                double dx = __dsub_rn((double)pj.x, (double)xi);
+                double dy = __dsub_rn((double)pj.y, (double)yi);
+                double dz = __dsub_rn((double)pj.z, (double)zi);
+                if (any_periodic) {
+                    // T = (n_a a + n_b b) + n_c c, each product and sum rounded on its own
+                    const double fa = (double)na, fb = (double)nb, fc = (double)nc;
+                    double tx = __dadd_rn(__dadd_rn(__dmul_rn(fa, geom.cell[0]), __dmul_rn(fb, geom.cell[3])), __dmul_rn(fc, geom.cell[6]));
+                    double ty = __dadd_rn(__dadd_rn(__dmul_rn(fa, geom.cell[1]), __dmul_rn(fb, geom.cell[4])), __dmul_rn(fc, geom.cell[7]));
+                    double tz = __dadd_rn(__dadd_rn(__dmul_rn(fa, geom.cell[2]), __dmul_rn(fb, geom.cell[5])), __dmul_rn(fc, geom.cell[8]));
+                    dx = __dadd_rn(dx, tx); dy = __dadd_rn(dy, ty); dz = __dadd_rn(dz, tz);
+                }
+                const double d2 = __dadd_rn(__dadd_rn(__dmul_rn(dx, dx), __dmul_rn(dy, dy)), __dmul_rn(dz, dz));
+                valid = (d2 < geom.rc2) && (d2 > 0.0);
+                if (valid && (abs(na) > 127 || abs(nb) > 127 || abs(nc) > 127)) {
+                    atomicOr(&counters->status, kStatusShiftRange);
+                    valid = false;
+                }
+                key = ((unsigned long long)(unsigned)__float_as_int(pj.w) << 24) |
+                      ((unsigned long long)(na + 128) << 16) | ((unsigned long long)(nb + 128) << 8) |
+                      (unsigned long long)(nc + 128);
+            }
+            f(valid, key);
         }
     }
 }

@@ -265,7 +265,7 @@ int launch_count(soap_t* h, const float* pos, const int32_t* num, int64_t N, con
     if (N > 0) species_bbox_kernel<<<blocks_for(N, 256, 1024), 256, 0, st>>>(pos, num, N, g, h->d_zlut, h->d_species_idx, h->d_bbox, h->d_counters);
     grid_setup_kernel<<<1, 1, 0, st>>>(h->d_bbox, g, N, (int)h->cap_cells, h->d_grid);
     if (N > 0) bin_count_kernel<<<blocks_for(N, 256), 256, 0, st>>>(pos, N, g, h->d_grid, h->d_atom_cell, h->d_atom_wrap, h->d_cell_count, h->d_counters);
-    scan_kernel<int><<<1, 1024, 0, st>>>(h->d_cell_count, h->d_cell_start, h->cap_cells, nullptr);
+    scan_kernel<int><<<1, 1024, 0, st>>>(h->d_cell_count, h->d_cell_start, h->cap_cells, nullptr, &h->d_grid->n_cells);
     if (N > 0) bin_fill_kernel<<<blocks_for(N, 256), 256, 0, st>>>(pos, N, h->d_atom_cell, h->d_atom_wrap, h->d_cell_start, h->d_cell_count, h->d_s_pos, h->d_s_wrap);
     if (C > 0) count_kernel<<<(unsigned)((C + 7) / 8), 256, 0, st>>>(pos, centers, C, g, h->d_grid, h->d_atom_cell, h->d_atom_wrap, h->d_cell_start, h->d_s_pos, h->d_s_wrap, h->d_pair_count,
                                                                               C <= kOrderMaxCenters ? h->d_size_hist : nullptr, h->d_counters);
@@ -606,7 +606,7 @@ int soap_neighbor_counts_static(const float* d_positions, int64_t n_atoms, doubl
     bbox_only_kernel<<<blocks_for(N, 256, 256), 256, 0, st>>>(d_positions, N, g, bbox);
     grid_setup_kernel<<<1, 1, 0, st>>>(bbox, g, N, kStaticMaxCells, grid);
     bin_count_kernel<<<blocks_for(N, 256), 256, 0, st>>>(d_positions, N, g, grid, atom_cell, atom_wrap, cell_count, counters);
-    scan_kernel<int><<<1, 1024, 0, st>>>(cell_count, cell_start, kStaticMaxCells, nullptr);
+    scan_kernel<int><<<1, 1024, 0, st>>>(cell_count, cell_start, kStaticMaxCells, nullptr, &grid->n_cells);
     bin_fill_kernel<<<blocks_for(N, 256), 256, 0, st>>>(d_positions, N, atom_cell, atom_wrap, cell_start, cell_count, s_pos, s_wrap);
     count_kernel<<<(unsigned)((N + 7) / 8), 256, 0, st>>>(d_positions, nullptr, N, g, grid, atom_cell, atom_wrap, cell_start, s_pos, s_wrap,
                                                          d_counts, nullptr, counters);
