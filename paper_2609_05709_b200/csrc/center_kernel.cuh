@@ -393,6 +393,9 @@ center_kernel(const CenterParams p) {
     auto product_rule = [&](auto acc_tag, int Z, float4 d, const float2* wG, float* out) {
         constexpr bool ACC = decltype(acc_tag)::value;
         const int F2 = 2 * F;
+        // position of the row start inside a 128-byte line, in floats: sweeps start on line boundaries
+        // where the row allows it (a warp store that straddles two lines costs two L1 wavefronts)
+        const int a_line = (int)((reinterpret_cast<size_t>(out) >> 2) & 31);
         auto put = [&](int f, float vx, float vy, float vz) {
             if (SOAP_DEBUG_SKIP & 128) vx = vy = vz = 1.f;
             if (ACC) { out[f] += vx; out[F + f] += vy; out[F2 + f] += vz; }
@@ -402,7 +405,7 @@ center_kernel(const CenterParams p) {
         for (int mu = 0; mu < S; ++mu) {
             for (int nu = mu; nu < S; ++nu) {
                 const int hi = lo + ((mu == nu) ? (NMAX * (NMAX + 1) / 2) * L1 : NMAX * NCH);
-                const int first = lo & ~31;
+                const int first = ((lo + a_line) & ~31) - a_line;
                 if (mu != Z && nu != Z) {
                     if (!ACC)
                         for (int f = first + lane; f < hi; f += 32)
