@@ -61,7 +61,7 @@ __global__ void species_bbox_kernel(const float* __restrict__ pos, const int* __
 // cell faces) is at least r_cut (1 + 1e-6) wherever more than one bin fits, so a
 // stencil of +-1 bin covers the sphere; short periodic axes get one bin and a
 // wider stencil of images.
-__global__ void grid_setup_kernel(const unsigned long long* bbox, Geometry geom, long long N, int cell_cap, GridParams* out) {
+__device__ inline GridParams choose_grid(const double hi_in[3], const double lo_in[3], const Geometry& geom, long long N, int cell_cap) {
     GridParams g;
     const double rc = geom.r_cut * (1.0 + 1e-6);
     double want[3];
@@ -71,7 +71,7 @@ __global__ void grid_setup_kernel(const unsigned long long* bbox, Geometry geom,
             g.smin[a] = 0.0;
             want[a] = floor(geom.height[a] / rc);
         } else {
-            double hi = N > 0 ? dec_double(bbox[a]) : 0.0, lo = N > 0 ? -dec_double(bbox[3 + a]) : 0.0;
+            double hi = N > 0 ? hi_in[a] : 0.0, lo = N > 0 ? lo_in[a] : 0.0;
             g.smin[a] = lo;
             want[a] = floor((hi - lo) * geom.height[a] / rc);
         }
@@ -88,14 +88,20 @@ __global__ void grid_setup_kernel(const unsigned long long* bbox, Geometry geom,
             double width = geom.height[a] / g.nb[a];
             g.R[a] = (int)ceil(rc / width);
         } else {
-            double hi = N > 0 ? dec_double(bbox[a]) : 0.0;
+            double hi = N > 0 ? hi_in[a] : 0.0;
             double span = hi - g.smin[a];
             g.sscale[a] = span > 0 ? g.nb[a] / span : 0.0;
             g.R[a] = g.nb[a] > 1 ? 1 : 0;
         }
     }
     g.n_cells = g.nb[0] * g.nb[1] * g.nb[2];
-    *out = g;
+    return g;
+}
+
+__global__ void grid_setup_kernel(const unsigned long long* bbox, Geometry geom, long long N, int cell_cap, GridParams* out) {
+    double hi[3], lo[3];
+    for (int a = 0; a < 3; ++a) { hi[a] = dec_double(bbox[a]); lo[a] = -dec_double(bbox[3 + a]); }
+    *out = choose_grid(hi, lo, geom, N, cell_cap);
 }
 
 __device__ inline void bin_of(const Geometry& geom, const GridParams& g, float x, float y, float z, int b[3], int w[3]) {
@@ -175,12 +181,167 @@ __global__ void scan_kernel(const int* __restrict__ in, OutT* __restrict__ out, 
     }
 }
 
+// Exclusive scan of long arrays in three launches: sums of tiles of kScanTile items, a one-block
+// scan of those sums, then every tile scans itself on top of its offset.
+constexpr int kScanTile = 4096;          // 1024 threads x 4 items
+__global__ void __launch_bounds__(1024) tile_sum_kernel(const int* __restrict__ in, long long n, int* __restrict__ tile_sums) {
+    __shared__ int ws[32];
+    const long long base = (long long)blockIdx.x * kScanTile;
+    int v = 0;
+    for (int k = 0; k < 4; ++k) {
+        const long long i = base + k * 1024 + threadIdx.x;
+        if (i < n) v += in[i];
+    }
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+    if ((threadIdx.x & 31) == 0) ws[threadIdx.x >> 5] = v;
+    __syncthreads();
+    if (threadIdx.x < 32) {
+        int t = ws[threadIdx.x];
+        for (int o = 16; o > 0; o >>= 1) t += __shfl_xor_sync(0xffffffffu, t, o);
+        if (threadIdx.x == 0) tile_sums[blockIdx.x] = t;
+    }
+}
+template <typename OutT>
+__global__ void __launch_bounds__(1024) tile_scan_kernel(const int* __restrict__ in, OutT* __restrict__ out, long long n,
+                                                         const long long* __restrict__ tile_offsets, long long n_tiles) {
+    __shared__ long long ws[32];
+    const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
+    const long long base = (long long)blockIdx.x * kScanTile + threadIdx.x * 4;      // 4 consecutive items per thread
+    int v[4];
+    long long mine = 0;
+    for (int k = 0; k < 4; ++k) { v[k] = base + k < n ? in[base + k] : 0; mine += v[k]; }
+    long long x = mine;
+    for (int o = 1; o < 32; o <<= 1) {
+        const long long y = __shfl_up_sync(0xffffffffu, x, o);
+        if (lane >= o) x += y;
+    }
+    if (lane == 31) ws[wid] = x;
+    __syncthreads();
+    if (wid == 0) {
+        long long t = ws[lane];
+        for (int o = 1; o < 32; o <<= 1) {
+            const long long y = __shfl_up_sync(0xffffffffu, t, o);
+            if (lane >= o) t += y;
+        }
+        ws[lane] = t;
+    }
+    __syncthreads();
+    long long run = tile_offsets[blockIdx.x] + (wid > 0 ? ws[wid - 1] : 0) + x - mine;
+    for (int k = 0; k < 4; ++k) {
+        if (base + k < n) out[base + k] = (OutT)run;
+        run += v[k];
+    }
+    if (blockIdx.x == 0 && threadIdx.x == 0) out[n] = (OutT)tile_offsets[n_tiles];
+}
+
 __global__ void bin_fill_kernel(const float* __restrict__ pos, long long N, const int* __restrict__ atom_cell,
                                 const int* __restrict__ atom_wrap, const int* __restrict__ cell_start, int* cell_count,
                                 float4* __restrict__ s_pos, int* __restrict__ s_wrap) {
     for (long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x; i < N; i += (long long)gridDim.x * blockDim.x) {
         int cell = atom_cell[i];
         int slot = cell_start[cell] + atomicSub(&cell_count[cell], 1) - 1;
+        s_pos[slot] = make_float4(pos[3 * i], pos[3 * i + 1], pos[3 * i + 2], __int_as_float((int)i));
+        s_wrap[slot] = atom_wrap[i];
+    }
+}
+
+// Small structures: species lookup, bounding box, grid choice, binning, bin scan and the sort of
+// the atoms by bin in ONE launch of a single CTA (five dependent launches otherwise; at a few
+// thousand atoms the launches, not the work, set the time).
+constexpr int kPrepThreads = 1024;
+constexpr long long kSmallPrepAtoms = 16384;
+__global__ void __launch_bounds__(kPrepThreads)
+small_prep_kernel(const float* __restrict__ pos, const int* __restrict__ numbers, long long N, Geometry geom,
+                  const int* __restrict__ z_lut, int* __restrict__ species_idx, int cell_cap, GridParams* grid_out,
+                  int* __restrict__ atom_cell, int* __restrict__ atom_wrap, int* cell_count, int* cell_start,
+                  float4* __restrict__ s_pos, int* __restrict__ s_wrap, Counters* counters) {
+    __shared__ double red[6][32];
+    __shared__ GridParams sg;
+    __shared__ long long warp_sums[32];
+    __shared__ long long carry_s;
+    const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
+    // ---- species and bounding box of the fractional coordinates ----
+    double hi[3] = {-1e300, -1e300, -1e300}, lo[3] = {-1e300, -1e300, -1e300};
+    bool bad = false;
+    for (long long i = tid; i < N; i += kPrepThreads) {
+        int z = numbers ? numbers[i] : 0;
+        int s = numbers ? ((z >= 0 && z < 128) ? z_lut[z] : -1) : 0;
+        if (s < 0) { bad = true; s = 0; }
+        if (species_idx) species_idx[i] = s;
+        double f[3];
+        frac_coords(geom, pos[3 * i], pos[3 * i + 1], pos[3 * i + 2], f);
+        for (int a = 0; a < 3; ++a) { hi[a] = fmax(hi[a], f[a]); lo[a] = fmax(lo[a], -f[a]); }
+    }
+    if (bad) atomicOr(&counters->status, kStatusUnknownSpecies);
+    for (int a = 0; a < 3; ++a) {
+        for (int o = 16; o > 0; o >>= 1) {
+            hi[a] = fmax(hi[a], __shfl_xor_sync(0xffffffffu, hi[a], o));
+            lo[a] = fmax(lo[a], __shfl_xor_sync(0xffffffffu, lo[a], o));
+        }
+        if (lane == 0) { red[a][wid] = hi[a]; red[3 + a][wid] = lo[a]; }
+    }
+    __syncthreads();
+    if (tid == 0) {
+        double h3[3], l3[3];
+        for (int a = 0; a < 3; ++a) {
+            double h = -1e300, l = -1e300;
+            for (int w = 0; w < kPrepThreads / 32; ++w) { h = fmax(h, red[a][w]); l = fmax(l, red[3 + a][w]); }
+            h3[a] = h; l3[a] = -l;
+        }
+        sg = choose_grid(h3, l3, geom, N, cell_cap);
+        *grid_out = sg;
+        carry_s = 0;
+    }
+    __syncthreads();
+    const GridParams g = sg;
+    // ---- bin counts ----
+    for (int c = tid; c <= g.n_cells; c += kPrepThreads) cell_count[c] = 0;
+    __syncthreads();
+    for (long long i = tid; i < N; i += kPrepThreads) {
+        int b[3], w[3];
+        bin_of(geom, g, pos[3 * i], pos[3 * i + 1], pos[3 * i + 2], b, w);
+        if (abs(w[0]) > 100 || abs(w[1]) > 100 || abs(w[2]) > 100) {
+            atomicOr(&counters->status, kStatusShiftRange);
+            w[0] = w[1] = w[2] = 0;
+        }
+        const int cell = (b[2] * g.nb[1] + b[1]) * g.nb[0] + b[0];
+        atom_cell[i] = cell;
+        atom_wrap[i] = pack3(w);
+        atomicAdd(&cell_count[cell], 1);
+    }
+    __syncthreads();
+    // ---- exclusive scan of the bin counts ----
+    for (int base = 0; base < g.n_cells; base += kPrepThreads) {
+        const int i = base + tid;
+        const long long v = i < g.n_cells ? (long long)cell_count[i] : 0;
+        long long x = v;
+        for (int o = 1; o < 32; o <<= 1) {
+            const long long y = __shfl_up_sync(0xffffffffu, x, o);
+            if (lane >= o) x += y;
+        }
+        if (lane == 31) warp_sums[wid] = x;
+        __syncthreads();
+        if (wid == 0) {
+            long long sacc = warp_sums[lane];
+            for (int o = 1; o < 32; o <<= 1) {
+                const long long y = __shfl_up_sync(0xffffffffu, sacc, o);
+                if (lane >= o) sacc += y;
+            }
+            warp_sums[lane] = sacc;
+        }
+        __syncthreads();
+        const long long carry = carry_s;
+        if (i < g.n_cells) cell_start[i] = (int)(carry + (wid > 0 ? warp_sums[wid - 1] : 0) + x - v);
+        __syncthreads();
+        if (tid == kPrepThreads - 1) carry_s = carry + warp_sums[31];
+        __syncthreads();
+    }
+    if (tid == 0) cell_start[g.n_cells] = (int)carry_s;
+    __syncthreads();
+    // ---- atoms sorted by bin ----
+    for (long long i = tid; i < N; i += kPrepThreads) {
+        const int cell = atom_cell[i];
+        const int slot = cell_start[cell] + atomicSub(&cell_count[cell], 1) - 1;
         s_pos[slot] = make_float4(pos[3 * i], pos[3 * i + 1], pos[3 * i + 2], __int_as_float((int)i));
         s_wrap[slot] = atom_wrap[i];
     }

@@ -70,7 +70,8 @@ struct soap_handle {
     float4* d_s_pos = nullptr;
     int *d_cell_count = nullptr, *d_cell_start = nullptr;
     int *d_pair_count = nullptr, *d_row_count = nullptr, *d_self_row = nullptr;
-    long long *d_pair_ptr = nullptr, *d_row_ptr = nullptr;
+    long long *d_pair_ptr = nullptr, *d_row_ptr = nullptr, *d_tile_offsets = nullptr;
+    int* d_tile_sums = nullptr;
     unsigned long long *d_pair_key = nullptr, *d_pair_tmp = nullptr;
     int* d_pair_row = nullptr;
     // plan
@@ -241,6 +242,8 @@ int ensure_scratch(soap_t* h, int64_t N, int64_t C, int64_t pairs) {
         CU(regrow(&h->d_order, cap));
         CU(regrow(&h->d_pair_ptr, cap + 1));
         CU(regrow(&h->d_row_ptr, cap + 1));
+        CU(regrow(&h->d_tile_sums, cap / kScanTile + 2));
+        CU(regrow(&h->d_tile_offsets, cap / kScanTile + 3));
         h->cap_centers = cap;
     }
     if (pairs > h->cap_pairs || h->cap_pairs == 0) {
@@ -257,19 +260,37 @@ int blocks_for(int64_t n, int threads, int cap = 4096) {
     return (int)std::max<int64_t>(1, std::min<int64_t>((n + threads - 1) / threads, cap));
 }
 
+// Exclusive scan of C per-centre counts into out[0..C] (out[C] = total, also to *total_dev).
+void scan_counts(soap_t* h, const int* counts, long long* out, int64_t C, long long* total_dev, cudaStream_t st) {
+    if (C <= 65536) {
+        scan_kernel<long long><<<1, 1024, 0, st>>>(counts, out, C, total_dev);
+        return;
+    }
+    const long long tiles = (C + kScanTile - 1) / kScanTile;
+    tile_sum_kernel<<<(unsigned)tiles, 1024, 0, st>>>(counts, C, h->d_tile_sums);
+    scan_kernel<long long><<<1, 1024, 0, st>>>(h->d_tile_sums, h->d_tile_offsets, tiles, total_dev);
+    tile_scan_kernel<long long><<<(unsigned)tiles, 1024, 0, st>>>(counts, out, C, h->d_tile_offsets, tiles);
+}
+
 // Cell list and pair counts: everything up to the scan of the per-centre counts.
 int launch_count(soap_t* h, const float* pos, const int32_t* num, int64_t N, const Geometry& g,
                  const int32_t* centers, int64_t C, cudaStream_t st) {
     CU(cudaMemsetAsync(h->d_bbox, 0, 64 + 2 * kSizeBins * sizeof(int), st));
-    CU(cudaMemsetAsync(h->d_cell_count, 0, (h->cap_cells + 1) * sizeof(int), st));
-    if (N > 0) species_bbox_kernel<<<blocks_for(N, 256, 1024), 256, 0, st>>>(pos, num, N, g, h->d_zlut, h->d_species_idx, h->d_bbox, h->d_counters);
-    grid_setup_kernel<<<1, 1, 0, st>>>(h->d_bbox, g, N, (int)h->cap_cells, h->d_grid);
-    if (N > 0) bin_count_kernel<<<blocks_for(N, 256), 256, 0, st>>>(pos, N, g, h->d_grid, h->d_atom_cell, h->d_atom_wrap, h->d_cell_count, h->d_counters);
-    scan_kernel<int><<<1, 1024, 0, st>>>(h->d_cell_count, h->d_cell_start, h->cap_cells, nullptr, &h->d_grid->n_cells);
-    if (N > 0) bin_fill_kernel<<<blocks_for(N, 256), 256, 0, st>>>(pos, N, h->d_atom_cell, h->d_atom_wrap, h->d_cell_start, h->d_cell_count, h->d_s_pos, h->d_s_wrap);
+    if (N <= kSmallPrepAtoms) {
+        small_prep_kernel<<<1, kPrepThreads, 0, st>>>(pos, num, N, g, h->d_zlut, h->d_species_idx, (int)h->cap_cells, h->d_grid,
+                                                      h->d_atom_cell, h->d_atom_wrap, h->d_cell_count, h->d_cell_start,
+                                                      h->d_s_pos, h->d_s_wrap, h->d_counters);
+    } else {
+        CU(cudaMemsetAsync(h->d_cell_count, 0, (h->cap_cells + 1) * sizeof(int), st));
+        species_bbox_kernel<<<blocks_for(N, 256, 1024), 256, 0, st>>>(pos, num, N, g, h->d_zlut, h->d_species_idx, h->d_bbox, h->d_counters);
+        grid_setup_kernel<<<1, 1, 0, st>>>(h->d_bbox, g, N, (int)h->cap_cells, h->d_grid);
+        bin_count_kernel<<<blocks_for(N, 256), 256, 0, st>>>(pos, N, g, h->d_grid, h->d_atom_cell, h->d_atom_wrap, h->d_cell_count, h->d_counters);
+        scan_kernel<int><<<1, 1024, 0, st>>>(h->d_cell_count, h->d_cell_start, h->cap_cells, nullptr, &h->d_grid->n_cells);
+        bin_fill_kernel<<<blocks_for(N, 256), 256, 0, st>>>(pos, N, h->d_atom_cell, h->d_atom_wrap, h->d_cell_start, h->d_cell_count, h->d_s_pos, h->d_s_wrap);
+    }
     if (C > 0) count_kernel<<<(unsigned)((C + 7) / 8), 256, 0, st>>>(pos, centers, C, g, h->d_grid, h->d_atom_cell, h->d_atom_wrap, h->d_cell_start, h->d_s_pos, h->d_s_wrap, h->d_pair_count,
                                                                               C <= kOrderMaxCenters ? h->d_size_hist : nullptr, h->d_counters);
-    scan_kernel<long long><<<1, 1024, 0, st>>>(h->d_pair_count, h->d_pair_ptr, C, &h->d_counters->n_pairs);
+    scan_counts(h, h->d_pair_count, h->d_pair_ptr, C, &h->d_counters->n_pairs, st);
     CU(cudaGetLastError());
     return SOAP_OK;
 }
@@ -281,7 +302,7 @@ int launch_fill(soap_t* h, const float* pos, const Geometry& g, const int32_t* c
         pos, centers, C, g, h->d_grid, h->d_atom_cell, h->d_atom_wrap, h->d_cell_start, h->d_s_pos, h->d_s_wrap,
         h->d_pair_ptr, h->cap_pairs, h->d_pair_tmp, h->d_pair_key, h->d_pair_row, h->d_row_count, h->d_self_row,
         h->d_size_hist, h->d_size_cursor, C <= kOrderMaxCenters ? h->d_order : nullptr, h->d_counters);
-    scan_kernel<long long><<<1, 1024, 0, st>>>(h->d_row_count, row_ptr_out, C, &h->d_counters->n_rows);
+    scan_counts(h, h->d_row_count, row_ptr_out, C, &h->d_counters->n_rows, st);
     CU(cudaGetLastError());
     return SOAP_OK;
 }
@@ -373,7 +394,7 @@ void soap_destroy(soap_t* h) {
     if (!h) return;
     void* ptrs[] = {h->d_table, h->d_self, h->d_anorm, h->d_dfact, h->d_kl, h->d_feat, h->d_zlut, h->d_inv_int, h->d_lm_of_t, h->d_l_of_lm, h->d_counters, h->d_bbox,
                     h->d_grid, h->d_species_idx, h->d_atom_cell, h->d_atom_wrap, h->d_s_wrap, h->d_s_pos, h->d_cell_count,
-                    h->d_cell_start, h->d_pair_count, h->d_row_count, h->d_self_row, h->d_order, h->d_pair_ptr, h->d_row_ptr,
+                    h->d_cell_start, h->d_pair_count, h->d_row_count, h->d_self_row, h->d_order, h->d_pair_ptr, h->d_row_ptr, h->d_tile_sums, h->d_tile_offsets,
                     h->d_pair_key, h->d_pair_tmp, h->d_pair_row};
     for (void* p : ptrs) if (p) cudaFree(p);
     if (h->h_counters) cudaFreeHost(h->h_counters);
