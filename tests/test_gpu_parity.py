@@ -111,6 +111,31 @@ def test_basis_size_sweep_small_cluster(pkg, n_max, l_max):
     check_derivatives(soap, oracle, s, sample=[0, 7, 20, 35])
 
 
+@pytest.mark.parametrize("r_cut,n_max,l_max", [(9.0, 4, 3), (12.5, 2, 2)])
+def test_large_neighbourhoods(pkg, r_cut, n_max, l_max):
+    """Several hundred neighbours per centre (the paper's own runs use r_cut = 10 A): more pairs than
+    one geometry batch of the per-centre kernel holds, and (at 12.5 A) more than the neighbour sort
+    keeps in shared memory."""
+    s = water_cluster(600, 7)
+    args = ([1, 8], r_cut, n_max, l_max, 0.5, GTO)
+    soap, oracle = pkg.Soap(*args), SoapOracle(*args)
+    inner = np.argsort(np.linalg.norm(s.positions, axis=1))          # centres deep inside the cluster first
+    sample = [int(inner[0]), int(inner[5]), 0, 1799]
+    lists = oracle.neighbor_list(s.positions, None, sample)
+    assert max(len(l) for l in lists) > (512 if r_cut > 12 else 128)
+    check_neighbors(soap, oracle, s, sample)
+    check_derivatives(soap, oracle, s, sample=sample)
+
+
+def test_eight_species(pkg):
+    rng = np.random.Generator(np.random.PCG64(3))
+    s = water_cluster(20, 9)
+    s.numbers = np.array([1, 6, 7, 8, 9, 15, 16, 17], np.int32)[rng.integers(0, 8, s.n_atoms)].astype(np.int32)
+    args = ([17, 1, 6, 7, 8, 9, 15, 16], 4.5, 3, 2, 0.5, POLYNOMIAL)
+    soap, oracle = pkg.Soap(*args), SoapOracle(*args)
+    check_derivatives(soap, oracle, s, sample=[0, 13, 31, 59])
+
+
 def test_config2_water_1000_sampled(pkg):
     s = water_cluster(1000, 0)
     args = ([1, 8], 6.0, 8, 6, 0.5, GTO)
