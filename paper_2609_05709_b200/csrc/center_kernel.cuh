@@ -38,9 +38,9 @@ namespace soap {
 // Universal small tables for the harmonic recursion (l_max <= 12), read with
 // warp-uniform indices, hence constant memory.  Each translation unit that
 // includes this file gets its own copy, filled in at load time.
-__device__ __constant__ float kc_anorm[91] = {0};    // [(l,m)] sqrt((2l+1)/4pi (l-m)!/(l+m)!) (times sqrt2 for m > 0)
+__device__ __constant__ float2 kc_norm[91] = {0};    // [(l,m)] a_lm = sqrt((2l+1)/4pi (l-m)!/(l+m)!) (sqrt2 for m > 0), (l+m) a_lm
+__device__ __constant__ float4 kc_step[91] = {0};    // [(l,m)] coefficients that advance columns m and m+1 from l to l+1
 __device__ __constant__ float kc_dfact[16] = {0};    // [m] (2m-1)!!
-__device__ __constant__ float kc_inv_int[32] = {0};  // [k] 1/k
 
 // Degree-5 table lookup: value and derivative with respect to the interval coordinate t.
 __device__ __forceinline__ void radial_lookup(const float* __restrict__ table, int qi, int n_ch, int ch, float t,
@@ -55,49 +55,51 @@ __device__ __forceinline__ void radial_lookup(const float* __restrict__ table, i
     dv = fmaf(dv, t, v); v = fmaf(v, t, a.x);
 }
 
-// Real solid harmonics of one pair per lane; this warp covers the columns
-// m = wid, wid + kWarps, ... of
+// Real solid harmonics of one pair per lane, one column m of
 //   S_{l,+m} = a_lm Q_l^m Re (x+iy)^m,   S_{l,-m} = a_lm Q_l^m Im (x+iy)^m,
 //   Q_l^m = r^(l-m) d^m P_l(t)/dt^m at t = z/r,
-//   (l-m) Q_l^m = (2l-1) z Q_{l-1}^m - (l+m-1) r^2 Q_{l-2}^m,   Q_m^m = (2m-1)!!,
+//   (l+1-m) Q_{l+1}^m = (2l+1) z Q_l^m - (l+m) r^2 Q_{l-1}^m,   Q_m^m = (2m-1)!!,
 //   dQ_l^m/dx = -x Q_{l-1}^{m+1},  dQ_l^m/dy = -y Q_{l-1}^{m+1},  dQ_l^m/dz = (l+m) Q_{l-1}^m.
-// Columns m and m+1 are advanced in lock step, so a step needs four registers.
+// Columns m and m+1 are advanced in lock step, so a step needs four registers; the rational
+// coefficients of the recurrences come from constant memory (all lanes use the same (l, m)).
 template <bool GRAD>
-__device__ __forceinline__ void harmonics_columns(int L, int wid, float4 d, float4* __restrict__ out4,
-                                                  float* __restrict__ out1) {
-    const float x = d.x, y = d.y, z = d.z, r2 = d.w * d.w;
-    for (int m = wid; m <= L; m += kWarps) {
-        float cm = 1.f, sm = 0.f, cp = 0.f, sp = 0.f;           // (x+iy)^m and (x+iy)^(m-1)
-        for (int t = 0; t < m; ++t) {
-            cp = cm; sp = sm;
-            const float cn = x * cm - y * sm;
-            sm = x * sm + y * cm;
-            cm = cn;
+__device__ __forceinline__ void harmonics_column(int L, int m, float x, float y, float z, float r2,
+                                                 float4* __restrict__ out4, float* __restrict__ out1) {
+    float cm = 1.f, sm = 0.f, cp = 0.f, sp = 0.f;               // (x+iy)^m and (x+iy)^(m-1)
+    for (int t = 0; t < m; ++t) {
+        cp = cm; sp = sm;
+        const float cn = x * cm - y * sm;
+        sm = x * sm + y * cm;
+        cm = cn;
+    }
+    float a1 = kc_dfact[m], a0 = 0.f;                           // Q_l^m, Q_{l-1}^m
+    float b1 = 0.f, b0 = 0.f;                                   // Q_l^{m+1}, Q_{l-1}^{m+1}
+    const float fm = (float)m;
+    int t = m * (m + 1) / 2 + m;                                // index of (l, m), l = m
+    for (int l = m; l <= L; ++l) {
+        const float2 nr = kc_norm[t];
+        const float aq = nr.x * a1;
+        const int lm0 = l * l + l;
+        if (!GRAD) {
+            out1[lm0 + m] = aq * cm;
+            if (m) out1[lm0 - m] = aq * sm;
+        } else {
+            const float qz = nr.y * a0;                         // a (l+m) Q_{l-1}^m  (a0 = 0 when l = m)
+            const float qx = nr.x * b0;                         // a Q_{l-1}^{m+1}
+            const float mq = fm * aq;
+            const float xq = x * qx, yq = y * qx;
+            out4[lm0 + m] = make_float4(aq * cm, mq * cp - xq * cm, -mq * sp - yq * cm, qz * cm);
+            if (m) out4[lm0 - m] = make_float4(aq * sm, mq * sp - xq * sm, mq * cp - yq * sm, qz * sm);
         }
-        float a1 = kc_dfact[m], a0 = 0.f;                  // Q_l^m, Q_{l-1}^m
-        float b1 = 0.f, b0 = 0.f;                               // Q_l^{m+1}, Q_{l-1}^{m+1}
-        const float fm = (float)m;
-        for (int l = m; l <= L; ++l) {
-            const float a = kc_anorm[l * (l + 1) / 2 + m];
-            const float aq = a * a1;
-            const int lm0 = l * l + l;
-            if (!GRAD) {
-                out1[lm0 + m] = aq * cm;
-                if (m) out1[lm0 - m] = aq * sm;
-            } else {
-                const float qz = a * (float)(l + m) * a0;       // a dQ/dz (a0 = 0 when l = m)
-                const float qx = a * b0;                        // a Q_{l-1}^{m+1}
-                const float mq = fm * aq;
-                out4[lm0 + m] = make_float4(aq * cm, mq * cp - x * qx * cm, -mq * sp - y * qx * cm, qz * cm);
-                if (m) out4[lm0 - m] = make_float4(aq * sm, mq * sp - x * qx * sm, mq * cp - y * qx * sm, qz * sm);
-            }
-            // advance both columns to l + 1
-            const float zz = (float)(2 * l + 1) * z;
-            const float an = (zz * a1 - (float)(l + m) * r2 * a0) * kc_inv_int[l + 1 - m];
-            a0 = a1; a1 = an;
-            const float bn = (l == m) ? kc_dfact[m + 1] : (zz * b1 - (float)(l + m + 1) * r2 * b0) * kc_inv_int[l - m];
+        // advance both columns to l + 1
+        const float4 st = kc_step[t];
+        const float an = st.x * z * a1 - st.y * r2 * a0;
+        a0 = a1; a1 = an;
+        if (GRAD) {
+            const float bn = (l == m) ? kc_dfact[m + 1] : st.z * z * b1 - st.w * r2 * b0;
             b0 = b1; b1 = bn;
         }
+        t += l + 1;
     }
 }
 
@@ -107,7 +109,15 @@ center_kernel(const CenterParams p) {
     constexpr int L1 = L + 1, LM = L1 * L1, LMP = LM | 1;      // odd row stride: no shared-memory bank conflicts
     constexpr int NMAX_BOUND = NMAX_T ? NMAX_T : 16;
     // pass-1 ownership: W_LM warps cover the lm index, SLOTS such groups split the n index
-    constexpr int W_LM = (LM + 31) / 32, SLOTS = kWarps / W_LM;
+#ifndef SOAP_SLOT_DIV_DERIV
+#define SOAP_SLOT_DIV_DERIV 2
+#endif
+#ifndef SOAP_SLOT_DIV_DESC
+#define SOAP_SLOT_DIV_DESC 2
+#endif
+    constexpr int W_LM = (LM + 31) / 32;
+    constexpr int SLOTS_FULL = kWarps / W_LM, SLOT_DIV = DERIV ? SOAP_SLOT_DIV_DERIV : SOAP_SLOT_DIV_DESC;
+    constexpr int SLOTS = SLOTS_FULL / SLOT_DIV > 0 ? SLOTS_FULL / SLOT_DIV : 1;
     constexpr int NPT_RAW = (NMAX_BOUND + SLOTS - 1) / SLOTS;      // radial functions per thread ...
     constexpr int NPT = NPT_RAW < 8 ? NPT_RAW : 8;                // ... at most 8 at a time (register budget)
     extern __shared__ __align__(16) float smem[];
@@ -235,8 +245,11 @@ center_kernel(const CenterParams p) {
                 else sG1[pr * NCH + ch] = v;
             }
         }
-        if (lane < pc)
-            harmonics_columns<GRAD>(L, wid, geo_d[g + lane], sSD4 + lane * LMP, sS + lane * LMP);
+        if (lane < pc) {
+            const float4 d = geo_d[g + lane];
+            for (int m = wid; m <= L; m += kWarps)
+                harmonics_column<GRAD>(L, m, d.x, d.y, d.z, d.w * d.w, sSD4 + lane * LMP, sS + lane * LMP);
+        }
     };
 
     // =========================== pass 1: c (and D) ===========================

@@ -9,13 +9,13 @@ inline bool center_has_fixed_nmax(bool deriv, int n_max) {
     if (deriv) return n_max >= 2 && n_max <= 12 && n_max % 2 == 0;
     return n_max == 8;
 }
-// tables for l_max = 12: anorm[91], dfact[16], inv_int[32]
-cudaError_t center_constants(int l_max, const float* anorm91, const float* dfact16, const float* inv32);
+// harmonic tables up to l = 12: anorm[91] (index l(l+1)/2 + m), dfact[16]
+cudaError_t center_constants(int l_max, const float* anorm91, const float* dfact16);
 cudaError_t center_set_smem(bool deriv, int l_max, int n_max, int bytes);
 cudaError_t center_launch(bool deriv, int l_max, int n_max, const CenterParams& p, unsigned grid, size_t smem, cudaStream_t st);
 
 #define SOAP_DECLARE_L(LV)                                                                                       \
-    cudaError_t center_constants_l##LV(const float* anorm91, const float* dfact16, const float* inv32);         \
+    cudaError_t center_constants_l##LV(const float* anorm91, const float* dfact16);         \
     cudaError_t center_set_smem_l##LV(bool deriv, int n_max, int bytes);                                        \
     cudaError_t center_launch_l##LV(bool deriv, int n_max, const CenterParams& p, unsigned grid, size_t smem, cudaStream_t st);
 SOAP_DECLARE_L(0) SOAP_DECLARE_L(1) SOAP_DECLARE_L(2) SOAP_DECLARE_L(3) SOAP_DECLARE_L(4) SOAP_DECLARE_L(5) SOAP_DECLARE_L(6)

@@ -18,9 +18,9 @@
 using namespace soap;
 
 namespace soap {
-cudaError_t center_constants(int l_max, const float* anorm91, const float* dfact16, const float* inv32) {
+cudaError_t center_constants(int l_max, const float* anorm91, const float* dfact16) {
     switch (l_max) {
-#define X(LV) case LV: return center_constants_l##LV(anorm91, dfact16, inv32);
+#define X(LV) case LV: return center_constants_l##LV(anorm91, dfact16);
         X(0) X(1) X(2) X(3) X(4) X(5) X(6) X(7) X(8) X(9) X(10) X(11) X(12)
 #undef X
     }
@@ -208,11 +208,10 @@ int ensure_device(soap_t* h) {
     }
     {
         // universal harmonic tables up to l = 12 (the handle's own tables stop at its l_max)
-        std::vector<float> anorm(91, 0.f), dfact(16, 0.f), inv(32, 0.f);
+        std::vector<float> anorm(91, 0.f), dfact(16, 0.f);
         for (size_t i = 0; i < h->basis.anorm.size(); ++i) anorm[i] = h->basis.anorm[i];
         for (size_t i = 0; i < h->basis.dfact.size(); ++i) dfact[i] = h->basis.dfact[i];
-        for (int k = 1; k < 32; ++k) inv[k] = 1.0f / k;
-        CU(center_constants(h->l_max, anorm.data(), dfact.data(), inv.data()));
+        CU(center_constants(h->l_max, anorm.data(), dfact.data()));
     }
     CU(center_set_smem(false, h->l_max, h->n_max, (int)h->smem_desc));
     CU(center_set_smem(true, h->l_max, h->n_max, (int)h->smem_deriv));
