@@ -250,6 +250,7 @@ __global__ void bin_fill_kernel(const float* __restrict__ pos, long long N, cons
 // thousand atoms the launches, not the work, set the time).
 constexpr int kPrepThreads = 1024;
 constexpr long long kSmallPrepAtoms = 16384;
+constexpr int kPrepSmemCells = 4096;
 __global__ void __launch_bounds__(kPrepThreads)
 small_prep_kernel(const float* __restrict__ pos, const int* __restrict__ numbers, long long N, Geometry geom,
                   const int* __restrict__ z_lut, int* __restrict__ species_idx, int cell_cap, GridParams* grid_out,
@@ -259,6 +260,7 @@ small_prep_kernel(const float* __restrict__ pos, const int* __restrict__ numbers
     __shared__ GridParams sg;
     __shared__ long long warp_sums[32];
     __shared__ long long carry_s;
+    __shared__ int s_cnt[kPrepSmemCells + 1], s_start[kPrepSmemCells + 1];   // bin counters on chip when they fit
     const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
     // ---- species and bounding box of the fractional coordinates ----
     double hi[3] = {-1e300, -1e300, -1e300}, lo[3] = {-1e300, -1e300, -1e300};
@@ -294,8 +296,10 @@ small_prep_kernel(const float* __restrict__ pos, const int* __restrict__ numbers
     }
     __syncthreads();
     const GridParams g = sg;
+    const bool on_chip = g.n_cells <= kPrepSmemCells;
+    int* cnt = on_chip ? s_cnt : cell_count;
     // ---- bin counts ----
-    for (int c = tid; c <= g.n_cells; c += kPrepThreads) cell_count[c] = 0;
+    for (int c = tid; c <= g.n_cells; c += kPrepThreads) cnt[c] = 0;
     __syncthreads();
     for (long long i = tid; i < N; i += kPrepThreads) {
         int b[3], w[3];
@@ -307,13 +311,13 @@ small_prep_kernel(const float* __restrict__ pos, const int* __restrict__ numbers
         const int cell = (b[2] * g.nb[1] + b[1]) * g.nb[0] + b[0];
         atom_cell[i] = cell;
         atom_wrap[i] = pack3(w);
-        atomicAdd(&cell_count[cell], 1);
+        atomicAdd(&cnt[cell], 1);
     }
     __syncthreads();
     // ---- exclusive scan of the bin counts ----
     for (int base = 0; base < g.n_cells; base += kPrepThreads) {
         const int i = base + tid;
-        const long long v = i < g.n_cells ? (long long)cell_count[i] : 0;
+        const long long v = i < g.n_cells ? (long long)cnt[i] : 0;
         long long x = v;
         for (int o = 1; o < 32; o <<= 1) {
             const long long y = __shfl_up_sync(0xffffffffu, x, o);
@@ -331,7 +335,11 @@ small_prep_kernel(const float* __restrict__ pos, const int* __restrict__ numbers
         }
         __syncthreads();
         const long long carry = carry_s;
-        if (i < g.n_cells) cell_start[i] = (int)(carry + (wid > 0 ? warp_sums[wid - 1] : 0) + x - v);
+        if (i < g.n_cells) {
+            const int st = (int)(carry + (wid > 0 ? warp_sums[wid - 1] : 0) + x - v);
+            cell_start[i] = st;
+            if (on_chip) s_start[i] = st;
+        }
         __syncthreads();
         if (tid == kPrepThreads - 1) carry_s = carry + warp_sums[31];
         __syncthreads();
@@ -339,9 +347,10 @@ small_prep_kernel(const float* __restrict__ pos, const int* __restrict__ numbers
     if (tid == 0) cell_start[g.n_cells] = (int)carry_s;
     __syncthreads();
     // ---- atoms sorted by bin ----
+    const int* starts = on_chip ? s_start : cell_start;
     for (long long i = tid; i < N; i += kPrepThreads) {
         const int cell = atom_cell[i];
-        const int slot = cell_start[cell] + atomicSub(&cell_count[cell], 1) - 1;
+        const int slot = starts[cell] + atomicSub(&cnt[cell], 1) - 1;
         s_pos[slot] = make_float4(pos[3 * i], pos[3 * i + 1], pos[3 * i + 2], __int_as_float((int)i));
         s_wrap[slot] = atom_wrap[i];
     }
