@@ -38,7 +38,22 @@ WORKLOADS = {
 DEFAULT_WORKLOAD = "water1000_gto_n8_l6_rc6"
 METRIC = "SOAP atoms/s, descriptor + Jacobian"
 UNIT = "atoms/s"
-KERNELS_PER_STEP = 10     # species_bbox, grid_setup, bin_count, scan, bin_fill, count, scan, fill, scan, center
+
+
+def kernels_per_step(n_atoms, n_centers):
+    """Kernel launches of one soap_derivatives call: the cell-list build is one launch up to 16384
+    atoms (five above), then count, scan, fill, scan (scans are three launches each above 65536
+    centres) and the fused per-centre kernel."""
+    prep = 1 if n_atoms <= 16384 else 5
+    scan = 1 if n_centers <= 65536 else 3
+    return prep + 1 + scan + 1 + scan + 1
+
+
+# DRAM traffic of the fused kernel from the ncu capture in profiles/center_kernel_water300.md
+# (dram__bytes_read.sum + dram__bytes_write.sum of one launch) and that launch's algorithmic bytes;
+# the full-size launch is scaled by its own algorithmic bytes (traffic is proportional to the rows written).
+NCU_SMALL_TRAFFIC_BYTES = 572.66e6 + 1.55e6
+NCU_SMALL_ALGORITHMIC_BYTES = 629088584
 
 
 def make_structure(name):
@@ -67,7 +82,7 @@ class ClockSampler:
     def start(self):
         try:
             self.proc = subprocess.Popen(["nvidia-smi", f"--id={self.index}", f"--query-gpu={self.QUERY}",
-                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                          "--format=csv,noheader,nounits", "-lms", "20"],
                                          stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
             threading.Thread(target=self._read, daemon=True).start()
         except OSError:
@@ -201,13 +216,19 @@ def run_cuda(args):
             dist.barrier()
         torch.cuda.synchronize()
 
-    for _ in range(max(args.warmup, 3)):
-        step()
-    soap.status()
-    # ---- device-resident timing: per-step CUDA events on the launching stream ----
+    # clocks are sampled from the warm-up to the end of the end-to-end leg (nvidia-smi needs a
+    # moment to deliver its first line, and the device-resident region lasts only tens of ms)
     sampler = ClockSampler(local)
     if rank == 0:
         sampler.start()
+    for _ in range(max(args.warmup, 3)):
+        step()
+    soap.status()
+    t_wait = time.time()
+    while rank == 0 and sampler.proc is not None and not sampler.lines and time.time() - t_wait < 2.0:
+        step()
+        torch.cuda.synchronize()
+    # ---- device-resident timing: per-step CUDA events on the launching stream ----
     barrier()
     step_ms, center_ms, nbr_ms = [], [], []
     for _ in range(args.steps):
@@ -222,7 +243,6 @@ def run_cuda(args):
         nbr_ms.append(a)
         center_ms.append(b)
     barrier()
-    clocks = sampler.stop() if rank == 0 else None
     soap.status()
     total_ms = sum(step_ms)
     # ---- end to end on host buffers: H2D of the inputs, compute, D2H of every output ----
@@ -244,6 +264,7 @@ def run_cuda(args):
         e1.synchronize()
         e2e_ms.append(e0.elapsed_time(e1))
     barrier()
+    clocks = sampler.stop() if rank == 0 else None
     e2e_total = sum(e2e_ms)
     total_ms, e2e_total = max_over_ranks([total_ms, e2e_total], device="cuda")     # slowest rank decides
     if rank != 0:
@@ -274,9 +295,11 @@ def run_cuda(args):
         "clocks": clocks,
         "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                 "ms_per_step": e2e_total / e2e_steps if e2e_steps else None, "steps": e2e_steps},
-        "gpu_launches": KERNELS_PER_STEP * args.steps,
+        "gpu_launches": kernels_per_step(C, C) * args.steps,
         "roofline": {"bound": "hbm", "kernel": "center_kernel<true>", "achieved": achieved, "peak": peak, "unit": "GB/s",
-                     "frac": achieved / peak, "peak_source": peak_src, "traffic": None,
+                     "frac": achieved / peak, "peak_source": peak_src,
+                     "traffic": alg_bytes * NCU_SMALL_TRAFFIC_BYTES / NCU_SMALL_ALGORITHMIC_BYTES,
+                     "traffic_source": "ncu capture on the 300-molecule cluster, scaled by algorithmic bytes",
                      "algorithmic_bytes_per_launch": alg_bytes, "kernel_ms": k_ms,
                      "neighbour_search_ms": statistics.mean(nbr_ms), "pairs": n_pairs, "rows": n_rows, "features": F},
         "cpu_baseline": {"value": cpu_value, "unit": UNIT, "cores": 1, "kind": "oracle",
