@@ -41,12 +41,10 @@ UNIT = "atoms/s"
 
 
 def kernels_per_step(n_atoms, n_centers):
-    """Kernel launches of one soap_derivatives call: the cell-list build is one launch up to 16384
-    atoms (five above), then count, scan, fill, scan (scans are three launches each above 65536
-    centres) and the fused per-centre kernel."""
-    prep = 1 if n_atoms <= 16384 else 5
-    scan = 1 if n_centers <= 65536 else 3
-    return prep + 1 + scan + 1 + scan + 1
+    """Kernel launches of one soap_derivatives call: the cell-list build (one launch up to 16384
+    atoms, five above), the pair kernel, the row scan with the launch order (one launch up to 65536
+    centres, three above) and the fused per-centre kernel."""
+    return (1 if n_atoms <= 16384 else 5) + 1 + (1 if n_centers <= 65536 else 3) + 1
 
 
 # DRAM traffic of the fused kernel from the ncu capture in profiles/center_kernel_water300.md

@@ -124,7 +124,7 @@ center_kernel(const CenterParams p) {
     const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
     const long long c_idx = p.order ? p.order[blockIdx.x] : blockIdx.x;
     // a failed neighbour build or an undersized output: write nothing
-    if (p.pair_ptr[p.n_centers] > p.pair_capacity) return;
+    if (p.counters->n_pairs > p.pair_capacity) return;
     if (DERIV && p.row_ptr[p.n_centers] > p.row_capacity) {
         if (c_idx == 0 && tid == 0) atomicOr(&p.counters->status, kStatusRowCapacity);
         return;
@@ -145,8 +145,8 @@ center_kernel(const CenterParams p) {
     const int ci = p.centers ? p.centers[c_idx] : (int)c_idx;
     const float xi = p.pos[3 * (long long)ci], yi = p.pos[3 * (long long)ci + 1], zi = p.pos[3 * (long long)ci + 2];
     const int zi_species = p.species_idx[ci];
-    const long long pair_base = p.pair_ptr[c_idx];
-    const int k_pairs = (int)(p.pair_ptr[c_idx + 1] - pair_base);
+    const long long pair_base = p.pair_start[c_idx];
+    const int k_pairs = p.pair_count[c_idx];
     const bool periodic = p.geom.pbc[0] | p.geom.pbc[1] | p.geom.pbc[2];
 
     for (int e = tid; e < CT * (DERIV ? 4 : 1); e += kThreads) {

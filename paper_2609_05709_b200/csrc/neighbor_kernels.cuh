@@ -98,7 +98,9 @@ __device__ inline GridParams choose_grid(const double hi_in[3], const double lo_
     return g;
 }
 
-__global__ void grid_setup_kernel(const unsigned long long* bbox, Geometry geom, long long N, int cell_cap, GridParams* out) {
+__global__ void grid_setup_kernel(const unsigned long long* bbox, Geometry geom, long long N, int cell_cap, GridParams* out,
+                                  Counters* counters) {
+    if (counters) { counters->n_pairs = 0; counters->n_rows = 0; }      // the pair cursor of this call
     double hi[3], lo[3];
     for (int a = 0; a < 3; ++a) { hi[a] = dec_double(bbox[a]); lo[a] = -dec_double(bbox[3 + a]); }
     *out = choose_grid(hi, lo, geom, N, cell_cap);
@@ -293,6 +295,8 @@ small_prep_kernel(const float* __restrict__ pos, const int* __restrict__ numbers
         sg = choose_grid(h3, l3, geom, N, cell_cap);
         *grid_out = sg;
         carry_s = 0;
+        counters->n_pairs = 0;                                            // the pair cursor of this call
+        counters->n_rows = 0;
     }
     __syncthreads();
     const GridParams g = sg;
@@ -449,16 +453,11 @@ __device__ inline void for_each_candidate(const Geometry& geom, const GridParams
     }
 }
 
-// Centres are handed to the per-centre kernel largest first (their CTAs differ in length by the
-// number of pairs): a histogram of pair counts in bins of 4, filled while counting, gives every
-// centre a slot.  Only used for moderate numbers of centres (the bins are global atomics).
-constexpr int kSizeBins = 256, kSizeBinShift = 2;
-
 // One warp per centre: number of pairs.
 __global__ void count_kernel(const float* __restrict__ pos, const int* __restrict__ centers, long long C, Geometry geom,
                              const GridParams* __restrict__ gp, const int* __restrict__ atom_cell, const int* __restrict__ atom_wrap,
                              const int* __restrict__ cell_start, const float4* __restrict__ s_pos, const int* __restrict__ s_wrap,
-                             int* __restrict__ pair_count, int* size_hist, Counters* counters) {
+                             int* __restrict__ pair_count, Counters* counters) {
     const GridParams g = *gp;
     const int lane = threadIdx.x & 31;
     const long long c = blockIdx.x * (long long)(blockDim.x >> 5) + (threadIdx.x >> 5);
@@ -474,36 +473,31 @@ __global__ void count_kernel(const float* __restrict__ pos, const int* __restric
     int cnt = 0;
     for_each_candidate(geom, g, cell_start, s_pos, s_wrap, xi, yi, zi, bi, wi, lane, counters,
                        [&](bool valid, unsigned long long) { cnt += __popc(__ballot_sync(0xffffffffu, valid)); });
-    if (lane == 0) {
-        pair_count[c] = cnt;
-        if (size_hist) atomicAdd(&size_hist[min(cnt >> kSizeBinShift, kSizeBins - 1)], 1);
-    }
+    if (lane == 0) pair_count[c] = cnt;
 }
 
 constexpr int kFillSmemKeys = 512;       // per warp; longer rows are sorted through global memory
 constexpr int kFillWarps = 4;
 
-// One warp per centre: collect the pairs, sort them by key, derive the Jacobian
-// row bookkeeping (distinct atoms, the centre's own position among them).
+// One warp per centre, one walk over the candidates: collect the pairs, reserve a segment of the
+// pair arrays with one atomic add (segments follow the order in which warps arrive, so the pair
+// arrays are addressed through pair_start / pair_count, not through a prefix sum), sort the keys,
+// derive the Jacobian row bookkeeping (distinct atoms, the centre's own position among them).
+// When the segment does not fit the planned capacity only the counts are produced and the status
+// word says so; the caller plans again with the totals.
 __global__ void __launch_bounds__(kFillWarps * 32)
-fill_kernel(const float* __restrict__ pos, const int* __restrict__ centers, long long C, Geometry geom,
-            const GridParams* __restrict__ gp, const int* __restrict__ atom_cell, const int* __restrict__ atom_wrap,
-            const int* __restrict__ cell_start, const float4* __restrict__ s_pos, const int* __restrict__ s_wrap,
-            const long long* __restrict__ pair_ptr, long long pair_capacity,
-            unsigned long long* pair_tmp, unsigned long long* pair_key, int* __restrict__ pair_row,
-            int* __restrict__ row_count, int* __restrict__ self_row, const int* size_hist, int* size_cursor,
-            int* __restrict__ order, Counters* counters) {
+pairs_kernel(const float* __restrict__ pos, const int* __restrict__ centers, long long C, Geometry geom,
+             const GridParams* __restrict__ gp, const int* __restrict__ atom_cell, const int* __restrict__ atom_wrap,
+             const int* __restrict__ cell_start, const float4* __restrict__ s_pos, const int* __restrict__ s_wrap,
+             long long pair_capacity, unsigned long long* pair_tmp, unsigned long long* pair_key, int* __restrict__ pair_row,
+             long long* __restrict__ pair_start, int* __restrict__ pair_count, int* __restrict__ row_count,
+             int* __restrict__ self_row, Counters* counters) {
     __shared__ unsigned long long s_raw[kFillWarps][kFillSmemKeys];
     __shared__ unsigned long long s_sorted[kFillWarps][kFillSmemKeys];
     const GridParams g = *gp;
     const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
     const long long c = blockIdx.x * (long long)kFillWarps + wid;
     if (c >= C) return;
-    if (pair_ptr[C] > pair_capacity) {                       // scratch too small: report, write nothing
-        if (c == 0 && lane == 0) atomicOr(&counters->status, kStatusPairCapacity);
-        if (lane == 0) { row_count[c] = 0; self_row[c] = 0; }
-        return;
-    }
     const int i = centers ? centers[c] : (int)c;
     const float xi = pos[3 * (long long)i], yi = pos[3 * (long long)i + 1], zi = pos[3 * (long long)i + 2];
     int bi[3], wi[3];
@@ -512,27 +506,42 @@ fill_kernel(const float* __restrict__ pos, const int* __restrict__ centers, long
         bi[0] = cell % g.nb[0]; bi[1] = (cell / g.nb[0]) % g.nb[1]; bi[2] = cell / (g.nb[0] * g.nb[1]);
         unpack3(atom_wrap[i], wi);
     }
-    const long long base = pair_ptr[c];
-    const int k = (int)(pair_ptr[c + 1] - base);
-    if (order) {
-        // slot = number of centres in larger bins + arrival number inside the own bin
-        const int bin = min(k >> kSizeBinShift, kSizeBins - 1);
-        int larger = 0;
-        for (int b = bin + 1 + lane; b < kSizeBins; b += 32) larger += size_hist[b];
-        for (int o = 16; o > 0; o >>= 1) larger += __shfl_xor_sync(0xffffffffu, larger, o);
-        if (lane == 0) order[larger + atomicAdd(&size_cursor[bin], 1)] = (int)c;
-    }
-    const bool in_smem = k <= kFillSmemKeys;
-    volatile unsigned long long* raw = in_smem ? s_raw[wid] : pair_tmp + base;
-    volatile unsigned long long* sorted = in_smem ? s_sorted[wid] : pair_key + base;
-    int cnt = 0;
+    // ---- walk the candidates; keep the keys on chip while they fit ----
+    int k = 0;
     for_each_candidate(geom, g, cell_start, s_pos, s_wrap, xi, yi, zi, bi, wi, lane, counters,
                        [&](bool valid, unsigned long long key) {
-                           unsigned m = __ballot_sync(0xffffffffu, valid);
-                           int at = cnt + __popc(m & ((1u << lane) - 1));
-                           if (valid && at < k) raw[at] = key;
-                           cnt += __popc(m);
+                           const unsigned m = __ballot_sync(0xffffffffu, valid);
+                           const int at = k + __popc(m & ((1u << lane) - 1));
+                           if (valid && at < kFillSmemKeys) s_raw[wid][at] = key;
+                           k += __popc(m);
                        });
+    long long base = 0;
+    if (lane == 0) base = (long long)atomicAdd(reinterpret_cast<unsigned long long*>(&counters->n_pairs), (unsigned long long)k);
+    base = __shfl_sync(0xffffffffu, base, 0);
+    const bool fits = base + k <= pair_capacity;
+    const bool in_smem = k <= kFillSmemKeys;
+    if (lane == 0) { pair_start[c] = base; pair_count[c] = fits ? k : 0; }
+    if (!fits) {
+        if (lane == 0) {
+            atomicOr(&counters->status, kStatusPairCapacity);
+            row_count[c] = k + 1;                         // upper bound; exact once the plan fits
+            self_row[c] = 0;
+        }
+        return;
+    }
+    if (!in_smem) {
+        // rare: more pairs than the on-chip buffer holds; walk again, now with a place to put them
+        int at0 = 0;
+        for_each_candidate(geom, g, cell_start, s_pos, s_wrap, xi, yi, zi, bi, wi, lane, counters,
+                           [&](bool valid, unsigned long long key) {
+                               const unsigned m = __ballot_sync(0xffffffffu, valid);
+                               const int at = at0 + __popc(m & ((1u << lane) - 1));
+                               if (valid && at < k) pair_tmp[base + at] = key;
+                               at0 += __popc(m);
+                           });
+    }
+    volatile unsigned long long* raw = in_smem ? s_raw[wid] : pair_tmp + base;
+    volatile unsigned long long* sorted = in_smem ? s_sorted[wid] : pair_key + base;
     __syncwarp();
     // rank sort (keys are distinct)
     bool self_in = false;
@@ -573,24 +582,80 @@ fill_kernel(const float* __restrict__ pos, const int* __restrict__ centers, long
     }
 }
 
-// Copies the sorted pair list out in a plain layout.
-__global__ void export_pairs_kernel(const long long* __restrict__ pair_ptr, const unsigned long long* __restrict__ pair_key,
-                                    long long C, long long capacity, long long* out_ptr, int* out_atom, int* out_shift,
-                                    Counters* counters) {
-    const long long total = pair_ptr[C];
-    for (long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x; i <= C; i += (long long)gridDim.x * blockDim.x)
-        out_ptr[i] = pair_ptr[i];
-    if (total > capacity) {
+// One block: exclusive scan of the row counts (rows of centre c start at row_ptr[c]) and the launch
+// order of the per-centre kernel, largest pair count first (bins of 4 pairs, counting sort), so that
+// the long CTAs do not end up alone at the tail of the launch.
+constexpr int kSizeBins = 256, kSizeBinShift = 2;
+__global__ void __launch_bounds__(1024)
+rows_order_kernel(const int* __restrict__ row_count, const int* __restrict__ pair_count, long long C,
+                  long long* __restrict__ row_ptr, int* __restrict__ order, Counters* counters) {
+    __shared__ long long warp_sums[32];
+    __shared__ long long carry_s;
+    __shared__ int hist[kSizeBins], first_slot[kSizeBins];
+    const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
+    if (tid == 0) carry_s = 0;
+    if (tid < kSizeBins) hist[tid] = 0;
+    __syncthreads();
+    for (long long base = 0; base < C; base += 1024) {
+        const long long i = base + tid;
+        const long long v = i < C ? (long long)row_count[i] : 0;
+        if (i < C) atomicAdd(&hist[min(pair_count[i] >> kSizeBinShift, kSizeBins - 1)], 1);
+        long long x = v;
+        for (int o = 1; o < 32; o <<= 1) {
+            const long long y = __shfl_up_sync(0xffffffffu, x, o);
+            if (lane >= o) x += y;
+        }
+        if (lane == 31) warp_sums[wid] = x;
+        __syncthreads();
+        if (wid == 0) {
+            long long sacc = warp_sums[lane];
+            for (int o = 1; o < 32; o <<= 1) {
+                const long long y = __shfl_up_sync(0xffffffffu, sacc, o);
+                if (lane >= o) sacc += y;
+            }
+            warp_sums[lane] = sacc;
+        }
+        __syncthreads();
+        const long long carry = carry_s;
+        if (i < C) row_ptr[i] = carry + (wid > 0 ? warp_sums[wid - 1] : 0) + x - v;
+        __syncthreads();
+        if (tid == 1023) carry_s = carry + warp_sums[31];
+        __syncthreads();
+    }
+    if (tid == 0) {
+        row_ptr[C] = carry_s;
+        counters->n_rows = carry_s;
+        int run = 0;
+        for (int b = kSizeBins - 1; b >= 0; --b) { first_slot[b] = run; run += hist[b]; }
+    }
+    __syncthreads();
+    if (order)
+        for (long long i = tid; i < C; i += 1024) {
+            const int b = min(pair_count[i] >> kSizeBinShift, kSizeBins - 1);
+            order[atomicAdd(&first_slot[b], 1)] = (int)i;
+        }
+}
+
+// Compact copy of the pair list (the pair arrays are addressed by segment): one warp per centre.
+__global__ void export_pairs_kernel(const long long* __restrict__ pair_start, const long long* __restrict__ out_ptr,
+                                    const unsigned long long* __restrict__ pair_key, long long C, long long capacity,
+                                    int* out_atom, int* out_shift, Counters* counters) {
+    if (out_ptr[C] > capacity) {
         if (blockIdx.x == 0 && threadIdx.x == 0) atomicOr(&counters->status, kStatusPairCapacity);
         return;
     }
-    for (long long e = blockIdx.x * (long long)blockDim.x + threadIdx.x; e < total; e += (long long)gridDim.x * blockDim.x) {
-        unsigned long long key = pair_key[e];
-        out_atom[e] = key_atom(key);
-        if (out_shift) {
-            int s[3];
-            key_shift(key, s);
-            out_shift[3 * e] = s[0]; out_shift[3 * e + 1] = s[1]; out_shift[3 * e + 2] = s[2];
+    const int lane = threadIdx.x & 31;
+    for (long long c = (blockIdx.x * (long long)blockDim.x + threadIdx.x) >> 5; c < C; c += ((long long)gridDim.x * blockDim.x) >> 5) {
+        const long long src = pair_start[c], dst = out_ptr[c];
+        const int k = (int)(out_ptr[c + 1] - dst);
+        for (int q = lane; q < k; q += 32) {
+            const unsigned long long key = pair_key[src + q];
+            out_atom[dst + q] = key_atom(key);
+            if (out_shift) {
+                int sft[3];
+                key_shift(key, sft);
+                out_shift[3 * (dst + q)] = sft[0]; out_shift[3 * (dst + q) + 1] = sft[1]; out_shift[3 * (dst + q) + 2] = sft[2];
+            }
         }
     }
 }

@@ -60,8 +60,8 @@ struct soap_handle {
     float *d_table = nullptr, *d_self = nullptr, *d_anorm = nullptr, *d_dfact = nullptr, *d_kl = nullptr, *d_inv_int = nullptr;
     int *d_feat = nullptr, *d_zlut = nullptr, *d_lm_of_t = nullptr, *d_l_of_lm = nullptr;
     Counters* d_counters = nullptr;
-    unsigned long long* d_bbox = nullptr;   // 6 words of bounding box, then the size histogram and its cursors
-    int *d_size_hist = nullptr, *d_size_cursor = nullptr, *d_order = nullptr;
+    unsigned long long* d_bbox = nullptr;   // 6 words of bounding box (structures above 16384 atoms)
+    int* d_order = nullptr;
     GridParams* d_grid = nullptr;
     Counters* h_counters = nullptr;      // pinned
     // scratch, grown on demand
@@ -70,7 +70,7 @@ struct soap_handle {
     float4* d_s_pos = nullptr;
     int *d_cell_count = nullptr, *d_cell_start = nullptr;
     int *d_pair_count = nullptr, *d_row_count = nullptr, *d_self_row = nullptr;
-    long long *d_pair_ptr = nullptr, *d_row_ptr = nullptr, *d_tile_offsets = nullptr;
+    long long *d_pair_ptr = nullptr, *d_pair_start = nullptr, *d_row_ptr = nullptr, *d_tile_offsets = nullptr;
     int* d_tile_sums = nullptr;
     unsigned long long *d_pair_key = nullptr, *d_pair_tmp = nullptr;
     int* d_pair_row = nullptr;
@@ -176,9 +176,7 @@ int ensure_device(soap_t* h) {
     CU(upload(&h->d_zlut, lut));
     CU(cudaMalloc((void**)&h->d_counters, sizeof(Counters)));
     CU(cudaMemset(h->d_counters, 0, sizeof(Counters)));
-    CU(cudaMalloc((void**)&h->d_bbox, 64 + 2 * kSizeBins * sizeof(int)));
-    h->d_size_hist = reinterpret_cast<int*>(reinterpret_cast<char*>(h->d_bbox) + 64);
-    h->d_size_cursor = h->d_size_hist + kSizeBins;
+    CU(cudaMalloc((void**)&h->d_bbox, 64));
     CU(cudaMalloc((void**)&h->d_grid, sizeof(GridParams)));
     CU(cudaMallocHost((void**)&h->h_counters, sizeof(Counters)));
     // shared-memory plan of the per-centre kernels
@@ -240,6 +238,7 @@ int ensure_scratch(soap_t* h, int64_t N, int64_t C, int64_t pairs) {
         CU(regrow(&h->d_self_row, cap));
         CU(regrow(&h->d_order, cap));
         CU(regrow(&h->d_pair_ptr, cap + 1));
+        CU(regrow(&h->d_pair_start, cap));
         CU(regrow(&h->d_row_ptr, cap + 1));
         CU(regrow(&h->d_tile_sums, cap / kScanTile + 2));
         CU(regrow(&h->d_tile_offsets, cap / kScanTile + 3));
@@ -271,37 +270,32 @@ void scan_counts(soap_t* h, const int* counts, long long* out, int64_t C, long l
     tile_scan_kernel<long long><<<(unsigned)tiles, 1024, 0, st>>>(counts, out, C, h->d_tile_offsets, tiles);
 }
 
-// Cell list and pair counts: everything up to the scan of the per-centre counts.
-int launch_count(soap_t* h, const float* pos, const int32_t* num, int64_t N, const Geometry& g,
-                 const int32_t* centers, int64_t C, cudaStream_t st) {
-    CU(cudaMemsetAsync(h->d_bbox, 0, 64 + 2 * kSizeBins * sizeof(int), st));
+// The whole neighbour search: cell list, sorted pair segments with their row bookkeeping, row
+// pointers (to `row_ptr_out`, the caller's array or the handle's) and the launch order.
+int launch_neighbors(soap_t* h, const float* pos, const int32_t* num, int64_t N, const Geometry& g,
+                     const int32_t* centers, int64_t C, long long* row_ptr_out, cudaStream_t st) {
     if (N <= kSmallPrepAtoms) {
         small_prep_kernel<<<1, kPrepThreads, 0, st>>>(pos, num, N, g, h->d_zlut, h->d_species_idx, (int)h->cap_cells, h->d_grid,
                                                       h->d_atom_cell, h->d_atom_wrap, h->d_cell_count, h->d_cell_start,
                                                       h->d_s_pos, h->d_s_wrap, h->d_counters);
     } else {
+        CU(cudaMemsetAsync(h->d_bbox, 0, 64, st));
         CU(cudaMemsetAsync(h->d_cell_count, 0, (h->cap_cells + 1) * sizeof(int), st));
         species_bbox_kernel<<<blocks_for(N, 256, 1024), 256, 0, st>>>(pos, num, N, g, h->d_zlut, h->d_species_idx, h->d_bbox, h->d_counters);
-        grid_setup_kernel<<<1, 1, 0, st>>>(h->d_bbox, g, N, (int)h->cap_cells, h->d_grid);
+        grid_setup_kernel<<<1, 1, 0, st>>>(h->d_bbox, g, N, (int)h->cap_cells, h->d_grid, h->d_counters);
         bin_count_kernel<<<blocks_for(N, 256), 256, 0, st>>>(pos, N, g, h->d_grid, h->d_atom_cell, h->d_atom_wrap, h->d_cell_count, h->d_counters);
         scan_kernel<int><<<1, 1024, 0, st>>>(h->d_cell_count, h->d_cell_start, h->cap_cells, nullptr, &h->d_grid->n_cells);
         bin_fill_kernel<<<blocks_for(N, 256), 256, 0, st>>>(pos, N, h->d_atom_cell, h->d_atom_wrap, h->d_cell_start, h->d_cell_count, h->d_s_pos, h->d_s_wrap);
     }
-    if (C > 0) count_kernel<<<(unsigned)((C + 7) / 8), 256, 0, st>>>(pos, centers, C, g, h->d_grid, h->d_atom_cell, h->d_atom_wrap, h->d_cell_start, h->d_s_pos, h->d_s_wrap, h->d_pair_count,
-                                                                              C <= kOrderMaxCenters ? h->d_size_hist : nullptr, h->d_counters);
-    scan_counts(h, h->d_pair_count, h->d_pair_ptr, C, &h->d_counters->n_pairs, st);
-    CU(cudaGetLastError());
-    return SOAP_OK;
-}
-
-// Sorted pair list and row bookkeeping; row_ptr goes to `row_ptr_out` (the caller's array or the handle's).
-int launch_fill(soap_t* h, const float* pos, const Geometry& g, const int32_t* centers, int64_t C,
-                long long* row_ptr_out, cudaStream_t st) {
-    if (C > 0) fill_kernel<<<(unsigned)((C + kFillWarps - 1) / kFillWarps), kFillWarps * 32, 0, st>>>(
+    if (C > 0) pairs_kernel<<<(unsigned)((C + kFillWarps - 1) / kFillWarps), kFillWarps * 32, 0, st>>>(
         pos, centers, C, g, h->d_grid, h->d_atom_cell, h->d_atom_wrap, h->d_cell_start, h->d_s_pos, h->d_s_wrap,
-        h->d_pair_ptr, h->cap_pairs, h->d_pair_tmp, h->d_pair_key, h->d_pair_row, h->d_row_count, h->d_self_row,
-        h->d_size_hist, h->d_size_cursor, C <= kOrderMaxCenters ? h->d_order : nullptr, h->d_counters);
-    scan_counts(h, h->d_row_count, row_ptr_out, C, &h->d_counters->n_rows, st);
+        h->cap_pairs, h->d_pair_tmp, h->d_pair_key, h->d_pair_row, h->d_pair_start, h->d_pair_count, h->d_row_count,
+        h->d_self_row, h->d_counters);
+    if (C <= kOrderMaxCenters) {
+        rows_order_kernel<<<1, 1024, 0, st>>>(h->d_row_count, h->d_pair_count, C, row_ptr_out, h->d_order, h->d_counters);
+    } else {
+        scan_counts(h, h->d_row_count, row_ptr_out, C, &h->d_counters->n_rows, st);
+    }
     CU(cudaGetLastError());
     return SOAP_OK;
 }
@@ -314,28 +308,34 @@ int check_inputs(soap_t* h, const float* pos, const int32_t* num, int64_t N, con
     return SOAP_OK;
 }
 
-// Plans scratch for a structure of this size: count, read the total back, grow.
+// Plans scratch for a structure of this size: run the search (with whatever capacity there is;
+// the counts come out right even when the pairs do not fit), read the totals back, grow.
 int plan(soap_t* h, const float* pos, const int32_t* num, int64_t N, const Geometry& g,
-         const int32_t* centers, int64_t C, cudaStream_t st, int64_t* n_pairs_out) {
+         const int32_t* centers, int64_t C, cudaStream_t st) {
     int rc = ensure_scratch(h, N, C, 0);
     if (rc) return rc;
-    rc = launch_count(h, pos, num, N, g, centers, C, st);
+    rc = launch_neighbors(h, pos, num, N, g, centers, C, h->d_row_ptr, st);
     if (rc) return rc;
     CU(cudaMemcpyAsync(h->h_counters, h->d_counters, sizeof(Counters), cudaMemcpyDeviceToHost, st));
     CU(cudaStreamSynchronize(st));
     const int64_t pairs = h->h_counters->n_pairs;
-    rc = ensure_scratch(h, N, C, pairs + pairs / 4 + 1024);
-    if (rc) return rc;
+    if (pairs > h->cap_pairs) {
+        rc = ensure_scratch(h, N, C, pairs + pairs / 4 + 1024);
+        if (rc) return rc;
+    }
+    // the planning run may have reported the shortage it was there to measure: forget that bit only
+    h->h_counters->status &= ~kStatusPairCapacity;
+    CU(cudaMemcpyAsync(&h->d_counters->status, &h->h_counters->status, sizeof(int), cudaMemcpyHostToDevice, st));
+    CU(cudaStreamSynchronize(st));
     h->planned_atoms = N;
     h->planned_centers = C;
-    if (n_pairs_out) *n_pairs_out = pairs;
     return SOAP_OK;
 }
 
 void fill_center_params(soap_t* h, CenterParams& cp, const float* pos, const int32_t* centers, int64_t C,
                         const Geometry& g, bool deriv) {
     cp.pos = pos; cp.centers = centers; cp.order = C <= kOrderMaxCenters ? h->d_order : nullptr; cp.species_idx = h->d_species_idx; cp.n_centers = C; cp.geom = g;
-    cp.pair_ptr = h->d_pair_ptr; cp.pair_key = h->d_pair_key; cp.pair_row = h->d_pair_row;
+    cp.pair_start = h->d_pair_start; cp.pair_count = h->d_pair_count; cp.pair_key = h->d_pair_key; cp.pair_row = h->d_pair_row;
     cp.row_ptr = h->d_row_ptr; cp.self_row = h->d_self_row;
     cp.pair_capacity = h->cap_pairs; cp.row_capacity = 0; cp.counters = h->d_counters;
     cp.table = h->d_table; cp.self_term = h->d_self; cp.anorm = h->d_anorm; cp.dfact = h->d_dfact; cp.kl = h->d_kl;
@@ -393,7 +393,7 @@ void soap_destroy(soap_t* h) {
     if (!h) return;
     void* ptrs[] = {h->d_table, h->d_self, h->d_anorm, h->d_dfact, h->d_kl, h->d_feat, h->d_zlut, h->d_inv_int, h->d_lm_of_t, h->d_l_of_lm, h->d_counters, h->d_bbox,
                     h->d_grid, h->d_species_idx, h->d_atom_cell, h->d_atom_wrap, h->d_s_wrap, h->d_s_pos, h->d_cell_count,
-                    h->d_cell_start, h->d_pair_count, h->d_row_count, h->d_self_row, h->d_order, h->d_pair_ptr, h->d_row_ptr, h->d_tile_sums, h->d_tile_offsets,
+                    h->d_cell_start, h->d_pair_count, h->d_row_count, h->d_self_row, h->d_order, h->d_pair_ptr, h->d_pair_start, h->d_row_ptr, h->d_tile_sums, h->d_tile_offsets,
                     h->d_pair_key, h->d_pair_tmp, h->d_pair_row};
     for (void* p : ptrs) if (p) cudaFree(p);
     if (h->h_counters) cudaFreeHost(h->h_counters);
@@ -434,9 +434,8 @@ int soap_neighbors(soap_t* h, const float* d_positions, const int32_t* d_numbers
     Geometry g;
     if ((rc = make_geometry(h, cell, g))) return rc;
     cudaStream_t st = (cudaStream_t)stream;
-    int64_t pairs = 0;
-    if ((rc = plan(h, d_positions, d_numbers, n_atoms, g, d_centers, n_centers, st, &pairs))) return rc;
-    if ((rc = launch_fill(h, d_positions, g, d_centers, n_centers, h->d_row_ptr, st))) return rc;
+    if ((rc = plan(h, d_positions, d_numbers, n_atoms, g, d_centers, n_centers, st))) return rc;
+    if ((rc = launch_neighbors(h, d_positions, d_numbers, n_atoms, g, d_centers, n_centers, h->d_row_ptr, st))) return rc;
     CU(cudaMemcpyAsync(h->h_counters, h->d_counters, sizeof(Counters), cudaMemcpyDeviceToHost, st));
     CU(cudaStreamSynchronize(st));
     h->last_centers = n_centers;
@@ -450,8 +449,10 @@ int soap_neighbor_list(soap_t* h, int64_t* d_pair_ptr, int32_t* d_pair_atom, int
     if (!h || !d_pair_ptr || !d_pair_atom || capacity_pairs < 0) return SOAP_ERR_INVALID_ARG;
     if (!h->tables_ready || h->planned_atoms < 0) return fail(h, SOAP_ERR_INVALID_ARG, "no neighbour list has been built yet");
     cudaStream_t st = (cudaStream_t)stream;
-    export_pairs_kernel<<<256, 256, 0, st>>>(h->d_pair_ptr, h->d_pair_key, h->last_centers, capacity_pairs,
-                                             (long long*)d_pair_ptr, d_pair_atom, d_pair_shift, h->d_counters);
+    // the pair arrays are addressed by segment: make the compact row pointers first, then gather
+    scan_counts(h, h->d_pair_count, (long long*)d_pair_ptr, h->last_centers, nullptr, st);
+    export_pairs_kernel<<<256, 256, 0, st>>>(h->d_pair_start, (const long long*)d_pair_ptr, h->d_pair_key, h->last_centers,
+                                             capacity_pairs, d_pair_atom, d_pair_shift, h->d_counters);
     CU(cudaGetLastError());
     return SOAP_OK;
 }
@@ -467,11 +468,9 @@ int soap_descriptor(soap_t* h, const float* d_positions, const int32_t* d_number
     cudaStream_t st = (cudaStream_t)stream;
     if (h->profiling) CU(cudaEventRecord(h->ev[0], st));
     if (h->planned_atoms != n_atoms || h->planned_centers != n_centers) {
-        if ((rc = plan(h, d_positions, d_numbers, n_atoms, g, d_centers, n_centers, st, nullptr))) return rc;
-    } else if ((rc = launch_count(h, d_positions, d_numbers, n_atoms, g, d_centers, n_centers, st))) {
-        return rc;
+        if ((rc = plan(h, d_positions, d_numbers, n_atoms, g, d_centers, n_centers, st))) return rc;
     }
-    if ((rc = launch_fill(h, d_positions, g, d_centers, n_centers, h->d_row_ptr, st))) return rc;
+    if ((rc = launch_neighbors(h, d_positions, d_numbers, n_atoms, g, d_centers, n_centers, h->d_row_ptr, st))) return rc;
     if (h->profiling) CU(cudaEventRecord(h->ev[1], st));
     h->last_centers = n_centers;
     if (n_centers > 0) {
@@ -497,11 +496,9 @@ int soap_derivatives(soap_t* h, const float* d_positions, const int32_t* d_numbe
     cudaStream_t st = (cudaStream_t)stream;
     if (h->profiling) CU(cudaEventRecord(h->ev[0], st));
     if (h->planned_atoms != n_atoms || h->planned_centers != n_centers) {
-        if ((rc = plan(h, d_positions, d_numbers, n_atoms, g, d_centers, n_centers, st, nullptr))) return rc;
-    } else if ((rc = launch_count(h, d_positions, d_numbers, n_atoms, g, d_centers, n_centers, st))) {
-        return rc;
+        if ((rc = plan(h, d_positions, d_numbers, n_atoms, g, d_centers, n_centers, st))) return rc;
     }
-    if ((rc = launch_fill(h, d_positions, g, d_centers, n_centers, (long long*)d_row_ptr, st))) return rc;
+    if ((rc = launch_neighbors(h, d_positions, d_numbers, n_atoms, g, d_centers, n_centers, (long long*)d_row_ptr, st))) return rc;
     if (h->profiling) CU(cudaEventRecord(h->ev[1], st));
     h->last_centers = n_centers;
     if (n_centers > 0) {
@@ -624,12 +621,12 @@ int soap_neighbor_counts_static(const float* d_positions, int64_t n_atoms, doubl
     if ((e = cudaMemsetAsync(base, 0, StaticLayout::header, st)) != cudaSuccess) return say(SOAP_ERR_CUDA, cudaGetErrorString(e));
     if ((e = cudaMemsetAsync(cell_count, 0, sizeof(int) * (kStaticMaxCells + 1), st)) != cudaSuccess) return say(SOAP_ERR_CUDA, cudaGetErrorString(e));
     bbox_only_kernel<<<blocks_for(N, 256, 256), 256, 0, st>>>(d_positions, N, g, bbox);
-    grid_setup_kernel<<<1, 1, 0, st>>>(bbox, g, N, kStaticMaxCells, grid);
+    grid_setup_kernel<<<1, 1, 0, st>>>(bbox, g, N, kStaticMaxCells, grid, nullptr);
     bin_count_kernel<<<blocks_for(N, 256), 256, 0, st>>>(d_positions, N, g, grid, atom_cell, atom_wrap, cell_count, counters);
     scan_kernel<int><<<1, 1024, 0, st>>>(cell_count, cell_start, kStaticMaxCells, nullptr, &grid->n_cells);
     bin_fill_kernel<<<blocks_for(N, 256), 256, 0, st>>>(d_positions, N, atom_cell, atom_wrap, cell_start, cell_count, s_pos, s_wrap);
     count_kernel<<<(unsigned)((N + 7) / 8), 256, 0, st>>>(d_positions, nullptr, N, g, grid, atom_cell, atom_wrap, cell_start, s_pos, s_wrap,
-                                                         d_counts, nullptr, counters);
+                                                         d_counts, counters);
     if ((e = cudaGetLastError()) != cudaSuccess) return say(SOAP_ERR_CUDA, cudaGetErrorString(e));
     return SOAP_OK;
 }

@@ -56,7 +56,8 @@ struct CenterParams {
     long long n_centers;
     Geometry geom;
     // neighbour data
-    const long long* pair_ptr;    // [C+1]
+    const long long* pair_start;  // [C] first pair of the centre's segment
+    const int* pair_count;        // [C]
     const unsigned long long* pair_key;
     const int* pair_row;
     const long long* row_ptr;     // [C+1]
