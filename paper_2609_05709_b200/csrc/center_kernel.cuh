@@ -32,6 +32,9 @@
 #ifndef SOAP_MIN_CTAS_DERIV
 #define SOAP_MIN_CTAS_DERIV 3          // resident CTAs per SM the derivative kernel is compiled for
 #endif
+#ifndef SOAP_MIN_CTAS_DESC
+#define SOAP_MIN_CTAS_DESC 6           // ... and the descriptor-only kernel (latency-bound: more warps help)
+#endif
 
 namespace soap {
 
@@ -104,7 +107,7 @@ __device__ __forceinline__ void harmonics_column(int L, int m, float x, float y,
 }
 
 template <bool DERIV, int L, int NMAX_T>
-__global__ void __launch_bounds__(kThreads, DERIV ? SOAP_MIN_CTAS_DERIV : 4)
+__global__ void __launch_bounds__(kThreads, DERIV ? SOAP_MIN_CTAS_DERIV : SOAP_MIN_CTAS_DESC)
 center_kernel(const CenterParams p) {
     constexpr int L1 = L + 1, LM = L1 * L1, LMP = LM | 1;      // odd row stride: no shared-memory bank conflicts
     constexpr int NMAX_BOUND = NMAX_T ? NMAX_T : 16;

@@ -57,8 +57,8 @@ struct soap_handle {
     // device state (created on first use)
     int device = -1;
     bool tables_ready = false;
-    float *d_table = nullptr, *d_self = nullptr, *d_anorm = nullptr, *d_dfact = nullptr, *d_kl = nullptr, *d_inv_int = nullptr;
-    int *d_feat = nullptr, *d_zlut = nullptr, *d_lm_of_t = nullptr, *d_l_of_lm = nullptr;
+    float *d_table = nullptr, *d_self = nullptr, *d_kl = nullptr;
+    int *d_feat = nullptr, *d_zlut = nullptr, *d_l_of_lm = nullptr;
     Counters* d_counters = nullptr;
     unsigned long long* d_bbox = nullptr;   // 6 words of bounding box (structures above 16384 atoms)
     int* d_order = nullptr;
@@ -155,20 +155,12 @@ int ensure_device(soap_t* h) {
     h->device = dev;
     CU(upload(&h->d_table, h->basis.table));
     CU(upload(&h->d_self, h->basis.self_term));
-    CU(upload(&h->d_anorm, h->basis.anorm));
-    CU(upload(&h->d_dfact, h->basis.dfact));
     CU(upload(&h->d_kl, h->basis.kl));
     CU(upload(&h->d_feat, h->feat_pack));
     {
-        std::vector<float> inv(32, 0.f);
-        for (int k = 1; k < 32; ++k) inv[k] = 1.0f / k;
-        CU(upload(&h->d_inv_int, inv));
-        std::vector<int> lm_of_t, l_of_lm;
-        for (int l = 0; l <= h->l_max; ++l) {
-            for (int m = 0; m <= l; ++m) lm_of_t.push_back((l << 4) | m);
+        std::vector<int> l_of_lm;
+        for (int l = 0; l <= h->l_max; ++l)
             for (int m = -l; m <= l; ++m) l_of_lm.push_back(l);
-        }
-        CU(upload(&h->d_lm_of_t, lm_of_t));
         CU(upload(&h->d_l_of_lm, l_of_lm));
     }
     std::vector<int> lut(128, -1);
@@ -338,8 +330,7 @@ void fill_center_params(soap_t* h, CenterParams& cp, const float* pos, const int
     cp.pair_start = h->d_pair_start; cp.pair_count = h->d_pair_count; cp.pair_key = h->d_pair_key; cp.pair_row = h->d_pair_row;
     cp.row_ptr = h->d_row_ptr; cp.self_row = h->d_self_row;
     cp.pair_capacity = h->cap_pairs; cp.row_capacity = 0; cp.counters = h->d_counters;
-    cp.table = h->d_table; cp.self_term = h->d_self; cp.anorm = h->d_anorm; cp.dfact = h->d_dfact; cp.kl = h->d_kl;
-    cp.inv_int = h->d_inv_int; cp.lm_of_t = h->d_lm_of_t; cp.l_of_lm = h->d_l_of_lm;
+    cp.table = h->d_table; cp.self_term = h->d_self; cp.kl = h->d_kl; cp.l_of_lm = h->d_l_of_lm;
     cp.feat_pack = h->d_feat; cp.nch_magic = (unsigned)((1ull << 32) / (unsigned)(h->n_max * (h->l_max + 1))) + 1u; cp.inv_h = (float)h->basis.inv_h; cp.n_intervals = h->basis.n_intervals;
     cp.S = h->S; cp.n_max = h->n_max; cp.l_max = h->l_max; cp.F = (int)h->F;
     cp.P = deriv ? h->P_deriv : h->P_desc;
@@ -391,7 +382,7 @@ int soap_create(soap_t** out, const int32_t* species, int n_species, double r_cu
 
 void soap_destroy(soap_t* h) {
     if (!h) return;
-    void* ptrs[] = {h->d_table, h->d_self, h->d_anorm, h->d_dfact, h->d_kl, h->d_feat, h->d_zlut, h->d_inv_int, h->d_lm_of_t, h->d_l_of_lm, h->d_counters, h->d_bbox,
+    void* ptrs[] = {h->d_table, h->d_self, h->d_kl, h->d_feat, h->d_zlut, h->d_l_of_lm, h->d_counters, h->d_bbox,
                     h->d_grid, h->d_species_idx, h->d_atom_cell, h->d_atom_wrap, h->d_s_wrap, h->d_s_pos, h->d_cell_count,
                     h->d_cell_start, h->d_pair_count, h->d_row_count, h->d_self_row, h->d_order, h->d_pair_ptr, h->d_pair_start, h->d_row_ptr, h->d_tile_sums, h->d_tile_offsets,
                     h->d_pair_key, h->d_pair_tmp, h->d_pair_row};

@@ -9,8 +9,7 @@ namespace soap {
 constexpr int kMaxSpecies = 8;
 constexpr int kThreads = 256;            // CTA size of the per-centre kernels
 constexpr int kWarps = kThreads / 32;
-constexpr int kMaxElemPerThread = 8;     // n_max (l_max+1)^2 / kThreads rounded up: 16*169/256 -> 11 is refused at create
-constexpr int kMaxChanRounds = 7;        // n_max (l_max+1) / 32 rounded up: 16*13/32
+constexpr int kMaxElemPerThread = 8;     // soap_create refuses n_max (l_max+1)^2 > 8 * kThreads (shared-memory budget of the tiles)
 
 // status bits (device, sticky until soap_status)
 constexpr int kStatusUnknownSpecies = 1;
@@ -67,10 +66,6 @@ struct CenterParams {
     // basis
     const float* table;           // [nint][n_ch][6]
     const float* self_term;       // [n_max]
-    const float* anorm;           // [(l,m)] harmonic normalisation
-    const float* dfact;           // [m] (2m-1)!!
-    const float* inv_int;         // [k] 1/k
-    const int* lm_of_t;           // [(l,m) index] -> l<<4 | m
     const int* l_of_lm;           // [lm] -> l
     const float* kl;
     const int* feat_pack;         // [F] n | n'<<5 | mu<<10 | nu<<14 | l<<18
