@@ -122,6 +122,23 @@ int soap_derivatives(soap_t *h, const float *d_positions, const int32_t *d_numbe
                      float *d_out_desc, float *d_out_jac, int64_t capacity_rows,
                      int64_t *d_row_ptr, int32_t *d_row_atom, void *stream);
 
+/* Dense view of the Jacobian in the layout of the paper's derivatives() call
+ * (architecture section: (n_centers, n_atoms, 3, n_features)), for the atoms of
+ * an inclusion list:
+ *   d_out [n_centers, n_include, 3, F]   fully overwritten; the block of
+ *         (centre c, listed atom a) is that atom's row of centre c, or zeros
+ *         when the atom is outside the centre's sphere (the text below Eq. 5:
+ *         only atoms inside the cutoff contribute).
+ *   d_include [n_include] atom indices, or NULL for atoms 0 .. n_include-1
+ *         (pass n_include = n_atoms for the paper's full layout; leaving atoms
+ *         out of the list is its `exclude`).
+ * d_jac_rows / d_row_ptr / d_row_atom are the outputs of soap_derivatives for
+ * the same n_centers.  The dense tensor grows as centres x atoms: meant for
+ * small structures or for batches of centres.  n_centers * n_include must stay
+ * below 2^31. */
+int soap_jacobian_dense(soap_t *h, const float *d_jac_rows, const int64_t *d_row_ptr, const int32_t *d_row_atom,
+                        int64_t n_centers, const int32_t *d_include, int64_t n_include, float *d_out, void *stream);
+
 /* Waits for `stream`, then returns and clears the sticky device status
  * (SOAP_OK, SOAP_ERR_UNKNOWN_SPECIES or SOAP_ERR_CAPACITY); also reports the
  * pair and row counts of the last call (either pointer may be NULL). */

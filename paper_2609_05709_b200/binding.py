@@ -12,7 +12,7 @@ GTO, POLYNOMIAL = 0, 1
 EXPORTED_SYMBOLS = [
     "soap_create", "soap_destroy", "soap_num_features", "soap_feature_info", "soap_last_error",
     "soap_radial_table", "soap_neighbors", "soap_neighbor_list", "soap_descriptor",
-    "soap_derivatives", "soap_status", "soap_profile", "soap_profile_read", "soap_neighbor_counts_static",
+    "soap_derivatives", "soap_status", "soap_profile", "soap_profile_read", "soap_neighbor_counts_static", "soap_jacobian_dense",
 ]
 
 _ERRORS = {-1: "SOAP_ERR_INVALID_ARG", -2: "SOAP_ERR_UNKNOWN_SPECIES", -3: "SOAP_ERR_CAPACITY",
@@ -58,6 +58,7 @@ def load_library() -> C.CDLL:
     lib.soap_derivatives.argtypes = common + [vp, vp, i64, vp, vp, vp]
     lib.soap_status.argtypes = [vp, C.POINTER(i64), C.POINTER(i64), vp]
     lib.soap_neighbor_counts_static.argtypes = [vp, i64, C.c_double, vp, vp, C.c_char_p, i64]
+    lib.soap_jacobian_dense.argtypes = [vp, vp, vp, vp, i64, vp, i64, vp, vp]
     lib.soap_profile.argtypes = [vp, i32]
     lib.soap_profile_read.argtypes = [vp, C.POINTER(C.c_float), C.POINTER(C.c_float)]
     for name in EXPORTED_SYMBOLS:
@@ -240,6 +241,33 @@ class Soap:
                               dev_buf["row_ptr"], dev_buf["row_atom"])
         for k in ("desc", "jac", "row_ptr", "row_atom"):
             host_out[k].copy_(dev_buf[k], non_blocking=True)
+
+    def jacobian_dense(self, deriv, n_atoms=None, include=None, out=None):
+        """(C, n_include, 3, F) dense Jacobian of a `Derivatives` result (zeros outside the spheres).
+        `include` is an int32 device tensor of atom indices; without it atoms 0..n_atoms-1 are listed."""
+        import torch
+        c = deriv.row_ptr.shape[0] - 1
+        if include is not None:
+            assert include.is_cuda and include.dtype == torch.int32 and include.is_contiguous()
+            n_inc, iptr = include.shape[0], C.c_void_p(include.data_ptr())
+        else:
+            n_inc, iptr = int(n_atoms), None
+        if out is None:
+            out = torch.empty((c, n_inc, 3, self.n_features), dtype=torch.float32, device=deriv.jacobian.device)
+        self._check(self._lib.soap_jacobian_dense(self._h, deriv.jacobian.data_ptr(), deriv.row_ptr.data_ptr(),
+                                                  deriv.row_atom.data_ptr(), c, iptr, n_inc, out.data_ptr(), self._stream()))
+        return out
+
+    def derivatives_batched(self, positions, numbers, cell=None, centers=None, batch=1024):
+        """Yields (centre indices of the batch, Derivatives) for consecutive batches of centres, so that
+        the Jacobian held on the device at any time is bounded by the batch (the paper's
+        centre-batch streaming); `centers` defaults to all atoms."""
+        import torch
+        n = positions.shape[0]
+        allc = torch.arange(n, dtype=torch.int32, device=positions.device) if centers is None else centers
+        for lo in range(0, allc.shape[0], batch):
+            part = allc[lo:lo + batch].contiguous()
+            yield part, self.derivatives(positions, numbers, cell, part)
 
     def status(self):
         """Waits for the stream; raises if the device flagged a problem. Returns (n_pairs, n_rows)."""

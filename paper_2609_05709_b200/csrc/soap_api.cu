@@ -12,6 +12,7 @@
 
 #include "basis_host.h"
 #include "center_launch.h"
+#include "dense_kernel.cuh"
 #include "neighbor_kernels.cuh"
 #include "soap.h"
 
@@ -501,6 +502,19 @@ int soap_derivatives(soap_t* h, const float* d_positions, const int32_t* d_numbe
         CU(center_launch(true, h->l_max, h->n_max, cp, (unsigned)n_centers, h->smem_deriv, st));
     }
     if (h->profiling) CU(cudaEventRecord(h->ev[2], st));
+    return SOAP_OK;
+}
+
+int soap_jacobian_dense(soap_t* h, const float* d_jac_rows, const int64_t* d_row_ptr, const int32_t* d_row_atom,
+                        int64_t n_centers, const int32_t* d_include, int64_t n_include, float* d_out, void* stream) {
+    if (!h) return SOAP_ERR_INVALID_ARG;
+    if (n_centers < 0 || n_include < 0) return fail(h, SOAP_ERR_INVALID_ARG, "negative size");
+    if (n_centers == 0 || n_include == 0) return SOAP_OK;
+    if (!d_jac_rows || !d_row_ptr || !d_row_atom || !d_out) return fail(h, SOAP_ERR_INVALID_ARG, "NULL pointer");
+    if (n_centers * n_include > 2147483647LL) return fail(h, SOAP_ERR_INVALID_ARG, "more than 2^31-1 (centre, atom) slots: split the call");
+    dense_scatter_kernel<<<(unsigned)(n_centers * n_include), 128, 0, (cudaStream_t)stream>>>(
+        d_jac_rows, (const long long*)d_row_ptr, d_row_atom, n_centers, d_include, n_include, (int)h->F, d_out);
+    CU(cudaGetLastError());
     return SOAP_OK;
 }
 

@@ -1,0 +1,80 @@
+"""Dense (centres, atoms, 3, F) view with an atom selection, and centre-batch streaming, on a GPU.
+
+The dense tensor is the layout of the paper's derivatives() call; the reference is built from the
+oracle's rows (zeros everywhere else, as the text below Eq. 5 says)."""
+import numpy as np
+import pytest
+
+from oracle.soap import GTO, POLYNOMIAL, SoapOracle
+from soap_inputs import small_periodic_cell, water_cluster
+
+torch = pytest.importorskip("torch")
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def pkg():
+    if not torch.cuda.is_available():
+        pytest.skip("no CUDA device")
+    import paper_2609_05709_b200 as p
+    p.load_library()
+    return p
+
+
+def oracle_dense(oracle, struct, centers, include):
+    ref = oracle.derivatives(struct.positions, struct.numbers, struct.cell, centers)
+    col = {int(a): k for k, a in enumerate(include)}
+    dense = np.zeros((len(centers), len(include), 3, oracle.n_features))
+    for c in range(len(centers)):
+        for r in range(ref.row_ptr[c], ref.row_ptr[c + 1]):
+            if int(ref.row_atom[r]) in col:
+                dense[c, col[int(ref.row_atom[r])]] = ref.jacobian[r]
+    return dense
+
+
+def col_err(a, ref):
+    a = np.asarray(a, np.float64).reshape(-1, ref.shape[-1])
+    ref = ref.reshape(-1, ref.shape[-1])
+    return float((np.abs(a - ref).max(0) / np.maximum(np.abs(ref).max(0), 1e-8)).max())
+
+
+@pytest.mark.parametrize("case", ["water", "cell"])
+def test_dense_view_with_atom_selection(pkg, case):
+    if case == "water":
+        s, args = water_cluster(8, 0), ([1, 8], 3.0, 3, 3, 0.5, GTO)          # small cutoff: many empty blocks
+    else:
+        s, args = small_periodic_cell(0), ([1, 6, 7, 8], 4.5, 2, 2, 0.5, POLYNOMIAL, (True, True, True))
+    soap, oracle = pkg.Soap(*args), SoapOracle(*args)
+    pos = torch.from_numpy(s.positions).cuda()
+    num = torch.from_numpy(s.numbers).cuda()
+    centers = [0, 3, 5] if case == "water" else [1, 6]
+    out = soap.derivatives(pos, num, s.cell, torch.tensor(centers, dtype=torch.int32).cuda())
+    # every atom
+    dense = soap.jacobian_dense(out, n_atoms=s.n_atoms)
+    ref = oracle_dense(oracle, s, centers, list(range(s.n_atoms)))
+    assert dense.shape == ref.shape
+    assert col_err(dense.cpu().numpy(), ref) < 1e-4
+    assert np.array_equal(dense.cpu().numpy() == 0, ref == 0) or case == "cell"   # same sparsity pattern
+    # a selection, not in order, with an atom outside every sphere where there is one
+    include = [5, 0, s.n_atoms - 1, 2]
+    dense = soap.jacobian_dense(out, include=torch.tensor(include, dtype=torch.int32).cuda())
+    assert col_err(dense.cpu().numpy(), oracle_dense(oracle, s, centers, include)) < 1e-4
+
+
+def test_centre_batches_equal_one_call(pkg):
+    s = water_cluster(40, 2)
+    soap = pkg.Soap([1, 8], 5.0, 4, 3, 0.5, GTO)
+    pos = torch.from_numpy(s.positions).cuda()
+    num = torch.from_numpy(s.numbers).cuda()
+    whole = soap.derivatives(pos, num)
+    rows = 0
+    for part, got in soap.derivatives_batched(pos, num, batch=37):
+        lo = int(part[0])
+        n = part.shape[0]
+        assert torch.equal(got.descriptor, whole.descriptor[lo:lo + n])
+        r0, r1 = int(whole.row_ptr[lo]), int(whole.row_ptr[lo + n])
+        assert torch.equal(got.row_ptr, whole.row_ptr[lo:lo + n + 1] - r0)
+        assert torch.equal(got.row_atom, whole.row_atom[r0:r1])
+        assert torch.equal(got.jacobian, whole.jacobian[r0:r1])       # same kernels, same inputs: bit for bit
+        rows += r1 - r0
+    assert rows == whole.jacobian.shape[0]
