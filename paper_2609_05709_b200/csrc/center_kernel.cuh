@@ -345,7 +345,42 @@ center_kernel(const CenterParams p) {
         int gp = ((lay.total - lay.sSD) / NV) / L1;                         // groups per slab
         gp = gp < 1 ? 1 : (gp > NP ? NP : gp);
         const bool staged = (lay.total - lay.sSD) >= NV * L1 && !(SOAP_DEBUG_SKIP & 8);
-        for (int q0 = 0; q0 < ((SOAP_DEBUG_SKIP & 8) ? 0 : NP); q0 += gp) {
+        // Descriptor-only build, whole row fits the staging area: a thread takes one (species pair, l, n)
+        // and all n' at once, so each coefficient of the n side is loaded once per m for the whole
+        // group (the generic loop below loads two operands per multiply-add).
+        const bool grouped = !DERIV && (lay.total - lay.sSD) >= F && !(SOAP_DEBUG_SKIP & 8);
+        if (grouped) {
+            const int NB = S * (S + 1) / 2;
+            for (int it = tid; it < NB * L1 * NMAX; it += kThreads) {
+                const int n1 = it % NMAX, rest = it / NMAX, b = rest % NB, l = rest / NB;   // l slowest: warps share 2l+1
+                int mu = 0, nu = 0, boff = 0;                                                // block b -> (mu, nu), feature offset
+                for (int k = 0, a2 = 0; a2 < S; ++a2)
+                    for (int b2 = a2; b2 < S; ++b2, ++k) {
+                        if (k == b) { mu = a2; nu = b2; }
+                        if (k < b) boff += (a2 == b2) ? (NMAX * (NMAX + 1) / 2) * L1 : NMAX * NCH;
+                    }
+                const int n2_lo = (mu == nu) ? n1 : 0;
+                const float* ar = c_t + (mu * NMAX + n1) * LMP + l * l;
+                const float* br = c_t + nu * NMAX * LMP + l * l;
+                float acc[NMAX_BOUND];
+#pragma unroll
+                for (int n2 = 0; n2 < NMAX_BOUND; ++n2) acc[n2] = 0.f;
+                for (int m = 0; m <= 2 * l; ++m) {
+                    const float ca = ar[m];
+#pragma unroll
+                    for (int n2 = 0; n2 < NMAX_BOUND; ++n2)
+                        if (n2 < NMAX && n2 >= n2_lo) acc[n2] = fmaf(ca, br[n2 * LMP + m], acc[n2]);
+                }
+                const float kl = __ldg(p.kl + l);
+                const int base = (mu == nu) ? boff + (n1 * NMAX - n1 * (n1 + 1) / 2) * L1 + l : boff + n1 * NCH + l;
+#pragma unroll
+                for (int n2 = 0; n2 < NMAX_BOUND; ++n2)
+                    if (n2 < NMAX && n2 >= n2_lo) slab[base + n2 * L1] = kl * acc[n2];
+            }
+            __syncthreads();
+            for (int e = tid; e < F; e += kThreads) desc_row[e] = slab[e];
+        }
+        for (int q0 = 0; q0 < ((SOAP_DEBUG_SKIP & 8) || grouped ? 0 : NP); q0 += gp) {
             const int nq = min(gp, NP - q0), nf = nq * L1, f0 = q0 * L1;
             for (int g = tid; g < nf; g += kThreads) {
                 const int l = g / nq, fl = (g - l * nq) * L1 + l;             // feature index inside the slab
