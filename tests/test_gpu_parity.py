@@ -211,6 +211,30 @@ def test_device_side_errors_are_reported(pkg):
         per.descriptor(pos, num)
 
 
+def test_denser_structure_than_planned_is_reported_and_replanned(pkg):
+    """Scratch is planned from the first structure of a given size; a later structure of the same
+    size with more pairs than the plan's headroom must be flagged, and planning again must fix it."""
+    loose = water_cluster(60, 0)
+    dense = water_cluster(60, 0)
+    dense.positions = (dense.positions * 0.6).astype(np.float32)          # same atoms, 4.6x the density
+    args = ([1, 8], 5.0, 3, 2, 0.5, GTO)
+    soap, oracle = pkg.Soap(*args), SoapOracle(*args)
+    num = torch.from_numpy(loose.numbers).cuda()
+    soap.descriptor(torch.from_numpy(loose.positions).cuda(), num)
+    p_loose, _ = soap.status()
+    pos_dense = torch.from_numpy(dense.positions).cuda()
+    soap.descriptor(pos_dense, num)                                       # same sizes: no new plan
+    with pytest.raises(pkg.SoapError) as e:
+        soap.status()
+    assert e.value.code == -3
+    p_dense, _ = soap.neighbors(pos_dense, num)                           # plans again
+    assert p_dense > 1.25 * p_loose + 1024
+    d = soap.descriptor(pos_dense, num)
+    soap.status()
+    ref = oracle.descriptor(dense.positions, dense.numbers, None, [0, 77, 179])
+    assert col_err(d[[0, 77, 179]].cpu().numpy(), ref, 0) < DESC_TOL
+
+
 def test_empty_structure(pkg):
     soap = pkg.Soap([1, 8], 5.0, 2, 2, 0.5)
     pos = torch.empty((0, 3), dtype=torch.float32, device="cuda")
