@@ -371,8 +371,8 @@ def run_suite(args):
                 r = time_case(s, [1, 8], 6.0, n_max, l_max, 0.5, 0, "derivatives", steps)
                 r["case"] = "map"
                 print(json.dumps(r), flush=True)
-    elif args.suite == "scaling":
-        for n_mol in (1000, 10000, 100000, 333334):
+    elif args.suite in ("scaling", "desc30k"):
+        for n_mol in ((10000,) if args.suite == "desc30k" else (1000, 10000, 100000, 333334)):
             s = water_cluster(n_mol, 0)
             r = time_case(s, [1, 8], 5.0, 8, 6, 0.5, 0, "descriptor", steps)
             r["case"] = "scaling"
@@ -396,10 +396,11 @@ def main():
     ap.add_argument("--workload", default=DEFAULT_WORKLOAD, choices=sorted(WORKLOADS))
     ap.add_argument("--kernel-only", action="store_true",
                     help="skip the end-to-end and CPU-baseline legs (for profiler captures)")
-    ap.add_argument("--suite", choices=["map", "scaling", "configs"],
+    ap.add_argument("--suite", choices=["map", "scaling", "configs", "desc30k"],
                     help="extra measurements beside the headline line: 'map' = descriptor+Jacobian over "
                          "n_max x l_max on the 1000-molecule cluster, 'scaling' = descriptor-only on "
-                         "3k..1M atoms, 'configs' = the periodic multi-species box and the tiny cluster; "
+                         "3k..1M atoms, 'configs' = the periodic multi-species box and the tiny cluster, "
+                         "'desc30k' = descriptor-only on 30,000 atoms alone (small enough for profiler captures); "
                          "prints one JSON line per case")
     args = ap.parse_args()
     if args.impl == "reference":
