@@ -32,4 +32,14 @@ Parity status of each function (what pins it, in tests/test_oracle_*.py):
 * soap.feature_table ....................................... the ORDER of the
   features rests on a reading of the paper's sentence on the nested loops
   (species pair, radial triangle, l fastest); the values do not depend on it.
+  With crossover off the table is the mu == nu subset (checked against the
+  full table).
+* modes.coefficient_vector / coefficient_derivatives ....... pinned
+  (the pinned coefficient routine, central finite differences of it, zero
+  row sums, zero blocks of foreign species); the ORDER of the coefficient
+  index (species, n, l, m) is a reading, the paper names none.
+* modes.average_descriptor / average_derivatives ........... pinned
+  (bilinear double sum over centre pairs for the inner average, one-centre
+  and translation-equivalent-centre reductions to the plain descriptor,
+  rotation / permutation invariance, central finite differences)
 """

@@ -32,7 +32,8 @@ class Derivatives:
 
 
 class SoapOracle:
-    def __init__(self, species, r_cut, n_max, l_max, sigma, rbf=GTO, pbc=(False, False, False)):
+    def __init__(self, species, r_cut, n_max, l_max, sigma, rbf=GTO, pbc=(False, False, False), crossover=True):
+        self.crossover = bool(crossover)
         self.species = sorted(int(z) for z in species)
         self.r_cut, self.n_max, self.l_max, self.sigma = float(r_cut), int(n_max), int(l_max), float(sigma)
         self.rbf = int(rbf)
@@ -47,10 +48,12 @@ class SoapOracle:
     def feature_table(self) -> np.ndarray:
         """Rows (mu, nu, n, n', l) in output order: species pairs mu <= nu,
         then the radial pair (n' >= n when mu == nu, every (n, n') otherwise),
-        then l fastest."""
+        then l fastest.  With `crossover` off only the pairs mu == nu are kept
+        (the constructor flag that decides whether off-diagonal species pairs
+        are retained)."""
         rows = []
         for mu in range(self.S):
-            for nu in range(mu, self.S):
+            for nu in range(mu, self.S if self.crossover else mu + 1):
                 for n in range(self.n_max):
                     for n2 in range(n if mu == nu else 0, self.n_max):
                         for l in range(self.l_max + 1):

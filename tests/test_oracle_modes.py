@@ -1,0 +1,121 @@
+"""Pins for the oracle's coefficient mode, averaged modes and the crossover flag."""
+import numpy as np
+import pytest
+
+from oracle import modes
+from oracle.soap import GTO, POLYNOMIAL, SoapOracle
+from soap_inputs import random_rotation, small_periodic_cell, water_cluster
+
+
+def _fd(fun, pos, h=1e-5):
+    """Central differences of fun(pos) with respect to every coordinate: (N, 3, ...)."""
+    out = []
+    for j in range(pos.shape[0]):
+        row = []
+        for k in range(3):
+            p1, p2 = pos.copy(), pos.copy()
+            p1[j, k] += h
+            p2[j, k] -= h
+            row.append((fun(p1) - fun(p2)) / (2 * h))
+        out.append(row)
+    return np.array(out)
+
+
+def test_crossover_off_keeps_exactly_the_same_species_blocks():
+    st = water_cluster(3, seed=5)
+    pos = st.positions.astype(np.float64)
+    full = SoapOracle([1, 8], 4.0, 3, 2, 0.5)
+    diag = SoapOracle([1, 8], 4.0, 3, 2, 0.5, crossover=False)
+    keep = np.nonzero(full.table[:, 0] == full.table[:, 1])[0]
+    assert diag.n_features == 2 * (3 * 4 // 2) * 3 == keep.size
+    assert np.array_equal(diag.table, full.table[keep])
+    a, b = full.derivatives(pos, st.numbers), diag.derivatives(pos, st.numbers)
+    assert np.array_equal(a.descriptor[:, keep], b.descriptor)
+    assert np.array_equal(a.row_atom, b.row_atom)
+    np.testing.assert_allclose(b.jacobian, a.jacobian[:, :, keep], rtol=0, atol=1e-15)
+
+
+@pytest.mark.parametrize("rbf", [GTO, POLYNOMIAL])
+def test_coefficient_jacobian_by_central_differences(rbf):
+    st = small_periodic_cell(seed=2, pbc=(True, True, False))      # short axes: images of the centre itself occur
+    pos = st.positions.astype(np.float64)
+    o = SoapOracle([1, 6, 7, 8], 4.2, 3, 3, 0.5, rbf, pbc=st.pbc)
+    der = modes.coefficient_derivatives(o, pos, st.numbers, st.cell)
+    dense = modes._dense(der, pos.shape[0])                        # [C, N, 3, W]
+    fd = _fd(lambda p: modes.coefficient_vector(o, p, st.numbers, st.cell), pos)   # [N, 3, C, W]
+    np.testing.assert_allclose(dense, np.transpose(fd, (2, 0, 1, 3)), rtol=0, atol=2e-8 * np.abs(dense).max())
+    # a rigid translation changes nothing: the rows of a centre sum to zero
+    assert np.abs(dense.sum(axis=1)).max() < 1e-12 * np.abs(dense).max()
+    # the descriptor of the coefficient mode is the pinned coefficient routine, flattened
+    np.testing.assert_array_equal(der.descriptor[3], o.coefficients(pos, st.numbers, st.cell, 3).reshape(-1))
+
+
+def test_coefficient_block_of_another_species_stays_zero():
+    pos = np.array([[0.0, 0.0, 0.0], [1.0, 0.2, -0.3], [-0.8, 1.1, 0.4]])
+    numbers = np.array([8, 1, 1])
+    o = SoapOracle([1, 8], 3.0, 2, 2, 0.4)
+    der = modes.coefficient_derivatives(o, pos, numbers, centers=[0])
+    J = der.jacobian.reshape(3, 3, 2, 2, 9)                        # rows: atoms 0, 1, 2
+    assert np.all(J[1:, :, 1] == 0) and np.abs(J[1:, :, 0]).max() > 0     # hydrogens move only the H block
+    assert np.all(J[0, :, 1] == 0)                                        # the O block holds the on-site constant only
+
+
+@pytest.mark.parametrize("mode", ["inner", "outer"])
+@pytest.mark.parametrize("rbf", [GTO, POLYNOMIAL])
+def test_averaged_jacobian_by_central_differences(mode, rbf):
+    st = small_periodic_cell(seed=4, pbc=(True, False, True))
+    pos = st.positions.astype(np.float64)
+    o = SoapOracle([1, 6, 7, 8], 4.0, 2, 3, 0.45, rbf, pbc=st.pbc)
+    centers = [0, 2, 3, 7]
+    desc, jac = modes.average_derivatives(o, mode, pos, st.numbers, st.cell, centers)
+    np.testing.assert_allclose(desc, modes.average_descriptor(o, mode, pos, st.numbers, st.cell, centers), rtol=1e-13)
+    fd = _fd(lambda p: modes.average_descriptor(o, mode, p, st.numbers, st.cell, centers), pos)
+    np.testing.assert_allclose(jac, fd, rtol=0, atol=3e-8 * np.abs(jac).max())
+    assert np.abs(jac.sum(axis=0)).max() < 1e-11 * np.abs(jac).max()
+
+
+def test_inner_average_is_the_mean_cross_power_spectrum():
+    """Eq. 4 is bilinear, so contracting the mean coefficients equals the mean over all ordered
+    pairs of centres (i, i') of K_l sum_m c_i c_i'."""
+    st = water_cluster(2, seed=9)
+    pos = st.positions.astype(np.float64)
+    o = SoapOracle([1, 8], 3.5, 2, 2, 0.5)
+    cs = [o.coefficients(pos, st.numbers, None, i) for i in range(6)]
+    acc = np.zeros(o.n_features)
+    for a in cs:
+        for b in cs:
+            for f, (mu, nu, n, n2, l) in enumerate(o.table):
+                sl = slice(l * l, (l + 1) ** 2)
+                acc[f] += np.pi * np.sqrt(8.0 / (2 * l + 1)) * np.dot(a[mu, n, sl], b[nu, n2, sl])
+    np.testing.assert_allclose(modes.average_descriptor(o, "inner", pos, st.numbers), acc / 36, rtol=1e-12)
+
+
+@pytest.mark.parametrize("mode", ["inner", "outer"])
+def test_averages_reduce_to_the_plain_descriptor(mode):
+    # one centre: nothing to average
+    st = water_cluster(3, seed=1)
+    pos = st.positions.astype(np.float64)
+    o = SoapOracle([1, 8], 4.0, 3, 2, 0.5)
+    plain = o.derivatives(pos, st.numbers, centers=[4])
+    desc, jac = modes.average_derivatives(o, mode, pos, st.numbers, centers=[4])
+    np.testing.assert_allclose(desc, plain.descriptor[0], rtol=1e-13)
+    np.testing.assert_allclose(jac, modes._dense(plain, pos.shape[0])[0], rtol=0, atol=1e-14)
+    # two atoms related by a lattice translation of half the doubled cell see the same environment
+    cell = np.diag([3.0, 3.2, 6.8])
+    p2 = np.array([[0.1, 0.2, 0.3], [0.1, 0.2, 3.7], [1.4, 1.9, 1.2], [1.4, 1.9, 4.6]])
+    z2 = np.array([8, 8, 1, 1])
+    op = SoapOracle([1, 8], 3.3, 2, 3, 0.5, pbc=(True, True, True))
+    np.testing.assert_allclose(modes.average_descriptor(op, mode, p2, z2, cell, [0, 1]),
+                               op.descriptor(p2, z2, cell, [0])[0], rtol=1e-12)
+
+
+@pytest.mark.parametrize("mode", ["inner", "outer"])
+def test_averages_are_rotation_and_permutation_invariant(mode):
+    st = water_cluster(3, seed=3)
+    pos = st.positions.astype(np.float64)
+    o = SoapOracle([1, 8], 4.0, 2, 4, 0.5)
+    ref = modes.average_descriptor(o, mode, pos, st.numbers)
+    R = random_rotation(np.random.default_rng(11))
+    np.testing.assert_allclose(modes.average_descriptor(o, mode, pos @ R.T, st.numbers), ref, rtol=1e-10, atol=1e-12)
+    perm = np.random.default_rng(0).permutation(pos.shape[0])
+    np.testing.assert_allclose(modes.average_descriptor(o, mode, pos[perm], st.numbers[perm]), ref, rtol=1e-12)
