@@ -139,6 +139,60 @@ int soap_derivatives(soap_t *h, const float *d_positions, const int32_t *d_numbe
 int soap_jacobian_dense(soap_t *h, const float *d_jac_rows, const int64_t *d_row_ptr, const int32_t *d_row_atom,
                         int64_t n_centers, const int32_t *d_include, int64_t n_include, float *d_out, void *stream);
 
+/* ---- output modes beyond the per-centre power spectrum (the interface section of the
+ *      paper: the crossover flag, the coefficient mode, the inner and outer averages) ---- */
+
+/* crossover = 0 keeps only the species pairs mu == nu (F = S n(n+1)/2 (l+1));
+ * the default keeps every pair mu <= nu.  Changes soap_num_features and
+ * soap_feature_info; waits for the device when tables are already uploaded.
+ * Not to be called while work on this handle is in flight. */
+int soap_set_crossover(soap_t *h, int crossover);
+
+/* Number of expansion coefficients per centre, W = S n_max (l_max+1)^2. */
+int soap_num_coefficients(const soap_t *h, int64_t *n_coefficients);
+
+/* Coefficient mode: the projection coefficients c^mu_nlm of Eq. 3 themselves
+ * (Eq. 13 / Eq. 18, on-site term included) instead of their contraction.
+ * d_out [n_centers, W], index (mu n_max + n)(l_max+1)^2 + l^2 + l + m with the
+ * real spherical harmonics m = -l..l (the paper fixes no order: this one is
+ * ours).  Otherwise like soap_descriptor. */
+int soap_coefficients(soap_t *h, const float *d_positions, const int32_t *d_numbers, int64_t n_atoms,
+                      const double *cell, const int32_t *d_centers, int64_t n_centers,
+                      float *d_out, void *stream);
+
+/* Coefficients and their Jacobian d c^mu_nlm / d R_j (Eq. 14 / Eq. 23) in the
+ * row format of soap_derivatives with W in place of F: d_out_coeff
+ * [n_centers, W], d_out_jac [capacity_rows, 3, W].  A neighbour's row is
+ * non-zero only in the block of its own species; the centre's row is minus
+ * the sum of the others.  Errors and capacities as in soap_derivatives. */
+int soap_coefficient_derivatives(soap_t *h, const float *d_positions, const int32_t *d_numbers, int64_t n_atoms,
+                                 const double *cell, const int32_t *d_centers, int64_t n_centers,
+                                 float *d_out_coeff, float *d_out_jac, int64_t capacity_rows,
+                                 int64_t *d_row_ptr, int32_t *d_row_atom, void *stream);
+
+enum { SOAP_AVERAGE_INNER = 1, SOAP_AVERAGE_OUTER = 2 };
+
+/* One averaged descriptor for the whole centre list, d_out [F]:
+ *   outer: the mean over the centres of their power spectra (Eq. 4);
+ *   inner: Eq. 4 applied to the mean over the centres of c^mu_nlm.
+ * n_centers >= 1.  Sums run in a fixed order (results repeat bit for bit).
+ * The handle keeps a workspace of n_centers max(F, W) floats. */
+int soap_descriptor_average(soap_t *h, int mode, const float *d_positions, const int32_t *d_numbers,
+                            int64_t n_atoms, const double *cell, const int32_t *d_centers,
+                            int64_t n_centers, float *d_out, void *stream);
+
+/* Averaged descriptor d_out_desc [F] and its Jacobian with respect to EVERY
+ * atom, d_out_jac [n_atoms, 3, F], fully overwritten (zero rows for atoms in
+ * no centre's sphere).  The per-centre rows (Eq. 5; for the inner average
+ * taken against the mean coefficients) go to a workspace inside the handle of
+ * n_rows 3 F floats, n_rows as soap_neighbors reports it, and are then summed
+ * per atom in centre order; SOAP_ERR_ALLOC when that does not fit the device
+ * (split the centre list and average the partial results by their weights).
+ * WAITS for the stream once (it reads the row total). */
+int soap_derivatives_average(soap_t *h, int mode, const float *d_positions, const int32_t *d_numbers,
+                             int64_t n_atoms, const double *cell, const int32_t *d_centers,
+                             int64_t n_centers, float *d_out_desc, float *d_out_jac, void *stream);
+
 /* Waits for `stream`, then returns and clears the sticky device status
  * (SOAP_OK, SOAP_ERR_UNKNOWN_SPECIES or SOAP_ERR_CAPACITY); also reports the
  * pair and row counts of the last call (either pointer may be NULL). */

@@ -8,11 +8,14 @@ from dataclasses import dataclass
 import numpy as np
 
 GTO, POLYNOMIAL = 0, 1
+AVERAGE_MODES = {"inner": 1, "outer": 2}
 
 EXPORTED_SYMBOLS = [
     "soap_create", "soap_destroy", "soap_num_features", "soap_feature_info", "soap_last_error",
     "soap_radial_table", "soap_neighbors", "soap_neighbor_list", "soap_descriptor",
     "soap_derivatives", "soap_status", "soap_profile", "soap_profile_read", "soap_neighbor_counts_static", "soap_jacobian_dense",
+    "soap_set_crossover", "soap_num_coefficients", "soap_coefficients", "soap_coefficient_derivatives",
+    "soap_descriptor_average", "soap_derivatives_average",
 ]
 
 _ERRORS = {-1: "SOAP_ERR_INVALID_ARG", -2: "SOAP_ERR_UNKNOWN_SPECIES", -3: "SOAP_ERR_CAPACITY",
@@ -59,6 +62,12 @@ def load_library() -> C.CDLL:
     lib.soap_status.argtypes = [vp, C.POINTER(i64), C.POINTER(i64), vp]
     lib.soap_neighbor_counts_static.argtypes = [vp, i64, C.c_double, vp, vp, C.c_char_p, i64]
     lib.soap_jacobian_dense.argtypes = [vp, vp, vp, vp, i64, vp, i64, vp, vp]
+    lib.soap_set_crossover.argtypes = [vp, i32]
+    lib.soap_num_coefficients.argtypes = [vp, C.POINTER(i64)]
+    lib.soap_coefficients.argtypes = common + [vp, vp]
+    lib.soap_coefficient_derivatives.argtypes = common + [vp, vp, i64, vp, vp, vp]
+    lib.soap_descriptor_average.argtypes = [vp, i32] + common[1:] + [vp, vp]
+    lib.soap_derivatives_average.argtypes = [vp, i32] + common[1:] + [vp, vp, vp]
     lib.soap_profile.argtypes = [vp, i32]
     lib.soap_profile_read.argtypes = [vp, C.POINTER(C.c_float), C.POINTER(C.c_float)]
     for name in EXPORTED_SYMBOLS:
@@ -98,7 +107,7 @@ class Derivatives:
 class Soap:
     """One descriptor configuration (the arguments of soap_create)."""
 
-    def __init__(self, species, r_cut, n_max, l_max, sigma, rbf=GTO, pbc=(False, False, False)):
+    def __init__(self, species, r_cut, n_max, l_max, sigma, rbf=GTO, pbc=(False, False, False), crossover=True):
         self._lib = load_library()
         self._h = C.c_void_p()
         sp = (C.c_int32 * len(species))(*[int(z) for z in species])
@@ -110,8 +119,12 @@ class Soap:
             self.close()
             raise SoapError(rc, msg)
         n = C.c_int64()
+        if not crossover:
+            self._check(self._lib.soap_set_crossover(self._h, 0))
         self._check(self._lib.soap_num_features(self._h, C.byref(n)))
         self.n_features = int(n.value)
+        self._check(self._lib.soap_num_coefficients(self._h, C.byref(n)))
+        self.n_coefficients = int(n.value)
         self.n_channels = int(n_max) * (int(l_max) + 1)
         self.pbc = tuple(bool(p) for p in pbc)
 
@@ -220,6 +233,59 @@ class Soap:
         self.derivatives_into(positions, numbers, cell, centers, desc, jac, row_ptr, row_atom)
         self.status()
         return Derivatives(desc, jac[:nrows], row_ptr, row_atom[:nrows])
+
+    # ------------------------------------------------------------------ other output modes
+    def coefficients(self, positions, numbers, cell=None, centers=None, out=None):
+        """(C, W) expansion coefficients c^mu_nlm, W = S n_max (l_max+1)^2."""
+        import torch
+        n, c, cptr = self._inputs(positions, numbers, centers)
+        keep, cellp = self._cell(cell)
+        if out is None:
+            out = torch.empty((c, self.n_coefficients), dtype=torch.float32, device=positions.device)
+        self._check(self._lib.soap_coefficients(self._h, positions.data_ptr(), numbers.data_ptr(), n, cellp, cptr, c,
+                                                out.data_ptr(), self._stream()))
+        return out
+
+    def coefficient_derivatives(self, positions, numbers, cell=None, centers=None) -> Derivatives:
+        """Coefficients and their Jacobian in the row format of `derivatives` (width W)."""
+        import torch
+        _, nrows = self.neighbors(positions, numbers, cell, centers)
+        n, c, cptr = self._inputs(positions, numbers, centers)
+        keep, cellp = self._cell(cell)
+        dev = positions.device
+        coeff = torch.empty((c, self.n_coefficients), dtype=torch.float32, device=dev)
+        jac = torch.empty((max(nrows, 1), 3, self.n_coefficients), dtype=torch.float32, device=dev)
+        row_ptr = torch.empty(c + 1, dtype=torch.int64, device=dev)
+        row_atom = torch.empty(max(nrows, 1), dtype=torch.int32, device=dev)
+        self._check(self._lib.soap_coefficient_derivatives(self._h, positions.data_ptr(), numbers.data_ptr(), n, cellp, cptr, c,
+                                                           coeff.data_ptr(), jac.data_ptr(), jac.shape[0], row_ptr.data_ptr(),
+                                                           row_atom.data_ptr(), self._stream()))
+        self.status()
+        return Derivatives(coeff, jac[:nrows], row_ptr, row_atom[:nrows])
+
+    def descriptor_average(self, mode, positions, numbers, cell=None, centers=None, out=None):
+        """(F,) averaged descriptor, mode "inner" or "outer"."""
+        import torch
+        n, c, cptr = self._inputs(positions, numbers, centers)
+        keep, cellp = self._cell(cell)
+        if out is None:
+            out = torch.empty(self.n_features, dtype=torch.float32, device=positions.device)
+        self._check(self._lib.soap_descriptor_average(self._h, AVERAGE_MODES[mode], positions.data_ptr(), numbers.data_ptr(), n,
+                                                      cellp, cptr, c, out.data_ptr(), self._stream()))
+        return out
+
+    def derivatives_average(self, mode, positions, numbers, cell=None, centers=None, out_desc=None, out_jac=None):
+        """Averaged descriptor (F,) and its Jacobian (n_atoms, 3, F)."""
+        import torch
+        n, c, cptr = self._inputs(positions, numbers, centers)
+        keep, cellp = self._cell(cell)
+        if out_desc is None:
+            out_desc = torch.empty(self.n_features, dtype=torch.float32, device=positions.device)
+        if out_jac is None:
+            out_jac = torch.empty((n, 3, self.n_features), dtype=torch.float32, device=positions.device)
+        self._check(self._lib.soap_derivatives_average(self._h, AVERAGE_MODES[mode], positions.data_ptr(), numbers.data_ptr(), n,
+                                                       cellp, cptr, c, out_desc.data_ptr(), out_jac.data_ptr(), self._stream()))
+        return out_desc, out_jac
 
     def profile(self, enable=True):
         self._check(self._lib.soap_profile(self._h, int(bool(enable))))

@@ -106,9 +106,11 @@ __device__ __forceinline__ void harmonics_column(int L, int m, float x, float y,
     }
 }
 
-template <bool DERIV, int L, int NMAX_T>
-__global__ void __launch_bounds__(kThreads, DERIV ? SOAP_MIN_CTAS_DERIV : SOAP_MIN_CTAS_DESC)
+// KIND: 0 descriptor only, 1 descriptor and Jacobian, 2 coefficients c^mu_nlm and their Jacobian
+template <int KIND, int L, int NMAX_T>
+__global__ void __launch_bounds__(kThreads, KIND ? SOAP_MIN_CTAS_DERIV : SOAP_MIN_CTAS_DESC)
 center_kernel(const CenterParams p) {
+    constexpr bool DERIV = KIND != 0, CC = KIND == 2;
     constexpr int L1 = L + 1, LM = L1 * L1, LMP = LM | 1;      // odd row stride: no shared-memory bank conflicts
     constexpr int NMAX_BOUND = NMAX_T ? NMAX_T : 16;
     // pass-1 ownership: W_LM warps cover the lm index, SLOTS such groups split the n index
@@ -149,7 +151,8 @@ center_kernel(const CenterParams p) {
     const float xi = p.pos[3 * (long long)ci], yi = p.pos[3 * (long long)ci + 1], zi = p.pos[3 * (long long)ci + 2];
     const int zi_species = p.species_idx[ci];
     const long long pair_base = p.pair_start[c_idx];
-    const int k_pairs = p.pair_count[c_idx];
+    // descriptor of given mean coefficients (inner average): no pairs to visit
+    const int k_pairs = (!DERIV && p.c_bar) ? 0 : p.pair_count[c_idx];
     const bool periodic = p.geom.pbc[0] | p.geom.pbc[1] | p.geom.pbc[2];
 
     for (int e = tid; e < CT * (DERIV ? 4 : 1); e += kThreads) {
@@ -158,7 +161,7 @@ center_kernel(const CenterParams p) {
 
     // same-species blocks: feature index -> (n1 L1 + l) | (n2 L1 + l) << 8, rows n1 of (NMAX - n1) L1 entries
     unsigned short* tri_dec = reinterpret_cast<unsigned short*>(smem + lay.tri);
-    if (DERIV)
+    if (DERIV && !CC)
         for (int e = tid; e < (NMAX * (NMAX + 1) / 2) * L1; e += kThreads) {
             int n1 = 0, r = e;
             while (r >= (NMAX - n1) * L1) { r -= (NMAX - n1) * L1; ++n1; }
@@ -327,8 +330,27 @@ center_kernel(const CenterParams p) {
     }
     __syncthreads();
     // on-site term: the centre's own Gaussian, l = 0 only (second term of Eq. 13)
-    if (tid < NMAX) c_t[(zi_species * NMAX + tid) * LMP] += __ldg(p.self_term + tid);
+    if (tid < NMAX && !p.c_bar) c_t[(zi_species * NMAX + tid) * LMP] += __ldg(p.self_term + tid);
     __syncthreads();
+    const int W = S * NE;                                                  // coefficients per centre
+    const int RW = CC ? W : F;                                             // width of an output row
+    if (p.c_bar) {
+        // inner average: the mean coefficients (on-site terms included) take the place of the centre's own
+        for (int e = tid; e < W; e += kThreads) {
+            const int row = e / LM;
+            c_t[row * LMP + (e - row * LM)] = __ldg(p.c_bar + e);
+        }
+        __syncthreads();
+    }
+    if ((!DERIV && p.emit_coeff) || CC) {
+        // coefficient mode: the tile itself is the result, index (mu n_max + n) (l_max+1)^2 + l^2 + l + m
+        float* crow = p.out_desc + (size_t)c_idx * W;
+        for (int e = tid; e < W; e += kThreads) {
+            const int row = e / LM;
+            crow[e] = c_t[row * LMP + (e - row * LM)];
+        }
+        if (!DERIV) return;
+    }
 
     // ============ power spectrum (Eq. 4) and the centre's own row ============
     // Threads walk the features l-major so that the lanes of a warp share the trip count 2l+1; the
@@ -336,8 +358,18 @@ center_kernel(const CenterParams p) {
     // pass through the (now idle) staging area in slabs, so that global memory is written in
     // feature order, whole sectors at a time.
     const long long row_base = DERIV ? p.row_ptr[c_idx] : 0;
-    {
-        float* desc_row = p.out_desc + (size_t)c_idx * F;
+    if (CC) {
+        // the centre's own row: minus the sum over the atoms that move relative to it
+        float* own = p.out_jac + (size_t)(row_base + p.self_row[c_idx]) * 3 * W;
+        for (int e = tid; e < 3 * W; e += kThreads) {
+            const int k = e / W, r = e - k * W, row = r / LM;
+            own[e] = -D_t[k * CT + row * LMP + (r - row * LM)];
+        }
+        if (tid == 0) p.row_atom[row_base + p.self_row[c_idx]] = ci;
+    } else {
+        // with given mean coefficients every centre would write the same descriptor: the first one does
+        const bool write_desc = !p.c_bar || c_idx == 0;
+        float* desc_row = p.out_desc + (p.c_bar ? (size_t)0 : (size_t)c_idx * F);
         float* own = DERIV ? p.out_jac + (size_t)(row_base + p.self_row[c_idx]) * 3 * F : nullptr;
         float* slab = smem + lay.sSD;
         constexpr int NV = DERIV ? 4 : 1;                                   // values per feature
@@ -350,12 +382,12 @@ center_kernel(const CenterParams p) {
         // group (the generic loop below loads two operands per multiply-add).
         const bool grouped = !DERIV && (lay.total - lay.sSD) >= F && !(SOAP_DEBUG_SKIP & 8);
         if (grouped) {
-            const int NB = S * (S + 1) / 2;
+            const int NB = p.crossover ? S * (S + 1) / 2 : S;
             for (int it = tid; it < NB * L1 * NMAX; it += kThreads) {
                 const int n1 = it % NMAX, rest = it / NMAX, b = rest % NB, l = rest / NB;   // l slowest: warps share 2l+1
                 int mu = 0, nu = 0, boff = 0;                                                // block b -> (mu, nu), feature offset
                 for (int k = 0, a2 = 0; a2 < S; ++a2)
-                    for (int b2 = a2; b2 < S; ++b2, ++k) {
+                    for (int b2 = a2; b2 < (p.crossover ? S : a2 + 1); ++b2, ++k) {
                         if (k == b) { mu = a2; nu = b2; }
                         if (k < b) boff += (a2 == b2) ? (NMAX * (NMAX + 1) / 2) * L1 : NMAX * NCH;
                     }
@@ -378,7 +410,8 @@ center_kernel(const CenterParams p) {
                     if (n2 < NMAX && n2 >= n2_lo) slab[base + n2 * L1] = kl * acc[n2];
             }
             __syncthreads();
-            for (int e = tid; e < F; e += kThreads) desc_row[e] = slab[e];
+            if (write_desc)
+                for (int e = tid; e < F; e += kThreads) desc_row[e] = slab[e];
         }
         for (int q0 = 0; q0 < ((SOAP_DEBUG_SKIP & 8) || grouped ? 0 : NP); q0 += gp) {
             const int nq = min(gp, NP - q0), nf = nq * L1, f0 = q0 * L1;
@@ -402,14 +435,14 @@ center_kernel(const CenterParams p) {
                     slab[fl] = kl * acc;
                     if (DERIV) { slab[nf + fl] = -kl * ax; slab[2 * nf + fl] = -kl * ay; slab[3 * nf + fl] = -kl * az; }
                 } else {
-                    desc_row[f0 + fl] = kl * acc;
+                    if (write_desc) desc_row[f0 + fl] = kl * acc;
                     if (DERIV) { own[f0 + fl] = -kl * ax; own[(size_t)F + f0 + fl] = -kl * ay; own[(size_t)2 * F + f0 + fl] = -kl * az; }
                 }
             }
             if (staged) {
                 __syncthreads();
                 for (int e = tid; e < nf; e += kThreads) {
-                    desc_row[f0 + e] = slab[e];
+                    if (write_desc) desc_row[f0 + e] = slab[e];
                     if (DERIV) {
                         own[f0 + e] = slab[nf + e];
                         own[(size_t)F + f0 + e] = slab[2 * nf + e];
@@ -424,10 +457,11 @@ center_kernel(const CenterParams p) {
     if (!DERIV) return;
     __syncthreads();
     // fold K_l into c for pass 2
-    for (int e = tid; e < S * NMAX * LM; e += kThreads) {
-        const int row = e / LM, lm = e - row * LM;
-        c_t[row * LMP + lm] *= __ldg(p.kl + __ldg(p.l_of_lm + lm));
-    }
+    if (!CC)
+        for (int e = tid; e < W; e += kThreads) {
+            const int row = e / LM, lm = e - row * LM;
+            c_t[row * LMP + lm] *= __ldg(p.kl + __ldg(p.l_of_lm + lm));
+        }
 
     // =========================== pass 2: the Jacobian rows ===========================
     const int NI = S * NCH, SN = S * NMAX;
@@ -454,7 +488,7 @@ center_kernel(const CenterParams p) {
         };
         int lo = 0;
         for (int mu = 0; mu < S; ++mu) {
-            for (int nu = mu; nu < S; ++nu) {
+            for (int nu = mu; nu < (p.crossover ? S : mu + 1); ++nu) {
                 const int hi = lo + ((mu == nu) ? (NMAX * (NMAX + 1) / 2) * L1 : NMAX * NCH);
                 const int first = ((lo + a_line) & ~31) - a_line;
                 if (mu != Z && nu != Z) {
@@ -543,6 +577,32 @@ center_kernel(const CenterParams p) {
         }
     };
 
+    // Coefficient mode: the row of a neighbour of species Z is grad c^Z_nlm = G_nl grad S_lm + Ghat_nl d S_lm
+    // (Eq. 14 / Eq. 23) in the block of Z and zero in the other blocks, written in aligned sweeps as above.
+    auto coeff_rule = [&](auto acc_tag, int Z, float4 d, const float2* wG, const float4* wSD, float* out) {
+        constexpr bool ACC = decltype(acc_tag)::value;
+        const int a_line = (int)((reinterpret_cast<size_t>(out) >> 2) & 31);
+        for (int s = 0; s < S; ++s) {
+            if (ACC && s != Z) continue;
+            const int lo = s * NE, hi = lo + NE;
+            const int first = ((lo + a_line) & ~31) - a_line;
+            for (int f = first + lane; f < hi; f += 32) {
+                if (f < lo) continue;
+                float vx = 0.f, vy = 0.f, vz = 0.f;
+                if (s == Z) {
+                    const int e = f - lo, n = e / LM, lm = e - n * LM;
+                    const int l = (int)sqrtf((float)lm);                  // lm = l^2 + l + m
+                    const float2 g = wG[n * L1 + l];
+                    const float4 h = wSD[lm];
+                    const float t = g.y * h.x;
+                    vx = fmaf(g.x, h.y, t * d.x); vy = fmaf(g.x, h.z, t * d.y); vz = fmaf(g.x, h.w, t * d.z);
+                }
+                if (ACC) { out[f] += vx; out[W + f] += vy; out[2 * W + f] += vz; }
+                else { out[f] = vx; out[W + f] = vy; out[2 * W + f] = vz; }
+            }
+        }
+    };
+
     // everything one warp does for one pair of the staged chunk
     auto do_pair = [&](int g, int pr) {
         const int4 gi = geo_i[g];
@@ -554,7 +614,7 @@ center_kernel(const CenterParams p) {
         const float4* wSD = sSD4 + pr * LMP;
         __syncwarp();
         // ---- U, V for every (nu, n', l) ----
-        if (SOAP_DEBUG_SKIP & 2) {
+        if (CC || (SOAP_DEBUG_SKIP & 2)) {
         } else if (SN <= 16) {
             // lane <-> (nu n', half): half 0 accumulates (U, Vx), half 1 (Vy, Vz)
             const int sn = lane >> 1, half = lane & 1;
@@ -593,12 +653,14 @@ center_kernel(const CenterParams p) {
         }
         __syncwarp();
         if (SOAP_DEBUG_SKIP & 1) return;
-        float* out = p.out_jac + (size_t)(row_base + row) * 3 * F;
+        float* out = p.out_jac + (size_t)(row_base + row) * 3 * RW;
         if (rw & kRowContinuation) {
-            product_rule(std::true_type{}, Z, d, wG, out);
+            if (CC) coeff_rule(std::true_type{}, Z, d, wG, wSD, out);
+            else product_rule(std::true_type{}, Z, d, wG, out);
         } else {
             if (lane == 0) p.row_atom[row_base + row] = geo_j[g];
-            product_rule(std::false_type{}, Z, d, wG, out);
+            if (CC) coeff_rule(std::false_type{}, Z, d, wG, wSD, out);
+            else product_rule(std::false_type{}, Z, d, wG, out);
         }
     };
 

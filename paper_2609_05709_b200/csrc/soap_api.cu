@@ -11,6 +11,7 @@
 #include <vector>
 
 #include "basis_host.h"
+#include "average_kernels.cuh"
 #include "center_launch.h"
 #include "dense_kernel.cuh"
 #include "neighbor_kernels.cuh"
@@ -27,17 +28,17 @@ cudaError_t center_constants(int l_max, const float* anorm91, const float* dfact
     }
     return cudaErrorInvalidValue;
 }
-cudaError_t center_set_smem(bool deriv, int l_max, int n_max, int bytes) {
+cudaError_t center_set_smem(int kind, int l_max, int n_max, int bytes) {
     switch (l_max) {
-#define X(LV) case LV: return center_set_smem_l##LV(deriv, n_max, bytes);
+#define X(LV) case LV: return center_set_smem_l##LV(kind, n_max, bytes);
         X(0) X(1) X(2) X(3) X(4) X(5) X(6) X(7) X(8) X(9) X(10) X(11) X(12)
 #undef X
     }
     return cudaErrorInvalidValue;
 }
-cudaError_t center_launch(bool deriv, int l_max, int n_max, const CenterParams& p, unsigned grid, size_t smem, cudaStream_t st) {
+cudaError_t center_launch(int kind, int l_max, int n_max, const CenterParams& p, unsigned grid, size_t smem, cudaStream_t st) {
     switch (l_max) {
-#define X(LV) case LV: return center_launch_l##LV(deriv, n_max, p, grid, smem, st);
+#define X(LV) case LV: return center_launch_l##LV(kind, n_max, p, grid, smem, st);
         X(0) X(1) X(2) X(3) X(4) X(5) X(6) X(7) X(8) X(9) X(10) X(11) X(12)
 #undef X
     }
@@ -51,6 +52,7 @@ struct soap_handle {
     int S = 0, n_max = 0, l_max = 0, rbf = 0;
     double r_cut = 0, sigma = 0;
     int pbc[3] = {0, 0, 0};
+    int crossover = 1;
     int64_t F = 0;
     HostBasis basis;
     std::vector<int> feat_pack;
@@ -75,6 +77,8 @@ struct soap_handle {
     int* d_tile_sums = nullptr;
     unsigned long long *d_pair_key = nullptr, *d_pair_tmp = nullptr;
     int* d_pair_row = nullptr;
+    void* d_work = nullptr;              // workspace of the averaged modes
+    size_t cap_work = 0;
     // plan
     int64_t planned_atoms = -1, planned_centers = -1;
     int64_t last_centers = 0;
@@ -204,8 +208,9 @@ int ensure_device(soap_t* h) {
         for (size_t i = 0; i < h->basis.dfact.size(); ++i) dfact[i] = h->basis.dfact[i];
         CU(center_constants(h->l_max, anorm.data(), dfact.data()));
     }
-    CU(center_set_smem(false, h->l_max, h->n_max, (int)h->smem_desc));
-    CU(center_set_smem(true, h->l_max, h->n_max, (int)h->smem_deriv));
+    CU(center_set_smem(kCenterDesc, h->l_max, h->n_max, (int)h->smem_desc));
+    CU(center_set_smem(kCenterDeriv, h->l_max, h->n_max, (int)h->smem_deriv));
+    CU(center_set_smem(kCenterCoeff, h->l_max, h->n_max, (int)h->smem_deriv));
     h->tables_ready = true;
     return SOAP_OK;
 }
@@ -335,7 +340,66 @@ void fill_center_params(soap_t* h, CenterParams& cp, const float* pos, const int
     cp.feat_pack = h->d_feat; cp.nch_magic = (unsigned)((1ull << 32) / (unsigned)(h->n_max * (h->l_max + 1))) + 1u; cp.inv_h = (float)h->basis.inv_h; cp.n_intervals = h->basis.n_intervals;
     cp.S = h->S; cp.n_max = h->n_max; cp.l_max = h->l_max; cp.F = (int)h->F;
     cp.P = deriv ? h->P_deriv : h->P_desc;
+    cp.crossover = h->crossover; cp.emit_coeff = 0; cp.c_bar = nullptr;
     cp.out_desc = nullptr; cp.out_jac = nullptr; cp.row_atom = nullptr;
+}
+
+// Feature table: species pairs mu <= nu (only mu == nu without crossover), radial pair (n' >= n on
+// the diagonal), l fastest.
+void build_feature_table(soap_t* h) {
+    h->feat_pack.clear();
+    for (int mu = 0; mu < h->S; ++mu)
+        for (int nu = mu; nu < (h->crossover ? h->S : mu + 1); ++nu)
+            for (int n = 0; n < h->n_max; ++n)
+                for (int n2 = (mu == nu ? n : 0); n2 < h->n_max; ++n2)
+                    for (int l = 0; l <= h->l_max; ++l)
+                        h->feat_pack.push_back(n | (n2 << 5) | (mu << 10) | (nu << 14) | (l << 18));
+    h->F = (int64_t)h->feat_pack.size();
+}
+
+// Everything before the per-centre kernel: argument checks, device set-up, planning when the sizes
+// changed, the neighbour search.
+int prepare(soap_t* h, const float* pos, const int32_t* num, int64_t N, const double* cell, const int32_t* centers,
+            int64_t C, long long* row_ptr_out, Geometry& g, cudaStream_t st) {
+    int rc = check_inputs(h, pos, num, N, centers, C);
+    if (rc) return rc;
+    if ((rc = ensure_device(h))) return rc;
+    if ((rc = make_geometry(h, cell, g))) return rc;
+    if (h->profiling) CU(cudaEventRecord(h->ev[0], st));
+    if (h->planned_atoms != N || h->planned_centers != C) {
+        if ((rc = plan(h, pos, num, N, g, centers, C, st))) return rc;
+    }
+    if ((rc = launch_neighbors(h, pos, num, N, g, centers, C, row_ptr_out ? row_ptr_out : h->d_row_ptr, st))) return rc;
+    if (h->profiling) CU(cudaEventRecord(h->ev[1], st));
+    h->last_centers = C;
+    return SOAP_OK;
+}
+
+int ensure_work(soap_t* h, size_t bytes) {
+    if (bytes <= h->cap_work) return SOAP_OK;
+    if (h->d_work) { cudaFree(h->d_work); h->d_work = nullptr; h->cap_work = 0; }
+    const size_t want = bytes + bytes / 16 + 4096;
+    if (cudaMalloc(&h->d_work, want) != cudaSuccess) {
+        cudaGetLastError();
+        return fail(h, SOAP_ERR_ALLOC, "the workspace of the averaged mode (" + std::to_string(want >> 20) +
+                                           " MiB: every Jacobian row of every centre) does not fit the device; use fewer centres per call");
+    }
+    h->cap_work = want;
+    return SOAP_OK;
+}
+
+size_t align256(size_t x) { return (x + 255) & ~(size_t)255; }
+
+// out[col] = mean over the rows of in[rows][width], summed in a fixed order
+int column_mean(soap_t* h, const float* in, int64_t rows, int width, double* partial, float* out, cudaStream_t st) {
+    int chunks = (int)std::max<int64_t>(1, std::min<int64_t>(kMeanMaxChunks, rows / 32));
+    const long long chunk_rows = (rows + chunks - 1) / chunks;
+    chunks = (int)((rows + chunk_rows - 1) / chunk_rows);
+    const unsigned gx = (unsigned)((width + kMeanThreads - 1) / kMeanThreads);
+    column_partial_kernel<<<dim3(gx, (unsigned)chunks), kMeanThreads, 0, st>>>(in, rows, width, chunk_rows, partial);
+    column_finish_kernel<<<gx, kMeanThreads, 0, st>>>(partial, chunks, width, 1.0 / (double)rows, out);
+    CU(cudaGetLastError());
+    return SOAP_OK;
 }
 
 }  // namespace
@@ -368,15 +432,7 @@ int soap_create(soap_t** out, const int32_t* species, int n_species, double r_cu
     if (rc) return bail(rc, err);
     if ((int64_t)n_max * (l_max + 1) * (l_max + 1) > (int64_t)kMaxElemPerThread * kThreads)
         return bail(SOAP_ERR_INVALID_ARG, "n_max (l_max+1)^2 must not exceed 2048");
-    // feature table: species pairs mu <= nu, radial pair (n' >= n on the diagonal), l fastest
-    for (int mu = 0; mu < h->S; ++mu)
-        for (int nu = mu; nu < h->S; ++nu)
-            for (int n = 0; n < n_max; ++n)
-                for (int n2 = (mu == nu ? n : 0); n2 < n_max; ++n2)
-                    for (int l = 0; l <= l_max; ++l) {
-                        h->feat_pack.push_back(n | (n2 << 5) | (mu << 10) | (nu << 14) | (l << 18));
-                    }
-    h->F = (int64_t)h->feat_pack.size();
+    build_feature_table(h);
     *out = h;
     return SOAP_OK;
 }
@@ -386,7 +442,7 @@ void soap_destroy(soap_t* h) {
     void* ptrs[] = {h->d_table, h->d_self, h->d_kl, h->d_feat, h->d_zlut, h->d_l_of_lm, h->d_counters, h->d_bbox,
                     h->d_grid, h->d_species_idx, h->d_atom_cell, h->d_atom_wrap, h->d_s_wrap, h->d_s_pos, h->d_cell_count,
                     h->d_cell_start, h->d_pair_count, h->d_row_count, h->d_self_row, h->d_order, h->d_pair_ptr, h->d_pair_start, h->d_row_ptr, h->d_tile_sums, h->d_tile_offsets,
-                    h->d_pair_key, h->d_pair_tmp, h->d_pair_row};
+                    h->d_pair_key, h->d_pair_tmp, h->d_pair_row, h->d_work};
     for (void* p : ptrs) if (p) cudaFree(p);
     if (h->h_counters) cudaFreeHost(h->h_counters);
     for (cudaEvent_t e : h->ev) if (e) cudaEventDestroy(e);
@@ -469,7 +525,7 @@ int soap_descriptor(soap_t* h, const float* d_positions, const int32_t* d_number
         CenterParams cp;
         fill_center_params(h, cp, d_positions, d_centers, n_centers, g, false);
         cp.out_desc = d_out;
-        CU(center_launch(false, h->l_max, h->n_max, cp, (unsigned)n_centers, h->smem_desc, st));
+        CU(center_launch(kCenterDesc, h->l_max, h->n_max, cp, (unsigned)n_centers, h->smem_desc, st));
     }
     if (h->profiling) CU(cudaEventRecord(h->ev[2], st));
     return SOAP_OK;
@@ -499,7 +555,7 @@ int soap_derivatives(soap_t* h, const float* d_positions, const int32_t* d_numbe
         cp.row_ptr = (const long long*)d_row_ptr;
         cp.row_capacity = capacity_rows;
         cp.out_desc = d_out_desc; cp.out_jac = d_out_jac; cp.row_atom = d_row_atom;
-        CU(center_launch(true, h->l_max, h->n_max, cp, (unsigned)n_centers, h->smem_deriv, st));
+        CU(center_launch(kCenterDeriv, h->l_max, h->n_max, cp, (unsigned)n_centers, h->smem_deriv, st));
     }
     if (h->profiling) CU(cudaEventRecord(h->ev[2], st));
     return SOAP_OK;
@@ -515,6 +571,167 @@ int soap_jacobian_dense(soap_t* h, const float* d_jac_rows, const int64_t* d_row
     dense_scatter_kernel<<<(unsigned)(n_centers * n_include), 128, 0, (cudaStream_t)stream>>>(
         d_jac_rows, (const long long*)d_row_ptr, d_row_atom, n_centers, d_include, n_include, (int)h->F, d_out);
     CU(cudaGetLastError());
+    return SOAP_OK;
+}
+
+int soap_set_crossover(soap_t* h, int crossover) {
+    if (!h) return SOAP_ERR_INVALID_ARG;
+    crossover = crossover ? 1 : 0;
+    if (crossover == h->crossover) return SOAP_OK;
+    h->crossover = crossover;
+    build_feature_table(h);
+    if (h->tables_ready) {
+        CU(cudaDeviceSynchronize());
+        cudaFree(h->d_feat);
+        h->d_feat = nullptr;
+        CU(upload(&h->d_feat, h->feat_pack));
+    }
+    return SOAP_OK;
+}
+
+int soap_num_coefficients(const soap_t* h, int64_t* n_coefficients) {
+    if (!h || !n_coefficients) return SOAP_ERR_INVALID_ARG;
+    *n_coefficients = (int64_t)h->S * h->n_max * (h->l_max + 1) * (h->l_max + 1);
+    return SOAP_OK;
+}
+
+int soap_coefficients(soap_t* h, const float* d_positions, const int32_t* d_numbers, int64_t n_atoms, const double* cell,
+                      const int32_t* d_centers, int64_t n_centers, float* d_out, void* stream) {
+    if (h && n_centers > 0 && !d_out) return fail(h, SOAP_ERR_INVALID_ARG, "d_out must not be NULL");
+    Geometry g;
+    cudaStream_t st = (cudaStream_t)stream;
+    int rc = prepare(h, d_positions, d_numbers, n_atoms, cell, d_centers, n_centers, nullptr, g, st);
+    if (rc) return rc;
+    if (n_centers > 0) {
+        CenterParams cp;
+        fill_center_params(h, cp, d_positions, d_centers, n_centers, g, false);
+        cp.out_desc = d_out;
+        cp.emit_coeff = 1;
+        CU(center_launch(kCenterDesc, h->l_max, h->n_max, cp, (unsigned)n_centers, h->smem_desc, st));
+    }
+    if (h->profiling) CU(cudaEventRecord(h->ev[2], st));
+    return SOAP_OK;
+}
+
+int soap_coefficient_derivatives(soap_t* h, const float* d_positions, const int32_t* d_numbers, int64_t n_atoms,
+                                 const double* cell, const int32_t* d_centers, int64_t n_centers, float* d_out_coeff,
+                                 float* d_out_jac, int64_t capacity_rows, int64_t* d_row_ptr, int32_t* d_row_atom,
+                                 void* stream) {
+    if (h && (!d_row_ptr || capacity_rows < 0)) return fail(h, SOAP_ERR_INVALID_ARG, "d_row_ptr must not be NULL");
+    if (h && n_centers > 0 && (!d_out_coeff || !d_out_jac || !d_row_atom)) return fail(h, SOAP_ERR_INVALID_ARG, "output pointers must not be NULL");
+    Geometry g;
+    cudaStream_t st = (cudaStream_t)stream;
+    int rc = prepare(h, d_positions, d_numbers, n_atoms, cell, d_centers, n_centers, (long long*)d_row_ptr, g, st);
+    if (rc) return rc;
+    if (n_centers > 0) {
+        CenterParams cp;
+        fill_center_params(h, cp, d_positions, d_centers, n_centers, g, true);
+        cp.row_ptr = (const long long*)d_row_ptr;
+        cp.row_capacity = capacity_rows;
+        cp.out_desc = d_out_coeff; cp.out_jac = d_out_jac; cp.row_atom = d_row_atom;
+        CU(center_launch(kCenterCoeff, h->l_max, h->n_max, cp, (unsigned)n_centers, h->smem_deriv, st));
+    }
+    if (h->profiling) CU(cudaEventRecord(h->ev[2], st));
+    return SOAP_OK;
+}
+
+int soap_descriptor_average(soap_t* h, int mode, const float* d_positions, const int32_t* d_numbers, int64_t n_atoms,
+                            const double* cell, const int32_t* d_centers, int64_t n_centers, float* d_out, void* stream) {
+    if (!h) return SOAP_ERR_INVALID_ARG;
+    if (mode != SOAP_AVERAGE_INNER && mode != SOAP_AVERAGE_OUTER) return fail(h, SOAP_ERR_INVALID_ARG, "mode must be SOAP_AVERAGE_INNER or SOAP_AVERAGE_OUTER");
+    if (n_centers < 1) return fail(h, SOAP_ERR_INVALID_ARG, "an average needs at least one centre");
+    if (!d_out) return fail(h, SOAP_ERR_INVALID_ARG, "d_out must not be NULL");
+    Geometry g;
+    cudaStream_t st = (cudaStream_t)stream;
+    int rc = prepare(h, d_positions, d_numbers, n_atoms, cell, d_centers, n_centers, nullptr, g, st);
+    if (rc) return rc;
+    const int F = (int)h->F, W = h->S * h->n_max * (h->l_max + 1) * (h->l_max + 1);
+    const bool inner = mode == SOAP_AVERAGE_INNER;
+    const int width = inner ? W : F;
+    const size_t o_rows = 0, o_partial = align256((size_t)n_centers * width * 4),
+                 o_cbar = o_partial + align256((size_t)kMeanMaxChunks * width * 8), total = o_cbar + align256((size_t)W * 4);
+    if ((rc = ensure_work(h, total))) return rc;
+    char* w = (char*)h->d_work;
+    CenterParams cp;
+    fill_center_params(h, cp, d_positions, d_centers, n_centers, g, false);
+    cp.out_desc = (float*)(w + o_rows);
+    cp.emit_coeff = inner ? 1 : 0;
+    CU(center_launch(kCenterDesc, h->l_max, h->n_max, cp, (unsigned)n_centers, h->smem_desc, st));
+    if ((rc = column_mean(h, (const float*)(w + o_rows), n_centers, width, (double*)(w + o_partial),
+                          inner ? (float*)(w + o_cbar) : d_out, st))) return rc;
+    if (inner) {
+        // Eq. 4 on the mean coefficients: one CTA, no pairs
+        cp.emit_coeff = 0;
+        cp.c_bar = (const float*)(w + o_cbar);
+        cp.out_desc = d_out;
+        cp.order = nullptr;
+        CU(center_launch(kCenterDesc, h->l_max, h->n_max, cp, 1u, h->smem_desc, st));
+    }
+    if (h->profiling) CU(cudaEventRecord(h->ev[2], st));
+    return SOAP_OK;
+}
+
+int soap_derivatives_average(soap_t* h, int mode, const float* d_positions, const int32_t* d_numbers, int64_t n_atoms,
+                             const double* cell, const int32_t* d_centers, int64_t n_centers, float* d_out_desc,
+                             float* d_out_jac, void* stream) {
+    if (!h) return SOAP_ERR_INVALID_ARG;
+    if (mode != SOAP_AVERAGE_INNER && mode != SOAP_AVERAGE_OUTER) return fail(h, SOAP_ERR_INVALID_ARG, "mode must be SOAP_AVERAGE_INNER or SOAP_AVERAGE_OUTER");
+    if (n_centers < 1) return fail(h, SOAP_ERR_INVALID_ARG, "an average needs at least one centre");
+    if (!d_out_desc || !d_out_jac) return fail(h, SOAP_ERR_INVALID_ARG, "output pointers must not be NULL");
+    Geometry g;
+    cudaStream_t st = (cudaStream_t)stream;
+    int rc = prepare(h, d_positions, d_numbers, n_atoms, cell, d_centers, n_centers, nullptr, g, st);
+    if (rc) return rc;
+    // the row total sizes the workspace; a structure that outgrew its plan is planned again
+    CU(cudaMemcpyAsync(h->h_counters, h->d_counters, sizeof(Counters), cudaMemcpyDeviceToHost, st));
+    CU(cudaStreamSynchronize(st));
+    if (h->h_counters->n_pairs > h->cap_pairs) {
+        h->planned_atoms = -1;
+        if ((rc = prepare(h, d_positions, d_numbers, n_atoms, cell, d_centers, n_centers, nullptr, g, st))) return rc;
+        CU(cudaMemcpyAsync(h->h_counters, h->d_counters, sizeof(Counters), cudaMemcpyDeviceToHost, st));
+        CU(cudaStreamSynchronize(st));
+    }
+    const int64_t rows = h->h_counters->n_rows;
+    const int F = (int)h->F, W = h->S * h->n_max * (h->l_max + 1) * (h->l_max + 1);
+    const bool inner = mode == SOAP_AVERAGE_INNER;
+    const int width = inner ? W : F;
+    const size_t o_jac = 0, o_atom = align256((size_t)rows * 3 * F * 4), o_rows = o_atom + align256((size_t)rows * 4),
+                 o_partial = o_rows + align256((size_t)n_centers * width * 4),
+                 o_cbar = o_partial + align256((size_t)kMeanMaxChunks * width * 8), total = o_cbar + align256((size_t)W * 4);
+    if ((rc = ensure_work(h, total))) return rc;
+    char* w = (char*)h->d_work;
+    CenterParams cp;
+    if (inner) {
+        fill_center_params(h, cp, d_positions, d_centers, n_centers, g, false);
+        cp.out_desc = (float*)(w + o_rows);
+        cp.emit_coeff = 1;
+        CU(center_launch(kCenterDesc, h->l_max, h->n_max, cp, (unsigned)n_centers, h->smem_desc, st));
+        if ((rc = column_mean(h, (const float*)(w + o_rows), n_centers, W, (double*)(w + o_partial), (float*)(w + o_cbar), st))) return rc;
+    }
+    fill_center_params(h, cp, d_positions, d_centers, n_centers, g, true);
+    cp.row_capacity = rows;
+    cp.out_jac = (float*)(w + o_jac);
+    cp.row_atom = (int*)(w + o_atom);
+    if (inner) {
+        // every centre differentiates against the mean coefficients; the first one writes the descriptor
+        cp.c_bar = (const float*)(w + o_cbar);
+        cp.out_desc = d_out_desc;
+    } else {
+        cp.out_desc = (float*)(w + o_rows);
+    }
+    CU(center_launch(kCenterDeriv, h->l_max, h->n_max, cp, (unsigned)n_centers, h->smem_deriv, st));
+    if (!inner && (rc = column_mean(h, (const float*)(w + o_rows), n_centers, F, (double*)(w + o_partial), d_out_desc, st))) return rc;
+    if (n_atoms > 0) {
+        const int width3 = 3 * F;
+        int slices = (int)std::max<int64_t>(1, std::min<int64_t>((1184 + n_atoms - 1) / n_atoms, (width3 + kAvgThreads - 1) / kAvgThreads));
+        const int slice = (((width3 + slices - 1) / slices) + 31) & ~31;
+        slices = (width3 + slice - 1) / slice;
+        average_rows_kernel<<<dim3((unsigned)n_atoms, (unsigned)slices), kAvgThreads, 0, st>>>(
+            (const float*)(w + o_jac), h->d_row_ptr, (const int*)(w + o_atom), n_centers, width3, slice,
+            (float)(1.0 / (double)n_centers), d_out_jac);
+        CU(cudaGetLastError());
+    }
+    if (h->profiling) CU(cudaEventRecord(h->ev[2], st));
     return SOAP_OK;
 }
 

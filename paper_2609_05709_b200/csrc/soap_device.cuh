@@ -74,9 +74,13 @@ struct CenterParams {
     int S, n_max, l_max, F;
     int P;                        // pairs per staged chunk (<= 32)
     unsigned nch_magic;           // floor(2^32 / (n_max (l_max+1))) + 1: x / n_ch == umulhi(x, magic) for x < 65536
+    // output mode
+    int crossover;                // 0: only the species pairs mu == nu are features
+    int emit_coeff;               // descriptor build: write the coefficients c^mu_nlm instead of the power spectrum
+    const float* c_bar;           // [S n_max (l_max+1)^2] or null: coefficients that replace the centre's own after pass 1
     // outputs
-    float* out_desc;              // [C,F]
-    float* out_jac;               // [rows,3,F]
+    float* out_desc;              // [C,F]  (coefficient mode: [C, S n_max (l_max+1)^2]; with c_bar: [F])
+    float* out_jac;               // [rows,3,F]  (coefficient mode: [rows, 3, S n_max (l_max+1)^2])
     int* row_atom;                // [rows]
 };
 
