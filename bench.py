@@ -309,13 +309,13 @@ def run_cuda(args):
         dist.destroy_process_group()
 
 
-def time_case(struct, species, r_cut, n_max, l_max, sigma, rbf, mode, steps, warmup=3):
+def time_case(struct, species, r_cut, n_max, l_max, sigma, rbf, mode, steps, warmup=3, crossover=True):
     """Device-resident timing of one configuration; returns a dict for the tables in the benchmark spec."""
     import torch
     import paper_2609_05709_b200 as pkg
     pbc = (True, True, True) if struct.cell is not None else (False, False, False)
-    soap = pkg.Soap(species, r_cut, n_max, l_max, sigma, rbf, pbc)
-    F, C = soap.n_features, struct.n_atoms
+    soap = pkg.Soap(species, r_cut, n_max, l_max, sigma, rbf, pbc, crossover=crossover)
+    F, C, W = soap.n_features, struct.n_atoms, soap.n_coefficients
     pos = torch.from_numpy(struct.positions).cuda()
     num = torch.from_numpy(struct.numbers).cuda()
     n_pairs, n_rows = soap.neighbors(pos, num, struct.cell)
@@ -326,9 +326,34 @@ def time_case(struct, species, r_cut, n_max, l_max, sigma, rbf, mode, steps, war
         row_atom = torch.empty(n_rows, dtype=torch.int32, device="cuda")
         step = lambda: soap.derivatives_into(pos, num, struct.cell, None, desc, jac, row_ptr, row_atom)
         alg_bytes = n_rows * 3 * F * 4 + C * F * 4 + n_rows * 4 + n_pairs * 24 + (C + 1) * 16
-    else:
+    elif mode == "descriptor":
         step = lambda: soap.descriptor(pos, num, struct.cell, None, out=desc)
         alg_bytes = C * F * 4 + n_pairs * 24 + (C + 1) * 8
+    elif mode == "coefficients":
+        coeff = torch.empty((C, W), device="cuda")
+        step = lambda: soap.coefficients(pos, num, struct.cell, None, out=coeff)
+        alg_bytes = C * W * 4 + n_pairs * 24 + (C + 1) * 8
+    elif mode == "coefficient_derivatives":
+        coeff = torch.empty((C, W), device="cuda")
+        jac = torch.empty((n_rows, 3, W), device="cuda")
+        row_ptr = torch.empty(C + 1, dtype=torch.int64, device="cuda")
+        row_atom = torch.empty(n_rows, dtype=torch.int32, device="cuda")
+        cellp = soap._cell(struct.cell)
+        step = lambda: soap._check(soap._lib.soap_coefficient_derivatives(
+            soap._h, pos.data_ptr(), num.data_ptr(), C, cellp[1], None, C, coeff.data_ptr(), jac.data_ptr(), n_rows,
+            row_ptr.data_ptr(), row_atom.data_ptr(), soap._stream()))
+        alg_bytes = n_rows * 3 * W * 4 + C * W * 4 + n_rows * 4 + n_pairs * 24 + (C + 1) * 16
+    elif mode in ("average_inner", "average_outer"):
+        avg = torch.empty(F, device="cuda")
+        step = lambda: soap.descriptor_average(mode[8:], pos, num, struct.cell, None, out=avg)
+        alg_bytes = F * 4 + n_pairs * 24 + (C + 1) * 8
+    else:
+        # averaged Jacobian: what must move is the result; the per-centre rows are an intermediate
+        # (written once, read once) that the figure 'intermediate_bytes' counts
+        avg = torch.empty(F, device="cuda")
+        jac = torch.empty((C, 3, F), device="cuda")
+        step = lambda: soap.derivatives_average(mode[8:13], pos, num, struct.cell, None, out_desc=avg, out_jac=jac)
+        alg_bytes = C * 3 * F * 4 + F * 4 + n_pairs * 24 + (C + 1) * 8
     flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
     soap.profile(True)
     for _ in range(warmup):
@@ -350,10 +375,12 @@ def time_case(struct, species, r_cut, n_max, l_max, sigma, rbf, mode, steps, war
     ms = statistics.median(total)
     peak, _ = measured_peaks()
     k_ms = statistics.median(kern)
-    out = {"mode": mode, "atoms": C, "n_max": n_max, "l_max": l_max, "features": F, "pairs": n_pairs, "rows": n_rows,
+    out = {"mode": mode, "crossover": bool(crossover), "atoms": C, "n_max": n_max, "l_max": l_max, "features": F, "pairs": n_pairs, "rows": n_rows,
            "ms_per_step": ms, "atoms_per_s": C / (ms * 1e-3), "kernel_ms": k_ms, "neighbour_search_ms": statistics.median(nbr),
            "algorithmic_bytes": alg_bytes, "kernel_GBps": alg_bytes / (k_ms * 1e-3) / 1e9,
            "hbm_frac_of_measured_peak": alg_bytes / (k_ms * 1e-3) / 1e9 / peak}
+    if mode.endswith("_derivatives") and mode.startswith("average"):
+        out["intermediate_bytes"] = 2 * n_rows * 3 * F * 4
     del soap
     torch.cuda.empty_cache()
     return out
@@ -377,6 +404,15 @@ def run_suite(args):
             r = time_case(s, [1, 8], 5.0, 8, 6, 0.5, 0, "descriptor", steps)
             r["case"] = "scaling"
             print(json.dumps(r), flush=True)
+    elif args.suite == "modes":
+        s = water_cluster(1000, 0)
+        base = ([1, 8], 6.0, 8, 6, 0.5, 0)
+        for mode, crossover in (("derivatives", False), ("descriptor", False), ("coefficients", True),
+                                ("coefficient_derivatives", True), ("average_inner", True), ("average_outer", True),
+                                ("average_inner_derivatives", True), ("average_outer_derivatives", True)):
+            r = time_case(s, *base, mode, steps, crossover=crossover)
+            r["case"] = "modes"
+            print(json.dumps(r), flush=True)
     else:
         for name in ("water8_gto_n4_l3_rc5", "water1000_gto_n8_l6_rc6", "chno2000_poly_n8_l8_rc5"):
             kind, n, species, r_cut, n_max, l_max, sigma, rbf = WORKLOADS[name]
@@ -396,11 +432,12 @@ def main():
     ap.add_argument("--workload", default=DEFAULT_WORKLOAD, choices=sorted(WORKLOADS))
     ap.add_argument("--kernel-only", action="store_true",
                     help="skip the end-to-end and CPU-baseline legs (for profiler captures)")
-    ap.add_argument("--suite", choices=["map", "scaling", "configs", "desc30k"],
+    ap.add_argument("--suite", choices=["map", "scaling", "configs", "desc30k", "modes"],
                     help="extra measurements beside the headline line: 'map' = descriptor+Jacobian over "
                          "n_max x l_max on the 1000-molecule cluster, 'scaling' = descriptor-only on "
                          "3k..1M atoms, 'configs' = the periodic multi-species box and the tiny cluster, "
-                         "'desc30k' = descriptor-only on 30,000 atoms alone (small enough for profiler captures); "
+                         "'desc30k' = descriptor-only on 30,000 atoms alone (small enough for profiler captures), "
+                         "'modes' = crossover off, coefficient mode and the averaged modes on the 1000-molecule cluster; "
                          "prints one JSON line per case")
     args = ap.parse_args()
     if args.impl == "reference":
