@@ -18,6 +18,7 @@ from dataclasses import dataclass
 import numpy as np
 
 from . import basis
+from . import weighting as _weighting
 from .harmonics import real_spherical_harmonics
 
 GTO, POLYNOMIAL = 0, 1
@@ -32,8 +33,10 @@ class Derivatives:
 
 
 class SoapOracle:
-    def __init__(self, species, r_cut, n_max, l_max, sigma, rbf=GTO, pbc=(False, False, False), crossover=True):
+    def __init__(self, species, r_cut, n_max, l_max, sigma, rbf=GTO, pbc=(False, False, False), crossover=True,
+                 weighting=None):
         self.crossover = bool(crossover)
+        self.weighting = dict(weighting) if weighting else None
         self.species = sorted(int(z) for z in species)
         self.r_cut, self.n_max, self.l_max, self.sigma = float(r_cut), int(n_max), int(l_max), float(sigma)
         self.rbf = int(rbf)
@@ -125,16 +128,23 @@ class SoapOracle:
 
     # ---------------------------------------------------------- coefficients
     def radial(self, d):
-        """F[n, l, j], dF/dd[n, l, j] of the chosen basis."""
+        """F[n, l, j], dF/dd[n, l, j] of the chosen basis, times the radial
+        weighting of the neighbour density when one is set."""
         if self.rbf == GTO:
-            return basis.gto_radial(d, self.r_cut, self.n_max, self.l_max, self.sigma)
-        return basis.poly_radial(d, self.r_cut, self.n_max, self.l_max, self.sigma)
+            F, dF = basis.gto_radial(d, self.r_cut, self.n_max, self.l_max, self.sigma)
+        else:
+            F, dF = basis.poly_radial(d, self.r_cut, self.n_max, self.l_max, self.sigma)
+        if self.weighting:
+            w, dw = _weighting.weight(self.weighting, d)
+            F, dF = F * w, dF * w + F * dw
+        return F, dF
 
     def onsite(self):
         """c_n00 contribution of the centre itself (position independent)."""
+        w0 = _weighting.onsite_weight(self.weighting)
         if self.rbf == GTO:
-            return basis.gto_onsite(self.r_cut, self.n_max, self.l_max, self.sigma)
-        return basis.poly_onsite(self.r_cut, self.n_max, self.sigma)
+            return w0 * basis.gto_onsite(self.r_cut, self.n_max, self.l_max, self.sigma)
+        return w0 * basis.poly_onsite(self.r_cut, self.n_max, self.sigma)
 
     def _species_index(self, numbers):
         lut = {z: s for s, z in enumerate(self.species)}

@@ -119,3 +119,106 @@ def test_averages_are_rotation_and_permutation_invariant(mode):
     np.testing.assert_allclose(modes.average_descriptor(o, mode, pos @ R.T, st.numbers), ref, rtol=1e-10, atol=1e-12)
     perm = np.random.default_rng(0).permutation(pos.shape[0])
     np.testing.assert_allclose(modes.average_descriptor(o, mode, pos[perm], st.numbers[perm]), ref, rtol=1e-12)
+
+
+# ----------------------------------------------------------------- radial weighting
+WEIGHTS = [
+    {"function": "poly", "r0": 3.6, "c": 1.3, "m": 2, "w0": 0.6},
+    {"function": "pow", "r0": 1.5, "c": 0.8, "d": 1.2, "m": 3, "w0": 1.4},
+    {"function": "exp", "r0": 0.9, "c": 2.0, "d": 0.5, "w0": 1.0},
+]
+
+
+def _w_plain(spec, d):
+    """The three weight functions typed out once more, scalar, for the pins."""
+    x = d / spec["r0"]
+    if spec["function"] == "poly":
+        return spec["c"] * (1 + 2 * x ** 3 - 3 * x ** 2) ** spec["m"] if x <= 1 else 0.0
+    if spec["function"] == "pow":
+        return spec["c"] / (spec["d"] + x ** spec["m"])
+    return spec["c"] / (spec["d"] + np.exp(-x))
+
+
+@pytest.mark.parametrize("spec", WEIGHTS)
+@pytest.mark.parametrize("rbf", [GTO, POLYNOMIAL])
+def test_weighted_coefficients_against_brute_force_projection(spec, rbf):
+    """Eq. 3 by 3-D quadrature with every neighbour Gaussian of Eq. 1 scaled by w(|r_j|) and the
+    centre's by w0; the radial functions come from the unweighted oracle through Eq. 3 itself:
+    g_nl(r) is recovered as the projection of a delta shell, i.e. taken from `basis`."""
+    from oracle import basis
+    from test_oracle_soap import _scipy_real_harmonics
+    r_cut, n_max, l_max, sigma = 4.0, 2, 2, 0.5
+    pos = np.array([[0.0, 0.0, 0.0], [1.1, 0.7, -0.9], [-1.6, 0.4, 1.2], [0.3, -2.2, 0.8], [2.4, 2.3, 1.7]])
+    numbers = np.array([1, 8, 1, 8, 1])
+    o = SoapOracle([1, 8], r_cut, n_max, l_max, sigma, rbf, weighting=spec)
+    c = o.coefficients(pos, numbers, None, 0)
+    r_hi = r_cut + 10 * sigma if rbf == GTO else r_cut
+    xr, wr = np.polynomial.legendre.leggauss(140)
+    r = 0.5 * r_hi * (xr + 1)
+    wr = 0.5 * r_hi * wr
+    xt, wt = np.polynomial.legendre.leggauss(80)
+    nphi = 160
+    phi = 2 * np.pi * np.arange(nphi) / nphi
+    ct, ph = np.meshgrid(xt, phi, indexing="ij")
+    st = np.sqrt(1 - ct * ct)
+    unit = np.stack([st * np.cos(ph), st * np.sin(ph), ct], -1)
+    Yg = _scipy_real_harmonics(l_max, np.arccos(ct), ph)
+    if rbf == GTO:
+        alpha = basis.gto_alpha(r_cut, n_max, l_max)
+        beta = basis.gto_beta(r_cut, n_max, l_max).astype(np.float64)
+        g = np.array([[beta[l, n] @ (r[None, :] ** l * np.exp(-alpha[l][:, None] * r[None, :] ** 2))
+                       for l in range(l_max + 1)] for n in range(n_max)])
+    else:
+        W = basis.poly_w(n_max).astype(np.float64)
+        N = basis.poly_norm(r_cut, n_max)
+        prim = np.array([(r_cut - r) ** (k + 2) / N[k - 1] for k in range(1, n_max + 1)])
+        g = np.repeat((W @ prim)[:, None, :], l_max + 1, axis=1)
+    ls = np.concatenate([[l] * (2 * l + 1) for l in range(l_max + 1)])
+    for mu, z in enumerate([1, 8]):
+        rho = np.zeros((r.size,) + ct.shape)
+        for j in range(5):
+            if numbers[j] != z:
+                continue
+            dj = np.linalg.norm(pos[j] - pos[0])
+            if j != 0 and dj >= r_cut:
+                continue
+            wj = spec["w0"] if j == 0 else _w_plain(spec, dj)
+            diff = r[:, None, None, None] * unit[None] - pos[j]
+            rho += wj * np.exp(-np.sum(diff * diff, -1) / (2 * sigma ** 2))
+        ang = np.einsum("mtp,rtp,t->mr", Yg, rho, wt) * (2 * np.pi / nphi)
+        ref = np.einsum("nmr,mr,r->nm", g[:, ls, :], ang, wr * r * r)
+        assert np.abs(c[mu] - ref).max() < 5e-9 * max(1.0, np.abs(ref).max())
+
+
+@pytest.mark.parametrize("spec", WEIGHTS)
+def test_weighted_jacobian_by_central_differences(spec):
+    st = small_periodic_cell(seed=6, pbc=(True, True, True))
+    pos = st.positions.astype(np.float64)
+    o = SoapOracle([1, 6, 7, 8], 4.0, 2, 3, 0.5, GTO, pbc=st.pbc, weighting=spec)
+    der = o.derivatives(pos, st.numbers, st.cell, [1, 5])
+    dense = modes._dense(der, pos.shape[0])
+    fd = _fd(lambda p: o.descriptor(p, st.numbers, st.cell, [1, 5]), pos)
+    np.testing.assert_allclose(dense, np.transpose(fd, (2, 0, 1, 3)), rtol=0, atol=3e-8 * np.abs(dense).max())
+
+
+def test_weight_that_vanishes_beyond_r0_removes_those_atoms():
+    spec = {"function": "poly", "r0": 2.5, "c": 1.0, "m": 1, "w0": 1.0}
+    st = water_cluster(4, seed=2)
+    pos = st.positions.astype(np.float64)
+    o = SoapOracle([1, 8], 5.0, 3, 3, 0.5, weighting=spec)
+    near = np.nonzero(np.linalg.norm(pos - pos[0], axis=1) <= 2.5)[0]      # atom 0 itself included
+    assert near.size < pos.shape[0]
+    np.testing.assert_allclose(o.descriptor(pos, st.numbers, centers=[0])[0],
+                               o.descriptor(pos[near], st.numbers[near], centers=[0])[0], rtol=1e-13)
+
+
+def test_constant_weight_scales_the_neighbour_terms():
+    st = water_cluster(3, seed=8)
+    pos = st.positions.astype(np.float64)
+    plain = SoapOracle([1, 8], 4.0, 2, 2, 0.5, POLYNOMIAL)
+    spec = {"function": "pow", "r0": 1.0, "c": 3.0, "d": 1.0, "m": 0.0, "w0": 0.5}        # w = 3 / (1 + 1) everywhere
+    weighted = SoapOracle([1, 8], 4.0, 2, 2, 0.5, POLYNOMIAL, weighting=spec)
+    c0 = plain.coefficients(pos, st.numbers, None, 2)
+    on = np.zeros_like(c0)
+    on[plain._species_index(st.numbers)[2], :, 0] = plain.onsite()
+    np.testing.assert_allclose(weighted.coefficients(pos, st.numbers, None, 2), 1.5 * (c0 - on) + 0.5 * on, rtol=1e-12)
