@@ -148,6 +148,22 @@ int soap_jacobian_dense(soap_t *h, const float *d_jac_rows, const int64_t *d_row
  * Not to be called while work on this handle is in flight. */
 int soap_set_crossover(soap_t *h, int crossover);
 
+enum { SOAP_WEIGHT_NONE = 0, SOAP_WEIGHT_POLY = 1, SOAP_WEIGHT_POW = 2, SOAP_WEIGHT_EXP = 3 };
+
+/* Radial weighting of the neighbour density (the `weighting` argument of the
+ * paper's constructor, which names the option and gives no formula; the forms
+ * are our reading): the Gaussian of a neighbour at distance dist from the
+ * centre (Eq. 1) is scaled by
+ *   POLY: c (1 + 2 x^3 - 3 x^2)^m for x = dist/r0 <= 1, else 0   (d unused)
+ *   POW:  c / (d + x^m)
+ *   EXP:  c / (d + exp(-x))                                         (m unused)
+ * and the centre's own Gaussian (on-site term of Eq. 13) by w0.  The weight
+ * multiplies the neighbour's whole term, so the Jacobian gains the product-rule
+ * term w'(dist).  Evaluated per pair in fp64 by a kernel of its own after the
+ * neighbour search.  SOAP_WEIGHT_NONE switches it off.  Not to be called while
+ * work on this handle is in flight (it may wait for the device and reallocate). */
+int soap_set_weighting(soap_t *h, int function, double r0, double c, double d, double m, double w0);
+
 /* Number of expansion coefficients per centre, W = S n_max (l_max+1)^2. */
 int soap_num_coefficients(const soap_t *h, int64_t *n_coefficients);
 

@@ -9,13 +9,14 @@ import numpy as np
 
 GTO, POLYNOMIAL = 0, 1
 AVERAGE_MODES = {"inner": 1, "outer": 2}
+WEIGHT_FUNCTIONS = {"poly": 1, "pow": 2, "exp": 3}
 
 EXPORTED_SYMBOLS = [
     "soap_create", "soap_destroy", "soap_num_features", "soap_feature_info", "soap_last_error",
     "soap_radial_table", "soap_neighbors", "soap_neighbor_list", "soap_descriptor",
     "soap_derivatives", "soap_status", "soap_profile", "soap_profile_read", "soap_neighbor_counts_static", "soap_jacobian_dense",
     "soap_set_crossover", "soap_num_coefficients", "soap_coefficients", "soap_coefficient_derivatives",
-    "soap_descriptor_average", "soap_derivatives_average",
+    "soap_descriptor_average", "soap_derivatives_average", "soap_set_weighting",
 ]
 
 _ERRORS = {-1: "SOAP_ERR_INVALID_ARG", -2: "SOAP_ERR_UNKNOWN_SPECIES", -3: "SOAP_ERR_CAPACITY",
@@ -63,6 +64,7 @@ def load_library() -> C.CDLL:
     lib.soap_neighbor_counts_static.argtypes = [vp, i64, C.c_double, vp, vp, C.c_char_p, i64]
     lib.soap_jacobian_dense.argtypes = [vp, vp, vp, vp, i64, vp, i64, vp, vp]
     lib.soap_set_crossover.argtypes = [vp, i32]
+    lib.soap_set_weighting.argtypes = [vp, i32] + [C.c_double] * 5
     lib.soap_num_coefficients.argtypes = [vp, C.POINTER(i64)]
     lib.soap_coefficients.argtypes = common + [vp, vp]
     lib.soap_coefficient_derivatives.argtypes = common + [vp, vp, i64, vp, vp, vp]
@@ -107,7 +109,10 @@ class Derivatives:
 class Soap:
     """One descriptor configuration (the arguments of soap_create)."""
 
-    def __init__(self, species, r_cut, n_max, l_max, sigma, rbf=GTO, pbc=(False, False, False), crossover=True):
+    def __init__(self, species, r_cut, n_max, l_max, sigma, rbf=GTO, pbc=(False, False, False), crossover=True,
+                 weighting=None):
+        """`weighting`: None or {"function": "poly" | "pow" | "exp", "r0", "c", "m", "d", "w0"} (see
+        soap_set_weighting in include/soap.h)."""
         self._lib = load_library()
         self._h = C.c_void_p()
         sp = (C.c_int32 * len(species))(*[int(z) for z in species])
@@ -121,6 +126,10 @@ class Soap:
         n = C.c_int64()
         if not crossover:
             self._check(self._lib.soap_set_crossover(self._h, 0))
+        if weighting:
+            self._check(self._lib.soap_set_weighting(
+                self._h, WEIGHT_FUNCTIONS[weighting["function"]], float(weighting["r0"]), float(weighting.get("c", 1.0)),
+                float(weighting.get("d", 1.0)), float(weighting.get("m", 1.0)), float(weighting.get("w0", 1.0))))
         self._check(self._lib.soap_num_features(self._h, C.byref(n)))
         self.n_features = int(n.value)
         self._check(self._lib.soap_num_coefficients(self._h, C.byref(n)))

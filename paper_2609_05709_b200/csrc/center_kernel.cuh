@@ -136,11 +136,12 @@ center_kernel(const CenterParams p) {
     }
     const int S = p.S, NMAX = NMAX_T ? NMAX_T : p.n_max, NCH = NMAX * L1, NE = NMAX * LM;
     const int CT = S * NMAX * LMP, P = p.P, F = p.F;
-    const SmemLayout lay = make_layout(S, NMAX, L, P, DERIV);
+    const SmemLayout lay = make_layout(S, NMAX, L, P, DERIV, p.pair_w != nullptr);
     float* c_t = smem + lay.c;                                             // [S][NMAX][LMP]
     float4* geo_d = reinterpret_cast<float4*>(smem + lay.geo);             // [GP] dx, dy, dz, r
     int4* geo_i = reinterpret_cast<int4*>(smem + lay.geo + 4 * kGeoPairs);   // [GP] interval, t bits, species|moving<<8, row word
     int* geo_j = reinterpret_cast<int*>(smem + lay.geo + 8 * kGeoPairs);     // [GP] neighbour atom
+    float2* geo_w = reinterpret_cast<float2*>(smem + lay.geo + kGeoWords);   // [GP] (w, w'/d), only with a radial weighting
     float* D_t = smem + lay.D;                                             // [3][CT]    (pass 1 and the centre's row)
     float* sS = smem + lay.sSD;                                            // [P][LMP]   values            (descriptor build)
     float4* sSD4 = reinterpret_cast<float4*>(smem + lay.sSD);              // [P][LMP]   (S, dSx, dSy, dSz) (derivative build)
@@ -183,6 +184,7 @@ center_kernel(const CenterParams p) {
     auto stage_geometry = [&](int g0, int gc) -> bool {
         int special = 0, sp = -1, rank = 0, rw = 0, j = 0;
         float4 dd = make_float4(0.f, 0.f, 0.f, 0.f);
+        float2 wgt = make_float2(1.f, 0.f);
         int qi = 0;
         float tt = 0.f;
         if (tid < kGeoPairs) {
@@ -202,6 +204,7 @@ center_kernel(const CenterParams p) {
                 const double r = sqrt(dx * dx + dy * dy + dz * dz);
                 dd = make_float4((float)dx, (float)dy, (float)dz, (float)r);
                 rw = p.pair_row[pair_base + g0 + tid];
+                if (p.pair_w) wgt = p.pair_w[pair_base + g0 + tid];
                 special = rw & (kRowSelfImage | kRowContinuation);
                 // interval and offset in the radial table, in fp64 so that the offset keeps its digits
                 const double u = r * (double)p.inv_h;
@@ -225,6 +228,7 @@ center_kernel(const CenterParams p) {
             geo_d[at] = dd;
             geo_i[at] = make_int4(qi, __float_as_int(tt), sp | ((rw & kRowSelfImage) ? 0 : 256), rw);
             geo_j[at] = j;
+            if (p.pair_w) geo_w[at] = wgt;
         }
         if (tid <= S) {
             int at = 0;
@@ -244,6 +248,17 @@ center_kernel(const CenterParams p) {
             const int4 gi = geo_i[g + pr];
             const float t = __int_as_float(gi.y);
             const float rinv_h = GRAD ? p.inv_h / geo_d[g + pr].w : 0.f;
+            if (p.pair_w) {
+                // radial weighting: G -> w G, Ghat -> w Ghat + (w'/d) G
+                const float2 w = geo_w[g + pr];
+                for (int ch = lane; ch < NCH; ch += 32) {
+                    float v, dv;
+                    radial_lookup(p.table, gi.x, NCH, ch, t, v, dv);
+                    if (GRAD) sG2[pr * NCH + ch] = make_float2(v * w.x, fmaf(dv * rinv_h, w.x, v * w.y));
+                    else sG1[pr * NCH + ch] = v * w.x;
+                }
+                continue;
+            }
             for (int ch = lane; ch < NCH; ch += 32) {
                 float v, dv;
                 radial_lookup(p.table, gi.x, NCH, ch, t, v, dv);
@@ -330,7 +345,7 @@ center_kernel(const CenterParams p) {
     }
     __syncthreads();
     // on-site term: the centre's own Gaussian, l = 0 only (second term of Eq. 13)
-    if (tid < NMAX && !p.c_bar) c_t[(zi_species * NMAX + tid) * LMP] += __ldg(p.self_term + tid);
+    if (tid < NMAX && !p.c_bar) c_t[(zi_species * NMAX + tid) * LMP] += p.w0 * __ldg(p.self_term + tid);
     __syncthreads();
     const int W = S * NE;                                                  // coefficients per centre
     const int RW = CC ? W : F;                                             // width of an output row

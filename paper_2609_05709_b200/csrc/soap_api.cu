@@ -16,6 +16,7 @@
 #include "dense_kernel.cuh"
 #include "neighbor_kernels.cuh"
 #include "soap.h"
+#include "weight_kernel.cuh"
 
 using namespace soap;
 
@@ -53,6 +54,8 @@ struct soap_handle {
     double r_cut = 0, sigma = 0;
     int pbc[3] = {0, 0, 0};
     int crossover = 1;
+    WeightParams weight = {0, 1.0, 1.0, 1.0, 1.0};   // radial weighting of the neighbour density (off)
+    double w0 = 1.0;
     int64_t F = 0;
     HostBasis basis;
     std::vector<int> feat_pack;
@@ -77,6 +80,7 @@ struct soap_handle {
     int* d_tile_sums = nullptr;
     unsigned long long *d_pair_key = nullptr, *d_pair_tmp = nullptr;
     int* d_pair_row = nullptr;
+    float2* d_pair_w = nullptr;          // per-pair weights, only with a radial weighting
     void* d_work = nullptr;              // workspace of the averaged modes
     size_t cap_work = 0;
     // plan
@@ -149,6 +153,39 @@ int make_geometry(soap_t* h, const double* cell, Geometry& g) {
     return SOAP_OK;
 }
 
+// Shared-memory plan of the per-centre kernels (depends on the basis and on whether pairs carry weights).
+int plan_smem(soap_t* h) {
+    // shared-memory plan of the per-centre kernels
+    int max_smem = 0;
+    CU(cudaDeviceGetAttribute(&max_smem, cudaDevAttrMaxSharedMemoryPerBlockOptin, h->device));
+    for (int deriv = 0; deriv < 2; ++deriv) {
+        // largest chunk that still leaves room for three CTAs per SM, else two, else whatever fits
+        int P = 32;
+        size_t bytes = 0;
+        const size_t budget3 = (size_t)228 * 1024 / 3 - 1024, budget2 = (size_t)228 * 1024 / 2 - 1024;
+        for (int pass = 0; pass < 3; ++pass) {
+            const size_t budget = pass == 0 ? budget3 : pass == 1 ? budget2 : (size_t)max_smem;
+            for (P = 32; P >= 4; P /= 2) {
+                bytes = (size_t)make_layout(h->S, h->n_max, h->l_max, P, deriv, h->weight.fn != 0).total * 4;
+                if (bytes <= budget) break;
+            }
+            if (P >= (pass == 2 ? 4 : 8) && bytes <= budget) break;
+            if (P < 4) P = 4;
+        }
+        if (const char* env = std::getenv("SOAP_B200_CHUNK")) {       // tuning knob: pairs staged per chunk (4..32)
+            const int v = std::atoi(env);
+            if (v >= 4 && v <= 32) P = v;
+        }
+        bytes = (size_t)make_layout(h->S, h->n_max, h->l_max, P, deriv, h->weight.fn != 0).total * 4;
+        if (bytes > (size_t)max_smem) return fail(h, SOAP_ERR_INVALID_ARG, "this basis does not fit the shared memory of the device");
+        if (deriv) { h->P_deriv = P; h->smem_deriv = bytes; } else { h->P_desc = P; h->smem_desc = bytes; }
+    }
+    CU(center_set_smem(kCenterDesc, h->l_max, h->n_max, (int)h->smem_desc));
+    CU(center_set_smem(kCenterDeriv, h->l_max, h->n_max, (int)h->smem_deriv));
+    CU(center_set_smem(kCenterCoeff, h->l_max, h->n_max, (int)h->smem_deriv));
+    return SOAP_OK;
+}
+
 int ensure_device(soap_t* h) {
     int dev = -1;
     cudaError_t e = cudaGetDevice(&dev);
@@ -176,31 +213,7 @@ int ensure_device(soap_t* h) {
     CU(cudaMalloc((void**)&h->d_bbox, 64));
     CU(cudaMalloc((void**)&h->d_grid, sizeof(GridParams)));
     CU(cudaMallocHost((void**)&h->h_counters, sizeof(Counters)));
-    // shared-memory plan of the per-centre kernels
-    int max_smem = 0;
-    CU(cudaDeviceGetAttribute(&max_smem, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev));
-    for (int deriv = 0; deriv < 2; ++deriv) {
-        // largest chunk that still leaves room for three CTAs per SM, else two, else whatever fits
-        int P = 32;
-        size_t bytes = 0;
-        const size_t budget3 = (size_t)228 * 1024 / 3 - 1024, budget2 = (size_t)228 * 1024 / 2 - 1024;
-        for (int pass = 0; pass < 3; ++pass) {
-            const size_t budget = pass == 0 ? budget3 : pass == 1 ? budget2 : (size_t)max_smem;
-            for (P = 32; P >= 4; P /= 2) {
-                bytes = (size_t)make_layout(h->S, h->n_max, h->l_max, P, deriv).total * 4;
-                if (bytes <= budget) break;
-            }
-            if (P >= (pass == 2 ? 4 : 8) && bytes <= budget) break;
-            if (P < 4) P = 4;
-        }
-        if (const char* env = std::getenv("SOAP_B200_CHUNK")) {       // tuning knob: pairs staged per chunk (4..32)
-            const int v = std::atoi(env);
-            if (v >= 4 && v <= 32) P = v;
-        }
-        bytes = (size_t)make_layout(h->S, h->n_max, h->l_max, P, deriv).total * 4;
-        if (bytes > (size_t)max_smem) return fail(h, SOAP_ERR_INVALID_ARG, "this basis does not fit the shared memory of the device");
-        if (deriv) { h->P_deriv = P; h->smem_deriv = bytes; } else { h->P_desc = P; h->smem_desc = bytes; }
-    }
+    if (int rc = plan_smem(h)) return rc;
     {
         // universal harmonic tables up to l = 12 (the handle's own tables stop at its l_max)
         std::vector<float> anorm(91, 0.f), dfact(16, 0.f);
@@ -208,9 +221,6 @@ int ensure_device(soap_t* h) {
         for (size_t i = 0; i < h->basis.dfact.size(); ++i) dfact[i] = h->basis.dfact[i];
         CU(center_constants(h->l_max, anorm.data(), dfact.data()));
     }
-    CU(center_set_smem(kCenterDesc, h->l_max, h->n_max, (int)h->smem_desc));
-    CU(center_set_smem(kCenterDeriv, h->l_max, h->n_max, (int)h->smem_deriv));
-    CU(center_set_smem(kCenterCoeff, h->l_max, h->n_max, (int)h->smem_deriv));
     h->tables_ready = true;
     return SOAP_OK;
 }
@@ -247,6 +257,7 @@ int ensure_scratch(soap_t* h, int64_t N, int64_t C, int64_t pairs) {
         CU(regrow(&h->d_pair_key, cap));
         CU(regrow(&h->d_pair_tmp, cap));
         CU(regrow(&h->d_pair_row, cap));
+        if (h->weight.fn) CU(regrow(&h->d_pair_w, cap));
         h->cap_pairs = cap;
     }
     return SOAP_OK;
@@ -341,6 +352,7 @@ void fill_center_params(soap_t* h, CenterParams& cp, const float* pos, const int
     cp.S = h->S; cp.n_max = h->n_max; cp.l_max = h->l_max; cp.F = (int)h->F;
     cp.P = deriv ? h->P_deriv : h->P_desc;
     cp.crossover = h->crossover; cp.emit_coeff = 0; cp.c_bar = nullptr;
+    cp.pair_w = h->weight.fn ? h->d_pair_w : nullptr; cp.w0 = (float)h->w0;
     cp.out_desc = nullptr; cp.out_jac = nullptr; cp.row_atom = nullptr;
 }
 
@@ -370,6 +382,11 @@ int prepare(soap_t* h, const float* pos, const int32_t* num, int64_t N, const do
         if ((rc = plan(h, pos, num, N, g, centers, C, st))) return rc;
     }
     if ((rc = launch_neighbors(h, pos, num, N, g, centers, C, row_ptr_out ? row_ptr_out : h->d_row_ptr, st))) return rc;
+    if (h->weight.fn && C > 0) {
+        pair_weight_kernel<<<(unsigned)((C + 7) / 8), 256, 0, st>>>(pos, centers, C, g, h->d_pair_start, h->d_pair_count, h->d_pair_key,
+                                                                   h->cap_pairs, h->d_counters, h->weight, h->d_pair_w);
+        CU(cudaGetLastError());
+    }
     if (h->profiling) CU(cudaEventRecord(h->ev[1], st));
     h->last_centers = C;
     return SOAP_OK;
@@ -442,7 +459,7 @@ void soap_destroy(soap_t* h) {
     void* ptrs[] = {h->d_table, h->d_self, h->d_kl, h->d_feat, h->d_zlut, h->d_l_of_lm, h->d_counters, h->d_bbox,
                     h->d_grid, h->d_species_idx, h->d_atom_cell, h->d_atom_wrap, h->d_s_wrap, h->d_s_pos, h->d_cell_count,
                     h->d_cell_start, h->d_pair_count, h->d_row_count, h->d_self_row, h->d_order, h->d_pair_ptr, h->d_pair_start, h->d_row_ptr, h->d_tile_sums, h->d_tile_offsets,
-                    h->d_pair_key, h->d_pair_tmp, h->d_pair_row, h->d_work};
+                    h->d_pair_key, h->d_pair_tmp, h->d_pair_row, h->d_work, h->d_pair_w};
     for (void* p : ptrs) if (p) cudaFree(p);
     if (h->h_counters) cudaFreeHost(h->h_counters);
     for (cudaEvent_t e : h->ev) if (e) cudaEventDestroy(e);
@@ -507,20 +524,11 @@ int soap_neighbor_list(soap_t* h, int64_t* d_pair_ptr, int32_t* d_pair_atom, int
 
 int soap_descriptor(soap_t* h, const float* d_positions, const int32_t* d_numbers, int64_t n_atoms, const double* cell,
                     const int32_t* d_centers, int64_t n_centers, float* d_out, void* stream) {
-    int rc = check_inputs(h, d_positions, d_numbers, n_atoms, d_centers, n_centers);
-    if (rc) return rc;
-    if (n_centers > 0 && !d_out) return fail(h, SOAP_ERR_INVALID_ARG, "d_out must not be NULL");
-    if ((rc = ensure_device(h))) return rc;
+    if (h && n_centers > 0 && !d_out) return fail(h, SOAP_ERR_INVALID_ARG, "d_out must not be NULL");
     Geometry g;
-    if ((rc = make_geometry(h, cell, g))) return rc;
     cudaStream_t st = (cudaStream_t)stream;
-    if (h->profiling) CU(cudaEventRecord(h->ev[0], st));
-    if (h->planned_atoms != n_atoms || h->planned_centers != n_centers) {
-        if ((rc = plan(h, d_positions, d_numbers, n_atoms, g, d_centers, n_centers, st))) return rc;
-    }
-    if ((rc = launch_neighbors(h, d_positions, d_numbers, n_atoms, g, d_centers, n_centers, h->d_row_ptr, st))) return rc;
-    if (h->profiling) CU(cudaEventRecord(h->ev[1], st));
-    h->last_centers = n_centers;
+    int rc = prepare(h, d_positions, d_numbers, n_atoms, cell, d_centers, n_centers, nullptr, g, st);
+    if (rc) return rc;
     if (n_centers > 0) {
         CenterParams cp;
         fill_center_params(h, cp, d_positions, d_centers, n_centers, g, false);
@@ -534,21 +542,12 @@ int soap_descriptor(soap_t* h, const float* d_positions, const int32_t* d_number
 int soap_derivatives(soap_t* h, const float* d_positions, const int32_t* d_numbers, int64_t n_atoms, const double* cell,
                      const int32_t* d_centers, int64_t n_centers, float* d_out_desc, float* d_out_jac,
                      int64_t capacity_rows, int64_t* d_row_ptr, int32_t* d_row_atom, void* stream) {
-    int rc = check_inputs(h, d_positions, d_numbers, n_atoms, d_centers, n_centers);
-    if (rc) return rc;
-    if (!d_row_ptr || capacity_rows < 0) return fail(h, SOAP_ERR_INVALID_ARG, "d_row_ptr must not be NULL");
-    if (n_centers > 0 && (!d_out_desc || !d_out_jac || !d_row_atom)) return fail(h, SOAP_ERR_INVALID_ARG, "output pointers must not be NULL");
-    if ((rc = ensure_device(h))) return rc;
+    if (h && (!d_row_ptr || capacity_rows < 0)) return fail(h, SOAP_ERR_INVALID_ARG, "d_row_ptr must not be NULL");
+    if (h && n_centers > 0 && (!d_out_desc || !d_out_jac || !d_row_atom)) return fail(h, SOAP_ERR_INVALID_ARG, "output pointers must not be NULL");
     Geometry g;
-    if ((rc = make_geometry(h, cell, g))) return rc;
     cudaStream_t st = (cudaStream_t)stream;
-    if (h->profiling) CU(cudaEventRecord(h->ev[0], st));
-    if (h->planned_atoms != n_atoms || h->planned_centers != n_centers) {
-        if ((rc = plan(h, d_positions, d_numbers, n_atoms, g, d_centers, n_centers, st))) return rc;
-    }
-    if ((rc = launch_neighbors(h, d_positions, d_numbers, n_atoms, g, d_centers, n_centers, (long long*)d_row_ptr, st))) return rc;
-    if (h->profiling) CU(cudaEventRecord(h->ev[1], st));
-    h->last_centers = n_centers;
+    int rc = prepare(h, d_positions, d_numbers, n_atoms, cell, d_centers, n_centers, (long long*)d_row_ptr, g, st);
+    if (rc) return rc;
     if (n_centers > 0) {
         CenterParams cp;
         fill_center_params(h, cp, d_positions, d_centers, n_centers, g, true);
@@ -585,6 +584,31 @@ int soap_set_crossover(soap_t* h, int crossover) {
         cudaFree(h->d_feat);
         h->d_feat = nullptr;
         CU(upload(&h->d_feat, h->feat_pack));
+    }
+    return SOAP_OK;
+}
+
+int soap_set_weighting(soap_t* h, int function, double r0, double c, double d, double m, double w0) {
+    if (!h) return SOAP_ERR_INVALID_ARG;
+    if (function < SOAP_WEIGHT_NONE || function > SOAP_WEIGHT_EXP) return fail(h, SOAP_ERR_INVALID_ARG, "unknown weighting function");
+    if (function != SOAP_WEIGHT_NONE) {
+        if (!(r0 > 0) || !std::isfinite(c) || !std::isfinite(w0)) return fail(h, SOAP_ERR_INVALID_ARG, "weighting needs r0 > 0 and finite c, w0");
+        if (function == SOAP_WEIGHT_POLY && !(m >= 0)) return fail(h, SOAP_ERR_INVALID_ARG, "poly weighting needs m >= 0");
+        if (function == SOAP_WEIGHT_POW && (!(m >= 0) || !(d > 0))) return fail(h, SOAP_ERR_INVALID_ARG, "pow weighting needs m >= 0 and d > 0");
+        if (function == SOAP_WEIGHT_EXP && !(d >= 0)) return fail(h, SOAP_ERR_INVALID_ARG, "exp weighting needs d >= 0");
+    }
+    const bool was = h->weight.fn != 0, now = function != SOAP_WEIGHT_NONE;
+    h->weight = WeightParams{function, now ? r0 : 1.0, now ? c : 1.0, d, m};
+    h->w0 = now ? w0 : 1.0;
+    if (was != now) {
+        // the pair scratch gains or loses the weight array and the kernels' shared memory changes
+        h->planned_atoms = -1;
+        if (h->tables_ready) {
+            CU(cudaDeviceSynchronize());
+            if (h->d_pair_w) { cudaFree(h->d_pair_w); h->d_pair_w = nullptr; }
+            if (now) CU(regrow(&h->d_pair_w, (size_t)std::max<int64_t>(h->cap_pairs, 1)));
+            if (int rc = plan_smem(h)) return rc;
+        }
     }
     return SOAP_OK;
 }

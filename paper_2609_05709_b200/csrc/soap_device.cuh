@@ -78,6 +78,9 @@ struct CenterParams {
     int crossover;                // 0: only the species pairs mu == nu are features
     int emit_coeff;               // descriptor build: write the coefficients c^mu_nlm instead of the power spectrum
     const float* c_bar;           // [S n_max (l_max+1)^2] or null: coefficients that replace the centre's own after pass 1
+    // radial weighting of the neighbour density: per pair (w(d), w'(d)/d), null when off; w0 scales the on-site term
+    const float2* pair_w;
+    float w0;
     // outputs
     float* out_desc;              // [C,F]  (coefficient mode: [C, S n_max (l_max+1)^2]; with c_bar: [F])
     float* out_jac;               // [rows,3,F]  (coefficient mode: [rows, 3, S n_max (l_max+1)^2])
@@ -101,12 +104,13 @@ struct SmemLayout {
     int c, geo, tri, D, wUV, sSD, sG, total;
 };
 __host__ __device__ inline int align4(int x) { return (x + 3) & ~3; }
-__host__ __device__ inline SmemLayout make_layout(int S, int n_max, int l_max, int P, bool deriv) {
+constexpr int kGeoWords = kGeoPairs * 9 + 44;   // geometry (9 words per pair), species segments (9 + 32 words, padded)
+__host__ __device__ inline SmemLayout make_layout(int S, int n_max, int l_max, int P, bool deriv, bool weighted = false) {
     const int L1 = l_max + 1, LMP = (L1 * L1) | 1, NCH = n_max * L1, CT = S * n_max * LMP;
     SmemLayout o;
     int off = 0;
     o.c = off; off = align4(off + CT);
-    o.geo = off; off = align4(off + kGeoPairs * 9 + (kMaxSpecies + 1) + (kGeoPairs / 32) * kMaxSpecies);   // + species segments
+    o.geo = off; off = align4(off + kGeoWords + (weighted ? 2 * kGeoPairs : 0));   // + per-pair weights
     o.tri = off; if (deriv) off = align4(off + ((n_max * (n_max + 1) / 2) * L1 + 1) / 2);   // 16-bit entries
     // the D tiles (pass 1, centre's row) and the per-warp U/V staging (pass 2) never live
     // at the same time and share space

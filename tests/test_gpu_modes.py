@@ -172,3 +172,45 @@ def test_average_argument_errors(pkg):
     out = torch.empty(soap.n_features, device="cuda")
     rc = soap._lib.soap_descriptor_average(soap._h, 7, pos.data_ptr(), num.data_ptr(), 6, None, None, 6, out.data_ptr(), None)
     assert rc == -1
+
+
+# ----------------------------------------------------------------- radial weighting
+WEIGHTS = [
+    {"function": "poly", "r0": 4.2, "c": 1.3, "m": 2, "w0": 0.6},
+    {"function": "poly", "r0": 3.1, "c": 1.0, "m": 1, "w0": 1.0},       # cuts inside the sphere, kink in w'' at r0
+    {"function": "pow", "r0": 1.5, "c": 0.8, "d": 1.2, "m": 3, "w0": 1.4},
+    {"function": "exp", "r0": 0.9, "c": 2.0, "d": 0.5, "w0": 1.0},
+]
+
+
+@pytest.mark.parametrize("spec", WEIGHTS)
+@pytest.mark.parametrize("case", ["water_gto", "periodic_poly"])
+def test_radial_weighting(pkg, spec, case):
+    if case == "water_gto":
+        s, args = water_cluster(15, 2), ([1, 8], 5.0, 6, 5, 0.5, GTO, (False, False, False))
+    else:
+        s, args = small_periodic_cell(7, (True, True, True)), ([1, 6, 7, 8], 4.5, 3, 3, 0.5, POLYNOMIAL, (True, True, True))
+    soap = pkg.Soap(*args, weighting=spec)
+    oracle = SoapOracle(*args, weighting=spec)
+    check_derivatives(soap, oracle, s)
+    pos, num = dev(s)
+    ref = modes.coefficient_derivatives(oracle, s.positions, s.numbers, s.cell)
+    out = soap.coefficient_derivatives(pos, num, s.cell)
+    assert col_err(out.descriptor.cpu().numpy(), ref.descriptor, 0) < DESC_TOL
+    assert col_err(out.jacobian.cpu().numpy(), ref.jacobian, (0, 1)) < JAC_TOL
+
+
+def test_weighting_can_be_switched_on_a_live_handle(pkg):
+    s = water_cluster(10, 5)
+    pos, num = dev(s)
+    args = ([1, 8], 5.0, 4, 4, 0.5, GTO)
+    soap = pkg.Soap(*args)
+    plain = soap.derivatives(pos, num)
+    spec = WEIGHTS[0]
+    soap._check(soap._lib.soap_set_weighting(soap._h, 1, spec["r0"], spec["c"], 1.0, float(spec["m"]), spec["w0"]))
+    check_derivatives(soap, SoapOracle(*args, weighting=spec), s)
+    soap._check(soap._lib.soap_set_weighting(soap._h, 0, 0.0, 0.0, 0.0, 0.0, 0.0))
+    again = soap.derivatives(pos, num)
+    assert torch.equal(again.jacobian, plain.jacobian) and torch.equal(again.descriptor, plain.descriptor)
+    with pytest.raises(pkg.SoapError, match="r0 > 0"):
+        soap._check(soap._lib.soap_set_weighting(soap._h, 2, -1.0, 1.0, 1.0, 1.0, 1.0))
