@@ -404,6 +404,21 @@ def run_suite(args):
             r = time_case(s, [1, 8], 5.0, 8, 6, 0.5, 0, "descriptor", steps)
             r["case"] = "scaling"
             print(json.dumps(r), flush=True)
+    elif args.suite == "driver":
+        # the multi-process driver on the GPUs of this machine (one worker per GPU): wall time between the
+        # start signal and the last result on the host, results travelling through shared memory
+        from paper_2609_05709_b200 import driver
+        s = water_cluster(1000, 0)
+        config = dict(species=[1, 8], r_cut=6.0, n_max=8, l_max=6, sigma=0.5)
+        world = max(1, min(args.gpus, torch.cuda.device_count()))
+        for derivatives, batch in ((True, 256), (True, 1024), (False, 1024)):
+            best = None
+            for _ in range(max(1, min(steps, 3))):
+                _, seconds = driver.generate(config, [s], batch=batch, derivatives=derivatives, world=world)
+                best = seconds if best is None else min(best, seconds)
+            print(json.dumps({"case": "driver", "workers": world, "atoms": s.n_atoms, "batch": batch,
+                              "mode": "derivatives" if derivatives else "descriptor", "seconds": best,
+                              "atoms_per_s": s.n_atoms / best}), flush=True)
     elif args.suite == "modes":
         s = water_cluster(1000, 0)
         base = ([1, 8], 6.0, 8, 6, 0.5, 0)
@@ -432,11 +447,12 @@ def main():
     ap.add_argument("--workload", default=DEFAULT_WORKLOAD, choices=sorted(WORKLOADS))
     ap.add_argument("--kernel-only", action="store_true",
                     help="skip the end-to-end and CPU-baseline legs (for profiler captures)")
-    ap.add_argument("--suite", choices=["map", "scaling", "configs", "desc30k", "modes"],
+    ap.add_argument("--suite", choices=["map", "scaling", "configs", "desc30k", "modes", "driver"],
                     help="extra measurements beside the headline line: 'map' = descriptor+Jacobian over "
                          "n_max x l_max on the 1000-molecule cluster, 'scaling' = descriptor-only on "
                          "3k..1M atoms, 'configs' = the periodic multi-species box and the tiny cluster, "
                          "'desc30k' = descriptor-only on 30,000 atoms alone (small enough for profiler captures), "
+                         "'driver' = the multi-process driver with --gpus workers, results on the host, "
                          "'modes' = crossover off, coefficient mode and the averaged modes on the 1000-molecule cluster; "
                          "prints one JSON line per case")
     args = ap.parse_args()
