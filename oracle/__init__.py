@@ -42,6 +42,9 @@ Parity status of each function (what pins it, in tests/test_oracle_*.py):
   (bilinear double sum over centre pairs for the inner average, one-centre
   and translation-equivalent-centre reductions to the plain descriptor,
   rotation / permutation invariance, central finite differences)
+* modes.site_derivatives (centres that are not atoms) ....... pinned
+  (a ghost atom of a species of its own placed at the point, central finite
+  differences)
 * weighting.weight (radial weighting of the density) ....... pinned
   (brute-force 3-D quadrature of Eq. 3 over weighted Gaussians, central
   finite differences, atoms beyond a vanishing weight drop out, constant

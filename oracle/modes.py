@@ -106,3 +106,41 @@ def average_derivatives(o: SoapOracle, mode: str, positions, numbers, cell=None,
         k = np.pi * np.sqrt(8.0 / (2 * l + 1))
         jac[:, :, f] = k * (dcbar[:, :, mu, n, sl] @ cbar[nu, n2, sl] + dcbar[:, :, nu, n2, sl] @ cbar[mu, n, sl])
     return o.power_spectrum(cbar), jac
+
+
+# ------------------------------------------------------------------ centres that are not atoms
+def site_derivatives(o: SoapOracle, positions, numbers, sites, cell=None) -> Derivatives:
+    """Descriptor and Jacobian for centres at arbitrary Cartesian points (the interface accepts
+    an explicit list of centres; a point that is no atom has no Gaussian of its own, hence no
+    on-site term, and no row of its own: it does not move with any atom).  Otherwise Eqs. 4
+    and 5 exactly as for atom centres.  A point that coincides with an atom drops that atom
+    (the neighbour test is 0 < d^2): use the atom as the centre instead."""
+    pos = np.asarray(positions, np.float64)
+    sp = o._species_index(numbers)
+    sites = np.asarray(sites, np.float64).reshape(-1, 3)
+    lists = o.neighbor_list(pos, cell, sites=sites)
+    LM = (o.l_max + 1) ** 2
+    desc = np.empty((len(sites), o.n_features))
+    row_ptr, row_atom, blocks = [0], [], []
+    for a, site in enumerate(sites):
+        nbrs = lists[a]
+        d = o._displacements(pos, cell, site, nbrs)
+        t, g = o._pair_terms(d, True)                                  # [pair, n, lm], [pair, dir, n, lm]
+        c = np.zeros((o.S, o.n_max, LM))
+        atoms = sorted(set(n[0] for n in nbrs))
+        local = {atom: r for r, atom in enumerate(atoms)}
+        dc = np.zeros((len(atoms), 3, o.S, o.n_max, LM))               # grad_j c^mu_nlm, images of an atom add up
+        for e, n in enumerate(nbrs):
+            c[sp[n[0]]] += t[e]
+            dc[local[n[0]], :, sp[n[0]]] += g[e]
+        desc[a] = o.power_spectrum(c)
+        J = np.empty((len(atoms), 3, o.n_features))
+        for f, (mu, nu, n1, n2, l) in enumerate(o.table):               # Eq. 5
+            sl = slice(l * l, (l + 1) ** 2)
+            k = np.pi * np.sqrt(8.0 / (2 * l + 1))
+            J[:, :, f] = k * (dc[:, :, mu, n1, sl] @ c[nu, n2, sl] + dc[:, :, nu, n2, sl] @ c[mu, n1, sl])
+        row_ptr.append(row_ptr[-1] + len(atoms))
+        row_atom.extend(atoms)
+        blocks.append(J)
+    jac = np.concatenate(blocks, axis=0) if blocks else np.zeros((0, 3, o.n_features))
+    return Derivatives(desc, np.array(row_ptr, np.int64), np.array(row_atom, np.int32), jac)

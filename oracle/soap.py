@@ -70,9 +70,11 @@ class SoapOracle:
         return [vol / np.linalg.norm(np.cross(cell[(a + 1) % 3], cell[(a + 2) % 3]))
                 for a in range(3)]
 
-    def neighbor_list(self, positions, cell=None, centers=None):
+    def neighbor_list(self, positions, cell=None, centers=None, sites=None):
         """For every centre the sorted list of (atom j, n_a, n_b, n_c) with
-        0 < |r_j + n_a a + n_b b + n_c c - r_i|^2 < r_cut^2.
+        0 < |r_j + n_a a + n_b b + n_c c - r_i|^2 < r_cut^2.  With `sites`
+        (an array of Cartesian points) the centres are those points instead of
+        atoms: r_i is the point.
 
         The displacement is formed as (r_j - r_i) + T with the lattice
         translation T = (n_a a + n_b b) + n_c c, each step rounded to fp64 in
@@ -81,11 +83,12 @@ class SoapOracle:
         pos = np.asarray(positions, np.float64)
         N = pos.shape[0]
         centers = np.arange(N) if centers is None else np.asarray(centers)
+        origins = pos[centers] if sites is None else np.asarray(sites, np.float64).reshape(-1, 3)
         rc2 = self.r_cut * self.r_cut
         periodic = cell is not None and any(self.pbc)
         if periodic:
             cell = np.asarray(cell, np.float64)
-            frac = pos @ np.linalg.inv(cell)
+            frac = np.concatenate([pos, origins]) @ np.linalg.inv(cell)
             spans = []
             heights = self._heights(cell)
             for a in range(3):
@@ -100,9 +103,9 @@ class SoapOracle:
         else:
             shifts = [(0, 0, 0)]
         out = []
-        for i in centers:
+        for origin in origins:
             found = []
-            base = pos - pos[i]                                   # r_j - r_i
+            base = pos - origin                                   # r_j - r_i
             for (na, nb, nc) in shifts:
                 if periodic:
                     T = (na * cell[0] + nb * cell[1]) + nc * cell[2]
@@ -116,10 +119,12 @@ class SoapOracle:
         return out
 
     def _displacements(self, pos, cell, i, nbrs):
+        """Displacements of the listed neighbours from atom i, or from the
+        point i when i is a length-3 array."""
         if not nbrs:
             return np.zeros((0, 3))
         j = np.array([t[0] for t in nbrs])
-        d = pos[j] - pos[i]
+        d = pos[j] - (pos[i] if np.ndim(i) == 0 else np.asarray(i, np.float64))
         if cell is not None and any(self.pbc):
             n = np.array([t[1:] for t in nbrs], dtype=np.float64)
             cell = np.asarray(cell, np.float64)

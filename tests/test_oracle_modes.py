@@ -222,3 +222,37 @@ def test_constant_weight_scales_the_neighbour_terms():
     on = np.zeros_like(c0)
     on[plain._species_index(st.numbers)[2], :, 0] = plain.onsite()
     np.testing.assert_allclose(weighted.coefficients(pos, st.numbers, None, 2), 1.5 * (c0 - on) + 0.5 * on, rtol=1e-12)
+
+
+# ----------------------------------------------------------------- centres that are not atoms
+def test_site_centres_equal_a_ghost_atom_of_a_species_of_its_own():
+    """A point centre sees what an atom of an otherwise absent species placed there sees, in every
+    feature that does not involve that species (its own Gaussian only enters its own block)."""
+    st = small_periodic_cell(seed=3, pbc=(True, True, True))
+    pos = st.positions.astype(np.float64)
+    sites = np.array([[0.7, 1.9, 2.2], [3.1, 0.2, 1.0]])
+    o = SoapOracle([1, 6, 7, 8], 4.0, 2, 3, 0.5, pbc=st.pbc)
+    got = modes.site_derivatives(o, pos, st.numbers, sites, st.cell)
+    og = SoapOracle([1, 6, 7, 8, 99], 4.0, 2, 3, 0.5, pbc=st.pbc)
+    keep = np.nonzero((og.table[:, 0] < 4) & (og.table[:, 1] < 4))[0]
+    assert np.array_equal(og.table[keep], o.table)
+    for a, site in enumerate(sites):
+        p2 = np.concatenate([pos, site[None]])
+        z2 = np.concatenate([st.numbers, [99]])
+        ref = og.derivatives(p2, z2, st.cell, [len(pos)])
+        np.testing.assert_allclose(got.descriptor[a], ref.descriptor[0][keep], rtol=1e-12, atol=1e-15)
+        rows = slice(got.row_ptr[a], got.row_ptr[a + 1])
+        real = ref.row_atom < len(pos)                                  # the ghost's own row has no counterpart
+        assert np.array_equal(got.row_atom[rows], ref.row_atom[real])
+        np.testing.assert_allclose(got.jacobian[rows], ref.jacobian[real][:, :, keep], rtol=1e-11, atol=1e-14)
+
+
+def test_site_jacobian_by_central_differences():
+    st = water_cluster(3, seed=4)
+    pos = st.positions.astype(np.float64)
+    sites = np.array([[0.3, -0.4, 0.9]])
+    o = SoapOracle([1, 8], 4.5, 3, 3, 0.5, POLYNOMIAL)
+    der = modes.site_derivatives(o, pos, st.numbers, sites)
+    dense = modes._dense(der, pos.shape[0])
+    fd = _fd(lambda p: modes.site_derivatives(o, p, st.numbers, sites).descriptor, pos)
+    np.testing.assert_allclose(dense, np.transpose(fd, (2, 0, 1, 3)), rtol=0, atol=3e-8 * np.abs(dense).max())
