@@ -148,6 +148,24 @@ int soap_jacobian_dense(soap_t *h, const float *d_jac_rows, const int64_t *d_row
  * Not to be called while work on this handle is in flight. */
 int soap_set_crossover(soap_t *h, int crossover);
 
+/* Centres at arbitrary points instead of at atoms (the interface accepts an
+ * explicit list of centres): d_sites [n_sites, 3] fp32 Cartesian, device.  A
+ * point has no Gaussian of its own, so there is no on-site term (Eq. 13, second
+ * term) and no Jacobian row for the centre: rows are the atoms in the sphere
+ * only.  A point that coincides with an atom drops that atom (the neighbour
+ * test is 0 < d^2): pass the atom as a centre to soap_derivatives instead.
+ * Everything else (arguments, sizing with soap_neighbors_at, errors, status)
+ * as in soap_neighbors / soap_descriptor / soap_derivatives. */
+int soap_neighbors_at(soap_t *h, const float *d_positions, const int32_t *d_numbers, int64_t n_atoms,
+                      const double *cell, const float *d_sites, int64_t n_sites,
+                      int64_t *n_pairs, int64_t *n_rows, void *stream);
+int soap_descriptor_at(soap_t *h, const float *d_positions, const int32_t *d_numbers, int64_t n_atoms,
+                       const double *cell, const float *d_sites, int64_t n_sites, float *d_out, void *stream);
+int soap_derivatives_at(soap_t *h, const float *d_positions, const int32_t *d_numbers, int64_t n_atoms,
+                        const double *cell, const float *d_sites, int64_t n_sites,
+                        float *d_out_desc, float *d_out_jac, int64_t capacity_rows,
+                        int64_t *d_row_ptr, int32_t *d_row_atom, void *stream);
+
 enum { SOAP_WEIGHT_NONE = 0, SOAP_WEIGHT_POLY = 1, SOAP_WEIGHT_POW = 2, SOAP_WEIGHT_EXP = 3 };
 
 /* Radial weighting of the neighbour density (the `weighting` argument of the

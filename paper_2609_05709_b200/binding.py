@@ -17,6 +17,7 @@ EXPORTED_SYMBOLS = [
     "soap_derivatives", "soap_status", "soap_profile", "soap_profile_read", "soap_neighbor_counts_static", "soap_jacobian_dense",
     "soap_set_crossover", "soap_num_coefficients", "soap_coefficients", "soap_coefficient_derivatives",
     "soap_descriptor_average", "soap_derivatives_average", "soap_set_weighting",
+    "soap_neighbors_at", "soap_descriptor_at", "soap_derivatives_at",
 ]
 
 _ERRORS = {-1: "SOAP_ERR_INVALID_ARG", -2: "SOAP_ERR_UNKNOWN_SPECIES", -3: "SOAP_ERR_CAPACITY",
@@ -63,6 +64,9 @@ def load_library() -> C.CDLL:
     lib.soap_status.argtypes = [vp, C.POINTER(i64), C.POINTER(i64), vp]
     lib.soap_neighbor_counts_static.argtypes = [vp, i64, C.c_double, vp, vp, C.c_char_p, i64]
     lib.soap_jacobian_dense.argtypes = [vp, vp, vp, vp, i64, vp, i64, vp, vp]
+    lib.soap_neighbors_at.argtypes = common + [C.POINTER(i64), C.POINTER(i64), vp]
+    lib.soap_descriptor_at.argtypes = common + [vp, vp]
+    lib.soap_derivatives_at.argtypes = common + [vp, vp, i64, vp, vp, vp]
     lib.soap_set_crossover.argtypes = [vp, i32]
     lib.soap_set_weighting.argtypes = [vp, i32] + [C.c_double] * 5
     lib.soap_num_coefficients.argtypes = [vp, C.POINTER(i64)]
@@ -240,6 +244,36 @@ class Soap:
         row_ptr = torch.empty(c + 1, dtype=torch.int64, device=dev)
         row_atom = torch.empty(max(nrows, 1), dtype=torch.int32, device=dev)
         self.derivatives_into(positions, numbers, cell, centers, desc, jac, row_ptr, row_atom)
+        self.status()
+        return Derivatives(desc, jac[:nrows], row_ptr, row_atom[:nrows])
+
+    # ------------------------------------------------------------------ centres that are not atoms
+    def derivatives_at(self, positions, numbers, sites, cell=None, jacobian=True):
+        """Descriptor (and Jacobian) for centres at the points `sites` (float32 device tensor (C, 3)):
+        no on-site term and no row for the centre itself.  Returns `Derivatives`, or the (C, F)
+        descriptor with jacobian=False."""
+        import torch
+        n, _, _ = self._inputs(positions, numbers, None)
+        assert sites.is_cuda and sites.dtype == torch.float32 and sites.is_contiguous() and sites.shape[-1] == 3
+        c, sptr = sites.shape[0], C.c_void_p(sites.data_ptr())
+        keep, cellp = self._cell(cell)
+        dev = positions.device
+        desc = torch.empty((c, self.n_features), dtype=torch.float32, device=dev)
+        if not jacobian:
+            self._check(self._lib.soap_descriptor_at(self._h, positions.data_ptr(), numbers.data_ptr(), n, cellp, sptr, c,
+                                                     desc.data_ptr(), self._stream()))
+            self.status()
+            return desc
+        npairs, nrows = C.c_int64(), C.c_int64()
+        self._check(self._lib.soap_neighbors_at(self._h, positions.data_ptr(), numbers.data_ptr(), n, cellp, sptr, c,
+                                                C.byref(npairs), C.byref(nrows), self._stream()))
+        nrows = int(nrows.value)
+        jac = torch.empty((max(nrows, 1), 3, self.n_features), dtype=torch.float32, device=dev)
+        row_ptr = torch.empty(c + 1, dtype=torch.int64, device=dev)
+        row_atom = torch.empty(max(nrows, 1), dtype=torch.int32, device=dev)
+        self._check(self._lib.soap_derivatives_at(self._h, positions.data_ptr(), numbers.data_ptr(), n, cellp, sptr, c,
+                                                  desc.data_ptr(), jac.data_ptr(), jac.shape[0], row_ptr.data_ptr(),
+                                                  row_atom.data_ptr(), self._stream()))
         self.status()
         return Derivatives(desc, jac[:nrows], row_ptr, row_atom[:nrows])
 

@@ -148,9 +148,10 @@ center_kernel(const CenterParams p) {
     float* sG1 = smem + lay.sG;                                            // [P][NCH]   G
     float2* sG2 = reinterpret_cast<float2*>(smem + lay.sG);                // [P][NCH]   (G, Ghat)
 
-    const int ci = p.centers ? p.centers[c_idx] : (int)c_idx;
-    const float xi = p.pos[3 * (long long)ci], yi = p.pos[3 * (long long)ci + 1], zi = p.pos[3 * (long long)ci + 2];
-    const int zi_species = p.species_idx[ci];
+    const int ci = p.sites ? -1 : (p.centers ? p.centers[c_idx] : (int)c_idx);
+    const float* pc = p.sites ? p.sites + 3 * c_idx : p.pos + 3 * (long long)ci;
+    const float xi = pc[0], yi = pc[1], zi = pc[2];
+    const int zi_species = p.sites ? 0 : p.species_idx[ci];
     const long long pair_base = p.pair_start[c_idx];
     // descriptor of given mean coefficients (inner average): no pairs to visit
     const int k_pairs = (!DERIV && p.c_bar) ? 0 : p.pair_count[c_idx];
@@ -345,7 +346,7 @@ center_kernel(const CenterParams p) {
     }
     __syncthreads();
     // on-site term: the centre's own Gaussian, l = 0 only (second term of Eq. 13)
-    if (tid < NMAX && !p.c_bar) c_t[(zi_species * NMAX + tid) * LMP] += p.w0 * __ldg(p.self_term + tid);
+    if (tid < NMAX && !p.c_bar && !p.sites) c_t[(zi_species * NMAX + tid) * LMP] += p.w0 * __ldg(p.self_term + tid);
     __syncthreads();
     const int W = S * NE;                                                  // coefficients per centre
     const int RW = CC ? W : F;                                             // width of an output row
@@ -373,19 +374,22 @@ center_kernel(const CenterParams p) {
     // pass through the (now idle) staging area in slabs, so that global memory is written in
     // feature order, whole sectors at a time.
     const long long row_base = DERIV ? p.row_ptr[c_idx] : 0;
+    const bool has_own = DERIV && !p.sites;          // a centre that is no atom has no row of its own
     if (CC) {
         // the centre's own row: minus the sum over the atoms that move relative to it
-        float* own = p.out_jac + (size_t)(row_base + p.self_row[c_idx]) * 3 * W;
-        for (int e = tid; e < 3 * W; e += kThreads) {
-            const int k = e / W, r = e - k * W, row = r / LM;
-            own[e] = -D_t[k * CT + row * LMP + (r - row * LM)];
+        if (has_own) {
+            float* own = p.out_jac + (size_t)(row_base + p.self_row[c_idx]) * 3 * W;
+            for (int e = tid; e < 3 * W; e += kThreads) {
+                const int k = e / W, r = e - k * W, row = r / LM;
+                own[e] = -D_t[k * CT + row * LMP + (r - row * LM)];
+            }
+            if (tid == 0) p.row_atom[row_base + p.self_row[c_idx]] = ci;
         }
-        if (tid == 0) p.row_atom[row_base + p.self_row[c_idx]] = ci;
     } else {
         // with given mean coefficients every centre would write the same descriptor: the first one does
         const bool write_desc = !p.c_bar || c_idx == 0;
         float* desc_row = p.out_desc + (p.c_bar ? (size_t)0 : (size_t)c_idx * F);
-        float* own = DERIV ? p.out_jac + (size_t)(row_base + p.self_row[c_idx]) * 3 * F : nullptr;
+        float* own = has_own ? p.out_jac + (size_t)(row_base + p.self_row[c_idx]) * 3 * F : nullptr;
         float* slab = smem + lay.sSD;
         constexpr int NV = DERIV ? 4 : 1;                                   // values per feature
         const int NP = F / L1;                                              // (species pair, n, n') groups
@@ -451,14 +455,14 @@ center_kernel(const CenterParams p) {
                     if (DERIV) { slab[nf + fl] = -kl * ax; slab[2 * nf + fl] = -kl * ay; slab[3 * nf + fl] = -kl * az; }
                 } else {
                     if (write_desc) desc_row[f0 + fl] = kl * acc;
-                    if (DERIV) { own[f0 + fl] = -kl * ax; own[(size_t)F + f0 + fl] = -kl * ay; own[(size_t)2 * F + f0 + fl] = -kl * az; }
+                    if (has_own) { own[f0 + fl] = -kl * ax; own[(size_t)F + f0 + fl] = -kl * ay; own[(size_t)2 * F + f0 + fl] = -kl * az; }
                 }
             }
             if (staged) {
                 __syncthreads();
                 for (int e = tid; e < nf; e += kThreads) {
                     if (write_desc) desc_row[f0 + e] = slab[e];
-                    if (DERIV) {
+                    if (has_own) {
                         own[f0 + e] = slab[nf + e];
                         own[(size_t)F + f0 + e] = slab[2 * nf + e];
                         own[(size_t)2 * F + f0 + e] = slab[3 * nf + e];
@@ -467,7 +471,7 @@ center_kernel(const CenterParams p) {
                 __syncthreads();
             }
         }
-        if (DERIV && tid == 0) p.row_atom[row_base + p.self_row[c_idx]] = ci;
+        if (has_own && tid == 0) p.row_atom[row_base + p.self_row[c_idx]] = ci;
     }
     if (!DERIV) return;
     __syncthreads();

@@ -486,7 +486,7 @@ constexpr int kFillWarps = 4;
 // When the segment does not fit the planned capacity only the counts are produced and the status
 // word says so; the caller plans again with the totals.
 __global__ void __launch_bounds__(kFillWarps * 32)
-pairs_kernel(const float* __restrict__ pos, const int* __restrict__ centers, long long C, Geometry geom,
+pairs_kernel(const float* __restrict__ pos, const int* __restrict__ centers, const float* __restrict__ sites, long long C, Geometry geom,
              const GridParams* __restrict__ gp, const int* __restrict__ atom_cell, const int* __restrict__ atom_wrap,
              const int* __restrict__ cell_start, const float4* __restrict__ s_pos, const int* __restrict__ s_wrap,
              long long pair_capacity, unsigned long long* pair_tmp, unsigned long long* pair_key, int* __restrict__ pair_row,
@@ -498,10 +498,19 @@ pairs_kernel(const float* __restrict__ pos, const int* __restrict__ centers, lon
     const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
     const long long c = blockIdx.x * (long long)kFillWarps + wid;
     if (c >= C) return;
-    const int i = centers ? centers[c] : (int)c;
-    const float xi = pos[3 * (long long)i], yi = pos[3 * (long long)i + 1], zi = pos[3 * (long long)i + 2];
+    // a centre is an atom, or (with `sites`) a point of its own: no atom index, no row of its own
+    const bool site = sites != nullptr;
+    const int i = site ? -1 : (centers ? centers[c] : (int)c);
+    const float* pc = site ? sites + 3 * c : pos + 3 * (long long)i;
+    const float xi = pc[0], yi = pc[1], zi = pc[2];
     int bi[3], wi[3];
-    {
+    if (site) {
+        bin_of(geom, g, xi, yi, zi, bi, wi);
+        if (abs(wi[0]) > 100 || abs(wi[1]) > 100 || abs(wi[2]) > 100) {
+            if (lane == 0) atomicOr(&counters->status, kStatusShiftRange);
+            wi[0] = wi[1] = wi[2] = 0;
+        }
+    } else {
         int cell = atom_cell[i];
         bi[0] = cell % g.nb[0]; bi[1] = (cell / g.nb[0]) % g.nb[1]; bi[2] = cell / (g.nb[0] * g.nb[1]);
         unpack3(atom_wrap[i], wi);
@@ -568,7 +577,7 @@ pairs_kernel(const float* __restrict__ pos, const int* __restrict__ centers, lon
         const unsigned m = __ballot_sync(0xffffffffu, isnew);
         const int u = uniq + __popc(m & ((1u << lane) - 1)) + (isnew ? 1 : 0) - 1;   // index among distinct atoms
         if (q < k) {
-            int row = u + ((!self_in && atom > i) ? 1 : 0);
+            int row = u + ((!site && !self_in && atom > i) ? 1 : 0);
             if (!isnew) row |= kRowContinuation;
             if (atom == i) row |= kRowSelfImage;
             pair_row[base + q] = row;
@@ -577,8 +586,8 @@ pairs_kernel(const float* __restrict__ pos, const int* __restrict__ centers, lon
         uniq += __popc(m);
     }
     if (lane == 0) {
-        row_count[c] = uniq + (self_in ? 0 : 1);
-        self_row[c] = below;
+        row_count[c] = uniq + ((site || self_in) ? 0 : 1);
+        self_row[c] = site ? -1 : below;
     }
 }
 

@@ -282,7 +282,7 @@ void scan_counts(soap_t* h, const int* counts, long long* out, int64_t C, long l
 // The whole neighbour search: cell list, sorted pair segments with their row bookkeeping, row
 // pointers (to `row_ptr_out`, the caller's array or the handle's) and the launch order.
 int launch_neighbors(soap_t* h, const float* pos, const int32_t* num, int64_t N, const Geometry& g,
-                     const int32_t* centers, int64_t C, long long* row_ptr_out, cudaStream_t st) {
+                     const int32_t* centers, const float* sites, int64_t C, long long* row_ptr_out, cudaStream_t st) {
     if (N <= kSmallPrepAtoms) {
         small_prep_kernel<<<1, kPrepThreads, 0, st>>>(pos, num, N, g, h->d_zlut, h->d_species_idx, (int)h->cap_cells, h->d_grid,
                                                       h->d_atom_cell, h->d_atom_wrap, h->d_cell_count, h->d_cell_start,
@@ -297,7 +297,7 @@ int launch_neighbors(soap_t* h, const float* pos, const int32_t* num, int64_t N,
         bin_fill_kernel<<<blocks_for(N, 256), 256, 0, st>>>(pos, N, h->d_atom_cell, h->d_atom_wrap, h->d_cell_start, h->d_cell_count, h->d_s_pos, h->d_s_wrap);
     }
     if (C > 0) pairs_kernel<<<(unsigned)((C + kFillWarps - 1) / kFillWarps), kFillWarps * 32, 0, st>>>(
-        pos, centers, C, g, h->d_grid, h->d_atom_cell, h->d_atom_wrap, h->d_cell_start, h->d_s_pos, h->d_s_wrap,
+        pos, centers, sites, C, g, h->d_grid, h->d_atom_cell, h->d_atom_wrap, h->d_cell_start, h->d_s_pos, h->d_s_wrap,
         h->cap_pairs, h->d_pair_tmp, h->d_pair_key, h->d_pair_row, h->d_pair_start, h->d_pair_count, h->d_row_count,
         h->d_self_row, h->d_counters);
     if (C <= kOrderMaxCenters) {
@@ -309,21 +309,22 @@ int launch_neighbors(soap_t* h, const float* pos, const int32_t* num, int64_t N,
     return SOAP_OK;
 }
 
-int check_inputs(soap_t* h, const float* pos, const int32_t* num, int64_t N, const int32_t* centers, int64_t C) {
+int check_inputs(soap_t* h, const float* pos, const int32_t* num, int64_t N, const int32_t* centers, int64_t C,
+                 const float* sites = nullptr) {
     if (!h) return SOAP_ERR_INVALID_ARG;
     if (N < 0 || C < 0 || N > 2000000000LL) return fail(h, SOAP_ERR_INVALID_ARG, "atom or centre count out of range");
     if (N > 0 && (!pos || !num)) return fail(h, SOAP_ERR_INVALID_ARG, "positions and numbers must not be NULL");
-    if (!centers && C != N) return fail(h, SOAP_ERR_INVALID_ARG, "without a centre list n_centers must equal n_atoms");
+    if (!centers && !sites && C != N) return fail(h, SOAP_ERR_INVALID_ARG, "without a centre list n_centers must equal n_atoms");
     return SOAP_OK;
 }
 
 // Plans scratch for a structure of this size: run the search (with whatever capacity there is;
 // the counts come out right even when the pairs do not fit), read the totals back, grow.
 int plan(soap_t* h, const float* pos, const int32_t* num, int64_t N, const Geometry& g,
-         const int32_t* centers, int64_t C, cudaStream_t st) {
+         const int32_t* centers, const float* sites, int64_t C, cudaStream_t st) {
     int rc = ensure_scratch(h, N, C, 0);
     if (rc) return rc;
-    rc = launch_neighbors(h, pos, num, N, g, centers, C, h->d_row_ptr, st);
+    rc = launch_neighbors(h, pos, num, N, g, centers, sites, C, h->d_row_ptr, st);
     if (rc) return rc;
     CU(cudaMemcpyAsync(h->h_counters, h->d_counters, sizeof(Counters), cudaMemcpyDeviceToHost, st));
     CU(cudaStreamSynchronize(st));
@@ -342,8 +343,8 @@ int plan(soap_t* h, const float* pos, const int32_t* num, int64_t N, const Geome
 }
 
 void fill_center_params(soap_t* h, CenterParams& cp, const float* pos, const int32_t* centers, int64_t C,
-                        const Geometry& g, bool deriv) {
-    cp.pos = pos; cp.centers = centers; cp.order = C <= kOrderMaxCenters ? h->d_order : nullptr; cp.species_idx = h->d_species_idx; cp.n_centers = C; cp.geom = g;
+                        const Geometry& g, bool deriv, const float* sites = nullptr) {
+    cp.pos = pos; cp.centers = centers; cp.sites = sites; cp.order = C <= kOrderMaxCenters ? h->d_order : nullptr; cp.species_idx = h->d_species_idx; cp.n_centers = C; cp.geom = g;
     cp.pair_start = h->d_pair_start; cp.pair_count = h->d_pair_count; cp.pair_key = h->d_pair_key; cp.pair_row = h->d_pair_row;
     cp.row_ptr = h->d_row_ptr; cp.self_row = h->d_self_row;
     cp.pair_capacity = h->cap_pairs; cp.row_capacity = 0; cp.counters = h->d_counters;
@@ -372,18 +373,18 @@ void build_feature_table(soap_t* h) {
 // Everything before the per-centre kernel: argument checks, device set-up, planning when the sizes
 // changed, the neighbour search.
 int prepare(soap_t* h, const float* pos, const int32_t* num, int64_t N, const double* cell, const int32_t* centers,
-            int64_t C, long long* row_ptr_out, Geometry& g, cudaStream_t st) {
-    int rc = check_inputs(h, pos, num, N, centers, C);
+            int64_t C, long long* row_ptr_out, Geometry& g, cudaStream_t st, const float* sites = nullptr) {
+    int rc = check_inputs(h, pos, num, N, centers, C, sites);
     if (rc) return rc;
     if ((rc = ensure_device(h))) return rc;
     if ((rc = make_geometry(h, cell, g))) return rc;
     if (h->profiling) CU(cudaEventRecord(h->ev[0], st));
     if (h->planned_atoms != N || h->planned_centers != C) {
-        if ((rc = plan(h, pos, num, N, g, centers, C, st))) return rc;
+        if ((rc = plan(h, pos, num, N, g, centers, sites, C, st))) return rc;
     }
-    if ((rc = launch_neighbors(h, pos, num, N, g, centers, C, row_ptr_out ? row_ptr_out : h->d_row_ptr, st))) return rc;
+    if ((rc = launch_neighbors(h, pos, num, N, g, centers, sites, C, row_ptr_out ? row_ptr_out : h->d_row_ptr, st))) return rc;
     if (h->weight.fn && C > 0) {
-        pair_weight_kernel<<<(unsigned)((C + 7) / 8), 256, 0, st>>>(pos, centers, C, g, h->d_pair_start, h->d_pair_count, h->d_pair_key,
+        pair_weight_kernel<<<(unsigned)((C + 7) / 8), 256, 0, st>>>(pos, centers, sites, C, g, h->d_pair_start, h->d_pair_count, h->d_pair_key,
                                                                    h->cap_pairs, h->d_counters, h->weight, h->d_pair_w);
         CU(cudaGetLastError());
     }
@@ -491,22 +492,35 @@ int soap_radial_table(const soap_t* h, double d, double* G, double* Ghat) {
     return SOAP_OK;
 }
 
-int soap_neighbors(soap_t* h, const float* d_positions, const int32_t* d_numbers, int64_t n_atoms, const double* cell,
-                   const int32_t* d_centers, int64_t n_centers, int64_t* n_pairs, int64_t* n_rows, void* stream) {
-    int rc = check_inputs(h, d_positions, d_numbers, n_atoms, d_centers, n_centers);
+static int neighbors_impl(soap_t* h, const float* d_positions, const int32_t* d_numbers, int64_t n_atoms, const double* cell,
+                          const int32_t* d_centers, const float* d_sites, int64_t n_centers, int64_t* n_pairs, int64_t* n_rows,
+                          void* stream) {
+    int rc = check_inputs(h, d_positions, d_numbers, n_atoms, d_centers, n_centers, d_sites);
     if (rc) return rc;
     if ((rc = ensure_device(h))) return rc;
     Geometry g;
     if ((rc = make_geometry(h, cell, g))) return rc;
     cudaStream_t st = (cudaStream_t)stream;
-    if ((rc = plan(h, d_positions, d_numbers, n_atoms, g, d_centers, n_centers, st))) return rc;
-    if ((rc = launch_neighbors(h, d_positions, d_numbers, n_atoms, g, d_centers, n_centers, h->d_row_ptr, st))) return rc;
+    if ((rc = plan(h, d_positions, d_numbers, n_atoms, g, d_centers, d_sites, n_centers, st))) return rc;
+    if ((rc = launch_neighbors(h, d_positions, d_numbers, n_atoms, g, d_centers, d_sites, n_centers, h->d_row_ptr, st))) return rc;
     CU(cudaMemcpyAsync(h->h_counters, h->d_counters, sizeof(Counters), cudaMemcpyDeviceToHost, st));
     CU(cudaStreamSynchronize(st));
     h->last_centers = n_centers;
     if (n_pairs) *n_pairs = h->h_counters->n_pairs;
     if (n_rows) *n_rows = h->h_counters->n_rows;
     return SOAP_OK;
+}
+
+int soap_neighbors(soap_t* h, const float* d_positions, const int32_t* d_numbers, int64_t n_atoms, const double* cell,
+                   const int32_t* d_centers, int64_t n_centers, int64_t* n_pairs, int64_t* n_rows, void* stream) {
+    return neighbors_impl(h, d_positions, d_numbers, n_atoms, cell, d_centers, nullptr, n_centers, n_pairs, n_rows, stream);
+}
+
+int soap_neighbors_at(soap_t* h, const float* d_positions, const int32_t* d_numbers, int64_t n_atoms, const double* cell,
+                      const float* d_sites, int64_t n_sites, int64_t* n_pairs, int64_t* n_rows, void* stream) {
+    if (h && n_sites > 0 && !d_sites) return fail(h, SOAP_ERR_INVALID_ARG, "d_sites must not be NULL");
+    static const float none[3] = {0.f, 0.f, 0.f};
+    return neighbors_impl(h, d_positions, d_numbers, n_atoms, cell, nullptr, d_sites ? d_sites : none, n_sites, n_pairs, n_rows, stream);
 }
 
 int soap_neighbor_list(soap_t* h, int64_t* d_pair_ptr, int32_t* d_pair_atom, int32_t* d_pair_shift,
@@ -522,18 +536,50 @@ int soap_neighbor_list(soap_t* h, int64_t* d_pair_ptr, int32_t* d_pair_atom, int
     return SOAP_OK;
 }
 
-int soap_descriptor(soap_t* h, const float* d_positions, const int32_t* d_numbers, int64_t n_atoms, const double* cell,
-                    const int32_t* d_centers, int64_t n_centers, float* d_out, void* stream) {
+static int descriptor_impl(soap_t* h, const float* d_positions, const int32_t* d_numbers, int64_t n_atoms, const double* cell,
+                           const int32_t* d_centers, const float* d_sites, int64_t n_centers, float* d_out, void* stream) {
     if (h && n_centers > 0 && !d_out) return fail(h, SOAP_ERR_INVALID_ARG, "d_out must not be NULL");
     Geometry g;
     cudaStream_t st = (cudaStream_t)stream;
-    int rc = prepare(h, d_positions, d_numbers, n_atoms, cell, d_centers, n_centers, nullptr, g, st);
+    int rc = prepare(h, d_positions, d_numbers, n_atoms, cell, d_centers, n_centers, nullptr, g, st, d_sites);
     if (rc) return rc;
     if (n_centers > 0) {
         CenterParams cp;
-        fill_center_params(h, cp, d_positions, d_centers, n_centers, g, false);
+        fill_center_params(h, cp, d_positions, d_centers, n_centers, g, false, d_sites);
         cp.out_desc = d_out;
         CU(center_launch(kCenterDesc, h->l_max, h->n_max, cp, (unsigned)n_centers, h->smem_desc, st));
+    }
+    if (h->profiling) CU(cudaEventRecord(h->ev[2], st));
+    return SOAP_OK;
+}
+
+int soap_descriptor(soap_t* h, const float* d_positions, const int32_t* d_numbers, int64_t n_atoms, const double* cell,
+                    const int32_t* d_centers, int64_t n_centers, float* d_out, void* stream) {
+    return descriptor_impl(h, d_positions, d_numbers, n_atoms, cell, d_centers, nullptr, n_centers, d_out, stream);
+}
+
+int soap_descriptor_at(soap_t* h, const float* d_positions, const int32_t* d_numbers, int64_t n_atoms, const double* cell,
+                       const float* d_sites, int64_t n_sites, float* d_out, void* stream) {
+    if (h && !d_sites) return n_sites == 0 ? SOAP_OK : fail(h, SOAP_ERR_INVALID_ARG, "d_sites must not be NULL");
+    return descriptor_impl(h, d_positions, d_numbers, n_atoms, cell, nullptr, d_sites, n_sites, d_out, stream);
+}
+
+static int derivatives_impl(soap_t* h, const float* d_positions, const int32_t* d_numbers, int64_t n_atoms, const double* cell,
+                            const int32_t* d_centers, const float* d_sites, int64_t n_centers, float* d_out_desc, float* d_out_jac,
+                            int64_t capacity_rows, int64_t* d_row_ptr, int32_t* d_row_atom, void* stream) {
+    if (h && (!d_row_ptr || capacity_rows < 0)) return fail(h, SOAP_ERR_INVALID_ARG, "d_row_ptr must not be NULL");
+    if (h && n_centers > 0 && (!d_out_desc || !d_out_jac || !d_row_atom)) return fail(h, SOAP_ERR_INVALID_ARG, "output pointers must not be NULL");
+    Geometry g;
+    cudaStream_t st = (cudaStream_t)stream;
+    int rc = prepare(h, d_positions, d_numbers, n_atoms, cell, d_centers, n_centers, (long long*)d_row_ptr, g, st, d_sites);
+    if (rc) return rc;
+    if (n_centers > 0) {
+        CenterParams cp;
+        fill_center_params(h, cp, d_positions, d_centers, n_centers, g, true, d_sites);
+        cp.row_ptr = (const long long*)d_row_ptr;
+        cp.row_capacity = capacity_rows;
+        cp.out_desc = d_out_desc; cp.out_jac = d_out_jac; cp.row_atom = d_row_atom;
+        CU(center_launch(kCenterDeriv, h->l_max, h->n_max, cp, (unsigned)n_centers, h->smem_deriv, st));
     }
     if (h->profiling) CU(cudaEventRecord(h->ev[2], st));
     return SOAP_OK;
@@ -542,22 +588,17 @@ int soap_descriptor(soap_t* h, const float* d_positions, const int32_t* d_number
 int soap_derivatives(soap_t* h, const float* d_positions, const int32_t* d_numbers, int64_t n_atoms, const double* cell,
                      const int32_t* d_centers, int64_t n_centers, float* d_out_desc, float* d_out_jac,
                      int64_t capacity_rows, int64_t* d_row_ptr, int32_t* d_row_atom, void* stream) {
-    if (h && (!d_row_ptr || capacity_rows < 0)) return fail(h, SOAP_ERR_INVALID_ARG, "d_row_ptr must not be NULL");
-    if (h && n_centers > 0 && (!d_out_desc || !d_out_jac || !d_row_atom)) return fail(h, SOAP_ERR_INVALID_ARG, "output pointers must not be NULL");
-    Geometry g;
-    cudaStream_t st = (cudaStream_t)stream;
-    int rc = prepare(h, d_positions, d_numbers, n_atoms, cell, d_centers, n_centers, (long long*)d_row_ptr, g, st);
-    if (rc) return rc;
-    if (n_centers > 0) {
-        CenterParams cp;
-        fill_center_params(h, cp, d_positions, d_centers, n_centers, g, true);
-        cp.row_ptr = (const long long*)d_row_ptr;
-        cp.row_capacity = capacity_rows;
-        cp.out_desc = d_out_desc; cp.out_jac = d_out_jac; cp.row_atom = d_row_atom;
-        CU(center_launch(kCenterDeriv, h->l_max, h->n_max, cp, (unsigned)n_centers, h->smem_deriv, st));
-    }
-    if (h->profiling) CU(cudaEventRecord(h->ev[2], st));
-    return SOAP_OK;
+    return derivatives_impl(h, d_positions, d_numbers, n_atoms, cell, d_centers, nullptr, n_centers, d_out_desc, d_out_jac,
+                            capacity_rows, d_row_ptr, d_row_atom, stream);
+}
+
+int soap_derivatives_at(soap_t* h, const float* d_positions, const int32_t* d_numbers, int64_t n_atoms, const double* cell,
+                        const float* d_sites, int64_t n_sites, float* d_out_desc, float* d_out_jac,
+                        int64_t capacity_rows, int64_t* d_row_ptr, int32_t* d_row_atom, void* stream) {
+    if (h && !d_sites && n_sites > 0) return fail(h, SOAP_ERR_INVALID_ARG, "d_sites must not be NULL");
+    static const float none[3] = {0.f, 0.f, 0.f};
+    return derivatives_impl(h, d_positions, d_numbers, n_atoms, cell, nullptr, d_sites ? d_sites : none, n_sites, d_out_desc,
+                            d_out_jac, capacity_rows, d_row_ptr, d_row_atom, stream);
 }
 
 int soap_jacobian_dense(soap_t* h, const float* d_jac_rows, const int64_t* d_row_ptr, const int32_t* d_row_atom,

@@ -50,6 +50,7 @@ struct CenterParams {
     // structure
     const float* pos;             // [N,3]
     const int* centers;           // [C] or null
+    const float* sites;           // [C,3] or null: centres at these points instead of at atoms (no on-site term, no own row)
     const int* order;             // [C] CTA -> centre slot (largest first) or null
     const int* species_idx;       // [N]
     long long n_centers;

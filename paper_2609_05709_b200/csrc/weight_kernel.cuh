@@ -39,7 +39,8 @@ __device__ inline void weight_eval(const WeightParams& wp, double dist, double& 
 // One warp per centre walks the centre's pair segment.  The displacement is formed exactly as in
 // the per-centre kernel.
 __global__ void __launch_bounds__(256)
-pair_weight_kernel(const float* __restrict__ pos, const int* __restrict__ centers, long long n_centers, Geometry geom,
+pair_weight_kernel(const float* __restrict__ pos, const int* __restrict__ centers, const float* __restrict__ sites,
+                   long long n_centers, Geometry geom,
                    const long long* __restrict__ pair_start, const int* __restrict__ pair_count,
                    const unsigned long long* __restrict__ pair_key, long long pair_capacity, const Counters* counters,
                    WeightParams wp, float2* __restrict__ pair_w) {
@@ -48,7 +49,8 @@ pair_weight_kernel(const float* __restrict__ pos, const int* __restrict__ center
     if (c_idx >= n_centers) return;
     const int lane = threadIdx.x & 31;
     const int ci = centers ? centers[c_idx] : (int)c_idx;
-    const float xi = pos[3 * (long long)ci], yi = pos[3 * (long long)ci + 1], zi = pos[3 * (long long)ci + 2];
+    const float* pc = sites ? sites + 3 * c_idx : pos + 3 * (long long)ci;
+    const float xi = pc[0], yi = pc[1], zi = pc[2];
     const long long base = pair_start[c_idx];
     const int k = pair_count[c_idx];
     const bool periodic = geom.pbc[0] | geom.pbc[1] | geom.pbc[2];

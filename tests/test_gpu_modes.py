@@ -214,3 +214,34 @@ def test_weighting_can_be_switched_on_a_live_handle(pkg):
     assert torch.equal(again.jacobian, plain.jacobian) and torch.equal(again.descriptor, plain.descriptor)
     with pytest.raises(pkg.SoapError, match="r0 > 0"):
         soap._check(soap._lib.soap_set_weighting(soap._h, 2, -1.0, 1.0, 1.0, 1.0, 1.0))
+
+
+# ----------------------------------------------------------------- centres that are not atoms
+@pytest.mark.parametrize("case", ["water_gto", "periodic_poly_weighted"])
+def test_centres_at_arbitrary_points(pkg, case):
+    rng = np.random.default_rng(12)
+    if case == "water_gto":
+        s, args, kw = water_cluster(20, 4), ([1, 8], 5.0, 6, 4, 0.5, GTO, (False, False, False)), {}
+        lo, hi = s.positions.min(axis=0), s.positions.max(axis=0)
+        sites = lo + rng.random((9, 3)) * (hi - lo)
+        sites[0] = hi + 2.0                # outside the bounding box of the atoms, still within reach
+        sites[1] = lo - 30.0               # sees nothing
+    else:
+        s, args = small_periodic_cell(9, (True, True, True)), ([1, 6, 7, 8], 4.5, 3, 3, 0.5, POLYNOMIAL, (True, True, True))
+        kw = {"weighting": {"function": "poly", "r0": 4.0, "c": 1.0, "m": 2, "w0": 1.0}}
+        sites = rng.random((6, 3)) * 12.0 - 4.0                       # several cells away as well
+    sites = sites.astype(np.float32)
+    soap, oracle = pkg.Soap(*args, **kw), SoapOracle(*args, **kw)
+    pos, num = dev(s)
+    ref = modes.site_derivatives(oracle, s.positions, s.numbers, sites, s.cell)
+    out = soap.derivatives_at(pos, num, torch.from_numpy(sites).cuda(), s.cell)
+    assert np.array_equal(out.row_ptr.cpu().numpy(), ref.row_ptr)
+    assert np.array_equal(out.row_atom.cpu().numpy(), ref.row_atom)
+    assert col_err(out.descriptor.cpu().numpy(), ref.descriptor, 0) < DESC_TOL
+    assert col_err(out.jacobian.cpu().numpy(), ref.jacobian, (0, 1)) < JAC_TOL
+    d = soap.derivatives_at(pos, num, torch.from_numpy(sites).cuda(), s.cell, jacobian=False)
+    assert torch.equal(d, out.descriptor)
+    if case == "water_gto":
+        assert np.all(out.descriptor[1].cpu().numpy() == 0) and ref.row_ptr[2] == ref.row_ptr[1]
+    # the same handle still serves atom centres afterwards
+    check_derivatives(soap, oracle, s, sample=[0, 3])
