@@ -326,6 +326,14 @@ def time_case(struct, species, r_cut, n_max, l_max, sigma, rbf, mode, steps, war
         row_atom = torch.empty(n_rows, dtype=torch.int32, device="cuda")
         step = lambda: soap.derivatives_into(pos, num, struct.cell, None, desc, jac, row_ptr, row_atom)
         alg_bytes = n_rows * 3 * F * 4 + C * F * 4 + n_rows * 4 + n_pairs * 24 + (C + 1) * 16
+    elif mode == "derivatives_compact":
+        pitch = soap.compact_pitch
+        own = torch.empty((C, 3, F), device="cuda")
+        jac = torch.empty((n_rows, 3, pitch), device="cuda")
+        row_ptr = torch.empty(C + 1, dtype=torch.int64, device="cuda")
+        row_atom = torch.empty(n_rows, dtype=torch.int32, device="cuda")
+        step = lambda: soap.derivatives_compact_into(pos, num, struct.cell, None, desc, own, jac, row_ptr, row_atom)
+        alg_bytes = n_rows * 3 * pitch * 4 + C * 3 * F * 4 + C * F * 4 + n_rows * 4 + n_pairs * 24 + (C + 1) * 16
     elif mode == "descriptor":
         step = lambda: soap.descriptor(pos, num, struct.cell, None, out=desc)
         alg_bytes = C * F * 4 + n_pairs * 24 + (C + 1) * 8
@@ -419,6 +427,14 @@ def run_suite(args):
             print(json.dumps({"case": "driver", "workers": world, "atoms": s.n_atoms, "batch": batch,
                               "mode": "derivatives" if derivatives else "descriptor", "seconds": best,
                               "atoms_per_s": s.n_atoms / best}), flush=True)
+    elif args.suite == "compact":
+        for name in ("water1000_gto_n8_l6_rc6", "chno2000_poly_n8_l8_rc5"):
+            kind, n, species, r_cut, n_max, l_max, sigma, rbf = WORKLOADS[name]
+            s = make_structure(name)
+            for mode in ("derivatives", "derivatives_compact"):
+                r = time_case(s, species, r_cut, n_max, l_max, sigma, rbf, mode, steps)
+                r["case"] = name
+                print(json.dumps(r), flush=True)
     elif args.suite == "modes":
         s = water_cluster(1000, 0)
         base = ([1, 8], 6.0, 8, 6, 0.5, 0)
@@ -447,11 +463,12 @@ def main():
     ap.add_argument("--workload", default=DEFAULT_WORKLOAD, choices=sorted(WORKLOADS))
     ap.add_argument("--kernel-only", action="store_true",
                     help="skip the end-to-end and CPU-baseline legs (for profiler captures)")
-    ap.add_argument("--suite", choices=["map", "scaling", "configs", "desc30k", "modes", "driver"],
+    ap.add_argument("--suite", choices=["map", "scaling", "configs", "desc30k", "modes", "driver", "compact"],
                     help="extra measurements beside the headline line: 'map' = descriptor+Jacobian over "
                          "n_max x l_max on the 1000-molecule cluster, 'scaling' = descriptor-only on "
                          "3k..1M atoms, 'configs' = the periodic multi-species box and the tiny cluster, "
                          "'desc30k' = descriptor-only on 30,000 atoms alone (small enough for profiler captures), "
+                         "'compact' = species-compact against full Jacobian rows on the water cluster and the four-species box, "
                          "'driver' = the multi-process driver with --gpus workers, results on the host, "
                          "'modes' = crossover off, coefficient mode and the averaged modes on the 1000-molecule cluster; "
                          "prints one JSON line per case")

@@ -148,6 +148,40 @@ int soap_jacobian_dense(soap_t *h, const float *d_jac_rows, const int64_t *d_row
  * Not to be called while work on this handle is in flight. */
 int soap_set_crossover(soap_t *h, int crossover);
 
+/* ---- species-compact Jacobian rows ----
+ * The row of a neighbour of species Z is zero in every species-pair block that
+ * does not involve Z (Eq. 5: grad_j c^mu vanishes unless atom j has species mu;
+ * the paper's kernels write those zeros explicitly).  The compact format leaves
+ * them out: a neighbour row holds, in feature order, only the blocks (mu, nu)
+ * with mu == Z or nu == Z: n_compact = one same-species block + (S-1) cross
+ * blocks, the same for every Z, against F = S same-species + S(S-1)/2 cross
+ * blocks.  Rows are stored with a pitch of n_compact rounded up to a multiple
+ * of 8 floats (padding written as zeros).  The centre's own row involves every
+ * block and goes, full width, to an array of its own. */
+int soap_num_compact_features(const soap_t *h, int64_t *n_compact, int64_t *pitch);
+
+/* map[j] = index of the full feature that column j of a compact row of species
+ * `species_index` (position in the sorted species list) holds; host memory,
+ * n_compact entries, ascending. */
+int soap_compact_feature_map(const soap_t *h, int species_index, int32_t *map);
+
+/* soap_derivatives with compact rows:
+ *   d_out_center [n_centers, 3, F]         the centre's own row (all blocks)
+ *   d_out_jac    [capacity_rows, 3, pitch] neighbour rows, compact; the slot of
+ *                the centre's own row (row_atom == the centre) is zero-filled
+ * row_ptr / row_atom / d_out_desc / errors as in soap_derivatives. */
+int soap_derivatives_compact(soap_t *h, const float *d_positions, const int32_t *d_numbers, int64_t n_atoms,
+                             const double *cell, const int32_t *d_centers, int64_t n_centers,
+                             float *d_out_desc, float *d_out_center, float *d_out_jac, int64_t capacity_rows,
+                             int64_t *d_row_ptr, int32_t *d_row_atom, void *stream);
+
+/* Expands compact rows to the full rows soap_derivatives writes:
+ * d_out_rows [n_rows, 3, F].  d_centers as in the producing call (NULL = all
+ * atoms); d_numbers the structure's atomic numbers. */
+int soap_compact_expand(soap_t *h, const int32_t *d_numbers, const int32_t *d_centers, int64_t n_centers,
+                        const float *d_center_rows, const float *d_jac_compact, const int64_t *d_row_ptr,
+                        const int32_t *d_row_atom, float *d_out_rows, void *stream);
+
 /* Centres at arbitrary points instead of at atoms (the interface accepts an
  * explicit list of centres): d_sites [n_sites, 3] fp32 Cartesian, device.  A
  * point has no Gaussian of its own, so there is no on-site term (Eq. 13, second

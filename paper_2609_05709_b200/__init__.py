@@ -5,8 +5,8 @@ in include/soap.h; this package only marshals arguments.  torch is used for
 device memory and streams.  There is no CPU fallback: if the shared library is
 missing, importing `Soap` raises.
 """
-from .binding import (GTO, POLYNOMIAL, Soap, SoapError, Derivatives, library_path, load_library,
+from .binding import (GTO, POLYNOMIAL, Soap, SoapError, Derivatives, CompactDerivatives, library_path, load_library,
                       neighbor_counts_static, EXPORTED_SYMBOLS)
 
-__all__ = ["GTO", "POLYNOMIAL", "Soap", "SoapError", "Derivatives", "library_path", "load_library",
+__all__ = ["GTO", "POLYNOMIAL", "Soap", "SoapError", "Derivatives", "CompactDerivatives", "library_path", "load_library",
            "neighbor_counts_static", "EXPORTED_SYMBOLS"]

@@ -18,6 +18,7 @@ EXPORTED_SYMBOLS = [
     "soap_set_crossover", "soap_num_coefficients", "soap_coefficients", "soap_coefficient_derivatives",
     "soap_descriptor_average", "soap_derivatives_average", "soap_set_weighting",
     "soap_neighbors_at", "soap_descriptor_at", "soap_derivatives_at",
+    "soap_num_compact_features", "soap_compact_feature_map", "soap_derivatives_compact", "soap_compact_expand",
 ]
 
 _ERRORS = {-1: "SOAP_ERR_INVALID_ARG", -2: "SOAP_ERR_UNKNOWN_SPECIES", -3: "SOAP_ERR_CAPACITY",
@@ -67,6 +68,10 @@ def load_library() -> C.CDLL:
     lib.soap_neighbors_at.argtypes = common + [C.POINTER(i64), C.POINTER(i64), vp]
     lib.soap_descriptor_at.argtypes = common + [vp, vp]
     lib.soap_derivatives_at.argtypes = common + [vp, vp, i64, vp, vp, vp]
+    lib.soap_num_compact_features.argtypes = [vp, C.POINTER(i64), C.POINTER(i64)]
+    lib.soap_compact_feature_map.argtypes = [vp, i32, C.POINTER(C.c_int32)]
+    lib.soap_derivatives_compact.argtypes = common + [vp, vp, vp, i64, vp, vp, vp]
+    lib.soap_compact_expand.argtypes = [vp, vp, vp, i64, vp, vp, vp, vp, vp, vp]
     lib.soap_set_crossover.argtypes = [vp, i32]
     lib.soap_set_weighting.argtypes = [vp, i32] + [C.c_double] * 5
     lib.soap_num_coefficients.argtypes = [vp, C.POINTER(i64)]
@@ -100,6 +105,15 @@ def neighbor_counts_static(positions, r_cut, out=None):
     if rc != 0:
         raise SoapError(rc, msg.value.decode())
     return out
+
+
+@dataclass
+class CompactDerivatives:
+    descriptor: "torch.Tensor"   # (C, F)
+    center_rows: "torch.Tensor"  # (C, 3, F) the centre's own row
+    jacobian: "torch.Tensor"     # (rows, 3, pitch) species-compact neighbour rows
+    row_ptr: "torch.Tensor"      # (C+1,)
+    row_atom: "torch.Tensor"     # (rows,)
 
 
 @dataclass
@@ -138,6 +152,9 @@ class Soap:
         self.n_features = int(n.value)
         self._check(self._lib.soap_num_coefficients(self._h, C.byref(n)))
         self.n_coefficients = int(n.value)
+        pitch = C.c_int64()
+        self._check(self._lib.soap_num_compact_features(self._h, C.byref(n), C.byref(pitch)))
+        self.n_compact, self.compact_pitch = int(n.value), int(pitch.value)
         self.n_channels = int(n_max) * (int(l_max) + 1)
         self.pbc = tuple(bool(p) for p in pbc)
 
@@ -246,6 +263,46 @@ class Soap:
         self.derivatives_into(positions, numbers, cell, centers, desc, jac, row_ptr, row_atom)
         self.status()
         return Derivatives(desc, jac[:nrows], row_ptr, row_atom[:nrows])
+
+    # ------------------------------------------------------------------ species-compact rows
+    def compact_feature_map(self, species_index):
+        out = np.empty(self.n_compact, np.int32)
+        self._check(self._lib.soap_compact_feature_map(self._h, int(species_index), out.ctypes.data_as(C.POINTER(C.c_int32))))
+        return out
+
+    def derivatives_compact_into(self, positions, numbers, cell, centers, desc, center_rows, jac, row_ptr, row_atom):
+        n, c, cptr = self._inputs(positions, numbers, centers)
+        keep, cellp = self._cell(cell)
+        self._check(self._lib.soap_derivatives_compact(self._h, positions.data_ptr(), numbers.data_ptr(), n, cellp, cptr, c,
+                                                       desc.data_ptr(), center_rows.data_ptr(), jac.data_ptr(), jac.shape[0],
+                                                       row_ptr.data_ptr(), row_atom.data_ptr(), self._stream()))
+
+    def derivatives_compact(self, positions, numbers, cell=None, centers=None) -> CompactDerivatives:
+        """Like `derivatives`, with neighbour rows that leave out the structurally zero species blocks."""
+        import torch
+        _, nrows = self.neighbors(positions, numbers, cell, centers)
+        c = positions.shape[0] if centers is None else centers.shape[0]
+        dev = positions.device
+        desc = torch.empty((c, self.n_features), dtype=torch.float32, device=dev)
+        center_rows = torch.empty((c, 3, self.n_features), dtype=torch.float32, device=dev)
+        jac = torch.empty((max(nrows, 1), 3, self.compact_pitch), dtype=torch.float32, device=dev)
+        row_ptr = torch.empty(c + 1, dtype=torch.int64, device=dev)
+        row_atom = torch.empty(max(nrows, 1), dtype=torch.int32, device=dev)
+        self.derivatives_compact_into(positions, numbers, cell, centers, desc, center_rows, jac, row_ptr, row_atom)
+        self.status()
+        return CompactDerivatives(desc, center_rows, jac[:nrows], row_ptr, row_atom[:nrows])
+
+    def compact_expand(self, numbers, centers, comp: "CompactDerivatives"):
+        """(rows, 3, F): the full rows `derivatives` would have written."""
+        import torch
+        rows = comp.jacobian.shape[0]
+        out = torch.empty((max(rows, 1), 3, self.n_features), dtype=torch.float32, device=comp.jacobian.device)
+        c = comp.row_ptr.shape[0] - 1
+        cptr = None if centers is None else C.c_void_p(centers.data_ptr())
+        self._check(self._lib.soap_compact_expand(self._h, numbers.data_ptr(), cptr, c, comp.center_rows.data_ptr(),
+                                                  comp.jacobian.data_ptr(), comp.row_ptr.data_ptr(), comp.row_atom.data_ptr(),
+                                                  out.data_ptr(), self._stream()))
+        return out[:rows]
 
     # ------------------------------------------------------------------ centres that are not atoms
     def derivatives_at(self, positions, numbers, sites, cell=None, jacobian=True):

@@ -106,11 +106,18 @@ __device__ __forceinline__ void harmonics_column(int L, int m, float x, float y,
     }
 }
 
-// KIND: 0 descriptor only, 1 descriptor and Jacobian, 2 coefficients c^mu_nlm and their Jacobian
-template <int KIND, int L, int NMAX_T>
+// KIND: 0 descriptor only, 1 descriptor and Jacobian, 2 coefficients c^mu_nlm and their Jacobian.
+// PLAIN: the default configuration (every species pair, atom centres, no weighting, full rows, own
+// coefficients); the options are then compile-time constants and their code drops out.
+template <int KIND, int L, int NMAX_T, bool PLAIN>
 __global__ void __launch_bounds__(kThreads, KIND ? SOAP_MIN_CTAS_DERIV : SOAP_MIN_CTAS_DESC)
 center_kernel(const CenterParams p) {
     constexpr bool DERIV = KIND != 0, CC = KIND == 2;
+    const bool o_compact = !PLAIN && p.compact, o_cross = PLAIN || p.crossover, o_emit = !PLAIN && p.emit_coeff;
+    const float* const o_cbar = PLAIN ? nullptr : p.c_bar;
+    const float* const o_sites = PLAIN ? nullptr : p.sites;
+    const float2* const o_pw = PLAIN ? nullptr : p.pair_w;
+    const float o_w0 = PLAIN ? 1.f : p.w0;
     constexpr int L1 = L + 1, LM = L1 * L1, LMP = LM | 1;      // odd row stride: no shared-memory bank conflicts
     constexpr int NMAX_BOUND = NMAX_T ? NMAX_T : 16;
     // pass-1 ownership: W_LM warps cover the lm index, SLOTS such groups split the n index
@@ -136,7 +143,7 @@ center_kernel(const CenterParams p) {
     }
     const int S = p.S, NMAX = NMAX_T ? NMAX_T : p.n_max, NCH = NMAX * L1, NE = NMAX * LM;
     const int CT = S * NMAX * LMP, P = p.P, F = p.F;
-    const SmemLayout lay = make_layout(S, NMAX, L, P, DERIV, p.pair_w != nullptr);
+    const SmemLayout lay = make_layout(S, NMAX, L, P, DERIV, o_pw != nullptr);
     float* c_t = smem + lay.c;                                             // [S][NMAX][LMP]
     float4* geo_d = reinterpret_cast<float4*>(smem + lay.geo);             // [GP] dx, dy, dz, r
     int4* geo_i = reinterpret_cast<int4*>(smem + lay.geo + 4 * kGeoPairs);   // [GP] interval, t bits, species|moving<<8, row word
@@ -148,13 +155,13 @@ center_kernel(const CenterParams p) {
     float* sG1 = smem + lay.sG;                                            // [P][NCH]   G
     float2* sG2 = reinterpret_cast<float2*>(smem + lay.sG);                // [P][NCH]   (G, Ghat)
 
-    const int ci = p.sites ? -1 : (p.centers ? p.centers[c_idx] : (int)c_idx);
-    const float* pc = p.sites ? p.sites + 3 * c_idx : p.pos + 3 * (long long)ci;
+    const int ci = o_sites ? -1 : (p.centers ? p.centers[c_idx] : (int)c_idx);
+    const float* pc = o_sites ? o_sites + 3 * c_idx : p.pos + 3 * (long long)ci;
     const float xi = pc[0], yi = pc[1], zi = pc[2];
-    const int zi_species = p.sites ? 0 : p.species_idx[ci];
+    const int zi_species = o_sites ? 0 : p.species_idx[ci];
     const long long pair_base = p.pair_start[c_idx];
     // descriptor of given mean coefficients (inner average): no pairs to visit
-    const int k_pairs = (!DERIV && p.c_bar) ? 0 : p.pair_count[c_idx];
+    const int k_pairs = (!DERIV && o_cbar) ? 0 : p.pair_count[c_idx];
     const bool periodic = p.geom.pbc[0] | p.geom.pbc[1] | p.geom.pbc[2];
 
     for (int e = tid; e < CT * (DERIV ? 4 : 1); e += kThreads) {
@@ -205,7 +212,7 @@ center_kernel(const CenterParams p) {
                 const double r = sqrt(dx * dx + dy * dy + dz * dz);
                 dd = make_float4((float)dx, (float)dy, (float)dz, (float)r);
                 rw = p.pair_row[pair_base + g0 + tid];
-                if (p.pair_w) wgt = p.pair_w[pair_base + g0 + tid];
+                if (o_pw) wgt = o_pw[pair_base + g0 + tid];
                 special = rw & (kRowSelfImage | kRowContinuation);
                 // interval and offset in the radial table, in fp64 so that the offset keeps its digits
                 const double u = r * (double)p.inv_h;
@@ -229,7 +236,7 @@ center_kernel(const CenterParams p) {
             geo_d[at] = dd;
             geo_i[at] = make_int4(qi, __float_as_int(tt), sp | ((rw & kRowSelfImage) ? 0 : 256), rw);
             geo_j[at] = j;
-            if (p.pair_w) geo_w[at] = wgt;
+            if (o_pw) geo_w[at] = wgt;
         }
         if (tid <= S) {
             int at = 0;
@@ -249,7 +256,7 @@ center_kernel(const CenterParams p) {
             const int4 gi = geo_i[g + pr];
             const float t = __int_as_float(gi.y);
             const float rinv_h = GRAD ? p.inv_h / geo_d[g + pr].w : 0.f;
-            if (p.pair_w) {
+            if (o_pw) {
                 // radial weighting: G -> w G, Ghat -> w Ghat + (w'/d) G
                 const float2 w = geo_w[g + pr];
                 for (int ch = lane; ch < NCH; ch += 32) {
@@ -346,19 +353,19 @@ center_kernel(const CenterParams p) {
     }
     __syncthreads();
     // on-site term: the centre's own Gaussian, l = 0 only (second term of Eq. 13)
-    if (tid < NMAX && !p.c_bar && !p.sites) c_t[(zi_species * NMAX + tid) * LMP] += p.w0 * __ldg(p.self_term + tid);
+    if (tid < NMAX && !o_cbar && !o_sites) c_t[(zi_species * NMAX + tid) * LMP] += o_w0 * __ldg(p.self_term + tid);
     __syncthreads();
     const int W = S * NE;                                                  // coefficients per centre
-    const int RW = CC ? W : F;                                             // width of an output row
-    if (p.c_bar) {
+    const int RW = CC ? W : (o_compact ? p.Fc : F);                        // width of an output row
+    if (o_cbar) {
         // inner average: the mean coefficients (on-site terms included) take the place of the centre's own
         for (int e = tid; e < W; e += kThreads) {
             const int row = e / LM;
-            c_t[row * LMP + (e - row * LM)] = __ldg(p.c_bar + e);
+            c_t[row * LMP + (e - row * LM)] = __ldg(o_cbar + e);
         }
         __syncthreads();
     }
-    if ((!DERIV && p.emit_coeff) || CC) {
+    if ((!DERIV && o_emit) || CC) {
         // coefficient mode: the tile itself is the result, index (mu n_max + n) (l_max+1)^2 + l^2 + l + m
         float* crow = p.out_desc + (size_t)c_idx * W;
         for (int e = tid; e < W; e += kThreads) {
@@ -374,7 +381,7 @@ center_kernel(const CenterParams p) {
     // pass through the (now idle) staging area in slabs, so that global memory is written in
     // feature order, whole sectors at a time.
     const long long row_base = DERIV ? p.row_ptr[c_idx] : 0;
-    const bool has_own = DERIV && !p.sites;          // a centre that is no atom has no row of its own
+    const bool has_own = DERIV && !o_sites;          // a centre that is no atom has no row of its own
     if (CC) {
         // the centre's own row: minus the sum over the atoms that move relative to it
         if (has_own) {
@@ -387,9 +394,17 @@ center_kernel(const CenterParams p) {
         }
     } else {
         // with given mean coefficients every centre would write the same descriptor: the first one does
-        const bool write_desc = !p.c_bar || c_idx == 0;
-        float* desc_row = p.out_desc + (p.c_bar ? (size_t)0 : (size_t)c_idx * F);
-        float* own = has_own ? p.out_jac + (size_t)(row_base + p.self_row[c_idx]) * 3 * F : nullptr;
+        const bool write_desc = !o_cbar || c_idx == 0;
+        float* desc_row = p.out_desc + (o_cbar ? (size_t)0 : (size_t)c_idx * F);
+        // species-compact rows: the centre's own row keeps every block and lives in an array of its own;
+        // its slot among the compact rows is zero-filled
+        float* own = !has_own ? nullptr
+                     : o_compact ? p.out_center + (size_t)c_idx * 3 * F
+                                 : p.out_jac + (size_t)(row_base + p.self_row[c_idx]) * 3 * F;
+        if (has_own && o_compact) {
+            float* slot = p.out_jac + (size_t)(row_base + p.self_row[c_idx]) * 3 * RW;
+            for (int e = tid; e < 3 * RW; e += kThreads) slot[e] = 0.f;
+        }
         float* slab = smem + lay.sSD;
         constexpr int NV = DERIV ? 4 : 1;                                   // values per feature
         const int NP = F / L1;                                              // (species pair, n, n') groups
@@ -401,12 +416,12 @@ center_kernel(const CenterParams p) {
         // group (the generic loop below loads two operands per multiply-add).
         const bool grouped = !DERIV && (lay.total - lay.sSD) >= F && !(SOAP_DEBUG_SKIP & 8);
         if (grouped) {
-            const int NB = p.crossover ? S * (S + 1) / 2 : S;
+            const int NB = o_cross ? S * (S + 1) / 2 : S;
             for (int it = tid; it < NB * L1 * NMAX; it += kThreads) {
                 const int n1 = it % NMAX, rest = it / NMAX, b = rest % NB, l = rest / NB;   // l slowest: warps share 2l+1
                 int mu = 0, nu = 0, boff = 0;                                                // block b -> (mu, nu), feature offset
                 for (int k = 0, a2 = 0; a2 < S; ++a2)
-                    for (int b2 = a2; b2 < (p.crossover ? S : a2 + 1); ++b2, ++k) {
+                    for (int b2 = a2; b2 < (o_cross ? S : a2 + 1); ++b2, ++k) {
                         if (k == b) { mu = a2; nu = b2; }
                         if (k < b) boff += (a2 == b2) ? (NMAX * (NMAX + 1) / 2) * L1 : NMAX * NCH;
                     }
@@ -496,21 +511,22 @@ center_kernel(const CenterParams p) {
     // image of the same atom already wrote it.
     auto product_rule = [&](auto acc_tag, int Z, float4 d, const float2* wG, float* out) {
         constexpr bool ACC = decltype(acc_tag)::value;
-        const int F2 = 2 * F;
+        const int PS = RW, PS2 = 2 * RW;                      // stride between the three direction planes
         // position of the row start inside a 128-byte line, in floats: sweeps start on line boundaries
         // where the row allows it (a warp store that straddles two lines costs two L1 wavefronts)
         const int a_line = (int)((reinterpret_cast<size_t>(out) >> 2) & 31);
         auto put = [&](int f, float vx, float vy, float vz) {
             if (SOAP_DEBUG_SKIP & 128) vx = vy = vz = 1.f;
-            if (ACC) { out[f] += vx; out[F + f] += vy; out[F2 + f] += vz; }
-            else { out[f] = vx; out[F + f] = vy; out[F2 + f] = vz; }
+            if (ACC) { out[f] += vx; out[PS + f] += vy; out[PS2 + f] += vz; }
+            else { out[f] = vx; out[PS + f] = vy; out[PS2 + f] = vz; }
         };
         int lo = 0;
         for (int mu = 0; mu < S; ++mu) {
-            for (int nu = mu; nu < (p.crossover ? S : mu + 1); ++nu) {
+            for (int nu = mu; nu < (o_cross ? S : mu + 1); ++nu) {
                 const int hi = lo + ((mu == nu) ? (NMAX * (NMAX + 1) / 2) * L1 : NMAX * NCH);
                 const int first = ((lo + a_line) & ~31) - a_line;
                 if (mu != Z && nu != Z) {
+                    if (o_compact) continue;                  // compact rows hold only the blocks that involve Z
                     if (!ACC)
                         for (int f = first + lane; f < hi; f += 32)
                             if (f >= lo) put(f, 0.f, 0.f, 0.f);
@@ -553,8 +569,8 @@ center_kernel(const CenterParams p) {
                                 if (prev ? (n1 >= 1) : (n1 < NMAX)) {
                                     const float2 g = gp[n1 * L1];
                                     const float vx = fmaf(g.x, u.y, g.y * xx), vy = fmaf(g.x, u.z, g.y * xy), vz = fmaf(g.x, u.w, g.y * xz);
-                                    if (ACC) { o[n1 * NCH] += vx; o[F + n1 * NCH] += vy; o[F2 + n1 * NCH] += vz; }
-                                    else { o[n1 * NCH] = vx; o[F + n1 * NCH] = vy; o[F2 + n1 * NCH] = vz; }
+                                    if (ACC) { o[n1 * NCH] += vx; o[PS + n1 * NCH] += vy; o[PS2 + n1 * NCH] += vz; }
+                                    else { o[n1 * NCH] = vx; o[PS + n1 * NCH] = vy; o[PS2 + n1 * NCH] = vz; }
                                 }
                             }
                         } else {
@@ -567,8 +583,8 @@ center_kernel(const CenterParams p) {
                                 if (prev ? (n1 >= 1) : (n1 < NMAX)) {
                                     const float4 u = up[n1 * L1];
                                     const float vx = fmaf(g.x, u.y, gx * u.x), vy = fmaf(g.x, u.z, gy * u.x), vz = fmaf(g.x, u.w, gz * u.x);
-                                    if (ACC) { o[n1 * NCH] += vx; o[F + n1 * NCH] += vy; o[F2 + n1 * NCH] += vz; }
-                                    else { o[n1 * NCH] = vx; o[F + n1 * NCH] = vy; o[F2 + n1 * NCH] = vz; }
+                                    if (ACC) { o[n1 * NCH] += vx; o[PS + n1 * NCH] += vy; o[PS2 + n1 * NCH] += vz; }
+                                    else { o[n1 * NCH] = vx; o[PS + n1 * NCH] = vy; o[PS2 + n1 * NCH] = vz; }
                                 }
                             }
                         }
@@ -594,6 +610,9 @@ center_kernel(const CenterParams p) {
                 lo = hi;
             }
         }
+        // compact rows are padded to a multiple of eight floats: the padding is written as zeros
+        if (o_compact && !ACC)
+            for (int f = lo + lane; f < RW; f += 32) put(f, 0.f, 0.f, 0.f);
     };
 
     // Coefficient mode: the row of a neighbour of species Z is grad c^Z_nlm = G_nl grad S_lm + Ghat_nl d S_lm

@@ -5,6 +5,11 @@
 namespace soap {
 // kernel kinds: descriptor only; descriptor and Jacobian; coefficients c^mu_nlm and their Jacobian
 constexpr int kCenterDesc = 0, kCenterDeriv = 1, kCenterCoeff = 2;
+// whether the parameters ask for nothing beyond the default configuration (the kernels instantiated with
+// PLAIN = true assume exactly this)
+inline bool center_params_plain(const CenterParams& p) {
+    return p.crossover && !p.compact && !p.emit_coeff && !p.c_bar && !p.sites && !p.pair_w && p.w0 == 1.f;
+}
 // n_max values with their own instantiation of the derivative kernel; others run the
 // variant that reads n_max at run time.
 inline bool center_has_fixed_nmax(bool deriv, int n_max) {
@@ -19,7 +24,7 @@ cudaError_t center_launch(int kind, int l_max, int n_max, const CenterParams& p,
 #define SOAP_DECLARE_L(LV)                                                                                       \
     cudaError_t center_constants_l##LV(const float* anorm91, const float* dfact16);         \
     cudaError_t center_set_smem_l##LV(int kind, int n_max, int bytes);                                        \
-    cudaError_t center_launch_l##LV(int kind, int n_max, const CenterParams& p, unsigned grid, size_t smem, cudaStream_t st);
+    cudaError_t center_launch_l##LV(int kind, int n_max, bool plain, const CenterParams& p, unsigned grid, size_t smem, cudaStream_t st);
 SOAP_DECLARE_L(0) SOAP_DECLARE_L(1) SOAP_DECLARE_L(2) SOAP_DECLARE_L(3) SOAP_DECLARE_L(4) SOAP_DECLARE_L(5) SOAP_DECLARE_L(6)
 SOAP_DECLARE_L(7) SOAP_DECLARE_L(8) SOAP_DECLARE_L(9) SOAP_DECLARE_L(10) SOAP_DECLARE_L(11) SOAP_DECLARE_L(12)
 #undef SOAP_DECLARE_L

@@ -39,7 +39,7 @@ cudaError_t center_set_smem(int kind, int l_max, int n_max, int bytes) {
 }
 cudaError_t center_launch(int kind, int l_max, int n_max, const CenterParams& p, unsigned grid, size_t smem, cudaStream_t st) {
     switch (l_max) {
-#define X(LV) case LV: return center_launch_l##LV(kind, n_max, p, grid, smem, st);
+#define X(LV) case LV: return center_launch_l##LV(kind, n_max, center_params_plain(p), p, grid, smem, st);
         X(0) X(1) X(2) X(3) X(4) X(5) X(6) X(7) X(8) X(9) X(10) X(11) X(12)
 #undef X
     }
@@ -59,6 +59,9 @@ struct soap_handle {
     int64_t F = 0;
     HostBasis basis;
     std::vector<int> feat_pack;
+    std::vector<int> compact_map;        // [S][Fc] full feature index of each column of a species-compact row
+    int64_t Fc = 0, Fc_pitch = 0;
+    int* d_compact_map = nullptr;
     std::string error;
     // device state (created on first use)
     int device = -1;
@@ -354,6 +357,7 @@ void fill_center_params(soap_t* h, CenterParams& cp, const float* pos, const int
     cp.P = deriv ? h->P_deriv : h->P_desc;
     cp.crossover = h->crossover; cp.emit_coeff = 0; cp.c_bar = nullptr;
     cp.pair_w = h->weight.fn ? h->d_pair_w : nullptr; cp.w0 = (float)h->w0;
+    cp.compact = 0; cp.Fc = (int)h->Fc_pitch; cp.out_center = nullptr;
     cp.out_desc = nullptr; cp.out_jac = nullptr; cp.row_atom = nullptr;
 }
 
@@ -368,6 +372,15 @@ void build_feature_table(soap_t* h) {
                     for (int l = 0; l <= h->l_max; ++l)
                         h->feat_pack.push_back(n | (n2 << 5) | (mu << 10) | (nu << 14) | (l << 18));
     h->F = (int64_t)h->feat_pack.size();
+    // columns of a species-compact row: the features whose species pair involves z, in feature order
+    h->compact_map.clear();
+    for (int z = 0; z < h->S; ++z)
+        for (int64_t f = 0; f < h->F; ++f) {
+            const int pk = h->feat_pack[f];
+            if (((pk >> 10) & 15) == z || ((pk >> 14) & 15) == z) h->compact_map.push_back((int)f);
+        }
+    h->Fc = (int64_t)h->compact_map.size() / h->S;       // the same for every species
+    h->Fc_pitch = (h->Fc + 7) & ~(int64_t)7;
 }
 
 // Everything before the per-centre kernel: argument checks, device set-up, planning when the sizes
@@ -460,7 +473,7 @@ void soap_destroy(soap_t* h) {
     void* ptrs[] = {h->d_table, h->d_self, h->d_kl, h->d_feat, h->d_zlut, h->d_l_of_lm, h->d_counters, h->d_bbox,
                     h->d_grid, h->d_species_idx, h->d_atom_cell, h->d_atom_wrap, h->d_s_wrap, h->d_s_pos, h->d_cell_count,
                     h->d_cell_start, h->d_pair_count, h->d_row_count, h->d_self_row, h->d_order, h->d_pair_ptr, h->d_pair_start, h->d_row_ptr, h->d_tile_sums, h->d_tile_offsets,
-                    h->d_pair_key, h->d_pair_tmp, h->d_pair_row, h->d_work, h->d_pair_w};
+                    h->d_pair_key, h->d_pair_tmp, h->d_pair_row, h->d_work, h->d_pair_w, h->d_compact_map};
     for (void* p : ptrs) if (p) cudaFree(p);
     if (h->h_counters) cudaFreeHost(h->h_counters);
     for (cudaEvent_t e : h->ev) if (e) cudaEventDestroy(e);
@@ -566,7 +579,8 @@ int soap_descriptor_at(soap_t* h, const float* d_positions, const int32_t* d_num
 
 static int derivatives_impl(soap_t* h, const float* d_positions, const int32_t* d_numbers, int64_t n_atoms, const double* cell,
                             const int32_t* d_centers, const float* d_sites, int64_t n_centers, float* d_out_desc, float* d_out_jac,
-                            int64_t capacity_rows, int64_t* d_row_ptr, int32_t* d_row_atom, void* stream) {
+                            int64_t capacity_rows, int64_t* d_row_ptr, int32_t* d_row_atom, void* stream,
+                            float* d_out_center = nullptr) {
     if (h && (!d_row_ptr || capacity_rows < 0)) return fail(h, SOAP_ERR_INVALID_ARG, "d_row_ptr must not be NULL");
     if (h && n_centers > 0 && (!d_out_desc || !d_out_jac || !d_row_atom)) return fail(h, SOAP_ERR_INVALID_ARG, "output pointers must not be NULL");
     Geometry g;
@@ -579,6 +593,7 @@ static int derivatives_impl(soap_t* h, const float* d_positions, const int32_t* 
         cp.row_ptr = (const long long*)d_row_ptr;
         cp.row_capacity = capacity_rows;
         cp.out_desc = d_out_desc; cp.out_jac = d_out_jac; cp.row_atom = d_row_atom;
+        if (d_out_center) { cp.compact = 1; cp.out_center = d_out_center; }
         CU(center_launch(kCenterDeriv, h->l_max, h->n_max, cp, (unsigned)n_centers, h->smem_deriv, st));
     }
     if (h->profiling) CU(cudaEventRecord(h->ev[2], st));
@@ -599,6 +614,44 @@ int soap_derivatives_at(soap_t* h, const float* d_positions, const int32_t* d_nu
     static const float none[3] = {0.f, 0.f, 0.f};
     return derivatives_impl(h, d_positions, d_numbers, n_atoms, cell, nullptr, d_sites ? d_sites : none, n_sites, d_out_desc,
                             d_out_jac, capacity_rows, d_row_ptr, d_row_atom, stream);
+}
+
+int soap_num_compact_features(const soap_t* h, int64_t* n_compact, int64_t* pitch) {
+    if (!h) return SOAP_ERR_INVALID_ARG;
+    if (n_compact) *n_compact = h->Fc;
+    if (pitch) *pitch = h->Fc_pitch;
+    return SOAP_OK;
+}
+
+int soap_compact_feature_map(const soap_t* h, int species_index, int32_t* map) {
+    if (!h || !map || species_index < 0 || species_index >= h->S) return SOAP_ERR_INVALID_ARG;
+    std::memcpy(map, h->compact_map.data() + (size_t)species_index * h->Fc, (size_t)h->Fc * sizeof(int32_t));
+    return SOAP_OK;
+}
+
+int soap_derivatives_compact(soap_t* h, const float* d_positions, const int32_t* d_numbers, int64_t n_atoms, const double* cell,
+                             const int32_t* d_centers, int64_t n_centers, float* d_out_desc, float* d_out_center,
+                             float* d_out_jac, int64_t capacity_rows, int64_t* d_row_ptr, int32_t* d_row_atom, void* stream) {
+    if (h && n_centers > 0 && !d_out_center) return fail(h, SOAP_ERR_INVALID_ARG, "d_out_center must not be NULL");
+    return derivatives_impl(h, d_positions, d_numbers, n_atoms, cell, d_centers, nullptr, n_centers, d_out_desc, d_out_jac,
+                            capacity_rows, d_row_ptr, d_row_atom, stream, n_centers > 0 ? d_out_center : nullptr);
+}
+
+int soap_compact_expand(soap_t* h, const int32_t* d_numbers, const int32_t* d_centers, int64_t n_centers,
+                        const float* d_center_rows, const float* d_jac_compact, const int64_t* d_row_ptr,
+                        const int32_t* d_row_atom, float* d_out_rows, void* stream) {
+    if (!h) return SOAP_ERR_INVALID_ARG;
+    if (n_centers < 0) return fail(h, SOAP_ERR_INVALID_ARG, "negative size");
+    if (n_centers == 0) return SOAP_OK;
+    if (!d_numbers || !d_center_rows || !d_jac_compact || !d_row_ptr || !d_row_atom || !d_out_rows) return fail(h, SOAP_ERR_INVALID_ARG, "NULL pointer");
+    int rc = ensure_device(h);
+    if (rc) return rc;
+    if (!h->d_compact_map) CU(upload(&h->d_compact_map, h->compact_map));
+    compact_expand_kernel<<<(unsigned)n_centers, 256, 0, (cudaStream_t)stream>>>(
+        d_jac_compact, d_center_rows, (const long long*)d_row_ptr, d_row_atom, d_centers, d_numbers, h->d_zlut,
+        h->d_compact_map, (int)h->Fc, (int)h->Fc_pitch, (int)h->F, d_out_rows);
+    CU(cudaGetLastError());
+    return SOAP_OK;
 }
 
 int soap_jacobian_dense(soap_t* h, const float* d_jac_rows, const int64_t* d_row_ptr, const int32_t* d_row_atom,
@@ -625,6 +678,7 @@ int soap_set_crossover(soap_t* h, int crossover) {
         cudaFree(h->d_feat);
         h->d_feat = nullptr;
         CU(upload(&h->d_feat, h->feat_pack));
+        if (h->d_compact_map) { cudaFree(h->d_compact_map); h->d_compact_map = nullptr; }
     }
     return SOAP_OK;
 }

@@ -79,6 +79,10 @@ struct CenterParams {
     int crossover;                // 0: only the species pairs mu == nu are features
     int emit_coeff;               // descriptor build: write the coefficients c^mu_nlm instead of the power spectrum
     const float* c_bar;           // [S n_max (l_max+1)^2] or null: coefficients that replace the centre's own after pass 1
+    // species-compact Jacobian rows: a neighbour's row holds only the blocks that involve its species (pitch Fc, a
+    // multiple of 8 floats); the centre's own full row goes to out_center [C,3,F]
+    int compact, Fc;
+    float* out_center;
     // radial weighting of the neighbour density: per pair (w(d), w'(d)/d), null when off; w0 scales the on-site term
     const float2* pair_w;
     float w0;

@@ -245,3 +245,58 @@ def test_centres_at_arbitrary_points(pkg, case):
         assert np.all(out.descriptor[1].cpu().numpy() == 0) and ref.row_ptr[2] == ref.row_ptr[1]
     # the same handle still serves atom centres afterwards
     check_derivatives(soap, oracle, s, sample=[0, 3])
+
+
+# ----------------------------------------------------------------- species-compact Jacobian rows
+@pytest.mark.parametrize("case", ["water", "chno_periodic", "crossover_off", "one_species"])
+def test_species_compact_rows(pkg, case):
+    kw = {}
+    if case == "water":
+        s, args = water_cluster(25, 6), ([1, 8], 6.0, 8, 6, 0.5, GTO)
+    elif case == "chno_periodic":
+        s, args = small_periodic_cell(4, (True, True, True)), ([1, 6, 7, 8], 4.5, 3, 3, 0.5, POLYNOMIAL, (True, True, True))
+    elif case == "crossover_off":
+        s, args, kw = water_cluster(10, 3), ([1, 8], 5.0, 5, 2, 0.5, GTO, (False, False, False)), {"crossover": False}
+    else:
+        s, args = water_cluster(6, 1), ([8], 5.0, 4, 3, 0.5, GTO)
+        s.numbers[:] = 8
+    soap, oracle = pkg.Soap(*args, **kw), SoapOracle(*args, **kw)
+    S = len(args[0])
+    tri = args[2] * (args[2] + 1) // 2 * (args[3] + 1)
+    cross = args[2] * args[2] * (args[3] + 1)
+    assert soap.n_compact == tri + (0 if case == "crossover_off" else (S - 1) * cross)
+    assert soap.compact_pitch % 8 == 0 and 0 <= soap.compact_pitch - soap.n_compact < 8
+    pos, num = dev(s)
+    sample = list(range(s.n_atoms)) if s.n_atoms <= 30 else [0, 5, 31, s.n_atoms - 1]
+    cen = torch.tensor(sample, dtype=torch.int32).cuda()
+    ref = oracle.derivatives(s.positions, s.numbers, s.cell, sample)
+    comp = soap.derivatives_compact(pos, num, s.cell, cen)
+    assert np.array_equal(comp.row_ptr.cpu().numpy(), ref.row_ptr)
+    assert np.array_equal(comp.row_atom.cpu().numpy(), ref.row_atom)
+    assert col_err(comp.descriptor.cpu().numpy(), ref.descriptor, 0) < DESC_TOL
+    # compact columns against the oracle through the column map, row by row; everything the
+    # compact format leaves out is an exact zero in the oracle's row
+    jac = comp.jacobian.cpu().numpy()
+    own = comp.center_rows.cpu().numpy()
+    sp = oracle._species_index(s.numbers)
+    maps = [soap.compact_feature_map(z) for z in range(S)]
+    full = np.zeros_like(ref.jacobian)
+    for a, i in enumerate(sample):
+        for r in range(ref.row_ptr[a], ref.row_ptr[a + 1]):
+            atom = ref.row_atom[r]
+            if atom == i:
+                full[r] = own[a]
+                assert np.all(jac[r] == 0)
+                continue
+            m = maps[sp[atom]]
+            assert np.all(np.delete(ref.jacobian[r], m, axis=1) == 0)
+            full[r][:, m] = jac[r][:, :soap.n_compact]
+            assert np.all(jac[r][:, soap.n_compact:] == 0)
+    assert col_err(full, ref.jacobian, (0, 1)) < JAC_TOL
+    # the expansion kernel gives the same rows; the dense entry point (another instantiation of the
+    # kernel, so not necessarily the same bits) agrees far inside the tolerance
+    exp = soap.compact_expand(num, cen, comp)
+    soap.status()
+    assert np.array_equal(exp.cpu().numpy(), full)
+    dense = soap.derivatives(pos, num, s.cell, cen)
+    assert col_err(dense.jacobian.cpu().numpy(), full.astype(np.float64), (0, 1)) < 1e-5
