@@ -525,6 +525,9 @@ center_kernel(const CenterParams p) {
             for (int nu = mu; nu < (o_cross ? S : mu + 1); ++nu) {
                 const int hi = lo + ((mu == nu) ? (NMAX * (NMAX + 1) / 2) * L1 : NMAX * NCH);
                 const int first = ((lo + a_line) & ~31) - a_line;
+                if ((SOAP_DEBUG_SKIP & 256) && mu != Z && nu != Z) { lo = hi; continue; }
+                if ((SOAP_DEBUG_SKIP & 32) && mu == nu && mu == Z) { lo = hi; continue; }
+                if ((SOAP_DEBUG_SKIP & 64) && mu != nu && (mu == Z || nu == Z)) { lo = hi; continue; }
                 if (mu != Z && nu != Z) {
                     if (o_compact) continue;                  // compact rows hold only the blocks that involve Z
                     if (!ACC)
