@@ -436,8 +436,10 @@ def run_suite(args):
                 r["case"] = name
                 print(json.dumps(r), flush=True)
     elif args.suite == "modes":
-        s = water_cluster(1000, 0)
-        base = ([1, 8], 6.0, 8, 6, 0.5, 0)
+        # on --workload (default: the 1000-molecule cluster; the 300-molecule one is small enough for profiler captures)
+        kind, n, species, r_cut, n_max, l_max, sigma, rbf = WORKLOADS[args.workload]
+        s = make_structure(args.workload)
+        base = (species, r_cut, n_max, l_max, sigma, rbf)
         for mode, crossover in (("derivatives", False), ("descriptor", False), ("coefficients", True),
                                 ("coefficient_derivatives", True), ("average_inner", True), ("average_outer", True),
                                 ("average_inner_derivatives", True), ("average_outer_derivatives", True)):

@@ -499,6 +499,10 @@ center_kernel(const CenterParams p) {
 
     // =========================== pass 2: the Jacobian rows ===========================
     const int NI = S * NCH, SN = S * NMAX;
+    // coefficient mode: table lm -> l in the (now idle) space of the D tiles; the loop below starts with a barrier
+    int* lm_to_l = reinterpret_cast<int*>(smem + lay.wUV);
+    if (CC)
+        for (int e = tid; e < LM; e += kThreads) lm_to_l[e] = __ldg(p.l_of_lm + e);
     float4* wUV = reinterpret_cast<float4*>(smem + lay.wUV) + wid * NI;       // [nu][n'][l]
 
     // Product rule of one pair (Eq. 5).  Lanes take consecutive features of the row in sweeps that
@@ -632,7 +636,7 @@ center_kernel(const CenterParams p) {
                 float vx = 0.f, vy = 0.f, vz = 0.f;
                 if (s == Z) {
                     const int e = f - lo, n = e / LM, lm = e - n * LM;
-                    const int l = (int)sqrtf((float)lm);                  // lm = l^2 + l + m
+                    const int l = lm_to_l[lm];                            // lm = l^2 + l + m
                     const float2 g = wG[n * L1 + l];
                     const float4 h = wSD[lm];
                     const float t = g.y * h.x;
