@@ -29,6 +29,10 @@
 #ifndef SOAP_DEBUG_SKIP
 #define SOAP_DEBUG_SKIP 0
 #endif
+#ifndef SOAP_TRI_UNROLL
+#define SOAP_TRI_UNROLL 2              // sweeps of a same-species block in flight per warp
+#endif
+constexpr int kTriUnroll = SOAP_TRI_UNROLL;
 #ifndef SOAP_MIN_CTAS_DERIV
 #define SOAP_MIN_CTAS_DERIV 3          // resident CTAs per SM the derivative kernel is compiled for
 #endif
@@ -539,7 +543,7 @@ center_kernel(const CenterParams p) {
                             if (f >= lo) put(f, 0.f, 0.f, 0.f);
                 } else if (mu == nu) {
                     const float4* UVz = wUV + Z * NCH;
-#pragma unroll 2
+#pragma unroll kTriUnroll
                     for (int f = first + lane; f < hi; f += 32) {
                         if (f < lo) continue;
                         const unsigned dec = tri_dec[f - lo];                 // (n1 L1 + l) | (n2 L1 + l) << 8
