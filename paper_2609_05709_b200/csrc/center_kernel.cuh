@@ -525,6 +525,7 @@ center_kernel(const CenterParams p) {
         const int a_line = (int)((reinterpret_cast<size_t>(out) >> 2) & 31);
         auto put = [&](int f, float vx, float vy, float vz) {
             if (SOAP_DEBUG_SKIP & 128) vx = vy = vz = 1.f;
+            if ((SOAP_DEBUG_SKIP & 2048) && vx == vx) return;      // keep the arithmetic, drop the stores
             if (ACC) { out[f] += vx; out[PS + f] += vy; out[PS2 + f] += vz; }
             else { out[f] = vx; out[PS + f] = vy; out[PS2 + f] = vz; }
         };
@@ -548,8 +549,12 @@ center_kernel(const CenterParams p) {
                         if (f < lo) continue;
                         const unsigned dec = tri_dec[f - lo];                 // (n1 L1 + l) | (n2 L1 + l) << 8
                         const int iA = dec & 255, iB = dec >> 8;
-                        const float2 g1 = wG[iA], g2 = wG[iB];
-                        const float4 u1 = UVz[iA], u2 = UVz[iB];
+                        float2 g1 = wG[iA], g2 = wG[iB];
+                        float4 u1 = UVz[iA], u2 = UVz[iB];
+                        if (SOAP_DEBUG_SKIP & 1024) {                        // no operand loads: values from the indices
+                            g1 = make_float2((float)iA, d.x); g2 = make_float2((float)iB, d.y);
+                            u1 = make_float4(d.x, d.y, d.z, (float)iA); u2 = make_float4(d.z, d.x, (float)iB, d.y);
+                        }
                         const float t = fmaf(g1.y, u2.x, g2.y * u1.x);      // Ghat_n1 U_n2 + Ghat_n2 U_n1
                         put(f, fmaf(g1.x, u2.y, fmaf(g2.x, u1.y, t * d.x)), fmaf(g1.x, u2.z, fmaf(g2.x, u1.z, t * d.y)),
                             fmaf(g1.x, u2.w, fmaf(g2.x, u1.w, t * d.z)));
@@ -581,7 +586,7 @@ center_kernel(const CenterParams p) {
                                     const float2 g = gp[n1 * L1];
                                     const float vx = fmaf(g.x, u.y, g.y * xx), vy = fmaf(g.x, u.z, g.y * xy), vz = fmaf(g.x, u.w, g.y * xz);
                                     if (ACC) { o[n1 * NCH] += vx; o[PS + n1 * NCH] += vy; o[PS2 + n1 * NCH] += vz; }
-                                    else { o[n1 * NCH] = vx; o[PS + n1 * NCH] = vy; o[PS2 + n1 * NCH] = vz; }
+                                    else if (!((SOAP_DEBUG_SKIP & 2048) && vx == vx)) { o[n1 * NCH] = vx; o[PS + n1 * NCH] = vy; o[PS2 + n1 * NCH] = vz; }
                                 }
                             }
                         } else {
@@ -595,7 +600,7 @@ center_kernel(const CenterParams p) {
                                     const float4 u = up[n1 * L1];
                                     const float vx = fmaf(g.x, u.y, gx * u.x), vy = fmaf(g.x, u.z, gy * u.x), vz = fmaf(g.x, u.w, gz * u.x);
                                     if (ACC) { o[n1 * NCH] += vx; o[PS + n1 * NCH] += vy; o[PS2 + n1 * NCH] += vz; }
-                                    else { o[n1 * NCH] = vx; o[PS + n1 * NCH] = vy; o[PS2 + n1 * NCH] = vz; }
+                                    else if (!((SOAP_DEBUG_SKIP & 2048) && vx == vx)) { o[n1 * NCH] = vx; o[PS + n1 * NCH] = vy; o[PS2 + n1 * NCH] = vz; }
                                 }
                             }
                         }
