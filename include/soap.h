@@ -19,7 +19,8 @@
  *  - `cell` is host memory, 9 doubles, rows = lattice vectors a, b, c; it may
  *    be NULL when no axis is periodic.  Positions need not be wrapped.
  *  - `d_centers` lists the centre atoms (indices into the structure); NULL
- *    means every atom, in order (then n_centers must equal n_atoms).
+ *    means every atom, in order (then n_centers must equal n_atoms; n_centers
+ *    = 0 is an empty list and does nothing).
  *  - `stream` is a cudaStream_t passed as void* (NULL = default stream).  All
  *    calls enqueue work on it and return without waiting, except where noted.
  *  - Feature order: species pairs mu <= nu (species sorted by atomic number),

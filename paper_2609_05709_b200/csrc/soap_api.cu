@@ -317,7 +317,7 @@ int check_inputs(soap_t* h, const float* pos, const int32_t* num, int64_t N, con
     if (!h) return SOAP_ERR_INVALID_ARG;
     if (N < 0 || C < 0 || N > 2000000000LL) return fail(h, SOAP_ERR_INVALID_ARG, "atom or centre count out of range");
     if (N > 0 && (!pos || !num)) return fail(h, SOAP_ERR_INVALID_ARG, "positions and numbers must not be NULL");
-    if (!centers && !sites && C != N) return fail(h, SOAP_ERR_INVALID_ARG, "without a centre list n_centers must equal n_atoms");
+    if (!centers && !sites && C != N && C != 0) return fail(h, SOAP_ERR_INVALID_ARG, "without a centre list n_centers must equal n_atoms");
     return SOAP_OK;
 }
 

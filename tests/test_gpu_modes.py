@@ -300,3 +300,32 @@ def test_species_compact_rows(pkg, case):
     assert np.array_equal(exp.cpu().numpy(), full)
     dense = soap.derivatives(pos, num, s.cell, cen)
     assert col_err(dense.jacobian.cpu().numpy(), full.astype(np.float64), (0, 1)) < 1e-5
+
+
+def test_new_entry_points_with_empty_inputs_and_null_pointers(pkg):
+    s = water_cluster(3, 0)
+    pos, num = dev(s)
+    soap = pkg.Soap([1, 8], 4.0, 2, 2, 0.5, GTO)
+    none = torch.empty(0, dtype=torch.int32, device="cuda")
+    assert soap.coefficients(pos, num, None, none).shape == (0, soap.n_coefficients)
+    out = soap.coefficient_derivatives(pos, num, None, none)
+    assert out.jacobian.shape[0] == 0 and out.row_ptr.cpu().tolist() == [0]
+    comp = soap.derivatives_compact(pos, num, None, none)
+    assert comp.jacobian.shape[0] == 0 and comp.row_ptr.cpu().tolist() == [0]
+    sites = torch.empty((0, 3), dtype=torch.float32, device="cuda")
+    at = soap.derivatives_at(pos, num, sites)
+    assert at.jacobian.shape[0] == 0 and at.descriptor.shape == (0, soap.n_features)
+    # an empty structure seen from a point: no neighbours, zero descriptor
+    nopos, nonum = torch.empty((0, 3), device="cuda"), torch.empty(0, dtype=torch.int32, device="cuda")
+    one = torch.zeros((1, 3), dtype=torch.float32, device="cuda")
+    d = soap.derivatives_at(nopos, nonum, one)
+    assert d.jacobian.shape[0] == 0 and torch.all(d.descriptor == 0)
+    # NULL outputs are refused before any launch
+    n = s.n_atoms
+    lib, h = soap._lib, soap._h
+    assert lib.soap_coefficients(h, pos.data_ptr(), num.data_ptr(), n, None, None, n, None, None) == -1
+    assert lib.soap_descriptor_at(h, pos.data_ptr(), num.data_ptr(), n, None, None, 2, None, None) == -1
+    assert lib.soap_derivatives_compact(h, pos.data_ptr(), num.data_ptr(), n, None, None, n, pos.data_ptr(), None,
+                                        pos.data_ptr(), 0, pos.data_ptr(), pos.data_ptr(), None) == -1
+    assert lib.soap_derivatives_average(h, 1, pos.data_ptr(), num.data_ptr(), n, None, None, n, None, None, None) == -1
+    soap.status()

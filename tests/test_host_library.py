@@ -85,3 +85,31 @@ def test_compute_calls_fail_loudly_without_a_device(pkg):
     rc = s._lib.soap_neighbors(s._h, ctypes.c_void_p(16), ctypes.c_void_p(16), 1, None, None, 1,
                                ctypes.byref(n), ctypes.byref(n), None)
     assert rc == -4      # SOAP_ERR_CUDA: no CPU path behind the ABI
+
+
+def test_options_change_the_host_side_tables(pkg):
+    """Crossover, compact-row maps and weighting arguments are host logic: no GPU involved."""
+    s = pkg.Soap([1, 6, 8], 5.0, 3, 2, 0.5)
+    o = SoapOracle([1, 6, 8], 5.0, 3, 2, 0.5)
+    tri, cross = 6 * 3, 9 * 3
+    assert s.n_features == 3 * tri + 3 * cross and s.n_coefficients == 3 * 3 * 9
+    assert s.n_compact == tri + 2 * cross and s.compact_pitch == (s.n_compact + 7) // 8 * 8
+    for z in range(3):
+        m = s.compact_feature_map(z)
+        want = [f for f, (mu, nu, *_rest) in enumerate(o.table) if mu == z or nu == z]
+        assert list(m) == want
+    with pytest.raises(pkg.SoapError):
+        s.compact_feature_map(3)
+    # crossover off: the table shrinks to the same-species blocks, the compact row is the whole row of its species
+    d = pkg.Soap([1, 6, 8], 5.0, 3, 2, 0.5, crossover=False)
+    od = SoapOracle([1, 6, 8], 5.0, 3, 2, 0.5, crossover=False)
+    assert d.n_features == 3 * tri == od.n_features and d.n_compact == tri
+    assert [d.feature_info(f) for f in range(d.n_features)] == [tuple(int(v) for v in r) for r in od.table]
+    assert list(d.compact_feature_map(1)) == list(range(tri, 2 * tri))
+    # weighting arguments are validated before anything touches a device
+    for bad in [{"function": "poly", "r0": 0.0, "m": 1}, {"function": "pow", "r0": 1.0, "m": -1, "d": 1.0},
+                {"function": "pow", "r0": 1.0, "m": 2, "d": 0.0}, {"function": "exp", "r0": 1.0, "d": -1.0}]:
+        with pytest.raises(pkg.SoapError) as e:
+            pkg.Soap([1, 8], 5.0, 2, 2, 0.5, weighting=bad)
+        assert e.value.code == -1
+    pkg.Soap([1, 8], 5.0, 2, 2, 0.5, weighting={"function": "exp", "r0": 1.0, "c": 2.0, "d": 0.5})
