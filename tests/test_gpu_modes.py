@@ -329,3 +329,53 @@ def test_new_entry_points_with_empty_inputs_and_null_pointers(pkg):
                                         pos.data_ptr(), 0, pos.data_ptr(), pos.data_ptr(), None) == -1
     assert lib.soap_derivatives_average(h, 1, pos.data_ptr(), num.data_ptr(), n, None, None, n, None, None, None) == -1
     soap.status()
+
+
+# ----------------------------------------------------------------- the modes at the benchmark's full sizes
+def test_modes_at_full_size_sampled(pkg):
+    """The configurations `bench.py --suite modes|compact` times (1000-molecule cluster, every centre on
+    the GPU), checked on sampled centres the oracle computes one by one."""
+    s = water_cluster(1000, 0)
+    args = ([1, 8], 6.0, 8, 6, 0.5, GTO)
+    soap, oracle = pkg.Soap(*args), SoapOracle(*args)
+    pos, num = dev(s)
+    sample = [0, 1, 1500, 2999] + list(range(77, 3000, 487))
+    sp = oracle._species_index(s.numbers)
+    # species-compact rows of all 3000 centres
+    comp = soap.derivatives_compact(pos, num)
+    ref = oracle.derivatives(s.positions, s.numbers, None, sample)
+    row_ptr, row_atom = comp.row_ptr.cpu().numpy(), comp.row_atom.cpu().numpy()
+    maps = [soap.compact_feature_map(z) for z in range(2)]
+    got = []
+    for b, a in enumerate(sample):
+        lo, hi = row_ptr[a], row_ptr[a + 1]
+        assert np.array_equal(row_atom[lo:hi], ref.row_atom[ref.row_ptr[b]:ref.row_ptr[b + 1]])
+        rows = comp.jacobian[lo:hi].cpu().numpy()
+        full = np.zeros((hi - lo, 3, soap.n_features), np.float32)
+        for r in range(hi - lo):
+            atom = row_atom[lo + r]
+            if atom == a:
+                full[r] = comp.center_rows[a].cpu().numpy()
+            else:
+                full[r][:, maps[sp[atom]]] = rows[r][:, :soap.n_compact]
+        got.append(full)
+    assert col_err(np.concatenate(got), ref.jacobian, (0, 1)) < JAC_TOL
+    assert col_err(comp.descriptor.cpu().numpy()[sample], ref.descriptor, 0) < DESC_TOL
+    del comp
+    # coefficient mode of all 3000 centres
+    out = soap.coefficient_derivatives(pos, num)
+    cref = modes.coefficient_derivatives(oracle, s.positions, s.numbers, None, sample)
+    row_ptr = out.row_ptr.cpu().numpy()
+    got = [out.jacobian[row_ptr[a]:row_ptr[a + 1]].cpu().numpy() for a in sample]
+    assert col_err(np.concatenate(got), cref.jacobian, (0, 1)) < JAC_TOL
+    assert col_err(out.descriptor.cpu().numpy()[sample], cref.descriptor, 0) < DESC_TOL
+    del out
+    # outer average over all centres: equals the mean of the per-centre results of the plain entry point
+    # (themselves checked against the oracle at this size in test_gpu_parity.py), in fp64
+    d, jac = soap.derivatives_average("outer", pos, num)
+    plain = soap.derivatives(pos, num)
+    acc = torch.zeros((3000, 3, soap.n_features), dtype=torch.float64, device="cuda")
+    acc.index_add_(0, plain.row_atom.long(), plain.jacobian.double())
+    want = (acc / 3000).cpu().numpy()
+    assert col_err(jac.cpu().numpy(), want, (0, 1)) < 1e-5
+    assert col_err(d.cpu().numpy()[None], plain.descriptor.double().mean(dim=0).cpu().numpy()[None], 0) < 1e-5
