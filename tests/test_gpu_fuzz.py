@@ -71,7 +71,7 @@ def draw(seed):
     return Structure(pos, numbers, cell, pbc), (species, r_cut, n_max, l_max, sigma, rbf, pbc), kw, rng
 
 
-@pytest.mark.parametrize("seed", range(60))
+@pytest.mark.parametrize("seed", range(80))
 def test_random_configuration(seed):
     if not torch.cuda.is_available():
         pytest.skip("no CUDA device")
@@ -94,8 +94,15 @@ def test_random_configuration(seed):
     d = soap.descriptor(pos, num, s.cell)
     soap.status()
     assert col_err(d.cpu().numpy(), ref.descriptor, 0) < DESC_TOL, tag
-    which = seed % 3
-    if which == 0:                                   # compact rows expand to the same rows
+    which = seed % 4
+    if which == 3:                                   # averaged descriptor and Jacobian
+        mode = "inner" if seed % 8 == 3 else "outer"
+        rd, rj = modes.average_derivatives(oracle, mode, s.positions, s.numbers, s.cell)
+        gd, gj = soap.derivatives_average(mode, pos, num, s.cell)
+        soap.status()
+        assert col_err(gd.cpu().numpy()[None], rd[None], 0) < DESC_TOL, tag
+        assert col_err(gj.cpu().numpy(), rj, (0, 1)) < JAC_TOL, tag
+    elif which == 0:                                   # compact rows expand to the same rows
         comp = soap.derivatives_compact(pos, num, s.cell)
         exp = soap.compact_expand(num, None, comp).cpu().numpy()
         soap.status()
