@@ -154,6 +154,17 @@ def test_config2_water_1000_sampled(pkg):
     assert torch.isfinite(out.jacobian).all() and torch.isfinite(out.descriptor).all()
 
 
+@pytest.mark.parametrize("l_max", [2, 4, 6, 8, 10, 12])
+@pytest.mark.parametrize("n_max", [2, 4, 6, 8, 10, 12])
+def test_config3_hyperparameter_map_cells_sampled(pkg, n_max, l_max):
+    """Every cell of the (n_max, l_max) map `bench.py --suite map` times, on the full 1000-molecule cluster:
+    every centre on the GPU, three of them against the oracle."""
+    s = water_cluster(1000, 0)
+    args = ([1, 8], 6.0, n_max, l_max, 0.5, GTO)
+    soap, oracle = pkg.Soap(*args), SoapOracle(*args)
+    check_derivatives(soap, oracle, s, sample=[5, 1499, 2990])
+
+
 def test_config4_multispecies_box_sampled(pkg):
     s = multispecies_box(2000, 0)
     args = ([6, 1, 7, 8], 5.0, 8, 8, 0.4, POLYNOMIAL, (True, True, True))
