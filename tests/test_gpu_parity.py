@@ -191,6 +191,33 @@ def test_config5_descriptor_only_30k(pkg):
     assert [int(x) for x in (ptr[1:] - ptr[:-1]).cpu()] == [len(l) for l in lists]
 
 
+def test_config5_descriptor_only_million_atoms_sampled(pkg):
+    """The largest size of the scaling benchmark (1,000,002 atoms): every centre on the GPU, a handful of
+    centres and their neighbour lists against the oracle, and whole-output properties."""
+    s = water_cluster(333334, 0)
+    assert s.n_atoms == 1000002
+    args = ([1, 8], 5.0, 8, 6, 0.5, GTO)
+    soap, oracle = pkg.Soap(*args), SoapOracle(*args)
+    pos, num = dev(s)
+    d = soap.descriptor(pos, num)
+    soap.status()
+    sample = [0, 1000001, 500000, 123456, 777777, 999000]
+    ref = oracle.descriptor(s.positions, s.numbers, None, sample)
+    assert col_err(d[sample].cpu().numpy(), ref, 0) < DESC_TOL
+    cen = torch.tensor(sample, dtype=torch.int32).cuda()
+    ptr, atom, _ = soap.neighbor_list(pos, num, None, cen)
+    lists = oracle.neighbor_list(s.positions, None, sample)
+    ptr, atom = ptr.cpu().numpy(), atom.cpu().numpy()
+    for a, lst in enumerate(lists):
+        assert [int(x) for x in atom[ptr[a]:ptr[a + 1]]] == [t[0] for t in lst]
+    # whole output: finite, and every feature with mu == nu and n == n' is a sum of squares
+    assert torch.isfinite(d).all()
+    diag = [f for f, (mu, nu, n, n2, l) in enumerate(oracle.table) if mu == nu and n == n2]
+    cols = d[:, torch.tensor(diag, device="cuda")]
+    assert float(cols.min()) >= 0.0
+    assert float(cols.amax(dim=0).min()) > 0.0
+
+
 def test_device_side_errors_are_reported(pkg):
     s = water_cluster(8, 0)
     soap = pkg.Soap([1, 8], 5.0, 2, 2, 0.5)
