@@ -310,7 +310,7 @@ def run_cuda(args):
 
 
 def time_case(struct, species, r_cut, n_max, l_max, sigma, rbf, mode, steps, warmup=3, crossover=True):
-    """Device-resident timing of one configuration; returns a dict for the tables in the benchmark spec."""
+    """Device-resident timing of one configuration; returns a dict (one row of the measured tables)."""
     import torch
     import paper_2609_05709_b200 as pkg
     pbc = (True, True, True) if struct.cell is not None else (False, False, False)
