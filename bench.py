@@ -427,6 +427,42 @@ def run_suite(args):
             print(json.dumps({"case": "driver", "workers": world, "atoms": s.n_atoms, "batch": batch,
                               "mode": "derivatives" if derivatives else "descriptor", "seconds": best,
                               "atoms_per_s": s.n_atoms / best}), flush=True)
+    elif args.suite == "graph":
+        # launch-bound small systems: one planned step recorded in a CUDA graph and replayed
+        import paper_2609_05709_b200 as pkg
+        for name in ("water8_gto_n4_l3_rc5", "water300_gto_n8_l6_rc6"):
+            kind, n, species, r_cut, n_max, l_max, sigma, rbf = WORKLOADS[name]
+            st = make_structure(name)
+            soap = pkg.Soap(species, r_cut, n_max, l_max, sigma, rbf)
+            pos, num = torch.from_numpy(st.positions).cuda(), torch.from_numpy(st.numbers).cuda()
+            C, F = st.n_atoms, soap.n_features
+            _, n_rows = soap.neighbors(pos, num)
+            desc = torch.empty((C, F), device="cuda")
+            jac = torch.empty((n_rows, 3, F), device="cuda")
+            row_ptr = torch.empty(C + 1, dtype=torch.int64, device="cuda")
+            row_atom = torch.empty(n_rows, dtype=torch.int32, device="cuda")
+            step = lambda: soap.derivatives_into(pos, num, None, None, desc, jac, row_ptr, row_atom)
+            for _ in range(3):
+                step()
+            torch.cuda.synchronize()
+            graph = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(graph):
+                step()
+            out = {"case": "graph", "workload": name, "atoms": C}
+            for label, fn in (("direct_ms", step), ("graph_replay_ms", graph.replay)):
+                for _ in range(5):
+                    fn()
+                times = []
+                for _ in range(max(steps, 20)):
+                    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                    e0.record()
+                    fn()
+                    e1.record()
+                    e1.synchronize()
+                    times.append(e0.elapsed_time(e1))
+                out[label] = statistics.median(times)
+            soap.status()
+            print(json.dumps(out), flush=True)
     elif args.suite == "compact":
         for name in ("water1000_gto_n8_l6_rc6", "chno2000_poly_n8_l8_rc5"):
             kind, n, species, r_cut, n_max, l_max, sigma, rbf = WORKLOADS[name]
@@ -465,12 +501,13 @@ def main():
     ap.add_argument("--workload", default=DEFAULT_WORKLOAD, choices=sorted(WORKLOADS))
     ap.add_argument("--kernel-only", action="store_true",
                     help="skip the end-to-end and CPU-baseline legs (for profiler captures)")
-    ap.add_argument("--suite", choices=["map", "scaling", "configs", "desc30k", "modes", "driver", "compact"],
+    ap.add_argument("--suite", choices=["map", "scaling", "configs", "desc30k", "modes", "driver", "compact", "graph"],
                     help="extra measurements beside the headline line: 'map' = descriptor+Jacobian over "
                          "n_max x l_max on the 1000-molecule cluster, 'scaling' = descriptor-only on "
                          "3k..1M atoms, 'configs' = the periodic multi-species box and the tiny cluster, "
                          "'desc30k' = descriptor-only on 30,000 atoms alone (small enough for profiler captures), "
                          "'compact' = species-compact against full Jacobian rows on the water cluster and the four-species box, "
+                         "'graph' = a planned step replayed from a CUDA graph on the small clusters, "
                          "'driver' = the multi-process driver with --gpus workers, results on the host, "
                          "'modes' = crossover off, coefficient mode and the averaged modes on the 1000-molecule cluster; "
                          "prints one JSON line per case")

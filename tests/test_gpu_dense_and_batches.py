@@ -78,3 +78,37 @@ def test_centre_batches_equal_one_call(pkg):
         assert torch.equal(got.jacobian, whole.jacobian[r0:r1])       # same kernels, same inputs: bit for bit
         rows += r1 - r0
     assert rows == whole.jacobian.shape[0]
+
+
+def test_a_planned_step_can_be_captured_in_a_cuda_graph_and_replayed(pkg):
+    """After the first call for a structure size the library neither allocates nor waits, so a step
+    can be recorded once and replayed on new positions of the same size (launch-bound small systems)."""
+    s = water_cluster(8, 3)
+    soap = pkg.Soap([1, 8], 5.0, 4, 3, 0.5, GTO)
+    pos = torch.from_numpy(s.positions).cuda()
+    num = torch.from_numpy(s.numbers).cuda()
+    n = s.n_atoms
+    _, nrows = soap.neighbors(pos, num)
+    cap = nrows + 64                                            # head-room: the moved structure may gain rows
+    desc = torch.empty((n, soap.n_features), device="cuda")
+    jac = torch.empty((cap, 3, soap.n_features), device="cuda")
+    row_ptr = torch.empty(n + 1, dtype=torch.int64, device="cuda")
+    row_atom = torch.empty(cap, dtype=torch.int32, device="cuda")
+    soap.derivatives_into(pos, num, None, None, desc, jac, row_ptr, row_atom)     # warm-up outside the capture
+    torch.cuda.synchronize()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph):
+        soap.derivatives_into(pos, num, None, None, desc, jac, row_ptr, row_atom)
+    # new coordinates in the captured input buffer, then replay
+    rng = np.random.default_rng(5)
+    moved = s.positions + rng.normal(scale=0.05, size=s.positions.shape).astype(np.float32)
+    pos.copy_(torch.from_numpy(moved).cuda())
+    graph.replay()
+    torch.cuda.synchronize()
+    soap.status()
+    got_desc, got_ptr = desc.clone(), row_ptr.clone()
+    rows = int(got_ptr[-1])
+    got_jac, got_atom = jac[:rows].clone(), row_atom[:rows].clone()
+    ref = soap.derivatives(torch.from_numpy(moved).cuda(), num)
+    assert torch.equal(got_ptr, ref.row_ptr) and torch.equal(got_atom, ref.row_atom)
+    assert torch.equal(got_desc, ref.descriptor) and torch.equal(got_jac, ref.jacobian)
