@@ -140,6 +140,11 @@ int soap_derivatives(soap_t *h, const float *d_positions, const int32_t *d_numbe
 int soap_jacobian_dense(soap_t *h, const float *d_jac_rows, const int64_t *d_row_ptr, const int32_t *d_row_atom,
                         int64_t n_centers, const int32_t *d_include, int64_t n_include, float *d_out, void *stream);
 
+/* The same scatter for rows of any width (`width` floats per direction): the
+ * dense (centre, atom, 3, W) view of soap_coefficient_derivatives' rows. */
+int soap_rows_dense(soap_t *h, const float *d_rows, int64_t width, const int64_t *d_row_ptr, const int32_t *d_row_atom,
+                    int64_t n_centers, const int32_t *d_include, int64_t n_include, float *d_out, void *stream);
+
 /* ---- output modes beyond the per-centre power spectrum (the interface section of the
  *      paper: the crossover flag, the coefficient mode, the inner and outer averages) ---- */
 

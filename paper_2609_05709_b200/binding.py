@@ -18,7 +18,7 @@ EXPORTED_SYMBOLS = [
     "soap_set_crossover", "soap_num_coefficients", "soap_coefficients", "soap_coefficient_derivatives",
     "soap_descriptor_average", "soap_derivatives_average", "soap_set_weighting",
     "soap_neighbors_at", "soap_descriptor_at", "soap_derivatives_at",
-    "soap_num_compact_features", "soap_compact_feature_map", "soap_derivatives_compact", "soap_compact_expand",
+    "soap_rows_dense", "soap_num_compact_features", "soap_compact_feature_map", "soap_derivatives_compact", "soap_compact_expand",
 ]
 
 _ERRORS = {-1: "SOAP_ERR_INVALID_ARG", -2: "SOAP_ERR_UNKNOWN_SPECIES", -3: "SOAP_ERR_CAPACITY",
@@ -65,6 +65,7 @@ def load_library() -> C.CDLL:
     lib.soap_status.argtypes = [vp, C.POINTER(i64), C.POINTER(i64), vp]
     lib.soap_neighbor_counts_static.argtypes = [vp, i64, C.c_double, vp, vp, C.c_char_p, i64]
     lib.soap_jacobian_dense.argtypes = [vp, vp, vp, vp, i64, vp, i64, vp, vp]
+    lib.soap_rows_dense.argtypes = [vp, vp, i64, vp, vp, i64, vp, i64, vp, vp]
     lib.soap_neighbors_at.argtypes = common + [C.POINTER(i64), C.POINTER(i64), vp]
     lib.soap_descriptor_at.argtypes = common + [vp, vp]
     lib.soap_derivatives_at.argtypes = common + [vp, vp, i64, vp, vp, vp]
@@ -418,10 +419,11 @@ class Soap:
             n_inc, iptr = include.shape[0], C.c_void_p(include.data_ptr())
         else:
             n_inc, iptr = int(n_atoms), None
+        width = deriv.jacobian.shape[2]                     # F, or W for the rows of the coefficient mode
         if out is None:
-            out = torch.empty((c, n_inc, 3, self.n_features), dtype=torch.float32, device=deriv.jacobian.device)
-        self._check(self._lib.soap_jacobian_dense(self._h, deriv.jacobian.data_ptr(), deriv.row_ptr.data_ptr(),
-                                                  deriv.row_atom.data_ptr(), c, iptr, n_inc, out.data_ptr(), self._stream()))
+            out = torch.empty((c, n_inc, 3, width), dtype=torch.float32, device=deriv.jacobian.device)
+        self._check(self._lib.soap_rows_dense(self._h, deriv.jacobian.data_ptr(), width, deriv.row_ptr.data_ptr(),
+                                              deriv.row_atom.data_ptr(), c, iptr, n_inc, out.data_ptr(), self._stream()))
         return out
 
     def derivatives_batched(self, positions, numbers, cell=None, centers=None, batch=1024):

@@ -654,17 +654,23 @@ int soap_compact_expand(soap_t* h, const int32_t* d_numbers, const int32_t* d_ce
     return SOAP_OK;
 }
 
+int soap_rows_dense(soap_t* h, const float* d_rows, int64_t width, const int64_t* d_row_ptr, const int32_t* d_row_atom,
+                    int64_t n_centers, const int32_t* d_include, int64_t n_include, float* d_out, void* stream) {
+    if (!h) return SOAP_ERR_INVALID_ARG;
+    if (n_centers < 0 || n_include < 0 || width < 1 || width > 2147483647LL / 3) return fail(h, SOAP_ERR_INVALID_ARG, "size out of range");
+    if (n_centers == 0 || n_include == 0) return SOAP_OK;
+    if (!d_rows || !d_row_ptr || !d_row_atom || !d_out) return fail(h, SOAP_ERR_INVALID_ARG, "NULL pointer");
+    if (n_centers * n_include > 2147483647LL) return fail(h, SOAP_ERR_INVALID_ARG, "more than 2^31-1 (centre, atom) slots: split the call");
+    dense_scatter_kernel<<<(unsigned)(n_centers * n_include), 128, 0, (cudaStream_t)stream>>>(
+        d_rows, (const long long*)d_row_ptr, d_row_atom, n_centers, d_include, n_include, (int)width, d_out);
+    CU(cudaGetLastError());
+    return SOAP_OK;
+}
+
 int soap_jacobian_dense(soap_t* h, const float* d_jac_rows, const int64_t* d_row_ptr, const int32_t* d_row_atom,
                         int64_t n_centers, const int32_t* d_include, int64_t n_include, float* d_out, void* stream) {
     if (!h) return SOAP_ERR_INVALID_ARG;
-    if (n_centers < 0 || n_include < 0) return fail(h, SOAP_ERR_INVALID_ARG, "negative size");
-    if (n_centers == 0 || n_include == 0) return SOAP_OK;
-    if (!d_jac_rows || !d_row_ptr || !d_row_atom || !d_out) return fail(h, SOAP_ERR_INVALID_ARG, "NULL pointer");
-    if (n_centers * n_include > 2147483647LL) return fail(h, SOAP_ERR_INVALID_ARG, "more than 2^31-1 (centre, atom) slots: split the call");
-    dense_scatter_kernel<<<(unsigned)(n_centers * n_include), 128, 0, (cudaStream_t)stream>>>(
-        d_jac_rows, (const long long*)d_row_ptr, d_row_atom, n_centers, d_include, n_include, (int)h->F, d_out);
-    CU(cudaGetLastError());
-    return SOAP_OK;
+    return soap_rows_dense(h, d_jac_rows, h->F, d_row_ptr, d_row_atom, n_centers, d_include, n_include, d_out, stream);
 }
 
 int soap_set_crossover(soap_t* h, int crossover) {
