@@ -21,6 +21,11 @@
 using namespace soap;
 
 namespace soap {
+// tuning knob: SOAP_B200_GENERAL=1 runs the default configuration through the general kernels as well
+static bool force_general() {
+    static const bool on = [] { const char* e = std::getenv("SOAP_B200_GENERAL"); return e && e[0] == '1'; }();
+    return on;
+}
 cudaError_t center_constants(int l_max, const float* anorm91, const float* dfact16) {
     switch (l_max) {
 #define X(LV) case LV: return center_constants_l##LV(anorm91, dfact16);
@@ -39,7 +44,7 @@ cudaError_t center_set_smem(int kind, int l_max, int n_max, int bytes) {
 }
 cudaError_t center_launch(int kind, int l_max, int n_max, const CenterParams& p, unsigned grid, size_t smem, cudaStream_t st) {
     switch (l_max) {
-#define X(LV) case LV: return center_launch_l##LV(kind, n_max, center_params_plain(p), p, grid, smem, st);
+#define X(LV) case LV: return center_launch_l##LV(kind, n_max, center_params_plain(p) && !force_general(), p, grid, smem, st);
         X(0) X(1) X(2) X(3) X(4) X(5) X(6) X(7) X(8) X(9) X(10) X(11) X(12)
 #undef X
     }
