@@ -559,7 +559,7 @@ center_kernel(const CenterParams p) {
                         put(f, fmaf(g1.x, u2.y, fmaf(g2.x, u1.y, t * d.x)), fmaf(g1.x, u2.z, fmaf(g2.x, u1.z, t * d.y)),
                             fmaf(g1.x, u2.w, fmaf(g2.x, u1.w, t * d.z)));
                     }
-                } else if ((NCH & 7) == 0) {
+                } else if ((NCH & 7) == 0 || (NMAX_T != 0 && NMAX_T <= 8)) {
                     // Cross-species block, n_ch a multiple of 8: rows n1 of n_ch floats follow each other, so
                     // windows of n_ch floats that start `shift` floats before a row start are sector-aligned
                     // for every n1.  A lane keeps one window position i: its (n2, l) = i - shift (mod n_ch)
@@ -567,7 +567,11 @@ center_kernel(const CenterParams p) {
                     // the lanes in front of the row start (i < shift) serve the tail of the previous row.
                     const bool first_term = (mu == Z);
                     const float4* UVo = wUV + (first_term ? nu : mu) * NCH;
-                    const int shift = lo & 7;
+                    // When n_ch is no multiple of 8 the rows start at changing sector offsets: no shift then, lanes
+                    // sit on the columns themselves and the warp stores are contiguous but not sector-aligned.
+                    // That still beats the per-feature decode below by 2 to 14 % up to n_max = 8; from
+                    // n_max = 10 on it loses (up to 24 %), so larger n_max keep the aligned sweeps.
+                    const int shift = (NCH & 7) == 0 ? (lo & 7) : 0;
                     for (int i0 = 0; i0 < NCH; i0 += 32) {
                         const int i = i0 + lane;
                         if (i >= NCH) break;
