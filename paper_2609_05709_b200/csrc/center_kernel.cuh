@@ -559,52 +559,65 @@ center_kernel(const CenterParams p) {
                         put(f, fmaf(g1.x, u2.y, fmaf(g2.x, u1.y, t * d.x)), fmaf(g1.x, u2.z, fmaf(g2.x, u1.z, t * d.y)),
                             fmaf(g1.x, u2.w, fmaf(g2.x, u1.w, t * d.z)));
                     }
-                } else if ((NCH & 7) == 0 || (NMAX_T != 0 && NMAX_T <= 8)) {
-                    // Cross-species block, n_ch a multiple of 8: rows n1 of n_ch floats follow each other, so
-                    // windows of n_ch floats that start `shift` floats before a row start are sector-aligned
-                    // for every n1.  A lane keeps one window position i: its (n2, l) = i - shift (mod n_ch)
-                    // is fixed, so the operand that depends on (n2, l) stays in registers over the n1 loop;
-                    // the lanes in front of the row start (i < shift) serve the tail of the previous row.
+                } else if ((NCH & 7) == 0 || (NMAX_T > 8 && (NCH & 3) == 0) || (NMAX_T != 0 && NMAX_T <= 8)) {
+                    // Cross-species block: rows n1 of n_ch floats follow each other.  A lane keeps one position i of
+                    // a window of about n_ch floats, so its (n2, l) is fixed and the operand that depends on (n2, l)
+                    // stays in registers over the unrolled n1 loop.
+                    //  * n_ch a multiple of 8: every row starts at the same offset inside a 32-byte sector; the
+                    //    windows start `shift` floats before the row starts, on sector boundaries, and the lanes in
+                    //    front of a row start (i < shift) serve the tail of the previous row.
+                    //  * n_ch a multiple of 4 only: the offset alternates between two values, so even and odd rows
+                    //    are done in two passes, each with its own shift and window length (taken from n_max = 9
+                    //    on, where it gains 7 to 8 %; with few rows per pass the set-up costs more than it saves,
+                    //    and a window must not be shorter than its shift).
+                    //  * otherwise (taken up to n_max = 8): no shift, lanes sit on the columns themselves; the warp
+                    //    stores are contiguous but not sector-aligned, which still beats decoding every feature by 2 to
+                    //    14 %; from n_max = 10 on it loses (up to 24 %), so those keep the aligned sweeps below.
                     const bool first_term = (mu == Z);
                     const float4* UVo = wUV + (first_term ? nu : mu) * NCH;
-                    // When n_ch is no multiple of 8 the rows start at changing sector offsets: no shift then, lanes
-                    // sit on the columns themselves and the warp stores are contiguous but not sector-aligned.
-                    // That still beats the per-feature decode below by 2 to 14 % up to n_max = 8; from
-                    // n_max = 10 on it loses (up to 24 %), so larger n_max keep the aligned sweeps.
-                    const int shift = (NCH & 7) == 0 ? (lo & 7) : 0;
-                    for (int i0 = 0; i0 < NCH; i0 += 32) {
-                        const int i = i0 + lane;
-                        if (i >= NCH) break;
-                        const bool prev = i < shift;                          // belongs to row n1 - 1
-                        const int j = prev ? i - shift + NCH : i - shift;      // n2 L1 + l
-                        const int l = j % L1;
-                        float* o = out + (lo - shift + i);
-                        if (first_term) {
-                            const float4 u = UVo[j];
-                            const float xx = u.x * d.x, xy = u.x * d.y, xz = u.x * d.z;
-                            const float2* gp = wG + l - (prev ? L1 : 0);
+                    const int T = (NCH & 7) == 0 ? 1 : ((NMAX_T > 8 && (NCH & 3) == 0) ? 2 : 0);
+                    const int TT = T ? T : 1;
 #pragma unroll
-                            for (int n1 = 0; n1 <= NMAX_BOUND; ++n1) {
-                                if (n1 > NMAX) break;
-                                if (prev ? (n1 >= 1) : (n1 < NMAX)) {
-                                    const float2 g = gp[n1 * L1];
-                                    const float vx = fmaf(g.x, u.y, g.y * xx), vy = fmaf(g.x, u.z, g.y * xy), vz = fmaf(g.x, u.w, g.y * xz);
-                                    if (ACC) { o[n1 * NCH] += vx; o[PS + n1 * NCH] += vy; o[PS2 + n1 * NCH] += vz; }
-                                    else if (!((SOAP_DEBUG_SKIP & 2048) && vx == vx)) { o[n1 * NCH] = vx; o[PS + n1 * NCH] = vy; o[PS2 + n1 * NCH] = vz; }
+                    for (int pp = 0; pp < 2; ++pp) {
+                        if (pp >= TT) break;
+                        const int shift = T ? ((a_line + lo + pp * NCH) & 7) : 0;
+                        const int wlen = NCH + shift - (T ? ((a_line + lo + (pp + 1) * NCH) & 7) : 0);
+                        for (int i0 = 0; i0 < wlen; i0 += 32) {
+                            const int i = i0 + lane;
+                            if (i >= wlen) break;
+                            const bool prev = i < shift;                          // belongs to row n1 - 1
+                            const int j = prev ? i - shift + NCH : i - shift;      // n2 L1 + l
+                            const int l = j % L1;
+                            float* o = out + (lo - shift + i);
+                            if (first_term) {
+                                const float4 u = UVo[j];
+                                const float xx = u.x * d.x, xy = u.x * d.y, xz = u.x * d.z;
+                                const float2* gp = wG + l - (prev ? L1 : 0);
+#pragma unroll
+                                for (int k = 0; k <= NMAX_BOUND; ++k) {
+                                    const int n1 = pp + k * TT;
+                                    if (n1 > NMAX) break;
+                                    if (prev ? (n1 >= 1) : (n1 < NMAX)) {
+                                        const float2 g = gp[n1 * L1];
+                                        const float vx = fmaf(g.x, u.y, g.y * xx), vy = fmaf(g.x, u.z, g.y * xy), vz = fmaf(g.x, u.w, g.y * xz);
+                                        if (ACC) { o[n1 * NCH] += vx; o[PS + n1 * NCH] += vy; o[PS2 + n1 * NCH] += vz; }
+                                        else if (!((SOAP_DEBUG_SKIP & 2048) && vx == vx)) { o[n1 * NCH] = vx; o[PS + n1 * NCH] = vy; o[PS2 + n1 * NCH] = vz; }
+                                    }
                                 }
-                            }
-                        } else {
-                            const float2 g = wG[j];
-                            const float gx = g.y * d.x, gy = g.y * d.y, gz = g.y * d.z;
-                            const float4* up = UVo + l - (prev ? L1 : 0);
+                            } else {
+                                const float2 g = wG[j];
+                                const float gx = g.y * d.x, gy = g.y * d.y, gz = g.y * d.z;
+                                const float4* up = UVo + l - (prev ? L1 : 0);
 #pragma unroll
-                            for (int n1 = 0; n1 <= NMAX_BOUND; ++n1) {
-                                if (n1 > NMAX) break;
-                                if (prev ? (n1 >= 1) : (n1 < NMAX)) {
-                                    const float4 u = up[n1 * L1];
-                                    const float vx = fmaf(g.x, u.y, gx * u.x), vy = fmaf(g.x, u.z, gy * u.x), vz = fmaf(g.x, u.w, gz * u.x);
-                                    if (ACC) { o[n1 * NCH] += vx; o[PS + n1 * NCH] += vy; o[PS2 + n1 * NCH] += vz; }
-                                    else if (!((SOAP_DEBUG_SKIP & 2048) && vx == vx)) { o[n1 * NCH] = vx; o[PS + n1 * NCH] = vy; o[PS2 + n1 * NCH] = vz; }
+                                for (int k = 0; k <= NMAX_BOUND; ++k) {
+                                    const int n1 = pp + k * TT;
+                                    if (n1 > NMAX) break;
+                                    if (prev ? (n1 >= 1) : (n1 < NMAX)) {
+                                        const float4 u = up[n1 * L1];
+                                        const float vx = fmaf(g.x, u.y, gx * u.x), vy = fmaf(g.x, u.z, gy * u.x), vz = fmaf(g.x, u.w, gz * u.x);
+                                        if (ACC) { o[n1 * NCH] += vx; o[PS + n1 * NCH] += vy; o[PS2 + n1 * NCH] += vz; }
+                                        else if (!((SOAP_DEBUG_SKIP & 2048) && vx == vx)) { o[n1 * NCH] = vx; o[PS + n1 * NCH] = vy; o[PS2 + n1 * NCH] = vz; }
+                                    }
                                 }
                             }
                         }
