@@ -34,6 +34,8 @@ WORKLOADS = {
     "water8_gto_n4_l3_rc5": ("water", 8, [1, 8], 5.0, 4, 3, 0.5, 0),
     "water300_gto_n8_l6_rc6": ("water", 300, [1, 8], 6.0, 8, 6, 0.5, 0),      # small case for ncu captures
     "chno2000_poly_n8_l8_rc5": ("box", 2000, [1, 6, 7, 8], 5.0, 8, 8, 0.4, 1),
+    # the paper's own headline parameters (r_cut 10, n_max 7, l_max 3; its sigma is not given): context only
+    "water1000_gto_n7_l3_rc10": ("water", 1000, [1, 8], 10.0, 7, 3, 0.5, 0),
 }
 DEFAULT_WORKLOAD = "water1000_gto_n8_l6_rc6"
 METRIC = "SOAP atoms/s, descriptor + Jacobian"
@@ -483,7 +485,7 @@ def run_suite(args):
             r["case"] = "modes"
             print(json.dumps(r), flush=True)
     else:
-        for name in ("water8_gto_n4_l3_rc5", "water1000_gto_n8_l6_rc6", "chno2000_poly_n8_l8_rc5"):
+        for name in ("water8_gto_n4_l3_rc5", "water1000_gto_n8_l6_rc6", "chno2000_poly_n8_l8_rc5", "water1000_gto_n7_l3_rc10"):
             kind, n, species, r_cut, n_max, l_max, sigma, rbf = WORKLOADS[name]
             s = make_structure(name)
             for mode in ("derivatives", "descriptor"):

@@ -154,6 +154,17 @@ def test_config2_water_1000_sampled(pkg):
     assert torch.isfinite(out.jacobian).all() and torch.isfinite(out.descriptor).all()
 
 
+def test_paper_parameters_water_1000_rcut10_sampled(pkg):
+    """The paper's own headline parameters (r_cut 10, n_max 7, l_max 3) on the 1000-molecule cluster:
+    several hundred neighbours per sphere, every centre on the GPU, sampled centres against the oracle."""
+    s = water_cluster(1000, 0)
+    args = ([1, 8], 10.0, 7, 3, 0.5, GTO)
+    soap, oracle = pkg.Soap(*args), SoapOracle(*args)
+    sample = [0, 1499, 2999, 777]
+    check_neighbors(soap, oracle, s, sample)
+    check_derivatives(soap, oracle, s, sample=sample)
+
+
 @pytest.mark.parametrize("l_max", [2, 4, 6, 8, 10, 12])
 @pytest.mark.parametrize("n_max", [2, 4, 6, 8, 10, 12])
 def test_config3_hyperparameter_map_cells_sampled(pkg, n_max, l_max):
