@@ -29,6 +29,9 @@
 #ifndef SOAP_DEBUG_SKIP
 #define SOAP_DEBUG_SKIP 0
 #endif
+#ifndef SOAP_WINDOW_MASK
+#define SOAP_WINDOW_MASK 3             // 3: windows for n_ch % 4 == 0 (two passes); 1: also n_ch % 2 == 0 (four passes)
+#endif
 #ifndef SOAP_TRI_UNROLL
 #define SOAP_TRI_UNROLL 2              // sweeps of a same-species block in flight per warp
 #endif
@@ -587,7 +590,7 @@ center_kernel(const CenterParams p) {
                         put(f, fmaf(g1.x, u2.y, fmaf(g2.x, u1.y, t * d.x)), fmaf(g1.x, u2.z, fmaf(g2.x, u1.z, t * d.y)),
                             fmaf(g1.x, u2.w, fmaf(g2.x, u1.w, t * d.z)));
                     }
-                } else if ((NCH & 7) == 0 || (NMAX_T > 8 && (NCH & 3) == 0) || (NMAX_T != 0 && NMAX_T <= 8)) {
+                } else if ((NCH & 7) == 0 || (NMAX_T > 8 && (NCH & (SOAP_WINDOW_MASK)) == 0) || (NMAX_T != 0 && NMAX_T <= 8)) {
                     // Cross-species block: rows n1 of n_ch floats follow each other.  A lane keeps one position i of
                     // a window of about n_ch floats, so its (n2, l) is fixed and the operand that depends on (n2, l)
                     // stays in registers over the unrolled n1 loop.
@@ -603,10 +606,10 @@ center_kernel(const CenterParams p) {
                     //    14 %; from n_max = 10 on it loses (up to 24 %), so those keep the aligned sweeps below.
                     const bool first_term = (mu == Z);
                     const float4* UVo = wUV + (first_term ? nu : mu) * NCH;
-                    const int T = (NCH & 7) == 0 ? 1 : ((NMAX_T > 8 && (NCH & 3) == 0) ? 2 : 0);
+                    const int T = (NCH & 7) == 0 ? 1 : ((NMAX_T > 8 && (NCH & 3) == 0) ? 2 : ((NMAX_T > 8 && (NCH & (SOAP_WINDOW_MASK)) == 0) ? 4 : 0));
                     const int TT = T ? T : 1;
 #pragma unroll
-                    for (int pp = 0; pp < 2; ++pp) {
+                    for (int pp = 0; pp < 4; ++pp) {
                         if (pp >= TT) break;
                         const int shift = T ? ((a_line + lo + pp * NCH) & 7) : 0;
                         const int wlen = NCH + shift - (T ? ((a_line + lo + (pp + 1) * NCH) & 7) : 0);
