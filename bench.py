@@ -465,6 +465,83 @@ def run_suite(args):
                 out[label] = statistics.median(times)
             soap.status()
             print(json.dumps(out), flush=True)
+    elif args.suite == "small":
+        # a stream of different small structures (launch-bound): descriptor + Jacobian of 256 eight-molecule water
+        # clusters, every structure into buffers of its own, on one stream and round-robin over eight streams
+        # (one library handle per stream; after the first call nothing allocates or waits)
+        import paper_2609_05709_b200 as pkg
+        structs = [water_cluster(8, seed) for seed in range(256)]
+        n, cap_rows = structs[0].n_atoms, structs[0].n_atoms ** 2
+        pos = [torch.from_numpy(st.positions).cuda() for st in structs]
+        num = torch.from_numpy(structs[0].numbers).cuda()
+        for n_streams in (1, 8):
+            streams = [torch.cuda.Stream() for _ in range(n_streams)]
+            handles = [pkg.Soap([1, 8], 5.0, 4, 3, 0.5, 0) for _ in range(n_streams)]
+            F = handles[0].n_features
+            outs = [(torch.empty((n, F), device="cuda"), torch.empty((cap_rows, 3, F), device="cuda"),
+                     torch.empty(n + 1, dtype=torch.int64, device="cuda"), torch.empty(cap_rows, dtype=torch.int32, device="cuda"))
+                    for _ in structs]
+            for h, st in zip(handles, streams):                 # plan once per handle, outside the timing
+                with torch.cuda.stream(st):
+                    h.neighbors(pos[0], num)
+            torch.cuda.synchronize()
+
+            def sweep():
+                for k, p_k in enumerate(pos):
+                    with torch.cuda.stream(streams[k % n_streams]):
+                        handles[k % n_streams].derivatives_into(p_k, num, None, None, *outs[k])
+
+            sweep()
+            torch.cuda.synchronize()
+            for h in handles:
+                h.status()
+            best = None
+            for _ in range(max(3, min(steps, 10))):
+                t0 = time.perf_counter()
+                sweep()
+                torch.cuda.synchronize()
+                dt = time.perf_counter() - t0
+                best = dt if best is None else min(best, dt)
+            print(json.dumps({"case": "small", "structures": len(structs), "atoms_each": n, "streams": n_streams,
+                              "seconds": best, "structures_per_s": len(structs) / best,
+                              "atoms_per_s": len(structs) * n / best, "us_per_structure": 1e6 * best / len(structs)}), flush=True)
+        # the same structures (and 16 times as many) as ONE list of atoms through the batch entry point
+        for copies in (1, 16):
+            soap = pkg.Soap([1, 8], 5.0, 4, 3, 0.5, 0)
+            allpos = torch.cat(pos * copies).contiguous()
+            allnum = num.repeat(len(structs) * copies).contiguous()
+            ptr = torch.arange(0, (len(structs) * copies + 1) * n, n, dtype=torch.int64, device="cuda")
+            N = allpos.shape[0]
+            import ctypes
+            npairs, nrows = ctypes.c_int64(), ctypes.c_int64()
+            soap._check(soap._lib.soap_neighbors_batch(soap._h, allpos.data_ptr(), allnum.data_ptr(), N, ptr.data_ptr(),
+                                                       ptr.shape[0] - 1, ctypes.byref(npairs), ctypes.byref(nrows), soap._stream()))
+            F = soap.n_features
+            desc = torch.empty((N, F), device="cuda")
+            jac = torch.empty((nrows.value, 3, F), device="cuda")
+            row_ptr = torch.empty(N + 1, dtype=torch.int64, device="cuda")
+            row_atom = torch.empty(nrows.value, dtype=torch.int32, device="cuda")
+            call = lambda: soap._check(soap._lib.soap_derivatives_batch(
+                soap._h, allpos.data_ptr(), allnum.data_ptr(), N, ptr.data_ptr(), ptr.shape[0] - 1, desc.data_ptr(),
+                jac.data_ptr(), nrows.value, row_ptr.data_ptr(), row_atom.data_ptr(), soap._stream()))
+            for _ in range(3):
+                call()
+            soap.status()
+            times = []
+            for _ in range(max(steps, 10)):
+                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                e0.record()
+                call()
+                e1.record()
+                e1.synchronize()
+                times.append(e0.elapsed_time(e1) * 1e-3)
+            best = statistics.median(times)
+            nst = len(structs) * copies
+            print(json.dumps({"case": "small", "structures": nst, "atoms_each": n, "streams": "one batch call",
+                              "seconds": best, "structures_per_s": nst / best, "atoms_per_s": nst * n / best,
+                              "us_per_structure": 1e6 * best / nst, "rows": nrows.value,
+                              "jacobian_GBps": nrows.value * 3 * F * 4 / best / 1e9}), flush=True)
+            del soap, desc, jac
     elif args.suite == "compact":
         for name in ("water1000_gto_n8_l6_rc6", "chno2000_poly_n8_l8_rc5"):
             kind, n, species, r_cut, n_max, l_max, sigma, rbf = WORKLOADS[name]
@@ -503,12 +580,13 @@ def main():
     ap.add_argument("--workload", default=DEFAULT_WORKLOAD, choices=sorted(WORKLOADS))
     ap.add_argument("--kernel-only", action="store_true",
                     help="skip the end-to-end and CPU-baseline legs (for profiler captures)")
-    ap.add_argument("--suite", choices=["map", "scaling", "configs", "desc30k", "modes", "driver", "compact", "graph"],
+    ap.add_argument("--suite", choices=["map", "scaling", "configs", "desc30k", "modes", "driver", "compact", "graph", "small"],
                     help="extra measurements beside the headline line: 'map' = descriptor+Jacobian over "
                          "n_max x l_max on the 1000-molecule cluster, 'scaling' = descriptor-only on "
                          "3k..1M atoms, 'configs' = the periodic multi-species box and the tiny cluster, "
                          "'desc30k' = descriptor-only on 30,000 atoms alone (small enough for profiler captures), "
                          "'compact' = species-compact against full Jacobian rows on the water cluster and the four-species box, "
+                         "'small' = a stream of 256 different 24-atom structures on one and on eight CUDA streams, "
                          "'graph' = a planned step replayed from a CUDA graph on the small clusters, "
                          "'driver' = the multi-process driver with --gpus workers, results on the host, "
                          "'modes' = crossover off, coefficient mode and the averaged modes on the 1000-molecule cluster; "

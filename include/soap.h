@@ -101,8 +101,13 @@ int soap_neighbor_list(soap_t *h, int64_t *d_pair_ptr, int32_t *d_pair_atom, int
                        int64_t capacity_pairs, void *stream);
 
 /* Descriptor only: d_out [n_centers, F] fp32, fully overwritten (Eq. 4).
- * Runs the neighbour search itself.  The first call for a structure size
- * plans scratch memory like soap_neighbors (allocates and waits once). */
+ * Runs the neighbour search itself.  A call for a structure with more atoms
+ * or centres than any before it on this handle first plans scratch memory
+ * like soap_neighbors (allocates and waits once); other calls only enqueue
+ * work.  If such a call meets more pairs than the planned scratch holds (a
+ * denser structure), soap_status reports SOAP_ERR_CAPACITY and the outputs
+ * of that call are invalid: call soap_neighbors for that structure, then
+ * repeat. */
 int soap_descriptor(soap_t *h, const float *d_positions, const int32_t *d_numbers, int64_t n_atoms,
                     const double *cell, const int32_t *d_centers, int64_t n_centers,
                     float *d_out, void *stream);
@@ -153,6 +158,28 @@ int soap_rows_dense(soap_t *h, const float *d_rows, int64_t width, const int64_t
  * soap_feature_info; waits for the device when tables are already uploaded.
  * Not to be called while work on this handle is in flight. */
 int soap_set_crossover(soap_t *h, int crossover);
+
+/* ---- many independent structures in one call ----
+ * The paper enumerates work as batches of centres drawn from one structure
+ * each and notes that small systems are bound by launch latency.  These entry
+ * points take many non-periodic structures as ONE list of atoms:
+ * d_struct_ptr [n_structs+1] (device, ascending, d_struct_ptr[0] = 0,
+ * d_struct_ptr[n_structs] = n_atoms) delimits the structures; every atom is a
+ * centre and sees only the atoms of its own structure (0 < d^2 < r_cut^2,
+ * the same fp64 test), found by a warp running over that structure - meant for
+ * molecules of up to a few hundred atoms.  Outputs as in soap_descriptor /
+ * soap_derivatives with atom and centre indices counted through the whole
+ * list; the launch count does not depend on the number of structures.  The
+ * handle must have no periodic axis.  Planning, capacities and errors as in
+ * soap_neighbors / soap_derivatives. */
+int soap_neighbors_batch(soap_t *h, const float *d_positions, const int32_t *d_numbers, int64_t n_atoms,
+                         const int64_t *d_struct_ptr, int64_t n_structs, int64_t *n_pairs, int64_t *n_rows,
+                         void *stream);
+int soap_descriptor_batch(soap_t *h, const float *d_positions, const int32_t *d_numbers, int64_t n_atoms,
+                          const int64_t *d_struct_ptr, int64_t n_structs, float *d_out, void *stream);
+int soap_derivatives_batch(soap_t *h, const float *d_positions, const int32_t *d_numbers, int64_t n_atoms,
+                           const int64_t *d_struct_ptr, int64_t n_structs, float *d_out_desc, float *d_out_jac,
+                           int64_t capacity_rows, int64_t *d_row_ptr, int32_t *d_row_atom, void *stream);
 
 /* ---- species-compact Jacobian rows ----
  * The row of a neighbour of species Z is zero in every species-pair block that

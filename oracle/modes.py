@@ -144,3 +144,25 @@ def site_derivatives(o: SoapOracle, positions, numbers, sites, cell=None) -> Der
         blocks.append(J)
     jac = np.concatenate(blocks, axis=0) if blocks else np.zeros((0, 3, o.n_features))
     return Derivatives(desc, np.array(row_ptr, np.int64), np.array(row_atom, np.int32), jac)
+
+
+# ------------------------------------------------------------------ many independent structures at once
+def batch_derivatives(o: SoapOracle, structures) -> Derivatives:
+    """Non-periodic structures treated as one list of atoms: every atom of every structure is a centre and
+    sees only the atoms of its own structure (the multi-GPU section enumerates work as batches of centres
+    drawn from one structure each; structures never interact).  Output rows as in
+    `SoapOracle.derivatives`, with atom indices counted through the concatenated list."""
+    desc, ptr, atoms, jac = [], [np.zeros(1, np.int64)], [], []
+    base_atom, base_row = 0, 0
+    for positions, numbers in structures:
+        d = o.derivatives(positions, numbers)
+        desc.append(d.descriptor)
+        ptr.append(d.row_ptr[1:] + base_row)
+        atoms.append(d.row_atom + base_atom)
+        jac.append(d.jacobian)
+        base_atom += len(numbers)
+        base_row += int(d.row_ptr[-1])
+    F = o.n_features
+    return Derivatives(np.concatenate(desc) if desc else np.zeros((0, F)), np.concatenate(ptr),
+                       (np.concatenate(atoms) if atoms else np.zeros(0)).astype(np.int32),
+                       np.concatenate(jac) if jac else np.zeros((0, 3, F)))

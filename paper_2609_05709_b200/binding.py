@@ -18,7 +18,8 @@ EXPORTED_SYMBOLS = [
     "soap_set_crossover", "soap_num_coefficients", "soap_coefficients", "soap_coefficient_derivatives",
     "soap_descriptor_average", "soap_derivatives_average", "soap_set_weighting",
     "soap_neighbors_at", "soap_descriptor_at", "soap_derivatives_at",
-    "soap_rows_dense", "soap_num_compact_features", "soap_compact_feature_map", "soap_derivatives_compact", "soap_compact_expand",
+    "soap_rows_dense", "soap_neighbors_batch", "soap_descriptor_batch", "soap_derivatives_batch",
+    "soap_num_compact_features", "soap_compact_feature_map", "soap_derivatives_compact", "soap_compact_expand",
 ]
 
 _ERRORS = {-1: "SOAP_ERR_INVALID_ARG", -2: "SOAP_ERR_UNKNOWN_SPECIES", -3: "SOAP_ERR_CAPACITY",
@@ -73,6 +74,9 @@ def load_library() -> C.CDLL:
     lib.soap_compact_feature_map.argtypes = [vp, i32, C.POINTER(C.c_int32)]
     lib.soap_derivatives_compact.argtypes = common + [vp, vp, vp, i64, vp, vp, vp]
     lib.soap_compact_expand.argtypes = [vp, vp, vp, i64, vp, vp, vp, vp, vp, vp]
+    lib.soap_neighbors_batch.argtypes = [vp, vp, vp, i64, vp, i64, C.POINTER(i64), C.POINTER(i64), vp]
+    lib.soap_descriptor_batch.argtypes = [vp, vp, vp, i64, vp, i64, vp, vp]
+    lib.soap_derivatives_batch.argtypes = [vp, vp, vp, i64, vp, i64, vp, vp, i64, vp, vp, vp]
     lib.soap_set_crossover.argtypes = [vp, i32]
     lib.soap_set_weighting.argtypes = [vp, i32] + [C.c_double] * 5
     lib.soap_num_coefficients.argtypes = [vp, C.POINTER(i64)]
@@ -262,6 +266,35 @@ class Soap:
         row_ptr = torch.empty(c + 1, dtype=torch.int64, device=dev)
         row_atom = torch.empty(max(nrows, 1), dtype=torch.int32, device=dev)
         self.derivatives_into(positions, numbers, cell, centers, desc, jac, row_ptr, row_atom)
+        self.status()
+        return Derivatives(desc, jac[:nrows], row_ptr, row_atom[:nrows])
+
+    # ------------------------------------------------------------------ many structures in one call
+    def derivatives_batch(self, positions, numbers, struct_ptr, jacobian=True):
+        """Many independent non-periodic structures as one list of atoms; `struct_ptr` is an int64 device
+        tensor (B+1,) of offsets.  Returns `Derivatives` over all atoms (indices through the whole list), or
+        the (N, F) descriptor with jacobian=False."""
+        import torch
+        n, _, _ = self._inputs(positions, numbers, None)
+        assert struct_ptr.is_cuda and struct_ptr.dtype == torch.int64 and struct_ptr.is_contiguous()
+        b, sp = struct_ptr.shape[0] - 1, C.c_void_p(struct_ptr.data_ptr())
+        dev = positions.device
+        desc = torch.empty((n, self.n_features), dtype=torch.float32, device=dev)
+        if not jacobian:
+            self._check(self._lib.soap_descriptor_batch(self._h, positions.data_ptr(), numbers.data_ptr(), n, sp, b,
+                                                        desc.data_ptr(), self._stream()))
+            self.status()
+            return desc
+        npairs, nrows = C.c_int64(), C.c_int64()
+        self._check(self._lib.soap_neighbors_batch(self._h, positions.data_ptr(), numbers.data_ptr(), n, sp, b,
+                                                   C.byref(npairs), C.byref(nrows), self._stream()))
+        nrows = int(nrows.value)
+        jac = torch.empty((max(nrows, 1), 3, self.n_features), dtype=torch.float32, device=dev)
+        row_ptr = torch.empty(n + 1, dtype=torch.int64, device=dev)
+        row_atom = torch.empty(max(nrows, 1), dtype=torch.int32, device=dev)
+        self._check(self._lib.soap_derivatives_batch(self._h, positions.data_ptr(), numbers.data_ptr(), n, sp, b,
+                                                     desc.data_ptr(), jac.data_ptr(), jac.shape[0], row_ptr.data_ptr(),
+                                                     row_atom.data_ptr(), self._stream()))
         self.status()
         return Derivatives(desc, jac[:nrows], row_ptr, row_atom[:nrows])
 

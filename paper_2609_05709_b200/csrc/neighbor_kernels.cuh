@@ -591,6 +591,74 @@ pairs_kernel(const float* __restrict__ pos, const int* __restrict__ centers, con
     }
 }
 
+// Many independent non-periodic structures in one launch: atoms of all structures in one list,
+// struct_ptr[b] .. struct_ptr[b+1]-1 the atoms of structure b, every atom a centre that sees only its own
+// structure.  One warp per centre runs over the atoms of its structure (brute force: the structures
+// this is for are small molecules, where the cutoff sphere holds most of the structure anyway), with the same
+// exact fp64 test as the cell-list path; neighbours come out in ascending atom order, so nothing is sorted.
+// Writes what pairs_kernel writes (keys with zero lattice translation) plus the species index of the centre.
+__global__ void __launch_bounds__(kFillWarps * 32)
+batch_pairs_kernel(const float* __restrict__ pos, const int* __restrict__ numbers, const int* __restrict__ z_lut,
+                   int* __restrict__ species_idx, const long long* __restrict__ struct_ptr, long long n_structs,
+                   long long N, double rc2, long long pair_capacity, unsigned long long* pair_key,
+                   int* __restrict__ pair_row, long long* __restrict__ pair_start, int* __restrict__ pair_count,
+                   int* __restrict__ row_count, int* __restrict__ self_row, Counters* counters) {
+    const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
+    const long long i = blockIdx.x * (long long)kFillWarps + wid;
+    if (i >= N) return;
+    if (lane == 0) {
+        const int z = numbers[i];
+        int s = (z >= 0 && z < 128) ? z_lut[z] : -1;
+        if (s < 0) { atomicOr(&counters->status, kStatusUnknownSpecies); s = 0; }
+        species_idx[i] = s;
+    }
+    // the structure that holds atom i: last b with struct_ptr[b] <= i
+    long long lo = 0, hi = n_structs;
+    while (hi - lo > 1) {
+        const long long mid = (lo + hi) >> 1;
+        if (struct_ptr[mid] <= i) lo = mid; else hi = mid;
+    }
+    const long long a = struct_ptr[lo], b = min(struct_ptr[lo + 1], N);
+    const double xi = pos[3 * i], yi = pos[3 * i + 1], zi = pos[3 * i + 2];
+    auto inside = [&](long long j) {
+        if (j >= b) return false;
+        const double dx = __dsub_rn((double)pos[3 * j], xi), dy = __dsub_rn((double)pos[3 * j + 1], yi),
+                     dz = __dsub_rn((double)pos[3 * j + 2], zi);
+        const double d2 = __dadd_rn(__dadd_rn(__dmul_rn(dx, dx), __dmul_rn(dy, dy)), __dmul_rn(dz, dz));
+        return d2 < rc2 && d2 > 0.0;
+    };
+    int k = 0, below = 0;
+    for (long long j0 = a; j0 < b; j0 += 32) {
+        const bool v = inside(j0 + lane);
+        k += __popc(__ballot_sync(0xffffffffu, v));
+        below += __popc(__ballot_sync(0xffffffffu, v && j0 + lane < i));
+    }
+    long long base = 0;
+    if (lane == 0) base = (long long)atomicAdd(reinterpret_cast<unsigned long long*>(&counters->n_pairs), (unsigned long long)k);
+    base = __shfl_sync(0xffffffffu, base, 0);
+    const bool fits = base + k <= pair_capacity;
+    if (lane == 0) {
+        pair_start[i] = base;
+        pair_count[i] = fits ? k : 0;
+        row_count[i] = k + 1;                     // the neighbours and the centre itself
+        self_row[i] = below;
+        if (!fits) atomicOr(&counters->status, kStatusPairCapacity);
+    }
+    if (!fits) return;
+    int at = 0;
+    for (long long j0 = a; j0 < b; j0 += 32) {
+        const long long j = j0 + lane;
+        const bool v = inside(j);
+        const unsigned m = __ballot_sync(0xffffffffu, v);
+        if (v) {
+            const int q = at + __popc(m & ((1u << lane) - 1));
+            pair_key[base + q] = ((unsigned long long)j << 24) | (128ull << 16) | (128ull << 8) | 128ull;
+            pair_row[base + q] = q + (j > i ? 1 : 0);        // rows in atom order, the centre's own among them
+        }
+        at += __popc(m);
+    }
+}
+
 // One block: exclusive scan of the row counts (rows of centre c start at row_ptr[c]) and the launch
 // order of the per-centre kernel, largest pair count first (bins of 4 pairs, counting sort), so that
 // the long CTAs do not end up alone at the tail of the launch.

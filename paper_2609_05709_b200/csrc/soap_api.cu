@@ -289,9 +289,22 @@ void scan_counts(soap_t* h, const int* counts, long long* out, int64_t C, long l
 
 // The whole neighbour search: cell list, sorted pair segments with their row bookkeeping, row
 // pointers (to `row_ptr_out`, the caller's array or the handle's) and the launch order.
+// With `batch` (struct_ptr [n_structs+1], device): many independent non-periodic structures in one list of atoms,
+// every atom a centre, neighbours only inside the own structure.
+struct Batch {
+    const long long* struct_ptr = nullptr;
+    int64_t n_structs = 0;
+};
+
 int launch_neighbors(soap_t* h, const float* pos, const int32_t* num, int64_t N, const Geometry& g,
-                     const int32_t* centers, const float* sites, int64_t C, long long* row_ptr_out, cudaStream_t st) {
-    if (N <= kSmallPrepAtoms) {
+                     const int32_t* centers, const float* sites, int64_t C, long long* row_ptr_out, cudaStream_t st,
+                     const Batch& batch = Batch()) {
+    if (batch.struct_ptr) {
+        CU(cudaMemsetAsync(&h->d_counters->n_pairs, 0, 2 * sizeof(long long), st));      // pair cursor and row total
+        if (N > 0) batch_pairs_kernel<<<(unsigned)((N + kFillWarps - 1) / kFillWarps), kFillWarps * 32, 0, st>>>(
+            pos, num, h->d_zlut, h->d_species_idx, batch.struct_ptr, batch.n_structs, N, g.rc2, h->cap_pairs, h->d_pair_key,
+            h->d_pair_row, h->d_pair_start, h->d_pair_count, h->d_row_count, h->d_self_row, h->d_counters);
+    } else if (N <= kSmallPrepAtoms) {
         small_prep_kernel<<<1, kPrepThreads, 0, st>>>(pos, num, N, g, h->d_zlut, h->d_species_idx, (int)h->cap_cells, h->d_grid,
                                                       h->d_atom_cell, h->d_atom_wrap, h->d_cell_count, h->d_cell_start,
                                                       h->d_s_pos, h->d_s_wrap, h->d_counters);
@@ -304,7 +317,7 @@ int launch_neighbors(soap_t* h, const float* pos, const int32_t* num, int64_t N,
         scan_kernel<int><<<1, 1024, 0, st>>>(h->d_cell_count, h->d_cell_start, h->cap_cells, nullptr, &h->d_grid->n_cells);
         bin_fill_kernel<<<blocks_for(N, 256), 256, 0, st>>>(pos, N, h->d_atom_cell, h->d_atom_wrap, h->d_cell_start, h->d_cell_count, h->d_s_pos, h->d_s_wrap);
     }
-    if (C > 0) pairs_kernel<<<(unsigned)((C + kFillWarps - 1) / kFillWarps), kFillWarps * 32, 0, st>>>(
+    if (C > 0 && !batch.struct_ptr) pairs_kernel<<<(unsigned)((C + kFillWarps - 1) / kFillWarps), kFillWarps * 32, 0, st>>>(
         pos, centers, sites, C, g, h->d_grid, h->d_atom_cell, h->d_atom_wrap, h->d_cell_start, h->d_s_pos, h->d_s_wrap,
         h->cap_pairs, h->d_pair_tmp, h->d_pair_key, h->d_pair_row, h->d_pair_start, h->d_pair_count, h->d_row_count,
         h->d_self_row, h->d_counters);
@@ -329,10 +342,10 @@ int check_inputs(soap_t* h, const float* pos, const int32_t* num, int64_t N, con
 // Plans scratch for a structure of this size: run the search (with whatever capacity there is;
 // the counts come out right even when the pairs do not fit), read the totals back, grow.
 int plan(soap_t* h, const float* pos, const int32_t* num, int64_t N, const Geometry& g,
-         const int32_t* centers, const float* sites, int64_t C, cudaStream_t st) {
+         const int32_t* centers, const float* sites, int64_t C, cudaStream_t st, const Batch& batch = Batch()) {
     int rc = ensure_scratch(h, N, C, 0);
     if (rc) return rc;
-    rc = launch_neighbors(h, pos, num, N, g, centers, sites, C, h->d_row_ptr, st);
+    rc = launch_neighbors(h, pos, num, N, g, centers, sites, C, h->d_row_ptr, st, batch);
     if (rc) return rc;
     CU(cudaMemcpyAsync(h->h_counters, h->d_counters, sizeof(Counters), cudaMemcpyDeviceToHost, st));
     CU(cudaStreamSynchronize(st));
@@ -345,8 +358,8 @@ int plan(soap_t* h, const float* pos, const int32_t* num, int64_t N, const Geome
     h->h_counters->status &= ~kStatusPairCapacity;
     CU(cudaMemcpyAsync(&h->d_counters->status, &h->h_counters->status, sizeof(int), cudaMemcpyHostToDevice, st));
     CU(cudaStreamSynchronize(st));
-    h->planned_atoms = N;
-    h->planned_centers = C;
+    h->planned_atoms = std::max<int64_t>(h->planned_atoms, N);
+    h->planned_centers = std::max<int64_t>(h->planned_centers, C);
     return SOAP_OK;
 }
 
@@ -391,16 +404,22 @@ void build_feature_table(soap_t* h) {
 // Everything before the per-centre kernel: argument checks, device set-up, planning when the sizes
 // changed, the neighbour search.
 int prepare(soap_t* h, const float* pos, const int32_t* num, int64_t N, const double* cell, const int32_t* centers,
-            int64_t C, long long* row_ptr_out, Geometry& g, cudaStream_t st, const float* sites = nullptr) {
+            int64_t C, long long* row_ptr_out, Geometry& g, cudaStream_t st, const float* sites = nullptr,
+            const Batch& batch = Batch()) {
     int rc = check_inputs(h, pos, num, N, centers, C, sites);
     if (rc) return rc;
+    if (batch.struct_ptr && (h->pbc[0] || h->pbc[1] || h->pbc[2]))
+        return fail(h, SOAP_ERR_INVALID_ARG, "batches of structures are for non-periodic structures");
     if ((rc = ensure_device(h))) return rc;
     if ((rc = make_geometry(h, cell, g))) return rc;
     if (h->profiling) CU(cudaEventRecord(h->ev[0], st));
-    if (h->planned_atoms != N || h->planned_centers != C) {
-        if ((rc = plan(h, pos, num, N, g, centers, sites, C, st))) return rc;
+    // plan (search once, read the totals, grow the scratch: allocates and waits) when this structure is larger
+    // than anything planned so far; smaller ones run in the scratch that is there, and if one of them turns out
+    // to have more pairs than that holds the status word says so
+    if (h->planned_atoms < 0 || N > h->planned_atoms || C > h->planned_centers) {
+        if ((rc = plan(h, pos, num, N, g, centers, sites, C, st, batch))) return rc;
     }
-    if ((rc = launch_neighbors(h, pos, num, N, g, centers, sites, C, row_ptr_out ? row_ptr_out : h->d_row_ptr, st))) return rc;
+    if ((rc = launch_neighbors(h, pos, num, N, g, centers, sites, C, row_ptr_out ? row_ptr_out : h->d_row_ptr, st, batch))) return rc;
     if (h->weight.fn && C > 0) {
         pair_weight_kernel<<<(unsigned)((C + 7) / 8), 256, 0, st>>>(pos, centers, sites, C, g, h->d_pair_start, h->d_pair_count, h->d_pair_key,
                                                                    h->cap_pairs, h->d_counters, h->weight, h->d_pair_w);
@@ -512,15 +531,17 @@ int soap_radial_table(const soap_t* h, double d, double* G, double* Ghat) {
 
 static int neighbors_impl(soap_t* h, const float* d_positions, const int32_t* d_numbers, int64_t n_atoms, const double* cell,
                           const int32_t* d_centers, const float* d_sites, int64_t n_centers, int64_t* n_pairs, int64_t* n_rows,
-                          void* stream) {
+                          void* stream, const Batch& batch = Batch()) {
     int rc = check_inputs(h, d_positions, d_numbers, n_atoms, d_centers, n_centers, d_sites);
     if (rc) return rc;
+    if (batch.struct_ptr && (h->pbc[0] || h->pbc[1] || h->pbc[2]))
+        return fail(h, SOAP_ERR_INVALID_ARG, "batches of structures are for non-periodic structures");
     if ((rc = ensure_device(h))) return rc;
     Geometry g;
     if ((rc = make_geometry(h, cell, g))) return rc;
     cudaStream_t st = (cudaStream_t)stream;
-    if ((rc = plan(h, d_positions, d_numbers, n_atoms, g, d_centers, d_sites, n_centers, st))) return rc;
-    if ((rc = launch_neighbors(h, d_positions, d_numbers, n_atoms, g, d_centers, d_sites, n_centers, h->d_row_ptr, st))) return rc;
+    if ((rc = plan(h, d_positions, d_numbers, n_atoms, g, d_centers, d_sites, n_centers, st, batch))) return rc;
+    if ((rc = launch_neighbors(h, d_positions, d_numbers, n_atoms, g, d_centers, d_sites, n_centers, h->d_row_ptr, st, batch))) return rc;
     CU(cudaMemcpyAsync(h->h_counters, h->d_counters, sizeof(Counters), cudaMemcpyDeviceToHost, st));
     CU(cudaStreamSynchronize(st));
     h->last_centers = n_centers;
@@ -555,11 +576,12 @@ int soap_neighbor_list(soap_t* h, int64_t* d_pair_ptr, int32_t* d_pair_atom, int
 }
 
 static int descriptor_impl(soap_t* h, const float* d_positions, const int32_t* d_numbers, int64_t n_atoms, const double* cell,
-                           const int32_t* d_centers, const float* d_sites, int64_t n_centers, float* d_out, void* stream) {
+                           const int32_t* d_centers, const float* d_sites, int64_t n_centers, float* d_out, void* stream,
+                           const Batch& batch = Batch()) {
     if (h && n_centers > 0 && !d_out) return fail(h, SOAP_ERR_INVALID_ARG, "d_out must not be NULL");
     Geometry g;
     cudaStream_t st = (cudaStream_t)stream;
-    int rc = prepare(h, d_positions, d_numbers, n_atoms, cell, d_centers, n_centers, nullptr, g, st, d_sites);
+    int rc = prepare(h, d_positions, d_numbers, n_atoms, cell, d_centers, n_centers, nullptr, g, st, d_sites, batch);
     if (rc) return rc;
     if (n_centers > 0) {
         CenterParams cp;
@@ -585,12 +607,12 @@ int soap_descriptor_at(soap_t* h, const float* d_positions, const int32_t* d_num
 static int derivatives_impl(soap_t* h, const float* d_positions, const int32_t* d_numbers, int64_t n_atoms, const double* cell,
                             const int32_t* d_centers, const float* d_sites, int64_t n_centers, float* d_out_desc, float* d_out_jac,
                             int64_t capacity_rows, int64_t* d_row_ptr, int32_t* d_row_atom, void* stream,
-                            float* d_out_center = nullptr) {
+                            float* d_out_center = nullptr, const Batch& batch = Batch()) {
     if (h && (!d_row_ptr || capacity_rows < 0)) return fail(h, SOAP_ERR_INVALID_ARG, "d_row_ptr must not be NULL");
     if (h && n_centers > 0 && (!d_out_desc || !d_out_jac || !d_row_atom)) return fail(h, SOAP_ERR_INVALID_ARG, "output pointers must not be NULL");
     Geometry g;
     cudaStream_t st = (cudaStream_t)stream;
-    int rc = prepare(h, d_positions, d_numbers, n_atoms, cell, d_centers, n_centers, (long long*)d_row_ptr, g, st, d_sites);
+    int rc = prepare(h, d_positions, d_numbers, n_atoms, cell, d_centers, n_centers, (long long*)d_row_ptr, g, st, d_sites, batch);
     if (rc) return rc;
     if (n_centers > 0) {
         CenterParams cp;
@@ -619,6 +641,49 @@ int soap_derivatives_at(soap_t* h, const float* d_positions, const int32_t* d_nu
     static const float none[3] = {0.f, 0.f, 0.f};
     return derivatives_impl(h, d_positions, d_numbers, n_atoms, cell, nullptr, d_sites ? d_sites : none, n_sites, d_out_desc,
                             d_out_jac, capacity_rows, d_row_ptr, d_row_atom, stream);
+}
+
+// ---- many independent structures in one call ----
+static int check_batch(soap_t* h, const int64_t* d_struct_ptr, int64_t n_structs, int64_t n_atoms) {
+    if (!h) return SOAP_ERR_INVALID_ARG;
+    if (n_structs < 0 || (n_atoms > 0 && n_structs < 1)) return fail(h, SOAP_ERR_INVALID_ARG, "n_structs must be at least 1 when there are atoms");
+    if (n_structs > 0 && !d_struct_ptr) return fail(h, SOAP_ERR_INVALID_ARG, "d_struct_ptr must not be NULL");
+    return SOAP_OK;
+}
+
+int soap_neighbors_batch(soap_t* h, const float* d_positions, const int32_t* d_numbers, int64_t n_atoms,
+                         const int64_t* d_struct_ptr, int64_t n_structs, int64_t* n_pairs, int64_t* n_rows, void* stream) {
+    int rc = check_batch(h, d_struct_ptr, n_structs, n_atoms);
+    if (rc) return rc;
+    static const long long none[2] = {0, 0};
+    Batch b;
+    b.struct_ptr = d_struct_ptr ? (const long long*)d_struct_ptr : none;
+    b.n_structs = n_structs;
+    return neighbors_impl(h, d_positions, d_numbers, n_atoms, nullptr, nullptr, nullptr, n_atoms, n_pairs, n_rows, stream, b);
+}
+
+int soap_descriptor_batch(soap_t* h, const float* d_positions, const int32_t* d_numbers, int64_t n_atoms,
+                          const int64_t* d_struct_ptr, int64_t n_structs, float* d_out, void* stream) {
+    int rc = check_batch(h, d_struct_ptr, n_structs, n_atoms);
+    if (rc) return rc;
+    static const long long none[2] = {0, 0};
+    Batch b;
+    b.struct_ptr = d_struct_ptr ? (const long long*)d_struct_ptr : none;
+    b.n_structs = n_structs;
+    return descriptor_impl(h, d_positions, d_numbers, n_atoms, nullptr, nullptr, nullptr, n_atoms, d_out, stream, b);
+}
+
+int soap_derivatives_batch(soap_t* h, const float* d_positions, const int32_t* d_numbers, int64_t n_atoms,
+                           const int64_t* d_struct_ptr, int64_t n_structs, float* d_out_desc, float* d_out_jac,
+                           int64_t capacity_rows, int64_t* d_row_ptr, int32_t* d_row_atom, void* stream) {
+    int rc = check_batch(h, d_struct_ptr, n_structs, n_atoms);
+    if (rc) return rc;
+    static const long long none[2] = {0, 0};
+    Batch b;
+    b.struct_ptr = d_struct_ptr ? (const long long*)d_struct_ptr : none;
+    b.n_structs = n_structs;
+    return derivatives_impl(h, d_positions, d_numbers, n_atoms, nullptr, nullptr, nullptr, n_atoms, d_out_desc, d_out_jac,
+                            capacity_rows, d_row_ptr, d_row_atom, stream, nullptr, b);
 }
 
 int soap_num_compact_features(const soap_t* h, int64_t* n_compact, int64_t* pitch) {

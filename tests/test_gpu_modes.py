@@ -379,3 +379,36 @@ def test_modes_at_full_size_sampled(pkg):
     want = (acc / 3000).cpu().numpy()
     assert col_err(jac.cpu().numpy(), want, (0, 1)) < 1e-5
     assert col_err(d.cpu().numpy()[None], plain.descriptor.double().mean(dim=0).cpu().numpy()[None], 0) < 1e-5
+
+
+# ----------------------------------------------------------------- many independent structures in one call
+@pytest.mark.parametrize("rbf", [GTO, POLYNOMIAL])
+def test_batch_of_structures(pkg, rbf):
+    rng = np.random.default_rng(21)
+    parts = []
+    for k, n_mol in enumerate([1, 8, 2, 5, 3, 12]):
+        s = water_cluster(n_mol, 40 + k)
+        parts.append((s.positions + rng.uniform(-3, 3, size=3).astype(np.float32), s.numbers))
+    parts.insert(2, (np.array([[0.3, 0.1, -0.2]], np.float32), np.array([8], np.int32)))        # a lone atom
+    parts.insert(4, (np.zeros((0, 3), np.float32), np.zeros(0, np.int32)))                      # an empty structure
+    args = ([1, 8], 4.5, 4, 3, 0.5, rbf)
+    soap, oracle = pkg.Soap(*args), SoapOracle(*args)
+    ref = modes.batch_derivatives(oracle, parts)
+    pos = torch.from_numpy(np.concatenate([p[0] for p in parts])).cuda()
+    num = torch.from_numpy(np.concatenate([p[1] for p in parts])).cuda()
+    ptr = torch.tensor(np.concatenate([[0], np.cumsum([len(p[1]) for p in parts])]), dtype=torch.int64).cuda()
+    out = soap.derivatives_batch(pos, num, ptr)
+    assert np.array_equal(out.row_ptr.cpu().numpy(), ref.row_ptr)
+    assert np.array_equal(out.row_atom.cpu().numpy(), ref.row_atom)
+    assert col_err(out.descriptor.cpu().numpy(), ref.descriptor, 0) < DESC_TOL
+    assert col_err(out.jacobian.cpu().numpy(), ref.jacobian, (0, 1)) < JAC_TOL
+    d = soap.derivatives_batch(pos, num, ptr, jacobian=False)
+    assert torch.equal(d, out.descriptor)
+    # each structure on its own through the ordinary entry point gives the same bits
+    lo = int(ptr[1])
+    single = soap.derivatives(pos[lo:int(ptr[2])].contiguous(), num[lo:int(ptr[2])].contiguous())
+    assert torch.equal(single.descriptor, out.descriptor[lo:int(ptr[2])])
+    # a periodic handle refuses batches
+    per = pkg.Soap([1, 8], 4.5, 2, 2, 0.5, GTO, (True, False, False))
+    with pytest.raises(pkg.SoapError, match="non-periodic"):
+        per.derivatives_batch(pos, num, ptr)

@@ -256,3 +256,16 @@ def test_site_jacobian_by_central_differences():
     dense = modes._dense(der, pos.shape[0])
     fd = _fd(lambda p: modes.site_derivatives(o, p, st.numbers, sites).descriptor, pos)
     np.testing.assert_allclose(dense, np.transpose(fd, (2, 0, 1, 3)), rtol=0, atol=3e-8 * np.abs(dense).max())
+
+
+# ----------------------------------------------------------------- many independent structures
+def test_batch_equals_one_structure_with_the_parts_far_apart():
+    a, b, c = water_cluster(2, seed=1), water_cluster(3, seed=2), water_cluster(1, seed=3)
+    o = SoapOracle([1, 8], 4.0, 2, 2, 0.5)
+    parts = [(s.positions.astype(np.float64), s.numbers) for s in (a, b, c)]
+    got = modes.batch_derivatives(o, parts)
+    merged = np.concatenate([parts[0][0], parts[1][0] + [100.0, 0, 0], parts[2][0] + [0, -200.0, 50.0]])
+    ref = o.derivatives(merged, np.concatenate([p[1] for p in parts]))
+    assert np.array_equal(got.row_ptr, ref.row_ptr) and np.array_equal(got.row_atom, ref.row_atom)
+    np.testing.assert_allclose(got.descriptor, ref.descriptor, rtol=1e-10, atol=1e-13)
+    np.testing.assert_allclose(got.jacobian, ref.jacobian, rtol=0, atol=1e-10 * np.abs(ref.jacobian).max())
