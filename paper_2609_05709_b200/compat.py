@@ -86,9 +86,52 @@ class SOAP:
         e = self._engine((False, False, False))
         return e.n_coefficients if self.average == "cc" else e.n_features
 
+    # ------------------------------------------------------------------ lists of structures
+    @staticmethod
+    def _is_list_of_systems(system):
+        if not isinstance(system, (list, tuple)) or len(system) == 0:
+            return False
+        first = system[0]
+        return hasattr(first, "positions") or (isinstance(first, (list, tuple)) and len(first) >= 2 and np.ndim(first[0]) == 2)
+
+    def _many(self, systems, derivatives):
+        """Non-periodic structures, every atom a centre, average 'off': one batch call for all of them."""
+        import torch
+        from .binding import Derivatives
+        parts = [self._unpack(s) for s in systems]
+        if self.average != "off" or any(any(p[3]) for p in parts):
+            return None
+        e = self._engine((False, False, False))
+        sizes = [p[0].shape[0] for p in parts]
+        pos = torch.cat([p[0] for p in parts]).contiguous()
+        num = torch.cat([p[1] for p in parts]).contiguous()
+        ptr = torch.tensor(np.concatenate([[0], np.cumsum(sizes)]), dtype=torch.int64, device=pos.device)
+        if not derivatives:
+            d = e.derivatives_batch(pos, num, ptr, jacobian=False)
+            return list(torch.split(d, sizes))
+        out = e.derivatives_batch(pos, num, ptr)
+        row_ptr = out.row_ptr
+        res, a = [], 0
+        for n in sizes:
+            r0, r1 = int(row_ptr[a]), int(row_ptr[a + n])
+            one = Derivatives(out.descriptor[a:a + n], out.jacobian[r0:r1], (row_ptr[a:a + n + 1] - r0).contiguous(),
+                              (out.row_atom[r0:r1] - a).contiguous())
+            res.append((e.jacobian_dense(one, n_atoms=n) if n else out.jacobian.new_zeros((0, 0, 3, e.n_features)), one.descriptor))
+            a += n
+        e.status()
+        return res
+
     # ------------------------------------------------------------------ descriptors
     def create(self, system, centers=None):
-        """(n_centres, n_features); one row, (1, n_features), for the inner and outer averages."""
+        """(n_centres, n_features); one row, (1, n_features), for the inner and outer averages.  A list of
+        structures gives a list of results (non-periodic structures with every atom a centre go through one
+        batch call)."""
+        if self._is_list_of_systems(system):
+            if centers is None:
+                many = self._many(system, False)
+                if many is not None:
+                    return many
+            return [self.create(s, None if centers is None else centers[k]) for k, s in enumerate(system)]
         pos, num, cell, pbc = self._unpack(system)
         e = self._engine(pbc)
         idx, sites = self._centers(centers, pos.device)
@@ -115,6 +158,12 @@ class SOAP:
         import torch
         if include is not None and exclude is not None:
             raise ValueError("give include or exclude, not both")
+        if self._is_list_of_systems(system):
+            many = self._many(system, True) if centers is None and include is None and exclude is None else None
+            if many is None:
+                many = [self.derivatives(s, None if centers is None else centers[k], include, exclude, True)
+                        for k, s in enumerate(system)]
+            return many if return_descriptor else [m[0] for m in many]
         pos, num, cell, pbc = self._unpack(system)
         n = pos.shape[0]
         e = self._engine(pbc)

@@ -93,3 +93,20 @@ def test_unsupported_arguments_are_refused(SOAP):
         SOAP(r_cut=4.0, n_max=2, l_max=2, species=[1], average="middle")
     with pytest.raises(ValueError):
         SOAP(r_cut=4.0, n_max=2, l_max=2, species=[1], device="cpu")
+
+
+def test_lists_of_structures_go_through_the_batch_path(SOAP):
+    structs = [water_cluster(n, 30 + n) for n in (2, 5, 1, 7)]
+    soap = SOAP(r_cut=4.5, n_max=3, l_max=3, sigma=0.5, species=[1, 8])
+    oracle = SoapOracle([1, 8], 4.5, 3, 3, 0.5, GTO)
+    descs = soap.create(structs)
+    both = soap.derivatives(structs)
+    assert len(descs) == len(both) == 4
+    for s, d, (jac, d2) in zip(structs, descs, both):
+        ref = oracle.derivatives(s.positions, s.numbers)
+        assert torch.equal(d, d2) and col_err(d.cpu().numpy(), ref.descriptor, 0) < DESC_TOL
+        assert jac.shape == (s.n_atoms, s.n_atoms, 3, oracle.n_features)
+        assert col_err(jac.cpu().numpy(), modes._dense(ref, s.n_atoms), (0, 1, 2)) < JAC_TOL
+    # with a selection the structures are taken one by one
+    sel = soap.derivatives(structs, include=[0, 1], return_descriptor=False)
+    assert sel[1].shape == (15, 2, 3, oracle.n_features) and torch.equal(sel[1], both[1][0][:, [0, 1]])
