@@ -94,6 +94,15 @@ def test_random_configuration(seed):
     d = soap.descriptor(pos, num, s.cell)
     soap.status()
     assert col_err(d.cpu().numpy(), ref.descriptor, 0) < DESC_TOL, tag
+    if seed % 5 == 4 and not any(s.pbc) and s.n_atoms >= 2:        # the structure cut in two, as a batch of two
+        cut = s.n_atoms // 2
+        parts = [(s.positions[:cut], s.numbers[:cut]), (s.positions[cut:], s.numbers[cut:])]
+        bref = modes.batch_derivatives(oracle, parts)
+        ptr = torch.tensor([0, cut, s.n_atoms], dtype=torch.int64, device="cuda")
+        b = soap.derivatives_batch(pos, num, ptr)
+        assert np.array_equal(b.row_atom.cpu().numpy(), bref.row_atom), tag
+        assert col_err(b.descriptor.cpu().numpy(), bref.descriptor, 0) < DESC_TOL, tag
+        assert col_err(b.jacobian.cpu().numpy(), bref.jacobian, (0, 1)) < JAC_TOL, tag
     which = seed % 4
     if which == 3:                                   # averaged descriptor and Jacobian
         mode = "inner" if seed % 8 == 3 else "outer"
