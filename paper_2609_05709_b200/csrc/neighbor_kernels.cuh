@@ -612,13 +612,17 @@ batch_pairs_kernel(const float* __restrict__ pos, const int* __restrict__ number
         if (s < 0) { atomicOr(&counters->status, kStatusUnknownSpecies); s = 0; }
         species_idx[i] = s;
     }
-    // the structure that holds atom i: last b with struct_ptr[b] <= i
-    long long lo = 0, hi = n_structs;
-    while (hi - lo > 1) {
-        const long long mid = (lo + hi) >> 1;
-        if (struct_ptr[mid] <= i) lo = mid; else hi = mid;
+    // the structure that holds atom i: last b with struct_ptr[b] <= i (no offsets: one structure, all atoms)
+    long long a = 0, b = N;
+    if (struct_ptr) {
+        long long lo = 0, hi = n_structs;
+        while (hi - lo > 1) {
+            const long long mid = (lo + hi) >> 1;
+            if (struct_ptr[mid] <= i) lo = mid; else hi = mid;
+        }
+        a = struct_ptr[lo];
+        b = min(struct_ptr[lo + 1], N);
     }
-    const long long a = struct_ptr[lo], b = min(struct_ptr[lo + 1], N);
     const double xi = pos[3 * i], yi = pos[3 * i + 1], zi = pos[3 * i + 2];
     auto inside = [&](long long j) {
         if (j >= b) return false;

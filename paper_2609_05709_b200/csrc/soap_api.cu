@@ -295,11 +295,15 @@ struct Batch {
     const long long* struct_ptr = nullptr;
     int64_t n_structs = 0;
 };
+// A single small non-periodic structure with every atom a centre takes the same brute-force pair kernel (one
+// launch instead of the two that build and walk a cell list).
+constexpr int64_t kBruteForceAtoms = 512;
 
 int launch_neighbors(soap_t* h, const float* pos, const int32_t* num, int64_t N, const Geometry& g,
                      const int32_t* centers, const float* sites, int64_t C, long long* row_ptr_out, cudaStream_t st,
                      const Batch& batch = Batch()) {
-    if (batch.struct_ptr) {
+    const bool brute = !batch.struct_ptr && !centers && !sites && N <= kBruteForceAtoms && !(g.pbc[0] | g.pbc[1] | g.pbc[2]);
+    if (batch.struct_ptr || brute) {
         CU(cudaMemsetAsync(&h->d_counters->n_pairs, 0, 2 * sizeof(long long), st));      // pair cursor and row total
         if (N > 0) batch_pairs_kernel<<<(unsigned)((N + kFillWarps - 1) / kFillWarps), kFillWarps * 32, 0, st>>>(
             pos, num, h->d_zlut, h->d_species_idx, batch.struct_ptr, batch.n_structs, N, g.rc2, h->cap_pairs, h->d_pair_key,
@@ -317,7 +321,7 @@ int launch_neighbors(soap_t* h, const float* pos, const int32_t* num, int64_t N,
         scan_kernel<int><<<1, 1024, 0, st>>>(h->d_cell_count, h->d_cell_start, h->cap_cells, nullptr, &h->d_grid->n_cells);
         bin_fill_kernel<<<blocks_for(N, 256), 256, 0, st>>>(pos, N, h->d_atom_cell, h->d_atom_wrap, h->d_cell_start, h->d_cell_count, h->d_s_pos, h->d_s_wrap);
     }
-    if (C > 0 && !batch.struct_ptr) pairs_kernel<<<(unsigned)((C + kFillWarps - 1) / kFillWarps), kFillWarps * 32, 0, st>>>(
+    if (C > 0 && !batch.struct_ptr && !brute) pairs_kernel<<<(unsigned)((C + kFillWarps - 1) / kFillWarps), kFillWarps * 32, 0, st>>>(
         pos, centers, sites, C, g, h->d_grid, h->d_atom_cell, h->d_atom_wrap, h->d_cell_start, h->d_s_pos, h->d_s_wrap,
         h->cap_pairs, h->d_pair_tmp, h->d_pair_key, h->d_pair_row, h->d_pair_start, h->d_pair_count, h->d_row_count,
         h->d_self_row, h->d_counters);
