@@ -42,11 +42,13 @@ METRIC = "SOAP atoms/s, descriptor + Jacobian"
 UNIT = "atoms/s"
 
 
-def kernels_per_step(n_atoms, n_centers):
-    """Kernel launches of one soap_derivatives call: the cell-list build (one launch up to 16384
-    atoms, five above), the pair kernel, the row scan with the launch order (one launch up to 65536
+def kernels_per_step(n_atoms, n_centers, periodic=False):
+    """Kernel launches of one soap_derivatives call over all atoms: the cell-list build (one launch up to
+    16384 atoms, five above; none for a non-periodic structure of up to 512 atoms, which takes the
+    brute-force pair kernel), the pair kernel, the row scan with the launch order (one launch up to 65536
     centres, three above) and the fused per-centre kernel."""
-    return (1 if n_atoms <= 16384 else 5) + 1 + (1 if n_centers <= 65536 else 3) + 1
+    build = 0 if (n_atoms <= 512 and not periodic) else (1 if n_atoms <= 16384 else 5)
+    return build + 1 + (1 if n_centers <= 65536 else 3) + 1
 
 
 # DRAM traffic of the fused kernel from the ncu capture in profiles/center_kernel_water300.md
@@ -295,7 +297,7 @@ def run_cuda(args):
         "clocks": clocks,
         "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                 "ms_per_step": e2e_total / e2e_steps if e2e_steps else None, "steps": e2e_steps},
-        "gpu_launches": kernels_per_step(C, C) * args.steps,
+        "gpu_launches": kernels_per_step(C, C, s.cell is not None) * args.steps,
         "roofline": {"bound": "hbm", "kernel": "center_kernel<true>", "achieved": achieved, "peak": peak, "unit": "GB/s",
                      "frac": achieved / peak, "peak_source": peak_src,
                      "traffic": alg_bytes * NCU_SMALL_TRAFFIC_BYTES / NCU_SMALL_ALGORITHMIC_BYTES,
