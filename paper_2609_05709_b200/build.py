@@ -13,7 +13,8 @@ LIB = os.path.join(HERE, "libsoap_b200.so")
 
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-O3", "-lineinfo", "-std=c++17",
               "--expt-relaxed-constexpr", "-Xcompiler", "-fPIC", "-Xptxas", "-v"]
-CUDA_UNITS = ["soap_api"] + [f"center_l{l}" for l in range(13)]
+# compiled in parallel, the longest first (compile time grows with l_max)
+CUDA_UNITS = [f"center_l{l}" for l in range(12, -1, -1)] + ["soap_api"]
 
 
 def _newer(target, sources):
