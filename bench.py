@@ -54,7 +54,7 @@ def kernels_per_step(n_atoms, n_centers, periodic=False):
 # DRAM traffic of the fused kernel from the ncu capture in profiles/center_kernel_water300.md
 # (dram__bytes_read.sum + dram__bytes_write.sum of one launch) and that launch's algorithmic bytes;
 # the full-size launch is scaled by its own algorithmic bytes (traffic is proportional to the rows written).
-NCU_SMALL_TRAFFIC_BYTES = 572.66e6 + 1.55e6
+NCU_SMALL_TRAFFIC_BYTES = 573.28e6 + 1.58e6
 NCU_SMALL_ALGORITHMIC_BYTES = 629088584
 
 
