@@ -477,6 +477,7 @@ __global__ void count_kernel(const float* __restrict__ pos, const int* __restric
 }
 
 constexpr int kFillSmemKeys = 512;       // per warp; longer rows are sorted through global memory
+constexpr int kFillSmemKeysSmall = 128;  // variant for structures with few pairs per centre: 4x less shared memory, more warps resident
 constexpr int kFillWarps = 4;
 
 // One warp per centre, one walk over the candidates: collect the pairs, reserve a segment of the
@@ -485,6 +486,7 @@ constexpr int kFillWarps = 4;
 // derive the Jacobian row bookkeeping (distinct atoms, the centre's own position among them).
 // When the segment does not fit the planned capacity only the counts are produced and the status
 // word says so; the caller plans again with the totals.
+template <int KEYS>
 __global__ void __launch_bounds__(kFillWarps * 32)
 pairs_kernel(const float* __restrict__ pos, const int* __restrict__ centers, const float* __restrict__ sites, long long C, Geometry geom,
              const GridParams* __restrict__ gp, const int* __restrict__ atom_cell, const int* __restrict__ atom_wrap,
@@ -492,8 +494,8 @@ pairs_kernel(const float* __restrict__ pos, const int* __restrict__ centers, con
              long long pair_capacity, unsigned long long* pair_tmp, unsigned long long* pair_key, int* __restrict__ pair_row,
              long long* __restrict__ pair_start, int* __restrict__ pair_count, int* __restrict__ row_count,
              int* __restrict__ self_row, Counters* counters) {
-    __shared__ unsigned long long s_raw[kFillWarps][kFillSmemKeys];
-    __shared__ unsigned long long s_sorted[kFillWarps][kFillSmemKeys];
+    __shared__ unsigned long long s_raw[kFillWarps][KEYS];
+    __shared__ unsigned long long s_sorted[kFillWarps][KEYS];
     const GridParams g = *gp;
     const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
     const long long c = blockIdx.x * (long long)kFillWarps + wid;
@@ -521,14 +523,14 @@ pairs_kernel(const float* __restrict__ pos, const int* __restrict__ centers, con
                        [&](bool valid, unsigned long long key) {
                            const unsigned m = __ballot_sync(0xffffffffu, valid);
                            const int at = k + __popc(m & ((1u << lane) - 1));
-                           if (valid && at < kFillSmemKeys) s_raw[wid][at] = key;
+                           if (valid && at < KEYS) s_raw[wid][at] = key;
                            k += __popc(m);
                        });
     long long base = 0;
     if (lane == 0) base = (long long)atomicAdd(reinterpret_cast<unsigned long long*>(&counters->n_pairs), (unsigned long long)k);
     base = __shfl_sync(0xffffffffu, base, 0);
     const bool fits = base + k <= pair_capacity;
-    const bool in_smem = k <= kFillSmemKeys;
+    const bool in_smem = k <= KEYS;
     if (lane == 0) { pair_start[c] = base; pair_count[c] = fits ? k : 0; }
     if (!fits) {
         if (lane == 0) {

@@ -93,6 +93,7 @@ struct soap_handle {
     size_t cap_work = 0;
     // plan
     int64_t planned_atoms = -1, planned_centers = -1;
+    int64_t pairs_per_center_hint = 0;   // average at the last plan (chooses the pair kernel variant)
     int64_t last_centers = 0;
     int P_desc = 16, P_deriv = 16;
     size_t smem_desc = 0, smem_deriv = 0;
@@ -321,10 +322,19 @@ int launch_neighbors(soap_t* h, const float* pos, const int32_t* num, int64_t N,
         scan_kernel<int><<<1, 1024, 0, st>>>(h->d_cell_count, h->d_cell_start, h->cap_cells, nullptr, &h->d_grid->n_cells);
         bin_fill_kernel<<<blocks_for(N, 256), 256, 0, st>>>(pos, N, h->d_atom_cell, h->d_atom_wrap, h->d_cell_start, h->d_cell_count, h->d_s_pos, h->d_s_wrap);
     }
-    if (C > 0 && !batch.struct_ptr && !brute) pairs_kernel<<<(unsigned)((C + kFillWarps - 1) / kFillWarps), kFillWarps * 32, 0, st>>>(
+    if (C > 0 && !batch.struct_ptr && !brute) {
+        // few pairs per centre at the last plan: the variant with the small on-chip key buffers (more warps resident)
+        if (h->pairs_per_center_hint > 0 && h->pairs_per_center_hint <= kFillSmemKeysSmall * 3 / 4)
+            pairs_kernel<kFillSmemKeysSmall><<<(unsigned)((C + kFillWarps - 1) / kFillWarps), kFillWarps * 32, 0, st>>>(
         pos, centers, sites, C, g, h->d_grid, h->d_atom_cell, h->d_atom_wrap, h->d_cell_start, h->d_s_pos, h->d_s_wrap,
         h->cap_pairs, h->d_pair_tmp, h->d_pair_key, h->d_pair_row, h->d_pair_start, h->d_pair_count, h->d_row_count,
         h->d_self_row, h->d_counters);
+        else
+            pairs_kernel<kFillSmemKeys><<<(unsigned)((C + kFillWarps - 1) / kFillWarps), kFillWarps * 32, 0, st>>>(
+        pos, centers, sites, C, g, h->d_grid, h->d_atom_cell, h->d_atom_wrap, h->d_cell_start, h->d_s_pos, h->d_s_wrap,
+        h->cap_pairs, h->d_pair_tmp, h->d_pair_key, h->d_pair_row, h->d_pair_start, h->d_pair_count, h->d_row_count,
+        h->d_self_row, h->d_counters);
+    }
     if (C <= kOrderMaxCenters) {
         rows_order_kernel<<<1, 1024, 0, st>>>(h->d_row_count, h->d_pair_count, C, row_ptr_out, h->d_order, h->d_counters);
     } else {
@@ -354,6 +364,7 @@ int plan(soap_t* h, const float* pos, const int32_t* num, int64_t N, const Geome
     CU(cudaMemcpyAsync(h->h_counters, h->d_counters, sizeof(Counters), cudaMemcpyDeviceToHost, st));
     CU(cudaStreamSynchronize(st));
     const int64_t pairs = h->h_counters->n_pairs;
+    h->pairs_per_center_hint = C > 0 ? (pairs + C - 1) / C : 0;
     if (pairs > h->cap_pairs) {
         rc = ensure_scratch(h, N, C, pairs + pairs / 4 + 1024);
         if (rc) return rc;
