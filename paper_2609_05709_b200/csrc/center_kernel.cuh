@@ -55,7 +55,8 @@ __device__ __constant__ float kc_dfact[16] = {0};    // [m] (2m-1)!!
 // Degree-5 table lookup: value and derivative with respect to the interval coordinate t.
 __device__ __forceinline__ void radial_lookup(const float* __restrict__ table, int qi, int n_ch, int ch, float t,
                                               float& v, float& dv) {
-    const float2* cf = reinterpret_cast<const float2*>(table + ((size_t)qi * n_ch + ch) * 6);
+    // 32-bit index arithmetic: the table has at most 4096 x 208 x 6 floats
+    const float2* cf = reinterpret_cast<const float2*>(table) + (unsigned)(qi * n_ch + ch) * 3u;
     const float2 a = __ldg(cf), b = __ldg(cf + 1), c = __ldg(cf + 2);
     v = c.y; dv = 0.f;
     dv = fmaf(dv, t, v); v = fmaf(v, t, c.x);
