@@ -202,6 +202,35 @@ def test_config5_descriptor_only_30k(pkg):
     assert [int(x) for x in (ptr[1:] - ptr[:-1]).cpu()] == [len(l) for l in lists]
 
 
+def test_jacobian_beyond_four_gigabytes_30k_atoms_sampled(pkg):
+    """Descriptor + Jacobian of 30,000 atoms: 1.4 million rows, 16 GB of output, so every offset into the
+    Jacobian passes 2^32 bytes; centres from the start, the middle and the very end against the oracle."""
+    s = water_cluster(10000, 0)
+    args = ([1, 8], 5.0, 8, 6, 0.5, GTO)
+    soap, oracle = pkg.Soap(*args), SoapOracle(*args)
+    pos, num = dev(s)
+    out = soap.derivatives(pos, num)
+    assert out.jacobian.numel() * 4 > 2 ** 33
+    sample = [0, 14999, 29990, 29999]
+    ref = oracle.derivatives(s.positions, s.numbers, None, sample)
+    row_ptr = out.row_ptr.cpu().numpy()
+    got = []
+    for b, a in enumerate(sample):
+        lo, hi = int(row_ptr[a]), int(row_ptr[a + 1])
+        assert np.array_equal(out.row_atom[lo:hi].cpu().numpy(), ref.row_atom[ref.row_ptr[b]:ref.row_ptr[b + 1]])
+        got.append(out.jacobian[lo:hi].cpu().numpy())
+    assert col_err(np.concatenate(got), ref.jacobian, (0, 1)) < JAC_TOL
+    assert col_err(out.descriptor[sample].cpu().numpy(), ref.descriptor, 0) < DESC_TOL
+    # translation sum rule on the last thousand centres (their rows sit at the end of the 16 GB)
+    lo, hi = int(row_ptr[29000]), int(row_ptr[30000])
+    seg = torch.repeat_interleave(torch.arange(1000, device="cuda"), out.row_ptr[29001:] - out.row_ptr[29000:-1])
+    sums = torch.zeros((1000, 3, soap.n_features), device="cuda", dtype=torch.float64)
+    sums.index_add_(0, seg, out.jacobian[lo:hi].double())
+    scale = out.jacobian[lo:hi].abs().amax(dim=(0, 1)).double().clamp_min(1e-8)
+    assert float((sums.abs().amax(dim=(0, 1)) / scale).max()) < 1e-4
+    del out
+
+
 def test_config5_descriptor_only_million_atoms_sampled(pkg):
     """The largest size of the scaling benchmark (1,000,002 atoms): every centre on the GPU, a handful of
     centres and their neighbour lists against the oracle, and whole-output properties."""
