@@ -21,6 +21,10 @@
  *  - `d_centers` lists the centre atoms (indices into the structure); NULL
  *    means every atom, in order (then n_centers must equal n_atoms; n_centers
  *    = 0 is an empty list and does nothing).
+ *  - A handle is not thread-safe and serves one stream at a time: its scratch
+ *    memory is reused by every call, so calls on one handle must be ordered
+ *    (same stream, or synchronised).  Use one handle per concurrent stream or
+ *    host thread; handles share nothing but read-only constant tables.
  *  - `stream` is a cudaStream_t passed as void* (NULL = default stream).  All
  *    calls enqueue work on it and return without waiting, except where noted.
  *  - Feature order: species pairs mu <= nu (species sorted by atomic number),
