@@ -303,6 +303,14 @@ int soap_derivatives_average(soap_t *h, int mode, const float *d_positions, cons
  * pair and row counts of the last call (either pointer may be NULL). */
 int soap_status(soap_t *h, int64_t *n_pairs, int64_t *n_rows, void *stream);
 
+/* Measurement aid (the paper has no counterpart): the FP32 multiply-add rate of
+ * the current device from a register-only loop (16 independent chains per
+ * thread, 8 CTAs of 256 threads per SM, about 20 ms), timed with CUDA events on
+ * `stream`; the call waits for it.  *tflops receives 2 x multiply-adds / time
+ * of the best of four repetitions, *milliseconds (may be NULL) that time.
+ * This is the denominator the descriptor-only build is measured against. */
+int soap_measure_fp32_peak(double *tflops, double *milliseconds, void *stream);
+
 /* Neighbour counts with NO allocation anywhere in the call (the paper has no
  * counterpart; this entry point exists for callers that must not allocate).
  * Some callers cannot call cudaMalloc, or anything that may: a host
@@ -324,7 +332,9 @@ int soap_status(soap_t *h, int64_t *n_pairs, int64_t *n_rows, void *stream);
  * routine, and enqueues its work on `stream` without waiting.  The first call
  * on a device also looks up the device address of the fixed array (once per
  * device, with that device current); make that first call outside any stream
- * capture.  All calls on one GPU share the one array, which keeps the last
+ * capture.  The looked-up address is cached per device and published
+ * atomically, so host threads may race on their first calls; it goes stale if
+ * the device is reset (cudaDeviceReset) while the library stays loaded.  All calls on one GPU share the one array, which keeps the last
  * call's contents (the call clears what must start at zero): two calls whose
  * work overlaps on the GPU - different streams, or different host threads on
  * different streams - race on it and give wrong counts.  Serialise them. */

@@ -6,7 +6,7 @@ device memory and streams.  There is no CPU fallback: if the shared library is
 missing, importing `Soap` raises.
 """
 from .binding import (GTO, POLYNOMIAL, Soap, SoapError, Derivatives, CompactDerivatives, library_path, load_library,
-                      neighbor_counts_static, EXPORTED_SYMBOLS)
+                      neighbor_counts_static, measure_fp32_peak, EXPORTED_SYMBOLS)
 
 __all__ = ["GTO", "POLYNOMIAL", "Soap", "SoapError", "Derivatives", "CompactDerivatives", "library_path", "load_library",
-           "neighbor_counts_static", "EXPORTED_SYMBOLS"]
+           "neighbor_counts_static", "measure_fp32_peak", "EXPORTED_SYMBOLS"]

@@ -20,6 +20,7 @@ EXPORTED_SYMBOLS = [
     "soap_neighbors_at", "soap_descriptor_at", "soap_derivatives_at",
     "soap_rows_dense", "soap_neighbors_batch", "soap_descriptor_batch", "soap_derivatives_batch",
     "soap_num_compact_features", "soap_compact_feature_map", "soap_derivatives_compact", "soap_compact_expand",
+    "soap_measure_fp32_peak",
 ]
 
 _ERRORS = {-1: "SOAP_ERR_INVALID_ARG", -2: "SOAP_ERR_UNKNOWN_SPECIES", -3: "SOAP_ERR_CAPACITY",
@@ -84,6 +85,7 @@ def load_library() -> C.CDLL:
     lib.soap_coefficient_derivatives.argtypes = common + [vp, vp, i64, vp, vp, vp]
     lib.soap_descriptor_average.argtypes = [vp, i32] + common[1:] + [vp, vp]
     lib.soap_derivatives_average.argtypes = [vp, i32] + common[1:] + [vp, vp, vp]
+    lib.soap_measure_fp32_peak.argtypes = [C.POINTER(C.c_double), C.POINTER(C.c_double), vp]
     lib.soap_profile.argtypes = [vp, i32]
     lib.soap_profile_read.argtypes = [vp, C.POINTER(C.c_float), C.POINTER(C.c_float)]
     for name in EXPORTED_SYMBOLS:
@@ -91,6 +93,17 @@ def load_library() -> C.CDLL:
             getattr(lib, name).restype = C.c_int
     _LIB = lib
     return lib
+
+
+def measure_fp32_peak():
+    """(TFLOP/s, ms) of the library's register-only FP32 multiply-add loop on the current device and stream."""
+    import torch
+    lib = load_library()
+    tf, ms = C.c_double(), C.c_double()
+    rc = lib.soap_measure_fp32_peak(C.byref(tf), C.byref(ms), C.c_void_p(torch.cuda.current_stream().cuda_stream))
+    if rc != 0:
+        raise SoapError(rc, "soap_measure_fp32_peak failed (is a CUDA device present?)")
+    return tf.value, ms.value
 
 
 def neighbor_counts_static(positions, r_cut, out=None):

@@ -12,9 +12,11 @@ INCLUDE = os.path.join(os.path.dirname(HERE), "include")
 LIB = os.path.join(HERE, "libsoap_b200.so")
 
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-O3", "-lineinfo", "-std=c++17",
-              "--expt-relaxed-constexpr", "-Xcompiler", "-fPIC", "-Xptxas", "-v"]
-# compiled in parallel, the longest first (compile time grows with l_max)
-CUDA_UNITS = [f"center_l{l}" for l in range(12, -1, -1)] + ["soap_api"]
+              "--expt-relaxed-constexpr", "-Xcompiler", "-fPIC", "-Xptxas", "-v", "-Xfatbin=-compress-all"]
+# compiled in parallel, the longest first (compile time grows with l_max): the per-centre kernels are compiled
+# once per l_max from one source each (-DSOAP_L=<l_max>)
+PER_L_SOURCES = ["center_kernels", "desc_kernels"]
+PLAIN_UNITS = ["soap_api", "peak_kernel"]
 
 
 def _newer(target, sources):
@@ -41,12 +43,19 @@ def build(force: bool = False, verbose: bool = False) -> str:
     obj = lambda name: os.path.join(CSRC, name + ".o")
     cmds = [["g++", "-O2", "-std=gnu++17", "-fPIC", "-ffp-contract=off", "-I", INCLUDE, "-I", CSRC,
              "-c", os.path.join(CSRC, "basis_host.cpp"), "-o", obj("basis_host")]]
-    for unit in CUDA_UNITS:
+    objects = []
+    for l in range(12, -1, -1):
+        for src in PER_L_SOURCES:
+            name = f"{src}_l{l}"
+            objects.append(name)
+            cmds.append([nvcc, *NVCC_FLAGS, f"-DSOAP_L={l}", "-I", INCLUDE, "-I", CSRC, "-c", os.path.join(CSRC, src + ".cu"), "-o", obj(name)])
+    for unit in PLAIN_UNITS:
+        objects.append(unit)
         cmds.append([nvcc, *NVCC_FLAGS, "-I", INCLUDE, "-I", CSRC, "-c", os.path.join(CSRC, unit + ".cu"), "-o", obj(unit)])
     log = []
     with ThreadPoolExecutor(max_workers=min(len(cmds), os.cpu_count() or 4)) as pool:
         list(pool.map(lambda c: _run(c, verbose, log), cmds))
-    _run([nvcc, "-shared", "-o", LIB, *[obj(u) for u in CUDA_UNITS], obj("basis_host"), "-lquadmath", "-cudart", "static"],
+    _run([nvcc, "-shared", "-o", LIB, *[obj(u) for u in objects], obj("basis_host"), "-lquadmath", "-cudart", "static"],
          verbose, log)
     if verbose:
         sys.stderr.write("\n".join(log))

@@ -23,7 +23,7 @@
 #include <cmath>
 #include <cstdio>
 
-#include "soap_errors.h"
+#include "soap.h"
 
 namespace soap {
 namespace {

@@ -1,6 +1,6 @@
-// The fused per-centre kernel: one CTA owns one centre atom and produces its
-// descriptor row (Eq. 4) and, in the derivative build, all of its Jacobian
-// rows (Eq. 5).  Nothing per pair ever goes to HBM: radial factors, solid
+// The fused per-centre derivative kernel: one CTA owns one centre atom and produces its
+// descriptor row (Eq. 4) and all of its Jacobian rows (Eq. 5).  (The descriptor-only
+// build has a kernel of its own, desc_kernel.cuh.)  Nothing per pair ever goes to HBM: radial factors, solid
 // harmonics and the precontracted U/V live in shared memory; the expansion
 // coefficients c^mu_nlm of the centre stay in shared memory for the CTA's life.
 //
@@ -26,22 +26,8 @@
 
 #include "soap_device.cuh"
 
-#ifndef SOAP_DEBUG_SKIP
-#define SOAP_DEBUG_SKIP 0
-#endif
-#ifndef SOAP_WINDOW_MASK
-#define SOAP_WINDOW_MASK 3             // 3: windows for n_ch % 4 == 0 (two passes); 1: also n_ch % 2 == 0 (four passes)
-#endif
-#ifndef SOAP_TRI_UNROLL
-#define SOAP_TRI_UNROLL 2              // sweeps of a same-species block in flight per warp
-#endif
-constexpr int kTriUnroll = SOAP_TRI_UNROLL;
-#ifndef SOAP_MIN_CTAS_DERIV
-#define SOAP_MIN_CTAS_DERIV 3          // resident CTAs per SM the derivative kernel is compiled for
-#endif
-#ifndef SOAP_MIN_CTAS_DESC
-#define SOAP_MIN_CTAS_DESC 6           // ... and the descriptor-only kernel (latency-bound: more warps help)
-#endif
+constexpr int kTriUnroll = 2;          // sweeps of a same-species block in flight per warp
+constexpr int kMinCtas = 3;            // resident CTAs per SM the kernel is compiled for
 
 namespace soap {
 
@@ -73,9 +59,7 @@ __device__ __forceinline__ void radial_lookup(const float* __restrict__ table, i
 //   dQ_l^m/dx = -x Q_{l-1}^{m+1},  dQ_l^m/dy = -y Q_{l-1}^{m+1},  dQ_l^m/dz = (l+m) Q_{l-1}^m.
 // Columns m and m+1 are advanced in lock step, so a step needs four registers; the rational
 // coefficients of the recurrences come from constant memory (all lanes use the same (l, m)).
-template <bool GRAD>
-__device__ __forceinline__ void harmonics_column(int L, int m, float x, float y, float z, float r2,
-                                                 float4* __restrict__ out4, float* __restrict__ out1) {
+__device__ __forceinline__ void harmonics_column(int L, int m, float x, float y, float z, float r2, float4* __restrict__ out4) {
     float cm = 1.f, sm = 0.f, cp = 0.f, sp = 0.f;               // (x+iy)^m and (x+iy)^(m-1)
     for (int t = 0; t < m; ++t) {
         cp = cm; sp = sm;
@@ -91,37 +75,31 @@ __device__ __forceinline__ void harmonics_column(int L, int m, float x, float y,
         const float2 nr = kc_norm[t];
         const float aq = nr.x * a1;
         const int lm0 = l * l + l;
-        if (!GRAD) {
-            out1[lm0 + m] = aq * cm;
-            if (m) out1[lm0 - m] = aq * sm;
-        } else {
-            const float qz = nr.y * a0;                         // a (l+m) Q_{l-1}^m  (a0 = 0 when l = m)
-            const float qx = nr.x * b0;                         // a Q_{l-1}^{m+1}
-            const float mq = fm * aq;
-            const float xq = x * qx, yq = y * qx;
-            out4[lm0 + m] = make_float4(aq * cm, mq * cp - xq * cm, -mq * sp - yq * cm, qz * cm);
-            if (m) out4[lm0 - m] = make_float4(aq * sm, mq * sp - xq * sm, mq * cp - yq * sm, qz * sm);
-        }
+        const float qz = nr.y * a0;                             // a (l+m) Q_{l-1}^m  (a0 = 0 when l = m)
+        const float qx = nr.x * b0;                             // a Q_{l-1}^{m+1}
+        const float mq = fm * aq;
+        const float xq = x * qx, yq = y * qx;
+        out4[lm0 + m] = make_float4(aq * cm, mq * cp - xq * cm, -mq * sp - yq * cm, qz * cm);
+        if (m) out4[lm0 - m] = make_float4(aq * sm, mq * sp - xq * sm, mq * cp - yq * sm, qz * sm);
         // advance both columns to l + 1
         const float4 st = kc_step[t];
         const float an = st.x * z * a1 - st.y * r2 * a0;
         a0 = a1; a1 = an;
-        if (GRAD) {
-            const float bn = (l == m) ? kc_dfact[m + 1] : st.z * z * b1 - st.w * r2 * b0;
-            b0 = b1; b1 = bn;
-        }
+        const float bn = (l == m) ? kc_dfact[m + 1] : st.z * z * b1 - st.w * r2 * b0;
+        b0 = b1; b1 = bn;
         t += l + 1;
     }
 }
 
-// KIND: 0 descriptor only, 1 descriptor and Jacobian, 2 coefficients c^mu_nlm and their Jacobian.
+// KIND: 1 descriptor and Jacobian, 2 coefficients c^mu_nlm and their Jacobian.
 // PLAIN: the default configuration (every species pair, atom centres, no weighting, full rows, own
 // coefficients); the options are then compile-time constants and their code drops out.
 template <int KIND, int L, int NMAX_T, bool PLAIN>
-__global__ void __launch_bounds__(kThreads, KIND ? SOAP_MIN_CTAS_DERIV : SOAP_MIN_CTAS_DESC)
+__global__ void __launch_bounds__(kThreads, kMinCtas)
 center_kernel(const CenterParams p) {
-    constexpr bool DERIV = KIND != 0, CC = KIND == 2;
-    const bool o_compact = !PLAIN && p.compact, o_cross = PLAIN || p.crossover, o_emit = !PLAIN && p.emit_coeff;
+    static_assert(KIND == 1 || KIND == 2, "descriptor-only builds run desc_kernel");
+    constexpr bool CC = KIND == 2;
+    const bool o_compact = !PLAIN && p.compact, o_cross = PLAIN || p.crossover;
     const float* const o_cbar = PLAIN ? nullptr : p.c_bar;
     const float* const o_sites = PLAIN ? nullptr : p.sites;
     const float2* const o_pw = PLAIN ? nullptr : p.pair_w;
@@ -129,14 +107,8 @@ center_kernel(const CenterParams p) {
     constexpr int L1 = L + 1, LM = L1 * L1, LMP = LM | 1;      // odd row stride: no shared-memory bank conflicts
     constexpr int NMAX_BOUND = NMAX_T ? NMAX_T : 16;
     // pass-1 ownership: W_LM warps cover the lm index, SLOTS such groups split the n index
-#ifndef SOAP_SLOT_DIV_DERIV
-#define SOAP_SLOT_DIV_DERIV 2
-#endif
-#ifndef SOAP_SLOT_DIV_DESC
-#define SOAP_SLOT_DIV_DESC 2
-#endif
     constexpr int W_LM = (LM + 31) / 32;
-    constexpr int SLOTS_FULL = kWarps / W_LM, SLOT_DIV = DERIV ? SOAP_SLOT_DIV_DERIV : SOAP_SLOT_DIV_DESC;
+    constexpr int SLOTS_FULL = kWarps / W_LM, SLOT_DIV = 2;
     constexpr int SLOTS = SLOTS_FULL / SLOT_DIV > 0 ? SLOTS_FULL / SLOT_DIV : 1;
     constexpr int NPT_RAW = (NMAX_BOUND + SLOTS - 1) / SLOTS;      // radial functions per thread ...
     constexpr int NPT = NPT_RAW < 8 ? NPT_RAW : 8;                // ... at most 8 at a time (register budget)
@@ -145,22 +117,20 @@ center_kernel(const CenterParams p) {
     const long long c_idx = p.order ? p.order[blockIdx.x] : blockIdx.x;
     // a failed neighbour build or an undersized output: write nothing
     if (p.counters->n_pairs > p.pair_capacity) return;
-    if (DERIV && p.row_ptr[p.n_centers] > p.row_capacity) {
+    if (p.row_ptr[p.n_centers] > p.row_capacity) {
         if (c_idx == 0 && tid == 0) atomicOr(&p.counters->status, kStatusRowCapacity);
         return;
     }
     const int S = p.S, NMAX = NMAX_T ? NMAX_T : p.n_max, NCH = NMAX * L1, NE = NMAX * LM;
     const int CT = S * NMAX * LMP, P = p.P, F = p.F;
-    const SmemLayout lay = make_layout(S, NMAX, L, P, DERIV, o_pw != nullptr);
+    const SmemLayout lay = make_layout(S, NMAX, L, P, true, o_pw != nullptr);
     float* c_t = smem + lay.c;                                             // [S][NMAX][LMP]
     float4* geo_d = reinterpret_cast<float4*>(smem + lay.geo);             // [GP] dx, dy, dz, r
     int4* geo_i = reinterpret_cast<int4*>(smem + lay.geo + 4 * kGeoPairs);   // [GP] interval, t bits, species|moving<<8, row word
     int* geo_j = reinterpret_cast<int*>(smem + lay.geo + 8 * kGeoPairs);     // [GP] neighbour atom
     float2* geo_w = reinterpret_cast<float2*>(smem + lay.geo + kGeoWords);   // [GP] (w, w'/d), only with a radial weighting
     float* D_t = smem + lay.D;                                             // [3][CT]    (pass 1 and the centre's row)
-    float* sS = smem + lay.sSD;                                            // [P][LMP]   values            (descriptor build)
-    float4* sSD4 = reinterpret_cast<float4*>(smem + lay.sSD);              // [P][LMP]   (S, dSx, dSy, dSz) (derivative build)
-    float* sG1 = smem + lay.sG;                                            // [P][NCH]   G
+    float4* sSD4 = reinterpret_cast<float4*>(smem + lay.sSD);              // [P][LMP]   (S, dSx, dSy, dSz)
     float2* sG2 = reinterpret_cast<float2*>(smem + lay.sG);                // [P][NCH]   (G, Ghat)
 
     const int ci = o_sites ? -1 : (p.centers ? p.centers[c_idx] : (int)c_idx);
@@ -168,17 +138,16 @@ center_kernel(const CenterParams p) {
     const float xi = pc[0], yi = pc[1], zi = pc[2];
     const int zi_species = o_sites ? 0 : p.species_idx[ci];
     const long long pair_base = p.pair_start[c_idx];
-    // descriptor of given mean coefficients (inner average): no pairs to visit
-    const int k_pairs = (!DERIV && o_cbar) ? 0 : p.pair_count[c_idx];
+    const int k_pairs = p.pair_count[c_idx];
     const bool periodic = p.geom.pbc[0] | p.geom.pbc[1] | p.geom.pbc[2];
 
-    for (int e = tid; e < CT * (DERIV ? 4 : 1); e += kThreads) {
+    for (int e = tid; e < CT * 4; e += kThreads) {
         if (e < CT) c_t[e] = 0.f; else D_t[e - CT] = 0.f;
     }
 
     // same-species blocks: feature index -> (n1 L1 + l) | (n2 L1 + l) << 8, rows n1 of (NMAX - n1) L1 entries
     unsigned short* tri_dec = reinterpret_cast<unsigned short*>(smem + lay.tri);
-    if (DERIV && !CC)
+    if (!CC)
         for (int e = tid; e < (NMAX * (NMAX + 1) / 2) * L1; e += kThreads) {
             int n1 = 0, r = e;
             while (r >= (NMAX - n1) * L1) { r -= (NMAX - n1) * L1; ++n1; }
@@ -257,35 +226,31 @@ center_kernel(const CenterParams p) {
     };
 
     // ---- radial factors and solid harmonics of the pairs g .. g + pc - 1 of the staged geometry ----
-    auto stage_chunk = [&](int g, int pc, auto grad_tag) {
-        constexpr bool GRAD = decltype(grad_tag)::value;
-        if (SOAP_DEBUG_SKIP & 16) return;
+    auto stage_chunk = [&](int g, int pc) {
         for (int pr = wid; pr < pc; pr += kWarps) {
             const int4 gi = geo_i[g + pr];
             const float t = __int_as_float(gi.y);
-            const float rinv_h = GRAD ? p.inv_h / geo_d[g + pr].w : 0.f;
+            const float rinv_h = p.inv_h / geo_d[g + pr].w;
             if (o_pw) {
                 // radial weighting: G -> w G, Ghat -> w Ghat + (w'/d) G
                 const float2 w = geo_w[g + pr];
                 for (int ch = lane; ch < NCH; ch += 32) {
                     float v, dv;
                     radial_lookup(p.table, gi.x, NCH, ch, t, v, dv);
-                    if (GRAD) sG2[pr * NCH + ch] = make_float2(v * w.x, fmaf(dv * rinv_h, w.x, v * w.y));
-                    else sG1[pr * NCH + ch] = v * w.x;
+                    sG2[pr * NCH + ch] = make_float2(v * w.x, fmaf(dv * rinv_h, w.x, v * w.y));
                 }
                 continue;
             }
             for (int ch = lane; ch < NCH; ch += 32) {
                 float v, dv;
                 radial_lookup(p.table, gi.x, NCH, ch, t, v, dv);
-                if (GRAD) sG2[pr * NCH + ch] = make_float2(v, dv * rinv_h);
-                else sG1[pr * NCH + ch] = v;
+                sG2[pr * NCH + ch] = make_float2(v, dv * rinv_h);
             }
         }
         if (lane < pc) {
             const float4 d = geo_d[g + lane];
             for (int m = wid; m <= L; m += kWarps)
-                harmonics_column<GRAD>(L, m, d.x, d.y, d.z, d.w * d.w, sSD4 + lane * LMP, sS + lane * LMP);
+                harmonics_column(L, m, d.x, d.y, d.z, d.w * d.w, sSD4 + lane * LMP);
         }
     };
 
@@ -311,29 +276,23 @@ center_kernel(const CenterParams p) {
                     if (n < NMAX) {
                         const int e = (cur * NMAX + n) * LMP + own_lm;
                         c_t[e] += ac[k];
-                        if (DERIV) { D_t[e] += ax[k]; D_t[CT + e] += ay[k]; D_t[2 * CT + e] += az[k]; }
+                        D_t[e] += ax[k]; D_t[CT + e] += ay[k]; D_t[2 * CT + e] += az[k];
                     }
                     ac[k] = ax[k] = ay[k] = az[k] = 0.f;
                 }
             };
             for (int q0 = 0; q0 < gc; q0 += P) {
                 const int pc = min(P, gc - q0);
-                stage_chunk(q0, pc, std::integral_constant<bool, DERIV>{});
+                stage_chunk(q0, pc);
                 __syncthreads();
-                if (owner && !(SOAP_DEBUG_SKIP & 4)) {
+                if (owner) {
                     for (int s = 0; s < S; ++s) {
                         const int a = max(seg[s], q0), b = min(seg[s + 1], q0 + pc);
                         if (a >= b) continue;
                         if (s != cur) { flush(); cur = s; }
                         for (int g = a; g < b; ++g) {
                             const int pr = g - q0;
-                            if (!DERIV) {
-                                const float h = sS[pr * LMP + own_lm];
-                                const float* gp = sG1 + pr * NCH + (n0 + own_slot) * L1 + own_l;
-#pragma unroll
-                                for (int k = 0; k < NPT; ++k)
-                                    if (n0 + own_slot + k * SLOTS < NMAX) ac[k] = fmaf(gp[k * SLOTS * L1], h, ac[k]);
-                            } else {
+                            {
                                 const float4 h = sSD4[pr * LMP + own_lm];
                                 const float4 d = geo_d[g];
                                 // an image of the centre does not move relative to it: no contribution to D
@@ -373,14 +332,13 @@ center_kernel(const CenterParams p) {
         }
         __syncthreads();
     }
-    if ((!DERIV && o_emit) || CC) {
+    if (CC) {
         // coefficient mode: the tile itself is the result, index (mu n_max + n) (l_max+1)^2 + l^2 + l + m
         float* crow = p.out_desc + (size_t)c_idx * W;
         for (int e = tid; e < W; e += kThreads) {
             const int row = e / LM;
             crow[e] = c_t[row * LMP + (e - row * LM)];
         }
-        if (!DERIV) return;
     }
 
     // ============ power spectrum (Eq. 4) and the centre's own row ============
@@ -388,8 +346,8 @@ center_kernel(const CenterParams p) {
     // centre's row is minus the sum over its neighbours: -K_l sum_m (D^mu c^nu + c^mu D^nu).  Results
     // pass through the (now idle) staging area in slabs, so that global memory is written in
     // feature order, whole sectors at a time.
-    const long long row_base = DERIV ? p.row_ptr[c_idx] : 0;
-    const bool has_own = DERIV && !o_sites;          // a centre that is no atom has no row of its own
+    const long long row_base = p.row_ptr[c_idx];
+    const bool has_own = !o_sites;                   // a centre that is no atom has no row of its own
     if (CC) {
         // the centre's own row: minus the sum over the atoms that move relative to it
         if (has_own) {
@@ -414,48 +372,12 @@ center_kernel(const CenterParams p) {
             for (int e = tid; e < 3 * RW; e += kThreads) slot[e] = 0.f;
         }
         float* slab = smem + lay.sSD;
-        constexpr int NV = DERIV ? 4 : 1;                                   // values per feature
+        constexpr int NV = 4;                                               // values per feature: p and the three components of the centre's row
         const int NP = F / L1;                                              // (species pair, n, n') groups
         int gp = ((lay.total - lay.sSD) / NV) / L1;                         // groups per slab
         gp = gp < 1 ? 1 : (gp > NP ? NP : gp);
-        const bool staged = (lay.total - lay.sSD) >= NV * L1 && !(SOAP_DEBUG_SKIP & 8);
-        // Descriptor-only build, whole row fits the staging area: a thread takes one (species pair, l, n)
-        // and all n' at once, so each coefficient of the n side is loaded once per m for the whole
-        // group (the generic loop below loads two operands per multiply-add).
-        const bool grouped = !DERIV && (lay.total - lay.sSD) >= F && !(SOAP_DEBUG_SKIP & 8);
-        if (grouped) {
-            const int NB = o_cross ? S * (S + 1) / 2 : S;
-            for (int it = tid; it < NB * L1 * NMAX; it += kThreads) {
-                const int n1 = it % NMAX, rest = it / NMAX, b = rest % NB, l = rest / NB;   // l slowest: warps share 2l+1
-                int mu = 0, nu = 0, boff = 0;                                                // block b -> (mu, nu), feature offset
-                for (int k = 0, a2 = 0; a2 < S; ++a2)
-                    for (int b2 = a2; b2 < (o_cross ? S : a2 + 1); ++b2, ++k) {
-                        if (k == b) { mu = a2; nu = b2; }
-                        if (k < b) boff += (a2 == b2) ? (NMAX * (NMAX + 1) / 2) * L1 : NMAX * NCH;
-                    }
-                const int n2_lo = (mu == nu) ? n1 : 0;
-                const float* ar = c_t + (mu * NMAX + n1) * LMP + l * l;
-                const float* br = c_t + nu * NMAX * LMP + l * l;
-                float acc[NMAX_BOUND];
-#pragma unroll
-                for (int n2 = 0; n2 < NMAX_BOUND; ++n2) acc[n2] = 0.f;
-                for (int m = 0; m <= 2 * l; ++m) {
-                    const float ca = ar[m];
-#pragma unroll
-                    for (int n2 = 0; n2 < NMAX_BOUND; ++n2)
-                        if (n2 < NMAX && n2 >= n2_lo) acc[n2] = fmaf(ca, br[n2 * LMP + m], acc[n2]);
-                }
-                const float kl = __ldg(p.kl + l);
-                const int base = (mu == nu) ? boff + (n1 * NMAX - n1 * (n1 + 1) / 2) * L1 + l : boff + n1 * NCH + l;
-#pragma unroll
-                for (int n2 = 0; n2 < NMAX_BOUND; ++n2)
-                    if (n2 < NMAX && n2 >= n2_lo) slab[base + n2 * L1] = kl * acc[n2];
-            }
-            __syncthreads();
-            if (write_desc)
-                for (int e = tid; e < F; e += kThreads) desc_row[e] = slab[e];
-        }
-        for (int q0 = 0; q0 < ((SOAP_DEBUG_SKIP & 8) || grouped ? 0 : NP); q0 += gp) {
+        const bool staged = (lay.total - lay.sSD) >= NV * L1;
+        for (int q0 = 0; q0 < NP; q0 += gp) {
             const int nq = min(gp, NP - q0), nf = nq * L1, f0 = q0 * L1;
             for (int g = tid; g < nf; g += kThreads) {
                 const int l = g / nq, fl = (g - l * nq) * L1 + l;             // feature index inside the slab
@@ -467,15 +389,13 @@ center_kernel(const CenterParams p) {
                 for (int m = 0; m <= 2 * l; ++m) {
                     const float ca = c_t[ia + m], cb = c_t[ib + m];
                     acc = fmaf(ca, cb, acc);
-                    if (DERIV) {
-                        ax = fmaf(D_t[ia + m], cb, fmaf(ca, D_t[ib + m], ax));
-                        ay = fmaf(D_t[CT + ia + m], cb, fmaf(ca, D_t[CT + ib + m], ay));
-                        az = fmaf(D_t[2 * CT + ia + m], cb, fmaf(ca, D_t[2 * CT + ib + m], az));
-                    }
+                    ax = fmaf(D_t[ia + m], cb, fmaf(ca, D_t[ib + m], ax));
+                    ay = fmaf(D_t[CT + ia + m], cb, fmaf(ca, D_t[CT + ib + m], ay));
+                    az = fmaf(D_t[2 * CT + ia + m], cb, fmaf(ca, D_t[2 * CT + ib + m], az));
                 }
                 if (staged) {
                     slab[fl] = kl * acc;
-                    if (DERIV) { slab[nf + fl] = -kl * ax; slab[2 * nf + fl] = -kl * ay; slab[3 * nf + fl] = -kl * az; }
+                    slab[nf + fl] = -kl * ax; slab[2 * nf + fl] = -kl * ay; slab[3 * nf + fl] = -kl * az;
                 } else {
                     if (write_desc) desc_row[f0 + fl] = kl * acc;
                     if (has_own) { own[f0 + fl] = -kl * ax; own[(size_t)F + f0 + fl] = -kl * ay; own[(size_t)2 * F + f0 + fl] = -kl * az; }
@@ -496,7 +416,6 @@ center_kernel(const CenterParams p) {
         }
         if (has_own && tid == 0) p.row_atom[row_base + p.self_row[c_idx]] = ci;
     }
-    if (!DERIV) return;
     __syncthreads();
     // fold K_l into c for pass 2
     if (!CC)
@@ -528,8 +447,6 @@ center_kernel(const CenterParams p) {
         // where the row allows it (a warp store that straddles two lines costs two L1 wavefronts)
         const int a_line = (int)((reinterpret_cast<size_t>(out) >> 2) & 31);
         auto put = [&](int f, float vx, float vy, float vz) {
-            if (SOAP_DEBUG_SKIP & 128) vx = vy = vz = 1.f;
-            if ((SOAP_DEBUG_SKIP & 2048) && vx == vx) return;      // keep the arithmetic, drop the stores
             if (ACC) { out[f] += vx; out[PS + f] += vy; out[PS2 + f] += vz; }
             else { out[f] = vx; out[PS + f] = vy; out[PS2 + f] = vz; }
         };
@@ -538,9 +455,6 @@ center_kernel(const CenterParams p) {
             for (int nu = mu; nu < (o_cross ? S : mu + 1); ++nu) {
                 const int hi = lo + ((mu == nu) ? (NMAX * (NMAX + 1) / 2) * L1 : NMAX * NCH);
                 const int first = ((lo + a_line) & ~31) - a_line;
-                if ((SOAP_DEBUG_SKIP & 256) && mu != Z && nu != Z) { lo = hi; continue; }
-                if ((SOAP_DEBUG_SKIP & 32) && mu == nu && mu == Z) { lo = hi; continue; }
-                if ((SOAP_DEBUG_SKIP & 64) && mu != nu && (mu == Z || nu == Z)) { lo = hi; continue; }
                 if (mu != Z && nu != Z) {
                     if (o_compact) continue;                  // compact rows hold only the blocks that involve Z
                     if (!ACC)
@@ -581,17 +495,13 @@ center_kernel(const CenterParams p) {
                         if (f < lo) continue;
                         const unsigned dec = tri_dec[f - lo];                 // (n1 L1 + l) | (n2 L1 + l) << 8
                         const int iA = dec & 255, iB = dec >> 8;
-                        float2 g1 = wG[iA], g2 = wG[iB];
-                        float4 u1 = UVz[iA], u2 = UVz[iB];
-                        if (SOAP_DEBUG_SKIP & 1024) {                        // no operand loads: values from the indices
-                            g1 = make_float2((float)iA, d.x); g2 = make_float2((float)iB, d.y);
-                            u1 = make_float4(d.x, d.y, d.z, (float)iA); u2 = make_float4(d.z, d.x, (float)iB, d.y);
-                        }
+                        const float2 g1 = wG[iA], g2 = wG[iB];
+                        const float4 u1 = UVz[iA], u2 = UVz[iB];
                         const float t = fmaf(g1.y, u2.x, g2.y * u1.x);      // Ghat_n1 U_n2 + Ghat_n2 U_n1
                         put(f, fmaf(g1.x, u2.y, fmaf(g2.x, u1.y, t * d.x)), fmaf(g1.x, u2.z, fmaf(g2.x, u1.z, t * d.y)),
                             fmaf(g1.x, u2.w, fmaf(g2.x, u1.w, t * d.z)));
                     }
-                } else if ((NCH & 7) == 0 || (NMAX_T > 8 && (NCH & (SOAP_WINDOW_MASK)) == 0) || (NMAX_T != 0 && NMAX_T <= 8)) {
+                } else if ((NCH & 7) == 0 || (NMAX_T > 8 && (NCH & 3) == 0) || (NMAX_T != 0 && NMAX_T <= 8)) {
                     // Cross-species block: rows n1 of n_ch floats follow each other.  A lane keeps one position i of
                     // a window of about n_ch floats, so its (n2, l) is fixed and the operand that depends on (n2, l)
                     // stays in registers over the unrolled n1 loop.
@@ -607,7 +517,7 @@ center_kernel(const CenterParams p) {
                     //    14 %; from n_max = 10 on it loses (up to 24 %), so those keep the aligned sweeps below.
                     const bool first_term = (mu == Z);
                     const float4* UVo = wUV + (first_term ? nu : mu) * NCH;
-                    const int T = (NCH & 7) == 0 ? 1 : ((NMAX_T > 8 && (NCH & 3) == 0) ? 2 : ((NMAX_T > 8 && (NCH & (SOAP_WINDOW_MASK)) == 0) ? 4 : 0));
+                    const int T = (NCH & 7) == 0 ? 1 : ((NMAX_T > 8 && (NCH & 3) == 0) ? 2 : ((NMAX_T > 8 && (NCH & 3) == 0) ? 4 : 0));
                     const int TT = T ? T : 1;
 #pragma unroll
                     for (int pp = 0; pp < 4; ++pp) {
@@ -633,7 +543,7 @@ center_kernel(const CenterParams p) {
                                         const float2 g = gp[n1 * L1];
                                         const float vx = fmaf(g.x, u.y, g.y * xx), vy = fmaf(g.x, u.z, g.y * xy), vz = fmaf(g.x, u.w, g.y * xz);
                                         if (ACC) { o[n1 * NCH] += vx; o[PS + n1 * NCH] += vy; o[PS2 + n1 * NCH] += vz; }
-                                        else if (!((SOAP_DEBUG_SKIP & 2048) && vx == vx)) { o[n1 * NCH] = vx; o[PS + n1 * NCH] = vy; o[PS2 + n1 * NCH] = vz; }
+                                        else { o[n1 * NCH] = vx; o[PS + n1 * NCH] = vy; o[PS2 + n1 * NCH] = vz; }
                                     }
                                 }
                             } else {
@@ -648,7 +558,7 @@ center_kernel(const CenterParams p) {
                                         const float4 u = up[n1 * L1];
                                         const float vx = fmaf(g.x, u.y, gx * u.x), vy = fmaf(g.x, u.z, gy * u.x), vz = fmaf(g.x, u.w, gz * u.x);
                                         if (ACC) { o[n1 * NCH] += vx; o[PS + n1 * NCH] += vy; o[PS2 + n1 * NCH] += vz; }
-                                        else if (!((SOAP_DEBUG_SKIP & 2048) && vx == vx)) { o[n1 * NCH] = vx; o[PS + n1 * NCH] = vy; o[PS2 + n1 * NCH] = vz; }
+                                        else { o[n1 * NCH] = vx; o[PS + n1 * NCH] = vy; o[PS2 + n1 * NCH] = vz; }
                                     }
                                 }
                             }
@@ -717,7 +627,7 @@ center_kernel(const CenterParams p) {
         const float4* wSD = sSD4 + pr * LMP;
         __syncwarp();
         // ---- U, V for every (nu, n', l) ----
-        if (CC || (SOAP_DEBUG_SKIP & 2)) {
+        if (CC) {
         } else if (SN <= 16) {
             // lane <-> (nu n', half): half 0 accumulates (U, Vx), half 1 (Vy, Vz)
             const int sn = lane >> 1, half = lane & 1;
@@ -755,7 +665,6 @@ center_kernel(const CenterParams p) {
             }
         }
         __syncwarp();
-        if (SOAP_DEBUG_SKIP & 1) return;
         float* out = p.out_jac + (size_t)(row_base + row) * 3 * RW;
         if (rw & kRowContinuation) {
             if (CC) coeff_rule(std::true_type{}, Z, d, wG, wSD, out);
@@ -773,7 +682,7 @@ center_kernel(const CenterParams p) {
         if (g0 > 0 || k_pairs > kGeoPairs) special = stage_geometry(g0, gc);     // otherwise still valid from pass 1
         for (int q0 = 0; q0 < gc; q0 += P) {
             const int pc = min(P, gc - q0);
-            stage_chunk(q0, pc, std::true_type{});
+            stage_chunk(q0, pc);
             __syncthreads();
             if (!special) {
                 // every pair has a row of its own: deal them out round-robin

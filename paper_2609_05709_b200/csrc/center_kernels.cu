@@ -1,4 +1,8 @@
-// Included by center_l*.cu with SOAP_L defined: every instantiation for one l_max.
+// Every instantiation of the fused per-centre derivative kernels for one l_max: compiled once per value of
+// SOAP_L (0..12), which the build passes on the command line.
+#ifndef SOAP_L
+#error "compile with -DSOAP_L=<l_max>"
+#endif
 #include "center_kernel.cuh"
 #include "center_launch.h"
 
@@ -40,13 +44,25 @@ cudaError_t SOAP_CAT(center_constants_l, SOAP_L)(const float* anorm91, const flo
     return cudaMemcpyToSymbol(kc_dfact, dfact16, 16 * sizeof(float));
 }
 
-// The plain kernels have their own instantiation for every n_max up to 12 (loops over n unroll, the
-// accumulators of pass 1 fit the registers exactly; the variant that reads n_max at run time is 1.5 to 2
-// times slower); the options run through general kernels: Jacobian builds instantiated for the n_max listed
-// below, everything else through the run-time variant or the one for n_max = 8.
-#define SOAP_FOR_FIXED_NMAX(X) X(1) X(2) X(3) X(4) X(5) X(6) X(7) X(8) X(9) X(10) X(11) X(12)
-// n_max values for which the general kernels (the ones that honour the options) are instantiated too
-#define SOAP_FOR_GENERAL_NMAX(X) X(2) X(4) X(6) X(7) X(8) X(10) X(12)
+// The plain kernels have their own instantiation for the usual n_max (loops over n unroll, the accumulators of
+// pass 1 fit the registers exactly; the variant that reads n_max at run time is 1.4 to 2 times slower and
+// serves every other n_max); the kernels that honour the options are instantiated for fewer n_max still.
+// Even l_max and l_max = 3 get the long lists, the other odd l_max the short ones.
+#if (SOAP_L % 2 == 0) || (SOAP_L == 3)
+#define SOAP_FOR_FIXED_NMAX(X) X(2) X(4) X(6) X(7) X(8) X(10) X(12)
+#define SOAP_FOR_GENERAL_NMAX(X) X(4) X(8)
+#else
+#define SOAP_FOR_FIXED_NMAX(X) X(4) X(8)
+#define SOAP_FOR_GENERAL_NMAX(X) X(8)
+#endif
+static bool center_has_fixed_nmax(int n_max) {
+    switch (n_max) {
+#define X(N) case N: return true;
+        SOAP_FOR_FIXED_NMAX(X)
+#undef X
+    }
+    return false;
+}
 static bool general_has_fixed_nmax(int n_max) {
     switch (n_max) {
 #define X(N) case N: return true;
@@ -66,22 +82,6 @@ cudaError_t SOAP_CAT(center_set_smem_l, SOAP_L)(int kind, int n_max, int bytes) 
 #undef X
         }
         return cudaSuccess;
-    }
-    if (kind == kCenterDesc) {
-        if ((e = set_one<0, 0, false>(bytes)) != cudaSuccess) return e;
-        switch (general_has_fixed_nmax(n_max) ? n_max : 0) {
-#define X(N) case N: e = set_one<0, N, false>(bytes); break;
-            SOAP_FOR_GENERAL_NMAX(X)
-#undef X
-            default: e = cudaSuccess;
-        }
-        if (e != cudaSuccess) return e;
-        switch (center_has_fixed_nmax(n_max) ? n_max : 0) {
-#define X(N) case N: return set_one<0, N, true>(bytes);
-            SOAP_FOR_FIXED_NMAX(X)
-#undef X
-            default: return set_one<0, 0, true>(bytes);
-        }
     }
     if ((e = set_one<1, 0, false>(bytes)) != cudaSuccess) return e;
     switch (general_has_fixed_nmax(n_max) ? n_max : 0) {
@@ -107,22 +107,6 @@ cudaError_t SOAP_CAT(center_launch_l, SOAP_L)(int kind, int n_max, bool plain, c
             SOAP_FOR_GENERAL_NMAX(X)
 #undef X
             default: return launch_one<2, 0, false>(p, grid, smem, st);
-        }
-    }
-    if (kind == kCenterDesc) {
-        if (!plain) {
-            switch (general_has_fixed_nmax(n_max) ? n_max : 0) {
-#define X(N) case N: return launch_one<0, N, false>(p, grid, smem, st);
-                SOAP_FOR_GENERAL_NMAX(X)
-#undef X
-                default: return launch_one<0, 0, false>(p, grid, smem, st);
-            }
-        }
-        switch (center_has_fixed_nmax(n_max) ? n_max : 0) {
-#define X(N) case N: return launch_one<0, N, true>(p, grid, smem, st);
-            SOAP_FOR_FIXED_NMAX(X)
-#undef X
-            default: return launch_one<0, 0, true>(p, grid, smem, st);
         }
     }
     if (!plain) {

@@ -3,16 +3,13 @@
 #include "soap_device.cuh"
 
 namespace soap {
-// kernel kinds: descriptor only; descriptor and Jacobian; coefficients c^mu_nlm and their Jacobian
-constexpr int kCenterDesc = 0, kCenterDeriv = 1, kCenterCoeff = 2;
+// kernel kinds: descriptor and Jacobian; coefficients c^mu_nlm and their Jacobian
+constexpr int kCenterDeriv = 1, kCenterCoeff = 2;
 // whether the parameters ask for nothing beyond the default configuration (the kernels instantiated with
 // PLAIN = true assume exactly this)
 inline bool center_params_plain(const CenterParams& p) {
     return p.crossover && !p.compact && !p.emit_coeff && !p.c_bar && !p.sites && !p.pair_w && p.w0 == 1.f;
 }
-// n_max values with their own instantiation of the plain kernels; larger ones run the variant that reads
-// n_max at run time.
-inline bool center_has_fixed_nmax(int n_max) { return n_max >= 1 && n_max <= 12; }
 // harmonic tables up to l = 12: anorm[91] (index l(l+1)/2 + m), dfact[16]
 cudaError_t center_constants(int l_max, const float* anorm91, const float* dfact16);
 cudaError_t center_set_smem(int kind, int l_max, int n_max, int bytes);

@@ -1,0 +1,411 @@
+// The descriptor-only kernel: expansion coefficients (Eq. 13 / Eqs. 18-19) and the power spectrum
+// (Eq. 4) of every centre, one WARP per centre, persistent CTAs that draw centres from a counter.
+//
+// This build is bound by FP32 arithmetic and by shared-memory bandwidth, not by HBM, so the layout is
+// chosen for few instructions and few shared-memory wavefronts per pair:
+//   * the radial table (value polynomials, re-laid as [interval][l][n][6]) sits in shared memory once
+//     per CTA when it fits, so that a lookup is three conflict-free 8-byte loads per lane;
+//   * pairs are taken species by species through a small ring (the pair list is re-read once per
+//     species), staged 16 at a time: solid harmonics with a lane per pair from the fully unrolled
+//     Q_l^m recursion, radial factors with lanes on the channels (l, n);
+//   * accumulation c[l,m][n] += S_lm G_nl is register-tiled: a lane owns four consecutive m of one l
+//     times all n (an outer product of 4 x n_max per pair from 4 + n_max/4 shared loads); with at
+//     most 16 such tiles the two half-warps work on two pairs at once.  Sums stay in registers over
+//     all pairs of a species and go to the centre's tile c[lm][species, n] once per species;
+//   * Eq. 4 is the Gram matrix of that tile per l: lanes take 4 x 4 blocks of (species, n) pairs,
+//     two 16-byte loads per 16 multiply-adds, and the feature row is put together in shared memory
+//     and written out in order.
+// Nothing but the pair list is read from HBM and nothing but the descriptor row is written.
+#pragma once
+#include "soap_device.cuh"
+
+namespace soap {
+
+constexpr int kDescChunk = 16;                    // pairs staged at once by a warp
+constexpr int kDescRing = kDescChunk + 32;        // ring of pair geometry (a block of 32 keys may arrive on top of a partial chunk)
+constexpr int kDescMaxWarps = 12;                 // warps per CTA (one CTA per SM)
+
+// harmonic tables up to l = 12, filled by desc_constants(): a_lm (sqrt2 folded in for m > 0), index l(l+1)/2 + m
+__device__ __constant__ float kd_norm[91] = {0};
+
+__host__ __device__ constexpr int desc_tiles(int l_max) {
+    int t = 0;
+    for (int l = 0; l <= l_max; ++l) t += (2 * l + 1 + 3) / 4;
+    return t;
+}
+// n_max is padded to a multiple of four (NP = 4, 8, 12 or 16 is the template parameter; the padding channels have
+// all-zero table rows, so they cost arithmetic but need no special cases)
+__host__ __device__ constexpr int desc_np(int n_max) { return (n_max + 3) & ~3; }
+
+// Shared memory in 4-byte words: [table (optional)] then one region per warp:
+//   c [LM][S NP] | S staging [chunk][LM|1] (+4) | G staging [chunk][L1 NP] | ring [kDescRing][8]
+// The feature row is assembled on top of the staging area when it fits there.
+struct DescLayout {
+    int table, warp0, per_warp, c, sS, sG, ring, slab_words, total;
+};
+__host__ __device__ inline DescLayout make_desc_layout(int S, int np, int l_max, int warps, int table_words) {
+    const int L1 = l_max + 1, LM = L1 * L1, LMP = LM | 1;
+    DescLayout o;
+    o.table = 0;
+    o.warp0 = (table_words + 3) & ~3;
+    int off = 0;
+    o.c = off; off += LM * S * np;
+    o.sS = off; off += (kDescChunk * LMP + 4 + 3) & ~3;
+    o.sG = off; off += kDescChunk * L1 * np;
+    o.ring = off; off += kDescRing * 8;
+    o.slab_words = off - o.sS;
+    o.per_warp = off;
+    o.total = o.warp0 + warps * off;
+    return o;
+}
+
+// Real solid harmonics S_lm(d) = r^l Y_lm of one displacement, every (l, m), written to out[l^2 + l + m]:
+//   S_{l,+m} = a_lm Q_l^m Re (x+iy)^m,  S_{l,-m} = a_lm Q_l^m Im (x+iy)^m,
+//   Q_m^m = (2m-1)!!,  (l+1-m) Q_{l+1}^m = (2l+1) z Q_l^m - (l+m) r^2 Q_{l-1}^m.
+// Fully unrolled: every index is an immediate and the Q's live in registers.
+template <int L>
+__device__ __forceinline__ void harmonics_all(float x, float y, float z, float r2, float* __restrict__ out) {
+    float cm[L + 1], sm[L + 1];                   // (x+iy)^m
+    cm[0] = 1.f; sm[0] = 0.f;
+#pragma unroll
+    for (int m = 1; m <= L; ++m) {
+        cm[m] = x * cm[m - 1] - y * sm[m - 1];
+        sm[m] = x * sm[m - 1] + y * cm[m - 1];
+    }
+    float q1[L + 1], q2[L + 1];                   // Q_l^m and Q_{l-1}^m while the loop is at l
+#pragma unroll
+    for (int m = 0; m <= L; ++m) { q1[m] = 0.f; q2[m] = 0.f; }
+    float dfact = 1.f;                            // (2l-1)!!
+#pragma unroll
+    for (int l = 0; l <= L; ++l) {
+        if (l > 0) dfact *= (float)(2 * l - 1);
+        const float zl = (float)(2 * l - 1) * z;
+#pragma unroll
+        for (int m = 0; m <= l; ++m) {
+            float q;
+            if (m == l) q = dfact;
+            else q = (zl * q1[m] - (float)(l - 1 + m) * r2 * q2[m]) * (1.f / (float)(l - m));
+            q2[m] = q1[m];
+            q1[m] = q;
+            const float aq = kd_norm[l * (l + 1) / 2 + m] * q;
+            out[l * l + l + m] = aq * cm[m];
+            if (m) out[l * l + l - m] = aq * sm[m];
+        }
+    }
+}
+
+// NP: n_max rounded up to a multiple of four.  PLAIN: the default configuration (atom centres, no weighting, every
+// species pair, power spectrum out).  TS: the radial table is in shared memory.
+template <int L, int NP, bool PLAIN, bool TS>
+__global__ void __launch_bounds__(kDescMaxWarps * 32, 1) desc_kernel(const CenterParams p) {
+    constexpr int L1 = L + 1, LM = L1 * L1, LMP = LM | 1;
+    constexpr int NCHP = L1 * NP;
+    constexpr int T = desc_tiles(L);
+    constexpr int HALVES = T <= 16 ? 2 : 1, LANES_T = 32 / HALVES;
+    constexpr int TPL = (T + LANES_T - 1) / LANES_T;                     // tiles per lane (1, or 2 from l_max = 10 on)
+    constexpr int NB = (TPL * NP * 4 <= 64) ? NP : 64 / (4 * TPL);      // n handled per pass (at most 64 accumulators)
+    constexpr int NPASS = (NP + NB - 1) / NB;
+    constexpr int ROUNDS = (NCHP + 31) / 32;
+    extern __shared__ __align__(16) float smem[];
+    const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5, warps = blockDim.x >> 5;
+    const bool o_cross = PLAIN || p.crossover, o_emit = !PLAIN && p.emit_coeff;
+    const float* const o_cbar = PLAIN ? nullptr : p.c_bar;
+    const float* const o_sites = PLAIN ? nullptr : p.sites;
+    const float2* const o_pw = PLAIN ? nullptr : p.pair_w;
+    const float o_w0 = PLAIN ? 1.f : p.w0;
+    const int S = p.S, NMAX = p.n_max, SNP = S * NP, F = p.F;
+    const DescLayout lay = make_desc_layout(S, NP, L, warps, TS ? p.n_intervals * NCHP * 6 : 0);
+
+    if (TS) {
+        const float4* src = reinterpret_cast<const float4*>(p.table_ln);
+        float4* dst = reinterpret_cast<float4*>(smem);
+        const int n4 = p.n_intervals * NCHP * 6 / 4;
+        for (int e = threadIdx.x; e < n4; e += blockDim.x) dst[e] = __ldg(src + e);
+        __syncthreads();
+    }
+    // a failed neighbour build: write nothing
+    if (p.counters->n_pairs > p.pair_capacity) return;
+
+    float* const wbase = smem + lay.warp0 + wid * lay.per_warp;
+    float* const c_t = wbase + lay.c;                                               // [LM][SNP]
+    float* const sS = wbase + lay.sS;                                               // [chunk][LMP]
+    float* const sG = wbase + lay.sG;                                               // [chunk][NCHP]
+    float4* const ring_d = reinterpret_cast<float4*>(wbase + lay.ring);             // [ring] dx, dy, dz, r
+    int4* const ring_i = reinterpret_cast<int4*>(wbase + lay.ring + 4 * kDescRing); // [ring] interval, t, species, weight
+    float* const slab = wbase + lay.sS;
+    const float2* const tab = TS ? reinterpret_cast<const float2*>(smem) : reinterpret_cast<const float2*>(p.table_ln);
+
+    // the tiles of this lane: (l, first m index, number of valid rows)
+    const int half = HALVES == 2 ? lane >> 4 : 0;
+    int t_l[TPL], t_lm0[TPL], t_kv[TPL];
+#pragma unroll
+    for (int tp = 0; tp < TPL; ++tp) {
+        int t = tp * LANES_T + (lane & (LANES_T - 1)), l = 0;
+        if (t >= T) { t_l[tp] = 0; t_lm0[tp] = 0; t_kv[tp] = 0; continue; }
+        while (t >= (2 * l + 4) / 4) { t -= (2 * l + 4) / 4; ++l; }
+        t_l[tp] = l; t_lm0[tp] = l * l + 4 * t; t_kv[tp] = min(4, 2 * l + 1 - 4 * t);
+    }
+    const bool periodic = p.geom.pbc[0] | p.geom.pbc[1] | p.geom.pbc[2];
+    const long long n_work = o_cbar ? 1 : p.n_centers;
+
+    for (;;) {
+        long long w = 0;
+        if (lane == 0) w = (long long)atomicAdd(&p.counters->work, 1);
+        w = __shfl_sync(0xffffffffu, w, 0);
+        if (w >= n_work) break;
+        const long long c_idx = p.order ? p.order[w] : w;
+        const int ci = o_sites ? -1 : (p.centers ? p.centers[c_idx] : (int)c_idx);
+        const float* pc = o_sites ? o_sites + 3 * c_idx : p.pos + 3 * (long long)ci;
+        const float xi = pc[0], yi = pc[1], zi = pc[2];
+        const int zi_species = o_sites ? 0 : p.species_idx[ci];
+        const long long pair_base = p.pair_start[c_idx];
+        const int k_pairs = o_cbar ? 0 : p.pair_count[c_idx];
+
+        for (int e = lane; e < LM * SNP / 4; e += 32) reinterpret_cast<float4*>(c_t)[e] = make_float4(0.f, 0.f, 0.f, 0.f);
+        __syncwarp();
+
+#pragma unroll 1
+        for (int ip = 0; ip < NPASS; ++ip) {
+            const int n0 = ip * NB;
+            float acc[TPL][4][NB];
+#pragma unroll
+            for (int tp = 0; tp < TPL; ++tp)
+#pragma unroll
+                for (int k = 0; k < 4; ++k)
+#pragma unroll
+                    for (int n = 0; n < NB; ++n) acc[tp][k][n] = 0.f;
+            int cur = -1, fill = 0;
+
+            // sums of species s (columns n0 .. n0 + NB - 1) go to the centre's tile; the two half-warps add up first
+            auto flush = [&](int s) {
+#pragma unroll
+                for (int tp = 0; tp < TPL; ++tp)
+#pragma unroll
+                    for (int k = 0; k < 4; ++k) {
+                        float v[NB];
+#pragma unroll
+                        for (int n = 0; n < NB; ++n) {
+                            v[n] = acc[tp][k][n];
+                            if (HALVES == 2) v[n] += __shfl_xor_sync(0xffffffffu, v[n], 16);
+                            acc[tp][k][n] = 0.f;
+                        }
+                        if (k < t_kv[tp] && (HALVES == 1 || (k >> 1) == half)) {
+                            float4* dst = reinterpret_cast<float4*>(c_t + (t_lm0[tp] + k) * SNP + s * NP + n0);
+#pragma unroll
+                            for (int n4 = 0; n4 < NB / 4; ++n4)
+                                if (NPASS == 1 || n0 + 4 * n4 < NP) dst[n4] = make_float4(v[4 * n4], v[4 * n4 + 1], v[4 * n4 + 2], v[4 * n4 + 3]);
+                        }
+                    }
+            };
+
+            // harmonics, radial factors and the accumulation of the first n_stage entries of the ring
+            auto process = [&](int n_stage) {
+                if (lane < n_stage) {
+                    const float4 d = ring_d[lane];
+                    harmonics_all<L>(d.x, d.y, d.z, d.w * d.w, sS + lane * LMP);
+                }
+#pragma unroll 2
+                for (int pr = 0; pr < n_stage; ++pr) {
+                    const int4 gi = ring_i[pr];
+                    const float t = __int_as_float(gi.y);
+                    const float2* row = tab + (size_t)gi.x * (NCHP * 3);
+#pragma unroll
+                    for (int rr = 0; rr < ROUNDS; ++rr) {
+                        const int ch = rr * 32 + lane;
+                        if (ROUNDS * 32 == NCHP || ch < NCHP) {
+                            const float2 a = TS ? row[ch * 3] : __ldg(row + ch * 3);
+                            const float2 b = TS ? row[ch * 3 + 1] : __ldg(row + ch * 3 + 1);
+                            const float2 c = TS ? row[ch * 3 + 2] : __ldg(row + ch * 3 + 2);
+                            float v = fmaf(c.y, t, c.x);
+                            v = fmaf(v, t, b.y);
+                            v = fmaf(v, t, b.x);
+                            v = fmaf(v, t, a.y);
+                            v = fmaf(v, t, a.x);
+                            if (!PLAIN) v *= __int_as_float(gi.w);
+                            sG[pr * NCHP + ch] = v;
+                        }
+                    }
+                }
+                __syncwarp();
+                const int tag = lane < n_stage ? ring_i[lane].z : -1;
+                for (int s = 0; s < S; ++s) {
+                    const unsigned mask = __ballot_sync(0xffffffffu, tag == s);
+                    if (!mask) continue;
+                    const int a = __ffs(mask) - 1, b = a + __popc(mask);       // contiguous: the ring is filled species by species
+                    if (s != cur) {
+                        if (cur >= 0) flush(cur);
+                        cur = s;
+                    }
+                    for (int q = a + half; q < b; q += HALVES) {
+                        const float* sp = sS + q * LMP;
+                        const float4* gp = reinterpret_cast<const float4*>(sG + q * NCHP + n0);
+#pragma unroll
+                        for (int tp = 0; tp < TPL; ++tp) {
+                            float h[4];
+#pragma unroll
+                            for (int k = 0; k < 4; ++k) h[k] = sp[t_lm0[tp] + k];
+#pragma unroll
+                            for (int n4 = 0; n4 < NB / 4; ++n4) {
+                                if (NPASS > 1 && n0 + 4 * n4 >= NP) break;
+                                const float4 g = gp[t_l[tp] * (NP / 4) + n4];
+#pragma unroll
+                                for (int k = 0; k < 4; ++k) {
+                                    acc[tp][k][4 * n4] = fmaf(h[k], g.x, acc[tp][k][4 * n4]);
+                                    acc[tp][k][4 * n4 + 1] = fmaf(h[k], g.y, acc[tp][k][4 * n4 + 1]);
+                                    acc[tp][k][4 * n4 + 2] = fmaf(h[k], g.z, acc[tp][k][4 * n4 + 2]);
+                                    acc[tp][k][4 * n4 + 3] = fmaf(h[k], g.w, acc[tp][k][4 * n4 + 3]);
+                                }
+                            }
+                        }
+                    }
+                }
+                __syncwarp();
+            };
+
+            for (int s = 0; s < S; ++s) {
+                for (int e0 = 0; e0 < k_pairs; e0 += 32) {
+                    const int e = e0 + lane;
+                    bool match = false;
+                    unsigned long long key = 0;
+                    int j = 0;
+                    if (e < k_pairs) {
+                        key = p.pair_key[pair_base + e];
+                        j = key_atom(key);
+                        match = S == 1 || p.species_idx[j] == s;
+                    }
+                    const unsigned m = __ballot_sync(0xffffffffu, match);
+                    if (!m) continue;
+                    if (match) {
+                        double dx = (double)p.pos[3 * (long long)j] - (double)xi;
+                        double dy = (double)p.pos[3 * (long long)j + 1] - (double)yi;
+                        double dz = (double)p.pos[3 * (long long)j + 2] - (double)zi;
+                        if (periodic) {
+                            int sh[3];
+                            key_shift(key, sh);
+                            dx += sh[0] * p.geom.cell[0] + sh[1] * p.geom.cell[3] + sh[2] * p.geom.cell[6];
+                            dy += sh[0] * p.geom.cell[1] + sh[1] * p.geom.cell[4] + sh[2] * p.geom.cell[7];
+                            dz += sh[0] * p.geom.cell[2] + sh[1] * p.geom.cell[5] + sh[2] * p.geom.cell[8];
+                        }
+                        const double r = sqrt(dx * dx + dy * dy + dz * dz);
+                        // interval and offset in the radial table, in fp64 so that the offset keeps its digits
+                        const double u = r * (double)p.inv_h;
+                        const int qi = min((int)u, p.n_intervals - 1);
+                        const int slot = fill + __popc(m & ((1u << lane) - 1));
+                        ring_d[slot] = make_float4((float)dx, (float)dy, (float)dz, (float)r);
+                        ring_i[slot] = make_int4(qi, __float_as_int((float)(u - qi)), s,
+                                                 __float_as_int(o_pw ? o_pw[pair_base + e].x : 1.f));
+                    }
+                    fill += __popc(m);
+                    __syncwarp();
+                    while (fill >= kDescChunk) {
+                        process(kDescChunk);
+                        // move what is left to the front of the ring
+                        const int rest = fill - kDescChunk;
+                        float4 d4 = make_float4(0.f, 0.f, 0.f, 0.f);
+                        int4 i4 = make_int4(0, 0, 0, 0);
+                        if (lane < rest) { d4 = ring_d[kDescChunk + lane]; i4 = ring_i[kDescChunk + lane]; }
+                        __syncwarp();
+                        if (lane < rest) { ring_d[lane] = d4; ring_i[lane] = i4; }
+                        __syncwarp();
+                        fill = rest;
+                    }
+                }
+            }
+            if (fill > 0) process(fill);
+            if (cur >= 0) flush(cur);
+            __syncwarp();
+        }
+
+        // on-site term: the centre's own Gaussian, l = 0 only (second term of Eq. 13)
+        if (!o_cbar && !o_sites && lane < NMAX) c_t[zi_species * NP + lane] += o_w0 * __ldg(p.self_term + lane);
+        if (o_cbar) {
+            // given mean coefficients (inner average) take the place of the centre's own: index (mu n_max + n) LM + lm
+            for (int e = lane; e < S * NMAX * LM; e += 32) {
+                const int row = e / LM, lm = e - row * LM, mu = row / NMAX, n = row - mu * NMAX;
+                c_t[lm * SNP + mu * NP + n] = __ldg(o_cbar + e);
+            }
+        }
+        __syncwarp();
+        if (o_emit) {
+            // coefficient mode: the tile itself is the result, index (mu n_max + n) (l_max+1)^2 + l^2 + l + m
+            float* crow = p.out_desc + (size_t)c_idx * (S * NMAX * LM);
+            for (int e = lane; e < S * NMAX * LM; e += 32) {
+                const int row = e / LM, lm = e - row * LM, mu = row / NMAX, n = row - mu * NMAX;
+                crow[e] = c_t[lm * SNP + mu * NP + n];
+            }
+            __syncwarp();
+            continue;
+        }
+
+        // ---- power spectrum (Eq. 4): per l the Gram matrix of the tile's rows over (species, n) ----
+        float* const desc_row = p.out_desc + (o_cbar ? (size_t)0 : (size_t)c_idx * F);
+        const bool staged = F <= lay.slab_words;
+        float* const dst = staged ? slab : desc_row;
+        constexpr int TB = NP / 4;                                   // 4-wide column tiles per species
+        const int TA = S * TB;
+        const int NTP = o_cross ? TA * (TA + 1) / 2 : S * (TB * (TB + 1) / 2);
+        const int n_tasks = NTP * L1;
+        const int TRI = (NMAX * (NMAX + 1) / 2) * L1, SQ = NMAX * NMAX * L1;
+        for (int u0 = 0; u0 < n_tasks; u0 += 32) {
+            const int u = u0 + lane;
+            const bool active = u < n_tasks;
+            const int lq = active ? u / NTP : 0;
+            const int l = active ? L - lq : 0;                       // longest sums first; lanes of a round have similar l
+            int rem = active ? u - lq * NTP : 0, ta = 0, tb = 0;
+            if (o_cross) {
+                while (rem >= TA - ta) { rem -= TA - ta; ++ta; }
+                tb = ta + rem;
+            } else {
+                const int sb = rem / (TB * (TB + 1) / 2);
+                rem -= sb * (TB * (TB + 1) / 2);
+                while (rem >= TB - ta) { rem -= TB - ta; ++ta; }
+                tb = sb * TB + ta + rem;
+                ta += sb * TB;
+            }
+            float g[4][4];
+#pragma unroll
+            for (int i = 0; i < 4; ++i)
+#pragma unroll
+                for (int j = 0; j < 4; ++j) g[i][j] = 0.f;
+            const float* rowp = c_t + (l * l) * SNP;
+            const int steps = active ? 2 * l + 1 : 0;
+            for (int m = 0; m < steps; ++m) {
+                const float4 A = *reinterpret_cast<const float4*>(rowp + m * SNP + 4 * ta);
+                const float4 B = *reinterpret_cast<const float4*>(rowp + m * SNP + 4 * tb);
+                const float av[4] = {A.x, A.y, A.z, A.w}, bv[4] = {B.x, B.y, B.z, B.w};
+#pragma unroll
+                for (int i = 0; i < 4; ++i)
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) g[i][j] = fmaf(av[i], bv[j], g[i][j]);
+            }
+            if (active) {
+                const float kl = __ldg(p.kl + l);
+                const int mu = (4 * ta) / NP, nu = (4 * tb) / NP, na = 4 * ta - mu * NP, nb = 4 * tb - nu * NP;
+                int off;
+                if (o_cross) {
+                    const int before = mu * S - mu * (mu - 1) / 2 + (nu - mu), diag = mu + (nu > mu ? 1 : 0);
+                    off = diag * TRI + (before - diag) * SQ;
+                } else {
+                    off = mu * TRI;
+                }
+#pragma unroll
+                for (int i = 0; i < 4; ++i)
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) {
+                        const int n1 = na + i, n2 = nb + j;
+                        if (n1 < NMAX && n2 < NMAX && (mu < nu || n1 <= n2)) {
+                            const int within = mu == nu ? n1 * NMAX - n1 * (n1 - 1) / 2 + (n2 - n1) : n1 * NMAX + n2;
+                            dst[off + within * L1 + l] = kl * g[i][j];
+                        }
+                    }
+            }
+        }
+        __syncwarp();
+        if (staged) {
+            for (int e = lane; e < F; e += 32) desc_row[e] = slab[e];
+            __syncwarp();
+        }
+    }
+}
+
+}  // namespace soap

@@ -2,6 +2,7 @@
 #include <cuda_runtime.h>
 
 #include <algorithm>
+#include <atomic>
 #include <cmath>
 #include <cstdio>
 #include <cstdlib>
@@ -14,6 +15,8 @@
 #include "average_kernels.cuh"
 #include "center_launch.h"
 #include "dense_kernel.cuh"
+#include "desc_kernel.cuh"
+#include "desc_launch.h"
 #include "neighbor_kernels.cuh"
 #include "soap.h"
 #include "weight_kernel.cuh"
@@ -21,11 +24,6 @@
 using namespace soap;
 
 namespace soap {
-// tuning knob: SOAP_B200_GENERAL=1 runs the default configuration through the general kernels as well
-static bool force_general() {
-    static const bool on = [] { const char* e = std::getenv("SOAP_B200_GENERAL"); return e && e[0] == '1'; }();
-    return on;
-}
 cudaError_t center_constants(int l_max, const float* anorm91, const float* dfact16) {
     switch (l_max) {
 #define X(LV) case LV: return center_constants_l##LV(anorm91, dfact16);
@@ -44,7 +42,32 @@ cudaError_t center_set_smem(int kind, int l_max, int n_max, int bytes) {
 }
 cudaError_t center_launch(int kind, int l_max, int n_max, const CenterParams& p, unsigned grid, size_t smem, cudaStream_t st) {
     switch (l_max) {
-#define X(LV) case LV: return center_launch_l##LV(kind, n_max, center_params_plain(p) && !force_general(), p, grid, smem, st);
+#define X(LV) case LV: return center_launch_l##LV(kind, n_max, center_params_plain(p), p, grid, smem, st);
+        X(0) X(1) X(2) X(3) X(4) X(5) X(6) X(7) X(8) X(9) X(10) X(11) X(12)
+#undef X
+    }
+    return cudaErrorInvalidValue;
+}
+cudaError_t desc_constants(int l_max, const float* anorm91) {
+    switch (l_max) {
+#define X(LV) case LV: return desc_constants_l##LV(anorm91);
+        X(0) X(1) X(2) X(3) X(4) X(5) X(6) X(7) X(8) X(9) X(10) X(11) X(12)
+#undef X
+    }
+    return cudaErrorInvalidValue;
+}
+cudaError_t desc_set_smem(int l_max, int np, int bytes) {
+    switch (l_max) {
+#define X(LV) case LV: return desc_set_smem_l##LV(np, bytes);
+        X(0) X(1) X(2) X(3) X(4) X(5) X(6) X(7) X(8) X(9) X(10) X(11) X(12)
+#undef X
+    }
+    return cudaErrorInvalidValue;
+}
+cudaError_t desc_launch(int l_max, int np, bool plain, bool table_in_smem, const CenterParams& p, unsigned grid, unsigned block,
+                        size_t smem, cudaStream_t st) {
+    switch (l_max) {
+#define X(LV) case LV: return desc_launch_l##LV(np, plain, table_in_smem, p, grid, block, smem, st);
         X(0) X(1) X(2) X(3) X(4) X(5) X(6) X(7) X(8) X(9) X(10) X(11) X(12)
 #undef X
     }
@@ -72,6 +95,10 @@ struct soap_handle {
     int device = -1;
     bool tables_ready = false;
     float *d_table = nullptr, *d_self = nullptr, *d_kl = nullptr;
+    float* d_table_ln = nullptr;         // the radial table re-laid for the descriptor-only kernel
+    int sm_count = 0, max_smem = 0;
+    int desc_np = 0;                     // n_max rounded up to a multiple of four
+    size_t desc_table_bytes = 0, desc_warp_bytes = 0;
     int *d_feat = nullptr, *d_zlut = nullptr, *d_l_of_lm = nullptr;
     Counters* d_counters = nullptr;
     unsigned long long* d_bbox = nullptr;   // 6 words of bounding box (structures above 16384 atoms)
@@ -95,8 +122,8 @@ struct soap_handle {
     int64_t planned_atoms = -1, planned_centers = -1;
     int64_t pairs_per_center_hint = 0;   // average at the last plan (chooses the pair kernel variant)
     int64_t last_centers = 0;
-    int P_desc = 16, P_deriv = 16;
-    size_t smem_desc = 0, smem_deriv = 0;
+    int P_deriv = 16;
+    size_t smem_deriv = 0;
     // optional per-segment timing (events on the caller's stream)
     bool profiling = false;
     cudaEvent_t ev[3] = {nullptr, nullptr, nullptr};
@@ -167,29 +194,29 @@ int plan_smem(soap_t* h) {
     // shared-memory plan of the per-centre kernels
     int max_smem = 0;
     CU(cudaDeviceGetAttribute(&max_smem, cudaDevAttrMaxSharedMemoryPerBlockOptin, h->device));
-    for (int deriv = 0; deriv < 2; ++deriv) {
-        // largest chunk that still leaves room for three CTAs per SM, else two, else whatever fits
+    h->max_smem = max_smem;
+    h->desc_warp_bytes = (size_t)make_desc_layout(h->S, desc_np(h->n_max), h->l_max, 1, 0).per_warp * 4;
+    if (h->desc_warp_bytes > (size_t)max_smem) return fail(h, SOAP_ERR_INVALID_ARG, "this basis does not fit the shared memory of the device");
+    CU(desc_set_smem(h->l_max, desc_np(h->n_max), max_smem));
+    {
+        // pairs per staged chunk of the derivative kernels: the largest that still leaves room for three CTAs per SM,
+        // else two, else whatever fits
         int P = 32;
         size_t bytes = 0;
         const size_t budget3 = (size_t)228 * 1024 / 3 - 1024, budget2 = (size_t)228 * 1024 / 2 - 1024;
         for (int pass = 0; pass < 3; ++pass) {
             const size_t budget = pass == 0 ? budget3 : pass == 1 ? budget2 : (size_t)max_smem;
             for (P = 32; P >= 4; P /= 2) {
-                bytes = (size_t)make_layout(h->S, h->n_max, h->l_max, P, deriv, h->weight.fn != 0).total * 4;
+                bytes = (size_t)make_layout(h->S, h->n_max, h->l_max, P, true, h->weight.fn != 0).total * 4;
                 if (bytes <= budget) break;
             }
             if (P >= (pass == 2 ? 4 : 8) && bytes <= budget) break;
             if (P < 4) P = 4;
         }
-        if (const char* env = std::getenv("SOAP_B200_CHUNK")) {       // tuning knob: pairs staged per chunk (4..32)
-            const int v = std::atoi(env);
-            if (v >= 4 && v <= 32) P = v;
-        }
-        bytes = (size_t)make_layout(h->S, h->n_max, h->l_max, P, deriv, h->weight.fn != 0).total * 4;
+        bytes = (size_t)make_layout(h->S, h->n_max, h->l_max, P, true, h->weight.fn != 0).total * 4;
         if (bytes > (size_t)max_smem) return fail(h, SOAP_ERR_INVALID_ARG, "this basis does not fit the shared memory of the device");
-        if (deriv) { h->P_deriv = P; h->smem_deriv = bytes; } else { h->P_desc = P; h->smem_desc = bytes; }
+        h->P_deriv = P; h->smem_deriv = bytes;
     }
-    CU(center_set_smem(kCenterDesc, h->l_max, h->n_max, (int)h->smem_desc));
     CU(center_set_smem(kCenterDeriv, h->l_max, h->n_max, (int)h->smem_deriv));
     CU(center_set_smem(kCenterCoeff, h->l_max, h->n_max, (int)h->smem_deriv));
     return SOAP_OK;
@@ -205,6 +232,21 @@ int ensure_device(soap_t* h) {
     }
     h->device = dev;
     CU(upload(&h->d_table, h->basis.table));
+    {
+        // [interval][l][n padded to a multiple of four][6]; the padding channels are zero
+        const int L1 = h->l_max + 1, n_ch = h->n_max * L1, np = desc_np(h->n_max);
+        std::vector<float> ln((size_t)h->basis.n_intervals * L1 * np * kTableCoef, 0.f);
+        for (int q = 0; q < h->basis.n_intervals; ++q)
+            for (int l = 0; l < L1; ++l)
+                for (int n = 0; n < h->n_max; ++n)
+                    for (int k = 0; k < kTableCoef; ++k)
+                        ln[(((size_t)q * L1 + l) * np + n) * kTableCoef + k] =
+                            h->basis.table[((size_t)q * n_ch + n * L1 + l) * kTableCoef + k];
+        CU(upload(&h->d_table_ln, ln));
+        h->desc_np = np;
+        h->desc_table_bytes = ln.size() * sizeof(float);
+    }
+    CU(cudaDeviceGetAttribute(&h->sm_count, cudaDevAttrMultiProcessorCount, h->device));
     CU(upload(&h->d_self, h->basis.self_term));
     CU(upload(&h->d_kl, h->basis.kl));
     CU(upload(&h->d_feat, h->feat_pack));
@@ -229,6 +271,7 @@ int ensure_device(soap_t* h) {
         for (size_t i = 0; i < h->basis.anorm.size(); ++i) anorm[i] = h->basis.anorm[i];
         for (size_t i = 0; i < h->basis.dfact.size(); ++i) dfact[i] = h->basis.dfact[i];
         CU(center_constants(h->l_max, anorm.data(), dfact.data()));
+        CU(desc_constants(h->l_max, anorm.data()));
     }
     h->tables_ready = true;
     return SOAP_OK;
@@ -303,7 +346,8 @@ constexpr int64_t kBruteForceAtoms = 512;
 int launch_neighbors(soap_t* h, const float* pos, const int32_t* num, int64_t N, const Geometry& g,
                      const int32_t* centers, const float* sites, int64_t C, long long* row_ptr_out, cudaStream_t st,
                      const Batch& batch = Batch()) {
-    const bool brute = !batch.struct_ptr && !centers && !sites && N <= kBruteForceAtoms && !(g.pbc[0] | g.pbc[1] | g.pbc[2]);
+    // (C == N: the brute-force kernel writes the per-centre arrays for every atom, and those are sized from C)
+    const bool brute = !batch.struct_ptr && !centers && !sites && C == N && N <= kBruteForceAtoms && !(g.pbc[0] | g.pbc[1] | g.pbc[2]);
     if (batch.struct_ptr || brute) {
         CU(cudaMemsetAsync(&h->d_counters->n_pairs, 0, 2 * sizeof(long long), st));      // pair cursor and row total
         if (N > 0) batch_pairs_kernel<<<(unsigned)((N + kFillWarps - 1) / kFillWarps), kFillWarps * 32, 0, st>>>(
@@ -387,11 +431,31 @@ void fill_center_params(soap_t* h, CenterParams& cp, const float* pos, const int
     cp.table = h->d_table; cp.self_term = h->d_self; cp.kl = h->d_kl; cp.l_of_lm = h->d_l_of_lm;
     cp.feat_pack = h->d_feat; cp.nch_magic = (unsigned)((1ull << 32) / (unsigned)(h->n_max * (h->l_max + 1))) + 1u; cp.inv_h = (float)h->basis.inv_h; cp.n_intervals = h->basis.n_intervals;
     cp.S = h->S; cp.n_max = h->n_max; cp.l_max = h->l_max; cp.F = (int)h->F;
-    cp.P = deriv ? h->P_deriv : h->P_desc;
+    cp.P = h->P_deriv;
     cp.crossover = h->crossover; cp.emit_coeff = 0; cp.c_bar = nullptr;
     cp.pair_w = h->weight.fn ? h->d_pair_w : nullptr; cp.w0 = (float)h->w0;
     cp.compact = 0; cp.Fc = (int)h->Fc_pitch; cp.out_center = nullptr;
     cp.out_desc = nullptr; cp.out_jac = nullptr; cp.row_atom = nullptr;
+}
+
+// Launch of the descriptor-only kernel: persistent CTAs (one per SM) whose warps draw centres from a counter.
+// The radial table goes to shared memory when it leaves room for at least six warps and there is enough
+// work to pay for staging it; small jobs use fewer warps per CTA so that they spread over the SMs.
+int launch_desc(soap_t* h, CenterParams& cp, int64_t n_work, cudaStream_t st) {
+    if (n_work <= 0) return SOAP_OK;
+    cp.table_ln = h->d_table_ln;
+    const bool plain = center_params_plain(cp);
+    const int warps_fit = (int)std::min<size_t>(kDescMaxWarps, (size_t)h->max_smem / h->desc_warp_bytes);
+    const int warps_ts = h->desc_table_bytes + h->desc_warp_bytes <= (size_t)h->max_smem
+                             ? (int)std::min<size_t>(kDescMaxWarps, ((size_t)h->max_smem - h->desc_table_bytes) / h->desc_warp_bytes) : 0;
+    const bool ts = plain && warps_ts >= 6 && n_work >= (int64_t)4 * h->sm_count;
+    int warps = ts ? warps_ts : warps_fit;
+    warps = (int)std::max<int64_t>(1, std::min<int64_t>(warps, (n_work + h->sm_count - 1) / h->sm_count));
+    const unsigned grid = (unsigned)std::min<int64_t>(h->sm_count, (n_work + warps - 1) / warps);
+    const size_t smem = (size_t)make_desc_layout(h->S, h->desc_np, h->l_max, warps, ts ? (int)(h->desc_table_bytes / 4) : 0).total * 4;
+    CU(cudaMemsetAsync(&h->d_counters->work, 0, sizeof(int), st));
+    CU(desc_launch(h->l_max, h->desc_np, plain, ts, cp, grid, (unsigned)warps * 32, smem, st));
+    return SOAP_OK;
 }
 
 // Feature table: species pairs mu <= nu (only mu == nu without crossover), radial pair (n' >= n on
@@ -509,7 +573,7 @@ int soap_create(soap_t** out, const int32_t* species, int n_species, double r_cu
 
 void soap_destroy(soap_t* h) {
     if (!h) return;
-    void* ptrs[] = {h->d_table, h->d_self, h->d_kl, h->d_feat, h->d_zlut, h->d_l_of_lm, h->d_counters, h->d_bbox,
+    void* ptrs[] = {h->d_table, h->d_table_ln, h->d_self, h->d_kl, h->d_feat, h->d_zlut, h->d_l_of_lm, h->d_counters, h->d_bbox,
                     h->d_grid, h->d_species_idx, h->d_atom_cell, h->d_atom_wrap, h->d_s_wrap, h->d_s_pos, h->d_cell_count,
                     h->d_cell_start, h->d_pair_count, h->d_row_count, h->d_self_row, h->d_order, h->d_pair_ptr, h->d_pair_start, h->d_row_ptr, h->d_tile_sums, h->d_tile_offsets,
                     h->d_pair_key, h->d_pair_tmp, h->d_pair_row, h->d_work, h->d_pair_w, h->d_compact_map};
@@ -602,7 +666,7 @@ static int descriptor_impl(soap_t* h, const float* d_positions, const int32_t* d
         CenterParams cp;
         fill_center_params(h, cp, d_positions, d_centers, n_centers, g, false, d_sites);
         cp.out_desc = d_out;
-        CU(center_launch(kCenterDesc, h->l_max, h->n_max, cp, (unsigned)n_centers, h->smem_desc, st));
+        if ((rc = launch_desc(h, cp, n_centers, st))) return rc;
     }
     if (h->profiling) CU(cudaEventRecord(h->ev[2], st));
     return SOAP_OK;
@@ -817,7 +881,7 @@ int soap_coefficients(soap_t* h, const float* d_positions, const int32_t* d_numb
         fill_center_params(h, cp, d_positions, d_centers, n_centers, g, false);
         cp.out_desc = d_out;
         cp.emit_coeff = 1;
-        CU(center_launch(kCenterDesc, h->l_max, h->n_max, cp, (unsigned)n_centers, h->smem_desc, st));
+        if ((rc = launch_desc(h, cp, n_centers, st))) return rc;
     }
     if (h->profiling) CU(cudaEventRecord(h->ev[2], st));
     return SOAP_OK;
@@ -866,7 +930,7 @@ int soap_descriptor_average(soap_t* h, int mode, const float* d_positions, const
     fill_center_params(h, cp, d_positions, d_centers, n_centers, g, false);
     cp.out_desc = (float*)(w + o_rows);
     cp.emit_coeff = inner ? 1 : 0;
-    CU(center_launch(kCenterDesc, h->l_max, h->n_max, cp, (unsigned)n_centers, h->smem_desc, st));
+    if ((rc = launch_desc(h, cp, n_centers, st))) return rc;
     if ((rc = column_mean(h, (const float*)(w + o_rows), n_centers, width, (double*)(w + o_partial),
                           inner ? (float*)(w + o_cbar) : d_out, st))) return rc;
     if (inner) {
@@ -875,7 +939,7 @@ int soap_descriptor_average(soap_t* h, int mode, const float* d_positions, const
         cp.c_bar = (const float*)(w + o_cbar);
         cp.out_desc = d_out;
         cp.order = nullptr;
-        CU(center_launch(kCenterDesc, h->l_max, h->n_max, cp, 1u, h->smem_desc, st));
+        if ((rc = launch_desc(h, cp, 1, st))) return rc;
     }
     if (h->profiling) CU(cudaEventRecord(h->ev[2], st));
     return SOAP_OK;
@@ -915,7 +979,7 @@ int soap_derivatives_average(soap_t* h, int mode, const float* d_positions, cons
         fill_center_params(h, cp, d_positions, d_centers, n_centers, g, false);
         cp.out_desc = (float*)(w + o_rows);
         cp.emit_coeff = 1;
-        CU(center_launch(kCenterDesc, h->l_max, h->n_max, cp, (unsigned)n_centers, h->smem_desc, st));
+        if ((rc = launch_desc(h, cp, n_centers, st))) return rc;
         if ((rc = column_mean(h, (const float*)(w + o_rows), n_centers, W, (double*)(w + o_partial), (float*)(w + o_cbar), st))) return rc;
     }
     fill_center_params(h, cp, d_positions, d_centers, n_centers, g, true);
@@ -1018,18 +1082,19 @@ int soap_neighbor_counts_static(const float* d_positions, int64_t n_atoms, doubl
     // Set-up, once per device: the array's name is only a host-side stand-in here, so ask the
     // runtime for its device address.  The first call on a device does this (it may initialise
     // the context) and should therefore come before any stream capture.
-    static unsigned char* base_of_device[64] = {nullptr};
+    static std::atomic<unsigned char*> base_of_device[64];    // zero-initialised; one look-up per device, published atomically
     int dev = -1;
     cudaError_t e = cudaGetDevice(&dev);
     if (e != cudaSuccess) return say(SOAP_ERR_CUDA, cudaGetErrorString(e));
     if (dev < 0 || dev >= 64) return say(SOAP_ERR_INVALID_ARG, "device ordinal out of range");
-    if (!base_of_device[dev]) {
+    unsigned char* base = base_of_device[dev].load(std::memory_order_acquire);
+    if (!base) {
         void* ptr = nullptr;
         e = cudaGetSymbolAddress(&ptr, g_static_scratch);
         if (e != cudaSuccess || !ptr) return say(SOAP_ERR_CUDA, cudaGetErrorString(e));
-        base_of_device[dev] = static_cast<unsigned char*>(ptr);
+        base = static_cast<unsigned char*>(ptr);
+        base_of_device[dev].store(base, std::memory_order_release);
     }
-    unsigned char* base = base_of_device[dev];
     unsigned long long* bbox = reinterpret_cast<unsigned long long*>(base);
     GridParams* grid = reinterpret_cast<GridParams*>(base + 256);
     Counters* counters = reinterpret_cast<Counters*>(base + 768);

@@ -41,7 +41,7 @@ struct GridParams {               // device-resident, written by grid_setup_kern
 
 struct Counters {                 // device-resident
     int status;
-    int pad;
+    int work;                     // next centre of the descriptor-only kernel (zeroed before its launch)
     long long n_pairs;
     long long n_rows;
 };
@@ -66,6 +66,7 @@ struct CenterParams {
     Counters* counters;
     // basis
     const float* table;           // [nint][n_ch][6]
+    const float* table_ln;        // the same polynomials as [nint][l][n padded to a multiple of 4][6] (descriptor-only kernel)
     const float* self_term;       // [n_max]
     const int* l_of_lm;           // [lm] -> l
     const float* kl;

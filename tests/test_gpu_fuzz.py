@@ -1,14 +1,17 @@
 """Seeded random sweep over the configuration space: species count, basis size, radial basis, periodicity,
-crossover, weighting, compact rows, point centres — each drawn configuration on a small random structure, GPU
+crossover, weighting, compact rows, point centres, each drawn configuration on a small random structure, GPU
 against the oracle.
 
-Tolerances as everywhere (1e-5 values, 1e-4 Jacobians, per output column), with one difference in the scale of a
-column.  These structures are tiny (2 to 19 atoms, often one or two atoms per species), so a whole column can sit
-near a node or in the tail of its radial function for every centre at once; the column's own maximum is then far
-below the size of the quantities it is computed from, and fp32 cannot be accurate relative to it (2e-5 to 6e-5 was
-seen on 5 of 60 draws, Jacobians within 1e-4 throughout).  The column scale is therefore floored at 1e-3 of the
-largest entry of the whole output instead of at 1e-8; a wrong index, sign or term shows up at order one on the large
-entries regardless."""
+Every comparison evaluates the stated metric (per output column, largest |error| over the largest |reference| of
+that column, the column scale floored at 1e-8 absolute) against 1e-5 for values and 1e-4 for Jacobians.  These
+structures are tiny (2 to 19 atoms, often one or two atoms per species), so a whole column can be a cancelling sum
+for every centre at once: its own maximum is then far below the size of the fp32 quantities it is computed from.
+Where the stated metric is exceeded the test therefore demands that
+  * the offending column's own maximum is below 1e-3 of the largest entry of the whole output, and
+  * the error is within tolerance once the column scale is floored at 1e-3 of that largest entry,
+and records the case; the recorded cases are listed at the end of the run (one line per seed and output, with both
+figures), so nothing is hidden by the floor.  A wrong index, sign or term shows at order one on the large entries
+under either metric."""
 import os
 
 import numpy as np
@@ -19,13 +22,26 @@ from oracle.soap import GTO, POLYNOMIAL, SoapOracle
 from soap_inputs import Structure
 from test_gpu_parity import DESC_TOL, JAC_TOL
 
+RELAXED = []          # (tag, what, stated error, relaxed error, column max / output max), printed by conftest at the end
 
-def col_err(a, ref, axes):
+
+def check(a, ref, axes, tol, tag, what):
     a = np.asarray(a, np.float64)
     if ref.size == 0:
-        return 0.0
-    floor = max(1e-3 * float(np.abs(ref).max()), 1e-8)
-    return float((np.abs(a - ref).max(axis=axes) / np.maximum(np.abs(ref).max(axis=axes), floor)).max())
+        return
+    err = np.abs(a - ref).max(axis=axes)
+    col = np.abs(ref).max(axis=axes)
+    top = float(np.abs(ref).max())
+    stated = err / np.maximum(col, 1e-8)
+    relaxed = err / np.maximum(col, max(1e-3 * top, 1e-8))
+    if float(stated.max()) < tol:
+        return
+    bad = stated >= tol
+    ratio = float((col[bad] / max(top, 1e-300)).max())
+    RELAXED.append((tag, what, float(stated.max()), float(relaxed.max()), ratio))
+    assert ratio < 1e-3, f"{tag}: {what}: stated metric {stated.max():.2e} on a column at {ratio:.1e} of the output's maximum"
+    assert float(relaxed.max()) < tol, f"{tag}: {what}: {relaxed.max():.2e} even with the column scale floored at 1e-3 of the maximum"
+
 
 torch = pytest.importorskip("torch")
 pytestmark = pytest.mark.gpu
@@ -91,11 +107,11 @@ def test_random_configuration(seed):
         raise
     assert np.array_equal(out.row_ptr.cpu().numpy(), ref.row_ptr), tag
     assert np.array_equal(out.row_atom.cpu().numpy(), ref.row_atom), tag
-    assert col_err(out.descriptor.cpu().numpy(), ref.descriptor, 0) < DESC_TOL, tag
-    assert col_err(out.jacobian.cpu().numpy(), ref.jacobian, (0, 1)) < JAC_TOL, tag
+    check(out.descriptor.cpu().numpy(), ref.descriptor, 0, DESC_TOL, tag, "descriptor")
+    check(out.jacobian.cpu().numpy(), ref.jacobian, (0, 1), JAC_TOL, tag, "Jacobian")
     d = soap.descriptor(pos, num, s.cell)
     soap.status()
-    assert col_err(d.cpu().numpy(), ref.descriptor, 0) < DESC_TOL, tag
+    check(d.cpu().numpy(), ref.descriptor, 0, DESC_TOL, tag, "descriptor-only call")
     if seed % 5 == 4 and not any(s.pbc) and s.n_atoms >= 2:        # the structure cut in two, as a batch of two
         cut = s.n_atoms // 2
         parts = [(s.positions[:cut], s.numbers[:cut]), (s.positions[cut:], s.numbers[cut:])]
@@ -103,31 +119,31 @@ def test_random_configuration(seed):
         ptr = torch.tensor([0, cut, s.n_atoms], dtype=torch.int64, device="cuda")
         b = soap.derivatives_batch(pos, num, ptr)
         assert np.array_equal(b.row_atom.cpu().numpy(), bref.row_atom), tag
-        assert col_err(b.descriptor.cpu().numpy(), bref.descriptor, 0) < DESC_TOL, tag
-        assert col_err(b.jacobian.cpu().numpy(), bref.jacobian, (0, 1)) < JAC_TOL, tag
+        check(b.descriptor.cpu().numpy(), bref.descriptor, 0, DESC_TOL, tag, "batch descriptor")
+        check(b.jacobian.cpu().numpy(), bref.jacobian, (0, 1), JAC_TOL, tag, "batch Jacobian")
     which = seed % 4
     if which == 3:                                   # averaged descriptor and Jacobian
         mode = "inner" if seed % 8 == 3 else "outer"
         rd, rj = modes.average_derivatives(oracle, mode, s.positions, s.numbers, s.cell)
         gd, gj = soap.derivatives_average(mode, pos, num, s.cell)
         soap.status()
-        assert col_err(gd.cpu().numpy()[None], rd[None], 0) < DESC_TOL, tag
-        assert col_err(gj.cpu().numpy(), rj, (0, 1)) < JAC_TOL, tag
+        check(gd.cpu().numpy()[None], rd[None], 0, DESC_TOL, tag, "averaged descriptor")
+        check(gj.cpu().numpy(), rj, (0, 1), JAC_TOL, tag, "averaged Jacobian")
     elif which == 0:                                   # compact rows expand to the same rows
         comp = soap.derivatives_compact(pos, num, s.cell)
         exp = soap.compact_expand(num, None, comp).cpu().numpy()
         soap.status()
-        assert col_err(exp, ref.jacobian, (0, 1)) < JAC_TOL, tag
+        check(exp, ref.jacobian, (0, 1), JAC_TOL, tag, "expanded compact rows")
     elif which == 1:                                 # coefficient mode
         cref = modes.coefficient_derivatives(oracle, s.positions, s.numbers, s.cell)
         c = soap.coefficient_derivatives(pos, num, s.cell)
-        assert col_err(c.descriptor.cpu().numpy(), cref.descriptor, 0) < DESC_TOL, tag
-        assert col_err(c.jacobian.cpu().numpy(), cref.jacobian, (0, 1)) < JAC_TOL, tag
+        check(c.descriptor.cpu().numpy(), cref.descriptor, 0, DESC_TOL, tag, "coefficients")
+        check(c.jacobian.cpu().numpy(), cref.jacobian, (0, 1), JAC_TOL, tag, "coefficient Jacobian")
     else:                                            # point centres
         span = s.positions.max(axis=0) - s.positions.min(axis=0) + 1.0
         sites = (s.positions.min(axis=0) - 0.5 + rng.random((3, 3)) * span).astype(np.float32)
         sref = modes.site_derivatives(oracle, s.positions, s.numbers, sites, s.cell)
         at = soap.derivatives_at(pos, num, torch.from_numpy(sites).cuda(), s.cell)
         assert np.array_equal(at.row_atom.cpu().numpy(), sref.row_atom), tag
-        assert col_err(at.descriptor.cpu().numpy(), sref.descriptor, 0) < DESC_TOL, tag
-        assert col_err(at.jacobian.cpu().numpy(), sref.jacobian, (0, 1)) < JAC_TOL, tag
+        check(at.descriptor.cpu().numpy(), sref.descriptor, 0, DESC_TOL, tag, "point-centre descriptor")
+        check(at.jacobian.cpu().numpy(), sref.jacobian, (0, 1), JAC_TOL, tag, "point-centre Jacobian")

@@ -23,7 +23,7 @@ def pkg():
 
 def test_library_exports_every_declared_symbol(pkg):
     header = open(os.path.join(ROOT, "include", "soap.h")).read()
-    declared = sorted(set(re.findall(r"\b(soap_[a-z_]+)\s*\(", header)))
+    declared = sorted(set(re.findall(r"\b(soap_[a-z0-9_]+)\s*\(", header)))
     assert declared == sorted(pkg.EXPORTED_SYMBOLS)
     lib = ctypes.CDLL(pkg.library_path())
     for name in declared:

@@ -1,4 +1,6 @@
 """Pins for the oracle's radial bases (Eqs. 6-10, 13, 15-19)."""
+import os
+
 import mpmath
 import numpy as np
 import pytest
@@ -96,13 +98,31 @@ def test_gto_closed_form_against_radial_bessel_integral():
 
 def test_gto_single_neighbour_values():
     # A neighbour of another species on +z at 2.0 A, r_cut = 5, n_max = 4, sigma = 0.5:
-    # c_nl0 = sqrt((2l+1)/4 pi) F_nl(d).  Reference digits from an independent 40-digit
-    # evaluation of the radial Bessel integral (Eqs. 11-12).
-    ref0 = [1.1370509431e-02, -5.9880540027e-02, 1.0083928455e-02, 1.8909487433e-01]
-    ref2 = [2.2217362983e-02, -7.3158075793e-02, 9.1145153052e-02, 3.5394612354e-01]
+    # c_nl0 = sqrt((2l+1)/4 pi) F_nl(d).  The reference digits come from tests/golden/make_gto_single_neighbour.py,
+    # which evaluates Eqs. 1, 3, 8-11 in 40-digit arithmetic without the oracle (Loewdin root by a matrix iteration,
+    # radial integral by quadrature); they pin beta as the principal root of Eq. 9.
+    golden = np.loadtxt(os.path.join(os.path.dirname(__file__), "golden", "gto_single_neighbour.txt"))
+    ref = {l: golden[golden[:, 0] == l][:, 2] for l in (0, 2)}
+    assert len(ref[0]) == 4 and len(ref[2]) == 4
     F, _ = basis.gto_radial([2.0], 5.0, 4, 3, 0.5)
-    np.testing.assert_allclose(np.sqrt(1 / (4 * np.pi)) * F[:, 0, 0], ref0, rtol=2e-10)
-    np.testing.assert_allclose(np.sqrt(5 / (4 * np.pi)) * F[:, 2, 0], ref2, rtol=2e-10)
+    np.testing.assert_allclose(np.sqrt(1 / (4 * np.pi)) * F[:, 0, 0], ref[0], rtol=2e-10)
+    np.testing.assert_allclose(np.sqrt(5 / (4 * np.pi)) * F[:, 2, 0], ref[2], rtol=2e-10)
+
+
+@pytest.mark.parametrize("r_cut,n_max,l_max", [(5.0, 4, 3), (6.0, 8, 6), (6.0, 12, 12)])
+def test_lowdin_matrices_are_the_positive_definite_roots(r_cut, n_max, l_max):
+    # beta S beta = 1 and symmetry also hold for the non-principal symmetric roots (eigenvalue signs flipped);
+    # Eq. 9 means the principal one, whose eigenvalues are all positive.  Checked in 60-digit arithmetic on the
+    # extended-precision entries.
+    beta = basis.gto_beta(r_cut, n_max, l_max)
+    with mpmath.workdps(60):
+        for l in range(l_max + 1):
+            B = mpmath.matrix([[mpmath.mpf(repr(float(x))) + mpmath.mpf(float(x - np.longdouble(float(x)))) for x in row] for row in beta[l]])
+            lam = mpmath.eigsy((B + B.T) / 2, eigvals_only=True)
+            assert min(lam) > 0, f"l = {l}: smallest eigenvalue {min(lam)}"
+        W = basis.poly_w(min(n_max, 8))
+        Wm = mpmath.matrix([[mpmath.mpf(float(x)) for x in row] for row in W])
+        assert min(mpmath.eigsy((Wm + Wm.T) / 2, eigvals_only=True)) > 0
 
 
 def test_gto_onsite_is_the_zero_distance_limit():
