@@ -1,17 +1,19 @@
 // The descriptor-only kernel: expansion coefficients (Eq. 13 / Eqs. 18-19) and the power spectrum
 // (Eq. 4) of every centre, one WARP per centre, persistent CTAs that draw centres from a counter.
 //
-// This build is bound by FP32 arithmetic and by shared-memory bandwidth, not by HBM, so the layout is
+// This build is bound by FP32 issue slots and by shared-memory bandwidth, not by HBM, so the layout is
 // chosen for few instructions and few shared-memory wavefronts per pair:
 //   * the radial table (value polynomials, re-laid as [interval][l][n][6]) sits in shared memory once
 //     per CTA when it fits, so that a lookup is three conflict-free 8-byte loads per lane;
-//   * pairs are taken species by species through a small ring (the pair list is re-read once per
-//     species), staged 16 at a time: solid harmonics with a lane per pair from the fully unrolled
-//     Q_l^m recursion, radial factors with lanes on the channels (l, n);
+//   * the pairs of a centre (up to 128 at a time) are fetched and their geometry formed in registers
+//     in one go, ranked by species with ballots, and staged 16 at a time in species order: solid
+//     harmonics with a lane per pair from the fully unrolled Q_l^m recursion, radial factors with
+//     lanes on the channels (l, n);
 //   * accumulation c[l,m][n] += S_lm G_nl is register-tiled: a lane owns four consecutive m of one l
-//     times all n (an outer product of 4 x n_max per pair from 4 + n_max/4 shared loads); with at
-//     most 16 such tiles the two half-warps work on two pairs at once.  Sums stay in registers over
-//     all pairs of a species and go to the centre's tile c[lm][species, n] once per species;
+//     times all n (an outer product of 4 x n_max per pair from one 16-byte load of S and n_max/4 of
+//     G); with at most 16 such tiles the two half-warps work on two pairs at once.  Sums stay in
+//     registers over all pairs of a species and are added to the centre's tile c[lm][species, n]
+//     once per species; the staging rows are laid out so that all these loads are conflict-free;
 //   * Eq. 4 is the Gram matrix of that tile per l: lanes take 4 x 4 blocks of (species, n) pairs,
 //     two 16-byte loads per 16 multiply-adds, and the feature row is put together in shared memory
 //     and written out in order.
@@ -22,49 +24,57 @@
 namespace soap {
 
 constexpr int kDescChunk = 16;                    // pairs staged at once by a warp
-constexpr int kDescRing = kDescChunk + 32;        // ring of pair geometry (a block of 32 keys may arrive on top of a partial chunk)
+constexpr int kDescGroup = 128;                   // pairs whose geometry a warp holds in registers (four per lane)
 constexpr int kDescMaxWarps = 12;                 // warps per CTA (one CTA per SM)
 
-// harmonic tables up to l = 12, filled by desc_constants(): a_lm (sqrt2 folded in for m > 0), index l(l+1)/2 + m
+// harmonic normalisation up to l = 12, filled by desc_constants(): a_lm (sqrt2 folded in for m > 0), index l(l+1)/2 + m
 __device__ __constant__ float kd_norm[91] = {0};
 
-__host__ __device__ constexpr int desc_tiles(int l_max) {
+// tiles of four consecutive m of one l: tile index of the first tile of row l, and their number up to l_max
+__host__ __device__ constexpr int desc_tile_base(int l) {
     int t = 0;
-    for (int l = 0; l <= l_max; ++l) t += (2 * l + 1 + 3) / 4;
+    for (int k = 0; k < l; ++k) t += (2 * k + 1 + 3) / 4;
     return t;
 }
+__host__ __device__ constexpr int desc_tiles(int l_max) { return desc_tile_base(l_max + 1); }
 // n_max is padded to a multiple of four (NP = 4, 8, 12 or 16 is the template parameter; the padding channels have
 // all-zero table rows, so they cost arithmetic but need no special cases)
 __host__ __device__ constexpr int desc_np(int n_max) { return (n_max + 3) & ~3; }
+// words per pair of the harmonics staging: the tiles, four words each, padded to an odd number of 16-byte chunks so
+// that the 16-byte stores of eight lanes (eight pairs) fall into eight different bank groups
+__host__ __device__ constexpr int desc_s_row(int l_max) { return 4 * (desc_tiles(l_max) | 1); }
+// words per l of the radial staging: n padded so that the 16-byte chunks of consecutive l fall into different bank groups
+__host__ __device__ constexpr int desc_g_l(int np) { return np + (((np / 4) & 1) ? 0 : 4); }
 
 // Shared memory in 4-byte words: [table (optional)] then one region per warp:
-//   c [LM][S NP] | S staging [chunk][LM|1] (+4) | G staging [chunk][L1 NP] | ring [kDescRing][8]
+//   c [LM][S NP] | S staging [chunk][s_row] | G staging [chunk][L1 g_l] | pair staging [chunk][8]
 // The feature row is assembled on top of the staging area when it fits there.
 struct DescLayout {
     int table, warp0, per_warp, c, sS, sG, ring, slab_words, total;
 };
 __host__ __device__ inline DescLayout make_desc_layout(int S, int np, int l_max, int warps, int table_words) {
-    const int L1 = l_max + 1, LM = L1 * L1, LMP = LM | 1;
+    const int L1 = l_max + 1, LM = L1 * L1;
     DescLayout o;
     o.table = 0;
     o.warp0 = (table_words + 3) & ~3;
     int off = 0;
     o.c = off; off += LM * S * np;
-    o.sS = off; off += (kDescChunk * LMP + 4 + 3) & ~3;
-    o.sG = off; off += kDescChunk * L1 * np;
-    o.ring = off; off += kDescRing * 8;
+    o.sS = off; off += kDescChunk * desc_s_row(l_max);
+    o.sG = off; off += kDescChunk * L1 * desc_g_l(np);
+    o.ring = off; off += kDescChunk * 8;
     o.slab_words = off - o.sS;
     o.per_warp = off;
     o.total = o.warp0 + warps * off;
     return o;
 }
 
-// Real solid harmonics S_lm(d) = r^l Y_lm of one displacement, every (l, m), written to out[l^2 + l + m]:
+// Real solid harmonics S_lm(d) = r^l Y_lm of one displacement, every (l, m), written as 16-byte tiles: tile
+// desc_tile_base(l) + j holds m = 4j - l .. 4j + 3 - l of row l (zeros beyond m = l):
 //   S_{l,+m} = a_lm Q_l^m Re (x+iy)^m,  S_{l,-m} = a_lm Q_l^m Im (x+iy)^m,
 //   Q_m^m = (2m-1)!!,  (l+1-m) Q_{l+1}^m = (2l+1) z Q_l^m - (l+m) r^2 Q_{l-1}^m.
 // Fully unrolled: every index is an immediate and the Q's live in registers.
 template <int L>
-__device__ __forceinline__ void harmonics_all(float x, float y, float z, float r2, float* __restrict__ out) {
+__device__ __forceinline__ void harmonics_tiles(float x, float y, float z, float r2, float4* __restrict__ out) {
     float cm[L + 1], sm[L + 1];                   // (x+iy)^m
     cm[0] = 1.f; sm[0] = 0.f;
 #pragma unroll
@@ -80,6 +90,9 @@ __device__ __forceinline__ void harmonics_all(float x, float y, float z, float r
     for (int l = 0; l <= L; ++l) {
         if (l > 0) dfact *= (float)(2 * l - 1);
         const float zl = (float)(2 * l - 1) * z;
+        float row[2 * L + 4];                     // S_{l,m} at index m + l
+#pragma unroll
+        for (int i = 0; i < 2 * L + 4; ++i) row[i] = 0.f;
 #pragma unroll
         for (int m = 0; m <= l; ++m) {
             float q;
@@ -88,9 +101,12 @@ __device__ __forceinline__ void harmonics_all(float x, float y, float z, float r
             q2[m] = q1[m];
             q1[m] = q;
             const float aq = kd_norm[l * (l + 1) / 2 + m] * q;
-            out[l * l + l + m] = aq * cm[m];
-            if (m) out[l * l + l - m] = aq * sm[m];
+            row[l + m] = aq * cm[m];
+            if (m) row[l - m] = aq * sm[m];
         }
+#pragma unroll
+        for (int j = 0; j < (2 * l + 4) / 4; ++j)
+            out[desc_tile_base(l) + j] = make_float4(row[4 * j], row[4 * j + 1], row[4 * j + 2], row[4 * j + 3]);
     }
 }
 
@@ -98,8 +114,9 @@ __device__ __forceinline__ void harmonics_all(float x, float y, float z, float r
 // species pair, power spectrum out).  TS: the radial table is in shared memory.
 template <int L, int NP, bool PLAIN, bool TS>
 __global__ void __launch_bounds__(kDescMaxWarps * 32, 1) desc_kernel(const CenterParams p) {
-    constexpr int L1 = L + 1, LM = L1 * L1, LMP = LM | 1;
-    constexpr int NCHP = L1 * NP;
+    constexpr int L1 = L + 1, LM = L1 * L1;
+    constexpr int NCHP = L1 * NP;                                        // channels (l, n), n padded
+    constexpr int SROW = desc_s_row(L), GL = desc_g_l(NP), GROW = L1 * GL;
     constexpr int T = desc_tiles(L);
     constexpr int HALVES = T <= 16 ? 2 : 1, LANES_T = 32 / HALVES;
     constexpr int TPL = (T + LANES_T - 1) / LANES_T;                     // tiles per lane (1, or 2 from l_max = 10 on)
@@ -128,22 +145,30 @@ __global__ void __launch_bounds__(kDescMaxWarps * 32, 1) desc_kernel(const Cente
 
     float* const wbase = smem + lay.warp0 + wid * lay.per_warp;
     float* const c_t = wbase + lay.c;                                               // [LM][SNP]
-    float* const sS = wbase + lay.sS;                                               // [chunk][LMP]
-    float* const sG = wbase + lay.sG;                                               // [chunk][NCHP]
-    float4* const ring_d = reinterpret_cast<float4*>(wbase + lay.ring);             // [ring] dx, dy, dz, r
-    int4* const ring_i = reinterpret_cast<int4*>(wbase + lay.ring + 4 * kDescRing); // [ring] interval, t, species, weight
+    float4* const sS4 = reinterpret_cast<float4*>(wbase + lay.sS);                  // [chunk][SROW / 4] tiles of four m
+    float* const sG = wbase + lay.sG;                                               // [chunk][L1][GL]
+    float4* const ring_d = reinterpret_cast<float4*>(wbase + lay.ring);             // [chunk] dx, dy, dz, r
+    int4* const ring_i = reinterpret_cast<int4*>(wbase + lay.ring + 4 * kDescChunk);// [chunk] interval, t, species, weight
     float* const slab = wbase + lay.sS;
     const float2* const tab = TS ? reinterpret_cast<const float2*>(smem) : reinterpret_cast<const float2*>(p.table_ln);
 
-    // the tiles of this lane: (l, first m index, number of valid rows)
+    // the tiles of this lane: l, tile index, first row (l^2 + 4 j) and number of valid rows
     const int half = HALVES == 2 ? lane >> 4 : 0;
-    int t_l[TPL], t_lm0[TPL], t_kv[TPL];
+    int t_l[TPL], t_idx[TPL], t_lm0[TPL], t_kv[TPL];
 #pragma unroll
     for (int tp = 0; tp < TPL; ++tp) {
         int t = tp * LANES_T + (lane & (LANES_T - 1)), l = 0;
+        t_idx[tp] = t < T ? t : 0;
         if (t >= T) { t_l[tp] = 0; t_lm0[tp] = 0; t_kv[tp] = 0; continue; }
         while (t >= (2 * l + 4) / 4) { t -= (2 * l + 4) / 4; ++l; }
         t_l[tp] = l; t_lm0[tp] = l * l + 4 * t; t_kv[tp] = min(4, 2 * l + 1 - 4 * t);
+    }
+    // where this lane puts the radial factors it evaluates: channel ch = l NP + n of round rr goes to word l GL + n
+    int g_word[ROUNDS];
+#pragma unroll
+    for (int rr = 0; rr < ROUNDS; ++rr) {
+        const int ch = rr * 32 + lane, l = ch / NP;
+        g_word[rr] = l * GL + (ch - l * NP);
     }
     const bool periodic = p.geom.pbc[0] | p.geom.pbc[1] | p.geom.pbc[2];
     const long long n_work = o_cbar ? 1 : p.n_centers;
@@ -164,156 +189,174 @@ __global__ void __launch_bounds__(kDescMaxWarps * 32, 1) desc_kernel(const Cente
         for (int e = lane; e < LM * SNP / 4; e += 32) reinterpret_cast<float4*>(c_t)[e] = make_float4(0.f, 0.f, 0.f, 0.f);
         __syncwarp();
 
-#pragma unroll 1
-        for (int ip = 0; ip < NPASS; ++ip) {
-            const int n0 = ip * NB;
-            float acc[TPL][4][NB];
+        for (int g0 = 0; g0 < k_pairs; g0 += kDescGroup) {
+            // ---- geometry of up to 128 pairs, four per lane, all loads in flight together ----
+            const int kg = min(kDescGroup, k_pairs - g0);
+            int sp[4], pos_sorted[4];
+            float4 dd[4];
+            int2 qt[4];                                                     // interval, offset bits
+            float ww[4];
+            unsigned long long key[4];
 #pragma unroll
-            for (int tp = 0; tp < TPL; ++tp)
+            for (int b = 0; b < 4; ++b) {
+                const int e = g0 + 32 * b + lane;
+                key[b] = e < k_pairs ? p.pair_key[pair_base + e] : 0ull;
+                ww[b] = (o_pw && e < k_pairs) ? o_pw[pair_base + e].x : 1.f;
+            }
 #pragma unroll
-                for (int k = 0; k < 4; ++k)
+            for (int b = 0; b < 4; ++b) {
+                const int e = g0 + 32 * b + lane;
+                sp[b] = -1;
+                dd[b] = make_float4(0.f, 0.f, 0.f, 0.f);
+                qt[b] = make_int2(0, 0);
+                pos_sorted[b] = -1;
+                if (e < k_pairs) {
+                    const int j = key_atom(key[b]);
+                    sp[b] = S == 1 ? 0 : p.species_idx[j];
+                    double dx = (double)p.pos[3 * (long long)j] - (double)xi;
+                    double dy = (double)p.pos[3 * (long long)j + 1] - (double)yi;
+                    double dz = (double)p.pos[3 * (long long)j + 2] - (double)zi;
+                    if (periodic) {
+                        int sh[3];
+                        key_shift(key[b], sh);
+                        dx += sh[0] * p.geom.cell[0] + sh[1] * p.geom.cell[3] + sh[2] * p.geom.cell[6];
+                        dy += sh[0] * p.geom.cell[1] + sh[1] * p.geom.cell[4] + sh[2] * p.geom.cell[7];
+                        dz += sh[0] * p.geom.cell[2] + sh[1] * p.geom.cell[5] + sh[2] * p.geom.cell[8];
+                    }
+                    const double r = sqrt(dx * dx + dy * dy + dz * dz);
+                    // interval and offset in the radial table, in fp64 so that the offset keeps its digits
+                    const double u = r * (double)p.inv_h;
+                    const int qi = min((int)u, p.n_intervals - 1);
+                    dd[b] = make_float4((float)dx, (float)dy, (float)dz, (float)r);
+                    qt[b] = make_int2(qi, __float_as_int((float)(u - qi)));
+                }
+            }
+            // position of every pair in species order (stable): ballots, no memory traffic
+            {
+                int base = 0;
+                for (int s = 0; s < S; ++s)
 #pragma unroll
-                    for (int n = 0; n < NB; ++n) acc[tp][k][n] = 0.f;
-            int cur = -1, fill = 0;
+                    for (int b = 0; b < 4; ++b) {
+                        const unsigned m = __ballot_sync(0xffffffffu, sp[b] == s);
+                        if (sp[b] == s) pos_sorted[b] = base + __popc(m & ((1u << lane) - 1));
+                        base += __popc(m);
+                    }
+            }
 
-            // sums of species s (columns n0 .. n0 + NB - 1) go to the centre's tile; the two half-warps add up first
-            auto flush = [&](int s) {
+#pragma unroll 1
+            for (int ip = 0; ip < NPASS; ++ip) {
+                const int n0 = ip * NB;
+                float acc[TPL][4][NB];
 #pragma unroll
                 for (int tp = 0; tp < TPL; ++tp)
 #pragma unroll
-                    for (int k = 0; k < 4; ++k) {
-                        float v[NB];
+                    for (int k = 0; k < 4; ++k)
 #pragma unroll
-                        for (int n = 0; n < NB; ++n) {
-                            v[n] = acc[tp][k][n];
-                            if (HALVES == 2) v[n] += __shfl_xor_sync(0xffffffffu, v[n], 16);
-                            acc[tp][k][n] = 0.f;
-                        }
-                        if (k < t_kv[tp] && (HALVES == 1 || (k >> 1) == half)) {
-                            float4* dst = reinterpret_cast<float4*>(c_t + (t_lm0[tp] + k) * SNP + s * NP + n0);
-#pragma unroll
-                            for (int n4 = 0; n4 < NB / 4; ++n4)
-                                if (NPASS == 1 || n0 + 4 * n4 < NP) dst[n4] = make_float4(v[4 * n4], v[4 * n4 + 1], v[4 * n4 + 2], v[4 * n4 + 3]);
-                        }
-                    }
-            };
+                        for (int n = 0; n < NB; ++n) acc[tp][k][n] = 0.f;
+                int cur = -1;
 
-            // harmonics, radial factors and the accumulation of the first n_stage entries of the ring
-            auto process = [&](int n_stage) {
-                if (lane < n_stage) {
-                    const float4 d = ring_d[lane];
-                    harmonics_all<L>(d.x, d.y, d.z, d.w * d.w, sS + lane * LMP);
-                }
-#pragma unroll 2
-                for (int pr = 0; pr < n_stage; ++pr) {
-                    const int4 gi = ring_i[pr];
-                    const float t = __int_as_float(gi.y);
-                    const float2* row = tab + (size_t)gi.x * (NCHP * 3);
+                // sums of species s (columns n0 .. n0 + NB - 1) are added to the centre's tile; the two half-warps add up first
+                auto flush = [&](int s) {
 #pragma unroll
-                    for (int rr = 0; rr < ROUNDS; ++rr) {
-                        const int ch = rr * 32 + lane;
-                        if (ROUNDS * 32 == NCHP || ch < NCHP) {
-                            const float2 a = TS ? row[ch * 3] : __ldg(row + ch * 3);
-                            const float2 b = TS ? row[ch * 3 + 1] : __ldg(row + ch * 3 + 1);
-                            const float2 c = TS ? row[ch * 3 + 2] : __ldg(row + ch * 3 + 2);
-                            float v = fmaf(c.y, t, c.x);
-                            v = fmaf(v, t, b.y);
-                            v = fmaf(v, t, b.x);
-                            v = fmaf(v, t, a.y);
-                            v = fmaf(v, t, a.x);
-                            if (!PLAIN) v *= __int_as_float(gi.w);
-                            sG[pr * NCHP + ch] = v;
+                    for (int tp = 0; tp < TPL; ++tp)
+#pragma unroll
+                        for (int k = 0; k < 4; ++k) {
+                            float v[NB];
+#pragma unroll
+                            for (int n = 0; n < NB; ++n) {
+                                v[n] = acc[tp][k][n];
+                                if (HALVES == 2) v[n] += __shfl_xor_sync(0xffffffffu, v[n], 16);
+                                acc[tp][k][n] = 0.f;
+                            }
+                            if (k < t_kv[tp] && (HALVES == 1 || (k >> 1) == half)) {
+                                float4* dst = reinterpret_cast<float4*>(c_t + (t_lm0[tp] + k) * SNP + s * NP + n0);
+#pragma unroll
+                                for (int n4 = 0; n4 < NB / 4; ++n4)
+                                    if (NPASS == 1 || n0 + 4 * n4 < NP) {
+                                        float4 o = dst[n4];
+                                        o.x += v[4 * n4]; o.y += v[4 * n4 + 1]; o.z += v[4 * n4 + 2]; o.w += v[4 * n4 + 3];
+                                        dst[n4] = o;
+                                    }
+                            }
+                        }
+                };
+
+                for (int c0 = 0; c0 < kg; c0 += kDescChunk) {
+                    const int n_stage = min(kDescChunk, kg - c0);
+                    // the pairs at sorted positions c0 .. c0 + 15 go to the staging slots
+#pragma unroll
+                    for (int b = 0; b < 4; ++b)
+                        if ((unsigned)(pos_sorted[b] - c0) < (unsigned)kDescChunk) {
+                            ring_d[pos_sorted[b] - c0] = dd[b];
+                            ring_i[pos_sorted[b] - c0] = make_int4(qt[b].x, qt[b].y, sp[b], __float_as_int(ww[b]));
+                        }
+                    __syncwarp();
+                    // solid harmonics: a lane per pair
+                    if (lane < n_stage) {
+                        const float4 d = ring_d[lane];
+                        harmonics_tiles<L>(d.x, d.y, d.z, d.w * d.w, sS4 + lane * (SROW / 4));
+                    }
+                    // radial factors: lanes on the channels, pairs in turn
+#pragma unroll 4
+                    for (int pr = 0; pr < n_stage; ++pr) {
+                        const int4 gi = ring_i[pr];
+                        const float t = __int_as_float(gi.y);
+                        const float2* row = tab + (size_t)gi.x * (NCHP * 3);
+#pragma unroll
+                        for (int rr = 0; rr < ROUNDS; ++rr) {
+                            const int ch = rr * 32 + lane;
+                            if (ROUNDS * 32 == NCHP || ch < NCHP) {
+                                const float2 a = TS ? row[ch * 3] : __ldg(row + ch * 3);
+                                const float2 b = TS ? row[ch * 3 + 1] : __ldg(row + ch * 3 + 1);
+                                const float2 c = TS ? row[ch * 3 + 2] : __ldg(row + ch * 3 + 2);
+                                float v = fmaf(c.y, t, c.x);
+                                v = fmaf(v, t, b.y);
+                                v = fmaf(v, t, b.x);
+                                v = fmaf(v, t, a.y);
+                                v = fmaf(v, t, a.x);
+                                if (!PLAIN) v *= __int_as_float(gi.w);
+                                sG[pr * GROW + g_word[rr]] = v;
+                            }
                         }
                     }
-                }
-                __syncwarp();
-                const int tag = lane < n_stage ? ring_i[lane].z : -1;
-                for (int s = 0; s < S; ++s) {
-                    const unsigned mask = __ballot_sync(0xffffffffu, tag == s);
-                    if (!mask) continue;
-                    const int a = __ffs(mask) - 1, b = a + __popc(mask);       // contiguous: the ring is filled species by species
-                    if (s != cur) {
-                        if (cur >= 0) flush(cur);
-                        cur = s;
-                    }
-                    for (int q = a + half; q < b; q += HALVES) {
-                        const float* sp = sS + q * LMP;
-                        const float4* gp = reinterpret_cast<const float4*>(sG + q * NCHP + n0);
+                    __syncwarp();
+                    const int tag = lane < n_stage ? ring_i[lane].z : -1;
+                    for (int s = 0; s < S; ++s) {
+                        const unsigned mask = __ballot_sync(0xffffffffu, tag == s);
+                        if (!mask) continue;
+                        const int a = __ffs(mask) - 1, b = a + __popc(mask);       // contiguous: staged in species order
+                        if (s != cur) {
+                            if (cur >= 0) flush(cur);
+                            cur = s;
+                        }
+#pragma unroll 2
+                        for (int q = a + half; q < b; q += HALVES) {
+                            const float4* sp4 = sS4 + q * (SROW / 4);
+                            const float4* gp = reinterpret_cast<const float4*>(sG + q * GROW + n0);
 #pragma unroll
-                        for (int tp = 0; tp < TPL; ++tp) {
-                            float h[4];
+                            for (int tp = 0; tp < TPL; ++tp) {
+                                const float4 h4 = sp4[t_idx[tp]];
+                                const float h[4] = {h4.x, h4.y, h4.z, h4.w};
 #pragma unroll
-                            for (int k = 0; k < 4; ++k) h[k] = sp[t_lm0[tp] + k];
+                                for (int n4 = 0; n4 < NB / 4; ++n4) {
+                                    if (NPASS > 1 && n0 + 4 * n4 >= NP) break;
+                                    const float4 g = gp[t_l[tp] * (GL / 4) + n4];
 #pragma unroll
-                            for (int n4 = 0; n4 < NB / 4; ++n4) {
-                                if (NPASS > 1 && n0 + 4 * n4 >= NP) break;
-                                const float4 g = gp[t_l[tp] * (NP / 4) + n4];
-#pragma unroll
-                                for (int k = 0; k < 4; ++k) {
-                                    acc[tp][k][4 * n4] = fmaf(h[k], g.x, acc[tp][k][4 * n4]);
-                                    acc[tp][k][4 * n4 + 1] = fmaf(h[k], g.y, acc[tp][k][4 * n4 + 1]);
-                                    acc[tp][k][4 * n4 + 2] = fmaf(h[k], g.z, acc[tp][k][4 * n4 + 2]);
-                                    acc[tp][k][4 * n4 + 3] = fmaf(h[k], g.w, acc[tp][k][4 * n4 + 3]);
+                                    for (int k = 0; k < 4; ++k) {
+                                        acc[tp][k][4 * n4] = fmaf(h[k], g.x, acc[tp][k][4 * n4]);
+                                        acc[tp][k][4 * n4 + 1] = fmaf(h[k], g.y, acc[tp][k][4 * n4 + 1]);
+                                        acc[tp][k][4 * n4 + 2] = fmaf(h[k], g.z, acc[tp][k][4 * n4 + 2]);
+                                        acc[tp][k][4 * n4 + 3] = fmaf(h[k], g.w, acc[tp][k][4 * n4 + 3]);
+                                    }
                                 }
                             }
                         }
                     }
-                }
-                __syncwarp();
-            };
-
-            for (int s = 0; s < S; ++s) {
-                for (int e0 = 0; e0 < k_pairs; e0 += 32) {
-                    const int e = e0 + lane;
-                    bool match = false;
-                    unsigned long long key = 0;
-                    int j = 0;
-                    if (e < k_pairs) {
-                        key = p.pair_key[pair_base + e];
-                        j = key_atom(key);
-                        match = S == 1 || p.species_idx[j] == s;
-                    }
-                    const unsigned m = __ballot_sync(0xffffffffu, match);
-                    if (!m) continue;
-                    if (match) {
-                        double dx = (double)p.pos[3 * (long long)j] - (double)xi;
-                        double dy = (double)p.pos[3 * (long long)j + 1] - (double)yi;
-                        double dz = (double)p.pos[3 * (long long)j + 2] - (double)zi;
-                        if (periodic) {
-                            int sh[3];
-                            key_shift(key, sh);
-                            dx += sh[0] * p.geom.cell[0] + sh[1] * p.geom.cell[3] + sh[2] * p.geom.cell[6];
-                            dy += sh[0] * p.geom.cell[1] + sh[1] * p.geom.cell[4] + sh[2] * p.geom.cell[7];
-                            dz += sh[0] * p.geom.cell[2] + sh[1] * p.geom.cell[5] + sh[2] * p.geom.cell[8];
-                        }
-                        const double r = sqrt(dx * dx + dy * dy + dz * dz);
-                        // interval and offset in the radial table, in fp64 so that the offset keeps its digits
-                        const double u = r * (double)p.inv_h;
-                        const int qi = min((int)u, p.n_intervals - 1);
-                        const int slot = fill + __popc(m & ((1u << lane) - 1));
-                        ring_d[slot] = make_float4((float)dx, (float)dy, (float)dz, (float)r);
-                        ring_i[slot] = make_int4(qi, __float_as_int((float)(u - qi)), s,
-                                                 __float_as_int(o_pw ? o_pw[pair_base + e].x : 1.f));
-                    }
-                    fill += __popc(m);
                     __syncwarp();
-                    while (fill >= kDescChunk) {
-                        process(kDescChunk);
-                        // move what is left to the front of the ring
-                        const int rest = fill - kDescChunk;
-                        float4 d4 = make_float4(0.f, 0.f, 0.f, 0.f);
-                        int4 i4 = make_int4(0, 0, 0, 0);
-                        if (lane < rest) { d4 = ring_d[kDescChunk + lane]; i4 = ring_i[kDescChunk + lane]; }
-                        __syncwarp();
-                        if (lane < rest) { ring_d[lane] = d4; ring_i[lane] = i4; }
-                        __syncwarp();
-                        fill = rest;
-                    }
                 }
+                if (cur >= 0) flush(cur);
+                __syncwarp();
             }
-            if (fill > 0) process(fill);
-            if (cur >= 0) flush(cur);
-            __syncwarp();
         }
 
         // on-site term: the centre's own Gaussian, l = 0 only (second term of Eq. 13)
@@ -381,23 +424,29 @@ __global__ void __launch_bounds__(kDescMaxWarps * 32, 1) desc_kernel(const Cente
             if (active) {
                 const float kl = __ldg(p.kl + l);
                 const int mu = (4 * ta) / NP, nu = (4 * tb) / NP, na = 4 * ta - mu * NP, nb = 4 * tb - nu * NP;
-                int off;
-                if (o_cross) {
-                    const int before = mu * S - mu * (mu - 1) / 2 + (nu - mu), diag = mu + (nu > mu ? 1 : 0);
-                    off = diag * TRI + (before - diag) * SQ;
+                if (mu < nu) {
+                    // off-diagonal species block: rows n1 of n_max (l_max+1) features
+                    const int before = mu * S - mu * (mu - 1) / 2 + (nu - mu), diag = mu + 1;
+                    float* o = dst + diag * TRI + (before - diag) * SQ + (na * NMAX + nb) * L1 + l;
+#pragma unroll
+                    for (int i = 0; i < 4; ++i)
+#pragma unroll
+                        for (int j = 0; j < 4; ++j)
+                            if (na + i < NMAX && nb + j < NMAX) o[(i * NMAX + j) * L1] = kl * g[i][j];
                 } else {
-                    off = mu * TRI;
-                }
+                    // diagonal species block: rows n1 hold n2 = n1 .. n_max - 1
+                    const int before = o_cross ? mu * S - mu * (mu - 1) / 2 : 0;
+                    float* o = dst + (o_cross ? mu * TRI + (before - mu) * SQ : mu * TRI) + l;
 #pragma unroll
-                for (int i = 0; i < 4; ++i)
+                    for (int i = 0; i < 4; ++i) {
+                        const int n1 = na + i, rs = n1 * NMAX - n1 * (n1 - 1) / 2 - n1;      // row start minus n1
 #pragma unroll
-                    for (int j = 0; j < 4; ++j) {
-                        const int n1 = na + i, n2 = nb + j;
-                        if (n1 < NMAX && n2 < NMAX && (mu < nu || n1 <= n2)) {
-                            const int within = mu == nu ? n1 * NMAX - n1 * (n1 - 1) / 2 + (n2 - n1) : n1 * NMAX + n2;
-                            dst[off + within * L1 + l] = kl * g[i][j];
+                        for (int j = 0; j < 4; ++j) {
+                            const int n2 = nb + j;
+                            if (n1 < NMAX && n2 < NMAX && n1 <= n2) o[(rs + n2) * L1] = kl * g[i][j];
                         }
                     }
+                }
             }
         }
         __syncwarp();

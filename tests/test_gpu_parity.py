@@ -29,6 +29,17 @@ def col_err(a, ref, axes):
     return float((np.abs(a - ref).max(axis=axes) / np.maximum(np.abs(ref).max(axis=axes), 1e-8)).max())
 
 
+def same_values(a, b, tol=DESC_TOL):
+    """Two builds of the same quantity by different kernels (the descriptor-only build has a kernel of its own,
+    with another order of summation): equal within the parity tolerance, column by column, not bit for bit."""
+    a = a.detach().cpu().numpy() if hasattr(a, "detach") else np.asarray(a)
+    b = b.detach().cpu().numpy() if hasattr(b, "detach") else np.asarray(b)
+    if a.shape != b.shape:
+        return False
+    a2, b2 = a.reshape(-1, a.shape[-1]).astype(np.float64), b.reshape(-1, b.shape[-1]).astype(np.float64)
+    return a2.size == 0 or col_err(a2, b2, 0) < tol
+
+
 def dev(struct):
     return torch.from_numpy(struct.positions).cuda(), torch.from_numpy(struct.numbers).cuda()
 
