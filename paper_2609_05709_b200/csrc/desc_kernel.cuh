@@ -3,8 +3,9 @@
 //
 // This build is bound by FP32 issue slots and by shared-memory bandwidth, not by HBM, so the layout is
 // chosen for few instructions and few shared-memory wavefronts per pair:
-//   * the radial table (value polynomials, re-laid as [interval][l][n][6]) sits in shared memory once
-//     per CTA when it fits, so that a lookup is three conflict-free 8-byte loads per lane;
+//   * the radial table (value polynomials, re-laid as [interval][l][n / 2][6][2]) sits in shared memory
+//     once per CTA when it fits; a lane evaluates two adjacent n at once from three conflict-free 16-byte
+//     loads and five packed multiply-adds (fma.rn.f32x2: one issue slot for two multiply-adds);
 //   * the pairs of a centre (up to 128 at a time) are fetched and their geometry formed in registers
 //     in one go, ranked by species with ballots, and staged 16 at a time in species order: solid
 //     harmonics with a lane per pair from the fully unrolled Q_l^m recursion, radial factors with
@@ -122,7 +123,7 @@ __global__ void __launch_bounds__(kDescMaxWarps * 32, 1) desc_kernel(const Cente
     constexpr int TPL = (T + LANES_T - 1) / LANES_T;                     // tiles per lane (1, or 2 from l_max = 10 on)
     constexpr int NB = (TPL * NP * 4 <= 64) ? NP : 64 / (4 * TPL);      // n handled per pass (at most 64 accumulators)
     constexpr int NPASS = (NP + NB - 1) / NB;
-    constexpr int ROUNDS = (NCHP + 31) / 32;
+    constexpr int CPAIRS = NCHP / 2, ROUNDS = (CPAIRS + 31) / 32;       // lanes take pairs of adjacent n
     extern __shared__ __align__(16) float smem[];
     const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5, warps = blockDim.x >> 5;
     const bool o_cross = PLAIN || p.crossover, o_emit = !PLAIN && p.emit_coeff;
@@ -150,7 +151,7 @@ __global__ void __launch_bounds__(kDescMaxWarps * 32, 1) desc_kernel(const Cente
     float4* const ring_d = reinterpret_cast<float4*>(wbase + lay.ring);             // [chunk] dx, dy, dz, r
     int4* const ring_i = reinterpret_cast<int4*>(wbase + lay.ring + 4 * kDescChunk);// [chunk] interval, t, species, weight
     float* const slab = wbase + lay.sS;
-    const float2* const tab = TS ? reinterpret_cast<const float2*>(smem) : reinterpret_cast<const float2*>(p.table_ln);
+    const float4* const tab = TS ? reinterpret_cast<const float4*>(smem) : reinterpret_cast<const float4*>(p.table_ln);
 
     // the tiles of this lane: l, tile index, first row (l^2 + 4 j) and number of valid rows
     const int half = HALVES == 2 ? lane >> 4 : 0;
@@ -163,12 +164,13 @@ __global__ void __launch_bounds__(kDescMaxWarps * 32, 1) desc_kernel(const Cente
         while (t >= (2 * l + 4) / 4) { t -= (2 * l + 4) / 4; ++l; }
         t_l[tp] = l; t_lm0[tp] = l * l + 4 * t; t_kv[tp] = min(4, 2 * l + 1 - 4 * t);
     }
-    // where this lane puts the radial factors it evaluates: channel ch = l NP + n of round rr goes to word l GL + n
+    // where this lane puts the radial factors it evaluates: the channel pair cp = l NP/2 + n/2 of round rr goes to
+    // words l GL + n, l GL + n + 1
     int g_word[ROUNDS];
 #pragma unroll
     for (int rr = 0; rr < ROUNDS; ++rr) {
-        const int ch = rr * 32 + lane, l = ch / NP;
-        g_word[rr] = l * GL + (ch - l * NP);
+        const int cp = rr * 32 + lane, l = cp / (NP / 2);
+        g_word[rr] = l * GL + 2 * (cp - l * (NP / 2));
     }
     const bool periodic = p.geom.pbc[0] | p.geom.pbc[1] | p.geom.pbc[2];
     const long long n_work = o_cbar ? 1 : p.n_centers;
@@ -246,14 +248,15 @@ __global__ void __launch_bounds__(kDescMaxWarps * 32, 1) desc_kernel(const Cente
 #pragma unroll 1
             for (int ip = 0; ip < NPASS; ++ip) {
                 const int n0 = ip * NB;
-                float acc[TPL][4][NB];
+                float2 acc[TPL][4][NB / 2];
 #pragma unroll
                 for (int tp = 0; tp < TPL; ++tp)
 #pragma unroll
                     for (int k = 0; k < 4; ++k)
 #pragma unroll
-                        for (int n = 0; n < NB; ++n) acc[tp][k][n] = 0.f;
+                        for (int n = 0; n < NB / 2; ++n) acc[tp][k][n] = make_float2(0.f, 0.f);
                 int cur = -1;
+                const bool single = k_pairs <= kDescGroup;            // one group: every (row, species) is written once
 
                 // sums of species s (columns n0 .. n0 + NB - 1) are added to the centre's tile; the two half-warps add up first
                 auto flush = [&](int s) {
@@ -264,17 +267,21 @@ __global__ void __launch_bounds__(kDescMaxWarps * 32, 1) desc_kernel(const Cente
                             float v[NB];
 #pragma unroll
                             for (int n = 0; n < NB; ++n) {
-                                v[n] = acc[tp][k][n];
+                                v[n] = (n & 1) ? acc[tp][k][n / 2].y : acc[tp][k][n / 2].x;
                                 if (HALVES == 2) v[n] += __shfl_xor_sync(0xffffffffu, v[n], 16);
-                                acc[tp][k][n] = 0.f;
                             }
+#pragma unroll
+                            for (int n = 0; n < NB / 2; ++n) acc[tp][k][n] = make_float2(0.f, 0.f);
                             if (k < t_kv[tp] && (HALVES == 1 || (k >> 1) == half)) {
                                 float4* dst = reinterpret_cast<float4*>(c_t + (t_lm0[tp] + k) * SNP + s * NP + n0);
 #pragma unroll
                                 for (int n4 = 0; n4 < NB / 4; ++n4)
                                     if (NPASS == 1 || n0 + 4 * n4 < NP) {
-                                        float4 o = dst[n4];
-                                        o.x += v[4 * n4]; o.y += v[4 * n4 + 1]; o.z += v[4 * n4 + 2]; o.w += v[4 * n4 + 3];
+                                        float4 o = make_float4(v[4 * n4], v[4 * n4 + 1], v[4 * n4 + 2], v[4 * n4 + 3]);
+                                        if (!single) {
+                                            const float4 old = dst[n4];
+                                            o.x += old.x; o.y += old.y; o.z += old.z; o.w += old.w;
+                                        }
                                         dst[n4] = o;
                                     }
                             }
@@ -301,21 +308,23 @@ __global__ void __launch_bounds__(kDescMaxWarps * 32, 1) desc_kernel(const Cente
                     for (int pr = 0; pr < n_stage; ++pr) {
                         const int4 gi = ring_i[pr];
                         const float t = __int_as_float(gi.y);
-                        const float2* row = tab + (size_t)gi.x * (NCHP * 3);
+                        const float2 tt = make_float2(t, t);
+                        const float4* row = tab + (size_t)gi.x * (NCHP * 6 / 4);
 #pragma unroll
                         for (int rr = 0; rr < ROUNDS; ++rr) {
-                            const int ch = rr * 32 + lane;
-                            if (ROUNDS * 32 == NCHP || ch < NCHP) {
-                                const float2 a = TS ? row[ch * 3] : __ldg(row + ch * 3);
-                                const float2 b = TS ? row[ch * 3 + 1] : __ldg(row + ch * 3 + 1);
-                                const float2 c = TS ? row[ch * 3 + 2] : __ldg(row + ch * 3 + 2);
-                                float v = fmaf(c.y, t, c.x);
-                                v = fmaf(v, t, b.y);
-                                v = fmaf(v, t, b.x);
-                                v = fmaf(v, t, a.y);
-                                v = fmaf(v, t, a.x);
-                                if (!PLAIN) v *= __int_as_float(gi.w);
-                                sG[pr * GROW + g_word[rr]] = v;
+                            const int cp = rr * 32 + lane;
+                            if (ROUNDS * 32 == CPAIRS || cp < CPAIRS) {
+                                // coefficients of t^0 .. t^5 of two adjacent n, interleaved: (c0, c0', c1, c1'), (c2, c2', c3, c3'), (c4, c4', c5, c5')
+                                const float4 A = TS ? row[cp * 3] : __ldg(row + cp * 3);
+                                const float4 B = TS ? row[cp * 3 + 1] : __ldg(row + cp * 3 + 1);
+                                const float4 C = TS ? row[cp * 3 + 2] : __ldg(row + cp * 3 + 2);
+                                float2 v = __ffma2_rn(make_float2(C.z, C.w), tt, make_float2(C.x, C.y));
+                                v = __ffma2_rn(v, tt, make_float2(B.z, B.w));
+                                v = __ffma2_rn(v, tt, make_float2(B.x, B.y));
+                                v = __ffma2_rn(v, tt, make_float2(A.z, A.w));
+                                v = __ffma2_rn(v, tt, make_float2(A.x, A.y));
+                                if (!PLAIN) { const float wgt = __int_as_float(gi.w); v.x *= wgt; v.y *= wgt; }
+                                *reinterpret_cast<float2*>(sG + pr * GROW + g_word[rr]) = v;
                             }
                         }
                     }
@@ -336,17 +345,16 @@ __global__ void __launch_bounds__(kDescMaxWarps * 32, 1) desc_kernel(const Cente
 #pragma unroll
                             for (int tp = 0; tp < TPL; ++tp) {
                                 const float4 h4 = sp4[t_idx[tp]];
-                                const float h[4] = {h4.x, h4.y, h4.z, h4.w};
+                                const float2 h[4] = {make_float2(h4.x, h4.x), make_float2(h4.y, h4.y), make_float2(h4.z, h4.z),
+                                                     make_float2(h4.w, h4.w)};
 #pragma unroll
                                 for (int n4 = 0; n4 < NB / 4; ++n4) {
                                     if (NPASS > 1 && n0 + 4 * n4 >= NP) break;
                                     const float4 g = gp[t_l[tp] * (GL / 4) + n4];
 #pragma unroll
                                     for (int k = 0; k < 4; ++k) {
-                                        acc[tp][k][4 * n4] = fmaf(h[k], g.x, acc[tp][k][4 * n4]);
-                                        acc[tp][k][4 * n4 + 1] = fmaf(h[k], g.y, acc[tp][k][4 * n4 + 1]);
-                                        acc[tp][k][4 * n4 + 2] = fmaf(h[k], g.z, acc[tp][k][4 * n4 + 2]);
-                                        acc[tp][k][4 * n4 + 3] = fmaf(h[k], g.w, acc[tp][k][4 * n4 + 3]);
+                                        acc[tp][k][2 * n4] = __ffma2_rn(h[k], make_float2(g.x, g.y), acc[tp][k][2 * n4]);
+                                        acc[tp][k][2 * n4 + 1] = __ffma2_rn(h[k], make_float2(g.z, g.w), acc[tp][k][2 * n4 + 1]);
                                     }
                                 }
                             }
@@ -384,17 +392,21 @@ __global__ void __launch_bounds__(kDescMaxWarps * 32, 1) desc_kernel(const Cente
         float* const desc_row = p.out_desc + (o_cbar ? (size_t)0 : (size_t)c_idx * F);
         const bool staged = F <= lay.slab_words;
         float* const dst = staged ? slab : desc_row;
+        // Lanes take blocks of 4 x 4 (species, n) pairs (ta <= tb in units of four columns); a block's place in the
+        // feature row does not depend on l, so it is decoded once, and the lanes then walk down the l (with few
+        // blocks, several l side by side: group g of the lanes takes l = l_max - g, l_max - g - G, ...).
         constexpr int TB = NP / 4;                                   // 4-wide column tiles per species
         const int TA = S * TB;
         const int NTP = o_cross ? TA * (TA + 1) / 2 : S * (TB * (TB + 1) / 2);
-        const int n_tasks = NTP * L1;
+        const int G = NTP <= 16 ? 32 / NTP : 1;                      // l's side by side
         const int TRI = (NMAX * (NMAX + 1) / 2) * L1, SQ = NMAX * NMAX * L1;
-        for (int u0 = 0; u0 < n_tasks; u0 += 32) {
-            const int u = u0 + lane;
-            const bool active = u < n_tasks;
-            const int lq = active ? u / NTP : 0;
-            const int l = active ? L - lq : 0;                       // longest sums first; lanes of a round have similar l
-            int rem = active ? u - lq * NTP : 0, ta = 0, tb = 0;
+        const float4* const c4 = reinterpret_cast<const float4*>(c_t);
+        for (int tp0 = 0; tp0 < NTP; tp0 += 32) {
+            const int grp = G > 1 ? lane / NTP : 0;
+            int rem = G > 1 ? lane - grp * NTP : tp0 + lane;
+            const bool active = grp < G && rem < NTP;
+            if (!active) rem = 0;
+            int ta = 0, tb = 0;
             if (o_cross) {
                 while (rem >= TA - ta) { rem -= TA - ta; ++ta; }
                 tb = ta + rem;
@@ -405,46 +417,51 @@ __global__ void __launch_bounds__(kDescMaxWarps * 32, 1) desc_kernel(const Cente
                 tb = sb * TB + ta + rem;
                 ta += sb * TB;
             }
-            float g[4][4];
+            // row i of the block starts at feature offset rowoff[i] (+ j (l_max+1) + l); bit 4 i + j of `valid` says
+            // whether (i, j) is a feature at all (n below n_max, and n' >= n inside a diagonal species block)
+            const int mu = (4 * ta) / NP, nu = (4 * tb) / NP, na = 4 * ta - mu * NP, nb = 4 * tb - nu * NP;
+            int rowoff[4];
+            unsigned valid = 0;
+            {
+                const int before = o_cross ? mu * S - mu * (mu - 1) / 2 + (nu - mu) : mu, diag = o_cross ? mu + (nu > mu ? 1 : 0) : mu;
+                const int base = diag * TRI + (before - diag) * SQ;
 #pragma unroll
-            for (int i = 0; i < 4; ++i)
+                for (int i = 0; i < 4; ++i) {
+                    const int n1 = na + i;
+                    rowoff[i] = base + (mu < nu ? n1 * NMAX + nb : n1 * NMAX - n1 * (n1 - 1) / 2 - n1 + nb) * L1;
 #pragma unroll
-                for (int j = 0; j < 4; ++j) g[i][j] = 0.f;
-            const float* rowp = c_t + (l * l) * SNP;
-            const int steps = active ? 2 * l + 1 : 0;
-            for (int m = 0; m < steps; ++m) {
-                const float4 A = *reinterpret_cast<const float4*>(rowp + m * SNP + 4 * ta);
-                const float4 B = *reinterpret_cast<const float4*>(rowp + m * SNP + 4 * tb);
-                const float av[4] = {A.x, A.y, A.z, A.w}, bv[4] = {B.x, B.y, B.z, B.w};
-#pragma unroll
-                for (int i = 0; i < 4; ++i)
-#pragma unroll
-                    for (int j = 0; j < 4; ++j) g[i][j] = fmaf(av[i], bv[j], g[i][j]);
+                    for (int j = 0; j < 4; ++j)
+                        if (active && n1 < NMAX && nb + j < NMAX && (mu < nu || n1 <= nb + j)) valid |= 1u << (4 * i + j);
+                }
             }
-            if (active) {
-                const float kl = __ldg(p.kl + l);
-                const int mu = (4 * ta) / NP, nu = (4 * tb) / NP, na = 4 * ta - mu * NP, nb = 4 * tb - nu * NP;
-                if (mu < nu) {
-                    // off-diagonal species block: rows n1 of n_max (l_max+1) features
-                    const int before = mu * S - mu * (mu - 1) / 2 + (nu - mu), diag = mu + 1;
-                    float* o = dst + diag * TRI + (before - diag) * SQ + (na * NMAX + nb) * L1 + l;
+            for (int l0 = L; l0 >= 0; l0 -= G) {
+                const int l = l0 - grp;                                // this lane's l (may fall below zero in the last trip)
+                const int steps = (active && l >= 0) ? 2 * l + 1 : 0;
+                float2 g[4][2];
 #pragma unroll
-                    for (int i = 0; i < 4; ++i)
-#pragma unroll
-                        for (int j = 0; j < 4; ++j)
-                            if (na + i < NMAX && nb + j < NMAX) o[(i * NMAX + j) * L1] = kl * g[i][j];
-                } else {
-                    // diagonal species block: rows n1 hold n2 = n1 .. n_max - 1
-                    const int before = o_cross ? mu * S - mu * (mu - 1) / 2 : 0;
-                    float* o = dst + (o_cross ? mu * TRI + (before - mu) * SQ : mu * TRI) + l;
+                for (int i = 0; i < 4; ++i) g[i][0] = g[i][1] = make_float2(0.f, 0.f);
+                const float4* rowp = c4 + (l >= 0 ? l * l : 0) * (SNP / 4);
+                for (int m = 0; m < steps; ++m) {
+                    const float4 A = rowp[m * (SNP / 4) + ta];
+                    const float4 B = rowp[m * (SNP / 4) + tb];
+                    const float2 b01 = make_float2(B.x, B.y), b23 = make_float2(B.z, B.w);
+                    const float av[4] = {A.x, A.y, A.z, A.w};
 #pragma unroll
                     for (int i = 0; i < 4; ++i) {
-                        const int n1 = na + i, rs = n1 * NMAX - n1 * (n1 - 1) / 2 - n1;      // row start minus n1
+                        const float2 aa = make_float2(av[i], av[i]);
+                        g[i][0] = __ffma2_rn(aa, b01, g[i][0]);
+                        g[i][1] = __ffma2_rn(aa, b23, g[i][1]);
+                    }
+                }
+                if (steps) {
+                    const float kl = __ldg(p.kl + l);
 #pragma unroll
-                        for (int j = 0; j < 4; ++j) {
-                            const int n2 = nb + j;
-                            if (n1 < NMAX && n2 < NMAX && n1 <= n2) o[(rs + n2) * L1] = kl * g[i][j];
-                        }
+                    for (int i = 0; i < 4; ++i) {
+                        float* o = dst + rowoff[i] + l;
+                        if (valid & (1u << (4 * i))) o[0] = kl * g[i][0].x;
+                        if (valid & (2u << (4 * i))) o[L1] = kl * g[i][0].y;
+                        if (valid & (4u << (4 * i))) o[2 * L1] = kl * g[i][1].x;
+                        if (valid & (8u << (4 * i))) o[3 * L1] = kl * g[i][1].y;
                     }
                 }
             }

@@ -233,14 +233,15 @@ int ensure_device(soap_t* h) {
     h->device = dev;
     CU(upload(&h->d_table, h->basis.table));
     {
-        // [interval][l][n padded to a multiple of four][6]; the padding channels are zero
+        // [interval][l][n / 2][6][2], n padded to a multiple of four: the coefficients of two adjacent n interleaved
+        // (the descriptor-only kernel evaluates them with packed multiply-adds); the padding channels are zero
         const int L1 = h->l_max + 1, n_ch = h->n_max * L1, np = desc_np(h->n_max);
         std::vector<float> ln((size_t)h->basis.n_intervals * L1 * np * kTableCoef, 0.f);
         for (int q = 0; q < h->basis.n_intervals; ++q)
             for (int l = 0; l < L1; ++l)
                 for (int n = 0; n < h->n_max; ++n)
                     for (int k = 0; k < kTableCoef; ++k)
-                        ln[(((size_t)q * L1 + l) * np + n) * kTableCoef + k] =
+                        ln[((((size_t)q * L1 + l) * (np / 2) + n / 2) * kTableCoef + k) * 2 + (n & 1)] =
                             h->basis.table[((size_t)q * n_ch + n * L1 + l) * kTableCoef + k];
         CU(upload(&h->d_table_ln, ln));
         h->desc_np = np;

@@ -66,7 +66,7 @@ struct CenterParams {
     Counters* counters;
     // basis
     const float* table;           // [nint][n_ch][6]
-    const float* table_ln;        // the same polynomials as [nint][l][n padded to a multiple of 4][6] (descriptor-only kernel)
+    const float* table_ln;        // the same polynomials as [nint][l][n / 2][6][2], n padded to a multiple of 4 (descriptor-only kernel)
     const float* self_term;       // [n_max]
     const int* l_of_lm;           // [lm] -> l
     const float* kl;
