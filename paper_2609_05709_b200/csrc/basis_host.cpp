@@ -261,34 +261,51 @@ int build_basis(int rbf, double r_cut, int n_max, int l_max, double sigma,
     out = HostBasis();
     out.rbf = rbf; out.n_max = n_max; out.l_max = l_max; out.r_cut = r_cut; out.sigma = sigma;
     const int L1 = l_max + 1, n_ch = n_max * L1;
-    // interval width about sigma/6: the degree-5 fit then sits at the fp32 rounding floor
+    quad nodes[kTableCoef], vinv[kTableCoef][kTableCoef];
+    vandermonde_inverse(nodes, vinv);
+    std::vector<quad> vals;
+    // Fits the per-interval polynomials on `nint` uniform intervals; `vals` keeps the samples, the last of
+    // which is the value at distance zero.
+    auto fit = [&](int nint, std::vector<float>& table) -> bool {
+        const quad inv_h = (quad)nint / (quad)r_cut;
+        std::vector<quad> d((size_t)nint * kTableCoef + 1);
+        for (int q = 0; q < nint; ++q)
+            for (int k = 0; k < kTableCoef; ++k)
+                d[(size_t)q * kTableCoef + k] = ((quad)q + nodes[k]) / inv_h;
+        d.back() = 0;                                               // for the on-site term
+        if (rbf == 0) gto_values(r_cut, n_max, l_max, sigma, d, vals);
+        else if (!poly_values(r_cut, n_max, l_max, sigma, d, vals)) return false;
+        table.resize((size_t)nint * n_ch * kTableCoef);
+        for (int q = 0; q < nint; ++q)
+            for (int c = 0; c < n_ch; ++c)
+                for (int j = 0; j < kTableCoef; ++j) {
+                    quad acc = 0;
+                    for (int k = 0; k < kTableCoef; ++k)
+                        acc += vinv[j][k] * vals[((size_t)q * kTableCoef + k) * n_ch + c];
+                    table[((size_t)q * n_ch + c) * kTableCoef + j] = (float)acc;
+                }
+        return true;
+    };
+    // The descriptor-only kernel keeps its table in shared memory and reads values only: intervals of about
+    // sigma/3 keep the degree-5 fit near 1e-7 of a channel's maximum (the fp32 rounding of the coefficients
+    // is 5e-8 by itself) at half the size.
+    int nint_v = (int)std::ceil(r_cut / (sigma / 3.0));
+    nint_v = std::min(std::max(nint_v, 8), 4096);
+    out.n_intervals_values = nint_v;
+    out.inv_h_values = nint_v / r_cut;
+    if (!fit(nint_v, out.table_values)) {
+        err = "polynomial overlap matrix is not positive definite at this n_max";
+        return SOAP_ERR_INVALID_ARG;
+    }
+    // interval width about sigma/6: the degree-5 fit (value and derivative) then sits at the fp32 rounding floor
     int nint = (int)std::ceil(r_cut / (sigma / 6.0));
     nint = std::min(std::max(nint, 16), 4096);
     out.n_intervals = nint;
     out.inv_h = nint / r_cut;
-
-    quad nodes[kTableCoef], vinv[kTableCoef][kTableCoef];
-    vandermonde_inverse(nodes, vinv);
-    std::vector<quad> d((size_t)nint * kTableCoef + 1), vals;
-    for (int q = 0; q < nint; ++q)
-        for (int k = 0; k < kTableCoef; ++k)
-            d[(size_t)q * kTableCoef + k] = ((quad)q + nodes[k]) / (quad)out.inv_h;
-    d.back() = 0;                                               // for the on-site term
-    if (rbf == 0) {
-        gto_values(r_cut, n_max, l_max, sigma, d, vals);
-    } else if (!poly_values(r_cut, n_max, l_max, sigma, d, vals)) {
+    if (!fit(nint, out.table)) {
         err = "polynomial overlap matrix is not positive definite at this n_max";
         return SOAP_ERR_INVALID_ARG;
     }
-    out.table.resize((size_t)nint * n_ch * kTableCoef);
-    for (int q = 0; q < nint; ++q)
-        for (int c = 0; c < n_ch; ++c)
-            for (int j = 0; j < kTableCoef; ++j) {
-                quad acc = 0;
-                for (int k = 0; k < kTableCoef; ++k)
-                    acc += vinv[j][k] * vals[((size_t)q * kTableCoef + k) * n_ch + c];
-                out.table[((size_t)q * n_ch + c) * kTableCoef + j] = (float)acc;
-            }
     // on-site term: a neighbour at distance zero, S_00 = 1/sqrt(4 pi)   (second term of Eq. 13)
     out.self_term.resize(n_max);
     for (int n = 0; n < n_max; ++n)

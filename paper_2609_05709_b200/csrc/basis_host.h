@@ -19,6 +19,10 @@ struct HostBasis {
     // real solid harmonic; table[(q * n_ch + n * (l_max+1) + l) * 6 + k] is the
     // coefficient of t^k on interval q, t = d * inv_h - q in [0, 1).
     std::vector<float> table;
+    // the same functions on wider intervals (values only are read from it): descriptor-only kernel
+    int n_intervals_values = 0;
+    double inv_h_values = 0;
+    std::vector<float> table_values;
     std::vector<float> self_term;                  // on-site c_n00, [n_max]
     std::vector<float> anorm;                      // harmonic normalisation, [(l,m), m<=l], sqrt2 folded in for m>0
     std::vector<float> dfact;                      // (2m-1)!!, [l_max+1]

@@ -192,7 +192,7 @@ center_kernel(const CenterParams p) {
                 if (o_pw) wgt = o_pw[pair_base + g0 + tid];
                 special = rw & (kRowSelfImage | kRowContinuation);
                 // interval and offset in the radial table, in fp64 so that the offset keeps its digits
-                const double u = r * (double)p.inv_h;
+                const double u = r * p.inv_h;
                 qi = min((int)u, p.n_intervals - 1);
                 tt = (float)(u - qi);
                 sp = p.species_idx[j];
@@ -230,7 +230,7 @@ center_kernel(const CenterParams p) {
         for (int pr = wid; pr < pc; pr += kWarps) {
             const int4 gi = geo_i[g + pr];
             const float t = __int_as_float(gi.y);
-            const float rinv_h = p.inv_h / geo_d[g + pr].w;
+            const float rinv_h = (float)p.inv_h / geo_d[g + pr].w;
             if (o_pw) {
                 // radial weighting: G -> w G, Ghat -> w Ghat + (w'/d) G
                 const float2 w = geo_w[g + pr];

@@ -1,13 +1,13 @@
 // The descriptor-only kernel: expansion coefficients (Eq. 13 / Eqs. 18-19) and the power spectrum
-// (Eq. 4) of every centre, one WARP per centre, persistent CTAs that draw centres from a counter.
+// (Eq. 4) of every centre, one WARP per centre, persistent CTAs whose warps take the centres in turn.
 //
 // This build is bound by FP32 issue slots and by shared-memory bandwidth, not by HBM, so the layout is
 // chosen for few instructions and few shared-memory wavefronts per pair:
 //   * the radial table (value polynomials, re-laid as [interval][l][n / 2][6][2]) sits in shared memory
 //     once per CTA when it fits; a lane evaluates two adjacent n at once from three conflict-free 16-byte
 //     loads and five packed multiply-adds (fma.rn.f32x2: one issue slot for two multiply-adds);
-//   * the pairs of a centre (up to 128 at a time) are fetched and their geometry formed in registers
-//     in one go, ranked by species with ballots, and staged 16 at a time in species order: solid
+//   * the pairs of a centre (up to 64 at a time) have their geometry formed in registers, are ranked by species with ballots, and staged 16 at a time in
+//     species order: solid
 //     harmonics with a lane per pair from the fully unrolled Q_l^m recursion, radial factors with
 //     lanes on the channels (l, n);
 //   * accumulation c[l,m][n] += S_lm G_nl is register-tiled: a lane owns four consecutive m of one l
@@ -25,8 +25,8 @@
 namespace soap {
 
 constexpr int kDescChunk = 16;                    // pairs staged at once by a warp
-constexpr int kDescGroup = 128;                   // pairs whose geometry a warp holds in registers (four per lane)
-constexpr int kDescMaxWarps = 12;                 // warps per CTA (one CTA per SM)
+constexpr int kDescGroup = 64;                    // pairs whose geometry a warp holds in registers (two per lane)
+constexpr int kDescMaxWarps = 16;                 // warps per CTA (one CTA per SM)
 
 // harmonic normalisation up to l = 12, filled by desc_constants(): a_lm (sqrt2 folded in for m > 0), index l(l+1)/2 + m
 __device__ __constant__ float kd_norm[91] = {0};
@@ -44,11 +44,23 @@ __host__ __device__ constexpr int desc_np(int n_max) { return (n_max + 3) & ~3; 
 // words per pair of the harmonics staging: the tiles, four words each, padded to an odd number of 16-byte chunks so
 // that the 16-byte stores of eight lanes (eight pairs) fall into eight different bank groups
 __host__ __device__ constexpr int desc_s_row(int l_max) { return 4 * (desc_tiles(l_max) | 1); }
-// words per l of the radial staging: n padded so that the 16-byte chunks of consecutive l fall into different bank groups
-__host__ __device__ constexpr int desc_g_l(int np) { return np + (((np / 4) & 1) ? 0 : 4); }
+// words per l of the radial staging.  Lanes that own tiles of different l read 16-byte chunks of different rows at
+// once, and these must fall into different bank groups: with an odd number of chunks per l they do; with two
+// (n_max up to 8) the two chunks of rows l >= 4 are swapped instead; with four the row is padded by one chunk.
+__host__ __device__ constexpr int desc_g_l(int np) { return np == 16 ? 20 : np; }
+__host__ __device__ constexpr int desc_g_swap(int np, int l) { return np == 8 ? (l >> 2) & 1 : 0; }
+
+// 16-byte chunks per row of the centre's coefficient tile c[lm][species, n]: S NP / 4 rounded up to a power of two.
+// Chunk k of row r sits at position (k + r / 4) mod that number, so that the lanes of a warp, which own rows four
+// apart, do not all hit one group of banks when they store their sums.
+__host__ __device__ constexpr int desc_c_chunks(int S, int np) {
+    int rc = 1;
+    while (rc < S * np / 4) rc <<= 1;
+    return rc;
+}
 
 // Shared memory in 4-byte words: [table (optional)] then one region per warp:
-//   c [LM][S NP] | S staging [chunk][s_row] | G staging [chunk][L1 g_l] | pair staging [chunk][8]
+//   c [LM][4 desc_c_chunks] | S staging [chunk][s_row] | G staging [chunk][L1 g_l] | pair staging [chunk][8]
 // The feature row is assembled on top of the staging area when it fits there.
 struct DescLayout {
     int table, warp0, per_warp, c, sS, sG, ring, slab_words, total;
@@ -59,7 +71,7 @@ __host__ __device__ inline DescLayout make_desc_layout(int S, int np, int l_max,
     o.table = 0;
     o.warp0 = (table_words + 3) & ~3;
     int off = 0;
-    o.c = off; off += LM * S * np;
+    o.c = off; off += LM * 4 * desc_c_chunks(S, np);
     o.sS = off; off += kDescChunk * desc_s_row(l_max);
     o.sG = off; off += kDescChunk * L1 * desc_g_l(np);
     o.ring = off; off += kDescChunk * 8;
@@ -131,7 +143,7 @@ __global__ void __launch_bounds__(kDescMaxWarps * 32, 1) desc_kernel(const Cente
     const float* const o_sites = PLAIN ? nullptr : p.sites;
     const float2* const o_pw = PLAIN ? nullptr : p.pair_w;
     const float o_w0 = PLAIN ? 1.f : p.w0;
-    const int S = p.S, NMAX = p.n_max, SNP = S * NP, F = p.F;
+    const int S = p.S, NMAX = p.n_max, F = p.F;
     const DescLayout lay = make_desc_layout(S, NP, L, warps, TS ? p.n_intervals * NCHP * 6 : 0);
 
     if (TS) {
@@ -145,7 +157,10 @@ __global__ void __launch_bounds__(kDescMaxWarps * 32, 1) desc_kernel(const Cente
     if (p.counters->n_pairs > p.pair_capacity) return;
 
     float* const wbase = smem + lay.warp0 + wid * lay.per_warp;
-    float* const c_t = wbase + lay.c;                                               // [LM][SNP]
+    float* const c_t = wbase + lay.c;                                               // [LM][4 RC], chunks rotated by row / 4
+    const int RC = desc_c_chunks(S, NP), rc_mask = RC - 1;
+    auto c_chunk = [&](int r, int k) { return r * RC + ((k + (r >> 2)) & rc_mask); };        // 16-byte chunk k of row r
+    auto c_word = [&](int r, int col) { return 4 * c_chunk(r, col >> 2) + (col & 3); };
     float4* const sS4 = reinterpret_cast<float4*>(wbase + lay.sS);                  // [chunk][SROW / 4] tiles of four m
     float* const sG = wbase + lay.sG;                                               // [chunk][L1][GL]
     float4* const ring_d = reinterpret_cast<float4*>(wbase + lay.ring);             // [chunk] dx, dy, dz, r
@@ -169,65 +184,86 @@ __global__ void __launch_bounds__(kDescMaxWarps * 32, 1) desc_kernel(const Cente
     int g_word[ROUNDS];
 #pragma unroll
     for (int rr = 0; rr < ROUNDS; ++rr) {
-        const int cp = rr * 32 + lane, l = cp / (NP / 2);
-        g_word[rr] = l * GL + 2 * (cp - l * (NP / 2));
+        const int cp = rr * 32 + lane, l = cp / (NP / 2), n = 2 * (cp - l * (NP / 2));
+        g_word[rr] = l * GL + 4 * ((n >> 2) ^ desc_g_swap(NP, l)) + (n & 3);
     }
     const bool periodic = p.geom.pbc[0] | p.geom.pbc[1] | p.geom.pbc[2];
     const long long n_work = o_cbar ? 1 : p.n_centers;
 
-    for (;;) {
-        long long w = 0;
-        if (lane == 0) w = (long long)atomicAdd(&p.counters->work, 1);
-        w = __shfl_sync(0xffffffffu, w, 0);
-        if (w >= n_work) break;
-        const long long c_idx = p.order ? p.order[w] : w;
+    // Centres are dealt out to the warps of the grid in turn (neighbouring warps take neighbouring centres).
+    constexpr int PPL = kDescGroup / 32;                                 // pairs per lane and group
+    struct Head { float xi, yi, zi; int zsp; long long pair_base; int k_pairs; };
+    struct Raw { unsigned long long key[PPL]; float wgt[PPL]; int spj[PPL]; float px[PPL], py[PPL], pz[PPL]; };
+    auto load_head = [&](long long c_idx) {
+        Head h;
         const int ci = o_sites ? -1 : (p.centers ? p.centers[c_idx] : (int)c_idx);
         const float* pc = o_sites ? o_sites + 3 * c_idx : p.pos + 3 * (long long)ci;
-        const float xi = pc[0], yi = pc[1], zi = pc[2];
-        const int zi_species = o_sites ? 0 : p.species_idx[ci];
-        const long long pair_base = p.pair_start[c_idx];
-        const int k_pairs = o_cbar ? 0 : p.pair_count[c_idx];
+        h.xi = pc[0]; h.yi = pc[1]; h.zi = pc[2];
+        h.zsp = o_sites ? 0 : p.species_idx[ci];
+        h.pair_base = p.pair_start[c_idx];
+        h.k_pairs = o_cbar ? 0 : p.pair_count[c_idx];
+        return h;
+    };
+    auto load_keys = [&](const Head& h, int g0, Raw& r) {
+#pragma unroll
+        for (int b = 0; b < PPL; ++b) {
+            const int e = g0 + 32 * b + lane;
+            r.key[b] = e < h.k_pairs ? p.pair_key[h.pair_base + e] : 0ull;
+            r.wgt[b] = (o_pw && e < h.k_pairs) ? o_pw[h.pair_base + e].x : 1.f;
+        }
+    };
+    auto load_atoms = [&](const Head& h, int g0, Raw& r) {
+#pragma unroll
+        for (int b = 0; b < PPL; ++b) {
+            const int e = g0 + 32 * b + lane;
+            r.spj[b] = -1; r.px[b] = r.py[b] = r.pz[b] = 0.f;
+            if (e < h.k_pairs) {
+                const int j = key_atom(r.key[b]);
+                r.spj[b] = S == 1 ? 0 : p.species_idx[j];
+                r.px[b] = p.pos[3 * (long long)j]; r.py[b] = p.pos[3 * (long long)j + 1]; r.pz[b] = p.pos[3 * (long long)j + 2];
+            }
+        }
+    };
+    const long long w_stride = (long long)gridDim.x * warps;
+    for (long long c_idx = (long long)blockIdx.x * warps + wid; c_idx < n_work; c_idx += w_stride) {
+        const Head hd = load_head(c_idx);
+        Raw raw;
+        const float xi = hd.xi, yi = hd.yi, zi = hd.zi;
+        const int zi_species = hd.zsp, k_pairs = hd.k_pairs;
 
-        for (int e = lane; e < LM * SNP / 4; e += 32) reinterpret_cast<float4*>(c_t)[e] = make_float4(0.f, 0.f, 0.f, 0.f);
+        for (int e = lane; e < LM * RC; e += 32) reinterpret_cast<float4*>(c_t)[e] = make_float4(0.f, 0.f, 0.f, 0.f);
         __syncwarp();
 
         for (int g0 = 0; g0 < k_pairs; g0 += kDescGroup) {
-            // ---- geometry of up to 128 pairs, four per lane, all loads in flight together ----
+            // ---- geometry of up to 64 pairs, two per lane ----
             const int kg = min(kDescGroup, k_pairs - g0);
-            int sp[4], pos_sorted[4];
-            float4 dd[4];
-            int2 qt[4];                                                     // interval, offset bits
-            float ww[4];
-            unsigned long long key[4];
+            load_keys(hd, g0, raw);
+            load_atoms(hd, g0, raw);
+            int sp[PPL], pos_sorted[PPL];
+            float4 dd[PPL];
+            int2 qt[PPL];                                                    // interval, offset bits
+            float ww[PPL];
 #pragma unroll
-            for (int b = 0; b < 4; ++b) {
-                const int e = g0 + 32 * b + lane;
-                key[b] = e < k_pairs ? p.pair_key[pair_base + e] : 0ull;
-                ww[b] = (o_pw && e < k_pairs) ? o_pw[pair_base + e].x : 1.f;
-            }
-#pragma unroll
-            for (int b = 0; b < 4; ++b) {
-                const int e = g0 + 32 * b + lane;
-                sp[b] = -1;
+            for (int b = 0; b < PPL; ++b) {
+                sp[b] = raw.spj[b];
+                ww[b] = raw.wgt[b];
                 dd[b] = make_float4(0.f, 0.f, 0.f, 0.f);
                 qt[b] = make_int2(0, 0);
                 pos_sorted[b] = -1;
-                if (e < k_pairs) {
-                    const int j = key_atom(key[b]);
-                    sp[b] = S == 1 ? 0 : p.species_idx[j];
-                    double dx = (double)p.pos[3 * (long long)j] - (double)xi;
-                    double dy = (double)p.pos[3 * (long long)j + 1] - (double)yi;
-                    double dz = (double)p.pos[3 * (long long)j + 2] - (double)zi;
+                if (sp[b] >= 0) {
+                    double dx = (double)raw.px[b] - (double)xi;
+                    double dy = (double)raw.py[b] - (double)yi;
+                    double dz = (double)raw.pz[b] - (double)zi;
                     if (periodic) {
                         int sh[3];
-                        key_shift(key[b], sh);
+                        key_shift(raw.key[b], sh);
                         dx += sh[0] * p.geom.cell[0] + sh[1] * p.geom.cell[3] + sh[2] * p.geom.cell[6];
                         dy += sh[0] * p.geom.cell[1] + sh[1] * p.geom.cell[4] + sh[2] * p.geom.cell[7];
                         dz += sh[0] * p.geom.cell[2] + sh[1] * p.geom.cell[5] + sh[2] * p.geom.cell[8];
                     }
                     const double r = sqrt(dx * dx + dy * dy + dz * dz);
                     // interval and offset in the radial table, in fp64 so that the offset keeps its digits
-                    const double u = r * (double)p.inv_h;
+                    const double u = r * p.inv_h;
                     const int qi = min((int)u, p.n_intervals - 1);
                     dd[b] = make_float4((float)dx, (float)dy, (float)dz, (float)r);
                     qt[b] = make_int2(qi, __float_as_int((float)(u - qi)));
@@ -238,7 +274,7 @@ __global__ void __launch_bounds__(kDescMaxWarps * 32, 1) desc_kernel(const Cente
                 int base = 0;
                 for (int s = 0; s < S; ++s)
 #pragma unroll
-                    for (int b = 0; b < 4; ++b) {
+                    for (int b = 0; b < PPL; ++b) {
                         const unsigned m = __ballot_sync(0xffffffffu, sp[b] == s);
                         if (sp[b] == s) pos_sorted[b] = base + __popc(m & ((1u << lane) - 1));
                         base += __popc(m);
@@ -273,16 +309,18 @@ __global__ void __launch_bounds__(kDescMaxWarps * 32, 1) desc_kernel(const Cente
 #pragma unroll
                             for (int n = 0; n < NB / 2; ++n) acc[tp][k][n] = make_float2(0.f, 0.f);
                             if (k < t_kv[tp] && (HALVES == 1 || (k >> 1) == half)) {
-                                float4* dst = reinterpret_cast<float4*>(c_t + (t_lm0[tp] + k) * SNP + s * NP + n0);
+                                float4* const c4w = reinterpret_cast<float4*>(c_t);
+                                const int r = t_lm0[tp] + k, k0 = (s * NP + n0) / 4;
 #pragma unroll
                                 for (int n4 = 0; n4 < NB / 4; ++n4)
                                     if (NPASS == 1 || n0 + 4 * n4 < NP) {
                                         float4 o = make_float4(v[4 * n4], v[4 * n4 + 1], v[4 * n4 + 2], v[4 * n4 + 3]);
+                                        float4* dst = c4w + c_chunk(r, k0 + n4);
                                         if (!single) {
-                                            const float4 old = dst[n4];
+                                            const float4 old = *dst;
                                             o.x += old.x; o.y += old.y; o.z += old.z; o.w += old.w;
                                         }
-                                        dst[n4] = o;
+                                        *dst = o;
                                     }
                             }
                         }
@@ -292,7 +330,7 @@ __global__ void __launch_bounds__(kDescMaxWarps * 32, 1) desc_kernel(const Cente
                     const int n_stage = min(kDescChunk, kg - c0);
                     // the pairs at sorted positions c0 .. c0 + 15 go to the staging slots
 #pragma unroll
-                    for (int b = 0; b < 4; ++b)
+                    for (int b = 0; b < PPL; ++b)
                         if ((unsigned)(pos_sorted[b] - c0) < (unsigned)kDescChunk) {
                             ring_d[pos_sorted[b] - c0] = dd[b];
                             ring_i[pos_sorted[b] - c0] = make_int4(qt[b].x, qt[b].y, sp[b], __float_as_int(ww[b]));
@@ -350,7 +388,7 @@ __global__ void __launch_bounds__(kDescMaxWarps * 32, 1) desc_kernel(const Cente
 #pragma unroll
                                 for (int n4 = 0; n4 < NB / 4; ++n4) {
                                     if (NPASS > 1 && n0 + 4 * n4 >= NP) break;
-                                    const float4 g = gp[t_l[tp] * (GL / 4) + n4];
+                                    const float4 g = gp[t_l[tp] * (GL / 4) + (n4 ^ desc_g_swap(NP, t_l[tp]))];
 #pragma unroll
                                     for (int k = 0; k < 4; ++k) {
                                         acc[tp][k][2 * n4] = __ffma2_rn(h[k], make_float2(g.x, g.y), acc[tp][k][2 * n4]);
@@ -368,12 +406,12 @@ __global__ void __launch_bounds__(kDescMaxWarps * 32, 1) desc_kernel(const Cente
         }
 
         // on-site term: the centre's own Gaussian, l = 0 only (second term of Eq. 13)
-        if (!o_cbar && !o_sites && lane < NMAX) c_t[zi_species * NP + lane] += o_w0 * __ldg(p.self_term + lane);
+        if (!o_cbar && !o_sites && lane < NMAX) c_t[c_word(0, zi_species * NP + lane)] += o_w0 * __ldg(p.self_term + lane);
         if (o_cbar) {
             // given mean coefficients (inner average) take the place of the centre's own: index (mu n_max + n) LM + lm
             for (int e = lane; e < S * NMAX * LM; e += 32) {
                 const int row = e / LM, lm = e - row * LM, mu = row / NMAX, n = row - mu * NMAX;
-                c_t[lm * SNP + mu * NP + n] = __ldg(o_cbar + e);
+                c_t[c_word(lm, mu * NP + n)] = __ldg(o_cbar + e);
             }
         }
         __syncwarp();
@@ -382,7 +420,7 @@ __global__ void __launch_bounds__(kDescMaxWarps * 32, 1) desc_kernel(const Cente
             float* crow = p.out_desc + (size_t)c_idx * (S * NMAX * LM);
             for (int e = lane; e < S * NMAX * LM; e += 32) {
                 const int row = e / LM, lm = e - row * LM, mu = row / NMAX, n = row - mu * NMAX;
-                crow[e] = c_t[lm * SNP + mu * NP + n];
+                crow[e] = c_t[c_word(lm, mu * NP + n)];
             }
             __syncwarp();
             continue;
@@ -440,10 +478,10 @@ __global__ void __launch_bounds__(kDescMaxWarps * 32, 1) desc_kernel(const Cente
                 float2 g[4][2];
 #pragma unroll
                 for (int i = 0; i < 4; ++i) g[i][0] = g[i][1] = make_float2(0.f, 0.f);
-                const float4* rowp = c4 + (l >= 0 ? l * l : 0) * (SNP / 4);
+                const int r0 = l >= 0 ? l * l : 0;
                 for (int m = 0; m < steps; ++m) {
-                    const float4 A = rowp[m * (SNP / 4) + ta];
-                    const float4 B = rowp[m * (SNP / 4) + tb];
+                    const float4 A = c4[c_chunk(r0 + m, ta)];
+                    const float4 B = c4[c_chunk(r0 + m, tb)];
                     const float2 b01 = make_float2(B.x, B.y), b23 = make_float2(B.z, B.w);
                     const float av[4] = {A.x, A.y, A.z, A.w};
 #pragma unroll

@@ -236,13 +236,13 @@ int ensure_device(soap_t* h) {
         // [interval][l][n / 2][6][2], n padded to a multiple of four: the coefficients of two adjacent n interleaved
         // (the descriptor-only kernel evaluates them with packed multiply-adds); the padding channels are zero
         const int L1 = h->l_max + 1, n_ch = h->n_max * L1, np = desc_np(h->n_max);
-        std::vector<float> ln((size_t)h->basis.n_intervals * L1 * np * kTableCoef, 0.f);
-        for (int q = 0; q < h->basis.n_intervals; ++q)
+        std::vector<float> ln((size_t)h->basis.n_intervals_values * L1 * np * kTableCoef, 0.f);
+        for (int q = 0; q < h->basis.n_intervals_values; ++q)
             for (int l = 0; l < L1; ++l)
                 for (int n = 0; n < h->n_max; ++n)
                     for (int k = 0; k < kTableCoef; ++k)
                         ln[((((size_t)q * L1 + l) * (np / 2) + n / 2) * kTableCoef + k) * 2 + (n & 1)] =
-                            h->basis.table[((size_t)q * n_ch + n * L1 + l) * kTableCoef + k];
+                            h->basis.table_values[((size_t)q * n_ch + n * L1 + l) * kTableCoef + k];
         CU(upload(&h->d_table_ln, ln));
         h->desc_np = np;
         h->desc_table_bytes = ln.size() * sizeof(float);
@@ -430,7 +430,7 @@ void fill_center_params(soap_t* h, CenterParams& cp, const float* pos, const int
     cp.row_ptr = h->d_row_ptr; cp.self_row = h->d_self_row;
     cp.pair_capacity = h->cap_pairs; cp.row_capacity = 0; cp.counters = h->d_counters;
     cp.table = h->d_table; cp.self_term = h->d_self; cp.kl = h->d_kl; cp.l_of_lm = h->d_l_of_lm;
-    cp.feat_pack = h->d_feat; cp.nch_magic = (unsigned)((1ull << 32) / (unsigned)(h->n_max * (h->l_max + 1))) + 1u; cp.inv_h = (float)h->basis.inv_h; cp.n_intervals = h->basis.n_intervals;
+    cp.feat_pack = h->d_feat; cp.nch_magic = (unsigned)((1ull << 32) / (unsigned)(h->n_max * (h->l_max + 1))) + 1u; cp.inv_h = h->basis.inv_h; cp.n_intervals = h->basis.n_intervals;
     cp.S = h->S; cp.n_max = h->n_max; cp.l_max = h->l_max; cp.F = (int)h->F;
     cp.P = h->P_deriv;
     cp.crossover = h->crossover; cp.emit_coeff = 0; cp.c_bar = nullptr;
@@ -439,12 +439,13 @@ void fill_center_params(soap_t* h, CenterParams& cp, const float* pos, const int
     cp.out_desc = nullptr; cp.out_jac = nullptr; cp.row_atom = nullptr;
 }
 
-// Launch of the descriptor-only kernel: persistent CTAs (one per SM) whose warps draw centres from a counter.
+// Launch of the descriptor-only kernel: persistent CTAs (one per SM) whose warps take the centres in turn.
 // The radial table goes to shared memory when it leaves room for at least six warps and there is enough
 // work to pay for staging it; small jobs use fewer warps per CTA so that they spread over the SMs.
 int launch_desc(soap_t* h, CenterParams& cp, int64_t n_work, cudaStream_t st) {
     if (n_work <= 0) return SOAP_OK;
     cp.table_ln = h->d_table_ln;
+    cp.inv_h = h->basis.inv_h_values; cp.n_intervals = h->basis.n_intervals_values;      // the value table has intervals of its own
     const bool plain = center_params_plain(cp);
     const int warps_fit = (int)std::min<size_t>(kDescMaxWarps, (size_t)h->max_smem / h->desc_warp_bytes);
     const int warps_ts = h->desc_table_bytes + h->desc_warp_bytes <= (size_t)h->max_smem
@@ -454,7 +455,6 @@ int launch_desc(soap_t* h, CenterParams& cp, int64_t n_work, cudaStream_t st) {
     warps = (int)std::max<int64_t>(1, std::min<int64_t>(warps, (n_work + h->sm_count - 1) / h->sm_count));
     const unsigned grid = (unsigned)std::min<int64_t>(h->sm_count, (n_work + warps - 1) / warps);
     const size_t smem = (size_t)make_desc_layout(h->S, h->desc_np, h->l_max, warps, ts ? (int)(h->desc_table_bytes / 4) : 0).total * 4;
-    CU(cudaMemsetAsync(&h->d_counters->work, 0, sizeof(int), st));
     CU(desc_launch(h->l_max, h->desc_np, plain, ts, cp, grid, (unsigned)warps * 32, smem, st));
     return SOAP_OK;
 }

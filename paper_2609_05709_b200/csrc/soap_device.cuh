@@ -41,7 +41,7 @@ struct GridParams {               // device-resident, written by grid_setup_kern
 
 struct Counters {                 // device-resident
     int status;
-    int work;                     // next centre of the descriptor-only kernel (zeroed before its launch)
+    int pad;
     long long n_pairs;
     long long n_rows;
 };
@@ -71,7 +71,7 @@ struct CenterParams {
     const int* l_of_lm;           // [lm] -> l
     const float* kl;
     const int* feat_pack;         // [F] n | n'<<5 | mu<<10 | nu<<14 | l<<18
-    float inv_h;
+    double inv_h;                 // intervals per Angstrom of the radial table in use
     int n_intervals;
     int S, n_max, l_max, F;
     int P;                        // pairs per staged chunk (<= 32)
