@@ -286,10 +286,11 @@ int build_basis(int rbf, double r_cut, int n_max, int l_max, double sigma,
                 }
         return true;
     };
-    // The descriptor-only kernel keeps its table in shared memory and reads values only: intervals of about
-    // sigma/3 keep the degree-5 fit near 1e-7 of a channel's maximum (the fp32 rounding of the coefficients
-    // is 5e-8 by itself) at half the size.
-    int nint_v = (int)std::ceil(r_cut / (sigma / 3.0));
+    // The descriptor-only kernel keeps its table in shared memory and reads values only: on intervals of sigma/4
+    // the degree-5 fit error (1e-8 of a channel's maximum) still sits below the fp32 rounding of the coefficients
+    // (5e-8), at two thirds of the size; sigma/3 would be smaller still but loses accuracy in the tails, where
+    // the functions are small.
+    int nint_v = (int)std::ceil(r_cut / (sigma / 4.0));
     nint_v = std::min(std::max(nint_v, 8), 4096);
     out.n_intervals_values = nint_v;
     out.inv_h_values = nint_v / r_cut;

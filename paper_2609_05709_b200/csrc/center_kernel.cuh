@@ -91,6 +91,16 @@ __device__ __forceinline__ void harmonics_column(int L, int m, float x, float y,
     }
 }
 
+// Bulk asynchronous copy shared -> global (the copy engine moves the bytes; one thread issues it).  Addresses and
+// size must be multiples of 16 bytes.  Copies of a thread are grouped by bulk_commit(); bulk_wait_read() returns
+// once the shared-memory source of all its groups has been read.
+__device__ __forceinline__ void bulk_store(float* dst, const float* src_shared, unsigned bytes) {
+    asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;"
+                 :: "l"(dst), "r"((unsigned)__cvta_generic_to_shared(src_shared)), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
+__device__ __forceinline__ void bulk_wait_read() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
+
 // KIND: 1 descriptor and Jacobian, 2 coefficients c^mu_nlm and their Jacobian.
 // PLAIN: the default configuration (every species pair, atom centres, no weighting, full rows, own
 // coefficients); the options are then compile-time constants and their code drops out.
@@ -144,6 +154,10 @@ center_kernel(const CenterParams p) {
     for (int e = tid; e < CT * 4; e += kThreads) {
         if (e < CT) c_t[e] = 0.f; else D_t[e - CT] = 0.f;
     }
+    // zeros for the bulk copies of pass 2 (made visible to the copy engine; the barriers of pass 1 order them)
+    const float* zero_buf = smem + lay.zero;
+    for (int e = tid; e < kZeroWords; e += kThreads) smem[lay.zero + e] = 0.f;
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
 
     // same-species blocks: feature index -> (n1 L1 + l) | (n2 L1 + l) << 8, rows n1 of (NMAX - n1) L1 entries
     unsigned short* tri_dec = reinterpret_cast<unsigned short*>(smem + lay.tri);
@@ -426,6 +440,10 @@ center_kernel(const CenterParams p) {
 
     // =========================== pass 2: the Jacobian rows ===========================
     const int NI = S * NCH, SN = S * NMAX;
+    // whether the zero blocks of a row can go out as bulk copies: every block boundary, the plane pitch and the
+    // row start must sit on 16 bytes
+    const bool bulk_ok = !CC && ((((NMAX * (NMAX + 1) / 2) * L1) | (NMAX * NCH) | RW) & 3) == 0 &&
+                         (reinterpret_cast<size_t>(p.out_jac) & 15) == 0;
     // coefficient mode: table lm -> l in the (now idle) space of the D tiles; the loop below starts with a barrier
     int* lm_to_l = reinterpret_cast<int*>(smem + lay.wUV);
     if (CC)
@@ -457,9 +475,19 @@ center_kernel(const CenterParams p) {
                 const int first = ((lo + a_line) & ~31) - a_line;
                 if (mu != Z && nu != Z) {
                     if (o_compact) continue;                  // compact rows hold only the blocks that involve Z
-                    if (!ACC)
-                        for (int f = first + lane; f < hi; f += 32)
-                            if (f >= lo) put(f, 0.f, 0.f, 0.f);
+                    if (!ACC) {
+                        if (bulk_ok) {
+                            // structural zeros: the lanes hand the plane segments (pieces of at most kZeroWords) to the copy engine
+                            const int parts = (hi - lo + kZeroWords - 1) / kZeroWords;
+                            for (int idx = lane; idx < 3 * parts; idx += 32) {
+                                const int k = idx / parts, f = lo + (idx - k * parts) * kZeroWords;
+                                bulk_store(out + k * PS + f, zero_buf, 4u * (unsigned)min(kZeroWords, hi - f));
+                            }
+                        } else {
+                            for (int f = first + lane; f < hi; f += 32)
+                                if (f >= lo) put(f, 0.f, 0.f, 0.f);
+                        }
+                    }
                 } else if (mu == nu && NMAX_T != 0 && NMAX_T <= 4) {
                     // small n_max: lanes on the columns (n2, l) with their own operand in registers, rows n1 <= n2
                     // in turn: fewer instructions than the table-driven sweeps below, stores contiguous but not
@@ -673,6 +701,7 @@ center_kernel(const CenterParams p) {
             if (lane == 0) p.row_atom[row_base + row] = geo_j[g];
             if (CC) coeff_rule(std::false_type{}, Z, d, wG, wSD, out);
             else product_rule(std::false_type{}, Z, d, wG, out);
+            if (bulk_ok) bulk_commit();
         }
     };
 
@@ -680,8 +709,12 @@ center_kernel(const CenterParams p) {
         const int gc = min(kGeoPairs, k_pairs - g0);
         __syncthreads();
         if (g0 > 0 || k_pairs > kGeoPairs) special = stage_geometry(g0, gc);     // otherwise still valid from pass 1
-        for (int q0 = 0; q0 < gc; q0 += P) {
-            const int pc = min(P, gc - q0);
+        // chunks of equal size, a multiple of the warp count: a short last chunk would leave most warps idle
+        // (68 pairs in chunks of 32 are 32 + 32 + 4; in three chunks of 24 every warp has three pairs or two)
+        const int n_chunks = (gc + P - 1) / P;
+        const int PB = min(P, (((gc + n_chunks - 1) / n_chunks) + kWarps - 1) & ~(kWarps - 1));
+        for (int q0 = 0; q0 < gc; q0 += PB) {
+            const int pc = min(PB, gc - q0);
             stage_chunk(q0, pc);
             __syncthreads();
             if (!special) {
@@ -699,6 +732,8 @@ center_kernel(const CenterParams p) {
             __syncthreads();
         }
     }
+    // the zeros in shared memory must outlive the copies that read them
+    if (bulk_ok) bulk_wait_read();
 }
 
 }  // namespace soap

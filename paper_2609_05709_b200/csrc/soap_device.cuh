@@ -106,8 +106,10 @@ __host__ __device__ inline void key_shift(unsigned long long k, int s[3]) {
 // single bank.
 constexpr int kGeoPairs = 128;           // pairs whose geometry is staged at once
 
+constexpr int kZeroWords = 1024;         // a block of zeros that bulk copies write into the structural-zero blocks of the rows
+
 struct SmemLayout {
-    int c, geo, tri, D, wUV, sSD, sG, total;
+    int c, geo, tri, zero, D, wUV, sSD, sG, total;
 };
 __host__ __device__ inline int align4(int x) { return (x + 3) & ~3; }
 constexpr int kGeoWords = kGeoPairs * 9 + 44;   // geometry (9 words per pair), species segments (9 + 32 words, padded)
@@ -118,6 +120,7 @@ __host__ __device__ inline SmemLayout make_layout(int S, int n_max, int l_max, i
     o.c = off; off = align4(off + CT);
     o.geo = off; off = align4(off + kGeoWords + (weighted ? 2 * kGeoPairs : 0));   // + per-pair weights
     o.tri = off; if (deriv) off = align4(off + ((n_max * (n_max + 1) / 2) * L1 + 1) / 2);   // 16-bit entries
+    o.zero = off; if (deriv) off += kZeroWords;
     // the D tiles (pass 1, centre's row) and the per-warp U/V staging (pass 2) never live
     // at the same time and share space
     o.D = off; o.wUV = off;
