@@ -300,7 +300,10 @@ int soap_derivatives_average(soap_t *h, int mode, const float *d_positions, cons
 
 /* Waits for `stream`, then returns and clears the sticky device status
  * (SOAP_OK, SOAP_ERR_UNKNOWN_SPECIES or SOAP_ERR_CAPACITY); also reports the
- * pair and row counts of the last call (either pointer may be NULL). */
+ * pair and row counts of the last call (either pointer may be NULL).  The
+ * descriptor-only calls build no Jacobian rows and keep their pairs unsorted:
+ * after one of them the row count is zero and soap_neighbor_list wants a
+ * soap_neighbors call first. */
 int soap_status(soap_t *h, int64_t *n_pairs, int64_t *n_rows, void *stream);
 
 /* Measurement aid (the paper has no counterpart): the FP32 multiply-add rate of

@@ -486,7 +486,9 @@ constexpr int kFillWarps = 4;
 // derive the Jacobian row bookkeeping (distinct atoms, the centre's own position among them).
 // When the segment does not fit the planned capacity only the counts are produced and the status
 // word says so; the caller plans again with the totals.
-template <int KEYS>
+// ROWS = false (descriptor-only calls, which sum over the pairs in any order and have no Jacobian rows): the keys
+// go out as they were found, unsorted, and the row bookkeeping is left out.
+template <int KEYS, bool ROWS>
 __global__ void __launch_bounds__(kFillWarps * 32)
 pairs_kernel(const float* __restrict__ pos, const int* __restrict__ centers, const float* __restrict__ sites, long long C, Geometry geom,
              const GridParams* __restrict__ gp, const int* __restrict__ atom_cell, const int* __restrict__ atom_wrap,
@@ -554,6 +556,10 @@ pairs_kernel(const float* __restrict__ pos, const int* __restrict__ centers, con
     volatile unsigned long long* raw = in_smem ? s_raw[wid] : pair_tmp + base;
     volatile unsigned long long* sorted = in_smem ? s_sorted[wid] : pair_key + base;
     __syncwarp();
+    if (!ROWS) {
+        for (int q = lane; q < k; q += 32) pair_key[base + q] = raw[q];
+        return;
+    }
     // rank sort (keys are distinct)
     bool self_in = false;
     for (int q = lane; q < k; q += 32) {

@@ -122,6 +122,7 @@ struct soap_handle {
     int64_t planned_atoms = -1, planned_centers = -1;
     int64_t pairs_per_center_hint = 0;   // average at the last plan (chooses the pair kernel variant)
     int64_t last_centers = 0;
+    bool list_sorted = false;            // whether the pair list of the last search is sorted (descriptor-only calls skip that)
     int P_deriv = 16;
     size_t smem_deriv = 0;
     // optional per-segment timing (events on the caller's stream)
@@ -346,7 +347,7 @@ constexpr int64_t kBruteForceAtoms = 512;
 
 int launch_neighbors(soap_t* h, const float* pos, const int32_t* num, int64_t N, const Geometry& g,
                      const int32_t* centers, const float* sites, int64_t C, long long* row_ptr_out, cudaStream_t st,
-                     const Batch& batch = Batch()) {
+                     const Batch& batch = Batch(), bool rows = true) {
     // (C == N: the brute-force kernel writes the per-centre arrays for every atom, and those are sized from C)
     const bool brute = !batch.struct_ptr && !centers && !sites && C == N && N <= kBruteForceAtoms && !(g.pbc[0] | g.pbc[1] | g.pbc[2]);
     if (batch.struct_ptr || brute) {
@@ -368,17 +369,22 @@ int launch_neighbors(soap_t* h, const float* pos, const int32_t* num, int64_t N,
         bin_fill_kernel<<<blocks_for(N, 256), 256, 0, st>>>(pos, N, h->d_atom_cell, h->d_atom_wrap, h->d_cell_start, h->d_cell_count, h->d_s_pos, h->d_s_wrap);
     }
     if (C > 0 && !batch.struct_ptr && !brute) {
-        // few pairs per centre at the last plan: the variant with the small on-chip key buffers (more warps resident)
-        if (h->pairs_per_center_hint > 0 && h->pairs_per_center_hint <= kFillSmemKeysSmall * 3 / 4)
-            pairs_kernel<kFillSmemKeysSmall><<<(unsigned)((C + kFillWarps - 1) / kFillWarps), kFillWarps * 32, 0, st>>>(
-        pos, centers, sites, C, g, h->d_grid, h->d_atom_cell, h->d_atom_wrap, h->d_cell_start, h->d_s_pos, h->d_s_wrap,
-        h->cap_pairs, h->d_pair_tmp, h->d_pair_key, h->d_pair_row, h->d_pair_start, h->d_pair_count, h->d_row_count,
-        h->d_self_row, h->d_counters);
-        else
-            pairs_kernel<kFillSmemKeys><<<(unsigned)((C + kFillWarps - 1) / kFillWarps), kFillWarps * 32, 0, st>>>(
-        pos, centers, sites, C, g, h->d_grid, h->d_atom_cell, h->d_atom_wrap, h->d_cell_start, h->d_s_pos, h->d_s_wrap,
-        h->cap_pairs, h->d_pair_tmp, h->d_pair_key, h->d_pair_row, h->d_pair_start, h->d_pair_count, h->d_row_count,
-        h->d_self_row, h->d_counters);
+        // few pairs per centre at the last plan: the variant with the small on-chip key buffers (more warps resident);
+        // descriptor-only calls take the variants without sorting and row bookkeeping
+        const bool small_keys = h->pairs_per_center_hint > 0 && h->pairs_per_center_hint <= kFillSmemKeysSmall * 3 / 4;
+        const unsigned grid = (unsigned)((C + kFillWarps - 1) / kFillWarps);
+#define SOAP_PAIRS_ARGS pos, centers, sites, C, g, h->d_grid, h->d_atom_cell, h->d_atom_wrap, h->d_cell_start, h->d_s_pos, h->d_s_wrap, \
+        h->cap_pairs, h->d_pair_tmp, h->d_pair_key, h->d_pair_row, h->d_pair_start, h->d_pair_count, h->d_row_count, h->d_self_row, h->d_counters
+        if (small_keys && rows) pairs_kernel<kFillSmemKeysSmall, true><<<grid, kFillWarps * 32, 0, st>>>(SOAP_PAIRS_ARGS);
+        else if (small_keys) pairs_kernel<kFillSmemKeysSmall, false><<<grid, kFillWarps * 32, 0, st>>>(SOAP_PAIRS_ARGS);
+        else if (rows) pairs_kernel<kFillSmemKeys, true><<<grid, kFillWarps * 32, 0, st>>>(SOAP_PAIRS_ARGS);
+        else pairs_kernel<kFillSmemKeys, false><<<grid, kFillWarps * 32, 0, st>>>(SOAP_PAIRS_ARGS);
+#undef SOAP_PAIRS_ARGS
+    }
+    if (!rows && !batch.struct_ptr && !brute) {
+        // no Jacobian rows wanted: no row pointers, no launch order
+        CU(cudaGetLastError());
+        return SOAP_OK;
     }
     if (C <= kOrderMaxCenters) {
         rows_order_kernel<<<1, 1024, 0, st>>>(h->d_row_count, h->d_pair_count, C, row_ptr_out, h->d_order, h->d_counters);
@@ -485,7 +491,7 @@ void build_feature_table(soap_t* h) {
 // changed, the neighbour search.
 int prepare(soap_t* h, const float* pos, const int32_t* num, int64_t N, const double* cell, const int32_t* centers,
             int64_t C, long long* row_ptr_out, Geometry& g, cudaStream_t st, const float* sites = nullptr,
-            const Batch& batch = Batch()) {
+            const Batch& batch = Batch(), bool rows = true) {
     int rc = check_inputs(h, pos, num, N, centers, C, sites);
     if (rc) return rc;
     if (batch.struct_ptr && (h->pbc[0] || h->pbc[1] || h->pbc[2]))
@@ -499,7 +505,8 @@ int prepare(soap_t* h, const float* pos, const int32_t* num, int64_t N, const do
     if (h->planned_atoms < 0 || N > h->planned_atoms || C > h->planned_centers) {
         if ((rc = plan(h, pos, num, N, g, centers, sites, C, st, batch))) return rc;
     }
-    if ((rc = launch_neighbors(h, pos, num, N, g, centers, sites, C, row_ptr_out ? row_ptr_out : h->d_row_ptr, st, batch))) return rc;
+    if ((rc = launch_neighbors(h, pos, num, N, g, centers, sites, C, row_ptr_out ? row_ptr_out : h->d_row_ptr, st, batch, rows))) return rc;
+    h->list_sorted = rows;
     if (h->weight.fn && C > 0) {
         pair_weight_kernel<<<(unsigned)((C + 7) / 8), 256, 0, st>>>(pos, centers, sites, C, g, h->d_pair_start, h->d_pair_count, h->d_pair_key,
                                                                    h->cap_pairs, h->d_counters, h->weight, h->d_pair_w);
@@ -622,6 +629,7 @@ static int neighbors_impl(soap_t* h, const float* d_positions, const int32_t* d_
     cudaStream_t st = (cudaStream_t)stream;
     if ((rc = plan(h, d_positions, d_numbers, n_atoms, g, d_centers, d_sites, n_centers, st, batch))) return rc;
     if ((rc = launch_neighbors(h, d_positions, d_numbers, n_atoms, g, d_centers, d_sites, n_centers, h->d_row_ptr, st, batch))) return rc;
+    h->list_sorted = true;
     CU(cudaMemcpyAsync(h->h_counters, h->d_counters, sizeof(Counters), cudaMemcpyDeviceToHost, st));
     CU(cudaStreamSynchronize(st));
     h->last_centers = n_centers;
@@ -646,6 +654,7 @@ int soap_neighbor_list(soap_t* h, int64_t* d_pair_ptr, int32_t* d_pair_atom, int
                        int64_t capacity_pairs, void* stream) {
     if (!h || !d_pair_ptr || !d_pair_atom || capacity_pairs < 0) return SOAP_ERR_INVALID_ARG;
     if (!h->tables_ready || h->planned_atoms < 0) return fail(h, SOAP_ERR_INVALID_ARG, "no neighbour list has been built yet");
+    if (!h->list_sorted) return fail(h, SOAP_ERR_INVALID_ARG, "the last call was descriptor-only and kept its pairs unsorted: call soap_neighbors first");
     cudaStream_t st = (cudaStream_t)stream;
     // the pair arrays are addressed by segment: make the compact row pointers first, then gather
     scan_counts(h, h->d_pair_count, (long long*)d_pair_ptr, h->last_centers, nullptr, st);
@@ -661,7 +670,7 @@ static int descriptor_impl(soap_t* h, const float* d_positions, const int32_t* d
     if (h && n_centers > 0 && !d_out) return fail(h, SOAP_ERR_INVALID_ARG, "d_out must not be NULL");
     Geometry g;
     cudaStream_t st = (cudaStream_t)stream;
-    int rc = prepare(h, d_positions, d_numbers, n_atoms, cell, d_centers, n_centers, nullptr, g, st, d_sites, batch);
+    int rc = prepare(h, d_positions, d_numbers, n_atoms, cell, d_centers, n_centers, nullptr, g, st, d_sites, batch, false);
     if (rc) return rc;
     if (n_centers > 0) {
         CenterParams cp;
@@ -875,7 +884,7 @@ int soap_coefficients(soap_t* h, const float* d_positions, const int32_t* d_numb
     if (h && n_centers > 0 && !d_out) return fail(h, SOAP_ERR_INVALID_ARG, "d_out must not be NULL");
     Geometry g;
     cudaStream_t st = (cudaStream_t)stream;
-    int rc = prepare(h, d_positions, d_numbers, n_atoms, cell, d_centers, n_centers, nullptr, g, st);
+    int rc = prepare(h, d_positions, d_numbers, n_atoms, cell, d_centers, n_centers, nullptr, g, st, nullptr, Batch(), false);
     if (rc) return rc;
     if (n_centers > 0) {
         CenterParams cp;
@@ -918,7 +927,7 @@ int soap_descriptor_average(soap_t* h, int mode, const float* d_positions, const
     if (!d_out) return fail(h, SOAP_ERR_INVALID_ARG, "d_out must not be NULL");
     Geometry g;
     cudaStream_t st = (cudaStream_t)stream;
-    int rc = prepare(h, d_positions, d_numbers, n_atoms, cell, d_centers, n_centers, nullptr, g, st);
+    int rc = prepare(h, d_positions, d_numbers, n_atoms, cell, d_centers, n_centers, nullptr, g, st, nullptr, Batch(), false);
     if (rc) return rc;
     const int F = (int)h->F, W = h->S * h->n_max * (h->l_max + 1) * (h->l_max + 1);
     const bool inner = mode == SOAP_AVERAGE_INNER;
