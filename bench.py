@@ -251,7 +251,7 @@ def run_cuda(args):
     import torch
     import torch.distributed as dist
     import paper_2609_05709_b200 as pkg
-    from paper_2609_05709_b200.replicas import job_throughput, max_over_ranks
+    from paper_2609_05709_b200.replicas import job_throughput, max_over_ranks, split_centers
 
     world = int(os.environ.get("WORLD_SIZE", "1"))
     rank = int(os.environ.get("RANK", "0"))
@@ -267,11 +267,16 @@ def run_cuda(args):
     pbc = (True, True, True) if s.cell is not None else (False, False, False)
     soap = pkg.Soap(species, r_cut, n_max, l_max, sigma, rbf, pbc)
     F = soap.n_features
-    C = s.n_atoms
+    # --shard: ONE structure for the whole job, every rank computes a contiguous range of its centres (no exchange:
+    # a centre needs only the atoms in its own sphere); otherwise every rank runs the whole structure (replicas)
+    shard = bool(args.shard) and world > 1
+    c_lo, c_hi = split_centers(s.n_atoms, world, rank) if shard else (0, s.n_atoms)
+    C = c_hi - c_lo
     pos_host = torch.from_numpy(s.positions).pin_memory()
     num_host = torch.from_numpy(s.numbers).pin_memory()
     pos, num = pos_host.cuda(), num_host.cuda()
-    n_pairs, n_rows = soap.neighbors(pos, num, s.cell)               # sizes scratch and the Jacobian (untimed, like construction)
+    centers = torch.arange(c_lo, c_hi, dtype=torch.int32, device="cuda") if shard else None
+    n_pairs, n_rows = soap.neighbors(pos, num, s.cell, centers)      # sizes scratch and the Jacobian (untimed, like construction)
     dev = {"pos": torch.empty_like(pos), "num": torch.empty_like(num),
            "desc": torch.empty((C, F), device="cuda"), "jac": torch.empty((n_rows, 3, F), device="cuda"),
            "row_ptr": torch.empty(C + 1, dtype=torch.int64, device="cuda"),
@@ -280,7 +285,7 @@ def run_cuda(args):
     soap.profile(True)
 
     def step():
-        soap.derivatives_into(pos, num, s.cell, None, dev["desc"], dev["jac"], dev["row_ptr"], dev["row_atom"])
+        soap.derivatives_into(pos, num, s.cell, centers, dev["desc"], dev["jac"], dev["row_ptr"], dev["row_atom"])
 
     def barrier():
         if world > 1:
@@ -322,7 +327,7 @@ def run_cuda(args):
     if e2e_steps:
         host_out = {k: torch.empty(v.shape, dtype=v.dtype).pin_memory() for k, v in dev.items() if k not in ("pos", "num")}
         for _ in range(2):
-            soap.derivatives_host(pos_host, num_host, s.cell, host_out, dev)
+            soap.derivatives_host(pos_host, num_host, s.cell, host_out, dev, centers)
     torch.cuda.synchronize()
     barrier()
     e2e_ms = []
@@ -343,8 +348,9 @@ def run_cuda(args):
             dist.destroy_process_group()
         return
     ms_per_step = total_ms / args.steps
-    value = job_throughput(C, world, ms_per_step)
-    e2e_value = job_throughput(C, world, e2e_total / e2e_steps) if e2e_steps else None
+    units, ranks = (s.n_atoms, 1) if shard else (C, world)           # sharded: the job is the one structure
+    value = job_throughput(units, ranks, ms_per_step)
+    e2e_value = job_throughput(units, ranks, e2e_total / e2e_steps) if e2e_steps else None
     # ---- roofline of the dominant kernel (the fused per-centre kernel): HBM-write bound ----
     # algorithmic bytes per launch: Jacobian rows + descriptor + row_atom written, pair list and positions read
     alg_bytes = n_rows * 3 * F * 4 + C * F * 4 + n_rows * 4 + n_pairs * (8 + 4 + 12) + (C + 1) * 16
@@ -385,8 +391,8 @@ def run_cuda(args):
             "fp32_floor_ms": 2.0 * desc_only["fma"] / (fp32_tflops * 1e12) * 1e3}
     print(json.dumps({
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3),
-        "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
-        "dtype": "f32", "data": "synthetic", "config": config_dict(name, s),
+        "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "strong" if shard else "weak", "vs_baseline": None,
+        "dtype": "f32", "data": "synthetic", "config": dict(config_dict(name, s), **({"parallelism": f"centres of one structure sharded over {world} GPUs, no exchange"} if shard else {})),
         "clocks": clocks,
         "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                 "ms_per_step": e2e_total / e2e_steps if e2e_steps else None, "steps": e2e_steps},
@@ -681,6 +687,9 @@ def main():
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="cuda", choices=["cuda", "reference"])
     ap.add_argument("--workload", default=DEFAULT_WORKLOAD, choices=sorted(WORKLOADS))
+    ap.add_argument("--shard", action="store_true",
+                    help="with --gpus N > 1: shard the centres of ONE structure over the ranks (strong scaling) "
+                         "instead of running N independent replicas")
     ap.add_argument("--kernel-only", action="store_true",
                     help="skip the end-to-end and CPU-baseline legs (for profiler captures)")
     ap.add_argument("--suite", choices=["map", "scaling", "configs", "desc30k", "modes", "driver", "compact", "graph", "small"],

@@ -443,14 +443,14 @@ class Soap:
         self._check(self._lib.soap_profile_read(self._h, C.byref(a), C.byref(b)))
         return float(a.value), float(b.value)
 
-    def derivatives_host(self, positions, numbers, cell, host_out, dev_buf):
+    def derivatives_host(self, positions, numbers, cell, host_out, dev_buf, centers=None):
         """End-to-end call on HOST buffers: copies the (pinned) inputs to the device,
         computes, and copies descriptor, Jacobian, row_ptr and row_atom back into the
         pinned tensors of `host_out`.  `dev_buf` holds the device staging tensors.
         Everything is enqueued on the current stream; the caller synchronises."""
         dev_buf["pos"].copy_(positions, non_blocking=True)
         dev_buf["num"].copy_(numbers, non_blocking=True)
-        self.derivatives_into(dev_buf["pos"], dev_buf["num"], cell, None, dev_buf["desc"], dev_buf["jac"],
+        self.derivatives_into(dev_buf["pos"], dev_buf["num"], cell, centers, dev_buf["desc"], dev_buf["jac"],
                               dev_buf["row_ptr"], dev_buf["row_atom"])
         for k in ("desc", "jac", "row_ptr", "row_atom"):
             host_out[k].copy_(dev_buf[k], non_blocking=True)

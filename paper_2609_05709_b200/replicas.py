@@ -25,7 +25,8 @@ def job_throughput(units_per_rank: int, world_size: int, slowest_ms: float) -> f
 
 
 def split_centers(n_centers: int, world_size: int, rank: int):
-    """Contiguous, near-equal range of centre indices for `rank` (for sharding one structure)."""
+    """Contiguous, near-equal range of centre indices for `rank`: how `bench.py --shard` cuts one structure
+    into one piece per GPU (a centre needs only the atoms inside its sphere, so nothing is exchanged)."""
     base, extra = divmod(n_centers, world_size)
     lo = rank * base + min(rank, extra)
     return lo, lo + base + (1 if rank < extra else 0)

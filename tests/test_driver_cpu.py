@@ -77,6 +77,27 @@ def test_two_workers_reproduce_the_single_call(derivatives):
             assert r.jacobian is None
 
 
+def test_three_workers_and_an_uneven_task_list():
+    """Seven tasks on three workers (3 + 2 + 2), one of the structures empty: the pieces still come back complete
+    and in order."""
+    structs = _structures()
+    empty = small_periodic_cell(3, (True, True, False))
+    empty.positions, empty.numbers = empty.positions[:0].copy(), empty.numbers[:0].copy()
+    structs.insert(1, empty)
+    tasks = driver.enumerate_tasks([int(s.positions.shape[0]) for s in structs], 2)
+    assert len(tasks) == 7 and [len(driver.tasks_of_rank(tasks, 3, r)) for r in range(3)] == [3, 2, 2]
+    results, _ = driver.generate(CONFIG, structs, batch=2, derivatives=True, world=3,
+                                 backend_factory=oracle_backend, timeout=180)
+    o = SoapOracle(**CONFIG)
+    assert len(results) == 3 and results[1].descriptor.shape[0] == 0
+    for s, r in zip(structs, results):
+        if s.positions.shape[0] == 0:
+            continue
+        ref = o.derivatives(s.positions, s.numbers, s.cell)
+        assert np.array_equal(r.descriptor, ref.descriptor) and np.array_equal(r.row_ptr, ref.row_ptr)
+        assert np.array_equal(r.row_atom, ref.row_atom) and np.array_equal(r.jacobian, ref.jacobian)
+
+
 def test_a_worker_that_fails_in_setup_ends_the_job():
     with pytest.raises(RuntimeError, match="worker 1 failed during set-up"):
         driver.generate(CONFIG, _structures(), batch=3, world=2, backend_factory=failing_backend, timeout=60)

@@ -1,5 +1,5 @@
 """The multi-GPU driver with its CUDA backend on the one GPU of the test box: a single worker process
-must reproduce the direct call bit for bit."""
+must reproduce the direct call bit for bit, and its results must match the oracle."""
 import numpy as np
 import pytest
 
@@ -29,3 +29,22 @@ def test_one_worker_equals_the_direct_call():
         assert np.array_equal(r.jacobian, ref.jacobian.cpu().numpy())
     desc_only, _ = driver.generate(config, structs[:1], batch=25, derivatives=False, world=1, timeout=300)
     assert same_values(desc_only[0].descriptor, results[0].descriptor) and desc_only[0].jacobian is None
+
+
+def test_one_worker_against_the_oracle():
+    """The driver's output (descriptor, rows, row bookkeeping, batches put together on the host) against the fp64
+    oracle, not against another call of the library."""
+    if not torch.cuda.is_available():
+        pytest.skip("no CUDA device")
+    from oracle.soap import SoapOracle
+    from paper_2609_05709_b200 import driver
+    from test_gpu_parity import DESC_TOL, JAC_TOL, col_err
+    config = dict(species=[1, 8], r_cut=4.5, n_max=4, l_max=3, sigma=0.5)
+    structs = [water_cluster(11, 5), water_cluster(3, 6)]
+    results, _ = driver.generate(config, structs, batch=7, derivatives=True, world=1, timeout=300)
+    oracle = SoapOracle([1, 8], 4.5, 4, 3, 0.5)
+    for s, r in zip(structs, results):
+        ref = oracle.derivatives(s.positions, s.numbers)
+        assert np.array_equal(r.row_ptr, ref.row_ptr) and np.array_equal(r.row_atom, ref.row_atom)
+        assert col_err(r.descriptor, ref.descriptor, 0) < DESC_TOL
+        assert col_err(r.jacobian, ref.jacobian, (0, 1)) < JAC_TOL

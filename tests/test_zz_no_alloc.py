@@ -39,6 +39,23 @@ def test_static_scratch_counts_match_twice_in_a_row():
         got = pkg.neighbor_counts_static(pos, r_cut, out=out)
         torch.cuda.synchronize()
         assert torch.equal(got, want)                            # integer work: exact
+    # nothing is allocated on the device by a call whose output tensor is the caller's
+    torch.cuda.synchronize()
+    free_before, _ = torch.cuda.mem_get_info()
+    pkg.neighbor_counts_static(pos, r_cut, out=out)
+    torch.cuda.synchronize()
+    free_after, _ = torch.cuda.mem_get_info()
+    assert free_after == free_before
+    # the largest structure the fixed scratch takes: 65536 atoms, spread thinly so that the bin grid hits its cap
+    rng = np.random.default_rng(5)
+    big = (rng.random((65536, 3)) * 400.0).astype(np.float32)
+    big[1] = big[0] + np.float32(0.5)                              # at least one pair for sure
+    bpos = torch.from_numpy(big).cuda()
+    bnum = torch.ones(65536, dtype=torch.int32, device="cuda")
+    ptr, _, _ = pkg.Soap([1], 6.0, 2, 1, 0.5).neighbor_list(bpos, bnum)
+    got = pkg.neighbor_counts_static(bpos, 6.0)
+    torch.cuda.synchronize()
+    assert torch.equal(got, (ptr[1:] - ptr[:-1]).to(torch.int32)) and int(got.sum()) >= 2
     # sizes beyond the fixed scratch are refused with a message and nothing runs
     lib = pkg.load_library()
     msg = ctypes.create_string_buffer(256)
