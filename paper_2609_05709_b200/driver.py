@@ -107,18 +107,11 @@ def cuda_backend(rank: int, config: dict):
         else:
             out = {"desc": soap.descriptor(pos, num, struct.cell, centers)}
             soap.status()
-        # one copy, device -> shared host memory the driver maps.  The shared segment is page-locked for the
-        # copy (registered with the CUDA runtime), so that the device writes it at PCIe speed instead of going
-        # through a pageable staging buffer; it is unregistered again before the handle travels to the driver.
+        # one copy, device -> shared host memory the driver maps (pageable: page-locking the segment for the copy
+        # with cudaHostRegister was measured and costs more than it saves when every task has buffers of its own)
         host = {k: torch.empty(v.shape, dtype=v.dtype).share_memory_() for k, v in out.items()}
-        cudart = torch.cuda.cudart()
         for k, v in out.items():
-            nbytes = host[k].numel() * host[k].element_size()
-            pinned = nbytes >= (1 << 20) and int(cudart.cudaHostRegister(host[k].data_ptr(), nbytes, 0)) == 0
             host[k].copy_(v)
-            if pinned:
-                torch.cuda.synchronize()
-                cudart.cudaHostUnregister(host[k].data_ptr())
         return host
 
     # warm-up: one tiny call so that module loading and first-launch costs are paid before the start signal
