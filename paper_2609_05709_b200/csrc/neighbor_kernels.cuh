@@ -453,6 +453,53 @@ __device__ inline void for_each_candidate(const Geometry& geom, const GridParams
     }
 }
 
+// The same walk for the common case (no periodic axis, stencil of +-1 bin): the three bins of a stencil row along
+// x are neighbours in the sorted atom array, so the 27 bins are 9 contiguous runs.  Every lane keeps the nine run
+// boundaries in registers, and a candidate finds its run with compares instead of shuffles.
+template <class F>
+__device__ inline void for_each_candidate_runs(const Geometry& geom, const GridParams& g, const int* __restrict__ cell_start,
+                                               const float4* __restrict__ s_pos, float xi, float yi, float zi,
+                                               const int bi[3], int lane, F f) {
+    // lane r < 9 fetches run r = (dy + 1) + 3 (dz + 1)
+    int start = 0, cnt = 0;
+    if (lane < 9) {
+        const int cy = bi[1] + lane % 3 - g.R[1], cz = bi[2] + lane / 3 - g.R[2];
+        const bool inside = cy >= 0 && cy < g.nb[1] && cz >= 0 && cz < g.nb[2] && (lane % 3 <= 2 * g.R[1]) && (lane / 3 <= 2 * g.R[2]);
+        if (inside) {
+            const int x0 = max(bi[0] - g.R[0], 0), x1 = min(bi[0] + g.R[0], g.nb[0] - 1);
+            const int row = (cz * g.nb[1] + cy) * g.nb[0];
+            start = cell_start[row + x0];
+            cnt = cell_start[row + x1 + 1] - start;
+        }
+    }
+    int r_start[9], r_end[9], total = 0;                 // run r covers candidates r_end[r] - count .. r_end[r] - 1
+#pragma unroll
+    for (int r = 0; r < 9; ++r) {
+        const int c = __shfl_sync(0xffffffffu, cnt, r);
+        r_start[r] = __shfl_sync(0xffffffffu, start, r) - total;      // atom index = r_start[r] + t for t inside run r
+        total += c;
+        r_end[r] = total;
+    }
+    for (int t0 = 0; t0 < total; t0 += 32) {
+        const int t = t0 + lane;
+        bool valid = false;
+        unsigned long long key = 0;
+        if (t < total) {
+            int at = r_start[8];
+#pragma unroll
+            for (int r = 7; r >= 0; --r) at = t < r_end[r] ? r_start[r] : at;
+            const float4 pj = s_pos[at + t];
+            const double dx = __dsub_rn((double)pj.x, (double)xi);
+            const double dy = __dsub_rn((double)pj.y, (double)yi);
+            const double dz = __dsub_rn((double)pj.z, (double)zi);
+            const double d2 = __dadd_rn(__dadd_rn(__dmul_rn(dx, dx), __dmul_rn(dy, dy)), __dmul_rn(dz, dz));
+            valid = (d2 < geom.rc2) && (d2 > 0.0);
+            key = ((unsigned long long)(unsigned)__float_as_int(pj.w) << 24) | 0x808080ull;
+        }
+        f(valid, key);
+    }
+}
+
 // One warp per centre: number of pairs.
 __global__ void count_kernel(const float* __restrict__ pos, const int* __restrict__ centers, long long C, Geometry geom,
                              const GridParams* __restrict__ gp, const int* __restrict__ atom_cell, const int* __restrict__ atom_wrap,
@@ -521,13 +568,15 @@ pairs_kernel(const float* __restrict__ pos, const int* __restrict__ centers, con
     }
     // ---- walk the candidates; keep the keys on chip while they fit ----
     int k = 0;
-    for_each_candidate(geom, g, cell_start, s_pos, s_wrap, xi, yi, zi, bi, wi, lane, counters,
-                       [&](bool valid, unsigned long long key) {
-                           const unsigned m = __ballot_sync(0xffffffffu, valid);
-                           const int at = k + __popc(m & ((1u << lane) - 1));
-                           if (valid && at < KEYS) s_raw[wid][at] = key;
-                           k += __popc(m);
-                       });
+    auto collect = [&](bool valid, unsigned long long key) {
+        const unsigned m = __ballot_sync(0xffffffffu, valid);
+        const int at = k + __popc(m & ((1u << lane) - 1));
+        if (valid && at < KEYS) s_raw[wid][at] = key;
+        k += __popc(m);
+    };
+    const bool runs = !(g.periodic[0] | g.periodic[1] | g.periodic[2]) && g.R[0] <= 1 && g.R[1] <= 1 && g.R[2] <= 1;
+    if (runs) for_each_candidate_runs(geom, g, cell_start, s_pos, xi, yi, zi, bi, lane, collect);
+    else for_each_candidate(geom, g, cell_start, s_pos, s_wrap, xi, yi, zi, bi, wi, lane, counters, collect);
     long long base = 0;
     if (lane == 0) base = (long long)atomicAdd(reinterpret_cast<unsigned long long*>(&counters->n_pairs), (unsigned long long)k);
     base = __shfl_sync(0xffffffffu, base, 0);
