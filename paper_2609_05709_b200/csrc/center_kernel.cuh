@@ -101,19 +101,22 @@ __device__ __forceinline__ void bulk_store(float* dst, const float* src_shared, 
 __device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
 __device__ __forceinline__ void bulk_wait_read() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
 
-// KIND: 1 descriptor and Jacobian, 2 coefficients c^mu_nlm and their Jacobian.
+// KIND: 1 descriptor and Jacobian, 2 coefficients c^mu_nlm and their Jacobian, 3 Jacobian of the inner average
+// (every atom a centre; given mean coefficients; one row per atom, no per-pair rows).
 // PLAIN: the default configuration (every species pair, atom centres, no weighting, full rows, own
 // coefficients); the options are then compile-time constants and their code drops out.
 template <int KIND, int L, int NMAX_T, bool PLAIN>
 __global__ void __launch_bounds__(kThreads, kMinCtas)
 center_kernel(const CenterParams p) {
-    static_assert(KIND == 1 || KIND == 2, "descriptor-only builds run desc_kernel");
+    static_assert(KIND >= 1 && KIND <= 3, "descriptor-only builds run desc_kernel");
     constexpr bool CC = KIND == 2;
     const bool o_compact = !PLAIN && p.compact, o_cross = PLAIN || p.crossover;
     const float* const o_cbar = PLAIN ? nullptr : p.c_bar;
     const float* const o_sites = PLAIN ? nullptr : p.sites;
     const float2* const o_pw = PLAIN ? nullptr : p.pair_w;
     const float o_w0 = PLAIN ? 1.f : p.w0;
+    constexpr bool o_inner = KIND == 3;
+    const float o_scale = o_inner ? p.own_scale : 1.f;
     constexpr int L1 = L + 1, LM = L1 * L1, LMP = LM | 1;      // odd row stride: no shared-memory bank conflicts
     constexpr int NMAX_BOUND = NMAX_T ? NMAX_T : 16;
     // pass-1 ownership: W_LM warps cover the lm index, SLOTS such groups split the n index
@@ -279,8 +282,13 @@ center_kernel(const CenterParams p) {
             __syncthreads();
             special = stage_geometry(g0, gc);
             float ac[NPT], ax[NPT], ay[NPT], az[NPT];
+            // inner average: q = sum over the neighbour centres i of grad_a c(i), the gradient of THEIR coefficients with
+            // respect to this atom a.  Centre i sees a at -d, and [G grad S + Ghat d S](-d) = (-1)^(l+1) [..](d), so q
+            // is built from the very terms that go into D; it belongs to the block of this atom's species
+            float qx[NPT], qy[NPT], qz[NPT];
+            const float q_sign = (own_l & 1) ? 1.f : -1.f;
 #pragma unroll
-            for (int k = 0; k < NPT; ++k) ac[k] = ax[k] = ay[k] = az[k] = 0.f;
+            for (int k = 0; k < NPT; ++k) ac[k] = ax[k] = ay[k] = az[k] = qx[k] = qy[k] = qz[k] = 0.f;
             int cur = -1;
             auto flush = [&]() {
                 if (cur < 0 || !owner) return;
@@ -322,6 +330,11 @@ center_kernel(const CenterParams p) {
                                         ax[k] = fmaf(gg.x, hy, fmaf(gg.y, tx, ax[k]));
                                         ay[k] = fmaf(gg.x, hz, fmaf(gg.y, ty, ay[k]));
                                         az[k] = fmaf(gg.x, hw, fmaf(gg.y, tz, az[k]));
+                                        if (o_inner) {
+                                            qx[k] = fmaf(q_sign, fmaf(gg.x, hy, gg.y * tx), qx[k]);
+                                            qy[k] = fmaf(q_sign, fmaf(gg.x, hz, gg.y * ty), qy[k]);
+                                            qz[k] = fmaf(q_sign, fmaf(gg.x, hw, gg.y * tz), qz[k]);
+                                        }
                                     }
                             }
                         }
@@ -330,6 +343,17 @@ center_kernel(const CenterParams p) {
                 __syncthreads();
             }
             flush();
+            if (o_inner && owner) {
+                // D - q in the block of this atom's species: minus the sum over ALL centres of grad_a c, the centre itself included
+#pragma unroll
+                for (int k = 0; k < NPT; ++k) {
+                    const int n = n0 + own_slot + k * SLOTS;
+                    if (n < NMAX) {
+                        const int e = (zi_species * NMAX + n) * LMP + own_lm;
+                        D_t[e] -= qx[k]; D_t[CT + e] -= qy[k]; D_t[2 * CT + e] -= qz[k];
+                    }
+                }
+            }
         }
     }
     __syncthreads();
@@ -379,6 +403,7 @@ center_kernel(const CenterParams p) {
         // species-compact rows: the centre's own row keeps every block and lives in an array of its own;
         // its slot among the compact rows is zero-filled
         float* own = !has_own ? nullptr
+                     : o_inner   ? p.out_jac + (size_t)ci * 3 * F              // row of atom a in the (atoms, 3, F) result
                      : o_compact ? p.out_center + (size_t)c_idx * 3 * F
                                  : p.out_jac + (size_t)(row_base + p.self_row[c_idx]) * 3 * F;
         if (has_own && o_compact) {
@@ -409,10 +434,14 @@ center_kernel(const CenterParams p) {
                 }
                 if (staged) {
                     slab[fl] = kl * acc;
-                    slab[nf + fl] = -kl * ax; slab[2 * nf + fl] = -kl * ay; slab[3 * nf + fl] = -kl * az;
+                    const float ks = -kl * o_scale;
+                    slab[nf + fl] = ks * ax; slab[2 * nf + fl] = ks * ay; slab[3 * nf + fl] = ks * az;
                 } else {
                     if (write_desc) desc_row[f0 + fl] = kl * acc;
-                    if (has_own) { own[f0 + fl] = -kl * ax; own[(size_t)F + f0 + fl] = -kl * ay; own[(size_t)2 * F + f0 + fl] = -kl * az; }
+                    if (has_own) {
+                        const float ks = -kl * o_scale;
+                        own[f0 + fl] = ks * ax; own[(size_t)F + f0 + fl] = ks * ay; own[(size_t)2 * F + f0 + fl] = ks * az;
+                    }
                 }
             }
             if (staged) {
@@ -428,8 +457,9 @@ center_kernel(const CenterParams p) {
                 __syncthreads();
             }
         }
-        if (has_own && tid == 0) p.row_atom[row_base + p.self_row[c_idx]] = ci;
+        if (has_own && !o_inner && tid == 0) p.row_atom[row_base + p.self_row[c_idx]] = ci;
     }
+    if (o_inner) return;             // the averaged row of this atom is complete: no per-pair rows
     __syncthreads();
     // fold K_l into c for pass 2
     if (!CC)

@@ -112,7 +112,8 @@ struct soap_handle {
     int *d_cell_count = nullptr, *d_cell_start = nullptr;
     int *d_pair_count = nullptr, *d_row_count = nullptr, *d_self_row = nullptr;
     long long *d_pair_ptr = nullptr, *d_pair_start = nullptr, *d_row_ptr = nullptr, *d_tile_offsets = nullptr;
-    int* d_tile_sums = nullptr;
+    int *d_tile_sums = nullptr, *d_cell_tile_sums = nullptr;
+    long long* d_cell_tile_offsets = nullptr;
     unsigned long long *d_pair_key = nullptr, *d_pair_tmp = nullptr;
     int* d_pair_row = nullptr;
     float2* d_pair_w = nullptr;          // per-pair weights, only with a radial weighting
@@ -220,6 +221,7 @@ int plan_smem(soap_t* h) {
     }
     CU(center_set_smem(kCenterDeriv, h->l_max, h->n_max, (int)h->smem_deriv));
     CU(center_set_smem(kCenterCoeff, h->l_max, h->n_max, (int)h->smem_deriv));
+    CU(center_set_smem(kCenterInner, h->l_max, h->n_max, (int)h->smem_deriv));
     return SOAP_OK;
 }
 
@@ -290,6 +292,8 @@ int ensure_scratch(soap_t* h, int64_t N, int64_t C, int64_t pairs) {
         int64_t cells = std::min<int64_t>(std::max<int64_t>(2 * cap, 4096), (int64_t)1 << 26);
         CU(regrow(&h->d_cell_count, cells + 1));
         CU(regrow(&h->d_cell_start, cells + 1));
+        CU(regrow(&h->d_cell_tile_sums, cells / kScanTile + 2));
+        CU(regrow(&h->d_cell_tile_offsets, cells / kScanTile + 3));
         h->cap_cells = cells;
         h->cap_atoms = cap;
     }
@@ -365,7 +369,13 @@ int launch_neighbors(soap_t* h, const float* pos, const int32_t* num, int64_t N,
         species_bbox_kernel<<<blocks_for(N, 256, 1024), 256, 0, st>>>(pos, num, N, g, h->d_zlut, h->d_species_idx, h->d_bbox, h->d_counters);
         grid_setup_kernel<<<1, 1, 0, st>>>(h->d_bbox, g, N, (int)h->cap_cells, h->d_grid, h->d_counters);
         bin_count_kernel<<<blocks_for(N, 256), 256, 0, st>>>(pos, N, g, h->d_grid, h->d_atom_cell, h->d_atom_wrap, h->d_cell_count, h->d_counters);
-        scan_kernel<int><<<1, 1024, 0, st>>>(h->d_cell_count, h->d_cell_start, h->cap_cells, nullptr, &h->d_grid->n_cells);
+        {
+            // exclusive scan of the bin counts over the whole (zero-filled) capacity, tile by tile
+            const long long tiles = (h->cap_cells + kScanTile - 1) / kScanTile;
+            tile_sum_kernel<<<(unsigned)tiles, 1024, 0, st>>>(h->d_cell_count, h->cap_cells, h->d_cell_tile_sums);
+            scan_kernel<long long><<<1, 1024, 0, st>>>(h->d_cell_tile_sums, h->d_cell_tile_offsets, tiles, nullptr);
+            tile_scan_kernel<int><<<(unsigned)tiles, 1024, 0, st>>>(h->d_cell_count, h->d_cell_start, h->cap_cells, h->d_cell_tile_offsets, tiles);
+        }
         bin_fill_kernel<<<blocks_for(N, 256), 256, 0, st>>>(pos, N, h->d_atom_cell, h->d_atom_wrap, h->d_cell_start, h->d_cell_count, h->d_s_pos, h->d_s_wrap);
     }
     if (C > 0 && !batch.struct_ptr && !brute) {
@@ -439,7 +449,7 @@ void fill_center_params(soap_t* h, CenterParams& cp, const float* pos, const int
     cp.feat_pack = h->d_feat; cp.nch_magic = (unsigned)((1ull << 32) / (unsigned)(h->n_max * (h->l_max + 1))) + 1u; cp.inv_h = h->basis.inv_h; cp.n_intervals = h->basis.n_intervals;
     cp.S = h->S; cp.n_max = h->n_max; cp.l_max = h->l_max; cp.F = (int)h->F;
     cp.P = h->P_deriv;
-    cp.crossover = h->crossover; cp.emit_coeff = 0; cp.c_bar = nullptr;
+    cp.crossover = h->crossover; cp.emit_coeff = 0; cp.c_bar = nullptr; cp.inner_rows = 0; cp.own_scale = 1.f;
     cp.pair_w = h->weight.fn ? h->d_pair_w : nullptr; cp.w0 = (float)h->w0;
     cp.compact = 0; cp.Fc = (int)h->Fc_pitch; cp.out_center = nullptr;
     cp.out_desc = nullptr; cp.out_jac = nullptr; cp.row_atom = nullptr;
@@ -584,7 +594,8 @@ void soap_destroy(soap_t* h) {
     void* ptrs[] = {h->d_table, h->d_table_ln, h->d_self, h->d_kl, h->d_feat, h->d_zlut, h->d_l_of_lm, h->d_counters, h->d_bbox,
                     h->d_grid, h->d_species_idx, h->d_atom_cell, h->d_atom_wrap, h->d_s_wrap, h->d_s_pos, h->d_cell_count,
                     h->d_cell_start, h->d_pair_count, h->d_row_count, h->d_self_row, h->d_order, h->d_pair_ptr, h->d_pair_start, h->d_row_ptr, h->d_tile_sums, h->d_tile_offsets,
-                    h->d_pair_key, h->d_pair_tmp, h->d_pair_row, h->d_work, h->d_pair_w, h->d_compact_map};
+                    h->d_pair_key, h->d_pair_tmp, h->d_pair_row, h->d_work, h->d_pair_w, h->d_compact_map,
+                    h->d_cell_tile_sums, h->d_cell_tile_offsets};
     for (void* p : ptrs) if (p) cudaFree(p);
     if (h->h_counters) cudaFreeHost(h->h_counters);
     for (cudaEvent_t e : h->ev) if (e) cudaEventDestroy(e);
@@ -966,6 +977,32 @@ int soap_derivatives_average(soap_t* h, int mode, const float* d_positions, cons
     cudaStream_t st = (cudaStream_t)stream;
     int rc = prepare(h, d_positions, d_numbers, n_atoms, cell, d_centers, n_centers, nullptr, g, st);
     if (rc) return rc;
+    if (mode == SOAP_AVERAGE_INNER && !d_centers && n_centers == n_atoms) {
+        // Inner average with every atom a centre: pbar = P(cbar) and d pbar / d r_a = dP/dcbar . (1/C) sum_i grad_a c(i).
+        // Centre i sees atom a where a sees i, mirrored, so the kernel of atom a collects that sum from its own
+        // pairs in pass 1 and contracts it with cbar like a centre's own row: no per-pair rows, no workspace for them.
+        const int W = h->S * h->n_max * (h->l_max + 1) * (h->l_max + 1);
+        const size_t o_rows = 0, o_partial = align256((size_t)n_centers * W * 4),
+                     o_cbar = o_partial + align256((size_t)kMeanMaxChunks * W * 8), total = o_cbar + align256((size_t)W * 4);
+        if ((rc = ensure_work(h, total))) return rc;
+        char* w = (char*)h->d_work;
+        CenterParams cp;
+        fill_center_params(h, cp, d_positions, d_centers, n_centers, g, false);
+        cp.out_desc = (float*)(w + o_rows);
+        cp.emit_coeff = 1;
+        if ((rc = launch_desc(h, cp, n_centers, st))) return rc;
+        if ((rc = column_mean(h, (const float*)(w + o_rows), n_centers, W, (double*)(w + o_partial), (float*)(w + o_cbar), st))) return rc;
+        fill_center_params(h, cp, d_positions, d_centers, n_centers, g, true);
+        cp.row_capacity = INT64_MAX;
+        cp.c_bar = (const float*)(w + o_cbar);
+        cp.out_desc = d_out_desc;
+        cp.out_jac = d_out_jac;
+        cp.inner_rows = 1;
+        cp.own_scale = (float)(1.0 / (double)n_centers);
+        CU(center_launch(kCenterInner, h->l_max, h->n_max, cp, (unsigned)n_centers, h->smem_deriv, st));
+        if (h->profiling) CU(cudaEventRecord(h->ev[2], st));
+        return SOAP_OK;
+    }
     // the row total sizes the workspace; a structure that outgrew its plan is planned again
     CU(cudaMemcpyAsync(h->h_counters, h->d_counters, sizeof(Counters), cudaMemcpyDeviceToHost, st));
     CU(cudaStreamSynchronize(st));

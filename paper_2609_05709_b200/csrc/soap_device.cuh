@@ -80,6 +80,10 @@ struct CenterParams {
     int crossover;                // 0: only the species pairs mu == nu are features
     int emit_coeff;               // descriptor build: write the coefficients c^mu_nlm instead of the power spectrum
     const float* c_bar;           // [S n_max (l_max+1)^2] or null: coefficients that replace the centre's own after pass 1
+    // inner average over ALL atoms as centres: the kernel writes, for its atom a, d pbar / d r_a = own_scale times the
+    // contraction of cbar with sum_i grad_a c(i) (pass 1 collects that sum) to out_jac[a], and no per-pair rows
+    int inner_rows;
+    float own_scale;
     // species-compact Jacobian rows: a neighbour's row holds only the blocks that involve its species (pitch Fc, a
     // multiple of 8 floats); the centre's own full row goes to out_center [C,3,F]
     int compact, Fc;
