@@ -480,33 +480,23 @@ __device__ inline void for_each_candidate_runs(const Geometry& geom, const GridP
         total += c;
         r_end[r] = total;
     }
-    // two candidates per lane and trip, so that two position loads are in flight
-    auto locate = [&](int t) {
-        int at = r_start[8];
+    for (int t0 = 0; t0 < total; t0 += 32) {
+        const int t = t0 + lane;
+        bool valid = false;
+        unsigned long long key = 0;
+        if (t < total) {
+            int at = r_start[8];
 #pragma unroll
-        for (int r = 7; r >= 0; --r) at = t < r_end[r] ? r_start[r] : at;
-        return at + t;
-    };
-    auto test = [&](bool have, const float4& pj, bool& valid, unsigned long long& key) {
-        const double dx = __dsub_rn((double)pj.x, (double)xi);
-        const double dy = __dsub_rn((double)pj.y, (double)yi);
-        const double dz = __dsub_rn((double)pj.z, (double)zi);
-        const double d2 = __dadd_rn(__dadd_rn(__dmul_rn(dx, dx), __dmul_rn(dy, dy)), __dmul_rn(dz, dz));
-        valid = have && (d2 < geom.rc2) && (d2 > 0.0);
-        key = ((unsigned long long)(unsigned)__float_as_int(pj.w) << 24) | 0x808080ull;
-    };
-    for (int t0 = 0; t0 < total; t0 += 64) {
-        const int ta = t0 + lane, tb = t0 + 32 + lane;
-        const bool ha = ta < total, hb = tb < total;
-        float4 pa = make_float4(0.f, 0.f, 0.f, 0.f), pb = pa;
-        if (ha) pa = s_pos[locate(ta)];
-        if (hb) pb = s_pos[locate(tb)];
-        bool va, vb;
-        unsigned long long ka, kb;
-        test(ha, pa, va, ka);
-        test(hb, pb, vb, kb);
-        f(va, ka);
-        if (t0 + 32 < total) f(vb, kb);
+            for (int r = 7; r >= 0; --r) at = t < r_end[r] ? r_start[r] : at;
+            const float4 pj = s_pos[at + t];
+            const double dx = __dsub_rn((double)pj.x, (double)xi);
+            const double dy = __dsub_rn((double)pj.y, (double)yi);
+            const double dz = __dsub_rn((double)pj.z, (double)zi);
+            const double d2 = __dadd_rn(__dadd_rn(__dmul_rn(dx, dx), __dmul_rn(dy, dy)), __dmul_rn(dz, dz));
+            valid = (d2 < geom.rc2) && (d2 > 0.0);
+            key = ((unsigned long long)(unsigned)__float_as_int(pj.w) << 24) | 0x808080ull;
+        }
+        f(valid, key);
     }
 }
 
