@@ -7,7 +7,10 @@ One step = one soap_derivatives call through the C ABI: cell-list neighbour sear
 expansion coefficients, power spectrum and every Jacobian row of all 3000 centres.
 Prints ONE JSON line (rank 0).  With --gpus N > 1 (launched under torch.distributed.run)
 every rank runs the same structure on its own GPU: the path has no exchange step, so
-ranks are independent replicas and the job throughput is N x structure / slowest rank.
+ranks are independent replicas and the job throughput is N x structure / slowest rank
+(--shard cuts the centres of ONE structure over the ranks instead).  The same line carries the
+descriptor-only half of the metric (soap_descriptor on a 1,000,002-atom cluster) with its FP32
+roofline, the FP32 rate measured in the run, and the oracle timed on every host core.
 
 --impl reference times the fp64 NumPy oracle on the host cores on a bounded sample of
 the same workload.
@@ -381,7 +384,7 @@ def run_cuda(args):
                               "unit": UNIT, "ms_per_step": desc_only["ms_per_step"], "workload": desc_only["workload"],
                               "atoms": desc_only["atoms"], "steps": desc_only["steps"]}
         extra["roofline_desc_only"] = {
-            "bound": "alu", "kernel": "desc_kernel<6,8,true>", "achieved": achieved_tf, "peak": fp32_tflops, "unit": "TFLOP/s",
+            "bound": "alu", "kernel": "desc_kernel<6,8,true,true>", "achieved": achieved_tf, "peak": fp32_tflops, "unit": "TFLOP/s",
             "frac": achieved_tf / fp32_tflops, "traffic": None,
             "peak_source": f"measured in this run: register-only FP32 multiply-add loop, {fp32_ms:.2f} ms "
                            f"(nominal 148 SM x 128 lanes x 2 x 1.965 GHz = {FP32_NOMINAL_TFLOPS:.1f})",
