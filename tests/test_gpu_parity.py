@@ -120,7 +120,7 @@ def test_centre_subset_and_isolated_atoms(pkg):
     check_derivatives(soap, oracle, s, centers)
 
 
-@pytest.mark.parametrize("n_max,l_max", [(2, 2), (6, 4), (8, 6), (10, 8), (12, 12), (1, 0), (5, 9)])
+@pytest.mark.parametrize("n_max,l_max", [(2, 2), (6, 4), (8, 6), (10, 8), (12, 12), (1, 0), (5, 9), (14, 2), (16, 1), (3, 11)])
 def test_basis_size_sweep_small_cluster(pkg, n_max, l_max):
     s = water_cluster(12, 5)
     args = ([1, 8], 6.0, n_max, l_max, 0.5, GTO)
