@@ -470,8 +470,8 @@ def time_case(struct, species, r_cut, n_max, l_max, sigma, rbf, mode, steps, war
         step = lambda: soap.descriptor_average(mode[8:], pos, num, struct.cell, None, out=avg)
         alg_bytes = F * 4 + n_pairs * 24 + (C + 1) * 8
     else:
-        # averaged Jacobian: what must move is the result; the per-centre rows are an intermediate
-        # (written once, read once) that the figure 'intermediate_bytes' counts
+        # averaged Jacobian: what must move is the result (with every atom a centre, as here, the kernels write one row
+        # per atom and nothing per pair; only centre subsets still pass per-centre rows through a workspace)
         avg = torch.empty(F, device="cuda")
         jac = torch.empty((C, 3, F), device="cuda")
         step = lambda: soap.derivatives_average(mode[8:13], pos, num, struct.cell, None, out_desc=avg, out_jac=jac)
@@ -501,8 +501,6 @@ def time_case(struct, species, r_cut, n_max, l_max, sigma, rbf, mode, steps, war
            "ms_per_step": ms, "atoms_per_s": C / (ms * 1e-3), "kernel_ms": k_ms, "neighbour_search_ms": statistics.median(nbr),
            "algorithmic_bytes": alg_bytes, "kernel_GBps": alg_bytes / (k_ms * 1e-3) / 1e9,
            "hbm_frac_of_measured_peak": alg_bytes / (k_ms * 1e-3) / 1e9 / peak}
-    if mode.endswith("_derivatives") and mode.startswith("average"):
-        out["intermediate_bytes"] = 2 * n_rows * 3 * F * 4
     del soap
     torch.cuda.empty_cache()
     return out

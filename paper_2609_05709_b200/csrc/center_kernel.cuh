@@ -102,21 +102,23 @@ __device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.comm
 __device__ __forceinline__ void bulk_wait_read() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
 
 // KIND: 1 descriptor and Jacobian, 2 coefficients c^mu_nlm and their Jacobian, 3 Jacobian of the inner average
-// (every atom a centre; given mean coefficients; one row per atom, no per-pair rows).
+// (every atom a centre; given mean coefficients; one row per atom, no per-pair rows), 4 Jacobian of the outer average
+// (every atom a centre; given the coefficients of all centres; one row per atom, no per-pair rows).
 // PLAIN: the default configuration (every species pair, atom centres, no weighting, full rows, own
 // coefficients); the options are then compile-time constants and their code drops out.
 template <int KIND, int L, int NMAX_T, bool PLAIN>
 __global__ void __launch_bounds__(kThreads, kMinCtas)
 center_kernel(const CenterParams p) {
-    static_assert(KIND >= 1 && KIND <= 3, "descriptor-only builds run desc_kernel");
+    static_assert(KIND >= 1 && KIND <= 4, "descriptor-only builds run desc_kernel");
     constexpr bool CC = KIND == 2;
     const bool o_compact = !PLAIN && p.compact, o_cross = PLAIN || p.crossover;
     const float* const o_cbar = PLAIN ? nullptr : p.c_bar;
     const float* const o_sites = PLAIN ? nullptr : p.sites;
     const float2* const o_pw = PLAIN ? nullptr : p.pair_w;
     const float o_w0 = PLAIN ? 1.f : p.w0;
-    constexpr bool o_inner = KIND == 3;
-    const float o_scale = o_inner ? p.own_scale : 1.f;
+    constexpr bool o_inner = KIND == 3, o_outer = KIND == 4;
+    constexpr bool o_atom_rows = o_inner || o_outer;               // the result has one row per atom, at the atom's index
+    const float o_scale = o_atom_rows ? p.own_scale : 1.f;
     constexpr int L1 = L + 1, LM = L1 * L1, LMP = LM | 1;      // odd row stride: no shared-memory bank conflicts
     constexpr int NMAX_BOUND = NMAX_T ? NMAX_T : 16;
     // pass-1 ownership: W_LM warps cover the lm index, SLOTS such groups split the n index
@@ -403,7 +405,7 @@ center_kernel(const CenterParams p) {
         // species-compact rows: the centre's own row keeps every block and lives in an array of its own;
         // its slot among the compact rows is zero-filled
         float* own = !has_own ? nullptr
-                     : o_inner   ? p.out_jac + (size_t)ci * 3 * F              // row of atom a in the (atoms, 3, F) result
+                     : o_atom_rows ? p.out_jac + (size_t)ci * 3 * F            // row of atom a in the (atoms, 3, F) result
                      : o_compact ? p.out_center + (size_t)c_idx * 3 * F
                                  : p.out_jac + (size_t)(row_base + p.self_row[c_idx]) * 3 * F;
         if (has_own && o_compact) {
@@ -457,10 +459,169 @@ center_kernel(const CenterParams p) {
                 __syncthreads();
             }
         }
-        if (has_own && !o_inner && tid == 0) p.row_atom[row_base + p.self_row[c_idx]] = ci;
+        if (has_own && !o_atom_rows && tid == 0) p.row_atom[row_base + p.self_row[c_idx]] = ci;
     }
     if (o_inner) return;             // the averaged row of this atom is complete: no per-pair rows
     __syncthreads();
+    if constexpr (o_outer) {
+        // Outer average with every atom a centre: d pbar / d r_a = (1/C) sum_i d p(i) / d r_a.  Besides its own row
+        // (written above) atom a has a row under every centre i that sees it, and those are the atoms that a sees.
+        // Centre i sees a at -d: S_lm(-d) = (-1)^l S_lm(d), grad S_lm(-d) = (-1)^(l+1) grad S_lm(d), and the
+        // displacement in Ghat d S changes sign as well, so the row of a under i is the product rule of this very
+        // pair with U, V contracted against c(i) instead of c(a), times (-1)^(l+1).  In rounds of one pair per warp:
+        // a warp copies c(i) to shared memory and forms U, V; then the threads, each with features of its own, add
+        // the pairs of the round in a fixed order (bit-repeatable).  Only the blocks that involve the species of a
+        // are touched; a thread keeps its sums in registers over all rounds when they are at most kSlots features
+        // per thread, else it adds to the row in global memory group by group, every round.
+        constexpr int kSlots = 4;
+        const int NI = S * NCH, SN = S * NMAX, Z = zi_species;
+        const int TRI = (NMAX * (NMAX + 1) / 2) * L1, SQ = NMAX * NCH;
+        const int NZ = TRI + (o_cross ? (S - 1) * SQ : 0);                     // features that involve species Z
+        float4* sUV = reinterpret_cast<float4*>(smem + lay.wUV);              // [kWarps][nu][n'][l]
+        float* c_copy = smem + lay.total + wid * CT;                          // [kWarps][S n_max][LMP], behind the usual layout
+        float* const row = p.out_jac + (size_t)ci * 3 * F;
+        // the x-th feature that involves Z: its place in the row and its operands, (radial index, U/V index) of one
+        // term, or of both in the same-species block (gB >= 0)
+        auto decode = [&](int x, int& f, int& gA, int& uA, int& gB, int& uB) {
+            gB = -1; uB = 0;
+            if (x < TRI) {
+                // block (Z, Z): after the blocks (mu, nu >= mu) of every mu < Z
+                f = o_cross ? Z * TRI + (Z * S - Z * (Z + 1) / 2) * SQ + x : Z * TRI + x;
+                const unsigned dec = tri_dec[x];
+                gA = dec & 255; gB = dec >> 8;
+                uA = Z * NCH + gB; uB = Z * NCH + gA;
+            } else {
+                const int y = x - TRI, o = y / SQ, e = y - o * SQ;
+                const int other = o < Z ? o : o + 1, mu = min(Z, other), nu = max(Z, other);
+                f = mu * TRI + (mu * S - mu * (mu + 1) / 2) * SQ + TRI + (nu - mu - 1) * SQ + e;
+                const int n1 = (int)__umulhi((unsigned)e, p.nch_magic);
+                const int j = e - n1 * NCH, i1 = n1 * L1 + (j % L1);
+                const bool first_term = mu == Z;                               // which factor belongs to atom a
+                gA = first_term ? i1 : j;
+                uA = other * NCH + (first_term ? j : i1);
+            }
+        };
+        const int n_groups = (NZ + kSlots * kThreads - 1) / (kSlots * kThreads);
+        const bool in_registers = n_groups == 1;
+        int sf[kSlots], sgA[kSlots], suA[kSlots], sgB[kSlots], suB[kSlots];
+        float ax[kSlots], ay[kSlots], az[kSlots];
+#pragma unroll
+        for (int k = 0; k < kSlots; ++k) {
+            ax[k] = ay[k] = az[k] = 0.f;
+            sf[k] = -1; sgA[k] = suA[k] = suB[k] = 0; sgB[k] = -1;
+            if (in_registers && k * kThreads + tid < NZ) decode(k * kThreads + tid, sf[k], sgA[k], suA[k], sgB[k], suB[k]);
+        }
+        for (int g0 = 0; g0 < k_pairs; g0 += kGeoPairs) {
+            const int gc = min(kGeoPairs, k_pairs - g0);
+            __syncthreads();
+            if (g0 > 0 || k_pairs > kGeoPairs) stage_geometry(g0, gc);        // otherwise still valid from pass 1
+            for (int q0 = 0; q0 < gc; q0 += P) {
+                const int pc = min(P, gc - q0);
+                stage_chunk(q0, pc);
+                __syncthreads();
+                for (int r0 = 0; r0 < pc; r0 += kWarps) {
+                    const int nr = min(kWarps, pc - r0);
+                    if (wid < nr) {
+                        const float* cj = p.c_all + (size_t)geo_j[q0 + r0 + wid] * W;   // every atom is a centre, in order
+                        for (int e = lane; e < W; e += 32) {
+                            const int r = e / LM;
+                            c_copy[r * LMP + (e - r * LM)] = __ldg(cj + e);
+                        }
+                        __syncwarp();
+                        const float4* wSD = sSD4 + (r0 + wid) * LMP;
+                        float4* wUV = sUV + wid * NI;
+                        if (SN <= 16) {
+                            // lane <-> (nu n', half): half 0 accumulates (U, Vx), half 1 (Vy, Vz)
+                            const int sn = lane >> 1, half = lane & 1;
+                            if (sn < SN) {
+                                const float* cp = c_copy + sn * LMP;
+                                const float2* hp = reinterpret_cast<const float2*>(wSD) + half;
+                                float2* up = reinterpret_cast<float2*>(wUV + sn * L1) + half;
+#pragma unroll
+                                for (int l = 0; l <= L; ++l) {
+                                    float2 acc = make_float2(0.f, 0.f);
+#pragma unroll
+                                    for (int m = 0; m <= 2 * l; ++m) {
+                                        const float cv = cp[l * l + m];
+                                        const float2 h = hp[2 * (l * l + m)];
+                                        acc.x = fmaf(cv, h.x, acc.x); acc.y = fmaf(cv, h.y, acc.y);
+                                    }
+                                    const float fl = ((l & 1) ? o_scale : -o_scale) * __ldg(p.kl + l);
+                                    up[2 * l] = make_float2(fl * acc.x, fl * acc.y);
+                                }
+                            }
+                        } else {
+                            for (int sn = lane; sn < SN; sn += 32) {
+                                const float* cp = c_copy + sn * LMP;
+#pragma unroll
+                                for (int l = 0; l <= L; ++l) {
+                                    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+                                    for (int m = 0; m <= 2 * l; ++m) {
+                                        const float cv = cp[l * l + m];
+                                        const float4 h = wSD[l * l + m];
+                                        acc.x = fmaf(cv, h.x, acc.x); acc.y = fmaf(cv, h.y, acc.y);
+                                        acc.z = fmaf(cv, h.z, acc.z); acc.w = fmaf(cv, h.w, acc.w);
+                                    }
+                                    const float fl = ((l & 1) ? o_scale : -o_scale) * __ldg(p.kl + l);
+                                    wUV[sn * L1 + l] = make_float4(fl * acc.x, fl * acc.y, fl * acc.z, fl * acc.w);
+                                }
+                            }
+                        }
+                    }
+                    __syncthreads();
+                    for (int grp = 0; grp < n_groups; ++grp) {
+                        if (!in_registers) {
+#pragma unroll
+                            for (int k = 0; k < kSlots; ++k) {
+                                const int x = (grp * kSlots + k) * kThreads + tid;
+                                sf[k] = -1;
+                                if (x < NZ) {
+                                    decode(x, sf[k], sgA[k], suA[k], sgB[k], suB[k]);
+                                    ax[k] = row[sf[k]]; ay[k] = row[(size_t)F + sf[k]]; az[k] = row[(size_t)2 * F + sf[k]];
+                                }
+                            }
+                        }
+                        for (int w = 0; w < nr; ++w) {
+                            const int g = q0 + r0 + w;
+                            if (!(geo_i[g].z & 256)) continue;                 // an image of a itself: part of its own row already
+                            const float4 d = geo_d[g];
+                            const float2* wG = sG2 + (r0 + w) * NCH;
+                            const float4* UV = sUV + w * NI;
+#pragma unroll
+                            for (int k = 0; k < kSlots; ++k) {
+                                if (sf[k] < 0) continue;
+                                const float2 g1 = wG[sgA[k]];
+                                const float4 u1 = UV[suA[k]];
+                                float t = g1.y * u1.x;
+                                if (sgB[k] >= 0) {
+                                    const float2 g2 = wG[sgB[k]];
+                                    const float4 u2 = UV[suB[k]];
+                                    t = fmaf(g2.y, u2.x, t);
+                                    ax[k] = fmaf(g2.x, u2.y, ax[k]); ay[k] = fmaf(g2.x, u2.z, ay[k]); az[k] = fmaf(g2.x, u2.w, az[k]);
+                                }
+                                ax[k] = fmaf(g1.x, u1.y, fmaf(t, d.x, ax[k]));
+                                ay[k] = fmaf(g1.x, u1.z, fmaf(t, d.y, ay[k]));
+                                az[k] = fmaf(g1.x, u1.w, fmaf(t, d.z, az[k]));
+                            }
+                        }
+                        if (!in_registers) {
+#pragma unroll
+                            for (int k = 0; k < kSlots; ++k)
+                                if (sf[k] >= 0) { row[sf[k]] = ax[k]; row[(size_t)F + sf[k]] = ay[k]; row[(size_t)2 * F + sf[k]] = az[k]; }
+                        }
+                    }
+                    __syncthreads();
+                }
+            }
+        }
+        if (in_registers) {
+#pragma unroll
+            for (int k = 0; k < kSlots; ++k)
+                if (sf[k] >= 0) { row[sf[k]] += ax[k]; row[(size_t)F + sf[k]] += ay[k]; row[(size_t)2 * F + sf[k]] += az[k]; }
+        }
+        return;
+    }
     // fold K_l into c for pass 2
     if (!CC)
         for (int e = tid; e < W; e += kThreads) {

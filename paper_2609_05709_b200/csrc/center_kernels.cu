@@ -78,6 +78,10 @@ cudaError_t SOAP_CAT(center_set_smem_l, SOAP_L)(int kind, int n_max, int bytes) 
         if ((e = set_one<3, 0, false>(bytes)) != cudaSuccess) return e;
         return set_one<3, 8, false>(bytes);
     }
+    if (kind == kCenterOuter) {
+        if ((e = set_one<4, 0, false>(bytes)) != cudaSuccess) return e;
+        return set_one<4, 8, false>(bytes);
+    }
     if (kind == kCenterCoeff) {
         if ((e = set_one<2, 0, false>(bytes)) != cudaSuccess) return e;
         switch (general_has_fixed_nmax(n_max) ? n_max : 0) {
@@ -107,6 +111,8 @@ cudaError_t SOAP_CAT(center_launch_l, SOAP_L)(int kind, int n_max, bool plain, c
                                               cudaStream_t st) {
     if (kind == kCenterInner)
         return n_max == 8 ? launch_one<3, 8, false>(p, grid, smem, st) : launch_one<3, 0, false>(p, grid, smem, st);
+    if (kind == kCenterOuter)
+        return n_max == 8 ? launch_one<4, 8, false>(p, grid, smem, st) : launch_one<4, 0, false>(p, grid, smem, st);
     if (kind == kCenterCoeff) {
         switch (general_has_fixed_nmax(n_max) ? n_max : 0) {
 #define X(N) case N: return launch_one<2, N, false>(p, grid, smem, st);

@@ -3,12 +3,13 @@
 #include "soap_device.cuh"
 
 namespace soap {
-// kernel kinds: descriptor and Jacobian; coefficients c^mu_nlm and their Jacobian; Jacobian of the inner average
-constexpr int kCenterDeriv = 1, kCenterCoeff = 2, kCenterInner = 3;
+// kernel kinds: descriptor and Jacobian; coefficients c^mu_nlm and their Jacobian; Jacobian of the inner average;
+// Jacobian of the outer average (the last two: every atom a centre, one row per atom)
+constexpr int kCenterDeriv = 1, kCenterCoeff = 2, kCenterInner = 3, kCenterOuter = 4;
 // whether the parameters ask for nothing beyond the default configuration (the kernels instantiated with
 // PLAIN = true assume exactly this)
 inline bool center_params_plain(const CenterParams& p) {
-    return p.crossover && !p.compact && !p.emit_coeff && !p.c_bar && !p.sites && !p.pair_w && p.w0 == 1.f && !p.inner_rows;
+    return p.crossover && !p.compact && !p.emit_coeff && !p.c_bar && !p.sites && !p.pair_w && p.w0 == 1.f && !p.inner_rows && !p.c_all;
 }
 // harmonic tables up to l = 12: anorm[91] (index l(l+1)/2 + m), dfact[16]
 cudaError_t center_constants(int l_max, const float* anorm91, const float* dfact16);

@@ -124,8 +124,9 @@ struct soap_handle {
     int64_t pairs_per_center_hint = 0;   // average at the last plan (chooses the pair kernel variant)
     int64_t last_centers = 0;
     bool list_sorted = false;            // whether the pair list of the last search is sorted (descriptor-only calls skip that)
-    int P_deriv = 16;
-    size_t smem_deriv = 0;
+    int P_deriv = 16, P_outer = 16;      // pairs per staged chunk: derivative kernels, kernel of the outer average
+    size_t smem_deriv = 0, smem_outer = 0;
+    bool outer_fast = false;             // whether the kernel of the outer average fits the shared memory
     // optional per-segment timing (events on the caller's stream)
     bool profiling = false;
     cudaEvent_t ev[3] = {nullptr, nullptr, nullptr};
@@ -200,28 +201,34 @@ int plan_smem(soap_t* h) {
     h->desc_warp_bytes = (size_t)make_desc_layout(h->S, desc_np(h->n_max), h->l_max, 1, 0).per_warp * 4;
     if (h->desc_warp_bytes > (size_t)max_smem) return fail(h, SOAP_ERR_INVALID_ARG, "this basis does not fit the shared memory of the device");
     CU(desc_set_smem(h->l_max, desc_np(h->n_max), max_smem));
-    {
-        // pairs per staged chunk of the derivative kernels: the largest that still leaves room for three CTAs per SM,
-        // else two, else whatever fits
+    // pairs per staged chunk of the derivative kernels: the largest that still leaves room for three CTAs per SM,
+    // else two, else whatever fits (`extra` bytes follow the usual layout); false if nothing fits
+    auto plan_chunk = [&](size_t extra, int& P_out, size_t& bytes_out) -> bool {
         int P = 32;
         size_t bytes = 0;
         const size_t budget3 = (size_t)228 * 1024 / 3 - 1024, budget2 = (size_t)228 * 1024 / 2 - 1024;
         for (int pass = 0; pass < 3; ++pass) {
             const size_t budget = pass == 0 ? budget3 : pass == 1 ? budget2 : (size_t)max_smem;
             for (P = 32; P >= 4; P /= 2) {
-                bytes = (size_t)make_layout(h->S, h->n_max, h->l_max, P, true, h->weight.fn != 0).total * 4;
+                bytes = (size_t)make_layout(h->S, h->n_max, h->l_max, P, true, h->weight.fn != 0).total * 4 + extra;
                 if (bytes <= budget) break;
             }
             if (P >= (pass == 2 ? 4 : 8) && bytes <= budget) break;
             if (P < 4) P = 4;
         }
-        bytes = (size_t)make_layout(h->S, h->n_max, h->l_max, P, true, h->weight.fn != 0).total * 4;
-        if (bytes > (size_t)max_smem) return fail(h, SOAP_ERR_INVALID_ARG, "this basis does not fit the shared memory of the device");
-        h->P_deriv = P; h->smem_deriv = bytes;
-    }
+        bytes = (size_t)make_layout(h->S, h->n_max, h->l_max, P, true, h->weight.fn != 0).total * 4 + extra;
+        P_out = P; bytes_out = bytes;
+        return bytes <= (size_t)max_smem;
+    };
+    if (!plan_chunk(0, h->P_deriv, h->smem_deriv)) return fail(h, SOAP_ERR_INVALID_ARG, "this basis does not fit the shared memory of the device");
     CU(center_set_smem(kCenterDeriv, h->l_max, h->n_max, (int)h->smem_deriv));
     CU(center_set_smem(kCenterCoeff, h->l_max, h->n_max, (int)h->smem_deriv));
     CU(center_set_smem(kCenterInner, h->l_max, h->n_max, (int)h->smem_deriv));
+    // the kernel of the outer average keeps, per warp, a copy of a neighbouring centre's coefficients behind the usual
+    // layout; a basis too large for that takes the general path (per-pair rows in a workspace)
+    const int LMP = ((h->l_max + 1) * (h->l_max + 1)) | 1;
+    h->outer_fast = plan_chunk((size_t)kWarps * h->S * h->n_max * LMP * 4, h->P_outer, h->smem_outer);
+    if (h->outer_fast) CU(center_set_smem(kCenterOuter, h->l_max, h->n_max, (int)h->smem_outer));
     return SOAP_OK;
 }
 
@@ -449,7 +456,7 @@ void fill_center_params(soap_t* h, CenterParams& cp, const float* pos, const int
     cp.feat_pack = h->d_feat; cp.nch_magic = (unsigned)((1ull << 32) / (unsigned)(h->n_max * (h->l_max + 1))) + 1u; cp.inv_h = h->basis.inv_h; cp.n_intervals = h->basis.n_intervals;
     cp.S = h->S; cp.n_max = h->n_max; cp.l_max = h->l_max; cp.F = (int)h->F;
     cp.P = h->P_deriv;
-    cp.crossover = h->crossover; cp.emit_coeff = 0; cp.c_bar = nullptr; cp.inner_rows = 0; cp.own_scale = 1.f;
+    cp.crossover = h->crossover; cp.emit_coeff = 0; cp.c_bar = nullptr; cp.inner_rows = 0; cp.own_scale = 1.f; cp.c_all = nullptr;
     cp.pair_w = h->weight.fn ? h->d_pair_w : nullptr; cp.w0 = (float)h->w0;
     cp.compact = 0; cp.Fc = (int)h->Fc_pitch; cp.out_center = nullptr;
     cp.out_desc = nullptr; cp.out_jac = nullptr; cp.row_atom = nullptr;
@@ -1000,6 +1007,32 @@ int soap_derivatives_average(soap_t* h, int mode, const float* d_positions, cons
         cp.inner_rows = 1;
         cp.own_scale = (float)(1.0 / (double)n_centers);
         CU(center_launch(kCenterInner, h->l_max, h->n_max, cp, (unsigned)n_centers, h->smem_deriv, st));
+        if (h->profiling) CU(cudaEventRecord(h->ev[2], st));
+        return SOAP_OK;
+    }
+    if (mode == SOAP_AVERAGE_OUTER && !d_centers && n_centers == n_atoms && h->outer_fast) {
+        // Outer average with every atom a centre: atom a gathers its own row and the rows that the centres it sees
+        // hold for it (they need those centres' coefficients, written first by the descriptor kernel): one row per
+        // atom, no per-pair rows, no workspace for them.
+        const int F = (int)h->F, W = h->S * h->n_max * (h->l_max + 1) * (h->l_max + 1);
+        const size_t o_coeff = 0, o_rows = align256((size_t)n_centers * W * 4),
+                     o_partial = o_rows + align256((size_t)n_centers * F * 4), total = o_partial + align256((size_t)kMeanMaxChunks * F * 8);
+        if ((rc = ensure_work(h, total))) return rc;
+        char* w = (char*)h->d_work;
+        CenterParams cp;
+        fill_center_params(h, cp, d_positions, d_centers, n_centers, g, false);
+        cp.out_desc = (float*)(w + o_coeff);
+        cp.emit_coeff = 1;
+        if ((rc = launch_desc(h, cp, n_centers, st))) return rc;
+        fill_center_params(h, cp, d_positions, d_centers, n_centers, g, true);
+        cp.row_capacity = INT64_MAX;
+        cp.c_all = (const float*)(w + o_coeff);
+        cp.out_desc = (float*)(w + o_rows);
+        cp.out_jac = d_out_jac;
+        cp.own_scale = (float)(1.0 / (double)n_centers);
+        cp.P = h->P_outer;
+        CU(center_launch(kCenterOuter, h->l_max, h->n_max, cp, (unsigned)n_centers, h->smem_outer, st));
+        if ((rc = column_mean(h, (const float*)(w + o_rows), n_centers, F, (double*)(w + o_partial), d_out_desc, st))) return rc;
         if (h->profiling) CU(cudaEventRecord(h->ev[2], st));
         return SOAP_OK;
     }

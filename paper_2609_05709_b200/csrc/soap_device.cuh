@@ -84,6 +84,10 @@ struct CenterParams {
     // contraction of cbar with sum_i grad_a c(i) (pass 1 collects that sum) to out_jac[a], and no per-pair rows
     int inner_rows;
     float own_scale;
+    // outer average over ALL atoms as centres: coefficients of every centre, [C][S n_max (l_max+1)^2] (index
+    // (mu n_max + n) (l_max+1)^2 + l^2 + l + m, on-site terms included); the kernel of atom a adds to its own row
+    // the rows that the centres it sees hold for it, all times own_scale, in out_jac[a]
+    const float* c_all;
     // species-compact Jacobian rows: a neighbour's row holds only the blocks that involve its species (pitch Fc, a
     // multiple of 8 floats); the centre's own full row goes to out_center [C,3,F]
     int compact, Fc;

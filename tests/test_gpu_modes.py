@@ -106,11 +106,18 @@ def test_coefficient_mode_centre_subset_into_poisoned_buffers(pkg):
 
 
 @pytest.mark.parametrize("mode", ["inner", "outer"])
-@pytest.mark.parametrize("case", ["water", "periodic_poly", "subset"])
+@pytest.mark.parametrize("case", ["water", "periodic_poly", "subset", "wide_rows", "large_basis"])
 def test_averaged_modes(pkg, mode, case):
     centers = None
     if case == "water":
         s, args = water_cluster(12, 4), ([1, 8], 5.0, 6, 4, 0.5, GTO)
+    elif case == "wide_rows":
+        # more features that involve one species than a thread of the outer-average kernel keeps in registers;
+        # a 4 A cell with r_cut 4 A: every atom also sees images of itself
+        s, args = small_periodic_cell(2), ([1, 6, 7, 8], 4.0, 8, 4, 0.5, POLYNOMIAL, (True, True, True))
+    elif case == "large_basis":
+        # the coefficients of a centre are too many for the shared memory of the outer-average kernel: general path
+        s, args = water_cluster(4, 6), ([1, 8, 9], 4.5, 12, 12, 0.5, GTO)
     elif case == "periodic_poly":
         s, args = small_periodic_cell(5, (True, False, True)), ([1, 6, 7, 8], 4.5, 3, 3, 0.5, POLYNOMIAL, (True, False, True))
     else:
