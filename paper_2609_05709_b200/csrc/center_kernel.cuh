@@ -693,7 +693,7 @@ center_kernel(const CenterParams p) {
                         float* o = out + lo + j;
 #pragma unroll
                         for (int n1 = 0; n1 < NMAX_BOUND; ++n1) {
-                            if (n1 >= NMAX) break;
+                            if (n1 >= NMAX || n1 * L1 > min(j0 + 31, NCH - 1)) break;           // no lane of this round has n2 >= n1
                             const int rel = (n1 * NMAX - n1 * (n1 - 1) / 2) * L1 - n1 * L1;     // row start minus n1 L1
                             if (n1 <= n2) {
                                 const float2 gi = wG[n1 * L1 + l];
@@ -896,12 +896,59 @@ center_kernel(const CenterParams p) {
         }
     };
 
+    const int PW = P / kWarps;             // pairs a warp stages for itself (the staging area holds P)
     for (int g0 = 0; g0 < k_pairs; g0 += kGeoPairs) {
         const int gc = min(kGeoPairs, k_pairs - g0);
         __syncthreads();
         if (g0 > 0 || k_pairs > kGeoPairs) special = stage_geometry(g0, gc);     // otherwise still valid from pass 1
-        // chunks of equal size, a multiple of the warp count: a short last chunk would leave most warps idle
-        // (68 pairs in chunks of 32 are 32 + 32 + 4; in three chunks of 24 every warp has three pairs or two)
+        // (measured on the 1000-molecule cluster: 1 to 4 % faster from n_max = 8 on up to l_max = 8; with fewer
+        // channels than lanes, or more columns m than the eight lanes of a pair, the staging by the whole CTA wins)
+        constexpr bool kPrivate = NMAX_T >= 8 && L <= 8;
+        if (kPrivate && !special && PW >= 1) {
+            // Every pair has a row of its own: the warps work without one another.  Warp w takes the pairs w, w + 8,
+            // ... of the batch, PW at a time: it stages their radial factors (lanes on channels) and harmonics (eight
+            // lanes per pair, on the columns m of the recursion) in its own part of the staging area, then writes
+            // their rows.  No CTA barrier until the next batch of geometry.
+            const int slot0 = wid * PW;
+            for (int gw = wid; gw < gc; gw += PW * kWarps) {
+                const int nb = min(PW, (gc - gw + kWarps - 1) / kWarps);
+                __syncwarp();
+                for (int pr = 0; pr < nb; ++pr) {
+                    const int g = gw + pr * kWarps;
+                    const int4 gi = geo_i[g];
+                    const float t = __int_as_float(gi.y);
+                    const float rinv_h = (float)p.inv_h / geo_d[g].w;
+                    float2* mG = sG2 + (slot0 + pr) * NCH;
+                    if (o_pw) {
+                        const float2 w = geo_w[g];
+                        for (int ch = lane; ch < NCH; ch += 32) {
+                            float v, dv;
+                            radial_lookup(p.table, gi.x, NCH, ch, t, v, dv);
+                            mG[ch] = make_float2(v * w.x, fmaf(dv * rinv_h, w.x, v * w.y));
+                        }
+                    } else {
+                        for (int ch = lane; ch < NCH; ch += 32) {
+                            float v, dv;
+                            radial_lookup(p.table, gi.x, NCH, ch, t, v, dv);
+                            mG[ch] = make_float2(v, dv * rinv_h);
+                        }
+                    }
+                }
+                {
+                    const int pr = lane >> 3;
+                    if (pr < nb) {
+                        const float4 d = geo_d[gw + pr * kWarps];
+                        for (int m = lane & 7; m <= L; m += 8)
+                            harmonics_column(L, m, d.x, d.y, d.z, d.w * d.w, sSD4 + (slot0 + pr) * LMP);
+                    }
+                }
+                __syncwarp();
+                for (int pr = 0; pr < nb; ++pr) do_pair(gw + pr * kWarps, slot0 + pr);
+            }
+            continue;
+        }
+        // Images of one atom share a row (or the staging area holds fewer pairs than there are warps): staged by the
+        // whole CTA in chunks of equal size, a multiple of the warp count.
         const int n_chunks = (gc + P - 1) / P;
         const int PB = min(P, (((gc + n_chunks - 1) / n_chunks) + kWarps - 1) & ~(kWarps - 1));
         for (int q0 = 0; q0 < gc; q0 += PB) {
@@ -909,10 +956,9 @@ center_kernel(const CenterParams p) {
             stage_chunk(q0, pc);
             __syncthreads();
             if (!special) {
-                // every pair has a row of its own: deal them out round-robin
                 for (int pr = wid; pr < pc; pr += kWarps) do_pair(q0 + pr, pr);
             } else {
-                // images of one atom share a row and must stay with one warp, in order;
+                // images of one atom must stay with one warp, in order;
                 // images of the centre itself do not move relative to it and are skipped
                 for (int pr = 0; pr < pc; ++pr) {
                     const int rw = geo_i[q0 + pr].w;
