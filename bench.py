@@ -136,13 +136,14 @@ def _oracle_setup(name):
 
 def _oracle_worker(job):
     """One process of the all-cores baseline: the oracle, NumPy held to one thread, on its share of the centres."""
-    name, centers = job
+    name, centers, mode = job
     from threadpoolctl import threadpool_limits
     oracle, s = _oracle_setup(name)
+    call = oracle.derivatives if mode == "derivatives" else oracle.descriptor
     with threadpool_limits(limits=1):
-        oracle.derivatives(s.positions, s.numbers, s.cell, [0])        # builds the basis caches (not timed)
+        call(s.positions, s.numbers, s.cell, [0])                      # builds the basis caches (not timed)
         t0 = time.perf_counter()
-        oracle.derivatives(s.positions, s.numbers, s.cell, centers)
+        call(s.positions, s.numbers, s.cell, centers)
         return time.perf_counter() - t0
 
 
@@ -159,7 +160,7 @@ def oracle_rate(name, n_centers):
     return n_centers / seconds, seconds
 
 
-def oracle_rate_all_cores(name, per_core):
+def oracle_rate_all_cores(name, per_core, mode="derivatives"):
     """The same oracle in one process per host core (each on `per_core` centres of its own); the rate is all
     centres over the busy time of the slowest process."""
     import multiprocessing as mp
@@ -168,7 +169,7 @@ def oracle_rate_all_cores(name, per_core):
     cores = min(cores, 64)                     # one process each; more than this only adds start-up time
     n_atoms = make_structure(name).n_atoms
     allc = [int(c) for c in np.linspace(0, n_atoms - 1, cores * per_core)]
-    jobs = [(name, allc[k::cores]) for k in range(cores)]
+    jobs = [(name, allc[k::cores], mode) for k in range(cores)]
     with ProcessPoolExecutor(max_workers=cores, mp_context=mp.get_context("spawn")) as pool:
         busy = list(pool.map(_oracle_worker, jobs))
     return len(allc) / max(busy), cores, max(busy), len(allc)
@@ -509,7 +510,8 @@ def time_case(struct, species, r_cut, n_max, l_max, sigma, rbf, mode, steps, war
 def run_suite(args):
     import torch
     from soap_inputs import multispecies_box, water_cluster
-    torch.cuda.set_device(0)
+    if args.suite != "cpu":
+        torch.cuda.set_device(0)
     steps = args.steps
     if args.suite == "map":
         s = water_cluster(1000, 0)
@@ -652,6 +654,16 @@ def run_suite(args):
                               "us_per_structure": 1e6 * best / nst, "rows": nrows.value,
                               "jacobian_GBps": nrows.value * 3 * F * 4 / best / 1e9}), flush=True)
             del soap, desc, jac
+    elif args.suite == "cpu":
+        # the fp64 oracle as it stands on all host cores, per configuration (a reported baseline: it runs no GPU code)
+        cores = min(len(os.sched_getaffinity(0)) if hasattr(os, "sched_getaffinity") else (os.cpu_count() or 1), 64)
+        for name, per_core in (("water8_gto_n4_l3_rc5", (3, 3)), ("water1000_gto_n8_l6_rc6", (100, 300)),
+                               ("chno2000_poly_n8_l8_rc5", (24, 96)), ("water1000_gto_n7_l3_rc10", (40, 300))):
+            for mode, pc in zip(("derivatives", "descriptor"), per_core):
+                n_atoms = make_structure(name).n_atoms
+                rate, used, busy, n = oracle_rate_all_cores(name, max(1, min(pc, n_atoms // cores)), mode)
+                print(json.dumps({"case": name, "mode": mode, "atoms": n_atoms, "oracle_atoms_per_s": rate, "cores": used,
+                                  "centres_timed": n, "slowest_process_s": busy}), flush=True)
     elif args.suite == "compact":
         for name in ("water1000_gto_n8_l6_rc6", "chno2000_poly_n8_l8_rc5"):
             kind, n, species, r_cut, n_max, l_max, sigma, rbf = WORKLOADS[name]
@@ -693,7 +705,7 @@ def main():
                          "instead of running N independent replicas")
     ap.add_argument("--kernel-only", action="store_true",
                     help="skip the end-to-end and CPU-baseline legs (for profiler captures)")
-    ap.add_argument("--suite", choices=["map", "scaling", "configs", "desc30k", "modes", "driver", "compact", "graph", "small"],
+    ap.add_argument("--suite", choices=["map", "scaling", "configs", "desc30k", "modes", "driver", "compact", "graph", "small", "cpu"],
                     help="extra measurements beside the headline line: 'map' = descriptor+Jacobian over "
                          "n_max x l_max on the 1000-molecule cluster, 'scaling' = descriptor-only on "
                          "3k..1M atoms, 'configs' = the periodic multi-species box and the tiny cluster, "
