@@ -37,6 +37,20 @@
  *    set, the outputs of that call are unspecified.
  *  - The library has no CPU fallback: without a CUDA device the compute
  *    calls return SOAP_ERR_CUDA.
+ *  - Arithmetic is fp32 (distances and table offsets fp64, tables built in
+ *    quad precision).  Accuracy against an fp64 evaluation of the same
+ *    equations, per feature column over the centres of a call: descriptor
+ *    within 1e-5 and Jacobian within 1e-4 of the column's largest magnitude,
+ *    for every column whose largest magnitude is at least 1e-3 of the largest
+ *    entry of the whole output.  A column that is smaller than that for every
+ *    centre at once (a few-atom structure whose neighbours all sit near a node
+ *    of one radial function, or whose terms cancel) carries the rounding of
+ *    the larger quantities it is computed from: its error is bounded relative
+ *    to 1e-3 of the output's largest entry, not to its own maximum (in a
+ *    500-draw random sweep over structures of 2 to 19 atoms, 489 draws were
+ *    within 1e-5 / 1e-4 of that scale and the worst of the others reached
+ *    3e-5 / 2e-4; structures of the benchmark sizes meet the column bound
+ *    with a margin of 4 to 10).
  */
 #ifndef SOAP_B200_H
 #define SOAP_B200_H
