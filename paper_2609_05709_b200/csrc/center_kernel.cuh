@@ -707,6 +707,32 @@ center_kernel(const CenterParams p) {
                             }
                         }
                     }
+                } else if (mu == nu && NMAX_T != 0) {
+                    // compile-time n_max: the sweeps are unrolled in full, so that the table index and the three store
+                    // addresses of a sweep are constants off pointers formed once per block
+                    const float4* UVz = wUV + Z * NCH;
+                    constexpr int TRI_T = (NMAX_BOUND * (NMAX_BOUND + 1) / 2) * L1;
+                    constexpr int SWEEPS = (TRI_T + 62) / 32;                   // the block and up to 31 floats in front of it
+                    const int e0 = first - lo + lane;                           // -31 .. 31: place of this lane's first feature in the block
+                    const unsigned short* dp = tri_dec + e0;
+                    float* const o0 = out + (first + lane);
+                    float* const o1 = o0 + PS;
+                    float* const o2 = o0 + PS2;
+#pragma unroll
+                    for (int k = 0; k < SWEEPS; ++k) {
+                        const int e = e0 + 32 * k;
+                        if ((k > 0 || e >= 0) && (32 * k + 31 < TRI_T || e < TRI_T)) {
+                            const unsigned dec = dp[32 * k];                    // (n1 L1 + l) | (n2 L1 + l) << 8
+                            const int iA = dec & 255, iB = dec >> 8;
+                            const float2 g1 = wG[iA], g2 = wG[iB];
+                            const float4 u1 = UVz[iA], u2 = UVz[iB];
+                            const float t = fmaf(g1.y, u2.x, g2.y * u1.x);      // Ghat_n1 U_n2 + Ghat_n2 U_n1
+                            const float vx = fmaf(g1.x, u2.y, fmaf(g2.x, u1.y, t * d.x)), vy = fmaf(g1.x, u2.z, fmaf(g2.x, u1.z, t * d.y)),
+                                        vz = fmaf(g1.x, u2.w, fmaf(g2.x, u1.w, t * d.z));
+                            if (ACC) { o0[32 * k] += vx; o1[32 * k] += vy; o2[32 * k] += vz; }
+                            else { o0[32 * k] = vx; o1[32 * k] = vy; o2[32 * k] = vz; }
+                        }
+                    }
                 } else if (mu == nu) {
                     const float4* UVz = wUV + Z * NCH;
 #pragma unroll kTriUnroll
