@@ -266,10 +266,21 @@ center_kernel(const CenterParams p) {
                 sG2[pr * NCH + ch] = make_float2(v, dv * rinv_h);
             }
         }
-        if (lane < pc) {
-            const float4 d = geo_d[g + lane];
-            for (int m = wid; m <= L; m += kWarps)
-                harmonics_column(L, m, d.x, d.y, d.z, d.w * d.w, sSD4 + lane * LMP);
+        if (P >= 32) {
+            // a warp per column: m is the same for all its lanes, so the recursion's coefficients are uniform reads
+            if (lane < pc) {
+                const float4 d = geo_d[g + lane];
+                for (int m = wid; m <= L; m += kWarps)
+                    harmonics_column(L, m, d.x, d.y, d.z, d.w * d.w, sSD4 + lane * LMP);
+            }
+        } else {
+            // a chunk holds at most P pairs (a power of two): the lanes of a warp take 32 / P columns side by side
+            const int cols = 32 / P, pr = lane & (P - 1), cg = lane / P;
+            if (pr < pc) {
+                const float4 d = geo_d[g + pr];
+                for (int m = wid * cols + cg; m <= L; m += kWarps * cols)
+                    harmonics_column(L, m, d.x, d.y, d.z, d.w * d.w, sSD4 + pr * LMP);
+            }
         }
     };
 
