@@ -224,8 +224,13 @@ __global__ void __launch_bounds__(kDescMaxWarps * 32, 1) desc_kernel(const Cente
             }
         }
     };
-    const long long w_stride = (long long)gridDim.x * warps;
-    for (long long c_idx = (long long)blockIdx.x * warps + wid; c_idx < n_work; c_idx += w_stride) {
+    // Full rounds give every warp of the grid one centre, CTA by CTA; the centres of the last, partial round are
+    // dealt out across the CTAs first, so that every SM gets its share of them instead of a few SMs a full round
+    const long long w_stride = (long long)gridDim.x * warps, full_rounds = n_work / w_stride;
+    for (long long round = 0; round <= full_rounds; ++round) {
+        const long long c_idx = round * w_stride + (round < full_rounds ? (long long)blockIdx.x * warps + wid
+                                                                         : (long long)wid * gridDim.x + blockIdx.x);
+        if (c_idx >= n_work) break;
         const Head hd = load_head(c_idx);
         Raw raw;
         const float xi = hd.xi, yi = hd.yi, zi = hd.zi;
