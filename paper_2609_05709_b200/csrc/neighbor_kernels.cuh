@@ -285,13 +285,18 @@ small_prep_kernel(const float* __restrict__ pos, const int* __restrict__ numbers
         if (lane == 0) { red[a][wid] = hi[a]; red[3 + a][wid] = lo[a]; }
     }
     __syncthreads();
+    if (wid == 0) {
+        // the 32 warps' maxima, one per lane
+        for (int a = 0; a < 6; ++a) {
+            double v = red[a][lane];
+            for (int o = 16; o > 0; o >>= 1) v = fmax(v, __shfl_xor_sync(0xffffffffu, v, o));
+            if (lane == 0) red[a][0] = v;
+        }
+    }
+    __syncthreads();
     if (tid == 0) {
         double h3[3], l3[3];
-        for (int a = 0; a < 3; ++a) {
-            double h = -1e300, l = -1e300;
-            for (int w = 0; w < kPrepThreads / 32; ++w) { h = fmax(h, red[a][w]); l = fmax(l, red[3 + a][w]); }
-            h3[a] = h; l3[a] = -l;
-        }
+        for (int a = 0; a < 3; ++a) { h3[a] = red[a][0]; l3[a] = -red[3 + a][0]; }
         sg = choose_grid(h3, l3, geom, N, cell_cap);
         *grid_out = sg;
         carry_s = 0;
@@ -763,8 +768,21 @@ rows_order_kernel(const int* __restrict__ row_count, const int* __restrict__ pai
     if (tid == 0) {
         row_ptr[C] = carry_s;
         counters->n_rows = carry_s;
-        int run = 0;
-        for (int b = kSizeBins - 1; b >= 0; --b) { first_slot[b] = run; run += hist[b]; }
+    }
+    if (wid == 0) {
+        // first slot of every size bin, largest bin first: lane k scans the bins 255 - 8k down to 248 - 8k, a warp
+        // scan adds what the lanes before it hold
+        constexpr int per_lane = kSizeBins / 32;
+        const int top = kSizeBins - 1 - lane * per_lane;
+        int mine = 0;
+        for (int k = 0; k < per_lane; ++k) mine += hist[top - k];
+        int incl = mine;
+        for (int o = 1; o < 32; o <<= 1) {
+            const int y = __shfl_up_sync(0xffffffffu, incl, o);
+            if (lane >= o) incl += y;
+        }
+        int run = incl - mine;
+        for (int k = 0; k < per_lane; ++k) { first_slot[top - k] = run; run += hist[top - k]; }
     }
     __syncthreads();
     if (order)
