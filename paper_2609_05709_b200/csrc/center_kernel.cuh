@@ -129,13 +129,6 @@ center_kernel(const CenterParams p) {
     constexpr int NPT = NPT_RAW < 8 ? NPT_RAW : 8;                // ... at most 8 at a time (register budget)
     extern __shared__ __align__(16) float smem[];
     const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
-    const long long c_idx = p.order ? p.order[blockIdx.x] : blockIdx.x;
-    // a failed neighbour build or an undersized output: write nothing
-    if (p.counters->n_pairs > p.pair_capacity) return;
-    if (p.row_ptr[p.n_centers] > p.row_capacity) {
-        if (c_idx == 0 && tid == 0) atomicOr(&p.counters->status, kStatusRowCapacity);
-        return;
-    }
     const int S = p.S, NMAX = NMAX_T ? NMAX_T : p.n_max, NCH = NMAX * L1, NE = NMAX * LM;
     const int CT = S * NMAX * LMP, P = p.P, F = p.F;
     const SmemLayout lay = make_layout(S, NMAX, L, P, true, o_pw != nullptr);
@@ -148,14 +141,7 @@ center_kernel(const CenterParams p) {
     float4* sSD4 = reinterpret_cast<float4*>(smem + lay.sSD);              // [P][LMP]   (S, dSx, dSy, dSz)
     float2* sG2 = reinterpret_cast<float2*>(smem + lay.sG);                // [P][NCH]   (G, Ghat)
 
-    const int ci = o_sites ? -1 : (p.centers ? p.centers[c_idx] : (int)c_idx);
-    const float* pc = o_sites ? o_sites + 3 * c_idx : p.pos + 3 * (long long)ci;
-    const float xi = pc[0], yi = pc[1], zi = pc[2];
-    const int zi_species = o_sites ? 0 : p.species_idx[ci];
-    const long long pair_base = p.pair_start[c_idx];
-    const int k_pairs = p.pair_count[c_idx];
-    const bool periodic = p.geom.pbc[0] | p.geom.pbc[1] | p.geom.pbc[2];
-
+    // ---- set-up that needs nothing from the kernels before this one (it may run while they finish) ----
     for (int e = tid; e < CT * 4; e += kThreads) {
         if (e < CT) c_t[e] = 0.f; else D_t[e - CT] = 0.f;
     }
@@ -173,6 +159,23 @@ center_kernel(const CenterParams p) {
             const int n2 = n1 + r / L1, l = r % L1;
             tri_dec[e] = (unsigned short)((n1 * L1 + l) | ((n2 * L1 + l) << 8));
         }
+
+    // ---- from here on the neighbour data of this call is read ----
+    grid_dependency_wait();
+    const long long c_idx = p.order ? p.order[blockIdx.x] : blockIdx.x;
+    // a failed neighbour build or an undersized output: write nothing
+    if (p.counters->n_pairs > p.pair_capacity) return;
+    if (p.row_ptr[p.n_centers] > p.row_capacity) {
+        if (c_idx == 0 && tid == 0) atomicOr(&p.counters->status, kStatusRowCapacity);
+        return;
+    }
+    const int ci = o_sites ? -1 : (p.centers ? p.centers[c_idx] : (int)c_idx);
+    const float* pc = o_sites ? o_sites + 3 * c_idx : p.pos + 3 * (long long)ci;
+    const float xi = pc[0], yi = pc[1], zi = pc[2];
+    const int zi_species = o_sites ? 0 : p.species_idx[ci];
+    const long long pair_base = p.pair_start[c_idx];
+    const int k_pairs = p.pair_count[c_idx];
+    const bool periodic = p.geom.pbc[0] | p.geom.pbc[1] | p.geom.pbc[2];
 
     // pass-1 ownership of this thread: one lm, and the radial functions slot, slot + SLOTS, ...
     const int own_slot = wid / W_LM, own_lm = (wid - own_slot * W_LM) * 32 + lane;

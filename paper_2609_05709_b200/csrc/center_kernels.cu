@@ -17,8 +17,9 @@ static cudaError_t set_one(int bytes) {
 }
 template <int KIND, int NM, bool PLAIN>
 static cudaError_t launch_one(const CenterParams& p, unsigned grid, size_t smem, cudaStream_t st) {
-    center_kernel<KIND, SOAP_L, NM, PLAIN><<<grid, kThreads, smem, st>>>(p);
-    return cudaGetLastError();
+    // the kernel waits on the device for the kernel before it (the row scan, as a rule): its launch and its
+    // set-up overlap that kernel's tail
+    return launch_dependent(center_kernel<KIND, SOAP_L, NM, PLAIN>, grid, kThreads, smem, st, p);
 }
 
 // Fills this translation unit's constant tables (once per process and device is enough;

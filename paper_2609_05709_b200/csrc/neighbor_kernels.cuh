@@ -263,6 +263,7 @@ small_prep_kernel(const float* __restrict__ pos, const int* __restrict__ numbers
     __shared__ long long warp_sums[32];
     __shared__ long long carry_s;
     __shared__ int s_cnt[kPrepSmemCells + 1], s_start[kPrepSmemCells + 1];   // bin counters on chip when they fit
+    grid_dependency_launch();                                                // the pair kernel may move in and wait
     const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
     // ---- species and bounding box of the fractional coordinates ----
     double hi[3] = {-1e300, -1e300, -1e300}, lo[3] = {-1e300, -1e300, -1e300};
@@ -550,6 +551,8 @@ pairs_kernel(const float* __restrict__ pos, const int* __restrict__ centers, con
              int* __restrict__ self_row, Counters* counters) {
     __shared__ unsigned long long s_raw[kFillWarps][KEYS];
     __shared__ unsigned long long s_sorted[kFillWarps][KEYS];
+    grid_dependency_launch();
+    grid_dependency_wait();                                                  // the cell list of the kernel before
     const GridParams g = *gp;
     const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
     const long long c = blockIdx.x * (long long)kFillWarps + wid;
@@ -665,6 +668,7 @@ batch_pairs_kernel(const float* __restrict__ pos, const int* __restrict__ number
                    long long N, double rc2, long long pair_capacity, unsigned long long* pair_key,
                    int* __restrict__ pair_row, long long* __restrict__ pair_start, int* __restrict__ pair_count,
                    int* __restrict__ row_count, int* __restrict__ self_row, Counters* counters) {
+    grid_dependency_launch();
     const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
     const long long i = blockIdx.x * (long long)kFillWarps + wid;
     if (i >= N) return;
@@ -736,14 +740,24 @@ rows_order_kernel(const int* __restrict__ row_count, const int* __restrict__ pai
     __shared__ long long carry_s;
     __shared__ int hist[kSizeBins], first_slot[kSizeBins];
     const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
+    grid_dependency_launch();
     if (tid == 0) carry_s = 0;
     if (tid < kSizeBins) hist[tid] = 0;
+    grid_dependency_wait();                                                  // the counts of the pair kernel
     __syncthreads();
-    for (long long base = 0; base < C; base += 1024) {
-        const long long i = base + tid;
-        const long long v = i < C ? (long long)row_count[i] : 0;
-        if (i < C) atomicAdd(&hist[min(pair_count[i] >> kSizeBinShift, kSizeBins - 1)], 1);
-        long long x = v;
+    // four consecutive centres per thread and trip: a few thousand centres are one trip, four barriers
+    constexpr int kPerThread = 4;
+    for (long long base = 0; base < C; base += 1024 * kPerThread) {
+        const long long i0 = base + (long long)tid * kPerThread;
+        long long v[kPerThread], x = 0;
+#pragma unroll
+        for (int k = 0; k < kPerThread; ++k) {
+            const long long i = i0 + k;
+            v[k] = i < C ? (long long)row_count[i] : 0;
+            if (i < C) atomicAdd(&hist[min(pair_count[i] >> kSizeBinShift, kSizeBins - 1)], 1);
+            x += v[k];
+        }
+        const long long mine = x;
         for (int o = 1; o < 32; o <<= 1) {
             const long long y = __shfl_up_sync(0xffffffffu, x, o);
             if (lane >= o) x += y;
@@ -760,7 +774,12 @@ rows_order_kernel(const int* __restrict__ row_count, const int* __restrict__ pai
         }
         __syncthreads();
         const long long carry = carry_s;
-        if (i < C) row_ptr[i] = carry + (wid > 0 ? warp_sums[wid - 1] : 0) + x - v;
+        long long at = carry + (wid > 0 ? warp_sums[wid - 1] : 0) + x - mine;
+#pragma unroll
+        for (int k = 0; k < kPerThread; ++k) {
+            if (i0 + k < C) row_ptr[i0 + k] = at;
+            at += v[k];
+        }
         __syncthreads();
         if (tid == 1023) carry_s = carry + warp_sums[31];
         __syncthreads();

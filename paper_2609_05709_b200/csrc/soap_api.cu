@@ -392,10 +392,11 @@ int launch_neighbors(soap_t* h, const float* pos, const int32_t* num, int64_t N,
         const unsigned grid = (unsigned)((C + kFillWarps - 1) / kFillWarps);
 #define SOAP_PAIRS_ARGS pos, centers, sites, C, g, h->d_grid, h->d_atom_cell, h->d_atom_wrap, h->d_cell_start, h->d_s_pos, h->d_s_wrap, \
         h->cap_pairs, h->d_pair_tmp, h->d_pair_key, h->d_pair_row, h->d_pair_start, h->d_pair_count, h->d_row_count, h->d_self_row, h->d_counters
-        if (small_keys && rows) pairs_kernel<kFillSmemKeysSmall, true><<<grid, kFillWarps * 32, 0, st>>>(SOAP_PAIRS_ARGS);
-        else if (small_keys) pairs_kernel<kFillSmemKeysSmall, false><<<grid, kFillWarps * 32, 0, st>>>(SOAP_PAIRS_ARGS);
-        else if (rows) pairs_kernel<kFillSmemKeys, true><<<grid, kFillWarps * 32, 0, st>>>(SOAP_PAIRS_ARGS);
-        else pairs_kernel<kFillSmemKeys, false><<<grid, kFillWarps * 32, 0, st>>>(SOAP_PAIRS_ARGS);
+        // (these kernels wait for the kernel before them on the device: their launch overlaps its tail)
+        if (small_keys && rows) CU(launch_dependent(pairs_kernel<kFillSmemKeysSmall, true>, grid, kFillWarps * 32, 0, st, SOAP_PAIRS_ARGS));
+        else if (small_keys) CU(launch_dependent(pairs_kernel<kFillSmemKeysSmall, false>, grid, kFillWarps * 32, 0, st, SOAP_PAIRS_ARGS));
+        else if (rows) CU(launch_dependent(pairs_kernel<kFillSmemKeys, true>, grid, kFillWarps * 32, 0, st, SOAP_PAIRS_ARGS));
+        else CU(launch_dependent(pairs_kernel<kFillSmemKeys, false>, grid, kFillWarps * 32, 0, st, SOAP_PAIRS_ARGS));
 #undef SOAP_PAIRS_ARGS
     }
     if (!rows && !batch.struct_ptr && !brute) {
@@ -404,7 +405,7 @@ int launch_neighbors(soap_t* h, const float* pos, const int32_t* num, int64_t N,
         return SOAP_OK;
     }
     if (C <= kOrderMaxCenters) {
-        rows_order_kernel<<<1, 1024, 0, st>>>(h->d_row_count, h->d_pair_count, C, row_ptr_out, h->d_order, h->d_counters);
+        CU(launch_dependent(rows_order_kernel, 1, 1024, 0, st, h->d_row_count, h->d_pair_count, C, row_ptr_out, h->d_order, h->d_counters));
     } else {
         scan_counts(h, h->d_row_count, row_ptr_out, C, &h->d_counters->n_rows, st);
     }

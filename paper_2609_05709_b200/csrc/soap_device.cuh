@@ -101,6 +101,28 @@ struct CenterParams {
     int* row_atom;                // [rows]
 };
 
+// Programmatic dependent launch: a kernel launched with the attribute cudaLaunchAttributeProgrammaticStreamSerialization
+// may start while the kernel before it in the stream still runs; it must call grid_dependency_wait() before it
+// touches anything that kernel (or one before it) wrote - the wait returns once that kernel has finished and its
+// writes are visible (at once when the launch carried no attribute).  grid_dependency_launch() lets the NEXT kernel
+// of the stream start; without it that happens when this kernel's blocks exit.
+#ifdef __CUDACC__
+__device__ __forceinline__ void grid_dependency_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void grid_dependency_launch() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
+// launch of a kernel that begins with grid_dependency_wait(), allowed to overlap the tail of its predecessor
+template <class... KArgs, class... Args>
+inline cudaError_t launch_dependent(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, Args&&... args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid; cfg.blockDim = block; cfg.dynamicSmemBytes = smem; cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr; cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
+#endif
+
 __host__ __device__ inline int key_atom(unsigned long long k) { return (int)(k >> 24); }
 __host__ __device__ inline void key_shift(unsigned long long k, int s[3]) {
     s[0] = (int)((k >> 16) & 255) - 128;
