@@ -153,6 +153,8 @@ __global__ void __launch_bounds__(kDescMaxWarps * 32, 1) desc_kernel(const Cente
         for (int e = threadIdx.x; e < n4; e += blockDim.x) dst[e] = __ldg(src + e);
         __syncthreads();
     }
+    // the table is this handle's own; everything below reads what the kernels before this one wrote
+    grid_dependency_wait();
     // a failed neighbour build: write nothing
     if (p.counters->n_pairs > p.pair_capacity) return;
 

@@ -27,10 +27,10 @@ static cudaError_t set_np(int bytes) {
 
 template <int NP>
 static cudaError_t launch_np(bool plain, bool ts, const CenterParams& p, unsigned grid, unsigned block, size_t smem, cudaStream_t st) {
-    if (plain && ts) desc_kernel<SOAP_L, NP, true, true><<<grid, block, smem, st>>>(p);
-    else if (plain) desc_kernel<SOAP_L, NP, true, false><<<grid, block, smem, st>>>(p);
-    else desc_kernel<SOAP_L, NP, false, false><<<grid, block, smem, st>>>(p);
-    return cudaGetLastError();
+    // (the kernel waits on the device for the kernel before it: launch and table staging overlap that kernel's tail)
+    if (plain && ts) return launch_dependent(desc_kernel<SOAP_L, NP, true, true>, grid, block, smem, st, p);
+    if (plain) return launch_dependent(desc_kernel<SOAP_L, NP, true, false>, grid, block, smem, st, p);
+    return launch_dependent(desc_kernel<SOAP_L, NP, false, false>, grid, block, smem, st, p);
 }
 
 cudaError_t SOAP_CAT(desc_constants_l, SOAP_L)(const float* anorm91) {
