@@ -112,3 +112,53 @@ def test_a_planned_step_can_be_captured_in_a_cuda_graph_and_replayed(pkg):
     ref = soap.derivatives(torch.from_numpy(moved).cuda(), num)
     assert torch.equal(got_ptr, ref.row_ptr) and torch.equal(got_atom, ref.row_atom)
     assert torch.equal(got_desc, ref.descriptor) and torch.equal(got_jac, ref.jacobian)
+
+
+def test_calls_queued_back_to_back_equal_calls_made_alone(pkg):
+    """The kernels of a call wait for one another on the device and start while their predecessor still runs.  Calls
+    of different sizes and kinds queued on one stream without a host wait in between, and on two streams at once
+    with a handle each, must give the bits of the same calls made alone."""
+    structs = [water_cluster(40, 1), water_cluster(6, 2), small_periodic_cell(3)]
+    args = [([1, 8], 5.0, 8, 6, 0.5, GTO), ([1, 8], 4.0, 4, 3, 0.5, GTO), ([1, 6, 7, 8], 4.5, 3, 3, 0.5, POLYNOMIAL, (True, True, True))]
+    soaps = [pkg.Soap(*a) for a in args]
+    dev = [(torch.from_numpy(s.positions).cuda(), torch.from_numpy(s.numbers).cuda(), s.cell) for s in structs]
+    alone = []
+    for soap, (pos, num, cell) in zip(soaps, dev):
+        d = soap.derivatives(pos, num, cell)
+        torch.cuda.synchronize()
+        p = soap.descriptor(pos, num, cell).clone()
+        torch.cuda.synchronize()
+        alone.append((d.descriptor.clone(), d.jacobian.clone(), d.row_ptr.clone(), d.row_atom.clone(), p))
+    def buffers(k):
+        ref = alone[k]
+        return [torch.empty_like(ref[0]), torch.empty_like(ref[1]), torch.empty_like(ref[2]), torch.empty_like(ref[3]), torch.empty_like(ref[4])]
+
+    for trial in range(5):
+        queued = []
+        for k in (0, 1, 2, 1, 0):
+            pos, num, cell = dev[k]
+            b = buffers(k)
+            soaps[k].derivatives_into(pos, num, cell, None, b[0], b[1], b[2], b[3])      # enqueues only: no host wait
+            soaps[k].descriptor(pos, num, cell, None, out=b[4])
+            queued.append((k, b))
+        torch.cuda.synchronize()
+        for k, b in queued:
+            soaps[k].status()
+            for got, ref in zip(b, alone[k]):
+                assert torch.equal(got, ref)
+    # two streams, a handle each, at the same time
+    other = pkg.Soap(*args[0])
+    streams = [torch.cuda.Stream(), torch.cuda.Stream()]
+    pos, num, cell = dev[0]
+    other.neighbors(pos, num, cell)                                # plans the second handle's scratch
+    torch.cuda.synchronize()
+    outs = []
+    for _ in range(4):
+        for soap, st in zip((soaps[0], other), streams):
+            with torch.cuda.stream(st):
+                b = buffers(0)
+                soap.derivatives_into(pos, num, cell, None, b[0], b[1], b[2], b[3])
+                outs.append(b)
+    torch.cuda.synchronize()
+    for b in outs:
+        assert torch.equal(b[0], alone[0][0]) and torch.equal(b[1], alone[0][1])
