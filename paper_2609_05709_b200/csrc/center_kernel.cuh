@@ -159,6 +159,16 @@ center_kernel(const CenterParams p) {
             const int n2 = n1 + r / L1, l = r % L1;
             tri_dec[e] = (unsigned short)((n1 * L1 + l) | ((n2 * L1 + l) << 8));
         }
+    // cross-species blocks (rows n1 of n_ch entries): feature index -> (n1 L1 + l) | (n2 L1 + l) << 8
+    // (measured on the 1000-molecule cluster: 3 to 7 % faster than decoding every feature by arithmetic at n_max = 10;
+    // up to n_max = 8 the lanes-on-columns path further down stays 1 to 6 % ahead)
+    constexpr bool kCrossTable = KIND != 2 && NMAX_T > 8 && NMAX_T <= 12 && ((NMAX_BOUND * L1) & 3) != 0;
+    unsigned short* x_dec = reinterpret_cast<unsigned short*>(smem + lay.xdec);
+    if (kCrossTable && S > 1)
+        for (int e = tid; e < NMAX * NCH; e += kThreads) {
+            const int n1 = e / NCH, j = e - n1 * NCH;
+            x_dec[e] = (unsigned short)((n1 * L1 + j % L1) | (j << 8));
+        }
 
     // ---- from here on the neighbour data of this call is read ----
     grid_dependency_wait();
@@ -759,6 +769,33 @@ center_kernel(const CenterParams p) {
                         const float t = fmaf(g1.y, u2.x, g2.y * u1.x);      // Ghat_n1 U_n2 + Ghat_n2 U_n1
                         put(f, fmaf(g1.x, u2.y, fmaf(g2.x, u1.y, t * d.x)), fmaf(g1.x, u2.z, fmaf(g2.x, u1.z, t * d.y)),
                             fmaf(g1.x, u2.w, fmaf(g2.x, u1.w, t * d.z)));
+                    }
+                } else if (kCrossTable) {
+                    // rows that do not all start on a sector boundary: sweeps aligned to the row start of the Jacobian
+                    // row, as in the same-species block, with the two operand indices of a feature from a table
+                    const bool first_term = (mu == Z);                        // which factor belongs to the moved atom
+                    const float4* UVo = wUV + (first_term ? nu : mu) * NCH;
+                    constexpr int SQ_T = NMAX_BOUND * NMAX_BOUND * L1, SWEEPS = (SQ_T + 62) / 32, kUnroll = 8;
+                    const int e0 = first - lo + lane;                           // -31 .. 31
+                    for (int k0 = 0; k0 < SWEEPS; k0 += kUnroll) {
+                        const unsigned short* dp = x_dec + e0 + 32 * k0;
+                        float* const o0 = out + (first + lane + 32 * k0);
+                        float* const o1 = o0 + PS;
+                        float* const o2 = o0 + PS2;
+#pragma unroll
+                        for (int kk = 0; kk < kUnroll; ++kk) {
+                            const int e = e0 + 32 * (k0 + kk);
+                            if (k0 + kk < SWEEPS && e >= 0 && e < SQ_T) {
+                                const unsigned dec = dp[32 * kk];
+                                const int i1 = dec & 255, j = dec >> 8;
+                                const float2 g = wG[first_term ? i1 : j];
+                                const float4 u = UVo[first_term ? j : i1];
+                                const float t = g.y * u.x;
+                                const float vx = fmaf(g.x, u.y, t * d.x), vy = fmaf(g.x, u.z, t * d.y), vz = fmaf(g.x, u.w, t * d.z);
+                                if (ACC) { o0[32 * kk] += vx; o1[32 * kk] += vy; o2[32 * kk] += vz; }
+                                else { o0[32 * kk] = vx; o1[32 * kk] = vy; o2[32 * kk] = vz; }
+                            }
+                        }
                     }
                 } else if ((NCH & 7) == 0 || (NMAX_T > 8 && (NCH & 3) == 0) || (NMAX_T != 0 && NMAX_T <= 8)) {
                     // Cross-species block: rows n1 of n_ch floats follow each other.  A lane keeps one position i of

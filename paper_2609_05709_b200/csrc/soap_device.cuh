@@ -139,8 +139,14 @@ constexpr int kGeoPairs = 128;           // pairs whose geometry is staged at on
 constexpr int kZeroWords = 1024;         // a block of zeros that bulk copies write into the structural-zero blocks of the rows
 
 struct SmemLayout {
-    int c, geo, tri, zero, D, wUV, sSD, sG, total;
+    int c, geo, tri, xdec, zero, D, wUV, sSD, sG, total;
 };
+// whether the cross-species blocks of the rows are written in table-driven sweeps (a decode table in shared
+// memory): several species, n_max from 9 to 12 and n_max (l_max+1) not a multiple of four (the other cases have
+// faster paths with an operand in registers)
+__host__ __device__ inline bool cross_table_wanted(int S, int n_max, int l_max) {
+    return S > 1 && n_max > 8 && n_max <= 12 && ((n_max * (l_max + 1)) & 3) != 0;
+}
 __host__ __device__ inline int align4(int x) { return (x + 3) & ~3; }
 constexpr int kGeoWords = kGeoPairs * 9 + 44;   // geometry (9 words per pair), species segments (9 + 32 words, padded)
 __host__ __device__ inline SmemLayout make_layout(int S, int n_max, int l_max, int P, bool deriv, bool weighted = false) {
@@ -150,6 +156,7 @@ __host__ __device__ inline SmemLayout make_layout(int S, int n_max, int l_max, i
     o.c = off; off = align4(off + CT);
     o.geo = off; off = align4(off + kGeoWords + (weighted ? 2 * kGeoPairs : 0));   // + per-pair weights
     o.tri = off; if (deriv) off = align4(off + ((n_max * (n_max + 1) / 2) * L1 + 1) / 2);   // 16-bit entries
+    o.xdec = off; if (deriv && cross_table_wanted(S, n_max, l_max)) off = align4(off + (n_max * NCH + 1) / 2);   // 16-bit entries
     o.zero = off; if (deriv) off += kZeroWords;
     // the D tiles (pass 1, centre's row) and the per-warp U/V staging (pass 2) never live
     // at the same time and share space
