@@ -617,15 +617,34 @@ pairs_kernel(const float* __restrict__ pos, const int* __restrict__ centers, con
         for (int q = lane; q < k; q += 32) pair_key[base + q] = raw[q];
         return;
     }
-    // rank sort (keys are distinct)
+    // rank sort (keys are distinct), two keys per lane and trip so that every key read serves two comparisons;
+    // without a periodic axis all keys carry the same lattice translation and the atom fields alone decide
     bool self_in = false;
-    for (int q = lane; q < k; q += 32) {
-        unsigned long long key = raw[q];
-        int rank = 0;
-        for (int r = 0; r < k; ++r) rank += raw[r] < key;
-        sorted[rank] = key;
-        if (in_smem) pair_key[base + rank] = key;
-        self_in |= key_atom(key) == i;
+    const bool atoms_only = !(geom.pbc[0] | geom.pbc[1] | geom.pbc[2]);
+    for (int q = lane; q < k; q += 64) {
+        const bool two = q + 32 < k;
+        const unsigned long long key0 = raw[q], key1 = two ? raw[q + 32] : ~0ull;
+        int rank0 = 0, rank1 = 0;
+        if (atoms_only) {
+            const unsigned a0 = (unsigned)(key0 >> 24), a1 = (unsigned)(key1 >> 24);
+            for (int r = 0; r < k; ++r) {
+                const unsigned a = (unsigned)(raw[r] >> 24);
+                rank0 += a < a0; rank1 += a < a1;
+            }
+        } else {
+            for (int r = 0; r < k; ++r) {
+                const unsigned long long v = raw[r];
+                rank0 += v < key0; rank1 += v < key1;
+            }
+        }
+        sorted[rank0] = key0;
+        if (in_smem) pair_key[base + rank0] = key0;
+        self_in |= key_atom(key0) == i;
+        if (two) {
+            sorted[rank1] = key1;
+            if (in_smem) pair_key[base + rank1] = key1;
+            self_in |= key_atom(key1) == i;
+        }
     }
     self_in = __any_sync(0xffffffffu, self_in);
     __syncwarp();
