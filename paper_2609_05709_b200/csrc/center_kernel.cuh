@@ -980,7 +980,7 @@ center_kernel(const CenterParams p) {
         if (g0 > 0 || k_pairs > kGeoPairs) special = stage_geometry(g0, gc);     // otherwise still valid from pass 1
         // (measured on the 1000-molecule cluster: 1 to 4 % faster from n_max = 8 on up to l_max = 8; with fewer
         // channels than lanes, or more columns m than the eight lanes of a pair, the staging by the whole CTA wins)
-        constexpr bool kPrivate = NMAX_T >= 8 && L <= 8;
+        constexpr bool kPrivate = !CC && NMAX_T >= 8 && L <= 8;      // (the coefficient rows are cheap per pair: staging by the CTA wins there)
         if (kPrivate && !special && PW >= 1) {
             // Every pair has a row of its own: the warps work without one another.  Warp w takes the pairs w, w + 8,
             // ... of the batch, PW at a time: it stages their radial factors (lanes on channels) and harmonics (eight
