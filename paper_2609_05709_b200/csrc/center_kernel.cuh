@@ -186,6 +186,10 @@ center_kernel(const CenterParams p) {
     const long long pair_base = p.pair_start[c_idx];
     const int k_pairs = p.pair_count[c_idx];
     const bool periodic = p.geom.pbc[0] | p.geom.pbc[1] | p.geom.pbc[2];
+    // the pairs are taken in batches of geometry of equal size (a multiple of eight, at most kGeoPairs): 274 pairs are
+    // 96 + 96 + 82, not 128 + 128 + 18
+    const int geo_batches = (k_pairs + kGeoPairs - 1) / kGeoPairs;
+    const int geo_batch = geo_batches > 1 ? min(kGeoPairs, (((k_pairs + geo_batches - 1) / geo_batches) + 7) & ~7) : kGeoPairs;
 
     // pass-1 ownership of this thread: one lm, and the radial functions slot, slot + SLOTS, ...
     const int own_slot = wid / W_LM, own_lm = (wid - own_slot * W_LM) * 32 + lane;
@@ -303,8 +307,8 @@ center_kernel(const CenterParams p) {
     // shared memory once per species and batch.
     bool special = false;
     for (int n0 = 0; n0 < NMAX; n0 += SLOTS * NPT) {             // one trip unless n_max > 8 SLOTS
-        for (int g0 = 0; g0 < k_pairs; g0 += kGeoPairs) {
-            const int gc = min(kGeoPairs, k_pairs - g0);
+        for (int g0 = 0; g0 < k_pairs; g0 += geo_batch) {
+            const int gc = min(geo_batch, k_pairs - g0);
             __syncthreads();
             special = stage_geometry(g0, gc);
             float ac[NPT], ax[NPT], ay[NPT], az[NPT];
@@ -535,8 +539,8 @@ center_kernel(const CenterParams p) {
             sf[k] = -1; sgA[k] = suA[k] = suB[k] = 0; sgB[k] = -1;
             if (in_registers && k * kThreads + tid < NZ) decode(k * kThreads + tid, sf[k], sgA[k], suA[k], sgB[k], suB[k]);
         }
-        for (int g0 = 0; g0 < k_pairs; g0 += kGeoPairs) {
-            const int gc = min(kGeoPairs, k_pairs - g0);
+        for (int g0 = 0; g0 < k_pairs; g0 += geo_batch) {
+            const int gc = min(geo_batch, k_pairs - g0);
             __syncthreads();
             if (g0 > 0 || k_pairs > kGeoPairs) stage_geometry(g0, gc);        // otherwise still valid from pass 1
             for (int q0 = 0; q0 < gc; q0 += P) {
@@ -974,8 +978,8 @@ center_kernel(const CenterParams p) {
     };
 
     const int PW = P / kWarps;             // pairs a warp stages for itself (the staging area holds P)
-    for (int g0 = 0; g0 < k_pairs; g0 += kGeoPairs) {
-        const int gc = min(kGeoPairs, k_pairs - g0);
+    for (int g0 = 0; g0 < k_pairs; g0 += geo_batch) {
+        const int gc = min(geo_batch, k_pairs - g0);
         __syncthreads();
         if (g0 > 0 || k_pairs > kGeoPairs) special = stage_geometry(g0, gc);     // otherwise still valid from pass 1
         // (measured on the 1000-molecule cluster: 1 to 4 % faster from n_max = 8 on up to l_max = 8; with fewer
