@@ -60,8 +60,10 @@ __host__ __device__ constexpr int desc_c_chunks(int S, int np) {
 }
 
 // Shared memory in 4-byte words: [table (optional)] then one region per warp:
-//   c [LM][4 desc_c_chunks] | S staging [chunk][s_row] | G staging [chunk][L1 g_l] | pair staging [chunk][8]
-// The feature row is assembled on top of the staging area when it fits there.
+//   c [LM][4 desc_c_chunks] | S staging [chunk][s_row] | G staging [chunk][L1 g_l] | pair staging [chunk][8 or 5]
+// The feature row is assembled on top of the staging area when it fits there.  With the table in shared memory (the
+// plain build on many centres) a staged pair is five words (dx, dy, dz, t; interval | species << 16) instead of
+// eight (dx, dy, dz, r; interval, t, species, weight): at the benchmark's basis that is what lets a 16th warp fit.
 struct DescLayout {
     int table, warp0, per_warp, c, sS, sG, ring, slab_words, total;
 };
@@ -74,7 +76,8 @@ __host__ __device__ inline DescLayout make_desc_layout(int S, int np, int l_max,
     o.c = off; off += LM * 4 * desc_c_chunks(S, np);
     o.sS = off; off += kDescChunk * desc_s_row(l_max);
     o.sG = off; off += kDescChunk * L1 * desc_g_l(np);
-    o.ring = off; off += kDescChunk * 8;
+    o.ring = off; off += kDescChunk * (table_words ? 5 : 8);
+    off = (off + 3) & ~3;
     o.slab_words = off - o.sS;
     o.per_warp = off;
     o.total = o.warp0 + warps * off;
@@ -167,6 +170,7 @@ __global__ void __launch_bounds__(kDescMaxWarps * 32, 1) desc_kernel(const Cente
     float* const sG = wbase + lay.sG;                                               // [chunk][L1][GL]
     float4* const ring_d = reinterpret_cast<float4*>(wbase + lay.ring);             // [chunk] dx, dy, dz, r
     int4* const ring_i = reinterpret_cast<int4*>(wbase + lay.ring + 4 * kDescChunk);// [chunk] interval, t, species, weight
+    int* const ring_q = reinterpret_cast<int*>(wbase + lay.ring + 4 * kDescChunk);  // TS: [chunk] interval | species << 16, and t in ring_d.w
     float* const slab = wbase + lay.sS;
     const float4* const tab = TS ? reinterpret_cast<const float4*>(smem) : reinterpret_cast<const float4*>(p.table_ln);
 
@@ -339,19 +343,26 @@ __global__ void __launch_bounds__(kDescMaxWarps * 32, 1) desc_kernel(const Cente
 #pragma unroll
                     for (int b = 0; b < PPL; ++b)
                         if ((unsigned)(pos_sorted[b] - c0) < (unsigned)kDescChunk) {
-                            ring_d[pos_sorted[b] - c0] = dd[b];
-                            ring_i[pos_sorted[b] - c0] = make_int4(qt[b].x, qt[b].y, sp[b], __float_as_int(ww[b]));
+                            if (TS) {
+                                ring_d[pos_sorted[b] - c0] = make_float4(dd[b].x, dd[b].y, dd[b].z, __int_as_float(qt[b].y));
+                                ring_q[pos_sorted[b] - c0] = qt[b].x | (sp[b] << 16);
+                            } else {
+                                ring_d[pos_sorted[b] - c0] = dd[b];
+                                ring_i[pos_sorted[b] - c0] = make_int4(qt[b].x, qt[b].y, sp[b], __float_as_int(ww[b]));
+                            }
                         }
                     __syncwarp();
                     // solid harmonics: a lane per pair
                     if (lane < n_stage) {
                         const float4 d = ring_d[lane];
-                        harmonics_tiles<L>(d.x, d.y, d.z, d.w * d.w, sS4 + lane * (SROW / 4));
+                        harmonics_tiles<L>(d.x, d.y, d.z, TS ? fmaf(d.x, d.x, fmaf(d.y, d.y, d.z * d.z)) : d.w * d.w, sS4 + lane * (SROW / 4));
                     }
                     // radial factors: lanes on the channels, pairs in turn
 #pragma unroll 4
                     for (int pr = 0; pr < n_stage; ++pr) {
-                        const int4 gi = ring_i[pr];
+                        int4 gi;
+                        if (TS) { gi = make_int4(ring_q[pr] & 0xffff, __float_as_int(ring_d[pr].w), 0, 0); }
+                        else gi = ring_i[pr];
                         const float t = __int_as_float(gi.y);
                         const float2 tt = make_float2(t, t);
                         const float4* row = tab + (size_t)gi.x * (NCHP * 6 / 4);
@@ -374,7 +385,7 @@ __global__ void __launch_bounds__(kDescMaxWarps * 32, 1) desc_kernel(const Cente
                         }
                     }
                     __syncwarp();
-                    const int tag = lane < n_stage ? ring_i[lane].z : -1;
+                    const int tag = lane < n_stage ? (TS ? ring_q[lane] >> 16 : ring_i[lane].z) : -1;
                     for (int s = 0; s < S; ++s) {
                         const unsigned mask = __ballot_sync(0xffffffffu, tag == s);
                         if (!mask) continue;

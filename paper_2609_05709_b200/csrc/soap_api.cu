@@ -472,8 +472,11 @@ int launch_desc(soap_t* h, CenterParams& cp, int64_t n_work, cudaStream_t st) {
     cp.inv_h = h->basis.inv_h_values; cp.n_intervals = h->basis.n_intervals_values;      // the value table has intervals of its own
     const bool plain = center_params_plain(cp);
     const int warps_fit = (int)std::min<size_t>(kDescMaxWarps, (size_t)h->max_smem / h->desc_warp_bytes);
-    const int warps_ts = h->desc_table_bytes + h->desc_warp_bytes <= (size_t)h->max_smem
-                             ? (int)std::min<size_t>(kDescMaxWarps, ((size_t)h->max_smem - h->desc_table_bytes) / h->desc_warp_bytes) : 0;
+    // (with the table in shared memory a warp's region is a little smaller: its staged pairs are five words, not eight)
+    const size_t table_pad = (h->desc_table_bytes + 15) & ~(size_t)15;
+    const size_t warp_bytes_ts = (size_t)make_desc_layout(h->S, h->desc_np, h->l_max, 1, (int)(h->desc_table_bytes / 4)).per_warp * 4;
+    const int warps_ts = h->desc_table_bytes > 0 && table_pad + warp_bytes_ts <= (size_t)h->max_smem
+                             ? (int)std::min<size_t>(kDescMaxWarps, ((size_t)h->max_smem - table_pad) / warp_bytes_ts) : 0;
     const bool ts = plain && warps_ts >= 6 && n_work >= (int64_t)4 * h->sm_count;
     int warps = ts ? warps_ts : warps_fit;
     warps = (int)std::max<int64_t>(1, std::min<int64_t>(warps, (n_work + h->sm_count - 1) / h->sm_count));
