@@ -27,6 +27,10 @@
  *    host thread; handles share nothing but read-only constant tables.
  *  - `stream` is a cudaStream_t passed as void* (NULL = default stream).  All
  *    calls enqueue work on it and return without waiting, except where noted.
+ *    Within a call the kernels use programmatic dependent launch (each waits on
+ *    the device for its predecessor before it reads that kernel's results);
+ *    towards other work on the stream a call behaves like any kernel sequence:
+ *    its first kernel starts after everything queued before it has finished.
  *  - Feature order: species pairs mu <= nu (species sorted by atomic number),
  *    then the radial pair (n, n') with n' >= n when mu == nu and all n, n'
  *    otherwise (n outer), then l fastest.  F = S n_max (S n_max + 1)/2 (l_max+1).
@@ -363,7 +367,11 @@ int soap_neighbor_counts_static(const float *d_positions, int64_t n_atoms, doubl
  * soap_descriptor and soap_derivatives record CUDA events on the caller's
  * stream around (a) the neighbour search and (b) the fused per-centre kernel.
  * soap_profile_read waits for the last call's events and returns both
- * durations in milliseconds.  Events cost about a microsecond; off by default. */
+ * durations in milliseconds.  Off by default: the kernels of a call are
+ * launched so that each may start while the one before it finishes (they wait
+ * for it on the device), and an event recorded between two launches keeps the
+ * second from starting early - a profiled call is a few microseconds slower,
+ * and its two durations can add up to more than an unprofiled call takes. */
 int soap_profile(soap_t *h, int enable);
 int soap_profile_read(soap_t *h, float *ms_neighbors, float *ms_center);
 
