@@ -348,9 +348,10 @@ center_kernel(const CenterParams p) {
                                 const float4 h = sSD4[pr * LMP + own_lm];
                                 const float4 d = geo_d[g];
                                 // an image of the centre does not move relative to it: no contribution to D
-                                const float mv = (geo_i[g].z & 256) ? 1.f : 0.f;
-                                const float hy = h.y * mv, hz = h.z * mv, hw = h.w * mv;
-                                const float tx = h.x * d.x * mv, ty = h.x * d.y * mv, tz = h.x * d.z * mv;
+                                // (only a batch with images or shared rows can hold one)
+                                const float mv = (!special || (geo_i[g].z & 256)) ? 1.f : 0.f;
+                                float hy = h.y, hz = h.z, hw = h.w, tx = h.x * d.x, ty = h.x * d.y, tz = h.x * d.z;
+                                if (special) { hy *= mv; hz *= mv; hw *= mv; tx *= mv; ty *= mv; tz *= mv; }
                                 const float2* gp = sG2 + pr * NCH + (n0 + own_slot) * L1 + own_l;
 #pragma unroll
                                 for (int k = 0; k < NPT; ++k)
